@@ -1,0 +1,269 @@
+/*
+ * CPU oracle for the routing hot path of GoodServe.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the hot path
+ * computes, written from the paper; it exists so that the CUDA library can be checked
+ * against it.  It shares no code with the CUDA path and nothing in the product may call it.
+ *
+ * What is stated here, and where the paper defines it:
+ *   - latency model  T(r,g) = q_g + p_g * (L_in_r - H_{r,g}) + d_g * L_out_r     (Eq. 2), with H = 0
+ *   - queue-delay smoothing  q_g <- alpha * w_g + (1 - alpha) * q_g              (Algorithm 1, EMA step)
+ *   - feasible set  C = { g : T(r,g) <= D_r }, restricted to instances whose memory
+ *     can hold the request                                                      (Algorithm 1; Sec. 3.1 constraints)
+ *   - just-enough choice  g* = argmax_{g in C} d_g                               (Algorithm 1; Sec. 3.4)
+ *   - fallback  g* = argmin_g (T(r,g) - D_r)  when C is empty                    (Algorithm 1)
+ *   - risk test: an ongoing request is flagged when its expected finish time under the
+ *     latest estimates exceeds its SLO                                          (Sec. 3.4, second step)
+ *
+ * Readings taken where the paper is silent (each is listed in the design document):
+ *   ties in argmax d_g and in argmin T go to the smallest instance index; d_g is the current
+ *   loaded per-token decode latency a_t + b_t * batch_g; w_g (observed wait) is modelled as
+ *   queued_prefill_tokens_g * p_g; the EMA steps once per routing round; the memory constraint
+ *   is  L_in + L_out <= free_kv_tokens_g ; the fallback prefers instances with KV room
+ *   (tier 2) and drops that preference only when no instance has room (tier 3); the risk
+ *   test is decode-only:  elapsed + d_assigned * max(pred_len - generated, 0) > slo.
+ *
+ * Two arithmetic modes, same steps:
+ *   *_f64 : every real operation in double from the float inputs (authority for values).
+ *   *_f32 : single precision with a fixed operation order, each operation rounded once
+ *           (fmaf / one multiply / one subtract) -- the precision in which the kernels take
+ *           their decisions, so integer results can be compared bit for bit.
+ *
+ * Invalid data never aborts: negative counts and negative/NaN q_ema are clamped to 0, an
+ * out-of-range type id is read as type 0, an out-of-range assigned instance is clamped into
+ * [0, M-1]; a status bit records that it happened.
+ *
+ * Build:  gcc -O2 -fPIC -shared -ffp-contract=off -fno-fast-math goodserve_oracle.c -lm
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <stdlib.h>
+
+enum { GSO_BAD_INSTANCE = 1, GSO_BAD_TYPE = 2, GSO_BAD_VALUE = 4 };
+
+static int32_t clamp_count(int32_t v, unsigned *status) {
+    if (v < 0) { *status |= GSO_BAD_VALUE; return 0; }
+    return v;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* per-instance coefficients of Eq. 2 for one routing round                              */
+/* ------------------------------------------------------------------------------------ */
+
+void gso_instance_table_f64(int32_t M, int32_t Tn,
+                            const int32_t *type_id, const int32_t *queued_prefill_tokens,
+                            const int32_t *decode_batch, const int32_t *free_kv_tokens,
+                            const float *q_ema_ms,
+                            const float *p_type, const float *a_type, const float *b_type,
+                            float ema_alpha,
+                            double *q, double *p, double *d, int64_t *kv, unsigned *status)
+{
+    double alpha = (double)ema_alpha;
+    for (int32_t g = 0; g < M; ++g) {
+        int32_t t = type_id[g];
+        if (t < 0 || t >= Tn) { *status |= GSO_BAD_TYPE; t = 0; }
+        double Qtok = (double)clamp_count(queued_prefill_tokens[g], status);
+        double B = (double)clamp_count(decode_batch[g], status);
+        double qe = (double)q_ema_ms[g];
+        if (!(qe >= 0.0)) { *status |= GSO_BAD_VALUE; qe = 0.0; }
+        p[g] = (double)p_type[t];
+        d[g] = (double)a_type[t] + (double)b_type[t] * B;
+        double w = Qtok * p[g];                            /* time to drain the queued prefill work */
+        q[g] = alpha * w + (1.0 - alpha) * qe;             /* EMA step */
+        kv[g] = (int64_t)clamp_count(free_kv_tokens[g], status);
+    }
+}
+
+void gso_instance_table_f32(int32_t M, int32_t Tn,
+                            const int32_t *type_id, const int32_t *queued_prefill_tokens,
+                            const int32_t *decode_batch, const int32_t *free_kv_tokens,
+                            const float *q_ema_ms,
+                            const float *p_type, const float *a_type, const float *b_type,
+                            float ema_alpha,
+                            float *q, float *p, float *d, int64_t *kv, unsigned *status)
+{
+    float one_minus_alpha = 1.0f - ema_alpha;
+    for (int32_t g = 0; g < M; ++g) {
+        int32_t t = type_id[g];
+        if (t < 0 || t >= Tn) { *status |= GSO_BAD_TYPE; t = 0; }
+        float Qtok = (float)clamp_count(queued_prefill_tokens[g], status);
+        float B = (float)clamp_count(decode_batch[g], status);
+        float qe = q_ema_ms[g];
+        if (!(qe >= 0.0f)) { *status |= GSO_BAD_VALUE; qe = 0.0f; }
+        p[g] = p_type[t];
+        d[g] = fmaf(b_type[t], B, a_type[t]);
+        float w = Qtok * p[g];
+        float keep = one_minus_alpha * qe;
+        q[g] = fmaf(ema_alpha, w, keep);
+        kv[g] = (int64_t)clamp_count(free_kv_tokens[g], status);
+    }
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Algorithm 1 for every request of a round: the literal loop over requests x instances  */
+/* ------------------------------------------------------------------------------------ */
+
+void gso_route_f64(int64_t N, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                   const float *slo_ms,
+                   int32_t M, const double *q, const double *p, const double *d, const int64_t *kv,
+                   int32_t *instance_idx, double *est_e2e_ms, double *slack_ms, uint8_t *tier,
+                   unsigned *status)
+{
+    for (int64_t r = 0; r < N; ++r) {
+        double x = (double)clamp_count(prompt_len[r], status);
+        double y = (double)clamp_count(pred_decode_len[r], status);
+        double D = (double)slo_ms[r];
+        int64_t need = (int64_t)x + (int64_t)y;
+
+        int32_t best_c = -1, best_k = -1, best_a = -1;   /* feasible / KV-ok / all */
+        double d_c = 0.0, T_c = 0.0, T_k = 0.0, T_a = 0.0;
+        for (int32_t g = 0; g < M; ++g) {
+            double T = q[g] + p[g] * x + d[g] * y;        /* Eq. 2, H = 0 */
+            int kv_ok = need <= kv[g];
+            if (kv_ok && T <= D) {                        /* g joins C */
+                if (best_c < 0 || d[g] > d_c) { best_c = g; d_c = d[g]; T_c = T; }
+            }
+            if (kv_ok && (best_k < 0 || T < T_k)) { best_k = g; T_k = T; }
+            if (best_a < 0 || T < T_a) { best_a = g; T_a = T; }
+        }
+        int32_t g_star; double T_star; uint8_t tr;
+        if (best_c >= 0)      { g_star = best_c; T_star = T_c; tr = 1; }
+        else if (best_k >= 0) { g_star = best_k; T_star = T_k; tr = 2; }
+        else                  { g_star = best_a; T_star = T_a; tr = 3; }
+        instance_idx[r] = g_star;
+        est_e2e_ms[r] = T_star;
+        slack_ms[r] = D - T_star;
+        if (tier) tier[r] = tr;
+    }
+}
+
+void gso_route_f32(int64_t N, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                   const float *slo_ms,
+                   int32_t M, const float *q, const float *p, const float *d, const int64_t *kv,
+                   int32_t *instance_idx, float *est_e2e_ms, float *slack_ms, uint8_t *tier,
+                   unsigned *status)
+{
+    for (int64_t r = 0; r < N; ++r) {
+        int32_t xi = clamp_count(prompt_len[r], status);
+        int32_t yi = clamp_count(pred_decode_len[r], status);
+        float x = (float)xi, y = (float)yi;
+        float D = slo_ms[r];
+        int64_t need = (int64_t)xi + (int64_t)yi;
+
+        int32_t best_c = -1, best_k = -1, best_a = -1;
+        float d_c = 0.0f, T_c = 0.0f, T_k = 0.0f, T_a = 0.0f;
+        for (int32_t g = 0; g < M; ++g) {
+            float T = fmaf(d[g], y, fmaf(p[g], x, q[g]));
+            int kv_ok = need <= kv[g];
+            if (kv_ok && T <= D) {
+                if (best_c < 0 || d[g] > d_c) { best_c = g; d_c = d[g]; T_c = T; }
+            }
+            if (kv_ok && (best_k < 0 || T < T_k)) { best_k = g; T_k = T; }
+            if (best_a < 0 || T < T_a) { best_a = g; T_a = T; }
+        }
+        int32_t g_star; float T_star; uint8_t tr;
+        if (best_c >= 0)      { g_star = best_c; T_star = T_c; tr = 1; }
+        else if (best_k >= 0) { g_star = best_k; T_star = T_k; tr = 2; }
+        else                  { g_star = best_a; T_star = T_a; tr = 3; }
+        instance_idx[r] = g_star;
+        est_e2e_ms[r] = T_star;
+        slack_ms[r] = D - T_star;
+        if (tier) tier[r] = tr;
+    }
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* SLO-violation risk test over the active requests (Sec. 3.4)                            */
+/* ------------------------------------------------------------------------------------ */
+
+static int32_t clamp_instance(int32_t g, int32_t M, unsigned *status) {
+    if (g < 0) { *status |= GSO_BAD_INSTANCE; return 0; }
+    if (g >= M) { *status |= GSO_BAD_INSTANCE; return M - 1; }
+    return g;
+}
+
+void gso_risk_f64(int64_t A, const int32_t *assigned_inst, const int32_t *generated_tokens,
+                  const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                  int32_t M, const double *d,
+                  uint8_t *flag, double *finish_ms, unsigned *status)
+{
+    for (int64_t i = 0; i < A; ++i) {
+        int32_t g = clamp_instance(assigned_inst[i], M, status);
+        int64_t gen = clamp_count(generated_tokens[i], status);
+        int64_t tot = clamp_count(pred_len[i], status);
+        int64_t rem = tot - gen; if (rem < 0) rem = 0;
+        double finish = (double)elapsed_ms[i] + d[g] * (double)rem;
+        flag[i] = (uint8_t)(finish > (double)slo_ms[i]);
+        if (finish_ms) finish_ms[i] = finish;
+    }
+}
+
+void gso_risk_f32(int64_t A, const int32_t *assigned_inst, const int32_t *generated_tokens,
+                  const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                  int32_t M, const float *d,
+                  uint8_t *flag, float *finish_ms, unsigned *status)
+{
+    for (int64_t i = 0; i < A; ++i) {
+        int32_t g = clamp_instance(assigned_inst[i], M, status);
+        int64_t gen = clamp_count(generated_tokens[i], status);
+        int64_t tot = clamp_count(pred_len[i], status);
+        int64_t rem = tot - gen; if (rem < 0) rem = 0;
+        float finish = fmaf(d[g], (float)rem, elapsed_ms[i]);
+        flag[i] = (uint8_t)(finish > slo_ms[i]);
+        if (finish_ms) finish_ms[i] = finish;
+    }
+}
+
+/* Migration candidates: ascending indices of flagged requests, and the packed flag words
+ * (bit i%32 of word i/32).  Returns the true count; writes at most `capacity` indices. */
+int64_t gso_compact(int64_t A, const uint8_t *flag, uint32_t *flag_bits,
+                    int32_t *cand_idx, int64_t capacity)
+{
+    int64_t count = 0;
+    if (flag_bits) for (int64_t w = 0; w < (A + 31) / 32; ++w) flag_bits[w] = 0u;
+    for (int64_t i = 0; i < A; ++i) {
+        if (!flag[i]) continue;
+        if (flag_bits) flag_bits[i >> 5] |= (uint32_t)1u << (i & 31);
+        if (cand_idx && count < capacity) cand_idx[count] = (int32_t)i;
+        ++count;
+    }
+    return count;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Between rounds of a stream: every routed request adds its prompt tokens to the chosen   */
+/* instance's prefill queue, one slot to its decode batch, and takes L_in + L_out tokens   */
+/* of KV room; the smoothed queue delay q_g of this round becomes the carried EMA state.   */
+/* ------------------------------------------------------------------------------------ */
+
+void gso_advance(int32_t M, int64_t N, const int32_t *instance_idx,
+                 const int32_t *prompt_len, const int32_t *pred_decode_len,
+                 int32_t *queued_prefill_tokens, int32_t *decode_batch, int32_t *free_kv_tokens,
+                 float *q_ema_ms, const float *q_round)
+{
+    const int64_t I32_MAX = 2147483647LL;
+    int64_t *dq = (int64_t *)calloc((size_t)M, sizeof(int64_t));   /* prompt tokens routed to g */
+    int64_t *db = (int64_t *)calloc((size_t)M, sizeof(int64_t));   /* requests routed to g */
+    int64_t *dk = (int64_t *)calloc((size_t)M, sizeof(int64_t));   /* KV tokens they will hold */
+    for (int64_t r = 0; r < N; ++r) {
+        int32_t g = instance_idx[r];
+        if (g < 0 || g >= M) continue;
+        int64_t x = prompt_len[r] < 0 ? 0 : prompt_len[r];
+        int64_t y = pred_decode_len[r] < 0 ? 0 : pred_decode_len[r];
+        dq[g] += x; db[g] += 1; dk[g] += x + y;
+    }
+    for (int32_t g = 0; g < M; ++g) {
+        int64_t Q = queued_prefill_tokens[g] < 0 ? 0 : queued_prefill_tokens[g];
+        int64_t B = decode_batch[g] < 0 ? 0 : decode_batch[g];
+        int64_t K = free_kv_tokens[g] < 0 ? 0 : free_kv_tokens[g];
+        Q += dq[g]; if (Q > I32_MAX) Q = I32_MAX;
+        B += db[g]; if (B > I32_MAX) B = I32_MAX;
+        K -= dk[g]; if (K < 0) K = 0;
+        queued_prefill_tokens[g] = (int32_t)Q;
+        decode_batch[g] = (int32_t)B;
+        free_kv_tokens[g] = (int32_t)K;
+        q_ema_ms[g] = q_round[g];
+    }
+    free(dq); free(db); free(dk);
+}

@@ -1,0 +1,493 @@
+"""Pins for the CPU oracle: everything here checks the oracle against something other than
+itself -- hand-worked fixtures, a declarative restatement of Algorithm 1's post-condition
+evaluated on exhaustive tiny grids, textbook special cases (numpy argmax/argmin/bincount),
+closed forms and invariants.  No GPU."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as W
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+PRECS = ("f64", "f32")
+
+
+# --------------------------------------------------------------------------------------
+# helpers
+# --------------------------------------------------------------------------------------
+
+def base_types():
+    return W.make_types(3, seed=0, perturb=False)
+
+
+def fixture_pool(kv=(100000, 100000, 100000)):
+    types = base_types()
+    type_id = np.array([0, 1, 2], np.int32)
+    queued = np.array([4000, 2000, 1000], np.int32)
+    batch = np.array([20, 10, 10], np.int32)
+    q_ema = (queued.astype(np.float64) * types.prefill_ms_per_tok[type_id]).astype(np.float32)
+    inst = W.InstanceState(type_id, queued, batch, np.array(kv, np.int32), q_ema)
+    return types, inst
+
+
+def read_rows(name):
+    rows = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+def latency_all_instances(q, p, d, x, y, prec):
+    """T(r, .) of Eq. 2 for one request.  In single precision each fused step rounds once;
+    a product of two floats is exact in double, so rounding the double sum gives that."""
+    if prec == "f64":
+        return q + p * float(x) + d * float(y)
+    t1 = (p.astype(np.float64) * float(x) + q).astype(np.float32)
+    return (d.astype(np.float64) * float(y) + t1).astype(np.float32).astype(np.float64)
+
+
+def check_postcondition(q, p, d, kv, x, y, D, idx, tier, prec="f64"):
+    """Declarative statement of what Algorithm 1 (with the adopted tie/KV readings) must
+    return, written as set conditions instead of a scan."""
+    q, p, d = (np.asarray(a, np.float64) for a in (q, p, d))
+    kv = np.asarray(kv, np.int64)
+    for r in range(len(x)):
+        T = latency_all_instances(q, p, d, x[r], y[r], prec)
+        ok = (int(x[r]) + int(y[r])) <= kv
+        feas = ok & (T <= float(D[r]))
+        g = int(idx[r])
+        if feas.any():
+            assert tier[r] == 1
+            assert feas[g]
+            better = feas & ((d > d[g]) | ((d == d[g]) & (np.arange(len(d)) < g)))
+            assert not better.any()
+        else:
+            pool = ok if ok.any() else np.ones_like(ok)
+            assert tier[r] == (2 if ok.any() else 3)
+            assert pool[g]
+            better = pool & ((T < T[g]) | ((T == T[g]) & (np.arange(len(d)) < g)))
+            assert not better.any()
+
+
+# --------------------------------------------------------------------------------------
+# hand-worked fixtures
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("alpha", [0.0, 0.3, 0.5, 1.0])
+def test_handworked_routing(prec, alpha):
+    for name, D, k0, k1, k2, g, est, slack, tier in read_rows("handworked_routing.txt"):
+        types, inst = fixture_pool((int(k0), int(k1), int(k2)))
+        tab = oracle.instance_table(types, inst, alpha, prec)
+        np.testing.assert_allclose(tab.q, [100, 100, 100], rtol=1e-6, err_msg=name)
+        np.testing.assert_allclose(tab.d, [9.0, 14.8, 26.5], rtol=1e-6, err_msg=name)
+        res = oracle.route(tab, [1000], [200], [float(D)])
+        assert res.instance_idx[0] == int(g), name
+        assert res.tier[0] == int(tier), name
+        assert res.est_e2e_ms[0] == pytest.approx(float(est), rel=1e-5), name
+        assert res.slack_ms[0] == pytest.approx(float(slack), rel=1e-4, abs=2e-3), name
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_handworked_risk(prec):
+    types, inst = fixture_pool()
+    tab = oracle.instance_table(types, inst, 0.5, prec)
+    for name, pred, gen, elapsed, slo, finish, flag in read_rows("handworked_risk.txt"):
+        res = oracle.risk(tab, [1], [int(gen)], [int(pred)], [float(elapsed)], [float(slo)])
+        assert res.finish_ms[0] == pytest.approx(float(finish), rel=1e-6), name
+        assert res.flag[0] == int(flag), name
+
+
+# --------------------------------------------------------------------------------------
+# closed form of Eq. 2 and of the instance coefficients
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_eq2_closed_form_and_linearity(prec):
+    wl = W.make_workload(1, n_requests=64, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    # a single-instance pool makes route() return T(r,g) itself
+    for g in (0, 17, 63):
+        one = oracle.InstanceTable(tab.q[g:g + 1], tab.p[g:g + 1], tab.d[g:g + 1],
+                                   tab.kv[g:g + 1], 0, prec)
+        x = np.array([0, 1, 0, 1000, 2000, 1000], np.int32)
+        y = np.array([0, 0, 1, 200, 200, 400], np.int32)
+        T = oracle.route(one, x, y, np.zeros(6, np.float32)).est_e2e_ms.astype(np.float64)
+        q, p, d = float(tab.q[g]), float(tab.p[g]), float(tab.d[g])
+        rel = 1e-12 if prec == "f64" else 1e-6
+        assert T[0] == pytest.approx(q, rel=rel)                      # intercept
+        assert T[1] - T[0] == pytest.approx(p, rel=1e-3, abs=1e-4)    # one more prompt token
+        assert T[2] - T[0] == pytest.approx(d, rel=1e-3, abs=1e-4)    # one more output token
+        assert T[3] == pytest.approx(q + 1000 * p + 200 * d, rel=rel)
+        assert T[4] - T[3] == pytest.approx(1000 * p, rel=1e-4)       # linear in L_in
+        assert T[5] - T[3] == pytest.approx(200 * d, rel=1e-4)        # linear in L_out
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_instance_coefficients(prec):
+    types, inst = fixture_pool()
+    inst.q_ema_ms[:] = [10.0, 20.0, 30.0]
+    w = np.array([100.0, 100.0, 100.0])
+    for alpha in (0.0, 0.25, 1.0):
+        tab = oracle.instance_table(types, inst, alpha, prec)
+        np.testing.assert_allclose(tab.q, alpha * w + (1 - alpha) * inst.q_ema_ms, rtol=1e-6)
+        np.testing.assert_allclose(tab.p, [0.025, 0.05, 0.1], rtol=1e-6)
+        assert list(tab.kv) == [100000] * 3
+    # alpha = 1 forgets the state, alpha = 0 keeps it
+    assert np.allclose(oracle.instance_table(types, inst, 1.0, prec).q, w, rtol=1e-6)
+    assert np.allclose(oracle.instance_table(types, inst, 0.0, prec).q, inst.q_ema_ms, rtol=1e-6)
+
+
+def test_invalid_data_is_clamped_and_reported():
+    types, inst = fixture_pool()
+    inst.type_id[1] = 7
+    inst.decode_batch[0] = -5
+    inst.q_ema_ms[2] = np.nan
+    tab = oracle.instance_table(types, inst, 0.5, "f64")
+    assert tab.status & oracle.BAD_TYPE and tab.status & oracle.BAD_VALUE
+    assert tab.d[0] == pytest.approx(8.0)             # batch read as 0
+    assert tab.p[1] == pytest.approx(0.025)           # type read as 0
+    assert tab.q[2] == pytest.approx(0.5 * 100.0)     # q_ema read as 0
+    res = oracle.route(tab, [-3], [10], [1e9])
+    assert res.status & oracle.BAD_VALUE
+    rk = oracle.risk(tab, [99, -1], [0, 0], [10, 10], [0.0, 0.0], [1e9, 1e9])
+    assert rk.status & oracle.BAD_INSTANCE
+    assert rk.finish_ms[0] == pytest.approx(10 * tab.d[2]) and rk.finish_ms[1] == pytest.approx(10 * tab.d[0])
+    # NaN deadline: nothing is feasible, the request falls back to the fastest instance
+    res = oracle.route(tab, [1000], [200], [np.nan])
+    assert res.tier[0] == 2 and res.instance_idx[0] == int(np.argmin(tab.q + 1000 * tab.p + 200 * tab.d))
+
+
+# --------------------------------------------------------------------------------------
+# Algorithm 1's post-condition on exhaustive tiny grids (brute force)
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_postcondition_exhaustive_tiny(prec):
+    types = base_types()
+    p_t = types.prefill_ms_per_tok
+    n_cases = 0
+    for M in (1, 2, 3, 4):
+        for tids in itertools.product(range(3), repeat=M):
+            if M == 4 and tids[0] != 0:
+                continue                                   # keep the run short
+            for code in range(2 ** M):                     # per instance: (batch, queue) pattern
+                batch = np.array([(code >> g) & 1 for g in range(M)], np.int32)
+                queued = np.array([20000 * ((code >> ((g + 1) % M)) & 1) for g in range(M)], np.int32)
+                kvs = np.array([0, 300, 100000, 100000][:M], np.int32)
+                tid = np.array(tids, np.int32)
+                q_ema = (queued * p_t[tid]).astype(np.float32)
+                inst = W.InstanceState(tid, queued, batch, kvs, q_ema)
+                tab = oracle.instance_table(types, inst, 0.5, prec)
+                x0, y0 = 200, 50
+                T = tab.q.astype(np.float64) + tab.p * x0 + tab.d * y0
+                # deadlines on, just below and just above every T value, plus extremes
+                Ds = np.concatenate([T, T * (1 - 1e-3), T * (1 + 1e-3), [0.0, 1e9]]).astype(np.float32)
+                x = np.full(len(Ds), x0, np.int32)
+                y = np.full(len(Ds), y0, np.int32)
+                x[-1], y[-1] = 400, 50                      # need 450 > kv 300 on g1
+                res = oracle.route(tab, x, y, Ds)
+                check_postcondition(tab.q, tab.p, tab.d, tab.kv, x, y, Ds, res.instance_idx, res.tier, prec)
+                n_cases += len(Ds)
+    assert n_cases > 5000
+
+
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("cfg_id", [0, 1])
+def test_postcondition_on_workload_sample(prec, cfg_id):
+    wl = W.make_workload(cfg_id, n_requests=256, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, wl.ema_alpha, prec)
+    r = wl.requests
+    res = oracle.route(tab, *r.columns())
+    check_postcondition(tab.q, tab.p, tab.d, tab.kv, r.prompt_len, r.pred_decode_len, r.slo_ms,
+                        res.instance_idx, res.tier, prec)
+    assert set(np.unique(res.tier)) <= {1, 2, 3}
+
+
+# --------------------------------------------------------------------------------------
+# special cases that reduce to library routines
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_infinite_deadline_picks_slowest_with_room(prec):
+    wl = W.make_workload(2, n_requests=512, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    r = wl.requests
+    res = oracle.route(tab, r.prompt_len, r.pred_decode_len, np.full(r.n, np.inf, np.float32))
+    need = r.prompt_len.astype(np.int64) + r.pred_decode_len
+    for i in range(r.n):
+        ok = need[i] <= tab.kv
+        assert ok.any()
+        expect = int(np.argmax(np.where(ok, tab.d, -np.inf)))     # first max = smallest index
+        assert res.instance_idx[i] == expect and res.tier[i] == 1
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_zero_deadline_is_min_latency_router(prec):
+    wl = W.make_workload(2, n_requests=512, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    r = wl.requests
+    res = oracle.route(tab, r.prompt_len, r.pred_decode_len, np.zeros(r.n, np.float32))
+    need = r.prompt_len.astype(np.int64) + r.pred_decode_len
+    real = np.float64 if prec == "f64" else np.float32
+    for i in range(r.n):
+        x, y = real(r.prompt_len[i]), real(r.pred_decode_len[i])
+        if prec == "f64":
+            T = tab.q + tab.p * x + tab.d * y
+        else:   # products of two floats are exact in double; one rounding per fused step
+            t1 = (tab.p.astype(np.float64) * np.float64(x) + tab.q).astype(np.float32)
+            T = (tab.d.astype(np.float64) * np.float64(y) + t1).astype(np.float32)
+        ok = need[i] <= tab.kv
+        expect = int(np.argmin(np.where(ok, T, np.inf)))
+        assert res.instance_idx[i] == expect and res.tier[i] == 2
+        assert res.est_e2e_ms[i] == T[expect]
+        assert res.slack_ms[i] == -T[expect]
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_single_type_equal_batches_first_short_queue(prec):
+    """One type, equal batches: p and d are common, so the feasible set is a threshold on q
+    and the just-enough pick is the first (smallest-index) instance whose queue fits."""
+    types = W.TypeTable(np.array([0.05], np.float32), np.array([14.0], np.float32),
+                        np.array([0.08], np.float32))
+    M = 16
+    rng = np.random.default_rng(5)
+    queued = rng.integers(0, 20000, M).astype(np.int32)
+    inst = W.InstanceState(np.zeros(M, np.int32), queued, np.full(M, 10, np.int32),
+                           np.full(M, 10 ** 6, np.int32), (queued * 0.05).astype(np.float32))
+    tab = oracle.instance_table(types, inst, 0.5, prec)
+    x, y = 500, 100
+    const = 500 * float(tab.p[0]) + 100 * float(tab.d[0])
+    for D in np.linspace(const - 10, const + 1100, 57):
+        res = oracle.route(tab, [x], [y], [D])
+        fits = np.nonzero(tab.q.astype(np.float64) <= np.float32(D) - const - 1e-3)[0]
+        tight = np.nonzero(np.abs(tab.q.astype(np.float64) - (np.float32(D) - const)) <= 1e-3)[0]
+        if len(tight):
+            continue                       # rounding decides; skip the knife edge
+        if len(fits):
+            assert res.tier[0] == 1 and res.instance_idx[0] == fits[0]
+        else:
+            assert res.tier[0] == 2 and res.instance_idx[0] == int(np.argmin(tab.q))
+
+
+# --------------------------------------------------------------------------------------
+# invariants
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_invariants_on_tight_workload(prec):
+    wl = W.make_workload(3, n_requests=2048, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    r = wl.requests
+    res = oracle.route(tab, *r.columns())
+    need = r.prompt_len.astype(np.int64) + r.pred_decode_len
+    x = r.prompt_len.astype(np.float64); y = r.pred_decode_len.astype(np.float64)
+    T = tab.q[None, :] + np.outer(x, tab.p) + np.outer(y, tab.d)
+    ok = need[:, None] <= tab.kv[None, :]
+    feas = ok & (T <= r.slo_ms[:, None].astype(np.float64) * (1 + (0 if prec == "f64" else 1e-6)))
+    strictly = ok & (T <= r.slo_ms[:, None].astype(np.float64) * (1 - 1e-6))
+    g = res.instance_idx
+    rows = np.arange(r.n)
+    # whenever some instance clearly meets the deadline, the chosen one meets it too
+    has = strictly.any(axis=1)
+    assert (res.tier[has] == 1).all()
+    assert feas[rows[has], g[has]].all() and (res.slack_ms[has] >= 0).all()
+    # fallback slack is the best achievable (largest) slack and is negative in tier 2
+    fb = res.tier == 2
+    assert fb.any() and (res.tier == 1).any()
+    best = np.max(np.where(ok, r.slo_ms[:, None].astype(np.float64) - T, -np.inf), axis=1)
+    np.testing.assert_allclose(res.slack_ms[fb], best[fb], rtol=1e-5, atol=1e-2)
+    assert (res.slack_ms[fb] < 0).all()
+    # est + slack = D
+    np.testing.assert_allclose(res.est_e2e_ms + res.slack_ms, r.slo_ms, rtol=1e-5)
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_chosen_capability_monotone_in_deadline(prec):
+    wl = W.make_workload(1, n_requests=8, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    for i in range(8):
+        x, y = wl.requests.prompt_len[i], wl.requests.pred_decode_len[i]
+        Ds = np.linspace(0, 6 * float(wl.requests.slo_ms[i]), 200).astype(np.float32)
+        res = oracle.route(tab, np.full(200, x), np.full(200, y), Ds)
+        t1 = res.tier == 1
+        dsel = tab.d[res.instance_idx]
+        assert (np.diff(dsel[t1]) >= 0).all()          # looser deadline -> never a faster pick
+        assert (np.diff(res.tier.astype(int)) <= 0).all()
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_permutation_and_degenerate_pools(prec):
+    wl = W.make_workload(1, n_requests=300, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    r = wl.requests
+    res = oracle.route(tab, *r.columns())
+    perm = np.random.default_rng(1).permutation(r.n)
+    res_p = oracle.route(tab, r.prompt_len[perm], r.pred_decode_len[perm], r.slo_ms[perm])
+    assert (res_p.instance_idx == res.instance_idx[perm]).all()
+    assert (res_p.est_e2e_ms == res.est_e2e_ms[perm]).all()
+    # relabelling instances (distinct d and distinct T almost surely) relabels the answer
+    gperm = np.random.default_rng(2).permutation(tab.n_instances)
+    tab_p = oracle.InstanceTable(tab.q[gperm], tab.p[gperm], tab.d[gperm], tab.kv[gperm], 0, prec)
+    res_g = oracle.route(tab_p, *r.columns())
+    same_d = tab.d[gperm[res_g.instance_idx]] == tab.d[res.instance_idx]
+    assert same_d.all()
+    np.testing.assert_array_equal(res_g.est_e2e_ms, res.est_e2e_ms)
+    # one instance: always 0; identical instances: always 0
+    one = oracle.InstanceTable(tab.q[:1], tab.p[:1], tab.d[:1], tab.kv[:1], 0, prec)
+    assert (oracle.route(one, *r.columns()).instance_idx == 0).all()
+    rep = oracle.InstanceTable(*(np.repeat(a[:1], 9) for a in (tab.q, tab.p, tab.d, tab.kv)), 0, prec)
+    assert (oracle.route(rep, *r.columns()).instance_idx == 0).all()
+
+
+def test_power_of_two_scaling_is_exact_in_f32():
+    """Scaling every time-valued input by 2^k is exact in binary floating point, so the
+    decisions are unchanged and the outputs scale exactly."""
+    wl = W.make_workload(1, n_requests=512, n_active=512)
+    s = np.float32(8.0)
+    t2 = W.TypeTable(wl.types.prefill_ms_per_tok * s, wl.types.tpot_a_ms * s, wl.types.tpot_b_ms * s)
+    i2 = wl.instances.copy(); i2.q_ema_ms *= s
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    tab2 = oracle.instance_table(t2, i2, 0.5, "f32")
+    r = wl.requests
+    a = oracle.route(tab, *r.columns())
+    b = oracle.route(tab2, r.prompt_len, r.pred_decode_len, r.slo_ms * s)
+    np.testing.assert_array_equal(a.instance_idx, b.instance_idx)
+    np.testing.assert_array_equal(a.tier, b.tier)
+    np.testing.assert_array_equal(a.est_e2e_ms * s, b.est_e2e_ms)
+    np.testing.assert_array_equal(a.slack_ms * s, b.slack_ms)
+    act = wl.active
+    ra = oracle.risk(tab, *act.columns())
+    rb = oracle.risk(tab2, act.assigned_inst, act.generated_tokens, act.pred_len,
+                     act.elapsed_ms * s, act.slo_ms * s)
+    np.testing.assert_array_equal(ra.flag, rb.flag)
+
+
+def test_f32_and_f64_agree_away_from_ties():
+    wl = W.make_workload(2, n_requests=4096, n_active=4096)
+    t64 = oracle.instance_table(wl.types, wl.instances, 0.5, "f64")
+    t32 = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    np.testing.assert_allclose(t32.q, t64.q, rtol=3e-7)
+    np.testing.assert_allclose(t32.d, t64.d, rtol=3e-7)
+    r = wl.requests
+    a = oracle.route(t64, *r.columns()); b = oracle.route(t32, *r.columns())
+    agree = a.instance_idx == b.instance_idx
+    assert agree.mean() > 0.999
+    np.testing.assert_allclose(b.est_e2e_ms[agree], a.est_e2e_ms[agree], rtol=1e-6)
+    ra = oracle.risk(t64, *wl.active.columns()); rb = oracle.risk(t32, *wl.active.columns())
+    assert (ra.flag == rb.flag).mean() > 0.9999
+
+
+# --------------------------------------------------------------------------------------
+# goodput objective (Eq. 1) on tiny inputs
+# --------------------------------------------------------------------------------------
+
+def test_single_request_attains_objective_optimum():
+    """For one request Eq. 1's optimum is 1 exactly when some instance with room meets the
+    deadline; the heuristic must reach indicator 1 in exactly those cases (brute force)."""
+    rng = np.random.default_rng(11)
+    types = base_types()
+    for _ in range(300):
+        M = int(rng.integers(1, 5))
+        tid = rng.integers(0, 3, M).astype(np.int32)
+        queued = rng.integers(0, 20000, M).astype(np.int32)
+        inst = W.InstanceState(tid, queued, rng.integers(0, 64, M).astype(np.int32),
+                               rng.integers(0, 3000, M).astype(np.int32),
+                               (queued * types.prefill_ms_per_tok[tid]).astype(np.float32))
+        tab = oracle.instance_table(types, inst, 0.5, "f64")
+        x, y = int(rng.integers(16, 2000)), int(rng.integers(8, 800))
+        D = np.float32(rng.uniform(500, 30000))
+        T = tab.q + tab.p * x + tab.d * y
+        optimum = int(any(T[g] <= D and x + y <= tab.kv[g] for g in range(M)))   # enumerate x_{r,g}
+        res = oracle.route(tab, [x], [y], [D])
+        g = res.instance_idx[0]
+        achieved = int(T[g] <= D and x + y <= tab.kv[g])
+        assert achieved == optimum
+
+
+# --------------------------------------------------------------------------------------
+# risk scan, compaction, state advance
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_risk_special_cases(prec):
+    wl = W.make_workload(1, n_requests=8, n_active=4096)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    a = wl.active
+    # nothing left to generate: flag <=> elapsed > slo
+    res = oracle.risk(tab, a.assigned_inst, a.pred_len, a.pred_len, a.elapsed_ms, a.slo_ms)
+    np.testing.assert_array_equal(res.flag, (a.elapsed_ms > a.slo_ms).astype(np.uint8))
+    res = oracle.risk(tab, a.assigned_inst, a.pred_len, a.pred_len, a.slo_ms * 2 + 1, a.slo_ms)
+    assert res.flag.all()
+    # not started: flag <=> d * y > D  (products of floats are exact in double)
+    zero = np.zeros(a.n, np.int32)
+    res = oracle.risk(tab, a.assigned_inst, zero, a.pred_len, np.zeros(a.n, np.float32), a.slo_ms)
+    dy = tab.d[a.assigned_inst].astype(np.float64) * a.pred_len
+    if prec == "f32":
+        dy = dy.astype(np.float32)
+    np.testing.assert_array_equal(res.flag, (dy > a.slo_ms).astype(np.uint8))
+    # flags are monotone: more elapsed time never clears a flag
+    base = oracle.risk(tab, *a.columns())
+    later = oracle.risk(tab, a.assigned_inst, a.generated_tokens, a.pred_len, a.elapsed_ms * 1.5, a.slo_ms)
+    assert (later.flag >= base.flag).all()
+    assert 0 < base.flag.mean() < 1
+
+
+def test_compaction_matches_numpy():
+    rng = np.random.default_rng(3)
+    for A in (0, 1, 31, 32, 33, 1000, 4097):
+        flag = (rng.random(A) < 0.3).astype(np.uint8)
+        bits, cand, count = oracle.compact(flag)
+        ref = np.nonzero(flag)[0]
+        np.testing.assert_array_equal(cand, ref)
+        assert count == len(ref)
+        unpacked = np.unpackbits(bits.view(np.uint8), bitorder="little")[:A]
+        np.testing.assert_array_equal(unpacked, flag)
+        _, cand_small, count_small = oracle.compact(flag, capacity=len(ref) // 2)
+        assert count_small == len(ref)
+        np.testing.assert_array_equal(cand_small, ref[:len(ref) // 2])
+
+
+def test_advance_matches_bincount_and_saturates():
+    wl = W.make_workload(1, n_requests=5000, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    r = wl.requests
+    res = oracle.route(tab, *r.columns())
+    before = wl.instances.copy()
+    oracle.advance(wl.instances, tab, res.instance_idx, r.prompt_len, r.pred_decode_len)
+    M = before.n_instances
+    dq = np.bincount(res.instance_idx, weights=r.prompt_len.astype(np.float64), minlength=M).astype(np.int64)
+    db = np.bincount(res.instance_idx, minlength=M)
+    dk = np.bincount(res.instance_idx, weights=(r.prompt_len.astype(np.float64) + r.pred_decode_len),
+                     minlength=M).astype(np.int64)
+    np.testing.assert_array_equal(wl.instances.queued_prefill_tokens, before.queued_prefill_tokens + dq)
+    np.testing.assert_array_equal(wl.instances.decode_batch, before.decode_batch + db)
+    np.testing.assert_array_equal(wl.instances.free_kv_tokens,
+                                  np.maximum(before.free_kv_tokens - dk, 0))
+    np.testing.assert_array_equal(wl.instances.q_ema_ms, tab.q)
+    # saturation, by hand: 3 requests of 2^30 prompt tokens onto one instance
+    types, inst = fixture_pool()
+    tabh = oracle.instance_table(types, inst, 0.5, "f32")
+    big = np.full(3, 2 ** 30, np.int32)
+    oracle.advance(inst, tabh, np.zeros(3, np.int32), big, np.full(3, 5, np.int32))
+    assert inst.queued_prefill_tokens[0] == 2 ** 31 - 1
+    assert inst.decode_batch[0] == 23 and inst.free_kv_tokens[0] == 0
+    assert inst.queued_prefill_tokens[1] == 2000 and inst.free_kv_tokens[1] == 100000
+
+
+def test_threaded_split_is_identical():
+    wl = W.make_workload(1, n_requests=10007, n_active=10007)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    a = oracle.route(tab, *wl.requests.columns(), threads=1)
+    b = oracle.route(tab, *wl.requests.columns(), threads=5)
+    np.testing.assert_array_equal(a.instance_idx, b.instance_idx)
+    np.testing.assert_array_equal(a.est_e2e_ms, b.est_e2e_ms)
+    ra = oracle.risk(tab, *wl.active.columns(), threads=1)
+    rb = oracle.risk(tab, *wl.active.columns(), threads=3)
+    np.testing.assert_array_equal(ra.flag, rb.flag)
