@@ -1,0 +1,227 @@
+/*
+ * goodserve.h -- C ABI of the GoodServe routing hot path on one NVIDIA B200 (sm_100a).
+ *
+ * Two operations of the paper's proxy router are provided as data-parallel GPU passes:
+ *
+ *   gs_route_batch   for every pending request r and every serving instance g, the
+ *                    end-to-end latency estimate  T(r,g) = q_g + p_g * L_in_r + d_g * L_out_r
+ *                    (Eq. 2 with no prefix-cache hit), the feasible set {g : T(r,g) <= D_r}
+ *                    restricted to instances with KV room, the "just-enough" choice
+ *                    argmax d_g over that set, and the fallback argmin T when the set is
+ *                    empty (Algorithm 1; Sec. 3.4).
+ *   gs_risk_scan     for every active request, the SLO-violation risk test of Sec. 3.4
+ *                    (expected finish time under the latest estimates exceeds the SLO) and
+ *                    the ascending list of flagged requests (migration candidates).
+ *   gs_advance_state between the rounds of a stream, folds one round's assignments back
+ *                    into the per-instance queue / batch / KV state and carries the smoothed
+ *                    queue delay of the EMA step (Algorithm 1) to the next round.
+ *
+ * Conventions that hold for every call unless its comment says otherwise
+ *   - Units: times in milliseconds (float), token counts int32.
+ *   - All array arguments of the device entry points are DEVICE pointers owned by the
+ *     caller; arrays must be 16-byte aligned (else GS_ERR_ALIGN).  The *_host variants take
+ *     HOST pointers (pinned memory makes their copies asynchronous) and stage through
+ *     buffers owned by the context.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Device entry points only enqueue work on it and return; they do not synchronise.
+ *   - Return value: GS_OK or a negative gs_error.  On an error nothing has been enqueued.
+ *   - Invalid DATA never faults or traps: negative token counts and negative/NaN q_ema are
+ *     read as 0, a type id outside [0, n_types) as type 0, an assigned instance outside
+ *     [0, n_instances) is clamped into range; a bit of the device status word records it
+ *     (gs_device_status).  A NaN deadline is never met, so such a request takes the fallback.
+ *   - One context serves one stream at a time; calls on one context must not overlap on the
+ *     GPU (they share the context's scratch memory).
+ */
+#ifndef GOODSERVE_H_
+#define GOODSERVE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define GS_API __attribute__((visibility("default")))
+#else
+#define GS_API
+#endif
+
+#define GS_MAX_INSTANCES 1024   /* instance table is staged whole in shared memory */
+#define GS_MAX_TYPES 16
+
+typedef struct gs_ctx gs_ctx;   /* opaque; owns only scratch memory and a status word */
+
+enum gs_error {
+    GS_OK = 0,
+    GS_ERR_INVALID_ARG = -1,    /* NULL pointer, negative size, n_instances < 1, ... */
+    GS_ERR_CAPACITY = -2,       /* n_instances or n_types above what the context was created for */
+    GS_ERR_CUDA = -3,           /* a CUDA runtime call failed; see gs_last_cuda_error */
+    GS_ERR_ALIGN = -4,          /* an array pointer is not 16-byte aligned */
+    GS_ERR_NO_DEVICE = -5       /* no usable CUDA device */
+};
+
+/* bits of the device status word */
+enum gs_dev_status {
+    GS_DEV_BAD_INSTANCE = 1,    /* assigned_inst outside [0, n_instances) was clamped */
+    GS_DEV_BAD_TYPE = 2,        /* type_id outside [0, n_types) was read as 0 */
+    GS_DEV_BAD_VALUE = 4,       /* negative count or negative/NaN q_ema was read as 0 */
+    GS_DEV_TIMEOUT = 8,         /* a bounded device-side wait expired (results of that call are invalid) */
+    GS_DEV_CAND_TRUNCATED = 16  /* more flagged requests than cand_capacity; list was cut */
+};
+
+/* gs_route_batch flags */
+#define GS_ROUTE_ACCUMULATE 1u  /* also add this round's assignments to the context's pending
+                                   per-instance deltas, to be applied by gs_advance_state */
+
+/* Per-instance serving state, structure of arrays, n_instances entries each.
+ * Together with the type table these give the coefficients of Eq. 2:
+ *   p_g = prefill_ms_per_tok[type_id[g]]
+ *   d_g = tpot_a_ms[t] + tpot_b_ms[t] * decode_batch[g]       (per-token decode latency under load)
+ *   w_g = queued_prefill_tokens[g] * p_g                      (stand-in for the observed wait)
+ *   q_g = alpha * w_g + (1 - alpha) * q_ema_ms[g]             (EMA step of Algorithm 1)
+ * free_kv_tokens[g] bounds L_in + L_out of a request placed on g (the memory constraint). */
+typedef struct gs_instances {
+    const int32_t *type_id;
+    const int32_t *queued_prefill_tokens;
+    const int32_t *decode_batch;
+    const int32_t *free_kv_tokens;
+    const float   *q_ema_ms;
+    int32_t        n_instances;      /* 1 .. GS_MAX_INSTANCES */
+} gs_instances;
+
+/* Per-GPU-type constants, n_types entries each (1 .. GS_MAX_TYPES). */
+typedef struct gs_types {
+    const float *prefill_ms_per_tok;
+    const float *tpot_a_ms;
+    const float *tpot_b_ms;
+    int32_t      n_types;
+} gs_types;
+
+/* Mutable view of the same instance state for gs_advance_state. */
+typedef struct gs_instances_mut {
+    int32_t *queued_prefill_tokens;
+    int32_t *decode_batch;
+    int32_t *free_kv_tokens;
+    float   *q_ema_ms;
+    int32_t  n_instances;
+} gs_instances_mut;
+
+/* Create a context on CUDA device `device` for pools of up to `max_instances` instances and
+ * `max_types` types.  Allocates the context's scratch memory (a few MB) with cudaMalloc.
+ * `*out` receives the context; destroy it with gs_destroy. */
+GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types);
+
+/* Frees everything the context owns.  The caller makes sure no call is still running. */
+GS_API int gs_destroy(gs_ctx *ctx);
+
+/* Static, never-NULL description of a gs_error code. */
+GS_API const char *gs_strerror(int code);
+
+/* cudaError_t of the last failed CUDA call of this context (0 if none), as int. */
+GS_API int gs_last_cuda_error(const gs_ctx *ctx);
+
+/* Synchronises `cuda_stream`, then reads and clears the device status word. */
+GS_API int gs_device_status(gs_ctx *ctx, void *cuda_stream, unsigned *out_bits);
+
+/* Number of kernels this context has launched since it was created. */
+GS_API int64_t gs_launch_count(const gs_ctx *ctx);
+
+/* Kernels of the library, for gs_timing_read. */
+enum gs_kernel {
+    GS_K_PROLOGUE = 0,       /* instance coefficients + preference order (per round) */
+    GS_K_ROUTE = 1,          /* pair scoring + selection */
+    GS_K_ADVANCE = 2,        /* state advance */
+    GS_K_RISK_FLAGS = 3,     /* risk test + flag words */
+    GS_K_RISK_OFFSETS = 4,   /* scan of per-chunk flag counts */
+    GS_K_RISK_SCATTER = 5,   /* ordered candidate list */
+    GS_K_COUNT = 6
+};
+
+/* Optional per-kernel timing for benchmarks.  While enabled (on != 0) every kernel launch of
+ * this context is bracketed by a pair of CUDA events on the launching stream.
+ * gs_timing_read waits for the recorded events, adds their durations to per-kernel totals,
+ * and returns the total milliseconds and number of launches of `kernel` since timing was
+ * last enabled.  Off by default; enabling it resets the totals. */
+GS_API int gs_timing_enable(gs_ctx *ctx, int on);
+GS_API int gs_timing_read(gs_ctx *ctx, int kernel, double *total_ms, int64_t *launches);
+
+/*
+ * One routing round (Algorithm 1 applied to every pending request against one snapshot of
+ * the instance state; the EMA step is taken once per round).
+ *
+ * Inputs, n_requests entries each:  prompt_len = L_in, pred_decode_len = predicted L_out,
+ * slo_ms = D_r.   Outputs, n_requests entries each:
+ *   out_instance_idx  g*            (index into the caller's instance arrays)
+ *   out_est_e2e_ms    T(r, g*)      computed as fma(d, L_out, fma(p, L_in, q)) in float
+ *   out_slack_ms      D_r - T(r, g*)
+ *   out_tier          (may be NULL) 1 = just-enough pick among feasible instances,
+ *                     2 = no feasible instance: minimum T among instances with KV room,
+ *                     3 = no instance has KV room: minimum T among all.
+ * Ties (equal d_g, or equal T in the fallback) go to the smallest instance index.
+ * Feasibility is T <= D (a request whose estimate equals its deadline is feasible).
+ * n_requests == 0 is valid and enqueues nothing.  Never writes the instance state.
+ */
+GS_API int gs_route_batch(gs_ctx *ctx,
+                   const int32_t *prompt_len, const int32_t *pred_decode_len,
+                   const float *slo_ms, int64_t n_requests,
+                   const gs_instances *inst, const gs_types *types, float ema_alpha,
+                   int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                   uint8_t *out_tier, unsigned flags, void *cuda_stream);
+
+/*
+ * Applies the deltas accumulated by gs_route_batch(..., GS_ROUTE_ACCUMULATE) since the last
+ * advance: per instance g,  queued_prefill_tokens += sum of L_in routed to g  (saturating at
+ * INT32_MAX), decode_batch += number of requests routed to g (saturating),
+ * free_kv_tokens = max(free_kv_tokens - sum of (L_in + L_out), 0), and q_ema_ms = q_g of the
+ * latest round.  Clears the pending deltas.  Integer sums, so the result does not depend on
+ * the order in which requests were processed.
+ */
+GS_API int gs_advance_state(gs_ctx *ctx, const gs_instances_mut *inst, void *cuda_stream);
+
+/*
+ * SLO-violation risk scan over n_active ongoing requests (Sec. 3.4).  Per request i:
+ *   rem    = max(pred_len[i] - generated_tokens[i], 0)      (pred_len is the re-estimated TOTAL)
+ *   finish = fma(d_{assigned_inst[i]}, rem, elapsed_ms[i])
+ *   flag   = finish > slo_ms[i]                              (strict: "exceeds")
+ * Outputs: out_flag_bits, ceil(n_active / 32) words, request i is bit (i % 32) of word
+ * (i / 32), unused high bits zero; out_cand_idx, the ascending indices of flagged requests,
+ * at most cand_capacity of them (may be NULL when cand_capacity == 0); out_cand_count, ONE
+ * int64 on the device that receives the TRUE number of flagged requests even when it exceeds
+ * cand_capacity (then GS_DEV_CAND_TRUNCATED is set).  n_active must be < 2^31.
+ */
+GS_API int gs_risk_scan(gs_ctx *ctx,
+                 const int32_t *assigned_inst, const int32_t *generated_tokens,
+                 const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                 int64_t n_active,
+                 const gs_instances *inst, const gs_types *types,
+                 uint32_t *out_flag_bits, int32_t *out_cand_idx, int64_t cand_capacity,
+                 int64_t *out_cand_count, void *cuda_stream);
+
+/*
+ * Host-buffer variants: every pointer (including those inside `inst` and `types`) is a HOST
+ * pointer.  The call copies the inputs to context-owned device buffers (grown with
+ * cudaMalloc when a larger size is first seen), runs the same kernels, copies the results
+ * back and synchronises `cuda_stream` before returning.  No alignment requirement.
+ * gs_risk_scan_host writes the true count to *out_cand_count (host) and returns at most
+ * cand_capacity indices.
+ */
+GS_API int gs_route_batch_host(gs_ctx *ctx,
+                        const int32_t *prompt_len, const int32_t *pred_decode_len,
+                        const float *slo_ms, int64_t n_requests,
+                        const gs_instances *inst, const gs_types *types, float ema_alpha,
+                        int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                        uint8_t *out_tier, void *cuda_stream);
+
+GS_API int gs_risk_scan_host(gs_ctx *ctx,
+                      const int32_t *assigned_inst, const int32_t *generated_tokens,
+                      const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                      int64_t n_active,
+                      const gs_instances *inst, const gs_types *types,
+                      uint32_t *out_flag_bits, int32_t *out_cand_idx, int64_t cand_capacity,
+                      int64_t *out_cand_count, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GOODSERVE_H_ */

@@ -1,0 +1,311 @@
+"""ctypes binding with the same names as the C ABI (see include/goodserve.h).
+
+Argument marshalling only: tensors are checked (device, dtype, contiguity) and their
+addresses handed to the library.  PyTorch supplies device memory and streams, nothing else.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+GS_ROUTE_ACCUMULATE = 1
+
+
+class DeviceStatus:
+    BAD_INSTANCE = 1
+    BAD_TYPE = 2
+    BAD_VALUE = 4
+    TIMEOUT = 8
+    CAND_TRUNCATED = 16
+
+
+class GoodServeError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"libgoodserve error {code}: {message}")
+        self.code = code
+
+
+class _Instances(C.Structure):
+    _fields_ = [("type_id", C.c_void_p), ("queued_prefill_tokens", C.c_void_p),
+                ("decode_batch", C.c_void_p), ("free_kv_tokens", C.c_void_p),
+                ("q_ema_ms", C.c_void_p), ("n_instances", C.c_int32)]
+
+
+class _Types(C.Structure):
+    _fields_ = [("prefill_ms_per_tok", C.c_void_p), ("tpot_a_ms", C.c_void_p),
+                ("tpot_b_ms", C.c_void_p), ("n_types", C.c_int32)]
+
+
+class _InstancesMut(C.Structure):
+    _fields_ = [("queued_prefill_tokens", C.c_void_p), ("decode_batch", C.c_void_p),
+                ("free_kv_tokens", C.c_void_p), ("q_ema_ms", C.c_void_p),
+                ("n_instances", C.c_int32)]
+
+
+def library_path() -> str:
+    return os.path.join(_PKG, "libgoodserve.so")
+
+
+_lib = None
+
+
+def load_library(build_if_missing: bool = True):
+    """Loads libgoodserve.so (building it with nvcc first if it is absent or stale).
+    Raises if that fails -- there is no other implementation to fall back to."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if build_if_missing:
+        from .build import build_library
+        try:
+            build_library()
+        except Exception as exc:                      # nvcc missing on a box that has the .so
+            if not os.path.exists(path):
+                raise RuntimeError(f"libgoodserve.so is missing and could not be built: {exc}") from exc
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} not found; run paper_2605_16867_b200/build.py")
+    lib = C.CDLL(path)
+    vp, i32, i64, f32, u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_uint
+    lib.gs_create.argtypes = [C.POINTER(vp), C.c_int, C.c_int, C.c_int]
+    lib.gs_destroy.argtypes = [vp]
+    lib.gs_strerror.argtypes = [C.c_int]
+    lib.gs_strerror.restype = C.c_char_p
+    lib.gs_last_cuda_error.argtypes = [vp]
+    lib.gs_device_status.argtypes = [vp, vp, C.POINTER(u32)]
+    lib.gs_launch_count.argtypes = [vp]
+    lib.gs_launch_count.restype = i64
+    route_args = [vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types), f32, vp, vp, vp, vp]
+    lib.gs_route_batch.argtypes = route_args + [u32, vp]
+    lib.gs_route_batch_host.argtypes = route_args + [vp]
+    lib.gs_advance_state.argtypes = [vp, C.POINTER(_InstancesMut), vp]
+    risk_args = [vp, vp, vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types), vp, vp, i64, vp, vp]
+    lib.gs_risk_scan.argtypes = risk_args
+    lib.gs_risk_scan_host.argtypes = risk_args
+    lib.gs_timing_enable.argtypes = [vp, C.c_int]
+    lib.gs_timing_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(i64)]
+    for name in ("gs_timing_enable", "gs_timing_read", "gs_create", "gs_destroy", "gs_last_cuda_error", "gs_device_status", "gs_route_batch",
+                 "gs_route_batch_host", "gs_advance_state", "gs_risk_scan", "gs_risk_scan_host"):
+        getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _dev_ptr(t: Optional[torch.Tensor], dtype: torch.dtype, n: Optional[int], name: str, device) -> Optional[int]:
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name}: expected a CUDA tensor")
+    if t.device != device:
+        raise ValueError(f"{name}: tensor is on {t.device}, context is on {device}")
+    if t.dtype != dtype or not t.is_contiguous() or t.dim() != 1:
+        raise TypeError(f"{name}: expected a contiguous 1-D {dtype} tensor, got {t.dtype} {tuple(t.shape)}")
+    if n is not None and t.numel() < n:
+        raise ValueError(f"{name}: needs {n} elements, has {t.numel()}")
+    return t.data_ptr()
+
+
+def _host_ptr(a, dtype, n: Optional[int], name: str) -> Optional[int]:
+    if a is None:
+        return None
+    if isinstance(a, torch.Tensor):
+        if a.is_cuda or not a.is_contiguous():
+            raise TypeError(f"{name}: expected a contiguous host tensor")
+        if n is not None and a.numel() < n:
+            raise ValueError(f"{name}: needs {n} elements, has {a.numel()}")
+        return a.data_ptr()
+    if not isinstance(a, np.ndarray) or a.dtype != dtype or not a.flags.c_contiguous:
+        raise TypeError(f"{name}: expected a contiguous numpy array of {dtype}")
+    if n is not None and a.size < n:
+        raise ValueError(f"{name}: needs {n} elements, has {a.size}")
+    return a.ctypes.data
+
+
+@dataclass
+class InstancePool:
+    """Device-resident pool description: per-instance state (SoA) and the type table."""
+    type_id: torch.Tensor
+    queued_prefill_tokens: torch.Tensor
+    decode_batch: torch.Tensor
+    free_kv_tokens: torch.Tensor
+    q_ema_ms: torch.Tensor
+    prefill_ms_per_tok: torch.Tensor
+    tpot_a_ms: torch.Tensor
+    tpot_b_ms: torch.Tensor
+
+    @property
+    def n_instances(self) -> int:
+        return int(self.type_id.numel())
+
+    @property
+    def n_types(self) -> int:
+        return int(self.prefill_ms_per_tok.numel())
+
+    @staticmethod
+    def from_host(types, inst, device) -> "InstancePool":
+        def up(a):
+            return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+        return InstancePool(up(inst.type_id), up(inst.queued_prefill_tokens), up(inst.decode_batch),
+                            up(inst.free_kv_tokens), up(inst.q_ema_ms), up(types.prefill_ms_per_tok),
+                            up(types.tpot_a_ms), up(types.tpot_b_ms))
+
+
+class GoodServe:
+    """One library context (gs_create / gs_destroy) bound to a CUDA device."""
+
+    def __init__(self, device: int = 0, max_instances: int = 1024, max_types: int = 16):
+        if not torch.cuda.is_available():
+            raise RuntimeError("GoodServe needs a CUDA device; there is no CPU implementation")
+        self._lib = load_library()
+        self.device = torch.device("cuda", device)
+        torch.cuda.init()
+        with torch.cuda.device(self.device):
+            torch.zeros(1, device=self.device)          # make sure the primary context exists
+        h = C.c_void_p()
+        self._check(self._lib.gs_create(C.byref(h), device, max_instances, max_types))
+        self._h = h
+
+    # -- plumbing ------------------------------------------------------------------------
+    def _check(self, rc: int):
+        if rc != 0:
+            raise GoodServeError(rc, self._lib.gs_strerror(rc).decode())
+
+    def _stream(self, stream) -> Optional[int]:
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        return s.cuda_stream or None
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.gs_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _pool_structs(self, pool: InstancePool):
+        M, Tn, dev = pool.n_instances, pool.n_types, self.device
+        i32, f32 = torch.int32, torch.float32
+        inst = _Instances(_dev_ptr(pool.type_id, i32, M, "type_id", dev),
+                          _dev_ptr(pool.queued_prefill_tokens, i32, M, "queued_prefill_tokens", dev),
+                          _dev_ptr(pool.decode_batch, i32, M, "decode_batch", dev),
+                          _dev_ptr(pool.free_kv_tokens, i32, M, "free_kv_tokens", dev),
+                          _dev_ptr(pool.q_ema_ms, f32, M, "q_ema_ms", dev), M)
+        types = _Types(_dev_ptr(pool.prefill_ms_per_tok, f32, Tn, "prefill_ms_per_tok", dev),
+                       _dev_ptr(pool.tpot_a_ms, f32, Tn, "tpot_a_ms", dev),
+                       _dev_ptr(pool.tpot_b_ms, f32, Tn, "tpot_b_ms", dev), Tn)
+        return inst, types
+
+    @staticmethod
+    def _host_pool_structs(types, inst):
+        M, Tn = int(inst.type_id.shape[0]), int(types.prefill_ms_per_tok.shape[0])
+        hi = _Instances(_host_ptr(inst.type_id, np.int32, M, "type_id"),
+                        _host_ptr(inst.queued_prefill_tokens, np.int32, M, "queued_prefill_tokens"),
+                        _host_ptr(inst.decode_batch, np.int32, M, "decode_batch"),
+                        _host_ptr(inst.free_kv_tokens, np.int32, M, "free_kv_tokens"),
+                        _host_ptr(inst.q_ema_ms, np.float32, M, "q_ema_ms"), M)
+        ht = _Types(_host_ptr(types.prefill_ms_per_tok, np.float32, Tn, "prefill_ms_per_tok"),
+                    _host_ptr(types.tpot_a_ms, np.float32, Tn, "tpot_a_ms"),
+                    _host_ptr(types.tpot_b_ms, np.float32, Tn, "tpot_b_ms"), Tn)
+        return hi, ht
+
+    # -- C ABI, same names ----------------------------------------------------------------
+    def route_batch(self, prompt_len, pred_decode_len, slo_ms, pool: InstancePool, ema_alpha: float,
+                    out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier=None,
+                    accumulate: bool = False, n_requests: Optional[int] = None, stream=None):
+        n = int(prompt_len.numel()) if n_requests is None else int(n_requests)
+        dev, i32, f32 = self.device, torch.int32, torch.float32
+        inst, types = self._pool_structs(pool)
+        self._check(self._lib.gs_route_batch(
+            self._h, _dev_ptr(prompt_len, i32, n, "prompt_len", dev),
+            _dev_ptr(pred_decode_len, i32, n, "pred_decode_len", dev),
+            _dev_ptr(slo_ms, f32, n, "slo_ms", dev), n, C.byref(inst), C.byref(types),
+            float(ema_alpha), _dev_ptr(out_instance_idx, i32, n, "out_instance_idx", dev),
+            _dev_ptr(out_est_e2e_ms, f32, n, "out_est_e2e_ms", dev),
+            _dev_ptr(out_slack_ms, f32, n, "out_slack_ms", dev),
+            _dev_ptr(out_tier, torch.uint8, n, "out_tier", dev),
+            GS_ROUTE_ACCUMULATE if accumulate else 0, self._stream(stream)))
+
+    def advance_state(self, pool: InstancePool, stream=None):
+        M, dev, i32 = pool.n_instances, self.device, torch.int32
+        mut = _InstancesMut(_dev_ptr(pool.queued_prefill_tokens, i32, M, "queued_prefill_tokens", dev),
+                            _dev_ptr(pool.decode_batch, i32, M, "decode_batch", dev),
+                            _dev_ptr(pool.free_kv_tokens, i32, M, "free_kv_tokens", dev),
+                            _dev_ptr(pool.q_ema_ms, torch.float32, M, "q_ema_ms", dev), M)
+        self._check(self._lib.gs_advance_state(self._h, C.byref(mut), self._stream(stream)))
+
+    def risk_scan(self, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms,
+                  pool: InstancePool, out_flag_bits, out_cand_idx, out_cand_count,
+                  cand_capacity: Optional[int] = None, n_active: Optional[int] = None, stream=None):
+        n = int(assigned_inst.numel()) if n_active is None else int(n_active)
+        cap = (0 if out_cand_idx is None else int(out_cand_idx.numel())) if cand_capacity is None else int(cand_capacity)
+        dev, i32, f32 = self.device, torch.int32, torch.float32
+        inst, types = self._pool_structs(pool)
+        self._check(self._lib.gs_risk_scan(
+            self._h, _dev_ptr(assigned_inst, i32, n, "assigned_inst", dev),
+            _dev_ptr(generated_tokens, i32, n, "generated_tokens", dev),
+            _dev_ptr(pred_len, i32, n, "pred_len", dev),
+            _dev_ptr(elapsed_ms, f32, n, "elapsed_ms", dev), _dev_ptr(slo_ms, f32, n, "slo_ms", dev), n,
+            C.byref(inst), C.byref(types),
+            _dev_ptr(out_flag_bits, i32, (n + 31) // 32, "out_flag_bits", dev),
+            _dev_ptr(out_cand_idx, i32, cap, "out_cand_idx", dev), cap,
+            _dev_ptr(out_cand_count, torch.int64, 1, "out_cand_count", dev), self._stream(stream)))
+
+    def route_batch_host(self, prompt_len, pred_decode_len, slo_ms, types, inst, ema_alpha: float,
+                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier=None, stream=None):
+        """Host-buffer variant: numpy arrays or (pinned) host tensors in and out."""
+        n = int(prompt_len.shape[0])
+        hi, ht = self._host_pool_structs(types, inst)
+        self._check(self._lib.gs_route_batch_host(
+            self._h, _host_ptr(prompt_len, np.int32, n, "prompt_len"),
+            _host_ptr(pred_decode_len, np.int32, n, "pred_decode_len"),
+            _host_ptr(slo_ms, np.float32, n, "slo_ms"), n, C.byref(hi), C.byref(ht), float(ema_alpha),
+            _host_ptr(out_instance_idx, np.int32, n, "out_instance_idx"),
+            _host_ptr(out_est_e2e_ms, np.float32, n, "out_est_e2e_ms"),
+            _host_ptr(out_slack_ms, np.float32, n, "out_slack_ms"),
+            _host_ptr(out_tier, np.uint8, n, "out_tier"), self._stream(stream)))
+
+    def risk_scan_host(self, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, types, inst,
+                       out_flag_bits, out_cand_idx, stream=None) -> int:
+        """Host-buffer variant; returns the true number of flagged requests."""
+        n = int(assigned_inst.shape[0])
+        cap = 0 if out_cand_idx is None else int(out_cand_idx.shape[0])
+        hi, ht = self._host_pool_structs(types, inst)
+        count = C.c_int64(0)
+        self._check(self._lib.gs_risk_scan_host(
+            self._h, _host_ptr(assigned_inst, np.int32, n, "assigned_inst"),
+            _host_ptr(generated_tokens, np.int32, n, "generated_tokens"),
+            _host_ptr(pred_len, np.int32, n, "pred_len"),
+            _host_ptr(elapsed_ms, np.float32, n, "elapsed_ms"), _host_ptr(slo_ms, np.float32, n, "slo_ms"), n,
+            C.byref(hi), C.byref(ht), _host_ptr(out_flag_bits, np.uint32, (n + 31) // 32, "out_flag_bits"),
+            _host_ptr(out_cand_idx, np.int32, cap, "out_cand_idx"), cap,
+            C.cast(C.byref(count), C.c_void_p), self._stream(stream)))
+        return int(count.value)
+
+    def device_status(self, stream=None) -> int:
+        bits = C.c_uint(0)
+        self._check(self._lib.gs_device_status(self._h, self._stream(stream), C.byref(bits)))
+        return int(bits.value)
+
+    def launch_count(self) -> int:
+        return int(self._lib.gs_launch_count(self._h))
+
+    def timing_enable(self, on: bool):
+        self._check(self._lib.gs_timing_enable(self._h, 1 if on else 0))
+
+    def timing_read(self, kernel: int):
+        """(total milliseconds, launches) of one kernel since timing was enabled."""
+        ms, n = C.c_double(0.0), C.c_int64(0)
+        self._check(self._lib.gs_timing_read(self._h, int(kernel), C.byref(ms), C.byref(n)))
+        return float(ms.value), int(n.value)
+
+    def last_cuda_error(self) -> int:
+        return int(self._lib.gs_last_cuda_error(self._h))

@@ -1,0 +1,397 @@
+// C-ABI entry points of libgoodserve: argument checks, context lifetime, kernel sequencing.
+#include <new>
+#include <stdint.h>
+#include <string.h>
+
+#include "gs_internal.cuh"
+
+namespace {
+
+inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+int cuda_fail(gs_ctx *ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda_error = (int)e;
+    return GS_ERR_CUDA;
+}
+
+// Makes the context's device current for the duration of a call.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+int check_pool(const gs_ctx *ctx, const gs_instances *inst, const gs_types *types, bool device_ptrs) {
+    if (!ctx || !inst || !types) return GS_ERR_INVALID_ARG;
+    if (inst->n_instances < 1 || types->n_types < 1) return GS_ERR_INVALID_ARG;
+    if (inst->n_instances > ctx->max_instances || types->n_types > ctx->max_types) return GS_ERR_CAPACITY;
+    const void *ptrs[] = {inst->type_id, inst->queued_prefill_tokens, inst->decode_batch,
+                          inst->free_kv_tokens, inst->q_ema_ms, types->prefill_ms_per_tok,
+                          types->tpot_a_ms, types->tpot_b_ms};
+    for (const void *p : ptrs) if (!p) return GS_ERR_INVALID_ARG;
+    if (device_ptrs)
+        for (int k = 0; k < 5; ++k) if (misaligned(ptrs[k])) return GS_ERR_ALIGN;
+    return GS_OK;
+}
+
+int ensure_stage(gs_ctx *ctx, size_t bytes) {
+    if (bytes <= ctx->stage_bytes) return GS_OK;
+    if (ctx->stage) { cudaFree(ctx->stage); ctx->stage = nullptr; ctx->stage_bytes = 0; }
+    const size_t want = bytes + bytes / 8 + 4096;
+    cudaError_t e = cudaMalloc(&ctx->stage, want);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->stage_bytes = want;
+    return GS_OK;
+}
+
+inline size_t pad256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+// Bump allocator over the staging buffer.
+struct Carver {
+    char *base; size_t off = 0;
+    template <typename T> T *take(size_t count) {
+        T *p = reinterpret_cast<T *>(base + off);
+        off += pad256(count * sizeof(T));
+        return p;
+    }
+};
+
+// Device copies of a host-side pool description; returns bytes needed when base == nullptr.
+struct PoolStage {
+    gs_instances inst;
+    gs_types types;
+};
+
+size_t pool_stage_bytes(int M, int Tn) { return 5 * pad256((size_t)M * 4) + 3 * pad256((size_t)Tn * 4); }
+
+cudaError_t stage_pool(Carver &c, const gs_instances *h_inst, const gs_types *h_types,
+                       PoolStage *out, cudaStream_t st) {
+    const int M = h_inst->n_instances, Tn = h_types->n_types;
+    int32_t *type_id = c.take<int32_t>(M), *queued = c.take<int32_t>(M), *batch = c.take<int32_t>(M),
+            *kv = c.take<int32_t>(M);
+    float *qe = c.take<float>(M), *p = c.take<float>(Tn), *a = c.take<float>(Tn), *b = c.take<float>(Tn);
+    const void *src[] = {h_inst->type_id, h_inst->queued_prefill_tokens, h_inst->decode_batch,
+                         h_inst->free_kv_tokens, h_inst->q_ema_ms, h_types->prefill_ms_per_tok,
+                         h_types->tpot_a_ms, h_types->tpot_b_ms};
+    void *dst[] = {type_id, queued, batch, kv, qe, p, a, b};
+    for (int k = 0; k < 8; ++k) {
+        cudaError_t e = cudaMemcpyAsync(dst[k], src[k], (size_t)(k < 5 ? M : Tn) * 4,
+                                        cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return e;
+    }
+    out->inst = gs_instances{type_id, queued, batch, kv, qe, M};
+    out->types = gs_types{p, a, b, Tn};
+    return cudaSuccess;
+}
+
+}  // namespace
+
+namespace gs {
+
+LaunchTimer::LaunchTimer(gs_ctx *c, int k, cudaStream_t s) : ctx(c), st(s), kernel(k) {
+    ctx->launches += 1;
+    if (!ctx->timing) return;
+    for (cudaEvent_t *ev : {&start, &stop}) {
+        if (!ctx->free_events->empty()) { *ev = ctx->free_events->back(); ctx->free_events->pop_back(); }
+        else if (cudaEventCreate(ev) != cudaSuccess) { *ev = nullptr; }
+    }
+    if (start && stop) cudaEventRecord(start, st);
+}
+
+LaunchTimer::~LaunchTimer() {
+    if (!ctx->timing || !start || !stop) return;
+    cudaEventRecord(stop, st);
+    ctx->pending->push_back({kernel, start, stop});
+}
+
+}  // namespace gs
+
+extern "C" {
+
+GS_API const char *gs_strerror(int code) {
+    switch (code) {
+        case GS_OK: return "ok";
+        case GS_ERR_INVALID_ARG: return "invalid argument (null pointer, negative size or empty pool)";
+        case GS_ERR_CAPACITY: return "pool larger than the context was created for";
+        case GS_ERR_CUDA: return "a CUDA runtime call failed (see gs_last_cuda_error)";
+        case GS_ERR_ALIGN: return "array pointer is not 16-byte aligned";
+        case GS_ERR_NO_DEVICE: return "no usable CUDA device";
+        default: return "unknown error code";
+    }
+}
+
+GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types) {
+    if (!out) return GS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (max_instances < 1 || max_types < 1) return GS_ERR_INVALID_ARG;
+    if (max_instances > GS_MAX_INSTANCES || max_types > GS_MAX_TYPES) return GS_ERR_CAPACITY;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev < 1 || device < 0 || device >= n_dev)
+        return GS_ERR_NO_DEVICE;
+    DeviceGuard guard(device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+
+    gs_ctx *ctx = new (std::nothrow) gs_ctx();
+    if (!ctx) return GS_ERR_INVALID_ARG;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->device = device;
+    ctx->max_instances = max_instances;
+    ctx->max_types = max_types;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) { delete ctx->pending; delete ctx->free_events; delete ctx; return GS_ERR_CUDA; }
+    ctx->n_sm = prop.multiProcessorCount;
+    ctx->pending = new (std::nothrow) std::vector<gs_ctx::TimedLaunch>();
+    ctx->free_events = new (std::nothrow) std::vector<cudaEvent_t>();
+    if (!ctx->pending || !ctx->free_events) { delete ctx->pending; delete ctx->free_events; delete ctx; return GS_ERR_INVALID_ARG; }
+    ctx->chunk_cap = ((size_t)gs::kMaxActive + gs::kRiskChunk - 1) / gs::kRiskChunk;
+
+    const size_t Mx = GS_MAX_INSTANCES;
+    gs::Scratch &s = ctx->s;
+    struct { void **p; size_t bytes; } allocs[] = {
+        {(void **)&s.rows, Mx * sizeof(gs::InstRow)},
+        {(void **)&s.row_g, Mx * sizeof(int)},
+        {(void **)&s.d_by_g, Mx * sizeof(float)},
+        {(void **)&s.q_by_g, Mx * sizeof(float)},
+        {(void **)&s.deltas, 3 * Mx * sizeof(unsigned long long)},
+        {(void **)&s.chunk_counts, (ctx->chunk_cap + 1) * sizeof(unsigned)},
+        {(void **)&s.status, 256},
+    };
+    for (auto &a : allocs) {
+        e = cudaMalloc(a.p, a.bytes);
+        if (e == cudaSuccess) e = cudaMemset(*a.p, 0, a.bytes);
+        if (e != cudaSuccess) { gs_destroy(ctx); return GS_ERR_CUDA; }
+    }
+    *out = ctx;
+    return GS_OK;
+}
+
+GS_API int gs_destroy(gs_ctx *ctx) {
+    if (!ctx) return GS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    gs::Scratch &s = ctx->s;
+    void *ptrs[] = {s.rows, s.row_g, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.status, ctx->stage};
+    for (void *p : ptrs) if (p) cudaFree(p);
+    if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
+    if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);
+    delete ctx->pending;
+    delete ctx->free_events;
+    delete ctx;
+    return GS_OK;
+}
+
+GS_API int gs_timing_enable(gs_ctx *ctx, int on) {
+    if (!ctx) return GS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    for (auto &t : *ctx->pending) { ctx->free_events->push_back(t.start); ctx->free_events->push_back(t.stop); }
+    ctx->pending->clear();
+    for (int k = 0; k < GS_K_COUNT; ++k) { ctx->time_ms[k] = 0.0; ctx->time_launches[k] = 0; }
+    ctx->timing = on != 0;
+    return GS_OK;
+}
+
+GS_API int gs_timing_read(gs_ctx *ctx, int kernel, double *total_ms, int64_t *launches) {
+    if (!ctx || kernel < 0 || kernel >= GS_K_COUNT || !total_ms || !launches) return GS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    for (auto &t : *ctx->pending) {
+        cudaError_t e = cudaEventSynchronize(t.stop);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, t.start, t.stop);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->time_ms[t.kernel] += (double)ms;
+        ctx->time_launches[t.kernel] += 1;
+        ctx->free_events->push_back(t.start);
+        ctx->free_events->push_back(t.stop);
+    }
+    ctx->pending->clear();
+    *total_ms = ctx->time_ms[kernel];
+    *launches = ctx->time_launches[kernel];
+    return GS_OK;
+}
+
+GS_API int gs_last_cuda_error(const gs_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+GS_API int64_t gs_launch_count(const gs_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+GS_API int gs_device_status(gs_ctx *ctx, void *cuda_stream, unsigned *out_bits) {
+    if (!ctx || !out_bits) return GS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess) e = cudaMemcpy(out_bits, ctx->s.status, sizeof(unsigned), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemset(ctx->s.status, 0, sizeof(unsigned));
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
+GS_API int gs_route_batch(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                   const float *slo_ms, int64_t n_requests,
+                   const gs_instances *inst, const gs_types *types, float ema_alpha,
+                   int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                   uint8_t *out_tier, unsigned flags, void *cuda_stream)
+{
+    int rc = check_pool(ctx, inst, types, true);
+    if (rc != GS_OK) return rc;
+    if (n_requests < 0 || (flags & ~GS_ROUTE_ACCUMULATE)) return GS_ERR_INVALID_ARG;
+    if (n_requests > 0) {
+        const void *ptrs[] = {prompt_len, pred_decode_len, slo_ms, out_instance_idx, out_est_e2e_ms, out_slack_ms};
+        for (const void *p : ptrs) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+        if (out_tier && misaligned(out_tier)) return GS_ERR_ALIGN;
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, inst->n_instances,
+                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier,
+                         (flags & GS_ROUTE_ACCUMULATE) != 0, st);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
+GS_API int gs_advance_state(gs_ctx *ctx, const gs_instances_mut *inst, void *cuda_stream) {
+    if (!ctx || !inst) return GS_ERR_INVALID_ARG;
+    if (inst->n_instances < 1) return GS_ERR_INVALID_ARG;
+    if (inst->n_instances > ctx->max_instances) return GS_ERR_CAPACITY;
+    const void *ptrs[] = {inst->queued_prefill_tokens, inst->decode_batch, inst->free_kv_tokens, inst->q_ema_ms};
+    for (const void *p : ptrs) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    cudaError_t e = gs::launch_advance(ctx, *inst, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
+GS_API int gs_risk_scan(gs_ctx *ctx, const int32_t *assigned_inst, const int32_t *generated_tokens,
+                 const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                 int64_t n_active, const gs_instances *inst, const gs_types *types,
+                 uint32_t *out_flag_bits, int32_t *out_cand_idx, int64_t cand_capacity,
+                 int64_t *out_cand_count, void *cuda_stream)
+{
+    int rc = check_pool(ctx, inst, types, true);
+    if (rc != GS_OK) return rc;
+    if (n_active < 0 || n_active > gs::kMaxActive || cand_capacity < 0 || !out_cand_count)
+        return GS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(out_cand_count) & 7u) return GS_ERR_ALIGN;
+    if (cand_capacity > 0 && !out_cand_idx) return GS_ERR_INVALID_ARG;
+    if (out_cand_idx && misaligned(out_cand_idx)) return GS_ERR_ALIGN;
+    if (n_active > 0) {
+        const void *ptrs[] = {assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, out_flag_bits};
+        for (const void *p : ptrs) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // the scan needs d_g only; the EMA weight does not enter it
+    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, 0.0f, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = gs::launch_risk(ctx, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, n_active,
+                        inst->n_instances, out_flag_bits, out_cand_idx, cand_capacity, out_cand_count, st);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
+GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                        const float *slo_ms, int64_t n_requests,
+                        const gs_instances *inst, const gs_types *types, float ema_alpha,
+                        int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                        uint8_t *out_tier, void *cuda_stream)
+{
+    int rc = check_pool(ctx, inst, types, false);
+    if (rc != GS_OK) return rc;
+    if (n_requests < 0) return GS_ERR_INVALID_ARG;
+    if (n_requests > 0 && (!prompt_len || !pred_decode_len || !slo_ms || !out_instance_idx ||
+                           !out_est_e2e_ms || !out_slack_ms)) return GS_ERR_INVALID_ARG;
+    if (n_requests == 0) return GS_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    const size_t n = (size_t)n_requests;
+    const size_t bytes = pool_stage_bytes(inst->n_instances, types->n_types) + 6 * pad256(n * 4) + pad256(n);
+    rc = ensure_stage(ctx, bytes);
+    if (rc != GS_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    Carver c{ctx->stage};
+    PoolStage pool;
+    cudaError_t e = stage_pool(c, inst, types, &pool, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    int32_t *dx = c.take<int32_t>(n), *dy = c.take<int32_t>(n);
+    float *dD = c.take<float>(n);
+    int32_t *didx = c.take<int32_t>(n);
+    float *dest = c.take<float>(n), *dslack = c.take<float>(n);
+    uint8_t *dtier = out_tier ? c.take<uint8_t>(n) : nullptr;
+    if ((e = cudaMemcpyAsync(dx, prompt_len, n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dy, pred_decode_len, n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dD, slo_ms, n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return cuda_fail(ctx, e);
+    rc = gs_route_batch(ctx, dx, dy, dD, n_requests, &pool.inst, &pool.types, ema_alpha,
+                        didx, dest, dslack, dtier, 0u, cuda_stream);
+    if (rc != GS_OK) return rc;
+    if ((e = cudaMemcpyAsync(out_instance_idx, didx, n * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(out_est_e2e_ms, dest, n * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(out_slack_ms, dslack, n * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return cuda_fail(ctx, e);
+    if (out_tier && (e = cudaMemcpyAsync(out_tier, dtier, n, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return cuda_fail(ctx, e);
+    e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
+GS_API int gs_risk_scan_host(gs_ctx *ctx, const int32_t *assigned_inst, const int32_t *generated_tokens,
+                      const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                      int64_t n_active, const gs_instances *inst, const gs_types *types,
+                      uint32_t *out_flag_bits, int32_t *out_cand_idx, int64_t cand_capacity,
+                      int64_t *out_cand_count, void *cuda_stream)
+{
+    int rc = check_pool(ctx, inst, types, false);
+    if (rc != GS_OK) return rc;
+    if (n_active < 0 || n_active > gs::kMaxActive || cand_capacity < 0 || !out_cand_count)
+        return GS_ERR_INVALID_ARG;
+    if (cand_capacity > 0 && !out_cand_idx) return GS_ERR_INVALID_ARG;
+    if (n_active > 0 && (!assigned_inst || !generated_tokens || !pred_len || !elapsed_ms || !slo_ms ||
+                         !out_flag_bits)) return GS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    const size_t n = (size_t)n_active;
+    const size_t words = (n + 31) / 32;
+    const size_t cap = (size_t)(cand_capacity < n_active ? cand_capacity : n_active);
+    const size_t bytes = pool_stage_bytes(inst->n_instances, types->n_types) + 5 * pad256(n * 4) +
+                         pad256(words * 4) + pad256(cap * 4) + 256;
+    rc = ensure_stage(ctx, bytes);
+    if (rc != GS_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    Carver c{ctx->stage};
+    PoolStage pool;
+    cudaError_t e = stage_pool(c, inst, types, &pool, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    int32_t *dg = c.take<int32_t>(n), *dgen = c.take<int32_t>(n), *dtot = c.take<int32_t>(n);
+    float *del = c.take<float>(n), *dslo = c.take<float>(n);
+    uint32_t *dbits = c.take<uint32_t>(words);
+    int32_t *dcand = c.take<int32_t>(cap);
+    int64_t *dcount = c.take<int64_t>(1);
+    const void *src[] = {assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms};
+    void *dst[] = {dg, dgen, dtot, del, dslo};
+    for (int k = 0; k < 5 && n > 0; ++k)
+        if ((e = cudaMemcpyAsync(dst[k], src[k], n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+            return cuda_fail(ctx, e);
+    rc = gs_risk_scan(ctx, dg, dgen, dtot, del, dslo, n_active, &pool.inst, &pool.types,
+                      dbits, cap ? dcand : nullptr, (int64_t)cap, dcount, cuda_stream);
+    if (rc != GS_OK) return rc;
+    int64_t count = 0;
+    if ((e = cudaMemcpyAsync(&count, dcount, sizeof(count), cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return cuda_fail(ctx, e);
+    if (words && (e = cudaMemcpyAsync(out_flag_bits, dbits, words * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return cuda_fail(ctx, e);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(ctx, e);
+    *out_cand_count = count;
+    const size_t n_out = (size_t)(count < (int64_t)cap ? count : (int64_t)cap);
+    if (n_out) {
+        e = cudaMemcpyAsync(out_cand_idx, dcand, n_out * 4, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    return GS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,313 @@
+"""GPU parity: the CUDA path, called through the C ABI (ctypes binding), against the CPU
+oracle on the same seeded inputs.  Integer results (instance index, tier, flag bits,
+candidate list, advanced state) are compared bit for bit with the oracle's fixed-order
+single-precision mode; latency estimates are compared with the fp64 oracle within 1e-5
+relative, and any index that differs from the fp64 oracle must be a documented near-tie."""
+import numpy as np
+import pytest
+
+import oracle
+import workloads as W
+from parity_util import (REL_TOL, assert_route_matches_f32_oracle, check_risk_against_f64,
+                         check_route_against_f64, gpu_risk, gpu_route, unpack_bits)
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def gs():
+    from paper_2605_16867_b200 import GoodServe
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    ctx = GoodServe(0)
+    yield ctx
+    ctx.close()
+
+
+def pool_of(gs, types, inst):
+    from paper_2605_16867_b200 import InstancePool
+    return InstancePool.from_host(types, inst, gs.device)
+
+
+def run_config(gs, wl, threads=8):
+    alpha = wl.ema_alpha
+    pool = pool_of(gs, wl.types, wl.instances)
+    t32 = oracle.instance_table(wl.types, wl.instances, alpha, "f32")
+    t64 = oracle.instance_table(wl.types, wl.instances, alpha, "f64")
+    got = gpu_route(gs, pool, wl.requests, alpha)
+    ref = oracle.route(t32, *wl.requests.columns(), threads=threads)
+    assert_route_matches_f32_oracle(got, ref)
+    n_tie = check_route_against_f64(got, t64, wl.requests)
+    # invariant: whenever any instance meets deadline and KV, the chosen one does
+    t1 = got.tier == 1
+    assert (got.slack_ms[t1] >= 0).all() and (got.slack_ms[got.tier == 2] < 0).all()
+
+    risk, _ = gpu_risk(gs, pool, wl.active)
+    rref = oracle.risk(t32, *wl.active.columns(), threads=threads)
+    bits, cand, count = oracle.compact(rref.flag)
+    np.testing.assert_array_equal(risk.flag_bits, bits)
+    assert risk.count == count
+    np.testing.assert_array_equal(risk.cand_idx, cand)
+    n_flag_tie = check_risk_against_f64(unpack_bits(risk.flag_bits, wl.active.n), t64, wl.active)
+    assert gs.device_status() == 0
+    print(f"cfg {wl.cfg.cfg_id}: N={wl.requests.n} M={wl.instances.n_instances} A={wl.active.n} "
+          f"tiers={[int((got.tier == k).sum()) for k in (1, 2, 3)]} flagged={count} "
+          f"near-tie index mismatches vs fp64={n_tie}, flag mismatches vs fp64={n_flag_tie}")
+
+
+@pytest.mark.parametrize("cfg_id", [0, 1, 2])
+def test_config_full_size(gs, cfg_id):
+    run_config(gs, W.make_workload(cfg_id))
+
+
+def test_config3_full_size(gs):
+    """Largest shape: 4,194,304 requests x 1,024 instances, 16,777,216 active requests."""
+    run_config(gs, W.make_workload(3))
+
+
+def test_config4_stream(gs):
+    """64 dependent rounds with state advance on the device, a risk scan after every 8th
+    round against the advanced state; the whole trajectory must match the oracle's."""
+    wl = W.make_workload(4)
+    alpha = wl.ema_alpha
+    pool = pool_of(gs, wl.types, wl.instances)
+    state = wl.instances.copy()
+    for k in range(wl.cfg.n_rounds):
+        req = W.make_round_requests(wl, k)
+        got = gpu_route(gs, pool, req, alpha, accumulate=True)
+        gs.advance_state(pool)
+        t32 = oracle.instance_table(wl.types, state, alpha, "f32")
+        ref = oracle.route(t32, *req.columns(), threads=8)
+        assert_route_matches_f32_oracle(got, ref)
+        if k % 16 == 0:
+            check_route_against_f64(got, oracle.instance_table(wl.types, state, alpha, "f64"), req)
+        oracle.advance(state, t32, ref.instance_idx, req.prompt_len, req.pred_decode_len)
+        for dev_col, host_col in zip((pool.queued_prefill_tokens, pool.decode_batch, pool.free_kv_tokens),
+                                     (state.queued_prefill_tokens, state.decode_batch, state.free_kv_tokens)):
+            np.testing.assert_array_equal(dev_col.cpu().numpy(), host_col, err_msg=f"round {k}")
+        np.testing.assert_array_equal(pool.q_ema_ms.cpu().numpy().view(np.uint32),
+                                      state.q_ema_ms.view(np.uint32), err_msg=f"round {k}")
+        if k % 8 == 7:
+            risk, _ = gpu_risk(gs, pool, wl.active)
+            t32n = oracle.instance_table(wl.types, state, alpha, "f32")
+            rref = oracle.risk(t32n, *wl.active.columns(), threads=8)
+            bits, cand, count = oracle.compact(rref.flag)
+            np.testing.assert_array_equal(risk.flag_bits, bits)
+            np.testing.assert_array_equal(risk.cand_idx, cand)
+            assert risk.count == count
+    assert gs.device_status() == 0
+
+
+def test_runs_are_deterministic(gs):
+    wl = W.make_workload(2, n_requests=300_000, n_active=1_000_000)
+    pool = pool_of(gs, wl.types, wl.instances)
+    a = gpu_route(gs, pool, wl.requests, 0.5)
+    b = gpu_route(gs, pool, wl.requests, 0.5)
+    for u, v in ((a.instance_idx, b.instance_idx), (a.est_e2e_ms, b.est_e2e_ms), (a.tier, b.tier)):
+        assert u.tobytes() == v.tobytes()
+    ra, _ = gpu_risk(gs, pool, wl.active)
+    rb, _ = gpu_risk(gs, pool, wl.active)
+    assert ra.flag_bits.tobytes() == rb.flag_bits.tobytes() and ra.cand_idx.tobytes() == rb.cand_idx.tobytes()
+
+
+# --------------------------------------------------------------------------------------
+# edge sizes
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("M", [1, 2, 3, 31, 32, 33, 127, 1023, 1024])
+@pytest.mark.parametrize("N", [1, 3, 4, 5, 31, 32, 33, 1000, 4099])
+def test_ragged_sizes(gs, M, N):
+    types, inst = W.make_pool(M, min(M, 8), seed=100 + M)
+    cfg = W.CONFIGS[3]
+    req = W.make_requests(cfg, types, seed=7 * M + N, n=N)
+    act = W.make_active(cfg, types, M, seed=11 * M + N, n=N)
+    pool = pool_of(gs, types, inst)
+    t32 = oracle.instance_table(types, inst, 0.25, "f32")
+    assert_route_matches_f32_oracle(gpu_route(gs, pool, req, 0.25), oracle.route(t32, *req.columns()))
+    risk, _ = gpu_risk(gs, pool, act)
+    bits, cand, count = oracle.compact(oracle.risk(t32, *act.columns()).flag)
+    np.testing.assert_array_equal(risk.flag_bits, bits)
+    np.testing.assert_array_equal(risk.cand_idx, cand)
+    assert risk.count == count
+
+
+def test_empty_inputs(gs):
+    types, inst = W.make_pool(16, 4, seed=1)
+    pool = pool_of(gs, types, inst)
+    e_i = torch.empty(0, dtype=torch.int32, device=gs.device)
+    e_f = torch.empty(0, dtype=torch.float32, device=gs.device)
+    gs.route_batch(e_i, e_i, e_f, pool, 0.5, e_i, e_f, e_f)
+    count = torch.full((1,), -1, dtype=torch.int64, device=gs.device)
+    gs.risk_scan(e_i, e_i, e_i, e_f, e_f, pool, e_i, None, count, cand_capacity=0)
+    assert int(count.item()) == 0 and gs.device_status() == 0
+
+
+def test_all_tiers_and_boundaries(gs):
+    """The hand-worked pool: every tier, KV exactly enough, deadline exactly met."""
+    from test_oracle_pins import fixture_pool, read_rows
+    for name, D, k0, k1, k2, g, est, slack, tier in read_rows("handworked_routing.txt"):
+        types, inst = fixture_pool((int(k0), int(k1), int(k2)))
+        pool = pool_of(gs, types, inst)
+        req = W.RequestBatch(np.array([1000], np.int32), np.array([200], np.int32), np.array([float(D)], np.float32))
+        got = gpu_route(gs, pool, req, 0.5)
+        assert got.instance_idx[0] == int(g) and got.tier[0] == int(tier), name
+        assert got.est_e2e_ms[0] == pytest.approx(float(est), rel=REL_TOL), name
+    types, inst = fixture_pool()
+    pool = pool_of(gs, types, inst)
+    for name, pred, gen, elapsed, slo, finish, flag in read_rows("handworked_risk.txt"):
+        act = W.ActiveSet(np.array([1], np.int32), np.array([int(gen)], np.int32), np.array([int(pred)], np.int32),
+                          np.array([float(elapsed)], np.float32), np.array([float(slo)], np.float32))
+        risk, _ = gpu_risk(gs, pool, act)
+        assert risk.count == int(flag), name
+
+
+def test_extreme_values(gs):
+    """Huge token counts (L_in + L_out above 2^31), infinite / NaN / negative deadlines."""
+    types, inst = W.make_pool(64, 4, seed=3)
+    inst.free_kv_tokens[:8] = 2 ** 31 - 1
+    pool = pool_of(gs, types, inst)
+    x = np.array([2 ** 31 - 1, 2 ** 30, 16, 16, 16, 2 ** 31 - 1, 0, 5], np.int32)
+    y = np.array([2 ** 31 - 1, 2 ** 30, 8, 8, 8, 0, 0, 7], np.int32)
+    D = np.array([1e30, np.inf, np.nan, -1.0, 0.0, 1e12, 1.0, np.inf], np.float32)
+    req = W.RequestBatch(x, y, D)
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    got = gpu_route(gs, pool, req, 0.5)
+    ref = oracle.route(t32, x, y, D)
+    np.testing.assert_array_equal(got.instance_idx, ref.instance_idx)
+    np.testing.assert_array_equal(got.tier, ref.tier)
+    np.testing.assert_array_equal(got.est_e2e_ms.view(np.uint32), ref.est_e2e_ms.view(np.uint32))
+    assert {1, 2, 3} <= set(got.tier.tolist())
+    assert gs.device_status() == 0
+
+
+def test_invalid_data_sets_status_bits(gs):
+    from paper_2605_16867_b200 import DeviceStatus
+    types, inst = W.make_pool(32, 4, seed=5)
+    inst.type_id[3] = 99
+    inst.decode_batch[4] = -2
+    inst.q_ema_ms[5] = np.nan
+    pool = pool_of(gs, types, inst)
+    cfg = W.CONFIGS[1]
+    req = W.make_requests(cfg, types, seed=1, n=500)
+    req.prompt_len[17] = -40
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    got = gpu_route(gs, pool, req, 0.5)
+    assert_route_matches_f32_oracle(got, oracle.route(t32, *req.columns()))
+    st = gs.device_status()
+    assert st & DeviceStatus.BAD_TYPE and st & DeviceStatus.BAD_VALUE
+    act = W.make_active(cfg, types, 32, seed=2, n=700)
+    act.assigned_inst[5] = 32
+    act.assigned_inst[6] = -1
+    act.generated_tokens[7] = -3
+    risk, _ = gpu_risk(gs, pool, act)
+    rref = oracle.risk(t32, *act.columns())
+    np.testing.assert_array_equal(unpack_bits(risk.flag_bits, act.n), rref.flag)
+    st = gs.device_status()
+    assert st & DeviceStatus.BAD_INSTANCE and st & DeviceStatus.BAD_VALUE
+    assert gs.device_status() == 0         # reading clears
+
+
+def test_candidate_buffer_too_small(gs):
+    from paper_2605_16867_b200 import DeviceStatus
+    wl = W.make_workload(1, n_requests=16, n_active=50_000)
+    pool = pool_of(gs, wl.types, wl.instances)
+    t32 = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    flag = oracle.risk(t32, *wl.active.columns()).flag
+    _, cand, count = oracle.compact(flag)
+    cap = count // 3
+    risk, raw = gpu_risk(gs, pool, wl.active, capacity=cap)
+    assert risk.count == count                      # the true count is still reported
+    np.testing.assert_array_equal(raw[:cap], cand[:cap])
+    assert gs.device_status() & DeviceStatus.CAND_TRUNCATED
+    # and nothing is written past the capacity
+    dev = gs.device
+    cols = [torch.from_numpy(c).to(dev) for c in wl.active.columns()]
+    bits = torch.zeros((wl.active.n + 31) // 32, dtype=torch.int32, device=dev)
+    buf = torch.full((cap + 64,), -9, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+    gs.risk_scan(*cols, pool, bits, buf, cnt, cand_capacity=cap)
+    torch.cuda.synchronize()
+    assert (buf[cap:].cpu().numpy() == -9).all()
+    gs.device_status()
+
+
+def test_accumulate_and_advance_saturate(gs):
+    types, inst = W.make_pool(4, 2, seed=9)
+    inst.free_kv_tokens[:] = 2 ** 31 - 1
+    inst.queued_prefill_tokens[:] = 5
+    pool = pool_of(gs, types, inst)
+    n = 64
+    req = W.RequestBatch(np.full(n, 2 ** 30, np.int32), np.full(n, 100, np.int32), np.full(n, np.inf, np.float32))
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    got = gpu_route(gs, pool, req, 0.5, accumulate=True)
+    gs.advance_state(pool)
+    ref = oracle.route(t32, *req.columns())
+    np.testing.assert_array_equal(got.instance_idx, ref.instance_idx)
+    state = inst.copy()
+    oracle.advance(state, t32, ref.instance_idx, req.prompt_len, req.pred_decode_len)
+    assert state.queued_prefill_tokens.max() == 2 ** 31 - 1 and state.free_kv_tokens.min() == 0
+    np.testing.assert_array_equal(pool.queued_prefill_tokens.cpu().numpy(), state.queued_prefill_tokens)
+    np.testing.assert_array_equal(pool.decode_batch.cpu().numpy(), state.decode_batch)
+    np.testing.assert_array_equal(pool.free_kv_tokens.cpu().numpy(), state.free_kv_tokens)
+    # a second advance with nothing pending changes only nothing
+    gs.advance_state(pool)
+    np.testing.assert_array_equal(pool.decode_batch.cpu().numpy(), state.decode_batch)
+
+
+def test_route_without_accumulate_leaves_state_alone(gs):
+    wl = W.make_workload(1, n_requests=4096, n_active=16)
+    pool = pool_of(gs, wl.types, wl.instances)
+    gpu_route(gs, pool, wl.requests, 0.5)
+    gs.advance_state(pool)
+    np.testing.assert_array_equal(pool.queued_prefill_tokens.cpu().numpy(), wl.instances.queued_prefill_tokens)
+    np.testing.assert_array_equal(pool.decode_batch.cpu().numpy(), wl.instances.decode_batch)
+
+
+def test_host_entry_points_match_device_ones(gs):
+    wl = W.make_workload(1, n_requests=20_001, n_active=70_003)
+    pool = pool_of(gs, wl.types, wl.instances)
+    dev = gpu_route(gs, pool, wl.requests, 0.5)
+    n = wl.requests.n
+    idx = np.empty(n, np.int32); est = np.empty(n, np.float32); slack = np.empty(n, np.float32)
+    tier = np.empty(n, np.uint8)
+    gs.route_batch_host(*wl.requests.columns(), wl.types, wl.instances, 0.5, idx, est, slack, tier)
+    np.testing.assert_array_equal(idx, dev.instance_idx)
+    np.testing.assert_array_equal(est, dev.est_e2e_ms)
+    np.testing.assert_array_equal(slack, dev.slack_ms)
+    np.testing.assert_array_equal(tier, dev.tier)
+    risk, _ = gpu_risk(gs, pool, wl.active)
+    bits = np.empty((wl.active.n + 31) // 32, np.uint32)
+    cand = np.empty(wl.active.n, np.int32)
+    count = gs.risk_scan_host(*wl.active.columns(), wl.types, wl.instances, bits, cand)
+    assert count == risk.count
+    np.testing.assert_array_equal(bits, risk.flag_bits)
+    np.testing.assert_array_equal(cand[:count], risk.cand_idx)
+
+
+def test_error_codes(gs):
+    from paper_2605_16867_b200 import GoodServe, GoodServeError, InstancePool
+    types, inst = W.make_pool(16, 4, seed=1)
+    pool = pool_of(gs, types, inst)
+    dev = gs.device
+    n = 64
+    xi = torch.zeros(n + 4, dtype=torch.int32, device=dev)
+    xf = torch.zeros(n + 4, dtype=torch.float32, device=dev)
+    with pytest.raises(GoodServeError) as e:      # misaligned view
+        gs.route_batch(xi[1:n + 1], xi[:n], xf[:n], pool, 0.5, xi[:n].clone(), xf[:n].clone(), xf[:n].clone())
+    assert e.value.code == -4
+    small = GoodServe(0, max_instances=8, max_types=2)
+    with pytest.raises(GoodServeError) as e:      # pool larger than the context
+        small.route_batch(xi[:n], xi[:n], xf[:n], pool, 0.5, xi[:n].clone(), xf[:n].clone(), xf[:n].clone())
+    assert e.value.code == -2
+    small.close()
+    with pytest.raises(GoodServeError) as e:
+        GoodServe(0, max_instances=4096)
+    assert e.value.code == -2
+    with pytest.raises((TypeError, ValueError)):  # wrong dtype is caught by the binding
+        gs.route_batch(xf[:n], xi[:n], xf[:n], pool, 0.5, xi[:n].clone(), xf[:n].clone(), xf[:n].clone())
+    # the context is still usable
+    cfg = W.CONFIGS[0]
+    req = W.make_requests(cfg, types, seed=0, n=100)
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    assert_route_matches_f32_oracle(gpu_route(gs, pool, req, 0.5), oracle.route(t32, *req.columns()))
