@@ -58,7 +58,8 @@ enum gs_error {
     GS_ERR_CAPACITY = -2,       /* n_instances or n_types above what the context was created for */
     GS_ERR_CUDA = -3,           /* a CUDA runtime call failed; see gs_last_cuda_error */
     GS_ERR_ALIGN = -4,          /* an array pointer is not 16-byte aligned */
-    GS_ERR_NO_DEVICE = -5       /* no usable CUDA device */
+    GS_ERR_NO_DEVICE = -5,      /* no usable CUDA device */
+    GS_ERR_TOO_LARGE = -6       /* gs_risk_scan_noalloc: n_active above GS_NOALLOC_MAX_ACTIVE */
 };
 
 /* bits of the device status word */
@@ -220,6 +221,42 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx,
                       const gs_instances *inst, const gs_types *types,
                       uint32_t *out_flag_bits, int32_t *out_cand_idx, int64_t cand_capacity,
                       int64_t *out_cand_count, void *cuda_stream);
+
+/*
+ * Risk scan without any allocation.  (The paper has no counterpart: this entry point exists
+ * only because of how some callers must run, not because of the method.)
+ *
+ * Who needs it: code that may not call cudaMalloc / cudaFree or anything that might -- a
+ * serving process that handed all device memory to its KV-cache allocator at start-up, a
+ * plugin running inside someone else's memory pool, a latency-critical loop where an
+ * allocation's implicit device synchronisation is unacceptable.  Such callers cannot create
+ * a gs_ctx (gs_create allocates), so this call takes none: the scratch that gs_risk_scan
+ * keeps in its context (per-instance decode latencies, per-chunk flag counts) lives instead
+ * in a fixed array inside the library image, about 72 KB that every GPU loading the library
+ * holds until the process exits.  It computes exactly what gs_risk_scan computes, with the
+ * same kernels; inputs, outputs and their layout are the same and still belong to the caller.
+ *
+ *   - Runs on the CURRENT device (cudaGetDevice) and enqueues on `cuda_stream`, which must
+ *     belong to it.  No cudaMalloc, cudaFree or allocating library routine is called.
+ *   - n_active may not exceed GS_NOALLOC_MAX_ACTIVE (the array is sized for that); a larger
+ *     value returns GS_ERR_TOO_LARGE and enqueues nothing.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress).  Make that first call outside any stream capture.
+ *   - All calls on one GPU share the one array, and it keeps the previous call's contents;
+ *     the call rewrites every word it later reads, so results never depend on earlier calls.
+ *     But two calls that overlap on the GPU (different streams, or different host threads)
+ *     race on the array and give wrong results: serialise them.
+ *   - out_status_bits (device pointer to one word, may be NULL) is OR-ed with gs_dev_status
+ *     bits; the caller zeroes it beforehand.  With NULL the bits are dropped.
+ */
+#define GS_NOALLOC_MAX_ACTIVE 16777216
+
+GS_API int gs_risk_scan_noalloc(const int32_t *assigned_inst, const int32_t *generated_tokens,
+                                const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                                int64_t n_active,
+                                const gs_instances *inst, const gs_types *types,
+                                uint32_t *out_flag_bits, int32_t *out_cand_idx, int64_t cand_capacity,
+                                int64_t *out_cand_count, unsigned *out_status_bits, void *cuda_stream);
 
 #ifdef __cplusplus
 }

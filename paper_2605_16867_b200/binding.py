@@ -90,6 +90,9 @@ def load_library(build_if_missing: bool = True):
     lib.gs_risk_scan_host.argtypes = risk_args
     lib.gs_timing_enable.argtypes = [vp, C.c_int]
     lib.gs_timing_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(i64)]
+    lib.gs_risk_scan_noalloc.argtypes = [vp, vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types),
+                                         vp, vp, i64, vp, vp, vp]
+    lib.gs_risk_scan_noalloc.restype = C.c_int
     for name in ("gs_timing_enable", "gs_timing_read", "gs_create", "gs_destroy", "gs_last_cuda_error", "gs_device_status", "gs_route_batch",
                  "gs_route_batch_host", "gs_advance_state", "gs_risk_scan", "gs_risk_scan_host"):
         getattr(lib, name).restype = C.c_int
@@ -309,3 +312,50 @@ class GoodServe:
 
     def last_cuda_error(self) -> int:
         return int(self._lib.gs_last_cuda_error(self._h))
+
+
+NOALLOC_MAX_ACTIVE = 16_777_216
+
+
+def risk_scan_noalloc(assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, pool: InstancePool,
+                      out_flag_bits, out_cand_idx, out_cand_count, out_status_bits=None,
+                      cand_capacity: Optional[int] = None, n_active: Optional[int] = None, stream=None):
+    """gs_risk_scan_noalloc: the risk scan for callers that must not allocate device memory.
+
+    Needs no GoodServe context (creating one allocates).  The scan's scratch is a fixed array
+    inside the library, shared by every call on the same GPU, so calls on one GPU must not
+    overlap; at most NOALLOC_MAX_ACTIVE requests per call.  Runs on the tensors' device, which
+    must be the current CUDA device.  This wrapper allocates nothing either: every tensor,
+    including the optional one-word ``out_status_bits`` (int32, zeroed by the caller), is the
+    caller's.
+    """
+    lib = load_library()
+    n = int(assigned_inst.numel()) if n_active is None else int(n_active)
+    cap = (0 if out_cand_idx is None else int(out_cand_idx.numel())) if cand_capacity is None else int(cand_capacity)
+    dev = assigned_inst.device
+    if torch.cuda.current_device() != dev.index:
+        raise ValueError("risk_scan_noalloc runs on the current device; make the tensors' device current")
+    i32, f32 = torch.int32, torch.float32
+    M, Tn = pool.n_instances, pool.n_types
+    inst = _Instances(_dev_ptr(pool.type_id, i32, M, "type_id", dev),
+                      _dev_ptr(pool.queued_prefill_tokens, i32, M, "queued_prefill_tokens", dev),
+                      _dev_ptr(pool.decode_batch, i32, M, "decode_batch", dev),
+                      _dev_ptr(pool.free_kv_tokens, i32, M, "free_kv_tokens", dev),
+                      _dev_ptr(pool.q_ema_ms, f32, M, "q_ema_ms", dev), M)
+    types = _Types(_dev_ptr(pool.prefill_ms_per_tok, f32, Tn, "prefill_ms_per_tok", dev),
+                   _dev_ptr(pool.tpot_a_ms, f32, Tn, "tpot_a_ms", dev),
+                   _dev_ptr(pool.tpot_b_ms, f32, Tn, "tpot_b_ms", dev), Tn)
+    s = torch.cuda.current_stream(dev) if stream is None else stream
+    rc = lib.gs_risk_scan_noalloc(
+        _dev_ptr(assigned_inst, i32, n, "assigned_inst", dev),
+        _dev_ptr(generated_tokens, i32, n, "generated_tokens", dev),
+        _dev_ptr(pred_len, i32, n, "pred_len", dev),
+        _dev_ptr(elapsed_ms, f32, n, "elapsed_ms", dev),
+        _dev_ptr(slo_ms, f32, n, "slo_ms", dev), n,
+        C.byref(inst), C.byref(types),
+        _dev_ptr(out_flag_bits, i32, (n + 31) // 32, "out_flag_bits", dev),
+        _dev_ptr(out_cand_idx, i32, cap, "out_cand_idx", dev), cap,
+        _dev_ptr(out_cand_count, torch.int64, 1, "out_cand_count", dev),
+        _dev_ptr(out_status_bits, i32, 1, "out_status_bits", dev), s.cuda_stream or None)
+    if rc != 0:
+        raise GoodServeError(rc, lib.gs_strerror(rc).decode())

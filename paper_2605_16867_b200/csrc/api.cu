@@ -121,6 +121,7 @@ GS_API const char *gs_strerror(int code) {
         case GS_ERR_CUDA: return "a CUDA runtime call failed (see gs_last_cuda_error)";
         case GS_ERR_ALIGN: return "array pointer is not 16-byte aligned";
         case GS_ERR_NO_DEVICE: return "no usable CUDA device";
+        case GS_ERR_TOO_LARGE: return "n_active exceeds GS_NOALLOC_MAX_ACTIVE, the fixed scratch of the no-allocation scan";
         default: return "unknown error code";
     }
 }

@@ -7,6 +7,8 @@
 // Pass 2 (scan_counts_kernel) turns the per-chunk counts into exclusive offsets and the total.
 // Pass 3 (scatter_candidates_kernel) re-reads only the flag words and writes the ascending
 // candidate list; positions inside a word come from popc of the lower lanes' bits.
+#include <mutex>
+
 #include "gs_internal.cuh"
 
 namespace gs {
@@ -198,4 +200,114 @@ cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *gen
     return cudaSuccess;
 }
 
+// ---------------------------------------------------------------------------------------
+// gs_risk_scan_noalloc: the same scan for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------------
+
+constexpr int64_t kNoAllocChunks = (GS_NOALLOC_MAX_ACTIVE + kRiskChunk - 1) / kRiskChunk;
+
+// All scratch of the no-allocation entry point.  It lives in the library image: every GPU
+// that loads the library holds these ~72 KB until the process exits.
+struct NoAllocScratch {
+    float d_by_g[GS_MAX_INSTANCES];
+    unsigned chunk_counts[kNoAllocChunks + 1];
+    unsigned status;
+};
+static __device__ __align__(256) NoAllocScratch g_noalloc_scratch;
+
+// Per-instance decode latency d_g = a_t + b_t * batch_g for the scan (the only coefficient
+// of Eq. 2 that the risk test of Sec. 3.4 uses), with the same clamping rules as elsewhere.
+__global__ void __launch_bounds__(GS_MAX_INSTANCES)
+decode_latency_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__ batch, int M,
+                      const float *__restrict__ a_type, const float *__restrict__ b_type, int n_types,
+                      float *__restrict__ d_by_g, unsigned *__restrict__ status)
+{
+    const int g = threadIdx.x;
+    if (g >= M) return;
+    unsigned bad = 0;
+    int t = type_id[g];
+    if (t < 0 || t >= n_types) { bad |= GS_DEV_BAD_TYPE; t = 0; }
+    int B = batch[g];
+    if (B < 0) { bad |= GS_DEV_BAD_VALUE; B = 0; }
+    d_by_g[g] = __fmaf_rn(b_type[t], __int2float_rn(B), a_type[t]);
+    if (bad) atomicOr(status, bad);
+}
+
 }  // namespace gs
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+// Device address of g_noalloc_scratch on each GPU, resolved on that GPU's first call.
+// In host code the symbol's name is only a handle, never an address a kernel may use.
+gs::NoAllocScratch *g_noalloc_ptr[kMaxDevices] = {};
+cudaError_t g_noalloc_err[kMaxDevices] = {};
+bool g_noalloc_ready[kMaxDevices] = {};
+std::mutex g_noalloc_mutex;     // guards the three tables above
+
+}  // namespace
+
+extern "C" GS_API int gs_risk_scan_noalloc(
+    const int32_t *assigned_inst, const int32_t *generated_tokens, const int32_t *pred_len,
+    const float *elapsed_ms, const float *slo_ms, int64_t n_active,
+    const gs_instances *inst, const gs_types *types,
+    uint32_t *out_flag_bits, int32_t *out_cand_idx, int64_t cand_capacity,
+    int64_t *out_cand_count, unsigned *out_status_bits, void *cuda_stream)
+{
+    using namespace gs;
+    if (!inst || !types || !out_cand_count || n_active < 0 || cand_capacity < 0) return GS_ERR_INVALID_ARG;
+    if (n_active > GS_NOALLOC_MAX_ACTIVE) return GS_ERR_TOO_LARGE;
+    if (inst->n_instances < 1 || types->n_types < 1) return GS_ERR_INVALID_ARG;
+    if (inst->n_instances > GS_MAX_INSTANCES || types->n_types > GS_MAX_TYPES) return GS_ERR_CAPACITY;
+    if (!inst->type_id || !inst->decode_batch || !types->tpot_a_ms || !types->tpot_b_ms) return GS_ERR_INVALID_ARG;
+    if (cand_capacity > 0 && !out_cand_idx) return GS_ERR_INVALID_ARG;
+    if (n_active > 0 && (!assigned_inst || !generated_tokens || !pred_len || !elapsed_ms || !slo_ms || !out_flag_bits))
+        return GS_ERR_INVALID_ARG;
+    const void *aligned16[] = {assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, out_flag_bits, out_cand_idx};
+    for (const void *p : aligned16) if (reinterpret_cast<uintptr_t>(p) & 15u) return GS_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(out_cand_count) & 7u) return GS_ERR_ALIGN;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GS_ERR_NO_DEVICE;
+    NoAllocScratch *sc = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_ready[dev]) {
+            // first call on this GPU (it is the current device): resolve the scratch's address here
+            void *p = nullptr;
+            g_noalloc_err[dev] = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+            g_noalloc_ptr[dev] = static_cast<NoAllocScratch *>(p);
+            g_noalloc_ready[dev] = true;
+        }
+        if (g_noalloc_err[dev] != cudaSuccess || !g_noalloc_ptr[dev]) return GS_ERR_CUDA;
+        sc = g_noalloc_ptr[dev];
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    unsigned *status = out_status_bits ? out_status_bits : &sc->status;
+    const int M = inst->n_instances;
+
+    decode_latency_kernel<<<1, GS_MAX_INSTANCES, 0, st>>>(inst->type_id, inst->decode_batch, M, types->tpot_a_ms,
+                                                        types->tpot_b_ms, types->n_types, sc->d_by_g, status);
+    if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
+    const int64_t n_chunks = (n_active + kRiskChunk - 1) / kRiskChunk;
+    const int64_t n_words = (n_active + 31) >> 5;
+    int n_sm = 0;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1) n_sm = 148;
+    int64_t blocks = (n_chunks + kRiskWarps - 1) / kRiskWarps;
+    if (blocks > (int64_t)n_sm * 8) blocks = (int64_t)n_sm * 8;
+    if (n_chunks > 0) {
+        // every count in [0, n_chunks) is rewritten by this pass, so stale contents do not matter
+        risk_flags_kernel<<<(unsigned)blocks, kRiskThreads, 0, st>>>(
+            assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, n_active, M, sc->d_by_g,
+            out_flag_bits, sc->chunk_counts, n_chunks, status);
+        if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
+    }
+    scan_counts_kernel<<<1, 1024, 0, st>>>(sc->chunk_counts, n_chunks, out_cand_count, cand_capacity, status);
+    if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
+    if (n_chunks > 0 && cand_capacity > 0) {
+        scatter_candidates_kernel<<<(unsigned)blocks, kRiskThreads, 0, st>>>(
+            out_flag_bits, n_words, sc->chunk_counts, n_chunks, out_cand_idx, cand_capacity);
+        if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
+    }
+    return GS_OK;
+}
