@@ -11,20 +11,26 @@
 
 namespace gs {
 
-// One row of the per-round instance table, in preference order (d descending, index
-// ascending): the coefficients of Eq. 2 plus the free KV tokens as raw int bits.
-struct __align__(16) InstRow {
+// One node of the per-round search structure.  A leaf is one instance: the coefficients of
+// Eq. 2 and its free KV tokens.  An inner node is a lower bound over the leaves below it
+// (min q, p, min d, all slightly shrunk; max kv).  Nodes are stored in depth-first order.
+// The parallel `meta` word is (instance index << 16) | target, instance index 0xFFFF marking
+// an inner node; target is where the walk continues when an inner node's bound fails, or,
+// for a leaf, the end of its type's subtree.
+struct __align__(16) Node {
     float q, p, d;
     int kv;
 };
+constexpr int kMaxNodes = 1536;         // >= 1024 leaves + all inner nodes for any type mix
 
 constexpr int kRiskChunk = 1024;        // requests per warp-chunk of the risk scan (32 flag words)
 constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 
 // Device scratch owned by a context.
 struct Scratch {
-    InstRow *rows;            // [max_instances] sorted by preference
-    int *row_g;               // [max_instances] original instance index of each row
+    Node *nodes;              // [kMaxNodes] search structure of the current round
+    unsigned *meta;           // [kMaxNodes]
+    int *table_info;          // {n_nodes, unsafe, n_instances, n_active_types}
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
     float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out
@@ -39,6 +45,7 @@ struct gs_ctx {
     int max_instances;
     int max_types;
     int n_sm;
+    int route_ctas_per_sm;
     gs::Scratch s;
     size_t chunk_cap;
     int64_t launches;
@@ -71,6 +78,7 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
                          const float *slo_ms, int64_t n, int n_instances,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, cudaStream_t st);
+cudaError_t configure_route(gs_ctx *ctx);
 cudaError_t launch_advance(gs_ctx *ctx, const gs_instances_mut &inst, cudaStream_t st);
 cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *generated,
                         const int32_t *pred_len, const float *elapsed, const float *slo,

@@ -1,20 +1,37 @@
 // gs_route_batch kernels: pair scoring (Eq. 2), feasibility, just-enough pick and fallback
 // (Algorithm 1) for every pending request of a round.
 //
-// One thread owns one request.  The per-round instance table (rows in preference order:
-// d descending, index ascending) is staged once per CTA in shared memory; every lane of a
-// warp walks the same rows, so each shared-memory read is a broadcast.  Because the
-// preference order does not depend on the request, argmax d_g over the feasible set is the
-// FIRST feasible row, and a lane stops scanning as soon as it has found one.
+// One thread owns four consecutive requests (128-bit column loads and stores).  The per-round
+// search structure built by the prologue is staged once per CTA in shared memory.  For each
+// request the thread walks it depth-first: an inner node whose lower bound already misses the
+// deadline (or whose largest free KV is too small) is skipped with everything below it; a
+// leaf is one instance, scored exactly as the definition says.  Within a type the leaves are
+// in preference order (d descending, index ascending), so the first feasible leaf of a type is
+// that type's best, and later types are left as soon as their leaves fall below the best d
+// found so far.  The walk therefore returns exactly argmax d_g over the feasible set.
+//
+// A request for which the walk finds nothing (no feasible instance: the fallback of
+// Algorithm 1) is queued in shared memory and finished by a whole warp that scores every
+// instance, lanes across instances, with shuffle reductions for the argmin.
 #include "gs_internal.cuh"
 
 namespace gs {
 
 constexpr int kRouteThreads = 256;
+constexpr int kReqPerThread = 4;
+constexpr int kRouteTile = kRouteThreads * kReqPerThread;
 
 // T(r,g) of Eq. 2 with H = 0, each step rounded once.
-__device__ __forceinline__ float latency(const InstRow &r, float x, float y) {
+__device__ __forceinline__ float latency(const Node &r, float x, float y) {
     return __fmaf_rn(r.d, y, __fmaf_rn(r.p, x, r.q));
+}
+
+__device__ __forceinline__ unsigned orderable_bits(float f) {
+    const unsigned b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float from_orderable_bits(unsigned o) {
+    return __uint_as_float((o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o);
 }
 
 // Adds one routed request to the CTA's pending-delta histogram.  Lanes of the warp that
@@ -36,69 +53,181 @@ __device__ __forceinline__ void accumulate_choice(unsigned long long *hist, int 
     }
 }
 
+// Depth-first walk for one request.  Returns the chosen instance or -1 (no feasible one).
+__device__ __forceinline__ int walk(const Node *__restrict__ nodes, const unsigned *__restrict__ meta,
+                                    int n_nodes, float x, float y, float D, unsigned need, float &T_out)
+{
+    int i = 0, g_best = -1;
+    float d_best = -1.0f, T_best = 0.f;
+    while (i < n_nodes) {
+        const Node nd = nodes[i];
+        const unsigned m = meta[i];
+        const float T = latency(nd, x, y);
+        const bool pass = (T <= D) && (need <= (unsigned)nd.kv);
+        const int inst = (int)(m >> 16);
+        const bool leaf = inst != 0xFFFF;
+        const bool worse = nd.d < d_best;
+        if (leaf && pass && !worse && (nd.d > d_best || inst < g_best || g_best < 0)) {
+            d_best = nd.d; g_best = inst; T_best = T;
+        }
+        const bool jump = leaf ? (pass || worse) : !pass;
+        i = jump ? (int)(m & 0xFFFFu) : i + 1;
+    }
+    T_out = T_best;
+    return g_best;
+}
+
 template <bool kAccumulate>
 __global__ void __launch_bounds__(kRouteThreads)
-route_scan_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
-                  const float *__restrict__ slo_ms, int64_t n, int M,
-                  const InstRow *__restrict__ rows, const int *__restrict__ row_g,
-                  int32_t *__restrict__ out_idx, float *__restrict__ out_est,
-                  float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
-                  unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
+route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
+             const float *__restrict__ slo_ms, int64_t n,
+             const Node *__restrict__ g_nodes, const unsigned *__restrict__ g_meta,
+             const int *__restrict__ table_info,
+             int32_t *__restrict__ out_idx, float *__restrict__ out_est,
+             float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
+             unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    InstRow *sh_rows = reinterpret_cast<InstRow *>(smem);
-    int *sh_g = reinterpret_cast<int *>(sh_rows + M);
+    const int n_nodes = table_info[0];
+    const bool unsafe = table_info[1] != 0;
+    const int M = table_info[2];
+    Node *sh_nodes = reinterpret_cast<Node *>(smem);
+    unsigned *sh_meta = reinterpret_cast<unsigned *>(sh_nodes + n_nodes);
+    int *sh_queue = reinterpret_cast<int *>(sh_meta + n_nodes);
+    int *sh_qcount = sh_queue + kRouteTile;
     unsigned long long *hist = reinterpret_cast<unsigned long long *>(
-        smem + (((size_t)M * (sizeof(InstRow) + sizeof(int)) + 15) & ~(size_t)15));
+        smem + (((size_t)n_nodes * (sizeof(Node) + sizeof(unsigned)) + (kRouteTile + 4) * sizeof(int) + 15) & ~(size_t)15));
 
-    for (int k = threadIdx.x; k < M; k += blockDim.x) {
-        sh_rows[k] = rows[k];
-        sh_g[k] = row_g[k];
+    for (int k = threadIdx.x; k < n_nodes; k += blockDim.x) {
+        sh_nodes[k] = g_nodes[k];
+        sh_meta[k] = g_meta[k];
     }
+    if (threadIdx.x == 0) *sh_qcount = 0;
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
     __syncthreads();
 
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int walk_nodes = unsafe ? 0 : n_nodes;
     unsigned bad = 0;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const int lane = threadIdx.x & 31;
-    // `base` is the warp's first request, so the trip count is uniform across the warp
-    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31); base < n; base += stride) {
-        const int64_t i = base + lane;
-        const bool valid = i < n;
-        int xi = valid ? prompt_len[i] : 0, yi = valid ? pred_decode_len[i] : 0;
-        if (xi < 0) { xi = 0; bad |= GS_DEV_BAD_VALUE; }
-        if (yi < 0) { yi = 0; bad |= GS_DEV_BAD_VALUE; }
-        const float D = valid ? slo_ms[i] : 0.f;
-        const float x = __int2float_rn(xi), y = __int2float_rn(yi);
-        const unsigned need = (unsigned)xi + (unsigned)yi;    // < 2^32, no overflow
+    const int64_t n_tiles = (n + kRouteTile - 1) / kRouteTile;
+    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const int64_t first = tile * kRouteTile + (int64_t)threadIdx.x * kReqPerThread;
+        int xi[kReqPerThread], yi[kReqPerThread];
+        float D[kReqPerThread];
+        if (first + kReqPerThread <= n) {
+            const int4 xv = __ldcs(reinterpret_cast<const int4 *>(prompt_len + first));
+            const int4 yv = __ldcs(reinterpret_cast<const int4 *>(pred_decode_len + first));
+            const float4 dv = __ldcs(reinterpret_cast<const float4 *>(slo_ms + first));
+            xi[0] = xv.x; xi[1] = xv.y; xi[2] = xv.z; xi[3] = xv.w;
+            yi[0] = yv.x; yi[1] = yv.y; yi[2] = yv.z; yi[3] = yv.w;
+            D[0] = dv.x; D[1] = dv.y; D[2] = dv.z; D[3] = dv.w;
+        } else {
+#pragma unroll
+            for (int j = 0; j < kReqPerThread; ++j) {
+                const bool v = first + j < n;
+                xi[j] = v ? prompt_len[first + j] : 0;
+                yi[j] = v ? pred_decode_len[first + j] : 0;
+                D[j] = v ? slo_ms[first + j] : 0.f;
+            }
+        }
+        int g_out[kReqPerThread];
+        float T_out[kReqPerThread];
+#pragma unroll
+        for (int j = 0; j < kReqPerThread; ++j) {
+            if (xi[j] < 0) { xi[j] = 0; bad |= GS_DEV_BAD_VALUE; }
+            if (yi[j] < 0) { yi[j] = 0; bad |= GS_DEV_BAD_VALUE; }
+            const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];      // < 2^32, no overflow
+            const bool valid = first + j < n;
+            g_out[j] = walk(sh_nodes, sh_meta, valid ? walk_nodes : 0, __int2float_rn(xi[j]),
+                            __int2float_rn(yi[j]), D[j], need, T_out[j]);
+            if (valid && g_out[j] < 0) sh_queue[atomicAdd(sh_qcount, 1)] = threadIdx.x * kReqPerThread + j;
+            if (kAccumulate) accumulate_choice(hist, M, valid ? g_out[j] : -1, (unsigned)xi[j], need);
+        }
+        if (first + kReqPerThread <= n) {
+            __stcs(reinterpret_cast<int4 *>(out_idx + first), make_int4(g_out[0], g_out[1], g_out[2], g_out[3]));
+            __stcs(reinterpret_cast<float4 *>(out_est + first), make_float4(T_out[0], T_out[1], T_out[2], T_out[3]));
+            __stcs(reinterpret_cast<float4 *>(out_slack + first),
+                   make_float4(__fsub_rn(D[0], T_out[0]), __fsub_rn(D[1], T_out[1]),
+                               __fsub_rn(D[2], T_out[2]), __fsub_rn(D[3], T_out[3])));
+            if (out_tier) *reinterpret_cast<uchar4 *>(out_tier + first) = make_uchar4(1, 1, 1, 1);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kReqPerThread; ++j)
+                if (first + j < n) {
+                    out_idx[first + j] = g_out[j];
+                    out_est[first + j] = T_out[j];
+                    out_slack[first + j] = __fsub_rn(D[j], T_out[j]);
+                    if (out_tier) out_tier[first + j] = 1;
+                }
+        }
+        __syncthreads();
 
-        int pick = -1;                         // row of the just-enough pick
-        float T_pick = 0.f;
-        int row_k = -1, row_a = -1;            // fallback rows: min T among KV-ok / among all
-        int g_k = 0, g_a = 0;
-        float T_k = 0.f, T_a = 0.f;
-        for (int k = 0; k < M; ++k) {
-            const InstRow r = sh_rows[k];
-            const float T = latency(r, x, y);
-            const bool kv_ok = need <= (unsigned)r.kv;
-            if (kv_ok && T <= D) { pick = k; T_pick = T; break; }
-            const int g = sh_g[k];
-            if (kv_ok && (row_k < 0 || T < T_k || (T == T_k && g < g_k))) { row_k = k; T_k = T; g_k = g; }
-            if (row_a < 0 || T < T_a || (T == T_a && g < g_a)) { row_a = k; T_a = T; g_a = g; }
+        // ---- requests with no feasible instance: one warp each, lanes across instances ----
+        const int n_queued = *sh_qcount;
+        for (int e = warp; e < n_queued; e += kRouteThreads / 32) {
+            const int64_t r = tile * kRouteTile + sh_queue[e];
+            int xr = prompt_len[r], yr = pred_decode_len[r];
+            if (xr < 0) xr = 0;
+            if (yr < 0) yr = 0;
+            const float Dr = slo_ms[r];
+            const float x = __int2float_rn(xr), y = __int2float_rn(yr);
+            const unsigned need = (unsigned)xr + (unsigned)yr;
+            unsigned long long k_feas = 0ull;                    // max over feasible: (d, smallest index)
+            unsigned long long k_room = ~0ull, k_all = ~0ull;    // min over KV-ok / all: (T, index)
+            float T_feas = 0.f;
+            for (int k = lane; k < n_nodes; k += 32) {
+                const unsigned m = sh_meta[k];
+                const unsigned inst = m >> 16;
+                if (inst == 0xFFFFu) continue;
+                const Node nd = sh_nodes[k];
+                const float T = latency(nd, x, y);
+                const bool room = need <= (unsigned)nd.kv;
+                const unsigned long long kt = ((unsigned long long)orderable_bits(T) << 32) | inst;
+                if (kt < k_all) k_all = kt;
+                if (room && kt < k_room) k_room = kt;
+                if (room && T <= Dr) {
+                    const unsigned long long kd = ((unsigned long long)orderable_bits(nd.d) << 32) | (0xFFFFu - inst);
+                    if (kd > k_feas) { k_feas = kd; T_feas = T; }
+                }
+            }
+            unsigned long long w_feas = k_feas, w_room = k_room, w_all = k_all;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const unsigned long long a = __shfl_xor_sync(0xFFFFFFFFu, w_feas, off);
+                const unsigned long long b = __shfl_xor_sync(0xFFFFFFFFu, w_room, off);
+                const unsigned long long c = __shfl_xor_sync(0xFFFFFFFFu, w_all, off);
+                if (a > w_feas) w_feas = a;
+                if (b < w_room) w_room = b;
+                if (c < w_all) w_all = c;
+            }
+            int g; float T; uint8_t tier;
+            if (w_feas != 0ull) {
+                const unsigned owner = __ballot_sync(0xFFFFFFFFu, k_feas == w_feas);
+                T = __shfl_sync(0xFFFFFFFFu, T_feas, __ffs(owner) - 1);
+                g = (int)(0xFFFFu - (unsigned)(w_feas & 0xFFFFu)); tier = 1;
+            } else if (w_room != ~0ull) {
+                g = (int)(w_room & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_room >> 32)); tier = 2;
+            } else {
+                g = (int)(w_all & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_all >> 32)); tier = 3;
+            }
+            if (lane == 0) {
+                out_idx[r] = g;
+                out_est[r] = T;
+                out_slack[r] = __fsub_rn(Dr, T);
+                if (out_tier) out_tier[r] = tier;
+                if (kAccumulate) {
+                    atomicAdd(&hist[g], (unsigned long long)(unsigned)xr);
+                    atomicAdd(&hist[M + g], 1ull);
+                    atomicAdd(&hist[2 * M + g], (unsigned long long)need);
+                }
+            }
         }
-        int row; float T; uint8_t tier;
-        if (pick >= 0)       { row = pick;  T = T_pick; tier = 1; }
-        else if (row_k >= 0) { row = row_k; T = T_k;    tier = 2; }
-        else                 { row = row_a; T = T_a;    tier = 3; }
-        const int g = sh_g[row];
-        if (valid) {
-            out_idx[i] = g;
-            out_est[i] = T;
-            out_slack[i] = __fsub_rn(D, T);
-            if (out_tier) out_tier[i] = tier;
-        }
-        if (kAccumulate) accumulate_choice(hist, M, valid ? g : -1, (unsigned)xi, need);
+        __syncthreads();
+        if (threadIdx.x == 0) *sh_qcount = 0;
+        // the next tile's first queue write happens after its walks; the barrier at the end of
+        // that tile's phase orders it after this reset only if we also fence here
+        __syncthreads();
     }
     if (bad) atomicOr(status, bad);
 
@@ -117,21 +246,35 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
                          bool accumulate, cudaStream_t st)
 {
     if (n == 0) return cudaSuccess;
-    size_t smem = (((size_t)M * (sizeof(InstRow) + sizeof(int)) + 15) & ~(size_t)15);
-    if (accumulate) smem += (size_t)3 * M * sizeof(unsigned long long);
-    int64_t blocks = (n + kRouteThreads - 1) / kRouteThreads;
-    const int64_t cap = (int64_t)ctx->n_sm * 8;
+    size_t smem = (((size_t)kMaxNodes * (sizeof(Node) + sizeof(unsigned)) + (kRouteTile + 4) * sizeof(int) + 15) & ~(size_t)15);
+    if (accumulate) smem += (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
+    const int64_t n_tiles = (n + kRouteTile - 1) / kRouteTile;
+    int64_t blocks = n_tiles;
+    const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm;
     if (blocks > cap) blocks = cap;
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     if (accumulate)
-        route_scan_kernel<true><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, M, ctx->s.rows, ctx->s.row_g,
+        route_kernel<true><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
+            prompt_len, pred_decode_len, slo_ms, n, ctx->s.nodes, ctx->s.meta, ctx->s.table_info,
             out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     else
-        route_scan_kernel<false><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, M, ctx->s.rows, ctx->s.row_g,
+        route_kernel<false><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
+            prompt_len, pred_decode_len, slo_ms, n, ctx->s.nodes, ctx->s.meta, ctx->s.table_info,
             out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     return cudaGetLastError();
+}
+
+// Raises the dynamic shared-memory limit of the route kernels (called once per context).
+cudaError_t configure_route(gs_ctx *ctx)
+{
+    const int max_smem = (int)((((size_t)kMaxNodes * (sizeof(Node) + sizeof(unsigned)) + (kRouteTile + 4) * sizeof(int) + 15) & ~(size_t)15) +
+                               (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long));
+    cudaError_t e = cudaFuncSetAttribute(route_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(route_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e != cudaSuccess) return e;
+    ctx->route_ctas_per_sm = 4;
+    return cudaSuccess;
 }
 
 // ---------------------------------------------------------------------------------------
