@@ -238,13 +238,15 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
+    # clocks are sampled from before the warm-up until a few samples under load exist: the
+    # timed region itself lasts only milliseconds, less than one nvidia-smi sampling period
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
 
     # ---- device-resident timed region: exactly K steps ------------------------------
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     gs.timing_enable(True)
     launches0 = gs.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -262,6 +264,10 @@ def run_gpu(args):
         if n:
             kernel_ms[name] = (ms, n)
     gs.timing_enable(False)
+    t_wait = time.perf_counter()
+    while len(sampler.rows) < 4 and time.perf_counter() - t_wait < 3.0:
+        step()                                   # keep the same load up for the sampler (untimed)
+        torch.cuda.synchronize(dev)
     clocks = sampler.stop()
     flagged = int(count.item())
     status = gs.device_status()
@@ -285,15 +291,19 @@ def run_gpu(args):
         return gs.risk_scan_host(*h_act, wl.types, wl.instances, h_bits, h_cand, stream=stream)
 
     e2e_steps = max(1, min(args.steps, 5))
-    e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    ev0.record(stream)
-    for _ in range(e2e_steps):
-        n_flag = e2e_step()
-    ev1.record(stream)
-    barrier()
-    e2e_ms = max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3)
+    n_flag = flagged
+    if args.no_e2e:
+        e2e_steps, e2e_ms = 0, float("nan")
+    else:
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        ev0.record(stream)
+        for _ in range(e2e_steps):
+            n_flag = e2e_step()
+        ev1.record(stream)
+        barrier()
+        e2e_ms = max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3)
     e2e_ms, e2e_pairs = aggregate_over_ranks(e2e_ms, float(e2e_steps) * N * M, dist)
     h2d = 3 * 4 * N + 5 * 4 * A + 2 * (5 * 4 * M + 3 * 4 * wl.types.n_types)
     d2h = 3 * 4 * N + 4 * ((A + 31) // 32) + 8 + 4 * n_flag
@@ -341,7 +351,8 @@ def run_gpu(args):
         "step_hbm_frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "flagged_fraction": flagged / A, "device_status": status,
         "roofline": roofline, "kernels": per_kernel,
-        "e2e": {"value": e2e_pairs / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": None if args.no_e2e else
+               {"value": e2e_pairs / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
         "gpu_launches": launches, "clocks": clocks,
     }
@@ -360,6 +371,7 @@ def main():
     ap.add_argument("--config", type=int, default=3, choices=sorted(W.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -11,25 +11,36 @@
 
 namespace gs {
 
-// One node of the per-round search structure.  A leaf is one instance: the coefficients of
-// Eq. 2 and its free KV tokens.  An inner node is a lower bound over the leaves below it
-// (min q, p, min d, all slightly shrunk; max kv).  Nodes are stored in depth-first order.
-// The parallel `meta` word is (instance index << 16) | target, instance index 0xFFFF marking
-// an inner node; target is where the walk continues when an inner node's bound fails, or,
-// for a leaf, the end of its type's subtree.
-struct __align__(16) Node {
+// Exact per-instance coefficients of Eq. 2 for the current round, in caller order.
+struct __align__(16) Row {
     float q, p, d;
     int kv;
 };
-constexpr int kMaxNodes = 1536;         // >= 1024 leaves + all inner nodes for any type mix
+
+// The per-round search structure (built by the prologue, walked by the route kernel) is an
+// array of 8-byte nodes in depth-first order, one subtree per GPU type.  Node words:
+//   x: lower bound of q over the rows below, low 11 bits = target node index (where the walk
+//      continues when this node's bound fails; for a leaf, the end of its type's subtree)
+//   y: lower bound of d over the rows below, low 11 bits = 0 for a block,
+//      kNodeLeafFlag | instance index for a leaf (one instance).
+constexpr unsigned kNodeTagMask = 0x7FFu;
+constexpr unsigned kNodeLeafFlag = 0x400u;
+constexpr int kMaxNodes = 1536;         // 1024 leaves + every block of 4/16/64/256 rows, any type mix
+
+// One GPU type's entry point: bound over all its rows, and its node range.
+struct __align__(16) TypeHeader {
+    float p_lo, q_lo, d_lo, d_max;
+    int begin, end, pad0, pad1;
+};
 
 constexpr int kRiskChunk = 1024;        // requests per warp-chunk of the risk scan (32 flag words)
 constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 
 // Device scratch owned by a context.
 struct Scratch {
-    Node *nodes;              // [kMaxNodes] search structure of the current round
-    unsigned *meta;           // [kMaxNodes]
+    Row *rows;                // [max_instances] exact coefficients, caller order
+    uint2 *nodes;             // [kMaxNodes] search structure of the current round
+    TypeHeader *headers;      // [GS_MAX_TYPES] in walk order (largest d first)
     int *table_info;          // {n_nodes, unsafe, n_instances, n_active_types}
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
     float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)

@@ -2,13 +2,18 @@
 // (Algorithm 1) for every pending request of a round.
 //
 // One thread owns four consecutive requests (128-bit column loads and stores).  The per-round
-// search structure built by the prologue is staged once per CTA in shared memory.  For each
-// request the thread walks it depth-first: an inner node whose lower bound already misses the
-// deadline (or whose largest free KV is too small) is skipped with everything below it; a
-// leaf is one instance, scored exactly as the definition says.  Within a type the leaves are
-// in preference order (d descending, index ascending), so the first feasible leaf of a type is
-// that type's best, and later types are left as soon as their leaves fall below the best d
-// found so far.  The walk therefore returns exactly argmax d_g over the feasible set.
+// tables built by the prologue are staged once per CTA in shared memory.  For each request:
+//   1. every GPU type is tested against a lower bound of T over all its instances (same
+//      shared-memory address for all lanes, so a broadcast); types that cannot meet the
+//      deadline are dropped;
+//   2. the surviving types' subtrees are walked depth-first: a block whose lower bound misses
+//      the deadline is skipped with everything below it; a row that passes the (slightly
+//      loose) bound test is scored exactly as the definition says, T = fma(d, y, fma(p, x, q)),
+//      and checked against the deadline and the instance's free KV.
+// Rows of a type are in preference order (d descending, index ascending), so the first
+// feasible row of a type is that type's best; a later type is left as soon as its rows fall
+// below the best d found so far.  The walk therefore returns exactly argmax d_g over the
+// feasible set, with ties to the smallest index.
 //
 // A request for which the walk finds nothing (no feasible instance: the fallback of
 // Algorithm 1) is queued in shared memory and finished by a whole warp that scores every
@@ -22,7 +27,7 @@ constexpr int kReqPerThread = 4;
 constexpr int kRouteTile = kRouteThreads * kReqPerThread;
 
 // T(r,g) of Eq. 2 with H = 0, each step rounded once.
-__device__ __forceinline__ float latency(const Node &r, float x, float y) {
+__device__ __forceinline__ float latency(const Row &r, float x, float y) {
     return __fmaf_rn(r.d, y, __fmaf_rn(r.p, x, r.q));
 }
 
@@ -53,25 +58,57 @@ __device__ __forceinline__ void accumulate_choice(unsigned long long *hist, int 
     }
 }
 
-// Depth-first walk for one request.  Returns the chosen instance or -1 (no feasible one).
-__device__ __forceinline__ int walk(const Node *__restrict__ nodes, const unsigned *__restrict__ meta,
-                                    int n_nodes, float x, float y, float D, unsigned need, float &T_out)
+// Shared-memory image of the round's tables.
+struct Tables {
+    const TypeHeader *headers;
+    const uint2 *nodes;
+    const Row *rows;
+    int n_types;
+};
+
+// Just-enough pick for one request.  Returns the chosen instance or -1 (no feasible one).
+__device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y, float D, unsigned need,
+                                             float &T_out)
 {
-    int i = 0, g_best = -1;
-    float d_best = -1.0f, T_best = 0.f;
-    while (i < n_nodes) {
-        const Node nd = nodes[i];
-        const unsigned m = meta[i];
-        const float T = latency(nd, x, y);
-        const bool pass = (T <= D) && (need <= (unsigned)nd.kv);
-        const int inst = (int)(m >> 16);
-        const bool leaf = inst != 0xFFFF;
-        const bool worse = nd.d < d_best;
-        if (leaf && pass && !worse && (nd.d > d_best || inst < g_best || g_best < 0)) {
-            d_best = nd.d; g_best = inst; T_best = T;
+    // 1. which types can hold a feasible instance at all
+    unsigned alive = 0;
+    for (int t = 0; t < tb.n_types; ++t) {
+        const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);   // p_lo, q_lo, d_lo, d_max
+        const float R = __fmaf_rn(-h.x, x, D);
+        if (__fmaf_rn(h.z, y, h.y) <= R + 1e-30f) alive |= 1u << t;
+    }
+    // 2. walk the surviving subtrees
+    int g_best = -1;
+    float d_best = -1.0f, T_best = 0.f, R = 0.f;
+    int i = 0, end = 0;
+    for (;;) {
+        if (i >= end) {                       // next surviving type, if any can still improve
+            if (alive == 0) break;
+            const int t = __ffs(alive) - 1;
+            alive &= alive - 1;
+            const TypeHeader h = tb.headers[t];
+            if (h.d_max < d_best) break;      // types are ordered by their largest d
+            i = h.begin; end = h.end;
+            R = __fmaf_rn(-h.p_lo, x, D) + 1e-30f;
         }
-        const bool jump = leaf ? (pass || worse) : !pass;
-        i = jump ? (int)(m & 0xFFFFu) : i + 1;
+        const uint2 nd = tb.nodes[i];
+        const unsigned target = nd.x & kNodeTagMask;
+        const bool pass = __fmaf_rn(__uint_as_float(nd.y), y, __uint_as_float(nd.x)) <= R;
+        const bool leaf = (nd.y & kNodeLeafFlag) != 0;
+        int next = (pass == leaf) ? (int)target : i + 1;     // block fails -> skip it; row passes -> see below
+        if (pass && leaf) {
+            const int inst = (int)(nd.y & (kNodeLeafFlag - 1));
+            const Row r = tb.rows[inst];
+            const float T = latency(r, x, y);
+            const bool feasible = (T <= D) && (need <= (unsigned)r.kv);
+            const bool worse = r.d < d_best;
+            if (feasible && !worse && (g_best < 0 || r.d > d_best || inst < g_best)) {
+                d_best = r.d; g_best = inst; T_best = T;
+            }
+            // feasible: the rest of this type ranks lower.  worse: so does everything after it.
+            next = (feasible || worse) ? (int)target : i + 1;
+        }
+        i = next;
     }
     T_out = T_best;
     return g_best;
@@ -81,8 +118,8 @@ template <bool kAccumulate>
 __global__ void __launch_bounds__(kRouteThreads)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
              const float *__restrict__ slo_ms, int64_t n,
-             const Node *__restrict__ g_nodes, const unsigned *__restrict__ g_meta,
-             const int *__restrict__ table_info,
+             const Row *__restrict__ g_rows, const uint2 *__restrict__ g_nodes,
+             const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
              int32_t *__restrict__ out_idx, float *__restrict__ out_est,
              float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
@@ -91,24 +128,27 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     const int n_nodes = table_info[0];
     const bool unsafe = table_info[1] != 0;
     const int M = table_info[2];
-    Node *sh_nodes = reinterpret_cast<Node *>(smem);
-    unsigned *sh_meta = reinterpret_cast<unsigned *>(sh_nodes + n_nodes);
-    int *sh_queue = reinterpret_cast<int *>(sh_meta + n_nodes);
+    const int n_act = table_info[3];
+    Row *sh_rows = reinterpret_cast<Row *>(smem);
+    TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
+    uint2 *sh_nodes = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
+    int *sh_queue = reinterpret_cast<int *>(sh_nodes + kMaxNodes);
     int *sh_qcount = sh_queue + kRouteTile;
-    unsigned long long *hist = reinterpret_cast<unsigned long long *>(
-        smem + (((size_t)n_nodes * (sizeof(Node) + sizeof(unsigned)) + (kRouteTile + 4) * sizeof(int) + 15) & ~(size_t)15));
+    unsigned long long *hist = reinterpret_cast<unsigned long long *>(sh_qcount + 4);
 
-    for (int k = threadIdx.x; k < n_nodes; k += blockDim.x) {
-        sh_nodes[k] = g_nodes[k];
-        sh_meta[k] = g_meta[k];
-    }
+    for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[k] = g_rows[k];
+    for (int k = threadIdx.x; k < n_nodes; k += blockDim.x) sh_nodes[k] = g_nodes[k];
+    if (threadIdx.x < n_act) sh_headers[threadIdx.x] = g_headers[threadIdx.x];
     if (threadIdx.x == 0) *sh_qcount = 0;
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
     __syncthreads();
 
+    Tables tb;
+    tb.headers = sh_headers; tb.nodes = sh_nodes; tb.rows = sh_rows;
+    tb.n_types = unsafe ? 0 : n_act;          // unusable bounds: every request takes the exhaustive path
+
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int walk_nodes = unsafe ? 0 : n_nodes;
     unsigned bad = 0;
     const int64_t n_tiles = (n + kRouteTile - 1) / kRouteTile;
     for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -128,7 +168,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 const bool v = first + j < n;
                 xi[j] = v ? prompt_len[first + j] : 0;
                 yi[j] = v ? pred_decode_len[first + j] : 0;
-                D[j] = v ? slo_ms[first + j] : 0.f;
+                D[j] = v ? slo_ms[first + j] : -1.0f;
             }
         }
         int g_out[kReqPerThread];
@@ -139,8 +179,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             if (yi[j] < 0) { yi[j] = 0; bad |= GS_DEV_BAD_VALUE; }
             const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];      // < 2^32, no overflow
             const bool valid = first + j < n;
-            g_out[j] = walk(sh_nodes, sh_meta, valid ? walk_nodes : 0, __int2float_rn(xi[j]),
-                            __int2float_rn(yi[j]), D[j], need, T_out[j]);
+            g_out[j] = pick_instance(tb, __int2float_rn(xi[j]), __int2float_rn(yi[j]), D[j], need, T_out[j]);
             if (valid && g_out[j] < 0) sh_queue[atomicAdd(sh_qcount, 1)] = threadIdx.x * kReqPerThread + j;
             if (kAccumulate) accumulate_choice(hist, M, valid ? g_out[j] : -1, (unsigned)xi[j], need);
         }
@@ -176,18 +215,16 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             unsigned long long k_feas = 0ull;                    // max over feasible: (d, smallest index)
             unsigned long long k_room = ~0ull, k_all = ~0ull;    // min over KV-ok / all: (T, index)
             float T_feas = 0.f;
-            for (int k = lane; k < n_nodes; k += 32) {
-                const unsigned m = sh_meta[k];
-                const unsigned inst = m >> 16;
-                if (inst == 0xFFFFu) continue;
-                const Node nd = sh_nodes[k];
-                const float T = latency(nd, x, y);
-                const bool room = need <= (unsigned)nd.kv;
-                const unsigned long long kt = ((unsigned long long)orderable_bits(T) << 32) | inst;
+            for (int inst = lane; inst < M; inst += 32) {
+                const Row row = sh_rows[inst];
+                const float T = latency(row, x, y);
+                const bool room = need <= (unsigned)row.kv;
+                const unsigned long long kt = ((unsigned long long)orderable_bits(T) << 32) | (unsigned)inst;
                 if (kt < k_all) k_all = kt;
                 if (room && kt < k_room) k_room = kt;
                 if (room && T <= Dr) {
-                    const unsigned long long kd = ((unsigned long long)orderable_bits(nd.d) << 32) | (0xFFFFu - inst);
+                    const unsigned long long kd =
+                        ((unsigned long long)orderable_bits(row.d) << 32) | (0xFFFFu - (unsigned)inst);
                     if (kd > k_feas) { k_feas = kd; T_feas = T; }
                 }
             }
@@ -225,8 +262,6 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         }
         __syncthreads();
         if (threadIdx.x == 0) *sh_qcount = 0;
-        // the next tile's first queue write happens after its walks; the barrier at the end of
-        // that tile's phase orders it after this reset only if we also fence here
         __syncthreads();
     }
     if (bad) atomicOr(status, bad);
@@ -240,14 +275,18 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     }
 }
 
+constexpr size_t kRouteSmemBase = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
+                                  (size_t)kMaxNodes * sizeof(uint2) + (kRouteTile + 4) * sizeof(int);
+constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
+
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                          const float *slo_ms, int64_t n, int M,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, cudaStream_t st)
 {
+    (void)M;
     if (n == 0) return cudaSuccess;
-    size_t smem = (((size_t)kMaxNodes * (sizeof(Node) + sizeof(unsigned)) + (kRouteTile + 4) * sizeof(int) + 15) & ~(size_t)15);
-    if (accumulate) smem += (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
+    const size_t smem = kRouteSmemBase + (accumulate ? kRouteSmemHist : 0);
     const int64_t n_tiles = (n + kRouteTile - 1) / kRouteTile;
     int64_t blocks = n_tiles;
     const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm;
@@ -255,25 +294,27 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     if (accumulate)
         route_kernel<true><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, ctx->s.nodes, ctx->s.meta, ctx->s.table_info,
-            out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
+            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.nodes, ctx->s.headers,
+            ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     else
         route_kernel<false><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, ctx->s.nodes, ctx->s.meta, ctx->s.table_info,
-            out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
+            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.nodes, ctx->s.headers,
+            ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     return cudaGetLastError();
 }
 
 // Raises the dynamic shared-memory limit of the route kernels (called once per context).
 cudaError_t configure_route(gs_ctx *ctx)
 {
-    const int max_smem = (int)((((size_t)kMaxNodes * (sizeof(Node) + sizeof(unsigned)) + (kRouteTile + 4) * sizeof(int) + 15) & ~(size_t)15) +
-                               (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long));
-    cudaError_t e = cudaFuncSetAttribute(route_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    cudaError_t e = cudaFuncSetAttribute(route_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(kRouteSmemBase + kRouteSmemHist));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    e = cudaFuncSetAttribute(route_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRouteSmemBase);
     if (e != cudaSuccess) return e;
-    ctx->route_ctas_per_sm = 4;
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false>, kRouteThreads, kRouteSmemBase);
+    if (e != cudaSuccess) return e;
+    ctx->route_ctas_per_sm = occ > 0 ? occ : 1;
     return cudaSuccess;
 }
 
