@@ -17,20 +17,25 @@ struct __align__(16) Row {
     int kv;
 };
 
-// The per-round search structure (built by the prologue, walked by the route kernel) is an
-// array of 8-byte nodes in depth-first order, one subtree per GPU type.  Node words:
-//   x: lower bound of q over the rows below, low 11 bits = target node index (where the walk
-//      continues when this node's bound fails; for a leaf, the end of its type's subtree)
-//   y: lower bound of d over the rows below, low 11 bits = 0 for a block,
-//      kNodeLeafFlag | instance index for a leaf (one instance).
-constexpr unsigned kNodeTagMask = 0x7FFu;
-constexpr unsigned kNodeLeafFlag = 0x400u;
-constexpr int kMaxNodes = 1536;         // 1024 leaves + every block of 4/16/64/256 rows, any type mix
+// Per-round search tables (built by the prologue, read by the route kernel).  Rows are
+// grouped by GPU type and, inside a type, kept in preference order (d descending, index
+// ascending); each type's rows are padded to a multiple of 16.
+//   row_bounds[i]   = {bits of q_lo, bits of d_lo | instance index}   (one row)
+//   block_bounds[b] = {q_lo, d_lo} over rows 4b .. 4b+3
+//   start_table[t * kStartSlots + s] = first group of 16 rows of type t worth looking at
+//                     when the largest d that can still meet the deadline falls in slot s
+constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low bits of a d word
+constexpr int kMaxPaddedRows = GS_MAX_INSTANCES + GS_MAX_TYPES * 16;
+constexpr int kMaxBlocks = kMaxPaddedRows / 4;
+constexpr int kStartSlots = 64;
 
-// One GPU type's entry point: bound over all its rows, and its node range.
+// One GPU type's entry: bound over all its rows, where its rows are, start-table geometry.
 struct __align__(16) TypeHeader {
     float p_lo, q_lo, d_lo, d_max;
-    int begin, end, pad0, pad1;
+    int base;           // first padded row (multiple of 16)
+    int n_groups;       // groups of 16 rows
+    float inv_w;        // slots per unit of d; 0 = no start table, begin at group 0
+    float d0;           // d at the low edge of slot 0
 };
 
 constexpr int kRiskChunk = 1024;        // requests per warp-chunk of the risk scan (32 flag words)
@@ -39,9 +44,11 @@ constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 // Device scratch owned by a context.
 struct Scratch {
     Row *rows;                // [max_instances] exact coefficients, caller order
-    uint2 *nodes;             // [kMaxNodes] search structure of the current round
-    TypeHeader *headers;      // [GS_MAX_TYPES] in walk order (largest d first)
-    int *table_info;          // {n_nodes, unsafe, n_instances, n_active_types}
+    uint2 *row_bounds;        // [kMaxPaddedRows]
+    float2 *block_bounds;     // [kMaxBlocks]
+    unsigned short *start_table;  // [GS_MAX_TYPES * kStartSlots]
+    TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)
+    int *table_info;          // {padded rows, unsafe, n_instances, n_active_types}
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
     float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out

@@ -1,20 +1,21 @@
 // Per-round instance prologue (one CTA):
 //   1. the coefficients of Eq. 2 for every instance and the EMA step of Algorithm 1
 //      (rows[g] = {q_g, p_g, d_g, free KV}, exact, in caller order);
-//   2. the search structure of the route kernel.  Instances are grouped by GPU type (types
+//   2. the search tables of the route kernel.  Instances are grouped by GPU type (types
 //      ordered by their largest d first) and, inside a type, put in preference order
-//      (d descending, index ascending).  Over the rows of a type sits a 4-ary hierarchy of
-//      blocks of 4, 16, 64, 256 consecutive rows; every block and every row becomes an
-//      8-byte node holding a lower bound (q_lo, d_lo) of the q and d of the rows below it.
-//      Nodes are stored in depth-first order with a skip target: "if nothing below this node
-//      can meet the deadline, continue at node X".
+//      (d descending, index ascending).  Per type the tables hold
+//        - a lower bound (q_lo, d_lo) for every row, tagged with the instance index,
+//        - a lower bound for every block of 4 consecutive rows,
+//        - a header with the bound over the whole type, and
+//        - a start table: for a threshold on d, the first group of 16 rows that can matter.
+//      A type's rows are padded to a multiple of 16 with entries that never pass a test.
 //
-// Bounds: q_lo <= q (1 - 2^-19) and d_lo <= d (1 - 2^-19), and the header keeps
-// p_lo = p (1 - 2^-19).  With all coefficients non-negative and each fused step of
-// T = fma(d, y, fma(p, x, q)) rounding by at most 2^-24 relative, the single-precision test
-// fma(d_lo, y, q_lo) > fma(-p_lo, x, D)  then implies  T(r,g) > D  for every row below.
-// The low 11 mantissa bits of the two words carry the skip target and the instance index;
-// the bound is lowered by one unit of the remaining mantissa first, so it stays a lower bound.
+// Bounds: q_lo <= q (1 - 2^-19), d_lo <= d (1 - 2^-19), p_lo = p (1 - 2^-19).  With all
+// coefficients non-negative and each fused step of T = fma(d, y, fma(p, x, q)) rounding by at
+// most 2^-24 relative, the single-precision test  fma(d_lo, y, q_lo) > fma(-p_lo, x, D)
+// implies  T(r,g) > D  for every row the bound covers.  The low bits of a row's d word
+// carry the instance index; the bound is lowered by one unit of the remaining mantissa
+// first, so it stays a lower bound.
 #include "gs_internal.cuh"
 
 namespace gs {
@@ -30,28 +31,13 @@ __device__ __forceinline__ unsigned orderable(float f) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// Number of nodes, inside a type's subtree, that precede every node of row s: s leaves and,
-// per level l = 1 .. levels-1, the blocks of 4^l rows that start before s.
-__device__ __forceinline__ int first_pos(int s, int levels) {
-    int pos = s;
-    for (int l = 1; l < levels; ++l) pos += (s + (1 << (2 * l)) - 1) >> (2 * l);
-    return pos;
-}
-
-// Position of the block of level `level` (0 = single row) that starts at row s: after every
-// higher-level block starting at the same row.
-__device__ __forceinline__ int node_pos(int level, int s, int levels) {
-    int pos = first_pos(s, levels);
-    for (int l = level + 1; l < levels; ++l) pos += (s & ((1 << (2 * l)) - 1)) == 0;
-    return pos;
-}
-
 constexpr float kShrink = 1.0f - 1.9073486328125e-6f;   // 1 - 2^-19
+constexpr unsigned kPadQ = 0x7FC00000u;                 // NaN: compares false with everything
 
-// Bit pattern of a lower bound of v >= 0 whose low kNodeTagBits bits are free for a tag.
+// Bit pattern of a lower bound of v >= 0 whose low tag bits are zero and may be overwritten.
 __device__ __forceinline__ unsigned lower_bound_bits(float v) {
-    const unsigned b = __float_as_uint(__fmul_rn(v, kShrink)) & ~kNodeTagMask;
-    return b >= (kNodeTagMask + 1u) ? b - (kNodeTagMask + 1u) : 0u;
+    const unsigned b = __float_as_uint(__fmul_rn(v, kShrink)) & ~kRowTagMask;
+    return b >= (kRowTagMask + 1u) ? b - (kRowTagMask + 1u) : 0u;
 }
 
 __global__ void __launch_bounds__(GS_MAX_INSTANCES)
@@ -64,18 +50,22 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
 {
     __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];
     __shared__ float sh_q[GS_MAX_INSTANCES], sh_d[GS_MAX_INSTANCES];       // by instance index
-    __shared__ float sh_nq[kMaxNodes];                                     // exact min q per node
+    __shared__ float sh_blk_d[kMaxBlocks];                                 // block d_lo as float
     __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES], sh_row0[GS_MAX_TYPES + 1];
-    __shared__ unsigned sh_dmax[GS_MAX_TYPES];
-    __shared__ int sh_base[GS_MAX_TYPES + 1], sh_levels[GS_MAX_TYPES];
+    __shared__ unsigned sh_dmax[GS_MAX_TYPES], sh_qmin[GS_MAX_TYPES];
+    __shared__ int sh_base[GS_MAX_TYPES + 1];                              // padded row offset per type
+    __shared__ float sh_inv_w[GS_MAX_TYPES], sh_d0[GS_MAX_TYPES];
     __shared__ int sh_unsafe, sh_n_act;
 
     const int g = threadIdx.x;
     unsigned bad = 0;
     float d = 0.f;
     int t = 0;
-    if (g < GS_MAX_TYPES) { sh_cnt[g] = 0; sh_dmax[g] = 0u; }
+    if (g < GS_MAX_TYPES) { sh_cnt[g] = 0; sh_dmax[g] = 0u; sh_qmin[g] = 0xFFFFFFFFu; }
     if (g == 0) sh_unsafe = 0;
+    // every table entry starts as padding
+    for (int i = g; i < kMaxPaddedRows; i += blockDim.x) s.row_bounds[i] = make_uint2(kPadQ, 0u);
+    for (int i = g; i < kMaxBlocks; i += blockDim.x) s.block_bounds[i] = make_float2(__uint_as_float(kPadQ), 0.f);
     __syncthreads();
 
     // ---- 1. coefficients ----------------------------------------------------------------
@@ -97,7 +87,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         s.rows[g] = row;
         s.d_by_g[g] = d;
         s.q_by_g[g] = q;
-        // the bounds of the search structure need finite, non-negative coefficients
+        // the bounds of the search tables need finite, non-negative coefficients
         const float big = 3.0e38f;
         if (!(q >= 0.f && q < big && p >= 0.f && p < big && d >= 0.f && d < big)) atomicOr(&sh_unsafe, 1);
         atomicAdd(&sh_cnt[t], 1);
@@ -105,7 +95,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     }
     __syncthreads();
 
-    // ---- 2. order of the types (largest d first; ties: smaller type id) and their geometry --
+    // ---- 2. order of the types (largest d first; ties: smaller type id), row offsets ------
     if (g < GS_MAX_TYPES) {
         int rank = GS_MAX_TYPES;           // unused types sort last
         if (sh_cnt[g] > 0) {
@@ -117,27 +107,20 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     }
     __syncthreads();
     if (g < GS_MAX_TYPES) {
-        // thread g handles the type at order position g: rows and nodes of the types before it
-        int n_act = 0, row0 = 0, base = 0, my_n = 0, my_type = -1;
+        // thread g handles the type at order position g
+        int n_act = 0, row0 = 0, base = 0, my_n = -1;
         for (int o = 0; o < GS_MAX_TYPES; ++o) {
             const int r = sh_rank[o], n = sh_cnt[o];
             if (n == 0) continue;
             ++n_act;
-            if (r == g) { my_n = n; my_type = o; }
-            if (r < g) {
-                int levels = 1;
-                while ((1 << (2 * levels)) < n) ++levels;
-                row0 += n;
-                base += first_pos(n, levels);
-            }
+            if (r == g) my_n = n;
+            if (r < g) { row0 += n; base += (n + 15) & ~15; }
         }
-        if (my_type >= 0) {
-            int levels = 1;
-            while ((1 << (2 * levels)) < my_n) ++levels;      // smallest L >= 1 with 4^L >= n
-            sh_row0[g] = row0; sh_base[g] = base; sh_levels[g] = levels;
+        if (my_n >= 0) {
+            sh_row0[g] = row0; sh_base[g] = base;
             if (g == n_act - 1) {
                 sh_row0[n_act] = row0 + my_n;
-                sh_base[n_act] = base + first_pos(my_n, levels);
+                sh_base[n_act] = base + ((my_n + 15) & ~15);
                 sh_n_act = n_act;
             }
         }
@@ -166,59 +149,86 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         }
     }
 
-    // ---- 4. leaves ------------------------------------------------------------------------
+    // ---- 4. row bounds, block bounds, per-type minimum of q --------------------------------
     const int n_act = sh_n_act;
-    int tr = 0, k = 0, levels = 0, n_t = 0, base = 0;
-    const bool is_row = g < M;
-    if (is_row) {
+    if (g < M) {
         const unsigned long long key = sh_key[g];
         const int inst = (int)(key & 0xFFFFull);
-        tr = (int)(key >> 48);
-        k = g - sh_row0[tr];
-        n_t = sh_row0[tr + 1] - sh_row0[tr];
-        levels = sh_levels[tr];
-        base = sh_base[tr];
-        const int pos = base + node_pos(0, k, levels);
-        const float rq = sh_q[inst];
-        sh_nq[pos] = rq;
-        s.nodes[pos] = make_uint2(lower_bound_bits(rq) | (unsigned)sh_base[tr + 1],
-                                  lower_bound_bits(sh_d[inst]) | kNodeLeafFlag | (unsigned)inst);
+        const int tr = (int)(key >> 48);
+        const int k = g - sh_row0[tr];
+        const int n_t = sh_row0[tr + 1] - sh_row0[tr];
+        const int base = sh_base[tr];
+        const float rq = sh_q[inst], rd = sh_d[inst];
+        s.row_bounds[base + k] = make_uint2(lower_bound_bits(rq), lower_bound_bits(rd) | (unsigned)inst);
+        if ((k & 3) == 0) {
+            // block of rows k .. k+3 (those that exist); rows are d-descending: the last has the least d
+            const int hi = min(k + 4, n_t);
+            float bq = rq;
+            for (int c = k + 1; c < hi; ++c) bq = fminf(bq, sh_q[(int)(sh_key[g + (c - k)] & 0xFFFFull)]);
+            const float bd = sh_d[(int)(sh_key[g + (hi - 1 - k)] & 0xFFFFull)];
+            const float bq_lo = __uint_as_float(lower_bound_bits(bq));
+            const float bd_lo = __uint_as_float(lower_bound_bits(bd));
+            s.block_bounds[(base + k) >> 2] = make_float2(bq_lo, bd_lo);
+            sh_blk_d[(base + k) >> 2] = bd_lo;
+            atomicMin(&sh_qmin[tr], orderable(bq));
+        }
     }
     __syncthreads();
 
-    // ---- 5. blocks, bottom-up; the thread of a block's first row builds the block ----------
-    for (int l = 1; l <= 5; ++l) {
-        const int w = 1 << (2 * l);
-        const bool type_level = (l == levels);              // covers the whole type: goes to the header
-        if (is_row && l <= levels && (k & (w - 1)) == 0 && (!type_level || k == 0)) {
-            const int hi = min(k + w, n_t);                 // rows [k, hi)
-            float bq = 3.4e38f;
-            for (int c = k; c < hi; c += (w >> 2)) bq = fminf(bq, sh_nq[base + node_pos(l - 1, c, levels)]);
-            const int last_inst = (int)(sh_key[sh_row0[tr] + hi - 1] & 0xFFFFull);   // smallest d
-            const float bd = sh_d[last_inst];
-            if (!type_level) {
-                const int pos = base + node_pos(l, k, levels);
-                sh_nq[pos] = bq;
-                const int skip = base + first_pos(hi, levels);
-                s.nodes[pos] = make_uint2(lower_bound_bits(bq) | (unsigned)skip, lower_bound_bits(bd));
-            } else {
-                const int first_inst = (int)(sh_key[sh_row0[tr]] & 0xFFFFull);
-                TypeHeader h;
-                h.p_lo = __fmul_rn(s.rows[first_inst].p, kShrink);
-                h.q_lo = __uint_as_float(lower_bound_bits(bq));
-                h.d_lo = __uint_as_float(lower_bound_bits(bd));
-                h.d_max = sh_d[first_inst];
-                h.begin = base;
-                h.end = sh_base[tr + 1];
-                h.pad0 = 0; h.pad1 = 0;
-                s.headers[tr] = h;
+    // ---- 5. headers --------------------------------------------------------------------------
+    if (g < n_act) {
+        const int tr = g;
+        const int n_t = sh_row0[tr + 1] - sh_row0[tr];
+        const int base = sh_base[tr];
+        const int first_inst = (int)(sh_key[sh_row0[tr]] & 0xFFFFull);
+        const int last_inst = (int)(sh_key[sh_row0[tr + 1] - 1] & 0xFFFFull);
+        const unsigned qo = sh_qmin[tr];                    // undo the monotone map (q >= 0 when safe)
+        const float qmin = __uint_as_float((qo & 0x80000000u) ? (qo & 0x7FFFFFFFu) : ~qo);
+        const int n_blocks = (n_t + 3) >> 2;
+        const int n_groups = (n_t + 15) >> 4;
+        // start table geometry: S slots between the least and the largest block bound of d
+        const float d_hi = sh_blk_d[base >> 2], d_low = sh_blk_d[(base >> 2) + n_blocks - 1];
+        float inv_w = 0.f;
+        if (n_groups > 1 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f))
+            inv_w = (float)kStartSlots / (d_hi - d_low);
+        sh_inv_w[tr] = inv_w; sh_d0[tr] = d_low;
+        TypeHeader h;
+        h.p_lo = __fmul_rn(s.rows[first_inst].p, kShrink);   // written in step 1 by this CTA
+        h.q_lo = __uint_as_float(lower_bound_bits(qmin));
+        h.d_lo = __uint_as_float(lower_bound_bits(sh_d[last_inst]));
+        h.d_max = sh_d[first_inst];
+        h.base = base;
+        h.n_groups = n_groups;
+        h.inv_w = inv_w;
+        h.d0 = d_low;
+        s.headers[tr] = h;
+    }
+    __syncthreads();
+
+    // ---- 6. start tables: slot -> first group of 16 rows whose blocks are not all above the slot
+    {
+        const int tr = g / kStartSlots, slot = g % kStartSlots;
+        if (tr < n_act) {
+            int start_group = 0;
+            const float inv_w = sh_inv_w[tr];
+            if (inv_w > 0.f) {
+                // two slots of margin absorb the rounding of the kernel's slot computation
+                const float edge = sh_d0[tr] + (float)(slot + 2) / inv_w;
+                const int b0 = sh_base[tr] >> 2;
+                const int n_blocks = (sh_row0[tr + 1] - sh_row0[tr] + 3) >> 2;
+                int lo = 0, hi = n_blocks;                  // blocks [0, lo) have d_lo > edge
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (sh_blk_d[b0 + mid] > edge) lo = mid + 1; else hi = mid;
+                }
+                start_group = lo >> 2;
             }
+            s.start_table[tr * kStartSlots + slot] = (unsigned short)start_group;
         }
-        __syncthreads();
     }
 
     if (g == 0) {
-        s.table_info[0] = sh_base[n_act];      // number of nodes
+        s.table_info[0] = sh_base[n_act];      // padded rows in use
         s.table_info[1] = sh_unsafe;
         s.table_info[2] = M;
         s.table_info[3] = n_act;

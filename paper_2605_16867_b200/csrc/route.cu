@@ -2,22 +2,25 @@
 // (Algorithm 1) for every pending request of a round.
 //
 // One thread owns four consecutive requests (128-bit column loads and stores).  The per-round
-// tables built by the prologue are staged once per CTA in shared memory.  For each request:
-//   1. every GPU type is tested against a lower bound of T over all its instances (same
-//      shared-memory address for all lanes, so a broadcast); types that cannot meet the
-//      deadline are dropped;
-//   2. the surviving types' subtrees are walked depth-first: a block whose lower bound misses
-//      the deadline is skipped with everything below it; a row that passes the (slightly
-//      loose) bound test is scored exactly as the definition says, T = fma(d, y, fma(p, x, q)),
-//      and checked against the deadline and the instance's free KV.
+// tables built by the prologue are staged once per CTA in shared memory.  For each request and
+// each GPU type in turn (types with the largest d first):
+//   1. the type is tested against a lower bound of T over all its instances (the same
+//      shared-memory address for all lanes: a broadcast) and dropped if it cannot meet the
+//      deadline or cannot beat the best d found so far;
+//   2. a start table turns the largest d that could still meet the deadline into the first
+//      group of 16 rows worth looking at;
+//   3. from there, four block bounds (4 rows each) are tested per step until one passes, the
+//      four rows of that block are tested against their own bounds, and a row that passes is
+//      scored exactly as the definition says, T = fma(d, y, fma(p, x, q)), and checked against
+//      the deadline and the instance's free KV.
 // Rows of a type are in preference order (d descending, index ascending), so the first
-// feasible row of a type is that type's best; a later type is left as soon as its rows fall
-// below the best d found so far.  The walk therefore returns exactly argmax d_g over the
-// feasible set, with ties to the smallest index.
+// feasible row of a type is that type's best.  Every bound is a true lower bound in the
+// kernel's own arithmetic, so nothing feasible is ever skipped and the result is exactly
+// argmax d_g over the feasible set, ties to the smallest index.
 //
-// A request for which the walk finds nothing (no feasible instance: the fallback of
-// Algorithm 1) is queued in shared memory and finished by a whole warp that scores every
-// instance, lanes across instances, with shuffle reductions for the argmin.
+// A request for which this finds nothing (no feasible instance: the fallback of Algorithm 1)
+// is queued in shared memory and finished by a whole warp that scores every instance, lanes
+// across instances, with shuffle reductions for the argmin.
 #include "gs_internal.cuh"
 
 namespace gs {
@@ -61,54 +64,83 @@ __device__ __forceinline__ void accumulate_choice(unsigned long long *hist, int 
 // Shared-memory image of the round's tables.
 struct Tables {
     const TypeHeader *headers;
-    const uint2 *nodes;
+    const float2 *block_bounds;
+    const uint2 *row_bounds;
+    const unsigned short *start_table;
     const Row *rows;
     int n_types;
 };
 
-// Just-enough pick for one request.  Returns the chosen instance or -1 (no feasible one).
+__device__ __forceinline__ bool bound_passes(float q_lo, float d_lo, float y, float R) {
+    return __fmaf_rn(d_lo, y, q_lo) <= R;
+}
+
+// Just-enough pick for one request; called by all 32 lanes of the warp together.
+// Returns the chosen instance or -1 (no feasible one, or a request this search does not take).
 __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y, float D, unsigned need,
                                              float &T_out)
 {
-    // 1. which types can hold a feasible instance at all
-    unsigned alive = 0;
+    int g_best = -1;
+    float d_best = -1.0f, T_best = 0.f;
+    const float ry = __frcp_rn(y);            // y == 0 never gets here with a live type (see caller)
     for (int t = 0; t < tb.n_types; ++t) {
         const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);   // p_lo, q_lo, d_lo, d_max
-        const float R = __fmaf_rn(-h.x, x, D);
-        if (__fmaf_rn(h.z, y, h.y) <= R + 1e-30f) alive |= 1u << t;
-    }
-    // 2. walk the surviving subtrees
-    int g_best = -1;
-    float d_best = -1.0f, T_best = 0.f, R = 0.f;
-    int i = 0, end = 0;
-    for (;;) {
-        if (i >= end) {                       // next surviving type, if any can still improve
-            if (alive == 0) break;
-            const int t = __ffs(alive) - 1;
-            alive &= alive - 1;
-            const TypeHeader h = tb.headers[t];
-            if (h.d_max < d_best) break;      // types are ordered by their largest d
-            i = h.begin; end = h.end;
-            R = __fmaf_rn(-h.p_lo, x, D) + 1e-30f;
-        }
-        const uint2 nd = tb.nodes[i];
-        const unsigned target = nd.x & kNodeTagMask;
-        const bool pass = __fmaf_rn(__uint_as_float(nd.y), y, __uint_as_float(nd.x)) <= R;
-        const bool leaf = (nd.y & kNodeLeafFlag) != 0;
-        int next = (pass == leaf) ? (int)target : i + 1;     // block fails -> skip it; row passes -> see below
-        if (pass && leaf) {
-            const int inst = (int)(nd.y & (kNodeLeafFlag - 1));
-            const Row r = tb.rows[inst];
-            const float T = latency(r, x, y);
-            const bool feasible = (T <= D) && (need <= (unsigned)r.kv);
-            const bool worse = r.d < d_best;
-            if (feasible && !worse && (g_best < 0 || r.d > d_best || inst < g_best)) {
-                d_best = r.d; g_best = inst; T_best = T;
+        const float R = __fmaf_rn(-h.x, x, D) + 1e-30f;
+        const bool live = bound_passes(h.y, h.z, y, R) && !(h.w < d_best);
+        if (!__any_sync(0xFFFFFFFFu, live)) continue;
+        if (live) {
+            const int4 g4 = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);  // base, n_groups, inv_w, d0
+            const int n_groups = g4.y;
+            const float inv_w = __int_as_float(g4.z);
+            int grp = 0;
+            if (inv_w > 0.f) {
+                // largest d that can still meet the deadline -> slot -> first group worth a look
+                const float z = (R - h.y) * ry;
+                const float sf = fminf(fmaxf((z - __int_as_float(g4.w)) * inv_w, 0.f), (float)(kStartSlots - 1));
+                grp = tb.start_table[t * kStartSlots + __float2int_rd(sf)];
             }
-            // feasible: the rest of this type ranks lower.  worse: so does everything after it.
-            next = (feasible || worse) ? (int)target : i + 1;
+            const float2 *blocks = tb.block_bounds + (g4.x >> 2);
+            const uint2 *rowb = tb.row_bounds + g4.x;
+            bool done = false;
+            while (!done) {
+                unsigned m = 0;
+                for (; grp < n_groups; ++grp) {
+                    const float4 a = *reinterpret_cast<const float4 *>(blocks + 4 * grp);
+                    const float4 b = *reinterpret_cast<const float4 *>(blocks + 4 * grp + 2);
+                    m = (bound_passes(a.x, a.y, y, R) ? 1u : 0u) | (bound_passes(a.z, a.w, y, R) ? 2u : 0u) |
+                        (bound_passes(b.x, b.y, y, R) ? 4u : 0u) | (bound_passes(b.z, b.w, y, R) ? 8u : 0u);
+                    if (m) break;
+                }
+                if (!m) break;                                   // type exhausted
+                do {
+                    const int blk = __ffs(m) - 1;
+                    m &= m - 1;
+                    const uint4 *rp = reinterpret_cast<const uint4 *>(rowb + 16 * grp + 4 * blk);
+                    const uint4 r0 = rp[0], r1 = rp[1];
+                    unsigned rm =
+                        (bound_passes(__uint_as_float(r0.x), __uint_as_float(r0.y), y, R) ? 1u : 0u) |
+                        (bound_passes(__uint_as_float(r0.z), __uint_as_float(r0.w), y, R) ? 2u : 0u) |
+                        (bound_passes(__uint_as_float(r1.x), __uint_as_float(r1.y), y, R) ? 4u : 0u) |
+                        (bound_passes(__uint_as_float(r1.z), __uint_as_float(r1.w), y, R) ? 8u : 0u);
+                    while (rm) {
+                        const int rr = __ffs(rm) - 1;
+                        rm &= rm - 1;
+                        const unsigned dw = rr == 0 ? r0.y : rr == 1 ? r0.w : rr == 2 ? r1.y : r1.w;
+                        const int inst = (int)(dw & kRowTagMask);
+                        const Row row = tb.rows[inst];
+                        const float T = latency(row, x, y);
+                        const bool feasible = (T <= D) && (need <= (unsigned)row.kv);
+                        const bool worse = row.d < d_best;
+                        if (feasible && !worse && (g_best < 0 || row.d > d_best || inst < g_best)) {
+                            d_best = row.d; g_best = inst; T_best = T;
+                        }
+                        // feasible: the rest of this type ranks lower.  worse: so does all that follows.
+                        if (feasible || worse) { done = true; rm = 0; m = 0; }
+                    }
+                } while (m);
+                ++grp;
+            }
         }
-        i = next;
     }
     T_out = T_best;
     return g_best;
@@ -118,26 +150,31 @@ template <bool kAccumulate>
 __global__ void __launch_bounds__(kRouteThreads)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
              const float *__restrict__ slo_ms, int64_t n,
-             const Row *__restrict__ g_rows, const uint2 *__restrict__ g_nodes,
+             const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
+             const float2 *__restrict__ g_block_bounds, const unsigned short *__restrict__ g_start_table,
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
              int32_t *__restrict__ out_idx, float *__restrict__ out_est,
              float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    const int n_nodes = table_info[0];
+    const int n_padded = table_info[0];
     const bool unsafe = table_info[1] != 0;
     const int M = table_info[2];
     const int n_act = table_info[3];
     Row *sh_rows = reinterpret_cast<Row *>(smem);
     TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
-    uint2 *sh_nodes = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
-    int *sh_queue = reinterpret_cast<int *>(sh_nodes + kMaxNodes);
+    uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
+    float2 *sh_block_bounds = reinterpret_cast<float2 *>(sh_row_bounds + kMaxPaddedRows);
+    unsigned short *sh_start = reinterpret_cast<unsigned short *>(sh_block_bounds + kMaxBlocks);
+    int *sh_queue = reinterpret_cast<int *>(sh_start + GS_MAX_TYPES * kStartSlots);
     int *sh_qcount = sh_queue + kRouteTile;
     unsigned long long *hist = reinterpret_cast<unsigned long long *>(sh_qcount + 4);
 
     for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[k] = g_rows[k];
-    for (int k = threadIdx.x; k < n_nodes; k += blockDim.x) sh_nodes[k] = g_nodes[k];
+    for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
+    for (int k = threadIdx.x; k < (n_padded >> 2); k += blockDim.x) sh_block_bounds[k] = g_block_bounds[k];
+    for (int k = threadIdx.x; k < n_act * kStartSlots; k += blockDim.x) sh_start[k] = g_start_table[k];
     if (threadIdx.x < n_act) sh_headers[threadIdx.x] = g_headers[threadIdx.x];
     if (threadIdx.x == 0) *sh_qcount = 0;
     if (kAccumulate)
@@ -145,7 +182,8 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     __syncthreads();
 
     Tables tb;
-    tb.headers = sh_headers; tb.nodes = sh_nodes; tb.rows = sh_rows;
+    tb.headers = sh_headers; tb.block_bounds = sh_block_bounds; tb.row_bounds = sh_row_bounds;
+    tb.start_table = sh_start; tb.rows = sh_rows;
     tb.n_types = unsafe ? 0 : n_act;          // unusable bounds: every request takes the exhaustive path
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -179,7 +217,10 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             if (yi[j] < 0) { yi[j] = 0; bad |= GS_DEV_BAD_VALUE; }
             const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];      // < 2^32, no overflow
             const bool valid = first + j < n;
-            g_out[j] = pick_instance(tb, __int2float_rn(xi[j]), __int2float_rn(yi[j]), D[j], need, T_out[j]);
+            // an empty slot, or L_out == 0 (the start table divides by it), skips the search;
+            // a real request that comes back empty-handed goes to the exhaustive path below
+            const float Dj = (valid && yi[j] > 0) ? D[j] : -1.0f;
+            g_out[j] = pick_instance(tb, __int2float_rn(xi[j]), __int2float_rn(yi[j]), Dj, need, T_out[j]);
             if (valid && g_out[j] < 0) sh_queue[atomicAdd(sh_qcount, 1)] = threadIdx.x * kReqPerThread + j;
             if (kAccumulate) accumulate_choice(hist, M, valid ? g_out[j] : -1, (unsigned)xi[j], need);
         }
@@ -276,7 +317,9 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
 }
 
 constexpr size_t kRouteSmemBase = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
-                                  (size_t)kMaxNodes * sizeof(uint2) + (kRouteTile + 4) * sizeof(int);
+                                  (size_t)kMaxPaddedRows * sizeof(uint2) + (size_t)kMaxBlocks * sizeof(float2) +
+                                  (size_t)GS_MAX_TYPES * kStartSlots * sizeof(unsigned short) +
+                                  (kRouteTile + 4) * sizeof(int);
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
 
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
@@ -294,11 +337,13 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     if (accumulate)
         route_kernel<true><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.nodes, ctx->s.headers,
+            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.row_bounds, ctx->s.block_bounds,
+            ctx->s.start_table, ctx->s.headers,
             ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     else
         route_kernel<false><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.nodes, ctx->s.headers,
+            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.row_bounds, ctx->s.block_bounds,
+            ctx->s.start_table, ctx->s.headers,
             ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     return cudaGetLastError();
 }
