@@ -157,7 +157,6 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
     struct { void **p; size_t bytes; } allocs[] = {
         {(void **)&s.rows, Mx * sizeof(gs::Row)},
         {(void **)&s.row_bounds, gs::kMaxPaddedRows * sizeof(uint2)},
-        {(void **)&s.block_bounds, gs::kMaxBlocks * sizeof(float2)},
         {(void **)&s.start_table, GS_MAX_TYPES * gs::kStartSlots * sizeof(unsigned short)},
         {(void **)&s.headers, GS_MAX_TYPES * sizeof(gs::TypeHeader)},
         {(void **)&s.table_info, 64},
@@ -181,7 +180,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.block_bounds, s.start_table, s.headers, s.table_info, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.start_table, s.headers, s.table_info, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.status, ctx->stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);

@@ -21,19 +21,25 @@ struct __align__(16) Row {
 // grouped by GPU type and, inside a type, kept in preference order (d descending, index
 // ascending); each type's rows are padded to a multiple of 16.
 //   row_bounds[i]   = {bits of q_lo, bits of d_lo | instance index}   (one row)
-//   block_bounds[b] = {q_lo, d_lo} over rows 4b .. 4b+3
-//   start_table[t * kStartSlots + s] = first group of 16 rows of type t worth looking at
+//   start_table[t * kStartSlots + s] = first row (a multiple of 8) of type t worth looking at
 //                     when the largest d that can still meet the deadline falls in slot s
+// Storage slot of padded row i.  Eight consecutive rows (64 bytes) are read together as four
+// 16-byte chunks; which chunk sits where is XOR-swizzled with the group number so that lanes
+// reading different groups in the same instruction spread over all shared-memory banks.
+__host__ __device__ __forceinline__ int row_slot(int i) {
+    const int group = i >> 3, pair = (i >> 1) & 3;
+    return (group << 3) | (((pair ^ ((group >> 1) & 3)) << 1) | (i & 1));
+}
+
 constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low bits of a d word
 constexpr int kMaxPaddedRows = GS_MAX_INSTANCES + GS_MAX_TYPES * 16;
-constexpr int kMaxBlocks = kMaxPaddedRows / 4;
-constexpr int kStartSlots = 64;
+constexpr int kStartSlots = 128;
 
 // One GPU type's entry: bound over all its rows, where its rows are, start-table geometry.
 struct __align__(16) TypeHeader {
     float p_lo, q_lo, d_lo, d_max;
     int base;           // first padded row (multiple of 16)
-    int n_groups;       // groups of 16 rows
+    int n_padded;       // rows including padding (multiple of 16)
     float inv_w;        // slots per unit of d; 0 = no start table, begin at group 0
     float d0;           // d at the low edge of slot 0
 };
@@ -45,7 +51,6 @@ constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 struct Scratch {
     Row *rows;                // [max_instances] exact coefficients, caller order
     uint2 *row_bounds;        // [kMaxPaddedRows]
-    float2 *block_bounds;     // [kMaxBlocks]
     unsigned short *start_table;  // [GS_MAX_TYPES * kStartSlots]
     TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)
     int *table_info;          // {padded rows, unsafe, n_instances, n_active_types}

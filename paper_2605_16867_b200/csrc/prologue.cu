@@ -5,9 +5,8 @@
 //      ordered by their largest d first) and, inside a type, put in preference order
 //      (d descending, index ascending).  Per type the tables hold
 //        - a lower bound (q_lo, d_lo) for every row, tagged with the instance index,
-//        - a lower bound for every block of 4 consecutive rows,
 //        - a header with the bound over the whole type, and
-//        - a start table: for a threshold on d, the first group of 16 rows that can matter.
+//        - a start table: for a threshold on d, the first group of 8 rows that can matter.
 //      A type's rows are padded to a multiple of 16 with entries that never pass a test.
 //
 // Bounds: q_lo <= q (1 - 2^-19), d_lo <= d (1 - 2^-19), p_lo = p (1 - 2^-19).  With all
@@ -50,7 +49,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
 {
     __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];
     __shared__ float sh_q[GS_MAX_INSTANCES], sh_d[GS_MAX_INSTANCES];       // by instance index
-    __shared__ float sh_blk_d[kMaxBlocks];                                 // block d_lo as float
+    __shared__ float sh_row_d[kMaxPaddedRows];                             // row d_lo as float (untagged)
     __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES], sh_row0[GS_MAX_TYPES + 1];
     __shared__ unsigned sh_dmax[GS_MAX_TYPES], sh_qmin[GS_MAX_TYPES];
     __shared__ int sh_base[GS_MAX_TYPES + 1];                              // padded row offset per type
@@ -65,7 +64,6 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     if (g == 0) sh_unsafe = 0;
     // every table entry starts as padding
     for (int i = g; i < kMaxPaddedRows; i += blockDim.x) s.row_bounds[i] = make_uint2(kPadQ, 0u);
-    for (int i = g; i < kMaxBlocks; i += blockDim.x) s.block_bounds[i] = make_float2(__uint_as_float(kPadQ), 0.f);
     __syncthreads();
 
     // ---- 1. coefficients ----------------------------------------------------------------
@@ -149,29 +147,22 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         }
     }
 
-    // ---- 4. row bounds, block bounds, per-type minimum of q --------------------------------
+    // ---- 4. row bounds, per-type minimum of q -------------------------------------------------
     const int n_act = sh_n_act;
     if (g < M) {
         const unsigned long long key = sh_key[g];
         const int inst = (int)(key & 0xFFFFull);
         const int tr = (int)(key >> 48);
         const int k = g - sh_row0[tr];
-        const int n_t = sh_row0[tr + 1] - sh_row0[tr];
         const int base = sh_base[tr];
-        const float rq = sh_q[inst], rd = sh_d[inst];
-        s.row_bounds[base + k] = make_uint2(lower_bound_bits(rq), lower_bound_bits(rd) | (unsigned)inst);
-        if ((k & 3) == 0) {
-            // block of rows k .. k+3 (those that exist); rows are d-descending: the last has the least d
-            const int hi = min(k + 4, n_t);
-            float bq = rq;
-            for (int c = k + 1; c < hi; ++c) bq = fminf(bq, sh_q[(int)(sh_key[g + (c - k)] & 0xFFFFull)]);
-            const float bd = sh_d[(int)(sh_key[g + (hi - 1 - k)] & 0xFFFFull)];
-            const float bq_lo = __uint_as_float(lower_bound_bits(bq));
-            const float bd_lo = __uint_as_float(lower_bound_bits(bd));
-            s.block_bounds[(base + k) >> 2] = make_float2(bq_lo, bd_lo);
-            sh_blk_d[(base + k) >> 2] = bd_lo;
-            atomicMin(&sh_qmin[tr], orderable(bq));
-        }
+        const float rq = sh_q[inst];
+        const unsigned d_bits = lower_bound_bits(sh_d[inst]);
+        s.row_bounds[row_slot(base + k)] = make_uint2(lower_bound_bits(rq), d_bits | (unsigned)inst);
+        sh_row_d[base + k] = __uint_as_float(d_bits);
+        // one shared-memory atomic per run of equal types inside the warp
+        const unsigned peers = __match_any_sync(__activemask(), tr);
+        const unsigned qmin = __reduce_min_sync(peers, orderable(rq));
+        if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicMin(&sh_qmin[tr], qmin);
     }
     __syncthreads();
 
@@ -181,49 +172,45 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         const int n_t = sh_row0[tr + 1] - sh_row0[tr];
         const int base = sh_base[tr];
         const int first_inst = (int)(sh_key[sh_row0[tr]] & 0xFFFFull);
-        const int last_inst = (int)(sh_key[sh_row0[tr + 1] - 1] & 0xFFFFull);
-        const unsigned qo = sh_qmin[tr];                    // undo the monotone map (q >= 0 when safe)
+        const unsigned qo = sh_qmin[tr];                    // undo the monotone map
         const float qmin = __uint_as_float((qo & 0x80000000u) ? (qo & 0x7FFFFFFFu) : ~qo);
-        const int n_blocks = (n_t + 3) >> 2;
-        const int n_groups = (n_t + 15) >> 4;
-        // start table geometry: S slots between the least and the largest block bound of d
-        const float d_hi = sh_blk_d[base >> 2], d_low = sh_blk_d[(base >> 2) + n_blocks - 1];
+        // start table geometry: kStartSlots slots between the least and the largest row bound of d
+        const float d_hi = sh_row_d[base], d_low = sh_row_d[base + n_t - 1];
         float inv_w = 0.f;
-        if (n_groups > 1 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f))
+        if (n_t > 16 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f))
             inv_w = (float)kStartSlots / (d_hi - d_low);
         sh_inv_w[tr] = inv_w; sh_d0[tr] = d_low;
         TypeHeader h;
         h.p_lo = __fmul_rn(s.rows[first_inst].p, kShrink);   // written in step 1 by this CTA
         h.q_lo = __uint_as_float(lower_bound_bits(qmin));
-        h.d_lo = __uint_as_float(lower_bound_bits(sh_d[last_inst]));
+        h.d_lo = d_low;
         h.d_max = sh_d[first_inst];
         h.base = base;
-        h.n_groups = n_groups;
+        h.n_padded = (n_t + 15) & ~15;
         h.inv_w = inv_w;
         h.d0 = d_low;
         s.headers[tr] = h;
     }
     __syncthreads();
 
-    // ---- 6. start tables: slot -> first group of 16 rows whose blocks are not all above the slot
-    {
-        const int tr = g / kStartSlots, slot = g % kStartSlots;
-        if (tr < n_act) {
-            int start_group = 0;
+    // ---- 6. start tables: slot -> first row (multiple of 8) not certainly above the slot -------
+    for (int e = g; e < n_act * kStartSlots; e += blockDim.x) {
+        const int tr = e / kStartSlots, slot = e % kStartSlots;
+        {
+            int start_row = 0;
             const float inv_w = sh_inv_w[tr];
             if (inv_w > 0.f) {
                 // two slots of margin absorb the rounding of the kernel's slot computation
                 const float edge = sh_d0[tr] + (float)(slot + 2) / inv_w;
-                const int b0 = sh_base[tr] >> 2;
-                const int n_blocks = (sh_row0[tr + 1] - sh_row0[tr] + 3) >> 2;
-                int lo = 0, hi = n_blocks;                  // blocks [0, lo) have d_lo > edge
+                const int b0 = sh_base[tr];
+                int lo = 0, hi = sh_row0[tr + 1] - sh_row0[tr];     // rows [0, lo) have d_lo > edge
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;
-                    if (sh_blk_d[b0 + mid] > edge) lo = mid + 1; else hi = mid;
+                    if (sh_row_d[b0 + mid] > edge) lo = mid + 1; else hi = mid;
                 }
-                start_group = lo >> 2;
+                start_row = lo & ~7;
             }
-            s.start_table[tr * kStartSlots + slot] = (unsigned short)start_group;
+            s.start_table[tr * kStartSlots + slot] = (unsigned short)start_row;
         }
     }
 

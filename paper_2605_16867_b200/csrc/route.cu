@@ -2,25 +2,24 @@
 // (Algorithm 1) for every pending request of a round.
 //
 // One thread owns four consecutive requests (128-bit column loads and stores).  The per-round
-// tables built by the prologue are staged once per CTA in shared memory.  For each request and
-// each GPU type in turn (types with the largest d first):
-//   1. the type is tested against a lower bound of T over all its instances (the same
-//      shared-memory address for all lanes: a broadcast) and dropped if it cannot meet the
-//      deadline or cannot beat the best d found so far;
-//   2. a start table turns the largest d that could still meet the deadline into the first
-//      group of 16 rows worth looking at;
-//   3. from there, four block bounds (4 rows each) are tested per step until one passes, the
-//      four rows of that block are tested against their own bounds, and a row that passes is
-//      scored exactly as the definition says, T = fma(d, y, fma(p, x, q)), and checked against
-//      the deadline and the instance's free KV.
+// tables built by the prologue are staged once per CTA in shared memory.  For each request:
+//   1. every GPU type is tested against a lower bound of T over all its instances (the same
+//      shared-memory address for all lanes: a broadcast); types that cannot meet the deadline
+//      are dropped;
+//   2. for each surviving type (largest d first, and only while it can still beat the best d
+//      found so far) a start table turns the largest d that could still meet the deadline
+//      into the first row worth looking at; from there the rows' own lower bounds are tested
+//      eight at a time, and the first row that passes is scored exactly as the definition
+//      says, T = fma(d, y, fma(p, x, q)), and checked against the deadline and the
+//      instance's free KV.
 // Rows of a type are in preference order (d descending, index ascending), so the first
 // feasible row of a type is that type's best.  Every bound is a true lower bound in the
 // kernel's own arithmetic, so nothing feasible is ever skipped and the result is exactly
 // argmax d_g over the feasible set, ties to the smallest index.
 //
 // A request for which this finds nothing (no feasible instance: the fallback of Algorithm 1)
-// is queued in shared memory and finished by a whole warp that scores every instance, lanes
-// across instances, with shuffle reductions for the argmin.
+// is finished right away by its whole warp, which scores every instance, lanes across
+// instances, with shuffle reductions for the argmin.
 #include "gs_internal.cuh"
 
 namespace gs {
@@ -64,82 +63,97 @@ __device__ __forceinline__ void accumulate_choice(unsigned long long *hist, int 
 // Shared-memory image of the round's tables.
 struct Tables {
     const TypeHeader *headers;
-    const float2 *block_bounds;
     const uint2 *row_bounds;
     const unsigned short *start_table;
     const Row *rows;
     int n_types;
 };
 
-__device__ __forceinline__ bool bound_passes(float q_lo, float d_lo, float y, float R) {
-    return __fmaf_rn(d_lo, y, q_lo) <= R;
+constexpr unsigned kNoRow = 0xFFFFFFFFu;
+
+// Scores one row exactly and folds it into the running best.  Returns true when the search of
+// this type is over: the row is feasible (later rows of the type rank lower) or already ranks
+// below the best found (so does everything after it).
+__device__ __forceinline__ bool score_row(const Tables &tb, int inst, float x, float y, float D, unsigned need,
+                                          int &g_best, float &d_best, float &T_best)
+{
+    const Row row = tb.rows[inst];
+    const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));      // Eq. 2, H = 0
+    const bool feasible = (T <= D) && (need <= (unsigned)row.kv);
+    const bool worse = row.d < d_best;
+    if (feasible && !worse && (g_best < 0 || row.d > d_best || inst < g_best)) {
+        d_best = row.d; g_best = inst; T_best = T;
+    }
+    return feasible || worse;
 }
 
-// Just-enough pick for one request; called by all 32 lanes of the warp together.
-// Returns the chosen instance or -1 (no feasible one, or a request this search does not take).
-__device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y, float D, unsigned need,
-                                             float &T_out)
+// Just-enough pick for one request.  Returns the chosen instance or -1 (no feasible one, or a
+// request this search does not take).  `Dm` is the deadline plus a hair (see the caller).
+__device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y, float D, float Dm,
+                                             unsigned need, float &T_out)
 {
-    int g_best = -1;
-    float d_best = -1.0f, T_best = 0.f;
-    const float ry = __frcp_rn(y);            // y == 0 never gets here with a live type (see caller)
+    // 1. which types can hold a feasible instance at all
+    unsigned alive = 0;
+#pragma unroll 2
     for (int t = 0; t < tb.n_types; ++t) {
         const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);   // p_lo, q_lo, d_lo, d_max
-        const float R = __fmaf_rn(-h.x, x, D) + 1e-30f;
-        const bool live = bound_passes(h.y, h.z, y, R) && !(h.w < d_best);
-        if (!__any_sync(0xFFFFFFFFu, live)) continue;
-        if (live) {
-            const int4 g4 = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);  // base, n_groups, inv_w, d0
-            const int n_groups = g4.y;
-            const float inv_w = __int_as_float(g4.z);
-            int grp = 0;
-            if (inv_w > 0.f) {
-                // largest d that can still meet the deadline -> slot -> first group worth a look
-                const float z = (R - h.y) * ry;
-                const float sf = fminf(fmaxf((z - __int_as_float(g4.w)) * inv_w, 0.f), (float)(kStartSlots - 1));
-                grp = tb.start_table[t * kStartSlots + __float2int_rd(sf)];
+        if (__fmaf_rn(h.z, y, h.y) <= __fmaf_rn(-h.x, x, Dm)) alive |= 1u << t;
+    }
+    int g_best = -1;
+    float d_best = -1.0f, T_best = 0.f;
+    const float ry = __frcp_rn(y);
+    // 2. search them, largest d first
+    while (alive) {
+        const int t = __ffs(alive) - 1;
+        alive &= alive - 1;
+        const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);
+        if (h.w < d_best) break;                                  // no later type can do better
+        const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, inv_w, d0
+        const float R = __fmaf_rn(-h.x, x, Dm);
+        const float inv_w = __int_as_float(geo.z);
+        int k = 0;
+        if (inv_w > 0.f) {
+            // largest d that can still meet the deadline -> slot -> first row worth a look
+            const float z = (R - h.y) * ry;
+            const float sf = fminf(fmaxf((z - __int_as_float(geo.w)) * inv_w, 0.f), (float)(kStartSlots - 1));
+            k = tb.start_table[t * kStartSlots + __float2int_rd(sf)];
+        }
+        const int k_end = geo.x + geo.y;
+        k += geo.x;                                         // padded row index, a multiple of 8
+        for (;;) {
+            // tag word of the first row, from k on, whose bound passes
+            unsigned first = kNoRow;
+            for (; k < k_end; k += 8) {
+                const char *grp = reinterpret_cast<const char *>(tb.row_bounds + k);
+                const int sw = (k >> 4) & 3;                // see row_slot()
+                const uint4 r0 = *reinterpret_cast<const uint4 *>(grp + ((0 ^ sw) << 4));
+                const uint4 r1 = *reinterpret_cast<const uint4 *>(grp + ((1 ^ sw) << 4));
+                const uint4 r2 = *reinterpret_cast<const uint4 *>(grp + ((2 ^ sw) << 4));
+                const uint4 r3 = *reinterpret_cast<const uint4 *>(grp + ((3 ^ sw) << 4));
+                first = __fmaf_rn(__uint_as_float(r3.w), y, __uint_as_float(r3.z)) <= R ? r3.w : first;
+                first = __fmaf_rn(__uint_as_float(r3.y), y, __uint_as_float(r3.x)) <= R ? r3.y : first;
+                first = __fmaf_rn(__uint_as_float(r2.w), y, __uint_as_float(r2.z)) <= R ? r2.w : first;
+                first = __fmaf_rn(__uint_as_float(r2.y), y, __uint_as_float(r2.x)) <= R ? r2.y : first;
+                first = __fmaf_rn(__uint_as_float(r1.w), y, __uint_as_float(r1.z)) <= R ? r1.w : first;
+                first = __fmaf_rn(__uint_as_float(r1.y), y, __uint_as_float(r1.x)) <= R ? r1.y : first;
+                first = __fmaf_rn(__uint_as_float(r0.w), y, __uint_as_float(r0.z)) <= R ? r0.w : first;
+                first = __fmaf_rn(__uint_as_float(r0.y), y, __uint_as_float(r0.x)) <= R ? r0.y : first;
+                if (first != kNoRow) break;
             }
-            const float2 *blocks = tb.block_bounds + (g4.x >> 2);
-            const uint2 *rowb = tb.row_bounds + g4.x;
-            bool done = false;
-            while (!done) {
-                unsigned m = 0;
-                for (; grp < n_groups; ++grp) {
-                    const float4 a = *reinterpret_cast<const float4 *>(blocks + 4 * grp);
-                    const float4 b = *reinterpret_cast<const float4 *>(blocks + 4 * grp + 2);
-                    m = (bound_passes(a.x, a.y, y, R) ? 1u : 0u) | (bound_passes(a.z, a.w, y, R) ? 2u : 0u) |
-                        (bound_passes(b.x, b.y, y, R) ? 4u : 0u) | (bound_passes(b.z, b.w, y, R) ? 8u : 0u);
-                    if (m) break;
-                }
-                if (!m) break;                                   // type exhausted
-                do {
-                    const int blk = __ffs(m) - 1;
-                    m &= m - 1;
-                    const uint4 *rp = reinterpret_cast<const uint4 *>(rowb + 16 * grp + 4 * blk);
-                    const uint4 r0 = rp[0], r1 = rp[1];
-                    unsigned rm =
-                        (bound_passes(__uint_as_float(r0.x), __uint_as_float(r0.y), y, R) ? 1u : 0u) |
-                        (bound_passes(__uint_as_float(r0.z), __uint_as_float(r0.w), y, R) ? 2u : 0u) |
-                        (bound_passes(__uint_as_float(r1.x), __uint_as_float(r1.y), y, R) ? 4u : 0u) |
-                        (bound_passes(__uint_as_float(r1.z), __uint_as_float(r1.w), y, R) ? 8u : 0u);
-                    while (rm) {
-                        const int rr = __ffs(rm) - 1;
-                        rm &= rm - 1;
-                        const unsigned dw = rr == 0 ? r0.y : rr == 1 ? r0.w : rr == 2 ? r1.y : r1.w;
-                        const int inst = (int)(dw & kRowTagMask);
-                        const Row row = tb.rows[inst];
-                        const float T = latency(row, x, y);
-                        const bool feasible = (T <= D) && (need <= (unsigned)row.kv);
-                        const bool worse = row.d < d_best;
-                        if (feasible && !worse && (g_best < 0 || row.d > d_best || inst < g_best)) {
-                            d_best = row.d; g_best = inst; T_best = T;
-                        }
-                        // feasible: the rest of this type ranks lower.  worse: so does all that follows.
-                        if (feasible || worse) { done = true; rm = 0; m = 0; }
-                    }
-                } while (m);
-                ++grp;
+            if (first == kNoRow) break;                     // type exhausted
+            // lanes meet again here, so the exact scoring runs once per warp, not once per step
+            if (score_row(tb, (int)(first & kRowTagMask), x, y, D, need, g_best, d_best, T_best)) break;
+            // rare: the bound passed but the row is not feasible (KV, or inside the bound's
+            // margin); go on row by row through the rest of these eight, then resume
+            bool over = false, seen = false;
+            for (int j = 0; j < 8 && !over; ++j) {
+                const uint2 rb = tb.row_bounds[row_slot(k + j)];
+                if (!seen) { seen = (rb.y == first); continue; }
+                if (__fmaf_rn(__uint_as_float(rb.y), y, __uint_as_float(rb.x)) <= R)
+                    over = score_row(tb, (int)(rb.y & kRowTagMask), x, y, D, need, g_best, d_best, T_best);
             }
+            if (over) break;
+            k += 8;
         }
     }
     T_out = T_best;
@@ -147,11 +161,11 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
 }
 
 template <bool kAccumulate>
-__global__ void __launch_bounds__(kRouteThreads)
+__global__ void __launch_bounds__(kRouteThreads, 4)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
              const float *__restrict__ slo_ms, int64_t n,
              const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
-             const float2 *__restrict__ g_block_bounds, const unsigned short *__restrict__ g_start_table,
+             const unsigned short *__restrict__ g_start_table,
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
              int32_t *__restrict__ out_idx, float *__restrict__ out_est,
              float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
@@ -165,32 +179,31 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     Row *sh_rows = reinterpret_cast<Row *>(smem);
     TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
     uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
-    float2 *sh_block_bounds = reinterpret_cast<float2 *>(sh_row_bounds + kMaxPaddedRows);
-    unsigned short *sh_start = reinterpret_cast<unsigned short *>(sh_block_bounds + kMaxBlocks);
-    int *sh_queue = reinterpret_cast<int *>(sh_start + GS_MAX_TYPES * kStartSlots);
-    int *sh_qcount = sh_queue + kRouteTile;
-    unsigned long long *hist = reinterpret_cast<unsigned long long *>(sh_qcount + 4);
+    unsigned short *sh_start = reinterpret_cast<unsigned short *>(sh_row_bounds + kMaxPaddedRows);
+    unsigned long long *hist = reinterpret_cast<unsigned long long *>(sh_start + GS_MAX_TYPES * kStartSlots);
 
     for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[k] = g_rows[k];
     for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
-    for (int k = threadIdx.x; k < (n_padded >> 2); k += blockDim.x) sh_block_bounds[k] = g_block_bounds[k];
     for (int k = threadIdx.x; k < n_act * kStartSlots; k += blockDim.x) sh_start[k] = g_start_table[k];
     if (threadIdx.x < n_act) sh_headers[threadIdx.x] = g_headers[threadIdx.x];
-    if (threadIdx.x == 0) *sh_qcount = 0;
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
     __syncthreads();
 
     Tables tb;
-    tb.headers = sh_headers; tb.block_bounds = sh_block_bounds; tb.row_bounds = sh_row_bounds;
+    tb.headers = sh_headers; tb.row_bounds = sh_row_bounds;
     tb.start_table = sh_start; tb.rows = sh_rows;
     tb.n_types = unsafe ? 0 : n_act;          // unusable bounds: every request takes the exhaustive path
 
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
     unsigned bad = 0;
-    const int64_t n_tiles = (n + kRouteTile - 1) / kRouteTile;
-    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        const int64_t first = tile * kRouteTile + (int64_t)threadIdx.x * kReqPerThread;
+    // a warp takes 128 consecutive requests at a time; nothing below needs a CTA barrier
+    constexpr int kWarpTile = 32 * kReqPerThread;
+    const int64_t n_wtiles = (n + kWarpTile - 1) / kWarpTile;
+    const int64_t warp_stride = (int64_t)gridDim.x * (kRouteThreads / 32);
+    for (int64_t wt = (int64_t)blockIdx.x * (kRouteThreads / 32) + (threadIdx.x >> 5); wt < n_wtiles;
+         wt += warp_stride) {
+        const int64_t first = wt * kWarpTile + (int64_t)lane * kReqPerThread;
         int xi[kReqPerThread], yi[kReqPerThread];
         float D[kReqPerThread];
         if (first + kReqPerThread <= n) {
@@ -211,17 +224,70 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         }
         int g_out[kReqPerThread];
         float T_out[kReqPerThread];
+        unsigned tiers = 0x01010101u;             // one byte per request
 #pragma unroll
         for (int j = 0; j < kReqPerThread; ++j) {
             if (xi[j] < 0) { xi[j] = 0; bad |= GS_DEV_BAD_VALUE; }
             if (yi[j] < 0) { yi[j] = 0; bad |= GS_DEV_BAD_VALUE; }
             const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];      // < 2^32, no overflow
             const bool valid = first + j < n;
+            const float x = __int2float_rn(xi[j]), y = __int2float_rn(yi[j]);
             // an empty slot, or L_out == 0 (the start table divides by it), skips the search;
-            // a real request that comes back empty-handed goes to the exhaustive path below
+            // a real request that comes back empty-handed goes to the exhaustive path below.
+            // (the hair added to the deadline of the bound tests keeps them safe when a bound's
+            // tag bits make a zero coefficient a denormal)
             const float Dj = (valid && yi[j] > 0) ? D[j] : -1.0f;
-            g_out[j] = pick_instance(tb, __int2float_rn(xi[j]), __int2float_rn(yi[j]), Dj, need, T_out[j]);
-            if (valid && g_out[j] < 0) sh_queue[atomicAdd(sh_qcount, 1)] = threadIdx.x * kReqPerThread + j;
+            g_out[j] = pick_instance(tb, x, y, Dj, Dj + 1e-30f, need, T_out[j]);
+
+            // ---- no feasible instance found: the whole warp scores every instance -------------
+            unsigned todo = __ballot_sync(0xFFFFFFFFu, valid && g_out[j] < 0);
+            while (todo) {
+                const int src = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const float xs = __shfl_sync(0xFFFFFFFFu, x, src), ys = __shfl_sync(0xFFFFFFFFu, y, src);
+                const float Ds = __shfl_sync(0xFFFFFFFFu, D[j], src);
+                const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
+                unsigned long long k_feas = 0ull;                    // max over feasible: (d, smallest index)
+                unsigned long long k_room = ~0ull, k_all = ~0ull;    // min over KV-ok / all: (T, index)
+                float T_feas = 0.f;
+                for (int inst = lane; inst < M; inst += 32) {
+                    const Row row = sh_rows[inst];
+                    const float T = latency(row, xs, ys);
+                    const bool room = needs <= (unsigned)row.kv;
+                    const unsigned long long kt = ((unsigned long long)orderable_bits(T) << 32) | (unsigned)inst;
+                    if (kt < k_all) k_all = kt;
+                    if (room && kt < k_room) k_room = kt;
+                    if (room && T <= Ds) {
+                        const unsigned long long kd =
+                            ((unsigned long long)orderable_bits(row.d) << 32) | (0xFFFFu - (unsigned)inst);
+                        if (kd > k_feas) { k_feas = kd; T_feas = T; }
+                    }
+                }
+                unsigned long long w_feas = k_feas, w_room = k_room, w_all = k_all;
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) {
+                    const unsigned long long a = __shfl_xor_sync(0xFFFFFFFFu, w_feas, off);
+                    const unsigned long long b = __shfl_xor_sync(0xFFFFFFFFu, w_room, off);
+                    const unsigned long long c = __shfl_xor_sync(0xFFFFFFFFu, w_all, off);
+                    if (a > w_feas) w_feas = a;
+                    if (b < w_room) w_room = b;
+                    if (c < w_all) w_all = c;
+                }
+                int g; float T; unsigned tier;
+                if (w_feas != 0ull) {
+                    const unsigned owner = __ballot_sync(0xFFFFFFFFu, k_feas == w_feas);
+                    T = __shfl_sync(0xFFFFFFFFu, T_feas, __ffs(owner) - 1);
+                    g = (int)(0xFFFFu - (unsigned)(w_feas & 0xFFFFu)); tier = 1;
+                } else if (w_room != ~0ull) {
+                    g = (int)(w_room & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_room >> 32)); tier = 2;
+                } else {
+                    g = (int)(w_all & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_all >> 32)); tier = 3;
+                }
+                if (lane == src) {
+                    g_out[j] = g; T_out[j] = T;
+                    tiers = (tiers & ~(0xFFu << (8 * j))) | (tier << (8 * j));
+                }
+            }
             if (kAccumulate) accumulate_choice(hist, M, valid ? g_out[j] : -1, (unsigned)xi[j], need);
         }
         if (first + kReqPerThread <= n) {
@@ -230,7 +296,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             __stcs(reinterpret_cast<float4 *>(out_slack + first),
                    make_float4(__fsub_rn(D[0], T_out[0]), __fsub_rn(D[1], T_out[1]),
                                __fsub_rn(D[2], T_out[2]), __fsub_rn(D[3], T_out[3])));
-            if (out_tier) *reinterpret_cast<uchar4 *>(out_tier + first) = make_uchar4(1, 1, 1, 1);
+            if (out_tier) *reinterpret_cast<unsigned *>(out_tier + first) = tiers;
         } else {
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j)
@@ -238,72 +304,9 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                     out_idx[first + j] = g_out[j];
                     out_est[first + j] = T_out[j];
                     out_slack[first + j] = __fsub_rn(D[j], T_out[j]);
-                    if (out_tier) out_tier[first + j] = 1;
+                    if (out_tier) out_tier[first + j] = (uint8_t)((tiers >> (8 * j)) & 0xFFu);
                 }
         }
-        __syncthreads();
-
-        // ---- requests with no feasible instance: one warp each, lanes across instances ----
-        const int n_queued = *sh_qcount;
-        for (int e = warp; e < n_queued; e += kRouteThreads / 32) {
-            const int64_t r = tile * kRouteTile + sh_queue[e];
-            int xr = prompt_len[r], yr = pred_decode_len[r];
-            if (xr < 0) xr = 0;
-            if (yr < 0) yr = 0;
-            const float Dr = slo_ms[r];
-            const float x = __int2float_rn(xr), y = __int2float_rn(yr);
-            const unsigned need = (unsigned)xr + (unsigned)yr;
-            unsigned long long k_feas = 0ull;                    // max over feasible: (d, smallest index)
-            unsigned long long k_room = ~0ull, k_all = ~0ull;    // min over KV-ok / all: (T, index)
-            float T_feas = 0.f;
-            for (int inst = lane; inst < M; inst += 32) {
-                const Row row = sh_rows[inst];
-                const float T = latency(row, x, y);
-                const bool room = need <= (unsigned)row.kv;
-                const unsigned long long kt = ((unsigned long long)orderable_bits(T) << 32) | (unsigned)inst;
-                if (kt < k_all) k_all = kt;
-                if (room && kt < k_room) k_room = kt;
-                if (room && T <= Dr) {
-                    const unsigned long long kd =
-                        ((unsigned long long)orderable_bits(row.d) << 32) | (0xFFFFu - (unsigned)inst);
-                    if (kd > k_feas) { k_feas = kd; T_feas = T; }
-                }
-            }
-            unsigned long long w_feas = k_feas, w_room = k_room, w_all = k_all;
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const unsigned long long a = __shfl_xor_sync(0xFFFFFFFFu, w_feas, off);
-                const unsigned long long b = __shfl_xor_sync(0xFFFFFFFFu, w_room, off);
-                const unsigned long long c = __shfl_xor_sync(0xFFFFFFFFu, w_all, off);
-                if (a > w_feas) w_feas = a;
-                if (b < w_room) w_room = b;
-                if (c < w_all) w_all = c;
-            }
-            int g; float T; uint8_t tier;
-            if (w_feas != 0ull) {
-                const unsigned owner = __ballot_sync(0xFFFFFFFFu, k_feas == w_feas);
-                T = __shfl_sync(0xFFFFFFFFu, T_feas, __ffs(owner) - 1);
-                g = (int)(0xFFFFu - (unsigned)(w_feas & 0xFFFFu)); tier = 1;
-            } else if (w_room != ~0ull) {
-                g = (int)(w_room & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_room >> 32)); tier = 2;
-            } else {
-                g = (int)(w_all & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_all >> 32)); tier = 3;
-            }
-            if (lane == 0) {
-                out_idx[r] = g;
-                out_est[r] = T;
-                out_slack[r] = __fsub_rn(Dr, T);
-                if (out_tier) out_tier[r] = tier;
-                if (kAccumulate) {
-                    atomicAdd(&hist[g], (unsigned long long)(unsigned)xr);
-                    atomicAdd(&hist[M + g], 1ull);
-                    atomicAdd(&hist[2 * M + g], (unsigned long long)need);
-                }
-            }
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) *sh_qcount = 0;
-        __syncthreads();
     }
     if (bad) atomicOr(status, bad);
 
@@ -317,9 +320,8 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
 }
 
 constexpr size_t kRouteSmemBase = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
-                                  (size_t)kMaxPaddedRows * sizeof(uint2) + (size_t)kMaxBlocks * sizeof(float2) +
-                                  (size_t)GS_MAX_TYPES * kStartSlots * sizeof(unsigned short) +
-                                  (kRouteTile + 4) * sizeof(int);
+                                  (size_t)kMaxPaddedRows * sizeof(uint2) +
+                                  (size_t)GS_MAX_TYPES * kStartSlots * sizeof(unsigned short);
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
 
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
@@ -330,19 +332,18 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     (void)M;
     if (n == 0) return cudaSuccess;
     const size_t smem = kRouteSmemBase + (accumulate ? kRouteSmemHist : 0);
-    const int64_t n_tiles = (n + kRouteTile - 1) / kRouteTile;
-    int64_t blocks = n_tiles;
+    int64_t blocks = (n + kRouteTile - 1) / kRouteTile;
     const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm;
     if (blocks > cap) blocks = cap;
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     if (accumulate)
         route_kernel<true><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.row_bounds, ctx->s.block_bounds,
+            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.row_bounds,
             ctx->s.start_table, ctx->s.headers,
             ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     else
         route_kernel<false><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.row_bounds, ctx->s.block_bounds,
+            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.row_bounds,
             ctx->s.start_table, ctx->s.headers,
             ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     return cudaGetLastError();
