@@ -150,7 +150,7 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
     ctx->pending = new (std::nothrow) std::vector<gs_ctx::TimedLaunch>();
     ctx->free_events = new (std::nothrow) std::vector<cudaEvent_t>();
     if (!ctx->pending || !ctx->free_events) { delete ctx->pending; delete ctx->free_events; delete ctx; return GS_ERR_INVALID_ARG; }
-    ctx->chunk_cap = ((size_t)gs::kMaxActive + gs::kRiskChunk - 1) / gs::kRiskChunk;
+    ctx->max_tiles = ((size_t)gs::kMaxActive + 8 * gs::kRiskChunk - 1) / (8 * gs::kRiskChunk);
 
     const size_t Mx = GS_MAX_INSTANCES;
     gs::Scratch &s = ctx->s;
@@ -163,7 +163,8 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
         {(void **)&s.d_by_g, Mx * sizeof(float)},
         {(void **)&s.q_by_g, Mx * sizeof(float)},
         {(void **)&s.deltas, 3 * Mx * sizeof(unsigned long long)},
-        {(void **)&s.chunk_counts, (ctx->chunk_cap + 1) * sizeof(unsigned)},
+        {(void **)&s.tile_status, ctx->max_tiles * sizeof(unsigned long long)},
+        {(void **)&s.ticket, 256},
         {(void **)&s.status, 256},
     };
     for (auto &a : allocs) {
@@ -180,7 +181,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.start_table, s.headers, s.table_info, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.start_table, s.headers, s.table_info, s.d_by_g, s.q_by_g, s.deltas, s.tile_status, s.ticket, s.status, ctx->stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);
@@ -290,11 +291,9 @@ GS_API int gs_risk_scan(gs_ctx *ctx, const int32_t *assigned_inst, const int32_t
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GS_ERR_NO_DEVICE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    // the scan needs d_g only; the EMA weight does not enter it
-    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, 0.0f, st);
-    if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = gs::launch_risk(ctx, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, n_active,
-                        inst->n_instances, out_flag_bits, out_cand_idx, cand_capacity, out_cand_count, st);
+    const cudaError_t e = gs::launch_risk(ctx, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms,
+                                          n_active, *inst, *types, out_flag_bits, out_cand_idx, cand_capacity,
+                                          out_cand_count, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 

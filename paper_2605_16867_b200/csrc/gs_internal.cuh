@@ -57,7 +57,8 @@ struct Scratch {
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
     float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out
-    unsigned *chunk_counts;   // [chunk_cap + 1] flagged requests per risk chunk, then offsets
+    unsigned long long *tile_status;  // [max_tiles] risk scan: published flag counts / prefixes
+    unsigned *ticket;         // risk scan: tile ticket counter
     unsigned *status;         // device status word
 };
 
@@ -70,7 +71,9 @@ struct gs_ctx {
     int n_sm;
     int route_ctas_per_sm;
     gs::Scratch s;
-    size_t chunk_cap;
+    size_t max_tiles;            // risk scan tiles the status array can hold
+    unsigned scan_epoch;         // tags the status words of the current scan
+    unsigned ticket_base;        // value of the ticket counter before the next scan
     int64_t launches;
     int last_cuda_error;
     // staging for the *_host entry points (device memory, grown on demand)
@@ -105,7 +108,7 @@ cudaError_t configure_route(gs_ctx *ctx);
 cudaError_t launch_advance(gs_ctx *ctx, const gs_instances_mut &inst, cudaStream_t st);
 cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *generated,
                         const int32_t *pred_len, const float *elapsed, const float *slo,
-                        int64_t n_active, int n_instances,
+                        int64_t n_active, const gs_instances &inst, const gs_types &types,
                         uint32_t *flag_bits, int32_t *cand_idx, int64_t cand_capacity,
                         int64_t *cand_count, cudaStream_t st);
 
