@@ -35,7 +35,7 @@ METRIC = "request-instance pairs scored/sec"
 UNIT = "pairs/s"
 ROUTE_BYTES_PER_REQUEST = 24      # 3 input columns + 3 output columns, 4 B each
 RISK_BYTES_PER_REQUEST = 20.125   # 5 input columns + 1 flag bit (candidate indices added per flag)
-KERNEL_NAMES = ("prologue", "route", "advance", "risk_scan")
+KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter")
 
 
 # --------------------------------------------------------------------------------------
@@ -320,7 +320,8 @@ def run_gpu(args):
         per_kernel[name] = {"launches": n, "avg_us": ms / n * 1e3}
     dominant = max(kernel_ms, key=lambda k: kernel_ms[k][0]) if kernel_ms else None
     alg_bytes = {"route": ROUTE_BYTES_PER_REQUEST * N + 20 * M,
-                 "risk_scan": 20 * A + 4 * ((A + 31) // 32) + 4 * flagged}
+                 "risk_flags": 20 * A + 4 * ((A + 31) // 32) + 4 * ((A + 1023) // 1024),
+                 "risk_scatter": 4 * ((A + 31) // 32) + 4 * flagged + 4 * ((A + 1023) // 1024)}
     roofline = None
     if dominant in alg_bytes:
         ms, n = kernel_ms[dominant]
@@ -334,7 +335,7 @@ def run_gpu(args):
             per_kernel[name]["algorithmic_GBps"] = gbs
             per_kernel[name]["frac_of_hbm_peak"] = gbs / peak
     route_ms = sum(kernel_ms[k][0] for k in ("prologue", "route") if k in kernel_ms) / args.steps
-    risk_ms = sum(kernel_ms[k][0] for k in ("risk_scan",) if k in kernel_ms) / args.steps
+    risk_ms = sum(kernel_ms[k][0] for k in ("risk_flags", "risk_scatter") if k in kernel_ms) / args.steps
     step_bytes = ROUTE_BYTES_PER_REQUEST * N + RISK_BYTES_PER_REQUEST * A + 4 * flagged
 
     line = {

@@ -133,8 +133,9 @@ enum gs_kernel {
     GS_K_PROLOGUE = 0,       /* instance coefficients + preference order (per round) */
     GS_K_ROUTE = 1,          /* pair scoring + selection */
     GS_K_ADVANCE = 2,        /* state advance */
-    GS_K_RISK_SCAN = 3,      /* risk test + flag words + ordered candidate list, one pass */
-    GS_K_COUNT = 4
+    GS_K_RISK_FLAGS = 3,     /* risk test + flag words + per-chunk flag counts */
+    GS_K_RISK_SCATTER = 4,   /* ordered candidate list */
+    GS_K_COUNT = 5
 };
 
 /* Optional per-kernel timing for benchmarks.  While enabled (on != 0) every kernel launch of
@@ -229,8 +230,8 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx,
  * plugin running inside someone else's memory pool, a latency-critical loop where an
  * allocation's implicit device synchronisation is unacceptable.  Such callers cannot create
  * a gs_ctx (gs_create allocates), so this call takes none: the scratch that gs_risk_scan
- * keeps in its context (the per-tile flag counts its kernel exchanges, a ticket counter) lives instead
- * in a fixed array inside the library image, about 16 KB that every GPU loading the library
+ * keeps in its context (the flag counts its two passes exchange) lives instead
+ * in a fixed array inside the library image, 66 KB that every GPU loading the library
  * holds until the process exits.  It computes exactly what gs_risk_scan computes, with the
  * same kernels; inputs, outputs and their layout are the same and still belong to the caller.
  *

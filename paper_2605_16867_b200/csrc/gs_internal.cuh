@@ -57,8 +57,8 @@ struct Scratch {
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
     float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out
-    unsigned long long *tile_status;  // [max_tiles] risk scan: published flag counts / prefixes
-    unsigned *ticket;         // risk scan: tile ticket counter
+    unsigned *chunk_counts;   // [max_chunks] risk scan: flags per chunk of 1024 requests
+    unsigned *group_totals;   // [2 * max_groups] risk scan: flags per 64 chunks, two parities
     unsigned *status;         // device status word
 };
 
@@ -71,9 +71,9 @@ struct gs_ctx {
     int n_sm;
     int route_ctas_per_sm;
     gs::Scratch s;
-    size_t max_tiles;            // risk scan tiles the status array can hold
-    unsigned scan_epoch;         // tags the status words of the current scan
-    unsigned ticket_base;        // value of the ticket counter before the next scan
+    size_t max_chunks, max_groups;   // capacity of the risk scan's count arrays
+    unsigned scan_epoch;             // its parity selects the group-total buffer of the next scan
+    int64_t scan_dirty[2];           // entries of each group-total buffer that may be non-zero
     int64_t launches;
     int last_cuda_error;
     // staging for the *_host entry points (device memory, grown on demand)
@@ -91,6 +91,7 @@ struct gs_ctx {
 namespace gs {
 
 // Brackets one kernel launch with events when timing is enabled; counts the launch.
+// (ctx may be null: then nothing is counted or timed)
 struct LaunchTimer {
     gs_ctx *ctx; cudaStream_t st; int kernel; cudaEvent_t start = nullptr, stop = nullptr;
     LaunchTimer(gs_ctx *c, int k, cudaStream_t s);

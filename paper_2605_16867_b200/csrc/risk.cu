@@ -1,21 +1,19 @@
 // gs_risk_scan: the SLO-violation risk test of Sec. 3.4 over all active requests and the
-// ordered compaction of the flagged ones (migration candidates), in ONE pass over the data.
+// ordered compaction of the flagged ones (migration candidates).
 //
-// A CTA takes tiles of 8192 requests (a ticket from a global counter, so a tile's predecessors
-// are always already running).  Each of its 8 warps streams 1024 requests of the five columns,
-// gathers d_g of the assigned instance from shared memory (computed per CTA from the raw
-// instance state: d_g = a_t + b_t * batch_g), and forms one flag word per 32 requests with a
-// warp ballot.  The tile's flag count is published and the tile's offset in the candidate list
-// is obtained by a decoupled look-back over the preceding tiles' published counts (each tile
-// first publishes its own count, then its inclusive prefix once known).  The candidate indices
-// are written straight from the flag words still in registers: a request's position is the
-// tile offset plus popc of the lower flags.
+// Pass 1 (risk_flags_kernel) streams the five request columns once.  Each CTA first computes
+// d_g = a_t + b_t * batch_g for every instance into shared memory; a warp then takes chunks of
+// 1024 requests, gathers d_g of the assigned instance, and emits one flag word per 32 requests
+// with a warp ballot.  It leaves the chunk's number of flags, and adds it to the total of the
+// chunk's group of 64 chunks.
+// Pass 2 (scatter_candidates_kernel) re-reads only the flag words.  Every warp owns a
+// contiguous run of chunks; it sums the group totals and chunk counts that precede its run
+// once, then keeps a running offset, and writes the ascending candidate list: a request's
+// position is that offset plus popc of the lower flags.
+// There is no device-side wait anywhere in the scan.
 //
-// The look-back is the only device-side wait.  It is bounded: after kSpinLimit polls the CTA
-// sets GS_DEV_TIMEOUT, publishes a prefix anyway so that nobody else waits on it, and goes on
-// (that call's candidate list is then invalid; every write stays in bounds).
-//
-// Tile status words carry the call's epoch, so the status array never needs clearing.
+// The group totals are double-buffered by call parity: pass 2 of one call clears the buffer
+// that pass 1 of the next call adds into.
 #include <mutex>
 
 #include "gs_internal.cuh"
@@ -25,37 +23,18 @@ namespace gs {
 constexpr int kRiskThreads = 256;
 constexpr int kRiskWarps = kRiskThreads / 32;
 constexpr int kRiskUnroll = 4;          // independent 32-request groups in flight per warp
-constexpr int kRiskTile = kRiskWarps * kRiskChunk;   // requests per CTA tile
-constexpr unsigned kSpinLimit = 4000000u;
-constexpr unsigned kFlagAggregate = 1u, kFlagPrefix = 2u;
-
-__device__ __forceinline__ unsigned long long pack_status(unsigned epoch, unsigned flag, unsigned value) {
-    return ((unsigned long long)((epoch << 2) | flag) << 32) | value;
-}
-
-__device__ __forceinline__ unsigned long long load_status(const unsigned long long *p) {
-    return *reinterpret_cast<const volatile unsigned long long *>(p);
-}
-
-__device__ __forceinline__ void store_status(unsigned long long *p, unsigned long long v) {
-    *reinterpret_cast<volatile unsigned long long *>(p) = v;
-}
+constexpr int kGroupShift = 6;          // 64 chunks per group
 
 __global__ void __launch_bounds__(kRiskThreads)
-risk_scan_kernel(const int32_t *__restrict__ assigned, const int32_t *__restrict__ generated,
-                 const int32_t *__restrict__ pred_len, const float *__restrict__ elapsed,
-                 const float *__restrict__ slo, int64_t n,
-                 const int32_t *__restrict__ type_id, const int32_t *__restrict__ batch, int M,
-                 const float *__restrict__ a_type, const float *__restrict__ b_type, int n_types,
-                 uint32_t *__restrict__ flag_bits, int32_t *__restrict__ cand_idx, int64_t cand_capacity,
-                 int64_t *__restrict__ cand_count,
-                 unsigned long long *__restrict__ tile_status, unsigned *__restrict__ ticket,
-                 unsigned ticket_base, unsigned epoch, unsigned n_tiles, unsigned *__restrict__ status)
+risk_flags_kernel(const int32_t *__restrict__ assigned, const int32_t *__restrict__ generated,
+                  const int32_t *__restrict__ pred_len, const float *__restrict__ elapsed,
+                  const float *__restrict__ slo, int64_t n,
+                  const int32_t *__restrict__ type_id, const int32_t *__restrict__ batch, int M,
+                  const float *__restrict__ a_type, const float *__restrict__ b_type, int n_types,
+                  uint32_t *__restrict__ flag_bits, unsigned *__restrict__ chunk_counts,
+                  unsigned *__restrict__ group_totals, int64_t n_chunks, unsigned *__restrict__ status)
 {
     __shared__ float sh_d[GS_MAX_INSTANCES];
-    __shared__ unsigned sh_wcount[kRiskWarps];      // flags per warp, then exclusive offsets
-    __shared__ unsigned sh_prefix, sh_tile;
-
     unsigned bad = 0;
     for (int g = threadIdx.x; g < M; g += blockDim.x) {
         int t = type_id[g];
@@ -65,21 +44,16 @@ risk_scan_kernel(const int32_t *__restrict__ assigned, const int32_t *__restrict
         sh_d[g] = __fmaf_rn(b_type[t], __int2float_rn(B), a_type[t]);   // loaded per-token decode latency
     }
     if (blockIdx.x != 0) bad = 0;           // one CTA reports bad pool data
+    __syncthreads();
+
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int64_t n_words = (n + 31) >> 5;
-    const uint32_t lt_mask = (1u << lane) - 1u;
 
-    for (;;) {
-        __syncthreads();                    // sh_d ready / previous tile done with sh_tile, sh_prefix
-        if (threadIdx.x == 0) sh_tile = atomicAdd(ticket, 1u) - ticket_base;
-        __syncthreads();
-        const unsigned tile = sh_tile;
-        if (tile >= n_tiles) break;
-
-        // ---- risk test: lane l ends up holding flag word l of the warp's 1024 requests ----
-        const int64_t first = ((int64_t)tile * kRiskWarps + warp) * kRiskChunk;
-        uint32_t my_word = 0;
+    for (int64_t chunk = (int64_t)blockIdx.x * kRiskWarps + warp; chunk < n_chunks;
+         chunk += (int64_t)gridDim.x * kRiskWarps) {
+        const int64_t first = chunk * kRiskChunk;
+        uint32_t my_word = 0;               // lane l ends up holding word l of the chunk
 #pragma unroll 1
         for (int w0 = 0; w0 < 32; w0 += kRiskUnroll) {
             int g[kRiskUnroll], gen[kRiskUnroll], tot[kRiskUnroll];
@@ -110,96 +84,87 @@ risk_scan_kernel(const int32_t *__restrict__ assigned, const int32_t *__restrict
                 if (lane == w0 + u) my_word = word;
             }
         }
-        const int64_t wi = (first >> 5) + lane;
-        if (wi < n_words) __stcs(flag_bits + wi, my_word);
+        const int64_t wi = chunk * 32 + lane;
+        if (wi < n_words) flag_bits[wi] = my_word;
+        const unsigned total = __reduce_add_sync(0xFFFFFFFFu, (unsigned)__popc(my_word));
+        if (lane == 0) {
+            chunk_counts[chunk] = total;
+            if (total) atomicAdd(group_totals + (chunk >> kGroupShift), total);
+        }
+    }
+    if (bad) atomicOr(status, bad);
+}
 
-        // flags in earlier words of this warp's chunk, and the chunk's total
-        const unsigned c = __popc(my_word);
+__global__ void __launch_bounds__(kRiskThreads)
+scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_words,
+                          const unsigned *__restrict__ chunk_counts,
+                          const unsigned *__restrict__ group_totals, unsigned *__restrict__ next_group_totals,
+                          int64_t n_clear, int64_t n_chunks, int64_t chunks_per_warp,
+                          int32_t *__restrict__ cand_idx, int64_t cand_capacity,
+                          int64_t *__restrict__ cand_count, unsigned *__restrict__ status)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t gwarp = (int64_t)blockIdx.x * kRiskWarps + (threadIdx.x >> 5);
+    const uint32_t lt_mask = (1u << lane) - 1u;
+
+    // clear what an earlier call left in the other parity's group totals, for the next call
+    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n_clear;
+         k += (int64_t)gridDim.x * blockDim.x)
+        next_group_totals[k] = 0u;
+
+    const int64_t c0 = gwarp * chunks_per_warp;
+    if (c0 >= n_chunks) return;
+    const int64_t c1 = min(c0 + chunks_per_warp, n_chunks);
+
+    // flags before chunk c0: whole groups, then the chunks of c0's own group
+    unsigned part = 0;
+    const int64_t g0 = c0 >> kGroupShift;
+    for (int64_t k = lane; k < g0; k += 32) part += group_totals[k];
+    for (int64_t k = (g0 << kGroupShift) + lane; k < c0; k += 32) part += chunk_counts[k];
+    int64_t base = (int64_t)__reduce_add_sync(0xFFFFFFFFu, part);
+
+    for (int64_t chunk = c0; chunk < c1; ++chunk) {
+        const int64_t wi = chunk * 32 + lane;
+        const uint32_t word = wi < n_words ? __ldcs(flag_bits + wi) : 0u;
+        const unsigned c = __popc(word);
         unsigned incl = c;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const unsigned v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
             if (lane >= off) incl += v;
         }
-        const unsigned word_off = incl - c;
-        if (lane == 31) sh_wcount[warp] = incl;
-        __syncthreads();
-
-        // ---- tile offset: publish the tile's count, look back over the tiles before it -------
-        if (warp == 0) {
-            const unsigned wc = lane < kRiskWarps ? sh_wcount[lane] : 0u;
-            unsigned winc = wc;
-#pragma unroll
-            for (int off = 1; off < kRiskWarps; off <<= 1) {
-                const unsigned v = __shfl_up_sync(0xFFFFFFFFu, winc, off);
-                if (lane >= off) winc += v;
-            }
-            const unsigned agg = __shfl_sync(0xFFFFFFFFu, winc, kRiskWarps - 1);
-            if (lane < kRiskWarps) sh_wcount[lane] = winc - wc;
-            if (lane == 0 && tile > 0) store_status(tile_status + tile, pack_status(epoch, kFlagAggregate, agg));
-            unsigned excl = 0;
-            long long look = (long long)tile - 1;      // lane l inspects tile look - l
-            unsigned spins = 0;
-            bool timed_out = false;
-            while (look >= 0) {
-                const long long idx = look - lane;
-                const unsigned long long w = idx >= 0 ? load_status(tile_status + idx)
-                                                      : pack_status(epoch, kFlagPrefix, 0u);
-                const unsigned hi = (unsigned)(w >> 32);
-                const bool ready = (hi >> 2) == epoch;
-                const unsigned ready_mask = __ballot_sync(0xFFFFFFFFu, ready);
-                const unsigned prefix_mask = __ballot_sync(0xFFFFFFFFu, ready && (hi & 3u) == kFlagPrefix);
-                // lanes up to and including the nearest tile that already knows its prefix
-                const int stop = prefix_mask ? __ffs(prefix_mask) - 1 : 31;
-                const unsigned need = stop == 31 ? 0xFFFFFFFFu : ((2u << stop) - 1u);
-                if ((ready_mask & need) == need) {
-                    excl += __reduce_add_sync(0xFFFFFFFFu, lane <= stop ? (unsigned)w : 0u);
-                    if (prefix_mask) break;
-                    look -= 32;
-                    continue;
-                }
-                if (++spins > kSpinLimit) { timed_out = true; break; }
-                __nanosleep(64);
-            }
-            if (lane == 0) {
-                if (timed_out) atomicOr(status, (unsigned)GS_DEV_TIMEOUT);
-                store_status(tile_status + tile, pack_status(epoch, kFlagPrefix, excl + agg));
-                sh_prefix = excl;
-                if (tile == n_tiles - 1) {
-                    *cand_count = (int64_t)(excl + agg);
-                    if ((int64_t)(excl + agg) > cand_capacity) atomicOr(status, (unsigned)GS_DEV_CAND_TRUNCATED);
-                }
-            }
-        }
-        __syncthreads();
-
-        // ---- candidates: ascending indices, straight from the flag words in registers --------
-        const int64_t base = (int64_t)sh_prefix + sh_wcount[warp];
+        const unsigned word_off = incl - c;                 // flags in earlier words of the chunk
         if (base < cand_capacity) {
 #pragma unroll 4
             for (int k = 0; k < 32; ++k) {
-                const uint32_t wk = __shfl_sync(0xFFFFFFFFu, my_word, k);
+                const uint32_t wk = __shfl_sync(0xFFFFFFFFu, word, k);
                 const unsigned ok = __shfl_sync(0xFFFFFFFFu, word_off, k);
                 if ((wk >> lane) & 1u) {
                     const int64_t pos = base + ok + __popc(wk & lt_mask);
-                    if (pos < cand_capacity) cand_idx[pos] = (int32_t)(first + (int64_t)k * 32 + lane);
+                    if (pos < cand_capacity)
+                        cand_idx[pos] = (int32_t)(chunk * kRiskChunk + (int64_t)k * 32 + lane);
                 }
             }
         }
+        base += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
-    if (bad) atomicOr(status, bad);
+    if (c1 == n_chunks && lane == 0) {      // the warp that owns the last chunk knows the total
+        *cand_count = base;
+        if (base > cand_capacity) atomicOr(status, (unsigned)GS_DEV_CAND_TRUNCATED);
+    }
 }
 
-// Host side of one scan: `state` holds the ticket counter, the epoch and the ticket base.
+// Host side of one scan; `epoch` (host) selects the group-total buffer of this call and
+// `dirty[b]` (host) is how many entries of buffer b may be non-zero.
 struct ScanLaunch {
-    unsigned long long *tile_status;
-    unsigned *ticket;
-    unsigned *epoch;        // host
-    unsigned *ticket_base;  // host
-    size_t max_tiles;
+    unsigned *chunk_counts;
+    unsigned *group_totals;     // two buffers of max_groups entries, both zero before the first call
+    size_t max_groups;
+    unsigned *epoch;
+    int64_t *dirty;
 };
 
-static cudaError_t enqueue_scan(const ScanLaunch &sl, int n_sm,
+static cudaError_t enqueue_scan(const ScanLaunch &sl, int n_sm, gs_ctx *timing_ctx,
                                 const int32_t *assigned, const int32_t *generated, const int32_t *pred_len,
                                 const float *elapsed, const float *slo, int64_t n,
                                 const gs_instances &inst, const gs_types &types,
@@ -207,24 +172,34 @@ static cudaError_t enqueue_scan(const ScanLaunch &sl, int n_sm,
                                 int64_t *cand_count, unsigned *status, cudaStream_t st)
 {
     if (n == 0) return cudaMemsetAsync(cand_count, 0, sizeof(int64_t), st);
-    const unsigned n_tiles = (unsigned)((n + kRiskTile - 1) / kRiskTile);
-    if (++*sl.epoch >= (1u << 30)) {
-        // epochs are about to repeat: forget every old status word
-        cudaError_t e = cudaMemsetAsync(sl.tile_status, 0, sl.max_tiles * sizeof(unsigned long long), st);
-        if (e != cudaSuccess) return e;
-        *sl.epoch = 1;
-    }
-    unsigned blocks = n_tiles;
-    const unsigned cap = (unsigned)n_sm * 8u;
+    const int64_t n_chunks = (n + kRiskChunk - 1) / kRiskChunk;
+    const int64_t n_words = (n + 31) >> 5;
+    const unsigned parity = (*sl.epoch)++ & 1u;
+    unsigned *totals = sl.group_totals + parity * sl.max_groups;
+    unsigned *next_totals = sl.group_totals + (parity ^ 1u) * sl.max_groups;
+    int64_t blocks = (n_chunks + kRiskWarps - 1) / kRiskWarps;
+    const int64_t cap = (int64_t)n_sm * 8;
     if (blocks > cap) blocks = cap;
-    risk_scan_kernel<<<blocks, kRiskThreads, 0, st>>>(
-        assigned, generated, pred_len, elapsed, slo, n, inst.type_id, inst.decode_batch, inst.n_instances,
-        types.tpot_a_ms, types.tpot_b_ms, types.n_types, flag_bits, cand_idx, cand_capacity, cand_count,
-        sl.tile_status, sl.ticket, *sl.ticket_base, *sl.epoch, n_tiles, status);
-    const cudaError_t e = cudaGetLastError();
-    // every tile takes one ticket and every CTA one more (the one that tells it to stop)
-    if (e == cudaSuccess) *sl.ticket_base += n_tiles + blocks;
-    return e;
+    cudaError_t e;
+    {
+        LaunchTimer timer(timing_ctx, GS_K_RISK_FLAGS, st);
+        risk_flags_kernel<<<(unsigned)blocks, kRiskThreads, 0, st>>>(
+            assigned, generated, pred_len, elapsed, slo, n, inst.type_id, inst.decode_batch, inst.n_instances,
+            types.tpot_a_ms, types.tpot_b_ms, types.n_types, flag_bits, sl.chunk_counts, totals, n_chunks, status);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    {
+        const int64_t warps = blocks * kRiskWarps;
+        const int64_t chunks_per_warp = (n_chunks + warps - 1) / warps;
+        LaunchTimer timer(timing_ctx, GS_K_RISK_SCATTER, st);
+        scatter_candidates_kernel<<<(unsigned)blocks, kRiskThreads, 0, st>>>(
+            flag_bits, n_words, sl.chunk_counts, totals, next_totals, sl.dirty[parity ^ 1u], n_chunks,
+            chunks_per_warp, cand_idx, cand_capacity, cand_count, status);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    sl.dirty[parity] = (n_chunks + (1 << kGroupShift) - 1) >> kGroupShift;
+    sl.dirty[parity ^ 1u] = 0;
+    return cudaSuccess;
 }
 
 cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *generated,
@@ -233,9 +208,8 @@ cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *gen
                         uint32_t *flag_bits, int32_t *cand_idx, int64_t cand_capacity,
                         int64_t *cand_count, cudaStream_t st)
 {
-    ScanLaunch sl{ctx->s.tile_status, ctx->s.ticket, &ctx->scan_epoch, &ctx->ticket_base, ctx->max_tiles};
-    LaunchTimer timer(ctx, GS_K_RISK_SCAN, st);
-    return enqueue_scan(sl, ctx->n_sm, assigned, generated, pred_len, elapsed, slo, n, inst, types,
+    ScanLaunch sl{ctx->s.chunk_counts, ctx->s.group_totals, ctx->max_groups, &ctx->scan_epoch, ctx->scan_dirty};
+    return enqueue_scan(sl, ctx->n_sm, ctx, assigned, generated, pred_len, elapsed, slo, n, inst, types,
                         flag_bits, cand_idx, cand_capacity, cand_count, ctx->s.status, st);
 }
 
@@ -243,15 +217,16 @@ cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *gen
 // gs_risk_scan_noalloc: the same scan for callers that cannot allocate device memory
 // ---------------------------------------------------------------------------------------
 
-constexpr size_t kNoAllocTiles = (GS_NOALLOC_MAX_ACTIVE + kRiskTile - 1) / kRiskTile;
+constexpr size_t kNoAllocChunks = (GS_NOALLOC_MAX_ACTIVE + kRiskChunk - 1) / kRiskChunk;
+constexpr size_t kNoAllocGroups = (kNoAllocChunks + (1u << kGroupShift) - 1) >> kGroupShift;
 
 // All scratch of the no-allocation entry point.  It lives in the library image: every GPU
-// that loads the library holds these ~16 KB until the process exits.  Zero-initialised; the
-// status words and the ticket counter keep their values between calls, which the epoch and
-// the ticket base account for.
+// that loads the library holds these 66 KB until the process exits.  Zero-initialised.  The
+// chunk counts are rewritten by every call before they are read; of the two group-total
+// buffers each call adds into one (cleared by the call before it) and clears the other.
 struct NoAllocScratch {
-    unsigned long long tile_status[kNoAllocTiles];
-    unsigned ticket;
+    unsigned chunk_counts[kNoAllocChunks];
+    unsigned group_totals[2 * kNoAllocGroups];
     unsigned status;
 };
 static __device__ __align__(256) NoAllocScratch g_noalloc_scratch;
@@ -268,7 +243,8 @@ struct NoAllocDevice {
     gs::NoAllocScratch *ptr = nullptr;
     cudaError_t err = cudaSuccess;
     bool ready = false;
-    unsigned epoch = 0, ticket_base = 0;
+    unsigned epoch = 0;
+    int64_t dirty[2] = {0, 0};
 };
 NoAllocDevice g_noalloc[kMaxDevices];
 std::mutex g_noalloc_mutex;     // guards g_noalloc
@@ -310,8 +286,8 @@ extern "C" GS_API int gs_risk_scan_noalloc(
     NoAllocScratch *sc = nd.ptr;
     int n_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1) n_sm = 148;
-    ScanLaunch sl{sc->tile_status, &sc->ticket, &nd.epoch, &nd.ticket_base, kNoAllocTiles};
-    const cudaError_t e = enqueue_scan(sl, n_sm, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms,
+    ScanLaunch sl{sc->chunk_counts, sc->group_totals, kNoAllocGroups, &nd.epoch, nd.dirty};
+    const cudaError_t e = enqueue_scan(sl, n_sm, nullptr, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms,
                                        n_active, *inst, *types, out_flag_bits, out_cand_idx, cand_capacity,
                                        out_cand_count, out_status_bits ? out_status_bits : &sc->status,
                                        (cudaStream_t)cuda_stream);

@@ -47,7 +47,7 @@ def test_noalloc_scan_equals_context_scan_on_consecutive_calls():
     big = W.make_workload(2, n_requests=16, n_active=1_500_000)
     small = W.make_workload(0, n_requests=16, n_active=1024)
     # first call: large; second: a different pool and a much smaller, ragged population, so
-    # whatever the first call left in the shared scratch (tile counts, ticket counter) would show up
+    # whatever the first call left in the shared scratch (chunk counts, group totals) would show up
     c1, s1, ctx1 = _scan_both_ways(gs, big, 1_500_000, 1_500_000)
     c2, s2, ctx2 = _scan_both_ways(gs, small, 1001, 1001)
     c3, s3, ctx3 = _scan_both_ways(gs, big, 700_001, 1000)       # truncated candidate list
