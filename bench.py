@@ -229,9 +229,23 @@ def run_gpu(args):
     count = torch.zeros(1, dtype=torch.int64, device=dev)
     stream = torch.cuda.current_stream(dev)
 
-    def step():
+    # The two halves of a step are independent (the scan reads the same instance snapshot and
+    # uses separate scratch), so the scan runs on a second stream beside the routing round: one
+    # is bound by instruction issue, the other by HBM.  --serial puts both on one stream.
+    side = None if args.serial else torch.cuda.Stream(dev)
+    fork, join = torch.cuda.Event(), torch.cuda.Event()
+
+    def step(overlap=True):
+        if side is None or not overlap:
+            gs.route_batch(*req, pool, alpha, out_idx, out_est, out_slack, None, stream=stream)
+            gs.risk_scan(*act, pool, flag_bits, cand, count, stream=stream)
+            return
+        fork.record(stream)
+        side.wait_event(fork)
+        gs.risk_scan(*act, pool, flag_bits, cand, count, stream=side)
         gs.route_batch(*req, pool, alpha, out_idx, out_est, out_slack, None, stream=stream)
-        gs.risk_scan(*act, pool, flag_bits, cand, count, stream=stream)
+        join.record(side)
+        stream.wait_event(join)
 
     def barrier():
         if dist is not None:
@@ -247,9 +261,8 @@ def run_gpu(args):
     barrier()
 
     # ---- device-resident timed region: exactly K steps ------------------------------
-    gs.timing_enable(True)
-    launches0 = gs.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = gs.launch_count()
     barrier()
     ev0.record(stream)
     for _ in range(args.steps):
@@ -258,6 +271,18 @@ def run_gpu(args):
     barrier()
     local_ms = ev0.elapsed_time(ev1)
     launches = gs.launch_count() - launches0
+
+    # ---- per-kernel durations: K more steps, one stream, every launch bracketed by events ----
+    # (kernels that share the GPU with another stream's kernel have no duration of their own,
+    # so the roofline figures come from this serial pass over the same inputs)
+    gs.timing_enable(True)
+    barrier()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(overlap=False)
+    ev1.record(stream)
+    barrier()
+    serial_ms_per_step = ev0.elapsed_time(ev1) / args.steps
     kernel_ms = {}
     for k, name in enumerate(KERNEL_NAMES):
         ms, n = gs.timing_read(k)
@@ -334,7 +359,7 @@ def run_gpu(args):
             gbs = alg_bytes[name] / (per_kernel[name]["avg_us"] * 1e-6) / 1e9
             per_kernel[name]["algorithmic_GBps"] = gbs
             per_kernel[name]["frac_of_hbm_peak"] = gbs / peak
-    route_ms = sum(kernel_ms[k][0] for k in ("prologue", "route") if k in kernel_ms) / args.steps
+    route_ms = sum(kernel_ms[k][0] for k in ("prologue", "route") if k in kernel_ms) / args.steps   # serial pass
     risk_ms = sum(kernel_ms[k][0] for k in ("risk_flags", "risk_scatter") if k in kernel_ms) / args.steps
     step_bytes = ROUTE_BYTES_PER_REQUEST * N + RISK_BYTES_PER_REQUEST * A + 4 * flagged
 
@@ -344,6 +369,7 @@ def run_gpu(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(args.config), "ema_alpha": alpha,
                    "l2": "inputs larger than L2: one step streams %.0f MB" % (step_bytes / 1e6),
+                   "streams": 1 if args.serial else 2,
                    "per_rank_seed": "config id + 1000 * rank", "sharding": "independent batches per rank, no collective"},
         "risk_scan_requests_per_s": world * A / (risk_ms * 1e-3) if risk_ms else None,
         "route_pairs_per_s": world * N * M / (route_ms * 1e-3) if route_ms else None,
@@ -351,6 +377,8 @@ def run_gpu(args):
         "step_hbm_frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "flagged_fraction": flagged / A, "device_status": status,
         "roofline": roofline, "kernels": per_kernel,
+        "kernel_timing": "serial pass of %d steps on one stream after the timed region, %.4f ms/step" % (
+            args.steps, serial_ms_per_step),
         "e2e": None if args.no_e2e else
                {"value": e2e_pairs / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
@@ -372,6 +400,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--serial", action="store_true", help="route and scan on one stream instead of two")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

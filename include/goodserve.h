@@ -29,8 +29,9 @@
  *     read as 0, a type id outside [0, n_types) as type 0, an assigned instance outside
  *     [0, n_instances) is clamped into range; a bit of the device status word records it
  *     (gs_device_status).  A NaN deadline is never met, so such a request takes the fallback.
- *   - One context serves one stream at a time; calls on one context must not overlap on the
- *     GPU (they share the context's scratch memory).
+ *   - Calls of the same kind on one context must not overlap on the GPU (they share the
+ *     context's scratch memory).  gs_route_batch / gs_advance_state on one stream and
+ *     gs_risk_scan on another may overlap each other: they use separate scratch.
  */
 #ifndef GOODSERVE_H_
 #define GOODSERVE_H_

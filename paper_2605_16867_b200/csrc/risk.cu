@@ -134,19 +134,26 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
             if (lane >= off) incl += v;
         }
         const unsigned word_off = incl - c;                 // flags in earlier words of the chunk
-        if (base < cand_capacity) {
-#pragma unroll 4
+        const unsigned total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        const int32_t idx0 = (int32_t)(chunk * kRiskChunk) + lane;      // n_active < 2^31
+        if (base + total <= cand_capacity) {
+            // whole chunk fits: 32-bit offsets from one 64-bit base, no per-element bound check
+            int32_t *out = cand_idx + base;
+#pragma unroll 8
             for (int k = 0; k < 32; ++k) {
                 const uint32_t wk = __shfl_sync(0xFFFFFFFFu, word, k);
                 const unsigned ok = __shfl_sync(0xFFFFFFFFu, word_off, k);
-                if ((wk >> lane) & 1u) {
-                    const int64_t pos = base + ok + __popc(wk & lt_mask);
-                    if (pos < cand_capacity)
-                        cand_idx[pos] = (int32_t)(chunk * kRiskChunk + (int64_t)k * 32 + lane);
-                }
+                if ((wk >> lane) & 1u) out[ok + __popc(wk & lt_mask)] = idx0 + 32 * k;
+            }
+        } else if (base < cand_capacity) {
+            for (int k = 0; k < 32; ++k) {
+                const uint32_t wk = __shfl_sync(0xFFFFFFFFu, word, k);
+                const unsigned ok = __shfl_sync(0xFFFFFFFFu, word_off, k);
+                const int64_t pos = base + ok + __popc(wk & lt_mask);
+                if (((wk >> lane) & 1u) && pos < cand_capacity) cand_idx[pos] = idx0 + 32 * k;
             }
         }
-        base += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        base += total;
     }
     if (c1 == n_chunks && lane == 0) {      // the warp that owns the last chunk knows the total
         *cand_count = base;
