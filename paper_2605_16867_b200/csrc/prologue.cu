@@ -48,6 +48,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 Scratch s)
 {
     __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];
+    __shared__ unsigned long long sh_key2[2][GS_MAX_INSTANCES];      // exchange buffers of the sort
     __shared__ float sh_q[GS_MAX_INSTANCES], sh_d[GS_MAX_INSTANCES];       // by instance index
     __shared__ float sh_row_d[kMaxPaddedRows];                             // row d_lo as float (untagged)
     __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES], sh_row0[GS_MAX_TYPES + 1];
@@ -125,27 +126,34 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     }
 
     // ---- 3. sort rows by (type order, d descending, index ascending) ---------------------
+    // bitonic network, one key per thread: partners closer than a warp exchange by shuffle,
+    // farther ones through shared memory (two buffers, so one barrier per exchange)
     int n_sort = 32;
     while (n_sort < M) n_sort <<= 1;
+    unsigned long long key = ~0ull;
+    if (g < M)
+        key = ((unsigned long long)sh_rank[t] << 48) | ((unsigned long long)(~orderable(d)) << 16) |
+              (unsigned long long)g;
     {
-        unsigned long long key = ~0ull;
-        if (g < M)
-            key = ((unsigned long long)sh_rank[t] << 48) | ((unsigned long long)(~orderable(d)) << 16) |
-                  (unsigned long long)g;
-        sh_key[g] = key;
-    }
-    __syncthreads();
-    for (int k = 2; k <= n_sort; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            const int partner = g ^ j;
-            if (g < n_sort && partner > g) {
-                const unsigned long long a = sh_key[g], b = sh_key[partner];
-                const bool ascending = (g & k) == 0;
-                if ((a > b) == ascending) { sh_key[g] = b; sh_key[partner] = a; }
+        int buf = 0;
+        for (int k = 2; k <= n_sort; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                unsigned long long other;
+                if (j >= 32) {
+                    sh_key2[buf][g] = key;
+                    __syncthreads();
+                    other = sh_key2[buf][g ^ j];
+                    buf ^= 1;
+                } else {
+                    other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
+                }
+                const bool keep_min = ((g & k) == 0) == ((g & j) == 0);
+                key = (keep_min == (other < key)) ? other : key;
             }
-            __syncthreads();
         }
     }
+    sh_key[g] = key;
+    __syncthreads();
 
     // ---- 4. row bounds, per-type minimum of q -------------------------------------------------
     const int n_act = sh_n_act;
