@@ -159,7 +159,7 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
     struct { void **p; size_t bytes; } allocs[] = {
         {(void **)&s.rows, Mx * sizeof(gs::Row)},
         {(void **)&s.row_bounds, gs::kMaxPaddedRows * sizeof(uint2)},
-        {(void **)&s.start_table, GS_MAX_TYPES * gs::kStartSlots * sizeof(unsigned short)},
+        {(void **)&s.start_table, (size_t)GS_MAX_TYPES * gs::kStartBuckets * gs::kStartSlots},
         {(void **)&s.headers, GS_MAX_TYPES * sizeof(gs::TypeHeader)},
         {(void **)&s.table_info, 64},
         {(void **)&s.d_by_g, Mx * sizeof(float)},
@@ -174,7 +174,10 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
         if (e == cudaSuccess) e = cudaMemset(*a.p, 0, a.bytes);
         if (e != cudaSuccess) { gs_destroy(ctx); return GS_ERR_CUDA; }
     }
-    if (gs::configure_route(ctx) != cudaSuccess) { gs_destroy(ctx); return GS_ERR_CUDA; }
+    if (gs::configure_route(ctx) != cudaSuccess || gs::configure_prologue() != cudaSuccess) {
+        gs_destroy(ctx);
+        return GS_ERR_CUDA;
+    }
     *out = ctx;
     return GS_OK;
 }
@@ -255,7 +258,7 @@ GS_API int gs_route_batch(gs_ctx *ctx, const int32_t *prompt_len, const int32_t 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, inst->n_instances,
+    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, types->n_types,
                          out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier,
                          (flags & GS_ROUTE_ACCUMULATE) != 0, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);

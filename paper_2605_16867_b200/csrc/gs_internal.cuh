@@ -21,8 +21,9 @@ struct __align__(16) Row {
 // grouped by GPU type and, inside a type, kept in preference order (d descending, index
 // ascending); each type's rows are padded to a multiple of 16.
 //   row_bounds[i]   = {bits of q_lo, bits of d_lo | instance index}   (one row)
-//   start_table[t * kStartSlots + s] = first row (a multiple of 8) of type t worth looking at
-//                     when the largest d that can still meet the deadline falls in slot s
+//   start_table[(t * kStartBuckets + b) * kStartSlots + s] = first group of 8 rows of type t
+//                     worth looking at when L_out falls in bucket b and the largest d that can
+//                     still meet the deadline falls in slot s
 // Storage slot of padded row i.  Eight consecutive rows (64 bytes) are read together as four
 // 16-byte chunks; which chunk sits where is XOR-swizzled with the group number so that lanes
 // reading different groups in the same instruction spread over all shared-memory banks.
@@ -33,7 +34,8 @@ __host__ __device__ __forceinline__ int row_slot(int i) {
 
 constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low bits of a d word
 constexpr int kMaxPaddedRows = GS_MAX_INSTANCES + GS_MAX_TYPES * 16;
-constexpr int kStartSlots = 128;
+constexpr int kStartSlots = 64;
+constexpr int kStartBuckets = 32;         // two per octave of L_out; the last one is open-ended
 
 // One GPU type's entry: bound over all its rows, where its rows are, start-table geometry.
 struct __align__(16) TypeHeader {
@@ -51,7 +53,7 @@ constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 struct Scratch {
     Row *rows;                // [max_instances] exact coefficients, caller order
     uint2 *row_bounds;        // [kMaxPaddedRows]
-    unsigned short *start_table;  // [GS_MAX_TYPES * kStartSlots]
+    unsigned char *start_table;   // [GS_MAX_TYPES * kStartBuckets * kStartSlots]
     TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)
     int *table_info;          // {padded rows, unsafe, n_instances, n_active_types}
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
@@ -69,7 +71,7 @@ struct gs_ctx {
     int max_instances;
     int max_types;
     int n_sm;
-    int route_ctas_per_sm;
+    int route_ctas_per_sm[GS_MAX_TYPES + 1];   // by number of types (sets the shared-memory size)
     gs::Scratch s;
     size_t max_chunks, max_groups;   // capacity of the risk scan's count arrays
     unsigned scan_epoch;             // its parity selects the group-total buffer of the next scan
@@ -102,10 +104,11 @@ struct LaunchTimer {
 cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_types &types,
                             float ema_alpha, cudaStream_t st);
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
-                         const float *slo_ms, int64_t n, int n_instances,
+                         const float *slo_ms, int64_t n, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, cudaStream_t st);
 cudaError_t configure_route(gs_ctx *ctx);
+cudaError_t configure_prologue();
 cudaError_t launch_advance(gs_ctx *ctx, const gs_instances_mut &inst, cudaStream_t st);
 cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *generated,
                         const int32_t *pred_len, const float *elapsed, const float *slo,

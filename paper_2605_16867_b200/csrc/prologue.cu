@@ -1,4 +1,4 @@
-// Per-round instance prologue (one CTA):
+// Per-round instance prologue, one CTA per GPU type:
 //   1. the coefficients of Eq. 2 for every instance and the EMA step of Algorithm 1
 //      (rows[g] = {q_g, p_g, d_g, free KV}, exact, in caller order);
 //   2. the search tables of the route kernel.  Instances are grouped by GPU type (types
@@ -6,8 +6,11 @@
 //      (d descending, index ascending).  Per type the tables hold
 //        - a lower bound (q_lo, d_lo) for every row, tagged with the instance index,
 //        - a header with the bound over the whole type, and
-//        - a start table: for a threshold on d, the first group of 8 rows that can matter.
+//        - a start table: for a range of L_out and a threshold on d, the first group of 8
+//          rows that can hold a feasible row at all.
 //      A type's rows are padded to a multiple of 16 with entries that never pass a test.
+// Every CTA derives all coefficients and the order of the types (cheap, and it keeps the
+// CTAs independent); the CTA at order position r then builds the tables of that type.
 //
 // Bounds: q_lo <= q (1 - 2^-19), d_lo <= d (1 - 2^-19), p_lo = p (1 - 2^-19).  With all
 // coefficients non-negative and each fused step of T = fma(d, y, fma(p, x, q)) rounding by at
@@ -15,9 +18,19 @@
 // implies  T(r,g) > D  for every row the bound covers.  The low bits of a row's d word
 // carry the instance index; the bound is lowered by one unit of the remaining mantissa
 // first, so it stays a lower bound.
+//
+// Start table.  Write R for fma(-p_lo, x, D), q0 for the type's least q_lo, y for L_out and
+// z = (R - q0) / y.  A row can pass its bound test only if  q_lo - q0 <= (z - d_lo) * y.
+// For all requests with y <= y_hi and z < z_edge the right side is at most
+// max(z_edge - d_lo, 0) * y_hi, so a row whose q_lo - q0 exceeds that is out for all of them,
+// and the search may begin at the first row that is not out.  The table is indexed by the
+// bucket of y (upper edge y_hi) and the slot of z (upper edge z_edge, widened by two slots
+// against the rounding of the kernel's own slot computation).
 #include "gs_internal.cuh"
 
 namespace gs {
+
+constexpr int kPrologueThreads = 256;
 
 __device__ __forceinline__ int clamp_count(int v, unsigned &bad) {
     if (v < 0) { bad |= GS_DEV_BAD_VALUE; return 0; }
@@ -39,7 +52,7 @@ __device__ __forceinline__ unsigned lower_bound_bits(float v) {
     return b >= (kRowTagMask + 1u) ? b - (kRowTagMask + 1u) : 0u;
 }
 
-__global__ void __launch_bounds__(GS_MAX_INSTANCES)
+__global__ void __launch_bounds__(kPrologueThreads)
 prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__ queued,
                 const int32_t *__restrict__ batch, const int32_t *__restrict__ free_kv,
                 const float *__restrict__ q_ema, int M,
@@ -47,29 +60,26 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 const float *__restrict__ b_type, int n_types, float alpha,
                 Scratch s)
 {
-    __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];
-    __shared__ unsigned long long sh_key2[2][GS_MAX_INSTANCES];      // exchange buffers of the sort
+    __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];                // my type's rows, sorted
     __shared__ float sh_q[GS_MAX_INSTANCES], sh_d[GS_MAX_INSTANCES];       // by instance index
-    __shared__ float sh_row_d[kMaxPaddedRows];                             // row d_lo as float (untagged)
-    __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES], sh_row0[GS_MAX_TYPES + 1];
-    __shared__ unsigned sh_dmax[GS_MAX_TYPES], sh_qmin[GS_MAX_TYPES];
-    __shared__ int sh_base[GS_MAX_TYPES + 1];                              // padded row offset per type
-    __shared__ float sh_inv_w[GS_MAX_TYPES], sh_d0[GS_MAX_TYPES];
-    __shared__ int sh_unsafe, sh_n_act;
+    __shared__ unsigned char sh_t[GS_MAX_INSTANCES];
+    __shared__ float sh_rq[GS_MAX_INSTANCES], sh_rd[GS_MAX_INSTANCES];     // my rows: q_lo, d_lo (untagged)
+    __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES];
+    __shared__ unsigned sh_dmax[GS_MAX_TYPES];
+    __shared__ unsigned sh_qmin;
+    __shared__ int sh_unsafe, sh_fill;
 
-    const int g = threadIdx.x;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    const bool writer = blockIdx.x == 0;       // one CTA writes what does not depend on the type
     unsigned bad = 0;
-    float d = 0.f;
-    int t = 0;
-    if (g < GS_MAX_TYPES) { sh_cnt[g] = 0; sh_dmax[g] = 0u; sh_qmin[g] = 0xFFFFFFFFu; }
-    if (g == 0) sh_unsafe = 0;
-    // every table entry starts as padding
-    for (int i = g; i < kMaxPaddedRows; i += blockDim.x) s.row_bounds[i] = make_uint2(kPadQ, 0u);
+    if (tid < GS_MAX_TYPES) { sh_cnt[tid] = 0; sh_dmax[tid] = 0u; }
+    if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; }
     __syncthreads();
 
-    // ---- 1. coefficients ----------------------------------------------------------------
-    if (g < M) {
-        t = type_id[g];
+    // ---- 1. coefficients of every instance ---------------------------------------------------
+    for (int g = tid; g < M; g += kPrologueThreads) {
+        int t = type_id[g];
         if (t < 0 || t >= n_types) { bad |= GS_DEV_BAD_TYPE; t = 0; }
         const float Qtok = __int2float_rn(clamp_count(queued[g], bad));
         const float B = __int2float_rn(clamp_count(batch[g], bad));
@@ -77,15 +87,17 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         if (!(qe >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; qe = 0.0f; }
         const int kv = clamp_count(free_kv[g], bad);
         const float p = p_type[t];
-        d = __fmaf_rn(b_type[t], B, a_type[t]);             // loaded per-token decode latency
-        const float w = __fmul_rn(Qtok, p);                 // time to drain the queued prefill
+        const float d = __fmaf_rn(b_type[t], B, a_type[t]);     // loaded per-token decode latency
+        const float w = __fmul_rn(Qtok, p);                     // time to drain the queued prefill
         const float keep = __fmul_rn(__fsub_rn(1.0f, alpha), qe);
-        const float q = __fmaf_rn(alpha, w, keep);          // EMA step
-        sh_q[g] = q; sh_d[g] = d;
-        Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
-        s.rows[g] = row;
-        s.d_by_g[g] = d;
-        s.q_by_g[g] = q;
+        const float q = __fmaf_rn(alpha, w, keep);              // EMA step
+        sh_q[g] = q; sh_d[g] = d; sh_t[g] = (unsigned char)t;
+        if (writer) {
+            Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
+            s.rows[g] = row;
+            s.d_by_g[g] = d;
+            s.q_by_g[g] = q;
+        }
         // the bounds of the search tables need finite, non-negative coefficients
         const float big = 3.0e38f;
         if (!(q >= 0.f && q < big && p >= 0.f && p < big && d >= 0.f && d < big)) atomicOr(&sh_unsafe, 1);
@@ -94,149 +106,161 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     }
     __syncthreads();
 
-    // ---- 2. order of the types (largest d first; ties: smaller type id), row offsets ------
-    if (g < GS_MAX_TYPES) {
+    // ---- 2. order of the types (largest d first; ties: smaller type id) ----------------------
+    if (tid < GS_MAX_TYPES) {
         int rank = GS_MAX_TYPES;           // unused types sort last
-        if (sh_cnt[g] > 0) {
+        if (sh_cnt[tid] > 0) {
             rank = 0;
             for (int o = 0; o < GS_MAX_TYPES; ++o)
-                if (sh_cnt[o] > 0 && (sh_dmax[o] > sh_dmax[g] || (sh_dmax[o] == sh_dmax[g] && o < g))) ++rank;
+                if (sh_cnt[o] > 0 && (sh_dmax[o] > sh_dmax[tid] || (sh_dmax[o] == sh_dmax[tid] && o < tid))) ++rank;
         }
-        sh_rank[g] = rank;
+        sh_rank[tid] = rank;
     }
     __syncthreads();
-    if (g < GS_MAX_TYPES) {
-        // thread g handles the type at order position g
-        int n_act = 0, row0 = 0, base = 0, my_n = -1;
-        for (int o = 0; o < GS_MAX_TYPES; ++o) {
-            const int r = sh_rank[o], n = sh_cnt[o];
-            if (n == 0) continue;
-            ++n_act;
-            if (r == g) my_n = n;
-            if (r < g) { row0 += n; base += (n + 15) & ~15; }
-        }
-        if (my_n >= 0) {
-            sh_row0[g] = row0; sh_base[g] = base;
-            if (g == n_act - 1) {
-                sh_row0[n_act] = row0 + my_n;
-                sh_base[n_act] = base + ((my_n + 15) & ~15);
-                sh_n_act = n_act;
-            }
-        }
+    // the type this CTA builds, the padded rows before it, the number of types in use
+    int my_type = -1, base = 0, n_act = 0, padded_total = 0;
+    for (int o = 0; o < GS_MAX_TYPES; ++o) {
+        const int r = sh_rank[o], n = sh_cnt[o];
+        if (n == 0) continue;
+        ++n_act;
+        padded_total += (n + 15) & ~15;
+        if (r == (int)blockIdx.x) my_type = o;
+        if (r < (int)blockIdx.x) base += (n + 15) & ~15;
     }
+    if (writer && tid == 0) {
+        s.table_info[0] = padded_total;
+        s.table_info[1] = sh_unsafe;
+        s.table_info[2] = M;
+        s.table_info[3] = n_act;
+        if (sh_unsafe) atomicOr(s.status, (unsigned)GS_DEV_BAD_VALUE);
+    }
+    if (writer && bad) atomicOr(s.status, bad);
+    if (my_type < 0) return;
+    const int tr = blockIdx.x;
+    const int n_t = sh_cnt[my_type];
+    const int n_padded = (n_t + 15) & ~15;
 
-    // ---- 3. sort rows by (type order, d descending, index ascending) ---------------------
-    // bitonic network, one key per thread: partners closer than a warp exchange by shuffle,
-    // farther ones through shared memory (two buffers, so one barrier per exchange)
+    // ---- 3. collect this type's rows and sort them by (d descending, index ascending) --------
     int n_sort = 32;
-    while (n_sort < M) n_sort <<= 1;
-    unsigned long long key = ~0ull;
-    if (g < M)
-        key = ((unsigned long long)sh_rank[t] << 48) | ((unsigned long long)(~orderable(d)) << 16) |
-              (unsigned long long)g;
-    {
-        int buf = 0;
-        for (int k = 2; k <= n_sort; k <<= 1) {
-            for (int j = k >> 1; j > 0; j >>= 1) {
-                unsigned long long other;
-                if (j >= 32) {
-                    sh_key2[buf][g] = key;
-                    __syncthreads();
-                    other = sh_key2[buf][g ^ j];
-                    buf ^= 1;
-                } else {
-                    other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
+    while (n_sort < n_t) n_sort <<= 1;
+    for (int g = tid; g < M; g += kPrologueThreads)
+        if (sh_t[g] == my_type)
+            sh_key[atomicAdd(&sh_fill, 1)] = ((unsigned long long)(~orderable(sh_d[g])) << 16) | (unsigned)g;
+    for (int k = n_t + tid; k < n_sort; k += kPrologueThreads) sh_key[k] = ~0ull;
+    __syncthreads();
+    for (int k = 2; k <= n_sort; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < n_sort; i += kPrologueThreads) {
+                const int partner = i ^ j;
+                if (partner > i) {
+                    const unsigned long long a = sh_key[i], b = sh_key[partner];
+                    if ((a > b) == ((i & k) == 0)) { sh_key[i] = b; sh_key[partner] = a; }
                 }
-                const bool keep_min = ((g & k) == 0) == ((g & j) == 0);
-                key = (keep_min == (other < key)) ? other : key;
             }
+            __syncthreads();
         }
     }
-    sh_key[g] = key;
-    __syncthreads();
 
-    // ---- 4. row bounds, per-type minimum of q -------------------------------------------------
-    const int n_act = sh_n_act;
-    if (g < M) {
-        const unsigned long long key = sh_key[g];
-        const int inst = (int)(key & 0xFFFFull);
-        const int tr = (int)(key >> 48);
-        const int k = g - sh_row0[tr];
-        const int base = sh_base[tr];
-        const float rq = sh_q[inst];
-        const unsigned d_bits = lower_bound_bits(sh_d[inst]);
-        s.row_bounds[row_slot(base + k)] = make_uint2(lower_bound_bits(rq), d_bits | (unsigned)inst);
-        sh_row_d[base + k] = __uint_as_float(d_bits);
-        // one shared-memory atomic per run of equal types inside the warp
-        const unsigned peers = __match_any_sync(__activemask(), tr);
-        const unsigned qmin = __reduce_min_sync(peers, orderable(rq));
-        if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicMin(&sh_qmin[tr], qmin);
+    // ---- 4. row bounds, least q of the type ---------------------------------------------------
+    unsigned my_qmin = 0xFFFFFFFFu;
+    for (int k = tid; k < n_padded; k += kPrologueThreads) {
+        uint2 entry = make_uint2(kPadQ, 0u);
+        if (k < n_t) {
+            const int inst = (int)(sh_key[k] & 0xFFFFull);
+            const unsigned q_bits = lower_bound_bits(sh_q[inst]), d_bits = lower_bound_bits(sh_d[inst]);
+            entry = make_uint2(q_bits, d_bits | (unsigned)inst);
+            sh_rq[k] = __uint_as_float(q_bits);
+            sh_rd[k] = __uint_as_float(d_bits);
+            my_qmin = min(my_qmin, q_bits);             // non-negative floats order like their bits
+        }
+        s.row_bounds[row_slot(base + k)] = entry;
     }
+    my_qmin = __reduce_min_sync(0xFFFFFFFFu, my_qmin);
+    if (lane == 0) atomicMin(&sh_qmin, my_qmin);
     __syncthreads();
 
-    // ---- 5. headers --------------------------------------------------------------------------
-    if (g < n_act) {
-        const int tr = g;
-        const int n_t = sh_row0[tr + 1] - sh_row0[tr];
-        const int base = sh_base[tr];
-        const int first_inst = (int)(sh_key[sh_row0[tr]] & 0xFFFFull);
-        const unsigned qo = sh_qmin[tr];                    // undo the monotone map
-        const float qmin = __uint_as_float((qo & 0x80000000u) ? (qo & 0x7FFFFFFFu) : ~qo);
-        // start table geometry: kStartSlots slots between the least and the largest row bound of d
-        const float d_hi = sh_row_d[base], d_low = sh_row_d[base + n_t - 1];
-        float inv_w = 0.f;
-        if (n_t > 16 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f))
-            inv_w = (float)kStartSlots / (d_hi - d_low);
-        sh_inv_w[tr] = inv_w; sh_d0[tr] = d_low;
+    // ---- 5. header ----------------------------------------------------------------------------
+    const float q0 = __uint_as_float(sh_qmin);
+    const float d_hi = sh_rd[0], d_low = sh_rd[n_t - 1];
+    float inv_w = 0.f;              // slots per unit of d; 0 = no start table (search from row 0)
+    if (n_t > 16 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f)) inv_w = (float)kStartSlots / (d_hi - d_low);
+    if (tid == 0) {
+        const int first_inst = (int)(sh_key[0] & 0xFFFFull);
         TypeHeader h;
-        h.p_lo = __fmul_rn(s.rows[first_inst].p, kShrink);   // written in step 1 by this CTA
-        h.q_lo = __uint_as_float(lower_bound_bits(qmin));
+        h.p_lo = __fmul_rn(p_type[my_type], kShrink);
+        h.q_lo = q0;
         h.d_lo = d_low;
         h.d_max = sh_d[first_inst];
         h.base = base;
-        h.n_padded = (n_t + 15) & ~15;
+        h.n_padded = n_padded;
         h.inv_w = inv_w;
         h.d0 = d_low;
         s.headers[tr] = h;
     }
-    __syncthreads();
 
-    // ---- 6. start tables: slot -> first row (multiple of 8) not certainly above the slot -------
-    for (int e = g; e < n_act * kStartSlots; e += blockDim.x) {
-        const int tr = e / kStartSlots, slot = e % kStartSlots;
-        {
-            int start_row = 0;
-            const float inv_w = sh_inv_w[tr];
-            if (inv_w > 0.f) {
-                // two slots of margin absorb the rounding of the kernel's slot computation
-                const float edge = sh_d0[tr] + (float)(slot + 2) / inv_w;
-                const int b0 = sh_base[tr];
-                int lo = 0, hi = sh_row0[tr + 1] - sh_row0[tr];     // rows [0, lo) have d_lo > edge
+    // ---- 6. start table -------------------------------------------------------------------------
+    // For bucket b put  H_k = (q_lo_k - q0) + y_hi d_lo_k.  A row can pass only if
+    // H_k <= y_hi z_edge (see the header comment; rows with d_lo above z_edge fail that too).
+    // With P_k the running minimum of H over rows 0..k, the first row that can pass is the first
+    // k with P_k <= y_hi z_edge: a binary search per slot.  Eight buckets are done at a time,
+    // one warp each for the running minima, then one (bucket, slot) cell per thread.
+    if (inv_w > 0.f) {
+        extern __shared__ float sh_pm[];                    // [8][n_t] running minima
+        const float w_slot = 1.0f / inv_w;
+        for (int b0 = 0; b0 < kStartBuckets; b0 += kPrologueThreads / 32) {
+            {
+                const int b = b0 + warp;
+                // bucket b holds y in [2^e (1 + m/2), 2^e (1 + (m+1)/2)),  e = b >> 1, m = b & 1;
+                // the last bucket has no upper edge: there only d_lo <= z_edge can be required
+                const bool open_ended = b == kStartBuckets - 1;
+                const float y_hi = ldexpf(1.0f + 0.5f * (float)((b & 1) + 1), b >> 1) * 1.00002f;
+                float carry = 3.4e38f;
+                for (int k0 = 0; k0 < n_t; k0 += 32) {
+                    const int k = k0 + lane;
+                    float h = 3.4e38f;
+                    if (k < n_t) h = open_ended ? sh_rd[k] : __fmaf_rn(y_hi, sh_rd[k], sh_rq[k] - q0);
+#pragma unroll
+                    for (int off = 1; off < 32; off <<= 1) h = fminf(h, __shfl_up_sync(0xFFFFFFFFu, h, off) + (lane >= off ? 0.f : 3.4e38f));
+                    h = fminf(h, carry);
+                    if (k < n_t) sh_pm[warp * n_t + k] = h;
+                    carry = __shfl_sync(0xFFFFFFFFu, h, 31);
+                }
+            }
+            __syncthreads();
+            for (int c = tid; c < (kPrologueThreads / 32) * kStartSlots; c += kPrologueThreads) {
+                const int bw = c / kStartSlots, slot = c % kStartSlots, b = b0 + bw;
+                const bool open_ended = b == kStartBuckets - 1;
+                const float y_hi = ldexpf(1.0f + 0.5f * (float)((b & 1) + 1), b >> 1) * 1.00002f;
+                const float z_edge = d_low + (float)(slot + 2) * w_slot;
+                const float limit = (open_ended ? z_edge : y_hi * z_edge) * 1.00002f;
+                const float *pm = sh_pm + bw * n_t;
+                int lo = 0, hi = n_t;                       // rows [0, lo) cannot pass
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;
-                    if (sh_row_d[b0 + mid] > edge) lo = mid + 1; else hi = mid;
+                    if (pm[mid] > limit) lo = mid + 1; else hi = mid;
                 }
-                start_row = lo & ~7;
+                // the top slot also takes every z beyond the table: nothing can be ruled out there
+                if (slot == kStartSlots - 1) lo = 0;
+                s.start_table[(tr * kStartBuckets + b) * kStartSlots + slot] = (unsigned char)(lo >> 3);
             }
-            s.start_table[tr * kStartSlots + slot] = (unsigned short)start_row;
+            __syncthreads();
         }
     }
+}
 
-    if (g == 0) {
-        s.table_info[0] = sh_base[n_act];      // padded rows in use
-        s.table_info[1] = sh_unsafe;
-        s.table_info[2] = M;
-        s.table_info[3] = n_act;
-    }
-    if (bad) atomicOr(s.status, bad);
-    if (g == 0 && sh_unsafe) atomicOr(s.status, (unsigned)GS_DEV_BAD_VALUE);
+size_t prologue_dynamic_smem() { return (size_t)(kPrologueThreads / 32) * GS_MAX_INSTANCES * sizeof(float); }
+
+cudaError_t configure_prologue()
+{
+    return cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)prologue_dynamic_smem());
 }
 
 cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_types &types,
                             float ema_alpha, cudaStream_t st)
 {
     LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
-    prologue_kernel<<<1, GS_MAX_INSTANCES, 0, st>>>(
+    prologue_kernel<<<GS_MAX_TYPES, kPrologueThreads, prologue_dynamic_smem(), st>>>(
         inst.type_id, inst.queued_prefill_tokens, inst.decode_batch, inst.free_kv_tokens,
         inst.q_ema_ms, inst.n_instances, types.prefill_ms_per_tok, types.tpot_a_ms,
         types.tpot_b_ms, types.n_types, ema_alpha, ctx->s);

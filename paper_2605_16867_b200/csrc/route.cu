@@ -7,8 +7,8 @@
 //      shared-memory address for all lanes: a broadcast); types that cannot meet the deadline
 //      are dropped;
 //   2. for each surviving type (largest d first, and only while it can still beat the best d
-//      found so far) a start table turns the largest d that could still meet the deadline
-//      into the first row worth looking at; from there the rows' own lower bounds are tested
+//      found so far) a start table turns L_out and the largest d that could still meet the
+//      deadline into the first row worth looking at; from there the rows' own lower bounds are tested
 //      eight at a time, and the first row that passes is scored exactly as the definition
 //      says, T = fma(d, y, fma(p, x, q)), and checked against the deadline and the
 //      instance's free KV.
@@ -64,7 +64,7 @@ __device__ __forceinline__ void accumulate_choice(unsigned long long *hist, int 
 struct Tables {
     const TypeHeader *headers;
     const uint2 *row_bounds;
-    const unsigned short *start_table;
+    const unsigned char *start_table;
     const Row *rows;
     int n_types;
 };
@@ -102,6 +102,8 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
     int g_best = -1;
     float d_best = -1.0f, T_best = 0.f;
     const float ry = __frcp_rn(y);
+    // bucket of L_out: exponent and top mantissa bit of y (y >= 1 here)
+    const int ybucket = min((int)(__float_as_uint(y) >> 22) - 254, kStartBuckets - 1);
     // 2. search them, largest d first
     while (alive) {
         const int t = __ffs(alive) - 1;
@@ -116,7 +118,7 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
             // largest d that can still meet the deadline -> slot -> first row worth a look
             const float z = (R - h.y) * ry;
             const float sf = fminf(fmaxf((z - __int_as_float(geo.w)) * inv_w, 0.f), (float)(kStartSlots - 1));
-            k = tb.start_table[t * kStartSlots + __float2int_rd(sf)];
+            k = 8 * tb.start_table[(t * kStartBuckets + ybucket) * kStartSlots + __float2int_rd(sf)];
         }
         const int k_end = geo.x + geo.y;
         k += geo.x;                                         // padded row index, a multiple of 8
@@ -163,9 +165,9 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
 template <bool kAccumulate>
 __global__ void __launch_bounds__(kRouteThreads, 4)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
-             const float *__restrict__ slo_ms, int64_t n,
+             const float *__restrict__ slo_ms, int64_t n, int n_types_alloc,
              const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
-             const unsigned short *__restrict__ g_start_table,
+             const unsigned char *__restrict__ g_start_table,
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
              int32_t *__restrict__ out_idx, float *__restrict__ out_est,
              float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
@@ -179,12 +181,13 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     Row *sh_rows = reinterpret_cast<Row *>(smem);
     TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
     uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
-    unsigned short *sh_start = reinterpret_cast<unsigned short *>(sh_row_bounds + kMaxPaddedRows);
-    unsigned long long *hist = reinterpret_cast<unsigned long long *>(sh_start + GS_MAX_TYPES * kStartSlots);
+    unsigned char *sh_start = reinterpret_cast<unsigned char *>(sh_row_bounds + kMaxPaddedRows);
+    unsigned long long *hist = reinterpret_cast<unsigned long long *>(sh_start + n_types_alloc * (kStartBuckets * kStartSlots));
 
     for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[k] = g_rows[k];
     for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
-    for (int k = threadIdx.x; k < n_act * kStartSlots; k += blockDim.x) sh_start[k] = g_start_table[k];
+    for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
+        reinterpret_cast<uint4 *>(sh_start)[k] = reinterpret_cast<const uint4 *>(g_start_table)[k];
     if (threadIdx.x < n_act) sh_headers[threadIdx.x] = g_headers[threadIdx.x];
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
@@ -319,48 +322,52 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     }
 }
 
-constexpr size_t kRouteSmemBase = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
-                                  (size_t)kMaxPaddedRows * sizeof(uint2) +
-                                  (size_t)GS_MAX_TYPES * kStartSlots * sizeof(unsigned short);
+constexpr size_t kRouteSmemFixed = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
+                                   (size_t)kMaxPaddedRows * sizeof(uint2);
+constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
 
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
-                         const float *slo_ms, int64_t n, int M,
+                         const float *slo_ms, int64_t n, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, cudaStream_t st)
 {
-    (void)M;
     if (n == 0) return cudaSuccess;
-    const size_t smem = kRouteSmemBase + (accumulate ? kRouteSmemHist : 0);
+    const size_t smem = kRouteSmemFixed + kRouteSmemPerType * n_types + (accumulate ? kRouteSmemHist : 0);
     int64_t blocks = (n + kRouteTile - 1) / kRouteTile;
-    const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm;
+    const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm[n_types];
     if (blocks > cap) blocks = cap;
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     if (accumulate)
         route_kernel<true><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.row_bounds,
+            prompt_len, pred_decode_len, slo_ms, n, n_types, ctx->s.rows, ctx->s.row_bounds,
             ctx->s.start_table, ctx->s.headers,
             ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     else
         route_kernel<false><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, ctx->s.rows, ctx->s.row_bounds,
+            prompt_len, pred_decode_len, slo_ms, n, n_types, ctx->s.rows, ctx->s.row_bounds,
             ctx->s.start_table, ctx->s.headers,
             ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
     return cudaGetLastError();
 }
 
-// Raises the dynamic shared-memory limit of the route kernels (called once per context).
+// Raises the dynamic shared-memory limit of the route kernels and looks up how many CTAs fit
+// on an SM for each table size (called once per context).
 cudaError_t configure_route(gs_ctx *ctx)
 {
+    const size_t max_smem = kRouteSmemFixed + kRouteSmemPerType * GS_MAX_TYPES;
     cudaError_t e = cudaFuncSetAttribute(route_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(kRouteSmemBase + kRouteSmemHist));
+                                         (int)(max_smem + kRouteSmemHist));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRouteSmemBase);
+    e = cudaFuncSetAttribute(route_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    int occ = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false>, kRouteThreads, kRouteSmemBase);
-    if (e != cudaSuccess) return e;
-    ctx->route_ctas_per_sm = occ > 0 ? occ : 1;
+    for (int t = 0; t <= GS_MAX_TYPES; ++t) {
+        int occ = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false>, kRouteThreads,
+                                                          kRouteSmemFixed + kRouteSmemPerType * t);
+        if (e != cudaSuccess) return e;
+        ctx->route_ctas_per_sm[t] = occ > 0 ? occ : 1;
+    }
     return cudaSuccess;
 }
 
