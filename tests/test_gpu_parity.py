@@ -311,3 +311,87 @@ def test_error_codes(gs):
     req = W.make_requests(cfg, types, seed=0, n=100)
     t32 = oracle.instance_table(types, inst, 0.5, "f32")
     assert_route_matches_f32_oracle(gpu_route(gs, pool, req, 0.5), oracle.route(t32, *req.columns()))
+
+
+# --------------------------------------------------------------------------------------
+# adversarial pools for the pruned search: the result must stay exactly the definition's
+# --------------------------------------------------------------------------------------
+
+def _canonical_T(tab32, x, y):
+    """T(r, g) for all (r, g) in the kernels' single-precision operation order (a product of
+    two floats is exact in double, so rounding the double sum once gives the fused result)."""
+    t1 = (np.outer(x.astype(np.float64), tab32.p.astype(np.float64)) + tab32.q.astype(np.float64)).astype(np.float32)
+    return (np.outer(y.astype(np.float64), tab32.d.astype(np.float64)) + t1.astype(np.float64)).astype(np.float32)
+
+
+def _random_pool(rng, M, Tn, scale_p=1.0, scale_d=1.0, equal_batches=False, zero_queue=False, scarce_kv=False):
+    types = W.TypeTable((rng.uniform(0.01, 0.2, Tn) * scale_p).astype(np.float32),
+                        (rng.uniform(4, 50, Tn) * scale_d).astype(np.float32),
+                        (rng.uniform(0.02, 0.3, Tn) * scale_d).astype(np.float32))
+    type_id = rng.integers(0, Tn, M).astype(np.int32)
+    queued = (np.zeros(M) if zero_queue else rng.integers(0, 20001, M)).astype(np.int32)
+    batch = (np.full(M, 7) if equal_batches else rng.integers(0, 65, M)).astype(np.int32)
+    kv = (rng.integers(0, 3000, M) if scarce_kv else rng.integers(0, 200001, M)).astype(np.int32)
+    q_ema = (queued * types.prefill_ms_per_tok[type_id] * rng.uniform(0.8, 1.2, M)).astype(np.float32)
+    return types, W.InstanceState(type_id, queued, batch, kv, q_ema)
+
+
+def _boundary_requests(rng, tab32, n):
+    """Requests whose deadline sits exactly on, one ulp below and one ulp above the estimate
+    of some instance, mixed with loose and hopeless ones."""
+    x = np.clip(np.rint(np.exp(rng.normal(6.5, 1.0, n))), 1, 1 << 20).astype(np.int32)
+    y = np.clip(np.rint(np.exp(rng.normal(5.0, 1.5, n))), 1, 1 << 20).astype(np.int32)
+    y[rng.random(n) < 0.02] = 0
+    x[rng.random(n) < 0.02] = 0
+    T = _canonical_T(tab32, x, y)
+    g = rng.integers(0, T.shape[1], n)
+    D = T[np.arange(n), g].copy()
+    kind = rng.integers(0, 6, n)
+    D = np.where(kind == 1, np.nextafter(D, np.float32(-np.inf)), D)
+    D = np.where(kind == 2, np.nextafter(D, np.float32(np.inf)), D)
+    D = np.where(kind == 3, D * rng.uniform(0.3, 3.0, n).astype(np.float32), D)
+    D = np.where(kind == 4, T.min(axis=1) * np.float32(0.999), D)
+    D = np.where(kind == 5, T.max(axis=1) * np.float32(1.001), D)
+    return W.RequestBatch(x, y, D.astype(np.float32))
+
+
+FUZZ_CASES = [
+    dict(M=1024, Tn=1), dict(M=1024, Tn=16), dict(M=1000, Tn=3), dict(M=513, Tn=8, scarce_kv=True),
+    dict(M=300, Tn=16, equal_batches=True), dict(M=128, Tn=1, equal_batches=True, zero_queue=True),
+    dict(M=64, Tn=2, zero_queue=True), dict(M=17, Tn=1), dict(M=16, Tn=1), dict(M=40, Tn=5, scarce_kv=True),
+    dict(M=777, Tn=7, scale_p=1e-6, scale_d=1e-5), dict(M=777, Tn=7, scale_p=1e4, scale_d=1e3),
+    dict(M=1024, Tn=8, scale_d=1e-3), dict(M=257, Tn=4, scale_p=0.0),
+]
+
+
+@pytest.mark.parametrize("case", range(len(FUZZ_CASES)))
+def test_pruned_search_is_exact_on_adversarial_pools(gs, case):
+    rng = np.random.default_rng(1000 + case)
+    types, inst = _random_pool(rng, **FUZZ_CASES[case])
+    pool = pool_of(gs, types, inst)
+    for alpha in (0.0, 0.5):
+        t32 = oracle.instance_table(types, inst, alpha, "f32")
+        req = _boundary_requests(rng, t32, 6000)
+        got = gpu_route(gs, pool, req, alpha)
+        ref = oracle.route(t32, *req.columns(), threads=4)
+        assert_route_matches_f32_oracle(got, ref)
+    assert gs.device_status() == 0
+
+
+def test_coefficients_the_bounds_cannot_use_take_the_exhaustive_path(gs):
+    """A negative type constant makes lower bounds meaningless; the kernel then scores every
+    instance for every request and still returns the definition's answer."""
+    from paper_2605_16867_b200 import DeviceStatus
+    rng = np.random.default_rng(77)
+    types, inst = _random_pool(rng, 200, 4)
+    types.tpot_a_ms[1] = -3.0
+    pool = pool_of(gs, types, inst)
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    cfg = W.CONFIGS[1]
+    req = W.make_requests(cfg, types, seed=3, n=5000)
+    req.slo_ms[:] = np.abs(req.slo_ms)
+    got = gpu_route(gs, pool, req, 0.5)
+    ref = oracle.route(t32, *req.columns())
+    np.testing.assert_array_equal(got.instance_idx, ref.instance_idx)
+    np.testing.assert_array_equal(got.tier, ref.tier)
+    assert gs.device_status() & DeviceStatus.BAD_VALUE
