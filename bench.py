@@ -36,6 +36,24 @@ UNIT = "pairs/s"
 ROUTE_BYTES_PER_REQUEST = 24      # 3 input columns + 3 output columns, 4 B each
 RISK_BYTES_PER_REQUEST = 20.125   # 5 input columns + 1 flag bit (candidate indices added per flag)
 KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter")
+ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-instruction per clock
+
+# Counters of one launch on config 3 taken with ncu (profiles/route_kernel_config3.md).  They
+# describe the kernel sources with this hash; after any change to those files they no longer
+# apply and the fields that use them become null until the kernel is profiled again.
+PROFILED_ROUTE = {"sources_sha1": "03458c74dc1f4239b529344bf78842b3d3547611", "config": 3,
+                  "dram_bytes_per_launch": 50_439_424 + 5_802_496,
+                  "warp_instructions_per_launch": 58_386_468}
+
+
+def kernel_sources_sha1() -> str:
+    import hashlib
+    h = hashlib.sha1()
+    base = os.path.join(ROOT, "paper_2605_16867_b200", "csrc")
+    for name in ("gs_internal.cuh", "prologue.cu", "route.cu"):
+        with open(os.path.join(base, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 # --------------------------------------------------------------------------------------
@@ -348,12 +366,23 @@ def run_gpu(args):
                  "risk_flags": 20 * A + 4 * ((A + 31) // 32) + 4 * ((A + 1023) // 1024),
                  "risk_scatter": 4 * ((A + 31) // 32) + 4 * flagged + 4 * ((A + 1023) // 1024)}
     roofline = None
+    issue = None
+    profiled = (PROFILED_ROUTE if PROFILED_ROUTE["sources_sha1"] == kernel_sources_sha1()
+                and PROFILED_ROUTE["config"] == args.config else None)
     if dominant in alg_bytes:
         ms, n = kernel_ms[dominant]
         achieved = alg_bytes[dominant] / (ms / n * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
-                    "algorithmic_bytes_per_launch": alg_bytes[dominant]}
+                    "frac": achieved / peak,
+                    "traffic": profiled["dram_bytes_per_launch"] if profiled and dominant == "route" else None,
+                    "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": alg_bytes[dominant]}
+    if profiled and "route" in kernel_ms:
+        ms, n = kernel_ms["route"]
+        rate = profiled["warp_instructions_per_launch"] / (ms / n * 1e-3)
+        issue = {"kernel": "route", "bound": "alu", "achieved": rate, "peak": ISSUE_PEAK_WARP_INST_PER_S,
+                 "unit": "warp-instructions/s", "frac": rate / ISSUE_PEAK_WARP_INST_PER_S,
+                 "warp_instructions_per_request": profiled["warp_instructions_per_launch"] / N,
+                 "note": "instruction count from ncu; peak = 148 SMs x 4 schedulers x 1.965 GHz"}
     for name in per_kernel:
         if name in alg_bytes:
             gbs = alg_bytes[name] / (per_kernel[name]["avg_us"] * 1e-6) / 1e9
@@ -376,7 +405,7 @@ def run_gpu(args):
         "route_requests_per_s": world * N / (route_ms * 1e-3) if route_ms else None,
         "step_hbm_frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "flagged_fraction": flagged / A, "device_status": status,
-        "roofline": roofline, "kernels": per_kernel,
+        "roofline": roofline, "issue": issue, "kernels": per_kernel,
         "kernel_timing": "serial pass of %d steps on one stream after the timed region, %.4f ms/step" % (
             args.steps, serial_ms_per_step),
         "e2e": None if args.no_e2e else
@@ -401,7 +430,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--serial", action="store_true", help="route and scan on one stream instead of two")
+    ap.add_argument("--print-kernel-hash", action="store_true", help="print the hash PROFILED_ROUTE refers to")
     args = ap.parse_args()
+    if args.print_kernel_hash:
+        print(kernel_sources_sha1())
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
