@@ -105,9 +105,7 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
 {
     const int lane = threadIdx.x & 31;
     const int64_t gwarp = (int64_t)blockIdx.x * kRiskWarps + (threadIdx.x >> 5);
-    const uint32_t lt_mask = (1u << lane) - 1u;
-
-    // clear what an earlier call left in the other parity's group totals, for the next call
+     // clear what an earlier call left in the other parity's group totals, for the next call
     for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n_clear;
          k += (int64_t)gridDim.x * blockDim.x)
         next_group_totals[k] = 0u;
@@ -119,13 +117,24 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
     // flags before chunk c0: whole groups, then the chunks of c0's own group
     unsigned part = 0;
     const int64_t g0 = c0 >> kGroupShift;
-    for (int64_t k = lane; k < g0; k += 32) part += group_totals[k];
-    for (int64_t k = (g0 << kGroupShift) + lane; k < c0; k += 32) part += chunk_counts[k];
+    for (int64_t k = lane; k < g0; k += 32 * 8) {           // eight independent loads in flight
+        unsigned v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = k + 32 * u < g0 ? group_totals[k + 32 * u] : 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) part += v[u];
+    }
+    {
+        const int64_t k = (g0 << kGroupShift) + lane;       // at most 64 chunks of c0's own group
+        part += (k < c0 ? chunk_counts[k] : 0u) + (k + 32 < c0 ? chunk_counts[k + 32] : 0u);
+    }
     int64_t base = (int64_t)__reduce_add_sync(0xFFFFFFFFu, part);
 
+    __shared__ unsigned short sh_stage[kRiskWarps][kRiskChunk];   // a chunk's flagged positions, in order
+    unsigned short *stage = sh_stage[threadIdx.x >> 5];
     for (int64_t chunk = c0; chunk < c1; ++chunk) {
         const int64_t wi = chunk * 32 + lane;
-        const uint32_t word = wi < n_words ? __ldcs(flag_bits + wi) : 0u;
+        uint32_t word = wi < n_words ? __ldcs(flag_bits + wi) : 0u;
         const unsigned c = __popc(word);
         unsigned incl = c;
 #pragma unroll
@@ -133,26 +142,22 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
             const unsigned v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
             if (lane >= off) incl += v;
         }
-        const unsigned word_off = incl - c;                 // flags in earlier words of the chunk
         const unsigned total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-        const int32_t idx0 = (int32_t)(chunk * kRiskChunk) + lane;      // n_active < 2^31
-        if (base + total <= cand_capacity) {
-            // whole chunk fits: 32-bit offsets from one 64-bit base, no per-element bound check
-            int32_t *out = cand_idx + base;
-#pragma unroll 8
-            for (int k = 0; k < 32; ++k) {
-                const uint32_t wk = __shfl_sync(0xFFFFFFFFu, word, k);
-                const unsigned ok = __shfl_sync(0xFFFFFFFFu, word_off, k);
-                if ((wk >> lane) & 1u) out[ok + __popc(wk & lt_mask)] = idx0 + 32 * k;
-            }
-        } else if (base < cand_capacity) {
-            for (int k = 0; k < 32; ++k) {
-                const uint32_t wk = __shfl_sync(0xFFFFFFFFu, word, k);
-                const unsigned ok = __shfl_sync(0xFFFFFFFFu, word_off, k);
-                const int64_t pos = base + ok + __popc(wk & lt_mask);
-                if (((wk >> lane) & 1u) && pos < cand_capacity) cand_idx[pos] = idx0 + 32 * k;
-            }
+        // each lane lists the set bits of its own word behind those of the lower words ...
+        unsigned at = incl - c;
+        const unsigned lane_base = (unsigned)lane << 5;
+        while (word) {
+            stage[at++] = (unsigned short)(lane_base + (__ffs(word) - 1));
+            word &= word - 1;
         }
+        __syncwarp();
+        // ... and the warp copies the list out with contiguous stores
+        const int32_t idx0 = (int32_t)(chunk * kRiskChunk);             // n_active < 2^31
+        const int64_t room = cand_capacity - base;
+        const unsigned n_out = room <= 0 ? 0u : (room < (int64_t)total ? (unsigned)room : total);
+        int32_t *out = cand_idx + base;
+        for (unsigned i = lane; i < n_out; i += 32) out[i] = idx0 + (int32_t)stage[i];
+        __syncwarp();
         base += total;
     }
     if (c1 == n_chunks && lane == 0) {      // the warp that owns the last chunk knows the total
