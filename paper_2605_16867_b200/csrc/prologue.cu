@@ -30,7 +30,8 @@
 
 namespace gs {
 
-constexpr int kPrologueThreads = 256;
+constexpr int kPrologueThreads = GS_MAX_INSTANCES;      // one thread per instance
+constexpr int kPmFloats = 8192;                         // shared-memory floats for the running minima
 
 __device__ __forceinline__ int clamp_count(int v, unsigned &bad) {
     if (v < 0) { bad |= GS_DEV_BAD_VALUE; return 0; }
@@ -44,6 +45,12 @@ __device__ __forceinline__ unsigned orderable(float f) {
 }
 
 constexpr float kShrink = 1.0f - 1.9073486328125e-6f;   // 1 - 2^-19
+
+// Upper edge of bucket b of L_out: buckets split every octave at 1.5, b = 2 * exponent + (mantissa >= 1.5).
+__device__ __forceinline__ float bucket_upper_edge(int b) {
+    const unsigned e = 127u + (unsigned)(b >> 1);
+    return __uint_as_float((b & 1) ? ((e + 1u) << 23) : ((e << 23) | 0x400000u));
+}
 constexpr unsigned kPadQ = 0x7FC00000u;                 // NaN: compares false with everything
 
 // Bit pattern of a lower bound of v >= 0 whose low tag bits are zero and may be overwritten.
@@ -61,12 +68,15 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 Scratch s)
 {
     __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];                // my type's rows, sorted
+    extern __shared__ unsigned long long sh_dyn[];                        // sort exchange buffers, then running minima
+    unsigned long long (*sh_xchg)[GS_MAX_INSTANCES] = reinterpret_cast<unsigned long long (*)[GS_MAX_INSTANCES]>(sh_dyn);
     __shared__ float sh_q[GS_MAX_INSTANCES], sh_d[GS_MAX_INSTANCES];       // by instance index
     __shared__ unsigned char sh_t[GS_MAX_INSTANCES];
     __shared__ float sh_rq[GS_MAX_INSTANCES], sh_rd[GS_MAX_INSTANCES];     // my rows: q_lo, d_lo (untagged)
     __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES];
     __shared__ unsigned sh_dmax[GS_MAX_TYPES];
     __shared__ unsigned sh_qmin;
+    __shared__ float sh_tp[GS_MAX_TYPES], sh_ta[GS_MAX_TYPES], sh_tb[GS_MAX_TYPES];   // type constants
     __shared__ int sh_unsafe, sh_fill;
 
     const int tid = threadIdx.x;
@@ -77,32 +87,51 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; }
     __syncthreads();
 
-    // ---- 1. coefficients of every instance ---------------------------------------------------
-    for (int g = tid; g < M; g += kPrologueThreads) {
-        int t = type_id[g];
-        if (t < 0 || t >= n_types) { bad |= GS_DEV_BAD_TYPE; t = 0; }
-        const float Qtok = __int2float_rn(clamp_count(queued[g], bad));
-        const float B = __int2float_rn(clamp_count(batch[g], bad));
-        float qe = q_ema[g];
-        if (!(qe >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; qe = 0.0f; }
-        const int kv = clamp_count(free_kv[g], bad);
-        const float p = p_type[t];
-        const float d = __fmaf_rn(b_type[t], B, a_type[t]);     // loaded per-token decode latency
-        const float w = __fmul_rn(Qtok, p);                     // time to drain the queued prefill
-        const float keep = __fmul_rn(__fsub_rn(1.0f, alpha), qe);
-        const float q = __fmaf_rn(alpha, w, keep);              // EMA step
-        sh_q[g] = q; sh_d[g] = d; sh_t[g] = (unsigned char)t;
-        if (writer) {
-            Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
-            s.rows[g] = row;
-            s.d_by_g[g] = d;
-            s.q_by_g[g] = q;
+    // ---- 1. coefficients of every instance (thread g owns instance g) -------------------------
+    // all global loads are issued before anything depends on them
+    const bool has = tid < M;
+    int r_type = 0, r_queued = 0, r_batch = 0, r_kv = 0;
+    float r_qema = 0.f;
+    if (has) {
+        r_type = type_id[tid]; r_queued = queued[tid]; r_batch = batch[tid];
+        r_kv = free_kv[tid]; r_qema = q_ema[tid];
+    }
+    if (tid < n_types) { sh_tp[tid] = p_type[tid]; sh_ta[tid] = a_type[tid]; sh_tb[tid] = b_type[tid]; }
+    __syncthreads();
+    {
+        int t = r_type;
+        if (has && (t < 0 || t >= n_types)) { bad |= GS_DEV_BAD_TYPE; t = 0; }
+        if (!has) t = -1;
+        float d = 0.f;
+        if (has) {
+            const float Qtok = __int2float_rn(clamp_count(r_queued, bad));
+            const float B = __int2float_rn(clamp_count(r_batch, bad));
+            float qe = r_qema;
+            if (!(qe >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; qe = 0.0f; }
+            const int kv = clamp_count(r_kv, bad);
+            const float p = sh_tp[t];
+            d = __fmaf_rn(sh_tb[t], B, sh_ta[t]);               // loaded per-token decode latency
+            const float w = __fmul_rn(Qtok, p);                 // time to drain the queued prefill
+            const float keep = __fmul_rn(__fsub_rn(1.0f, alpha), qe);
+            const float q = __fmaf_rn(alpha, w, keep);          // EMA step
+            sh_q[tid] = q; sh_d[tid] = d; sh_t[tid] = (unsigned char)t;
+            if (writer) {
+                Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
+                s.rows[tid] = row;
+                s.d_by_g[tid] = d;
+                s.q_by_g[tid] = q;
+            }
+            // the bounds of the search tables need finite, non-negative coefficients
+            const float big = 3.0e38f;
+            if (!(q >= 0.f && q < big && p >= 0.f && p < big && d >= 0.f && d < big)) atomicOr(&sh_unsafe, 1);
         }
-        // the bounds of the search tables need finite, non-negative coefficients
-        const float big = 3.0e38f;
-        if (!(q >= 0.f && q < big && p >= 0.f && p < big && d >= 0.f && d < big)) atomicOr(&sh_unsafe, 1);
-        atomicAdd(&sh_cnt[t], 1);
-        atomicMax(&sh_dmax[t], orderable(d));
+        // instances per type and each type's largest d: one shared-memory atomic per type and warp
+        const unsigned peers = __match_any_sync(0xFFFFFFFFu, t);
+        const unsigned dmax = __reduce_max_sync(peers, orderable(d));
+        if (t >= 0 && lane == __ffs(peers) - 1) {
+            atomicAdd(&sh_cnt[t], __popc(peers));
+            atomicMax(&sh_dmax[t], dmax);
+        }
     }
     __syncthreads();
 
@@ -141,25 +170,35 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     const int n_padded = (n_t + 15) & ~15;
 
     // ---- 3. collect this type's rows and sort them by (d descending, index ascending) --------
+    // bitonic network, one key per thread: partners closer than a warp exchange by shuffle,
+    // farther ones through shared memory (two buffers, so one barrier per exchange)
     int n_sort = 32;
     while (n_sort < n_t) n_sort <<= 1;
-    for (int g = tid; g < M; g += kPrologueThreads)
-        if (sh_t[g] == my_type)
-            sh_key[atomicAdd(&sh_fill, 1)] = ((unsigned long long)(~orderable(sh_d[g])) << 16) | (unsigned)g;
-    for (int k = n_t + tid; k < n_sort; k += kPrologueThreads) sh_key[k] = ~0ull;
+    if (has && sh_t[tid] == my_type)
+        sh_key[atomicAdd(&sh_fill, 1)] = ((unsigned long long)(~orderable(sh_d[tid])) << 16) | (unsigned)tid;
     __syncthreads();
-    for (int k = 2; k <= n_sort; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = tid; i < n_sort; i += kPrologueThreads) {
-                const int partner = i ^ j;
-                if (partner > i) {
-                    const unsigned long long a = sh_key[i], b = sh_key[partner];
-                    if ((a > b) == ((i & k) == 0)) { sh_key[i] = b; sh_key[partner] = a; }
+    {
+        unsigned long long key = tid < n_t ? sh_key[tid] : ~0ull;
+        int buf = 0;
+        for (int k = 2; k <= n_sort; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                unsigned long long other;
+                if (j >= 32) {
+                    sh_xchg[buf][tid] = key;
+                    __syncthreads();
+                    other = sh_xchg[buf][tid ^ j];
+                    buf ^= 1;
+                } else {
+                    other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
                 }
+                const bool keep_min = ((tid & k) == 0) == ((tid & j) == 0);
+                key = (keep_min == (other < key)) ? other : key;
             }
-            __syncthreads();
         }
+        __syncthreads();
+        sh_key[tid] = key;
     }
+    __syncthreads();
 
     // ---- 4. row bounds, least q of the type ---------------------------------------------------
     unsigned my_qmin = 0xFFFFFFFFu;
@@ -187,7 +226,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     if (tid == 0) {
         const int first_inst = (int)(sh_key[0] & 0xFFFFull);
         TypeHeader h;
-        h.p_lo = __fmul_rn(p_type[my_type], kShrink);
+        h.p_lo = __fmul_rn(sh_tp[my_type], kShrink);
         h.q_lo = q0;
         h.d_lo = d_low;
         h.d_max = sh_d[first_inst];
@@ -205,32 +244,39 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     // k with P_k <= y_hi z_edge: a binary search per slot.  Eight buckets are done at a time,
     // one warp each for the running minima, then one (bucket, slot) cell per thread.
     if (inv_w > 0.f) {
-        extern __shared__ float sh_pm[];                    // [8][n_t] running minima
+        float *sh_pm = reinterpret_cast<float *>(sh_dyn);   // [buckets per batch][n_t] running minima
         const float w_slot = 1.0f / inv_w;
-        for (int b0 = 0; b0 < kStartBuckets; b0 += kPrologueThreads / 32) {
-            {
+        int per_batch = kPmFloats / n_t;                    // n_t <= 1024: at least 8
+        if (per_batch > kStartBuckets) per_batch = kStartBuckets;
+        __syncthreads();                                    // the sort is done with sh_dyn
+        for (int b0 = 0; b0 < kStartBuckets; b0 += per_batch) {
+            if (warp < per_batch && b0 + warp < kStartBuckets) {
                 const int b = b0 + warp;
                 // bucket b holds y in [2^e (1 + m/2), 2^e (1 + (m+1)/2)),  e = b >> 1, m = b & 1;
                 // the last bucket has no upper edge: there only d_lo <= z_edge can be required
                 const bool open_ended = b == kStartBuckets - 1;
-                const float y_hi = ldexpf(1.0f + 0.5f * (float)((b & 1) + 1), b >> 1) * 1.00002f;
+                const float y_hi = bucket_upper_edge(b) * 1.00002f;
                 float carry = 3.4e38f;
                 for (int k0 = 0; k0 < n_t; k0 += 32) {
                     const int k = k0 + lane;
                     float h = 3.4e38f;
                     if (k < n_t) h = open_ended ? sh_rd[k] : __fmaf_rn(y_hi, sh_rd[k], sh_rq[k] - q0);
 #pragma unroll
-                    for (int off = 1; off < 32; off <<= 1) h = fminf(h, __shfl_up_sync(0xFFFFFFFFu, h, off) + (lane >= off ? 0.f : 3.4e38f));
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const float up = __shfl_up_sync(0xFFFFFFFFu, h, off);
+                        if (lane >= off) h = fminf(h, up);
+                    }
                     h = fminf(h, carry);
                     if (k < n_t) sh_pm[warp * n_t + k] = h;
                     carry = __shfl_sync(0xFFFFFFFFu, h, 31);
                 }
             }
             __syncthreads();
-            for (int c = tid; c < (kPrologueThreads / 32) * kStartSlots; c += kPrologueThreads) {
+            for (int c = tid; c < per_batch * kStartSlots; c += kPrologueThreads) {
                 const int bw = c / kStartSlots, slot = c % kStartSlots, b = b0 + bw;
+                if (b >= kStartBuckets) break;
                 const bool open_ended = b == kStartBuckets - 1;
-                const float y_hi = ldexpf(1.0f + 0.5f * (float)((b & 1) + 1), b >> 1) * 1.00002f;
+                const float y_hi = bucket_upper_edge(b) * 1.00002f;
                 const float z_edge = d_low + (float)(slot + 2) * w_slot;
                 const float limit = (open_ended ? z_edge : y_hi * z_edge) * 1.00002f;
                 const float *pm = sh_pm + bw * n_t;
@@ -248,7 +294,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     }
 }
 
-size_t prologue_dynamic_smem() { return (size_t)(kPrologueThreads / 32) * GS_MAX_INSTANCES * sizeof(float); }
+size_t prologue_dynamic_smem() { return (size_t)kPmFloats * sizeof(float); }   // >= 2 sort buffers
 
 cudaError_t configure_prologue()
 {

@@ -25,7 +25,10 @@
 namespace gs {
 
 constexpr int kRouteThreads = 256;
-constexpr int kReqPerThread = 4;
+#ifndef GS_REQ_PER_THREAD
+#define GS_REQ_PER_THREAD 4
+#endif
+constexpr int kReqPerThread = GS_REQ_PER_THREAD;
 constexpr int kRouteTile = kRouteThreads * kReqPerThread;
 
 // T(r,g) of Eq. 2 with H = 0, each step rounded once.
@@ -209,7 +212,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         const int64_t first = wt * kWarpTile + (int64_t)lane * kReqPerThread;
         int xi[kReqPerThread], yi[kReqPerThread];
         float D[kReqPerThread];
-        if (first + kReqPerThread <= n) {
+        if (kReqPerThread == 4 && first + kReqPerThread <= n) {
             const int4 xv = __ldcs(reinterpret_cast<const int4 *>(prompt_len + first));
             const int4 yv = __ldcs(reinterpret_cast<const int4 *>(pred_decode_len + first));
             const float4 dv = __ldcs(reinterpret_cast<const float4 *>(slo_ms + first));
@@ -293,7 +296,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             }
             if (kAccumulate) accumulate_choice(hist, M, valid ? g_out[j] : -1, (unsigned)xi[j], need);
         }
-        if (first + kReqPerThread <= n) {
+        if (kReqPerThread == 4 && first + kReqPerThread <= n) {
             __stcs(reinterpret_cast<int4 *>(out_idx + first), make_int4(g_out[0], g_out[1], g_out[2], g_out[3]));
             __stcs(reinterpret_cast<float4 *>(out_est + first), make_float4(T_out[0], T_out[1], T_out[2], T_out[3]));
             __stcs(reinterpret_cast<float4 *>(out_slack + first),
