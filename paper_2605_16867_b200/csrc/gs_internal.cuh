@@ -20,7 +20,7 @@ struct __align__(16) Row {
 // Per-round search tables (built by the prologue, read by the route kernel).  Rows are
 // grouped by GPU type and, inside a type, kept in preference order (d descending, index
 // ascending); each type's rows are padded to a multiple of 16.
-//   row_bounds[i]   = {bits of q_lo, bits of d_lo | instance index}   (one row)
+//   row_bounds[i]   = {bits of q_lo | instance index, bits of d_lo}   (one row)
 //   start_table[(t * kStartBuckets + b) * kStartSlots + s] = first group of 8 rows of type t
 //                     worth looking at when L_out falls in bucket b and the largest d that can
 //                     still meet the deadline falls in slot s
@@ -32,7 +32,7 @@ __host__ __device__ __forceinline__ int row_slot(int i) {
     return (group << 3) | (((pair ^ ((group >> 1) & 3)) << 1) | (i & 1));
 }
 
-constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low bits of a d word
+constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low bits of a q word
 constexpr int kMaxPaddedRows = GS_MAX_INSTANCES + GS_MAX_TYPES * 16;
 constexpr int kStartSlots = 64;
 constexpr int kStartBuckets = 32;         // two per octave of L_out; the last one is open-ended

@@ -15,8 +15,8 @@
 // Bounds: q_lo <= q (1 - 2^-19), d_lo <= d (1 - 2^-19), p_lo = p (1 - 2^-19).  With all
 // coefficients non-negative and each fused step of T = fma(d, y, fma(p, x, q)) rounding by at
 // most 2^-24 relative, the single-precision test  fma(d_lo, y, q_lo) > fma(-p_lo, x, D)
-// implies  T(r,g) > D  for every row the bound covers.  The low bits of a row's d word
-// carry the instance index; the bound is lowered by one unit of the remaining mantissa
+// implies  T(r,g) > D  for every row the bound covers.  The low bits of a row's q word
+// carry the instance index; that bound is lowered by one unit of the remaining mantissa
 // first, so it stays a lower bound.
 //
 // Start table.  Write R for fma(-p_lo, x, D), q0 for the type's least q_lo, y for L_out and
@@ -58,6 +58,9 @@ __device__ __forceinline__ unsigned lower_bound_bits(float v) {
     const unsigned b = __float_as_uint(__fmul_rn(v, kShrink)) & ~kRowTagMask;
     return b >= (kRowTagMask + 1u) ? b - (kRowTagMask + 1u) : 0u;
 }
+
+// Lower bound of v >= 0 at full precision (no tag).
+__device__ __forceinline__ float lower_bound(float v) { return __fmul_rn(v, kShrink); }
 
 __global__ void __launch_bounds__(kPrologueThreads)
 prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__ queued,
@@ -206,10 +209,12 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         uint2 entry = make_uint2(kPadQ, 0u);
         if (k < n_t) {
             const int inst = (int)(sh_key[k] & 0xFFFFull);
-            const unsigned q_bits = lower_bound_bits(sh_q[inst]), d_bits = lower_bound_bits(sh_d[inst]);
-            entry = make_uint2(q_bits, d_bits | (unsigned)inst);
+            // the tag rides on q: d multiplies L_out, so its bound is kept at full precision
+            const unsigned q_bits = lower_bound_bits(sh_q[inst]);
+            const float d_lo = lower_bound(sh_d[inst]);
+            entry = make_uint2(q_bits | (unsigned)inst, __float_as_uint(d_lo));
             sh_rq[k] = __uint_as_float(q_bits);
-            sh_rd[k] = __uint_as_float(d_bits);
+            sh_rd[k] = d_lo;
             my_qmin = min(my_qmin, q_bits);             // non-negative floats order like their bits
         }
         s.row_bounds[row_slot(base + k)] = entry;

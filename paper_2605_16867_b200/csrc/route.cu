@@ -135,14 +135,14 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
                 const uint4 r1 = *reinterpret_cast<const uint4 *>(grp + ((1 ^ sw) << 4));
                 const uint4 r2 = *reinterpret_cast<const uint4 *>(grp + ((2 ^ sw) << 4));
                 const uint4 r3 = *reinterpret_cast<const uint4 *>(grp + ((3 ^ sw) << 4));
-                first = __fmaf_rn(__uint_as_float(r3.w), y, __uint_as_float(r3.z)) <= R ? r3.w : first;
-                first = __fmaf_rn(__uint_as_float(r3.y), y, __uint_as_float(r3.x)) <= R ? r3.y : first;
-                first = __fmaf_rn(__uint_as_float(r2.w), y, __uint_as_float(r2.z)) <= R ? r2.w : first;
-                first = __fmaf_rn(__uint_as_float(r2.y), y, __uint_as_float(r2.x)) <= R ? r2.y : first;
-                first = __fmaf_rn(__uint_as_float(r1.w), y, __uint_as_float(r1.z)) <= R ? r1.w : first;
-                first = __fmaf_rn(__uint_as_float(r1.y), y, __uint_as_float(r1.x)) <= R ? r1.y : first;
-                first = __fmaf_rn(__uint_as_float(r0.w), y, __uint_as_float(r0.z)) <= R ? r0.w : first;
-                first = __fmaf_rn(__uint_as_float(r0.y), y, __uint_as_float(r0.x)) <= R ? r0.y : first;
+                first = __fmaf_rn(__uint_as_float(r3.w), y, __uint_as_float(r3.z)) <= R ? r3.z : first;
+                first = __fmaf_rn(__uint_as_float(r3.y), y, __uint_as_float(r3.x)) <= R ? r3.x : first;
+                first = __fmaf_rn(__uint_as_float(r2.w), y, __uint_as_float(r2.z)) <= R ? r2.z : first;
+                first = __fmaf_rn(__uint_as_float(r2.y), y, __uint_as_float(r2.x)) <= R ? r2.x : first;
+                first = __fmaf_rn(__uint_as_float(r1.w), y, __uint_as_float(r1.z)) <= R ? r1.z : first;
+                first = __fmaf_rn(__uint_as_float(r1.y), y, __uint_as_float(r1.x)) <= R ? r1.x : first;
+                first = __fmaf_rn(__uint_as_float(r0.w), y, __uint_as_float(r0.z)) <= R ? r0.z : first;
+                first = __fmaf_rn(__uint_as_float(r0.y), y, __uint_as_float(r0.x)) <= R ? r0.x : first;
                 if (first != kNoRow) break;
             }
             if (first == kNoRow) break;                     // type exhausted
@@ -153,9 +153,9 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
             bool over = false, seen = false;
             for (int j = 0; j < 8 && !over; ++j) {
                 const uint2 rb = tb.row_bounds[row_slot(k + j)];
-                if (!seen) { seen = (rb.y == first); continue; }
+                if (!seen) { seen = (rb.x == first); continue; }
                 if (__fmaf_rn(__uint_as_float(rb.y), y, __uint_as_float(rb.x)) <= R)
-                    over = score_row(tb, (int)(rb.y & kRowTagMask), x, y, D, need, g_best, d_best, T_best);
+                    over = score_row(tb, (int)(rb.x & kRowTagMask), x, y, D, need, g_best, d_best, T_best);
             }
             if (over) break;
             k += 8;
