@@ -211,3 +211,32 @@ def advance(inst, table_f32: InstanceTable, instance_idx, prompt_len, pred_decod
     _L().gso_advance(C.c_int32(inst.n_instances), C.c_int64(idx.shape[0]), _p(idx), _p(x), _p(y),
                      _p(inst.queued_prefill_tokens), _p(inst.decode_batch),
                      _p(inst.free_kv_tokens), _p(inst.q_ema_ms), _p(table_f32.q))
+
+
+@dataclass
+class RerouteResult:
+    new_instance: np.ndarray   # int32[n_cand], -1 = no strictly faster instance exists
+    est_ms: np.ndarray         # real[n_cand]: estimated remaining time on the target
+    slack_ms: np.ndarray       # real[n_cand]: (slo - elapsed) - est
+    tier: np.ndarray           # uint8[n_cand]: 0 no move, 1 just-enough, 2 / 3 fallback
+    status: int
+
+
+def reroute(table: InstanceTable, cand_idx, assigned_inst, generated_tokens, pred_len, elapsed_ms,
+            slo_ms, prompt_len) -> RerouteResult:
+    """Re-routing of flagged requests among strictly faster instances (see the C source)."""
+    cand = _c(cand_idx, np.int32)
+    g = _c(assigned_inst, np.int32); gen = _c(generated_tokens, np.int32)
+    tot = _c(pred_len, np.int32); el = _c(elapsed_ms, np.float32); slo = _c(slo_ms, np.float32)
+    x = _c(prompt_len, np.int32)
+    n = cand.shape[0]
+    real = np.float64 if table.precision == "f64" else np.float32
+    out = RerouteResult(np.empty(n, np.int32), np.empty(n, real), np.empty(n, real), np.empty(n, np.uint8), 0)
+    status = C.c_uint(0)
+    if n:
+        fn = getattr(_L(), f"gso_reroute_{table.precision}")
+        fn(C.c_int64(n), _p(cand), _p(g), _p(gen), _p(tot), _p(el), _p(slo), _p(x),
+           C.c_int32(table.n_instances), _p(table.q), _p(table.p), _p(table.d), _p(table.kv),
+           _p(out.new_instance), _p(out.est_ms), _p(out.slack_ms), _p(out.tier), C.byref(status))
+    out.status = status.value
+    return out

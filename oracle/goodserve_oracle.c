@@ -267,3 +267,73 @@ void gso_advance(int32_t M, int64_t N, const int32_t *instance_idx,
     }
     free(dq); free(db); free(dk);
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Re-routing of flagged requests (Sec. 3.4): a request whose expected finish exceeds its */
+/* SLO is re-routed "to another GPU with stronger processing capability (still following  */
+/* the just-enough heuristic)"; the migration moves token IDs, so the target re-prefills   */
+/* the whole context (prompt + tokens generated so far).                                   */
+/*                                                                                        */
+/* Reading: for candidate i on instance c                                                  */
+/*   x' = prompt_len + generated,  y' = max(pred_len - generated, 0),  D' = slo - elapsed  */
+/*   eligible instances  G_i = { g : d_g < d_c }        (strictly faster per output token) */
+/*   Algorithm 1 over G_i with (x', y', D'):  tier 1 just-enough pick, tier 2 / 3 fallback */
+/*   to the smallest T among eligible instances with / without KV room;                    */
+/*   G_i empty (already on the fastest instance): no move, instance -1, tier 0.            */
+/* ------------------------------------------------------------------------------------ */
+
+#define GSO_REROUTE_BODY(REAL, LAT)                                                           \
+    for (int64_t j = 0; j < n_cand; ++j) {                                                    \
+        int64_t i = cand_idx[j];                                                              \
+        int32_t c = clamp_instance(assigned_inst[i], M, status);                              \
+        int64_t gen = clamp_count(generated_tokens[i], status);                               \
+        int64_t tot = clamp_count(pred_len[i], status);                                       \
+        int64_t xin = clamp_count(prompt_len[i], status);                                     \
+        int64_t rem = tot - gen; if (rem < 0) rem = 0;                                        \
+        int64_t xi = xin + gen;                                                               \
+        REAL x = (REAL)xi, y = (REAL)rem;                                                     \
+        REAL D = (REAL)slo_ms[i] - (REAL)elapsed_ms[i];                                       \
+        int64_t need = xi + rem;                                                              \
+        int32_t best_c = -1, best_k = -1, best_a = -1;                                        \
+        REAL d_c = 0, T_c = 0, T_k = 0, T_a = 0;                                              \
+        for (int32_t g = 0; g < M; ++g) {                                                     \
+            if (!(d[g] < d[c])) continue;                  /* only strictly faster instances */ \
+            REAL T = LAT;                                                                     \
+            int kv_ok = need <= kv[g];                                                        \
+            if (kv_ok && T <= D) {                                                            \
+                if (best_c < 0 || d[g] > d_c) { best_c = g; d_c = d[g]; T_c = T; }            \
+            }                                                                                 \
+            if (kv_ok && (best_k < 0 || T < T_k)) { best_k = g; T_k = T; }                    \
+            if (best_a < 0 || T < T_a) { best_a = g; T_a = T; }                               \
+        }                                                                                     \
+        int32_t g_star = -1; REAL T_star = 0; uint8_t tr = 0;                                 \
+        if (best_c >= 0)      { g_star = best_c; T_star = T_c; tr = 1; }                      \
+        else if (best_k >= 0) { g_star = best_k; T_star = T_k; tr = 2; }                      \
+        else if (best_a >= 0) { g_star = best_a; T_star = T_a; tr = 3; }                      \
+        new_instance[j] = g_star;                                                             \
+        est_ms[j] = T_star;                                                                   \
+        slack_ms[j] = tr ? D - T_star : 0;                                                    \
+        if (tier) tier[j] = tr;                                                               \
+    }
+
+void gso_reroute_f64(int64_t n_cand, const int32_t *cand_idx,
+                     const int32_t *assigned_inst, const int32_t *generated_tokens,
+                     const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                     const int32_t *prompt_len,
+                     int32_t M, const double *q, const double *p, const double *d, const int64_t *kv,
+                     int32_t *new_instance, double *est_ms, double *slack_ms, uint8_t *tier,
+                     unsigned *status)
+{
+    GSO_REROUTE_BODY(double, q[g] + p[g] * x + d[g] * y)
+}
+
+void gso_reroute_f32(int64_t n_cand, const int32_t *cand_idx,
+                     const int32_t *assigned_inst, const int32_t *generated_tokens,
+                     const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                     const int32_t *prompt_len,
+                     int32_t M, const float *q, const float *p, const float *d, const int64_t *kv,
+                     int32_t *new_instance, float *est_ms, float *slack_ms, uint8_t *tier,
+                     unsigned *status)
+{
+    GSO_REROUTE_BODY(float, fmaf(d[g], y, fmaf(p[g], x, q[g])))
+}

@@ -491,3 +491,72 @@ def test_threaded_split_is_identical():
     ra = oracle.risk(tab, *wl.active.columns(), threads=1)
     rb = oracle.risk(tab, *wl.active.columns(), threads=3)
     np.testing.assert_array_equal(ra.flag, rb.flag)
+
+
+# --------------------------------------------------------------------------------------
+# re-routing of flagged requests
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_handworked_reroute(prec):
+    for name, cur, elapsed, slo, k0, k1, g, est, slack, tier in read_rows("handworked_reroute.txt"):
+        types, inst = fixture_pool((int(k0), int(k1), 100000))
+        tab = oracle.instance_table(types, inst, 0.5, prec)
+        res = oracle.reroute(tab, [0], [int(cur)], [50], [200], [float(elapsed)], [float(slo)], [1000])
+        assert res.new_instance[0] == int(g), name
+        assert res.tier[0] == int(tier), name
+        assert res.est_ms[0] == pytest.approx(float(est), rel=1e-5), name
+        assert res.slack_ms[0] == pytest.approx(float(slack), rel=1e-4, abs=2e-3), name
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_reroute_equals_routing_over_the_faster_instances(prec):
+    """Independent pin: restricted to the strictly faster instances, re-routing IS Algorithm 1
+    on the transformed request (x' = prompt + generated, y' = remaining, D' = slo - elapsed),
+    so it must agree with route() run on the sub-pool of eligible instances."""
+    wl = W.make_workload(1, n_requests=8, n_active=3000)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    a = wl.active
+    prompt = W.make_requests(wl.cfg, wl.types, seed=99, n=a.n).prompt_len
+    flag = oracle.risk(tab, *a.columns()).flag
+    cand = np.nonzero(flag)[0].astype(np.int32)
+    res = oracle.reroute(tab, cand, *a.columns(), prompt)
+    real = np.float64 if prec == "f64" else np.float32
+    seen_tiers = set()
+    for j, i in enumerate(cand[:600]):
+        c = a.assigned_inst[i]
+        elig = np.nonzero(tab.d < tab.d[c])[0]
+        if len(elig) == 0:
+            assert res.new_instance[j] == -1 and res.tier[j] == 0
+            seen_tiers.add(0)
+            continue
+        sub = oracle.InstanceTable(tab.q[elig], tab.p[elig], tab.d[elig], tab.kv[elig], 0, prec)
+        x = np.array([prompt[i] + a.generated_tokens[i]], np.int32)
+        y = np.array([max(a.pred_len[i] - a.generated_tokens[i], 0)], np.int32)
+        D = np.array([real(a.slo_ms[i]) - real(a.elapsed_ms[i])], np.float32)
+        if prec == "f32":
+            assert real(D[0]) == np.float32(a.slo_ms[i]) - np.float32(a.elapsed_ms[i])
+        ref = oracle.route(sub, x, y, D)
+        assert res.new_instance[j] == elig[ref.instance_idx[0]]
+        assert res.tier[j] == ref.tier[0]
+        if prec == "f32":
+            assert res.est_ms[j] == ref.est_e2e_ms[0]
+        else:
+            assert res.est_ms[j] == pytest.approx(ref.est_e2e_ms[0], rel=1e-6)
+        seen_tiers.add(int(res.tier[j]))
+    assert {1, 2} <= seen_tiers
+
+
+def test_reroute_never_moves_to_a_slower_or_equal_instance():
+    wl = W.make_workload(2, n_requests=8, n_active=20000)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, "f64")
+    a = wl.active
+    prompt = W.make_requests(wl.cfg, wl.types, seed=5, n=a.n).prompt_len
+    cand = np.nonzero(oracle.risk(tab, *a.columns()).flag)[0].astype(np.int32)
+    res = oracle.reroute(tab, cand, *a.columns(), prompt)
+    moved = res.new_instance >= 0
+    assert moved.any()
+    assert (tab.d[res.new_instance[moved]] < tab.d[a.assigned_inst[cand[moved]]]).all()
+    assert (res.tier[moved] > 0).all() and (res.tier[~moved] == 0).all()
+    t1 = res.tier == 1
+    assert (res.slack_ms[t1] >= 0).all()
