@@ -35,7 +35,7 @@ METRIC = "request-instance pairs scored/sec"
 UNIT = "pairs/s"
 ROUTE_BYTES_PER_REQUEST = 24      # 3 input columns + 3 output columns, 4 B each
 RISK_BYTES_PER_REQUEST = 20.125   # 5 input columns + 1 flag bit (candidate indices added per flag)
-KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter")
+KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter", "reroute")
 ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-instruction per clock
 
 # Counters of one launch on config 3 taken with ncu (profiles/route_kernel_config3.md).  They

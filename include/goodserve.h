@@ -136,7 +136,8 @@ enum gs_kernel {
     GS_K_ADVANCE = 2,        /* state advance */
     GS_K_RISK_FLAGS = 3,     /* risk test + flag words + per-chunk flag counts */
     GS_K_RISK_SCATTER = 4,   /* ordered candidate list */
-    GS_K_COUNT = 5
+    GS_K_REROUTE = 5,        /* re-routing of the candidates */
+    GS_K_COUNT = 6
 };
 
 /* Optional per-kernel timing for benchmarks.  While enabled (on != 0) every kernel launch of
@@ -198,6 +199,33 @@ GS_API int gs_risk_scan(gs_ctx *ctx,
                  const gs_instances *inst, const gs_types *types,
                  uint32_t *out_flag_bits, int32_t *out_cand_idx, int64_t cand_capacity,
                  int64_t *out_cand_count, void *cuda_stream);
+
+/*
+ * Re-routing of the scan's candidates (Sec. 3.4: a request whose expected finish exceeds its
+ * SLO is re-routed to another instance with stronger processing capability, still by the
+ * just-enough rule; the migration moves token IDs, so the target re-prefills the context).
+ *
+ * cand_idx / cand_count are gs_risk_scan's outputs (device; at most cand_capacity entries are
+ * read); the five active columns are those given to the scan, prompt_len[n_active] is the
+ * requests' L_in.  For candidate j = request i = cand_idx[j] on instance c = assigned_inst[i]:
+ *   x' = prompt_len[i] + generated_tokens[i]      tokens the target has to prefill again
+ *   y' = max(pred_len[i] - generated_tokens[i], 0) tokens left to decode
+ *   D' = slo_ms[i] - elapsed_ms[i]                 time left
+ *   eligible instances: d_g < d_c  (strictly lower per-token decode latency than where it runs)
+ * and Algorithm 1 is applied to (x', y', D') over the eligible instances only.  Outputs, one
+ * entry per candidate (cand_capacity entries each): out_new_instance (-1: no eligible instance,
+ * the request is already on the fastest one), out_est_ms = T(x', y', g*), out_slack_ms = D' - T,
+ * out_tier (may be NULL): 0 no move, 1 just-enough pick, 2 / 3 fallback among eligible
+ * instances with / without KV room.  Uses the instance snapshot given here (EMA step included).
+ */
+GS_API int gs_reroute_candidates(gs_ctx *ctx,
+                                 const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,
+                                 const int32_t *assigned_inst, const int32_t *generated_tokens,
+                                 const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                                 const int32_t *prompt_len, int64_t n_active,
+                                 const gs_instances *inst, const gs_types *types, float ema_alpha,
+                                 int32_t *out_new_instance, float *out_est_ms, float *out_slack_ms,
+                                 uint8_t *out_tier, void *cuda_stream);
 
 /*
  * Host-buffer variants: every pointer (including those inside `inst` and `types`) is a HOST

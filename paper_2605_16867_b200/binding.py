@@ -90,6 +90,9 @@ def load_library(build_if_missing: bool = True):
     lib.gs_risk_scan_host.argtypes = risk_args
     lib.gs_timing_enable.argtypes = [vp, C.c_int]
     lib.gs_timing_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(i64)]
+    lib.gs_reroute_candidates.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, C.POINTER(_Instances),
+                                          C.POINTER(_Types), f32, vp, vp, vp, vp, vp]
+    lib.gs_reroute_candidates.restype = C.c_int
     lib.gs_risk_scan_noalloc.argtypes = [vp, vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types),
                                          vp, vp, i64, vp, vp, vp]
     lib.gs_risk_scan_noalloc.restype = C.c_int
@@ -261,6 +264,28 @@ class GoodServe:
             _dev_ptr(out_flag_bits, i32, (n + 31) // 32, "out_flag_bits", dev),
             _dev_ptr(out_cand_idx, i32, cap, "out_cand_idx", dev), cap,
             _dev_ptr(out_cand_count, torch.int64, 1, "out_cand_count", dev), self._stream(stream)))
+
+    def reroute_candidates(self, cand_idx, cand_count, assigned_inst, generated_tokens, pred_len, elapsed_ms,
+                           slo_ms, prompt_len, pool: InstancePool, ema_alpha: float,
+                           out_new_instance, out_est_ms, out_slack_ms, out_tier=None,
+                           cand_capacity: Optional[int] = None, stream=None):
+        """gs_reroute_candidates: cand_idx / cand_count are risk_scan's device outputs."""
+        cap = int(cand_idx.numel()) if cand_capacity is None else int(cand_capacity)
+        n = int(assigned_inst.numel())
+        dev, i32, f32 = self.device, torch.int32, torch.float32
+        inst, types = self._pool_structs(pool)
+        self._check(self._lib.gs_reroute_candidates(
+            self._h, _dev_ptr(cand_idx, i32, cap, "cand_idx", dev),
+            _dev_ptr(cand_count, torch.int64, 1, "cand_count", dev), cap,
+            _dev_ptr(assigned_inst, i32, n, "assigned_inst", dev),
+            _dev_ptr(generated_tokens, i32, n, "generated_tokens", dev),
+            _dev_ptr(pred_len, i32, n, "pred_len", dev), _dev_ptr(elapsed_ms, f32, n, "elapsed_ms", dev),
+            _dev_ptr(slo_ms, f32, n, "slo_ms", dev), _dev_ptr(prompt_len, i32, n, "prompt_len", dev), n,
+            C.byref(inst), C.byref(types), float(ema_alpha),
+            _dev_ptr(out_new_instance, i32, cap, "out_new_instance", dev),
+            _dev_ptr(out_est_ms, f32, cap, "out_est_ms", dev),
+            _dev_ptr(out_slack_ms, f32, cap, "out_slack_ms", dev),
+            _dev_ptr(out_tier, torch.uint8, cap, "out_tier", dev), self._stream(stream)))
 
     def route_batch_host(self, prompt_len, pred_decode_len, slo_ms, types, inst, ema_alpha: float,
                          out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier=None, stream=None):

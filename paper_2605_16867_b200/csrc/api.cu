@@ -302,6 +302,36 @@ GS_API int gs_risk_scan(gs_ctx *ctx, const int32_t *assigned_inst, const int32_t
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 
+GS_API int gs_reroute_candidates(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count,
+                                 int64_t cand_capacity,
+                                 const int32_t *assigned_inst, const int32_t *generated_tokens,
+                                 const int32_t *pred_len, const float *elapsed_ms, const float *slo_ms,
+                                 const int32_t *prompt_len, int64_t n_active,
+                                 const gs_instances *inst, const gs_types *types, float ema_alpha,
+                                 int32_t *out_new_instance, float *out_est_ms, float *out_slack_ms,
+                                 uint8_t *out_tier, void *cuda_stream)
+{
+    int rc = check_pool(ctx, inst, types, true);
+    if (rc != GS_OK) return rc;
+    if (cand_capacity < 0 || n_active < 0 || n_active > gs::kMaxActive || !cand_count) return GS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(cand_count) & 7u) return GS_ERR_ALIGN;
+    if (cand_capacity > 0) {
+        if (n_active == 0) return GS_ERR_INVALID_ARG;
+        const void *ptrs[] = {cand_idx, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, prompt_len,
+                              out_new_instance, out_est_ms, out_slack_ms};
+        for (const void *p : ptrs) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = gs::launch_reroute(ctx, cand_idx, cand_count, cand_capacity, assigned_inst, generated_tokens, pred_len,
+                           elapsed_ms, slo_ms, prompt_len, n_active, types->n_types,
+                           out_new_instance, out_est_ms, out_slack_ms, out_tier, st);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
 GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                         const float *slo_ms, int64_t n_requests,
                         const gs_instances *inst, const gs_types *types, float ema_alpha,

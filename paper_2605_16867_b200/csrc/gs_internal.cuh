@@ -107,6 +107,11 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
                          const float *slo_ms, int64_t n, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, cudaStream_t st);
+cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,
+                           const int32_t *assigned, const int32_t *generated, const int32_t *pred_len,
+                           const float *elapsed, const float *slo, const int32_t *prompt_len, int64_t n_active,
+                           int n_types, int32_t *out_inst, float *out_est, float *out_slack, uint8_t *out_tier,
+                           cudaStream_t st);
 cudaError_t configure_route(gs_ctx *ctx);
 cudaError_t configure_prologue();
 cudaError_t launch_advance(gs_ctx *ctx, const gs_instances_mut &inst, cudaStream_t st);

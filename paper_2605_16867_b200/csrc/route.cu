@@ -74,15 +74,24 @@ struct Tables {
 
 constexpr unsigned kNoRow = 0xFFFFFFFFu;
 
+// Bound test of one row: false only if the row certainly cannot be chosen.
+template <bool kCapped>
+__device__ __forceinline__ bool row_may_pass(unsigned q_word, unsigned d_word, float y, float R, float d_cap) {
+    const float d_lo = __uint_as_float(d_word);
+    return __fmaf_rn(d_lo, y, __uint_as_float(q_word)) <= R && (!kCapped || d_lo < d_cap);
+}
+
 // Scores one row exactly and folds it into the running best.  Returns true when the search of
 // this type is over: the row is feasible (later rows of the type rank lower) or already ranks
 // below the best found (so does everything after it).
+// With kCapped only instances with d < d_cap are eligible (re-routing to a faster instance).
+template <bool kCapped>
 __device__ __forceinline__ bool score_row(const Tables &tb, int inst, float x, float y, float D, unsigned need,
-                                          int &g_best, float &d_best, float &T_best)
+                                          float d_cap, int &g_best, float &d_best, float &T_best)
 {
     const Row row = tb.rows[inst];
     const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));      // Eq. 2, H = 0
-    const bool feasible = (T <= D) && (need <= (unsigned)row.kv);
+    const bool feasible = (T <= D) && (need <= (unsigned)row.kv) && (!kCapped || row.d < d_cap);
     const bool worse = row.d < d_best;
     if (feasible && !worse && (g_best < 0 || row.d > d_best || inst < g_best)) {
         d_best = row.d; g_best = inst; T_best = T;
@@ -92,15 +101,17 @@ __device__ __forceinline__ bool score_row(const Tables &tb, int inst, float x, f
 
 // Just-enough pick for one request.  Returns the chosen instance or -1 (no feasible one, or a
 // request this search does not take).  `Dm` is the deadline plus a hair (see the caller).
+template <bool kCapped>
 __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y, float D, float Dm,
-                                             unsigned need, float &T_out)
+                                             unsigned need, float d_cap, float &T_out)
 {
     // 1. which types can hold a feasible instance at all
     unsigned alive = 0;
 #pragma unroll 2
     for (int t = 0; t < tb.n_types; ++t) {
         const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);   // p_lo, q_lo, d_lo, d_max
-        if (__fmaf_rn(h.z, y, h.y) <= __fmaf_rn(-h.x, x, Dm)) alive |= 1u << t;
+        // (a type whose least d_lo is not below the cap has no eligible instance: d_lo <= d)
+        if (__fmaf_rn(h.z, y, h.y) <= __fmaf_rn(-h.x, x, Dm) && (!kCapped || h.z < d_cap)) alive |= 1u << t;
     }
     int g_best = -1;
     float d_best = -1.0f, T_best = 0.f;
@@ -135,27 +146,27 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
                 const uint4 r1 = *reinterpret_cast<const uint4 *>(grp + ((1 ^ sw) << 4));
                 const uint4 r2 = *reinterpret_cast<const uint4 *>(grp + ((2 ^ sw) << 4));
                 const uint4 r3 = *reinterpret_cast<const uint4 *>(grp + ((3 ^ sw) << 4));
-                first = __fmaf_rn(__uint_as_float(r3.w), y, __uint_as_float(r3.z)) <= R ? r3.z : first;
-                first = __fmaf_rn(__uint_as_float(r3.y), y, __uint_as_float(r3.x)) <= R ? r3.x : first;
-                first = __fmaf_rn(__uint_as_float(r2.w), y, __uint_as_float(r2.z)) <= R ? r2.z : first;
-                first = __fmaf_rn(__uint_as_float(r2.y), y, __uint_as_float(r2.x)) <= R ? r2.x : first;
-                first = __fmaf_rn(__uint_as_float(r1.w), y, __uint_as_float(r1.z)) <= R ? r1.z : first;
-                first = __fmaf_rn(__uint_as_float(r1.y), y, __uint_as_float(r1.x)) <= R ? r1.x : first;
-                first = __fmaf_rn(__uint_as_float(r0.w), y, __uint_as_float(r0.z)) <= R ? r0.z : first;
-                first = __fmaf_rn(__uint_as_float(r0.y), y, __uint_as_float(r0.x)) <= R ? r0.x : first;
+                first = row_may_pass<kCapped>(r3.z, r3.w, y, R, d_cap) ? r3.z : first;
+                first = row_may_pass<kCapped>(r3.x, r3.y, y, R, d_cap) ? r3.x : first;
+                first = row_may_pass<kCapped>(r2.z, r2.w, y, R, d_cap) ? r2.z : first;
+                first = row_may_pass<kCapped>(r2.x, r2.y, y, R, d_cap) ? r2.x : first;
+                first = row_may_pass<kCapped>(r1.z, r1.w, y, R, d_cap) ? r1.z : first;
+                first = row_may_pass<kCapped>(r1.x, r1.y, y, R, d_cap) ? r1.x : first;
+                first = row_may_pass<kCapped>(r0.z, r0.w, y, R, d_cap) ? r0.z : first;
+                first = row_may_pass<kCapped>(r0.x, r0.y, y, R, d_cap) ? r0.x : first;
                 if (first != kNoRow) break;
             }
             if (first == kNoRow) break;                     // type exhausted
             // lanes meet again here, so the exact scoring runs once per warp, not once per step
-            if (score_row(tb, (int)(first & kRowTagMask), x, y, D, need, g_best, d_best, T_best)) break;
+            if (score_row<kCapped>(tb, (int)(first & kRowTagMask), x, y, D, need, d_cap, g_best, d_best, T_best)) break;
             // rare: the bound passed but the row is not feasible (KV, or inside the bound's
             // margin); go on row by row through the rest of these eight, then resume
             bool over = false, seen = false;
             for (int j = 0; j < 8 && !over; ++j) {
                 const uint2 rb = tb.row_bounds[row_slot(k + j)];
                 if (!seen) { seen = (rb.x == first); continue; }
-                if (__fmaf_rn(__uint_as_float(rb.y), y, __uint_as_float(rb.x)) <= R)
-                    over = score_row(tb, (int)(rb.x & kRowTagMask), x, y, D, need, g_best, d_best, T_best);
+                if (row_may_pass<kCapped>(rb.x, rb.y, y, R, d_cap))
+                    over = score_row<kCapped>(tb, (int)(rb.x & kRowTagMask), x, y, D, need, d_cap, g_best, d_best, T_best);
             }
             if (over) break;
             k += 8;
@@ -163,6 +174,83 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
     }
     T_out = T_best;
     return g_best;
+}
+
+// Copies the round's tables into shared memory (all threads of the CTA; the caller
+// synchronises).  Returns the first shared-memory byte after them.
+__device__ __forceinline__ unsigned char *stage_tables(unsigned char *smem, int n_types_alloc,
+                                                       const Row *__restrict__ g_rows,
+                                                       const uint2 *__restrict__ g_row_bounds,
+                                                       const unsigned char *__restrict__ g_start_table,
+                                                       const TypeHeader *__restrict__ g_headers,
+                                                       const int *__restrict__ table_info, Tables &tb)
+{
+    const int n_padded = table_info[0];
+    const bool unsafe = table_info[1] != 0;
+    const int M = table_info[2];
+    const int n_act = table_info[3];
+    Row *sh_rows = reinterpret_cast<Row *>(smem);
+    TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
+    uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
+    unsigned char *sh_start = reinterpret_cast<unsigned char *>(sh_row_bounds + kMaxPaddedRows);
+    for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[k] = g_rows[k];
+    for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
+    for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
+        reinterpret_cast<uint4 *>(sh_start)[k] = reinterpret_cast<const uint4 *>(g_start_table)[k];
+    if (threadIdx.x < n_act) sh_headers[threadIdx.x] = g_headers[threadIdx.x];
+    tb.headers = sh_headers; tb.row_bounds = sh_row_bounds;
+    tb.start_table = sh_start; tb.rows = sh_rows;
+    tb.n_types = unsafe ? 0 : n_act;          // unusable bounds: every request takes the exhaustive path
+    return sh_start + n_types_alloc * (kStartBuckets * kStartSlots);
+}
+
+// The definition evaluated in full by one warp for one request (same arguments in all lanes):
+// lanes across instances, shuffle reductions.  tier 1: feasible instance with the largest d
+// (ties: smallest index); tier 2 / 3: smallest T among instances with KV room / among all
+// (ties: smallest index); tier 0 (kCapped only): no instance with d < d_cap exists.
+template <bool kCapped>
+__device__ __forceinline__ void exhaustive_pick(const Row *rows, int M, float xs, float ys, float Ds,
+                                                unsigned needs, float d_cap, int lane,
+                                                int &g, float &T, unsigned &tier)
+{
+    unsigned long long k_feas = 0ull;                    // max over feasible: (d, smallest index)
+    unsigned long long k_room = ~0ull, k_all = ~0ull;    // min over KV-ok / all: (T, index)
+    float T_feas = 0.f;
+    for (int inst = lane; inst < M; inst += 32) {
+        const Row row = rows[inst];
+        if (kCapped && !(row.d < d_cap)) continue;
+        const float Tr = latency(row, xs, ys);
+        const bool room = needs <= (unsigned)row.kv;
+        const unsigned long long kt = ((unsigned long long)orderable_bits(Tr) << 32) | (unsigned)inst;
+        if (kt < k_all) k_all = kt;
+        if (room && kt < k_room) k_room = kt;
+        if (room && Tr <= Ds) {
+            const unsigned long long kd =
+                ((unsigned long long)orderable_bits(row.d) << 32) | (0xFFFFu - (unsigned)inst);
+            if (kd > k_feas) { k_feas = kd; T_feas = Tr; }
+        }
+    }
+    unsigned long long w_feas = k_feas, w_room = k_room, w_all = k_all;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long a = __shfl_xor_sync(0xFFFFFFFFu, w_feas, off);
+        const unsigned long long b = __shfl_xor_sync(0xFFFFFFFFu, w_room, off);
+        const unsigned long long c = __shfl_xor_sync(0xFFFFFFFFu, w_all, off);
+        if (a > w_feas) w_feas = a;
+        if (b < w_room) w_room = b;
+        if (c < w_all) w_all = c;
+    }
+    if (w_feas != 0ull) {
+        const unsigned owner = __ballot_sync(0xFFFFFFFFu, k_feas == w_feas);
+        T = __shfl_sync(0xFFFFFFFFu, T_feas, __ffs(owner) - 1);
+        g = (int)(0xFFFFu - (unsigned)(w_feas & 0xFFFFu)); tier = 1;
+    } else if (w_room != ~0ull) {
+        g = (int)(w_room & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_room >> 32)); tier = 2;
+    } else if (w_all != ~0ull) {
+        g = (int)(w_all & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_all >> 32)); tier = 3;
+    } else {
+        g = -1; T = 0.f; tier = 0;
+    }
 }
 
 template <bool kAccumulate>
@@ -177,29 +265,15 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    const int n_padded = table_info[0];
-    const bool unsafe = table_info[1] != 0;
     const int M = table_info[2];
-    const int n_act = table_info[3];
-    Row *sh_rows = reinterpret_cast<Row *>(smem);
-    TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
-    uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
-    unsigned char *sh_start = reinterpret_cast<unsigned char *>(sh_row_bounds + kMaxPaddedRows);
-    unsigned long long *hist = reinterpret_cast<unsigned long long *>(sh_start + n_types_alloc * (kStartBuckets * kStartSlots));
-
-    for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[k] = g_rows[k];
-    for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
-    for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
-        reinterpret_cast<uint4 *>(sh_start)[k] = reinterpret_cast<const uint4 *>(g_start_table)[k];
-    if (threadIdx.x < n_act) sh_headers[threadIdx.x] = g_headers[threadIdx.x];
+    Tables tb;
+    unsigned char *after_tables = stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_start_table, g_headers,
+                                               table_info, tb);
+    const Row *sh_rows = tb.rows;
+    unsigned long long *hist = reinterpret_cast<unsigned long long *>(after_tables);
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
     __syncthreads();
-
-    Tables tb;
-    tb.headers = sh_headers; tb.row_bounds = sh_row_bounds;
-    tb.start_table = sh_start; tb.rows = sh_rows;
-    tb.n_types = unsafe ? 0 : n_act;          // unusable bounds: every request takes the exhaustive path
 
     const int lane = threadIdx.x & 31;
     unsigned bad = 0;
@@ -243,7 +317,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             // (the hair added to the deadline of the bound tests keeps them safe when a bound's
             // tag bits make a zero coefficient a denormal)
             const float Dj = (valid && yi[j] > 0) ? D[j] : -1.0f;
-            g_out[j] = pick_instance(tb, x, y, Dj, Dj + 1e-30f, need, T_out[j]);
+            g_out[j] = pick_instance<false>(tb, x, y, Dj, Dj + 1e-30f, need, 0.f, T_out[j]);
 
             // ---- no feasible instance found: the whole warp scores every instance -------------
             unsigned todo = __ballot_sync(0xFFFFFFFFu, valid && g_out[j] < 0);
@@ -253,42 +327,8 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 const float xs = __shfl_sync(0xFFFFFFFFu, x, src), ys = __shfl_sync(0xFFFFFFFFu, y, src);
                 const float Ds = __shfl_sync(0xFFFFFFFFu, D[j], src);
                 const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
-                unsigned long long k_feas = 0ull;                    // max over feasible: (d, smallest index)
-                unsigned long long k_room = ~0ull, k_all = ~0ull;    // min over KV-ok / all: (T, index)
-                float T_feas = 0.f;
-                for (int inst = lane; inst < M; inst += 32) {
-                    const Row row = sh_rows[inst];
-                    const float T = latency(row, xs, ys);
-                    const bool room = needs <= (unsigned)row.kv;
-                    const unsigned long long kt = ((unsigned long long)orderable_bits(T) << 32) | (unsigned)inst;
-                    if (kt < k_all) k_all = kt;
-                    if (room && kt < k_room) k_room = kt;
-                    if (room && T <= Ds) {
-                        const unsigned long long kd =
-                            ((unsigned long long)orderable_bits(row.d) << 32) | (0xFFFFu - (unsigned)inst);
-                        if (kd > k_feas) { k_feas = kd; T_feas = T; }
-                    }
-                }
-                unsigned long long w_feas = k_feas, w_room = k_room, w_all = k_all;
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) {
-                    const unsigned long long a = __shfl_xor_sync(0xFFFFFFFFu, w_feas, off);
-                    const unsigned long long b = __shfl_xor_sync(0xFFFFFFFFu, w_room, off);
-                    const unsigned long long c = __shfl_xor_sync(0xFFFFFFFFu, w_all, off);
-                    if (a > w_feas) w_feas = a;
-                    if (b < w_room) w_room = b;
-                    if (c < w_all) w_all = c;
-                }
                 int g; float T; unsigned tier;
-                if (w_feas != 0ull) {
-                    const unsigned owner = __ballot_sync(0xFFFFFFFFu, k_feas == w_feas);
-                    T = __shfl_sync(0xFFFFFFFFu, T_feas, __ffs(owner) - 1);
-                    g = (int)(0xFFFFu - (unsigned)(w_feas & 0xFFFFu)); tier = 1;
-                } else if (w_room != ~0ull) {
-                    g = (int)(w_room & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_room >> 32)); tier = 2;
-                } else {
-                    g = (int)(w_all & 0xFFFFFFFFull); T = from_orderable_bits((unsigned)(w_all >> 32)); tier = 3;
-                }
+                exhaustive_pick<false>(sh_rows, M, xs, ys, Ds, needs, 0.f, lane, g, T, tier);
                 if (lane == src) {
                     g_out[j] = g; T_out[j] = T;
                     tiers = (tiers & ~(0xFFu << (8 * j))) | (tier << (8 * j));
@@ -354,6 +394,99 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------
+// re-routing of the scan's candidates among strictly faster instances (Sec. 3.4)
+// ---------------------------------------------------------------------------------------
+
+// One thread per candidate: gathers the flagged request's columns through cand_idx, turns it
+// into the request that a token-ID migration would pose to the target (re-prefill prompt +
+// generated tokens, decode what is left, within the time that is left) and runs the same
+// search as the routing round, restricted to instances with d < d of the current instance.
+__global__ void __launch_bounds__(kRouteThreads, 4)
+reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__ cand_count, int64_t cand_capacity,
+               const int32_t *__restrict__ assigned, const int32_t *__restrict__ generated,
+               const int32_t *__restrict__ pred_len, const float *__restrict__ elapsed,
+               const float *__restrict__ slo, const int32_t *__restrict__ prompt_len, int64_t n_active,
+               int n_types_alloc,
+               const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
+               const unsigned char *__restrict__ g_start_table,
+               const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
+               int32_t *__restrict__ out_inst, float *__restrict__ out_est,
+               float *__restrict__ out_slack, uint8_t *__restrict__ out_tier, unsigned *__restrict__ status)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int M = table_info[2];
+    Tables tb;
+    stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_start_table, g_headers, table_info, tb);
+    __syncthreads();
+
+    int64_t n = *cand_count;
+    if (n > cand_capacity) n = cand_capacity;
+    const int lane = threadIdx.x & 31;
+    unsigned bad = 0;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31); base < n; base += stride) {
+        const int64_t j = base + lane;
+        const bool valid = j < n;
+        int64_t i = valid ? (int64_t)cand_idx[j] : 0;
+        if (i < 0 || i >= n_active) { i = 0; if (valid) bad |= GS_DEV_BAD_INSTANCE; }
+        int c = assigned[i], gen = generated[i], tot = pred_len[i], xin = prompt_len[i];
+        if (c < 0) { c = 0; bad |= GS_DEV_BAD_INSTANCE; }
+        if (c >= M) { c = M - 1; bad |= GS_DEV_BAD_INSTANCE; }
+        if (gen < 0) { gen = 0; bad |= GS_DEV_BAD_VALUE; }
+        if (tot < 0) { tot = 0; bad |= GS_DEV_BAD_VALUE; }
+        if (xin < 0) { xin = 0; bad |= GS_DEV_BAD_VALUE; }
+        const unsigned rem = (unsigned)max(tot - gen, 0);
+        const unsigned xu = (unsigned)xin + (unsigned)gen;                    // < 2^32
+        const unsigned long long need64 = (unsigned long long)xu + rem;
+        const unsigned need = need64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (unsigned)need64;   // kv < 2^31 anyway
+        const float x = __uint2float_rn(xu), y = __uint2float_rn(rem);
+        const float D = __fsub_rn(slo[i], elapsed[i]);                        // time left
+        const float d_cap = tb.rows[c].d;
+        float T = 0.f;
+        const float Ds = (valid && rem > 0) ? D : -1.0f;      // see route_kernel: L_out == 0 skips the search
+        int g = pick_instance<true>(tb, x, y, Ds, Ds + 1e-30f, need, d_cap, T);
+        unsigned tier = 1;
+        unsigned todo = __ballot_sync(0xFFFFFFFFu, valid && g < 0);
+        while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const float xs = __shfl_sync(0xFFFFFFFFu, x, src), ys = __shfl_sync(0xFFFFFFFFu, y, src);
+            const float Dsrc = __shfl_sync(0xFFFFFFFFu, D, src), caps = __shfl_sync(0xFFFFFFFFu, d_cap, src);
+            const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
+            int gg; float TT; unsigned tt;
+            exhaustive_pick<true>(tb.rows, M, xs, ys, Dsrc, needs, caps, lane, gg, TT, tt);
+            if (lane == src) { g = gg; T = TT; tier = tt; }
+        }
+        if (valid) {
+            out_inst[j] = g;
+            out_est[j] = T;
+            out_slack[j] = tier ? __fsub_rn(D, T) : 0.f;
+            if (out_tier) out_tier[j] = (uint8_t)tier;
+        }
+    }
+    if (bad) atomicOr(status, bad);
+}
+
+cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,
+                           const int32_t *assigned, const int32_t *generated, const int32_t *pred_len,
+                           const float *elapsed, const float *slo, const int32_t *prompt_len, int64_t n_active,
+                           int n_types, int32_t *out_inst, float *out_est, float *out_slack, uint8_t *out_tier,
+                           cudaStream_t st)
+{
+    if (cand_capacity == 0) return cudaSuccess;
+    const size_t smem = kRouteSmemFixed + kRouteSmemPerType * n_types;
+    int64_t blocks = (cand_capacity + kRouteThreads - 1) / kRouteThreads;
+    const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm[n_types];
+    if (blocks > cap) blocks = cap;
+    LaunchTimer timer(ctx, GS_K_REROUTE, st);
+    reroute_kernel<<<(unsigned)blocks, kRouteThreads, smem, st>>>(
+        cand_idx, cand_count, cand_capacity, assigned, generated, pred_len, elapsed, slo, prompt_len, n_active,
+        n_types, ctx->s.rows, ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info,
+        out_inst, out_est, out_slack, out_tier, ctx->s.status);
+    return cudaGetLastError();
+}
+
 // Raises the dynamic shared-memory limit of the route kernels and looks up how many CTAs fit
 // on an SM for each table size (called once per context).
 cudaError_t configure_route(gs_ctx *ctx)
@@ -363,6 +496,8 @@ cudaError_t configure_route(gs_ctx *ctx)
                                          (int)(max_smem + kRouteSmemHist));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(route_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
     for (int t = 0; t <= GS_MAX_TYPES; ++t) {
         int occ = 0;

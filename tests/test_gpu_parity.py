@@ -395,3 +395,93 @@ def test_coefficients_the_bounds_cannot_use_take_the_exhaustive_path(gs):
     np.testing.assert_array_equal(got.instance_idx, ref.instance_idx)
     np.testing.assert_array_equal(got.tier, ref.tier)
     assert gs.device_status() & DeviceStatus.BAD_VALUE
+
+
+# --------------------------------------------------------------------------------------
+# re-routing of the scan's candidates (Sec. 3.4)
+# --------------------------------------------------------------------------------------
+
+def gpu_scan_and_reroute(gs, pool, act, prompt, alpha):
+    dev = gs.device
+    cols = [torch.from_numpy(c).to(dev) for c in act.columns()]
+    x = torch.from_numpy(prompt).to(dev)
+    n = act.n
+    bits = torch.zeros(max((n + 31) // 32, 1), dtype=torch.int32, device=dev)
+    cand = torch.full((max(n, 1),), -9, dtype=torch.int32, device=dev)
+    count = torch.zeros(1, dtype=torch.int64, device=dev)
+    gs.risk_scan(*cols, pool, bits, cand, count)
+    new_inst = torch.full((max(n, 1),), -7, dtype=torch.int32, device=dev)
+    est = torch.full((max(n, 1),), float("nan"), dtype=torch.float32, device=dev)
+    slack = torch.full((max(n, 1),), float("nan"), dtype=torch.float32, device=dev)
+    tier = torch.full((max(n, 1),), 9, dtype=torch.uint8, device=dev)
+    gs.reroute_candidates(cand, count, *cols, x, pool, alpha, new_inst, est, slack, tier)
+    torch.cuda.synchronize(dev)
+    c = int(count.item())
+    return (cand.cpu().numpy()[:c], new_inst.cpu().numpy(), est.cpu().numpy(), slack.cpu().numpy(),
+            tier.cpu().numpy(), c)
+
+
+def check_reroute(gs, types, inst, act, prompt, alpha=0.5):
+    pool = pool_of(gs, types, inst)
+    t32 = oracle.instance_table(types, inst, alpha, "f32")
+    t64 = oracle.instance_table(types, inst, alpha, "f64")
+    cand, new_inst, est, slack, tier, c = gpu_scan_and_reroute(gs, pool, act, prompt, alpha)
+    ref_cand = np.nonzero(oracle.risk(t32, *act.columns(), threads=8).flag)[0].astype(np.int32)
+    np.testing.assert_array_equal(cand, ref_cand)
+    ref = oracle.reroute(t32, ref_cand, *act.columns(), prompt)
+    np.testing.assert_array_equal(new_inst[:c], ref.new_instance)
+    np.testing.assert_array_equal(tier[:c], ref.tier)
+    np.testing.assert_array_equal(est[:c].view(np.uint32), ref.est_ms.view(np.uint32))
+    np.testing.assert_array_equal(slack[:c].view(np.uint32), ref.slack_ms.view(np.uint32))
+    assert (new_inst[c:] == -7).all() and (tier[c:] == 9).all()       # nothing past the count is touched
+    ref64 = oracle.reroute(t64, ref_cand, *act.columns(), prompt)
+    agree = ref64.new_instance == ref.new_instance
+    same = agree & (ref.tier > 0)
+    err = np.abs(est[:c][same] - ref64.est_ms[same]) / np.maximum(np.abs(ref64.est_ms[same]), 1e-30)
+    assert err.size == 0 or err.max() <= REL_TOL
+    assert agree.size == 0 or agree.mean() > 0.999       # the two precisions part only at near-ties
+    return ref
+
+
+@pytest.mark.parametrize("cfg_id", [0, 1, 2])
+def test_reroute_full_size(gs, cfg_id):
+    wl = W.make_workload(cfg_id)
+    prompt = W.make_requests(wl.cfg, wl.types, seed=500 + cfg_id, n=wl.active.n).prompt_len
+    ref = check_reroute(gs, wl.types, wl.instances, wl.active, prompt)
+    print(f"cfg {cfg_id}: {len(ref.tier)} candidates, tiers 0..3 = {[int((ref.tier == k).sum()) for k in range(4)]}")
+    assert gs.device_status() == 0
+
+
+def test_reroute_config3_sample(gs):
+    """Largest pool (1,024 instances of 8 types) on 2,097,152 active requests."""
+    wl = W.make_workload(3, n_requests=16, n_active=2_097_152)
+    prompt = W.make_requests(wl.cfg, wl.types, seed=503, n=wl.active.n).prompt_len
+    ref = check_reroute(gs, wl.types, wl.instances, wl.active, prompt)
+    assert {0, 1, 2} <= set(ref.tier.tolist())
+
+
+def test_reroute_handworked(gs):
+    from test_oracle_pins import fixture_pool, read_rows
+    for name, cur, elapsed, slo, k0, k1, g, est, slack, tier in read_rows("handworked_reroute.txt"):
+        types, inst = fixture_pool((int(k0), int(k1), 100000))
+        act = W.ActiveSet(np.array([int(cur)], np.int32), np.array([50], np.int32), np.array([200], np.int32),
+                          np.array([float(elapsed)], np.float32), np.array([float(slo)], np.float32))
+        pool = pool_of(gs, types, inst)
+        cand, new_inst, e, s, t, c = gpu_scan_and_reroute(gs, pool, act, np.array([1000], np.int32), 0.5)
+        if c == 0:          # the request is not at risk where it runs: nothing to re-route
+            continue
+        assert new_inst[0] == int(g) and t[0] == int(tier), name
+        assert e[0] == pytest.approx(float(est), rel=REL_TOL), name
+
+
+@pytest.mark.parametrize("case", [0, 3, 4, 7, 8, 10])
+def test_reroute_on_adversarial_pools(gs, case):
+    rng = np.random.default_rng(2000 + case)
+    types, inst = _random_pool(rng, **FUZZ_CASES[case])
+    cfg = W.CONFIGS[3]
+    act = W.make_active(cfg, types, inst.n_instances, seed=case, n=20_000)
+    act.generated_tokens[::7] = 0
+    act.generated_tokens[1::11] = act.pred_len[1::11]            # nothing left to decode
+    prompt = np.clip(np.rint(np.exp(rng.normal(6.5, 1.2, act.n))), 0, 1 << 20).astype(np.int32)
+    check_reroute(gs, types, inst, act, prompt, alpha=0.25)
+    assert gs.device_status() == 0
