@@ -307,6 +307,28 @@ def run_gpu(args):
         if n:
             kernel_ms[name] = (ms, n)
     gs.timing_enable(False)
+
+    # ---- the step after the scan (not part of the timed step): re-route its candidates ----
+    reroute = None
+    if not args.no_reroute:
+        a_prompt = torch.from_numpy(W.make_requests(cfg, wl.types, seed=rank_seed(args.config, rank) + 7,
+                                                    n=A).prompt_len).to(dev)
+        r_inst = torch.empty(A, dtype=torch.int32, device=dev)
+        r_est = torch.empty(A, dtype=torch.float32, device=dev)
+        r_slack = torch.empty(A, dtype=torch.float32, device=dev)
+        gs.reroute_candidates(cand, count, *act, a_prompt, pool, alpha, r_inst, r_est, r_slack, stream=stream)
+        barrier()
+        gs.timing_enable(True)
+        for _ in range(max(3, args.steps // 2)):
+            gs.reroute_candidates(cand, count, *act, a_prompt, pool, alpha, r_inst, r_est, r_slack, stream=stream)
+        barrier()
+        ms, n_l = gs.timing_read(KERNEL_NAMES.index("reroute"))
+        gs.timing_enable(False)
+        n_cand = int(count.item())
+        reroute = {"candidates": n_cand, "avg_us": ms / n_l * 1e3,
+                   "candidates_per_s": n_cand / (ms / n_l * 1e-3),
+                   "algorithmic_GBps": n_cand * (4 + 24 + 12) / (ms / n_l * 1e-3) / 1e9}
+        del a_prompt, r_inst, r_est, r_slack
     t_wait = time.perf_counter()
     while len(sampler.rows) < 4 and time.perf_counter() - t_wait < 3.0:
         step()                                   # keep the same load up for the sampler (untimed)
@@ -405,7 +427,7 @@ def run_gpu(args):
         "route_requests_per_s": world * N / (route_ms * 1e-3) if route_ms else None,
         "step_hbm_frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "flagged_fraction": flagged / A, "device_status": status,
-        "roofline": roofline, "issue": issue, "kernels": per_kernel,
+        "roofline": roofline, "issue": issue, "kernels": per_kernel, "reroute": reroute,
         "kernel_timing": "serial pass of %d steps on one stream after the timed region, %.4f ms/step" % (
             args.steps, serial_ms_per_step),
         "e2e": None if args.no_e2e else
@@ -429,6 +451,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-reroute", action="store_true", help="skip the untimed re-route measurement")
     ap.add_argument("--serial", action="store_true", help="route and scan on one stream instead of two")
     ap.add_argument("--print-kernel-hash", action="store_true", help="print the hash PROFILED_ROUTE refers to")
     args = ap.parse_args()
