@@ -18,8 +18,10 @@
 // argmax d_g over the feasible set, ties to the smallest index.
 //
 // A request for which this finds nothing (no feasible instance: the fallback of Algorithm 1)
-// is finished right away by its whole warp, which scores every instance, lanes across
-// instances, with shuffle reductions for the argmin.
+// is finished by the same thread with a branch-and-bound minimum of T over the same tables.
+// Only requests that the tables cannot serve (L_out == 0, or coefficients for which the bounds
+// do not hold) are handed to their whole warp, which scores every instance, lanes across
+// instances, with shuffle reductions.
 #include "gs_internal.cuh"
 
 namespace gs {
@@ -73,6 +75,12 @@ struct Tables {
 };
 
 constexpr unsigned kNoRow = 0xFFFFFFFFu;
+// Lanes of a warp that must need the fallback before each runs its own search; below that the
+// warp-wide scoring of every instance is the shorter way.
+#ifndef GS_THREAD_FALLBACK_MIN
+#define GS_THREAD_FALLBACK_MIN 3
+#endif
+constexpr int kThreadFallbackMin = GS_THREAD_FALLBACK_MIN;
 
 // Bound test of one row: false only if the row certainly cannot be chosen.
 template <bool kCapped>
@@ -174,6 +182,79 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
     }
     T_out = T_best;
     return g_best;
+}
+
+// Fallback of Algorithm 1 for one request, by one thread: the smallest T among instances with
+// KV room (tier 2), else among all (tier 3); ties to the smallest index.  Branch and bound over
+// the same tables: the best T found so far plays the deadline's part in the bound tests, so a
+// row is skipped only when its exactly-rounded T is proven larger.  Types are visited fastest
+// first and each type's rows from its smallest d upwards, which is where the minimum lives;
+// the walk up a type stops at the first group whose smallest d alone already exceeds the best.
+// Returns -1 with tier 0 only when kCapped and no instance has d < d_cap.
+struct Pick { int g; float T; unsigned tier; };
+
+template <bool kCapped>
+__device__ __forceinline__ Pick fallback_pick(const TypeHeader *headers, const uint2 *row_bounds, const Row *rows,
+                                           int n_types, float x, float y, unsigned need, float d_cap)
+{
+    Tables tb;
+    tb.headers = headers; tb.row_bounds = row_bounds; tb.rows = rows; tb.start_table = nullptr; tb.n_types = n_types;
+    unsigned tier_out = 0;
+    int g_best = -1;
+    float T_best = __int_as_float(0x7F800000);            // +inf
+#pragma unroll 1
+    for (int pass = 0; pass < 2 && g_best < 0; ++pass) {  // pass 0: instances with KV room only
+        const bool any_kv = pass == 1;
+#pragma unroll 1
+        for (int t = tb.n_types - 1; t >= 0; --t) {
+            const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);   // p_lo, q_lo, d_lo, d_max
+            if (kCapped && !(h.z < d_cap)) continue;
+            float R = __fmaf_rn(-h.x, x, T_best) + 1e-30f;
+            if (!(__fmaf_rn(h.z, y, h.y) <= R)) continue;
+            const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, ..
+#pragma unroll 1
+            for (int k = geo.x + geo.y - 8; k >= geo.x; k -= 8) {
+                const char *grp = reinterpret_cast<const char *>(tb.row_bounds + k);
+                const int sw = (k >> 4) & 3;                // see row_slot()
+                uint4 r[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) r[c] = *reinterpret_cast<const uint4 *>(grp + ((c ^ sw) << 4));
+                // rows k .. k+7 in order: (r[0].x,y) (r[0].z,w) (r[1].x,y) ...; larger d first.
+                // the last real row of the group has the group's smallest d: if even q0 with that
+                // d misses the best, so does everything from here up
+                float d_min = 0.f;                          // a group of padding only: nothing to conclude
+                bool have = false;
+#pragma unroll
+                for (int c = 3; c >= 0; --c) {              // padding (NaN q) only follows a type's last row
+                    if (!have && __uint_as_float(r[c].z) == __uint_as_float(r[c].z)) { d_min = __uint_as_float(r[c].w); have = true; }
+                    if (!have && __uint_as_float(r[c].x) == __uint_as_float(r[c].x)) { d_min = __uint_as_float(r[c].y); have = true; }
+                }
+                if (!(__fmaf_rn(d_min, y, h.y) <= R)) break;
+#pragma unroll
+                for (int c = 3; c >= 0; --c) {
+#pragma unroll
+                    for (int e = 1; e >= 0; --e) {
+                        const unsigned qw = e ? r[c].z : r[c].x, dw = e ? r[c].w : r[c].y;
+                        if (!row_may_pass<kCapped>(qw, dw, y, R, d_cap)) continue;
+                        const int inst = (int)(qw & kRowTagMask);
+                        const Row row = tb.rows[inst];
+                        if (kCapped && !(row.d < d_cap)) continue;
+                        if (!any_kv && !(need <= (unsigned)row.kv)) continue;
+                        const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));   // Eq. 2, H = 0
+                        if (T < T_best || (T == T_best && inst < g_best) || g_best < 0) {
+                            T_best = T; g_best = inst;
+                            R = __fmaf_rn(-h.x, x, T_best) + 1e-30f;
+                        }
+                    }
+                }
+            }
+        }
+        tier_out = any_kv ? 3u : 2u;
+    }
+    if (g_best < 0) { tier_out = 0u; T_best = 0.f; }
+    Pick r;
+    r.g = g_best; r.T = T_best; r.tier = tier_out;
+    return r;
 }
 
 // Copies the round's tables into shared memory (all threads of the CTA; the caller
@@ -318,23 +399,56 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             // tag bits make a zero coefficient a denormal)
             const float Dj = (valid && yi[j] > 0) ? D[j] : -1.0f;
             g_out[j] = pick_instance<false>(tb, x, y, Dj, Dj + 1e-30f, need, 0.f, T_out[j]);
-
-            // ---- no feasible instance found: the whole warp scores every instance -------------
-            unsigned todo = __ballot_sync(0xFFFFFFFFu, valid && g_out[j] < 0);
-            while (todo) {
-                const int src = __ffs(todo) - 1;
-                todo &= todo - 1;
-                const float xs = __shfl_sync(0xFFFFFFFFu, x, src), ys = __shfl_sync(0xFFFFFFFFu, y, src);
-                const float Ds = __shfl_sync(0xFFFFFFFFu, D[j], src);
-                const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
-                int g; float T; unsigned tier;
-                exhaustive_pick<false>(sh_rows, M, xs, ys, Ds, needs, 0.f, lane, g, T, tier);
-                if (lane == src) {
-                    g_out[j] = g; T_out[j] = T;
-                    tiers = (tiers & ~(0xFFu << (8 * j))) | (tier << (8 * j));
+        }
+        // ---- requests still without an instance: nothing is feasible (the fallback of
+        // Algorithm 1), or L_out == 0, or tables whose bounds cannot be used ----------------------
+        unsigned pend = 0, mine = 0;                 // bit j: request j of this lane is open / may search by itself
+#pragma unroll
+        for (int j = 0; j < kReqPerThread; ++j) {
+            const bool open = first + j < n && g_out[j] < 0;
+            pend |= (unsigned)open << j;
+            mine |= (unsigned)(open && yi[j] > 0 && tb.n_types > 0) << j;
+        }
+        if (__any_sync(0xFFFFFFFFu, pend != 0)) {
+            // several in the warp: each lane searches for its own; few: the warp shares each one
+            const int n_fall = (int)__reduce_add_sync(0xFFFFFFFFu, (unsigned)__popc(mine));
+            if (n_fall >= kThreadFallbackMin) {
+#pragma unroll
+                for (int j = 0; j < kReqPerThread; ++j)
+                    if ((mine >> j) & 1u) {
+                        const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];
+                        const Pick r = fallback_pick<false>(tb.headers, tb.row_bounds, tb.rows, tb.n_types,
+                                                            __int2float_rn(xi[j]), __int2float_rn(yi[j]), need, 0.f);
+                        g_out[j] = r.g; T_out[j] = r.T;
+                        tiers = (tiers & ~(0xFFu << (8 * j))) | (r.tier << (8 * j));
+                        pend &= ~(1u << j);
+                    }
+            }
+#pragma unroll
+            for (int j = 0; j < kReqPerThread; ++j) {
+                unsigned todo = __ballot_sync(0xFFFFFFFFu, (pend >> j) & 1u);
+                const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];
+                while (todo) {
+                    const int src = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const float xs = __shfl_sync(0xFFFFFFFFu, __int2float_rn(xi[j]), src);
+                    const float ys = __shfl_sync(0xFFFFFFFFu, __int2float_rn(yi[j]), src);
+                    const float Ds = __shfl_sync(0xFFFFFFFFu, D[j], src);
+                    const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
+                    int g; float T; unsigned tier;
+                    exhaustive_pick<false>(sh_rows, M, xs, ys, Ds, needs, 0.f, lane, g, T, tier);
+                    if (lane == src) {
+                        g_out[j] = g; T_out[j] = T;
+                        tiers = (tiers & ~(0xFFu << (8 * j))) | (tier << (8 * j));
+                    }
                 }
             }
-            if (kAccumulate) accumulate_choice(hist, M, valid ? g_out[j] : -1, (unsigned)xi[j], need);
+        }
+        if (kAccumulate) {
+#pragma unroll
+            for (int j = 0; j < kReqPerThread; ++j)
+                accumulate_choice(hist, M, first + j < n ? g_out[j] : -1, (unsigned)xi[j],
+                                  (unsigned)xi[j] + (unsigned)yi[j]);
         }
         if (kReqPerThread == 4 && first + kReqPerThread <= n) {
             __stcs(reinterpret_cast<int4 *>(out_idx + first), make_int4(g_out[0], g_out[1], g_out[2], g_out[3]));
@@ -447,7 +561,15 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
         const float Ds = (valid && rem > 0) ? D : -1.0f;      // see route_kernel: L_out == 0 skips the search
         int g = pick_instance<true>(tb, x, y, Ds, Ds + 1e-30f, need, d_cap, T);
         unsigned tier = 1;
-        unsigned todo = __ballot_sync(0xFFFFFFFFu, valid && g < 0);
+        bool settled = g >= 0;
+        const bool fall = valid && !settled && rem > 0 && tb.n_types > 0;
+        const int n_fall = __popc(__ballot_sync(0xFFFFFFFFu, fall));           // all lanes vote
+        if (fall && n_fall >= kThreadFallbackMin) {
+            const Pick r = fallback_pick<true>(tb.headers, tb.row_bounds, tb.rows, tb.n_types, x, y, need, d_cap);
+            g = r.g; T = r.T; tier = r.tier;                                // may settle on "no move"
+            settled = true;
+        }
+        unsigned todo = __ballot_sync(0xFFFFFFFFu, valid && !settled);
         while (todo) {
             const int src = __ffs(todo) - 1;
             todo &= todo - 1;

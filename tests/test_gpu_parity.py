@@ -378,6 +378,32 @@ def test_pruned_search_is_exact_on_adversarial_pools(gs, case):
     assert gs.device_status() == 0
 
 
+@pytest.mark.parametrize("share", [1.0, 0.3, 0.01])
+@pytest.mark.parametrize("scarce_kv", [False, True])
+def test_fallback_heavy_and_sparse_batches(gs, share, scarce_kv):
+    """Batches in which all, many or only a few requests have no feasible instance: the
+    fallback's minimum of T (with and without KV room) is the definition's whichever way the
+    kernel chooses to compute it, ties to the smallest index."""
+    rng = np.random.default_rng(4242)
+    types, inst = _random_pool(rng, 1024, 8, scarce_kv=scarce_kv)
+    inst.queued_prefill_tokens[::3] = 0            # groups of instances with equal estimates
+    inst.q_ema_ms[::3] = 0.0
+    inst.decode_batch[::3] = 5
+    pool = pool_of(gs, types, inst)
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    n = 20000
+    x = np.clip(np.rint(np.exp(rng.normal(6.5, 1.0, n))), 1, 1 << 18).astype(np.int32)
+    y = np.clip(np.rint(np.exp(rng.normal(5.0, 1.5, n))), 1, 1 << 18).astype(np.int32)
+    T = _canonical_T(t32, x, y)
+    hopeless = rng.random(n) < share
+    D = np.where(hopeless, T.min(axis=1) * np.float32(0.9), T.max(axis=1) * np.float32(1.1)).astype(np.float32)
+    req = W.RequestBatch(x, y, D)
+    got = gpu_route(gs, pool, req, 0.5)
+    ref = oracle.route(t32, *req.columns(), threads=4)
+    assert_route_matches_f32_oracle(got, ref)
+    assert (ref.tier[hopeless] >= 2).all() and (3 in set(ref.tier.tolist())) == scarce_kv
+
+
 def test_coefficients_the_bounds_cannot_use_take_the_exhaustive_path(gs):
     """A negative type constant makes lower bounds meaningless; the kernel then scores every
     instance for every request and still returns the definition's answer."""
