@@ -153,6 +153,45 @@ def route(table: InstanceTable, prompt_len, pred_decode_len, slo_ms, threads: in
     return out
 
 
+def route_prefix(table: InstanceTable, prompt_len, pred_decode_len, slo_ms, prefix_inst, prefix_hit_len,
+                 threads: int = 1) -> RouteResult:
+    """Algorithm 1 with the prefix-cache term of Eq. 2.  ``prefix_inst`` / ``prefix_hit_len`` are
+    int32 arrays of shape (n_slots, N): the instances on which request r has a cached prefix and
+    the hit lengths (see the C file for the reading of empty, invalid and duplicate slots)."""
+    x = _c(prompt_len, np.int32); y = _c(pred_decode_len, np.int32); D = _c(slo_ms, np.float32)
+    N = x.shape[0]
+    pi = _c(prefix_inst, np.int32).reshape(-1, N) if N else np.zeros((0, 0), np.int32)
+    ph = _c(prefix_hit_len, np.int32).reshape(-1, N) if N else np.zeros((0, 0), np.int32)
+    assert pi.shape == ph.shape
+    K = pi.shape[0]
+    real = np.float64 if table.precision == "f64" else np.float32
+    out = RouteResult(np.empty(N, np.int32), np.empty(N, real), np.empty(N, real),
+                      np.empty(N, np.uint8), 0)
+    if N == 0:
+        return out
+    fn = getattr(_L(), f"gso_route_prefix_{table.precision}")
+    threads = max(1, min(int(threads), N))
+    bounds = np.linspace(0, N, threads + 1).astype(np.int64)
+    stats = [C.c_uint(0) for _ in range(threads)]
+
+    def run(i):
+        lo, hi = int(bounds[i]), int(bounds[i + 1])
+        pi_c = np.ascontiguousarray(pi[:, lo:hi]); ph_c = np.ascontiguousarray(ph[:, lo:hi])
+        fn(C.c_int64(hi - lo), _p(x[lo:hi]), _p(y[lo:hi]), _p(D[lo:hi]), C.c_int32(K), _p(pi_c), _p(ph_c),
+           C.c_int32(table.n_instances), _p(table.q), _p(table.p), _p(table.d), _p(table.kv),
+           _p(out.instance_idx[lo:hi]), _p(out.est_e2e_ms[lo:hi]), _p(out.slack_ms[lo:hi]),
+           _p(out.tier[lo:hi]), C.byref(stats[i]))
+
+    if threads == 1:
+        run(0)
+    else:
+        with ThreadPoolExecutor(threads) as ex:
+            list(ex.map(run, range(threads)))
+    for s in stats:
+        out.status |= s.value
+    return out
+
+
 @dataclass
 class RiskResult:
     flag: np.ndarray        # uint8[A]

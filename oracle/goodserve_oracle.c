@@ -6,7 +6,8 @@
  * against it.  It shares no code with the CUDA path and nothing in the product may call it.
  *
  * What is stated here, and where the paper defines it:
- *   - latency model  T(r,g) = q_g + p_g * (L_in_r - H_{r,g}) + d_g * L_out_r     (Eq. 2), with H = 0
+ *   - latency model  T(r,g) = q_g + p_g * (L_in_r - H_{r,g}) + d_g * L_out_r     (Eq. 2); H = 0 in
+ *     gso_route_*, sparse per-request hits in gso_route_prefix_*
  *   - queue-delay smoothing  q_g <- alpha * w_g + (1 - alpha) * q_g              (Algorithm 1, EMA step)
  *   - feasible set  C = { g : T(r,g) <= D_r }, restricted to instances whose memory
  *     can hold the request                                                      (Algorithm 1; Sec. 3.1 constraints)
@@ -336,4 +337,99 @@ void gso_reroute_f32(int64_t n_cand, const int32_t *cand_idx,
                      unsigned *status)
 {
     GSO_REROUTE_BODY(float, fmaf(d[g], y, fmaf(p[g], x, q[g])))
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Algorithm 1 with the prefix-cache term of Eq. 2                                        */
+/*                                                                                        */
+/* H_{r,g} arrives in sparse form: n_slots (instance, hit length) pairs per request,      */
+/* slot-major arrays of n_slots * N entries (slot k of request r at k * N + r).           */
+/* Reading:                                                                               */
+/*   - a slot with a negative instance is empty; an instance >= M names nothing and is    */
+/*     ignored (status bit);                                                              */
+/*   - a hit length is clamped into [0, L_in] (a negative one, or one longer than the     */
+/*     prompt, sets a status bit);                                                        */
+/*   - an instance named by several slots keeps its longest hit;                          */
+/*   - every other pair has H = 0;                                                        */
+/*   - the memory constraint is unchanged: L_in + L_out <= free KV tokens.                */
+/* Everything else is the loop of gso_route_* with T taken from the full Eq. 2.           */
+/* ------------------------------------------------------------------------------------ */
+
+/* ReusePrefix(r, g): the hit length of request r on instance g */
+static int32_t reuse_prefix(int64_t r, int32_t g, int64_t N, int32_t n_slots,
+                            const int32_t *prefix_inst, const int32_t *prefix_hit_len, int32_t L_in)
+{
+    int32_t H = 0;
+    for (int32_t k = 0; k < n_slots; ++k) {
+        if (prefix_inst[(int64_t)k * N + r] != g) continue;
+        int32_t h = prefix_hit_len[(int64_t)k * N + r];
+        if (h < 0) h = 0;
+        if (h > L_in) h = L_in;
+        if (h > H) H = h;
+    }
+    return H;
+}
+
+/* status bits for the slots of request r (kept apart from the search so that it stays plain) */
+static void check_slots(int64_t r, int64_t N, int32_t n_slots, int32_t M, const int32_t *prefix_inst,
+                        const int32_t *prefix_hit_len, int32_t L_in, unsigned *status)
+{
+    for (int32_t k = 0; k < n_slots; ++k) {
+        int32_t g = prefix_inst[(int64_t)k * N + r];
+        if (g < 0) continue;
+        if (g >= M) { *status |= GSO_BAD_INSTANCE; continue; }
+        int32_t h = prefix_hit_len[(int64_t)k * N + r];
+        if (h < 0 || h > L_in) *status |= GSO_BAD_VALUE;
+    }
+}
+
+#define GSO_ROUTE_PREFIX_BODY(REAL, LAT)                                                      \
+    for (int64_t r = 0; r < N; ++r) {                                                         \
+        int32_t xi = clamp_count(prompt_len[r], status);                                      \
+        int32_t yi = clamp_count(pred_decode_len[r], status);                                 \
+        REAL y = (REAL)yi;                                                                    \
+        REAL D = (REAL)slo_ms[r];                                                             \
+        int64_t need = (int64_t)xi + (int64_t)yi;                                             \
+        check_slots(r, N, n_slots, M, prefix_inst, prefix_hit_len, xi, status);               \
+        int32_t best_c = -1, best_k = -1, best_a = -1;                                        \
+        REAL d_c = 0, T_c = 0, T_k = 0, T_a = 0;                                              \
+        for (int32_t g = 0; g < M; ++g) {                                                     \
+            int32_t H = reuse_prefix(r, g, N, n_slots, prefix_inst, prefix_hit_len, xi);      \
+            REAL xh = (REAL)(xi - H);                      /* tokens left to prefill on g */  \
+            REAL T = LAT;                                  /* Eq. 2 */                        \
+            int kv_ok = need <= kv[g];                                                        \
+            if (kv_ok && T <= D) {                                                            \
+                if (best_c < 0 || d[g] > d_c) { best_c = g; d_c = d[g]; T_c = T; }            \
+            }                                                                                 \
+            if (kv_ok && (best_k < 0 || T < T_k)) { best_k = g; T_k = T; }                    \
+            if (best_a < 0 || T < T_a) { best_a = g; T_a = T; }                               \
+        }                                                                                     \
+        int32_t g_star; REAL T_star; uint8_t tr;                                              \
+        if (best_c >= 0)      { g_star = best_c; T_star = T_c; tr = 1; }                      \
+        else if (best_k >= 0) { g_star = best_k; T_star = T_k; tr = 2; }                      \
+        else                  { g_star = best_a; T_star = T_a; tr = 3; }                      \
+        instance_idx[r] = g_star;                                                             \
+        est_e2e_ms[r] = T_star;                                                               \
+        slack_ms[r] = D - T_star;                                                             \
+        if (tier) tier[r] = tr;                                                               \
+    }
+
+void gso_route_prefix_f64(int64_t N, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                          const float *slo_ms, int32_t n_slots, const int32_t *prefix_inst,
+                          const int32_t *prefix_hit_len,
+                          int32_t M, const double *q, const double *p, const double *d, const int64_t *kv,
+                          int32_t *instance_idx, double *est_e2e_ms, double *slack_ms, uint8_t *tier,
+                          unsigned *status)
+{
+    GSO_ROUTE_PREFIX_BODY(double, q[g] + p[g] * xh + d[g] * y)
+}
+
+void gso_route_prefix_f32(int64_t N, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                          const float *slo_ms, int32_t n_slots, const int32_t *prefix_inst,
+                          const int32_t *prefix_hit_len,
+                          int32_t M, const float *q, const float *p, const float *d, const int64_t *kv,
+                          int32_t *instance_idx, float *est_e2e_ms, float *slack_ms, uint8_t *tier,
+                          unsigned *status)
+{
+    GSO_ROUTE_PREFIX_BODY(float, fmaf(d[g], y, fmaf(p[g], xh, q[g])))
 }

@@ -560,3 +560,155 @@ def test_reroute_never_moves_to_a_slower_or_equal_instance():
     assert (res.tier[moved] > 0).all() and (res.tier[~moved] == 0).all()
     t1 = res.tier == 1
     assert (res.slack_ms[t1] >= 0).all()
+
+
+# --------------------------------------------------------------------------------------
+# prefix-cache term of Eq. 2 (sparse H)
+# --------------------------------------------------------------------------------------
+
+def parse_slots(text):
+    if text == "-":
+        return np.zeros((0, 1), np.int32), np.zeros((0, 1), np.int32)
+    pairs = [tuple(int(v) for v in item.split(":")) for item in text.split(",")]
+    return (np.array([[g] for g, _ in pairs], np.int32), np.array([[h] for _, h in pairs], np.int32))
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_handworked_prefix(prec):
+    for name, x, y, D, k0, k1, k2, slots, g, est, slack, tier in read_rows("handworked_prefix.txt"):
+        types, inst = fixture_pool((int(k0), int(k1), int(k2)))
+        tab = oracle.instance_table(types, inst, 0.5, prec)
+        pi, ph = parse_slots(slots)
+        res = oracle.route_prefix(tab, [int(x)], [int(y)], [float(D)], pi, ph)
+        assert res.instance_idx[0] == int(g), name
+        assert res.tier[0] == int(tier), name
+        assert res.est_e2e_ms[0] == pytest.approx(float(est), rel=1e-5), name
+        assert res.slack_ms[0] == pytest.approx(float(slack), rel=1e-4, abs=2e-3), name
+        assert (res.status != 0) == (name in ("hit_longer_than_prompt", "empty_and_unknown_slots")), name
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_prefix_without_hits_is_plain_routing(prec):
+    wl = W.make_workload(1, n_requests=3000, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, prec)
+    cols = wl.requests.columns()
+    plain = oracle.route(tab, *cols)
+    n = len(cols[0])
+    rng = np.random.default_rng(5)
+    some_inst = rng.integers(0, tab.n_instances, (2, n)).astype(np.int32)
+    for pi, ph in ((np.zeros((0, n), np.int32), np.zeros((0, n), np.int32)),          # no slots at all
+                   (np.full((2, n), -1, np.int32), np.full((2, n), 77, np.int32)),    # only empty slots
+                   (some_inst, np.zeros((2, n), np.int32))):                          # hits of length 0
+        res = oracle.route_prefix(tab, *cols, pi, ph)
+        for a, b in ((res.instance_idx, plain.instance_idx), (res.tier, plain.tier),
+                     (res.est_e2e_ms, plain.est_e2e_ms), (res.slack_ms, plain.slack_ms)):
+            np.testing.assert_array_equal(a, b)
+        assert res.status == 0
+
+
+def dense_hits(pi, ph, x, M):
+    """H as a dense (N, M) matrix, built with numpy scatter-max (not the oracle's slot loop)."""
+    n = len(x)
+    H = np.zeros((n, M), np.int64)
+    for k in range(pi.shape[0]):
+        ok = (pi[k] >= 0) & (pi[k] < M)
+        rows = np.nonzero(ok)[0]
+        np.maximum.at(H, (rows, pi[k][rows]), np.clip(ph[k][rows], 0, x[rows]))
+    return H
+
+
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("n_slots", [1, 3])
+def test_prefix_matches_dense_statement(prec, n_slots):
+    """Eq. 2 evaluated over a dense H matrix with numpy, then the declarative post-condition of
+    Algorithm 1 on that T: nothing preferred over the answer exists."""
+    rng = np.random.default_rng(31 + n_slots)
+    wl = W.make_workload(1, n_requests=1500, n_active=8)
+    inst = wl.instances.copy()
+    inst.free_kv_tokens[rng.random(inst.n_instances) < 0.5] = 300        # all three tiers occur
+    tab = oracle.instance_table(wl.types, inst, 0.5, prec)
+    x, y, D = (a.copy() for a in wl.requests.columns())
+    D[::3] *= 0.4
+    x[::40] = 1 << 22                                                   # no instance has room for these
+    M = tab.n_instances
+    pi = rng.integers(-1, M + 1, (n_slots, len(x))).astype(np.int32)     # -1 = empty, M = unknown
+    ph = rng.integers(-5, 20000, (n_slots, len(x))).astype(np.int32)     # some negative, some > L_in
+    # a third of the deadlines sit just below the hit-free estimate of the request's first
+    # cached instance, so that the hit decides whether that instance is feasible
+    g0 = np.clip(pi[0], 0, M - 1)
+    T_plain = tab.q[g0].astype(np.float64) + tab.p[g0] * x.astype(np.float64) + tab.d[g0] * y.astype(np.float64)
+    D[1::3] = (T_plain * 0.9995).astype(np.float32)[1::3]
+    res = oracle.route_prefix(tab, x, y, D, pi, ph)
+    H = dense_hits(pi, ph, x, M)
+    q, p, d = (np.asarray(a, np.float64) for a in (tab.q, tab.p, tab.d))
+    xh = (x[:, None] - H).astype(np.float64)
+    if prec == "f64":
+        T = q + p * xh + d * y[:, None].astype(np.float64)
+    else:
+        t1 = (p * xh + q).astype(np.float32)
+        T = (d * y[:, None].astype(np.float64) + t1).astype(np.float32).astype(np.float64)
+    idx_all = np.arange(M)
+    seen = set()
+    for r in range(len(x)):
+        ok = (int(x[r]) + int(y[r])) <= np.asarray(tab.kv)
+        feas = ok & (T[r] <= float(D[r]))
+        g = int(res.instance_idx[r])
+        if feas.any():
+            assert res.tier[r] == 1 and feas[g]
+            assert not (feas & ((d > d[g]) | ((d == d[g]) & (idx_all < g)))).any()
+        else:
+            pool = ok if ok.any() else np.ones_like(ok)
+            assert res.tier[r] == (2 if ok.any() else 3) and pool[g]
+            assert not (pool & ((T[r] < T[r, g]) | ((T[r] == T[r, g]) & (idx_all < g)))).any()
+        assert res.est_e2e_ms[r] == pytest.approx(T[r, g], rel=1e-12 if prec == "f64" else 0, abs=0)
+        seen.add(int(res.tier[r]))
+    assert seen == {1, 2, 3}
+    assert res.status == (4 | 1)        # out-of-range hit lengths and unknown instances were seen
+    plain = oracle.route(tab, x, y, D)
+    assert (plain.instance_idx != res.instance_idx).mean() > 0.05       # the hits do change answers
+
+
+def test_constant_hit_on_one_instance_is_a_queue_credit():
+    """If every request has the same hit h on instance g, Eq. 2 reads
+    (q_g - p_g h) + p_g L_in + d_g L_out on g: plain routing against a table whose q_g is
+    lowered by p_g h.  Checked against route() (pinned above) in double precision."""
+    wl = W.make_workload(1, n_requests=4000, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, "f64")
+    x, y, D = wl.requests.columns()
+    g, h = 5, 16                                   # every prompt has at least 16 tokens
+    assert x.min() >= h
+    pi = np.full((1, len(x)), g, np.int32)
+    ph = np.full((1, len(x)), h, np.int32)
+    res = oracle.route_prefix(tab, x, y, D, pi, ph)
+    q2 = tab.q.copy()
+    q2[g] -= tab.p[g] * h
+    ref = oracle.route(oracle.InstanceTable(q2, tab.p, tab.d, tab.kv, 0, "f64"), x, y, D)
+    same = res.instance_idx == ref.instance_idx
+    assert same.mean() > 0.999                     # rounding order may flip an exact tie, nothing else
+    np.testing.assert_allclose(res.est_e2e_ms[same], ref.est_e2e_ms[same], rtol=1e-12)
+    np.testing.assert_array_equal(res.tier[same], ref.tier[same])
+
+
+def test_prefix_single_instance_closed_form():
+    types, inst = fixture_pool()
+    one = W.InstanceState(*(a[1:2].copy() for a in inst.columns()))
+    tab = oracle.instance_table(types, one, 0.5, "f64")
+    x = np.array([1000, 1000, 50, 0], np.int32)
+    y = np.array([200, 0, 7, 9], np.int32)
+    hit = np.array([640, 1000, 48, 0], np.int32)
+    res = oracle.route_prefix(tab, x, y, np.full(4, 1e9, np.float32), np.zeros((1, 4), np.int32), hit[None, :])
+    p = float(np.float32(0.05))
+    d = 14.0 + float(np.float32(0.08)) * 10
+    q = 0.5 * (2000 * p) + 0.5 * float(np.float32(2000 * p))        # EMA step on the carried (float) state
+    np.testing.assert_allclose(res.est_e2e_ms, q + p * (x - hit) + d * y, rtol=1e-12)
+
+
+def test_prefix_threaded_split_is_identical():
+    wl = W.make_workload(1, n_requests=5001, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    cols = wl.requests.columns()
+    pi, ph = W.make_prefix_hits(wl.requests, tab.n_instances, seed=1, n_slots=2)
+    a = oracle.route_prefix(tab, *cols, pi, ph)
+    b = oracle.route_prefix(tab, *cols, pi, ph, threads=7)
+    for u, v in ((a.instance_idx, b.instance_idx), (a.est_e2e_ms, b.est_e2e_ms), (a.tier, b.tier)):
+        np.testing.assert_array_equal(u, v)

@@ -61,6 +61,7 @@ CONFIGS: Dict[int, Config] = {
 # stream ids (second word of the Philox key)
 _S_TYPES, _S_INST, _S_PROMPT, _S_DECODE, _S_SLO, _S_MIX = 1, 2, 3, 4, 5, 6
 _S_A_INST, _S_A_PRED, _S_A_GEN, _S_A_PROMPT, _S_A_SLO, _S_A_ELAPSED = 10, 11, 12, 13, 14, 15
+_S_PFX_HAS, _S_PFX_INST, _S_PFX_LEN = 20, 21, 22
 _ROUND_STRIDE = 1000  # stream ids of round k are offset by k * _ROUND_STRIDE
 
 
@@ -221,6 +222,29 @@ def make_requests(cfg: Config, types: TypeTable, seed: int, n: Optional[int] = N
     scale = _rng(seed, _S_SLO + off).uniform(cfg.slo_lo, cfg.slo_hi, size=n)
     slo = (scale * _unloaded_latency_ms(types, prompt, decode)).astype(np.float32)
     return RequestBatch(prompt, decode, slo)
+
+
+def make_prefix_hits(requests: RequestBatch, n_instances: int, seed: int, n_slots: int = 1,
+                     hit_share: float = 0.35, block: int = 16) -> Tuple[np.ndarray, np.ndarray]:
+    """Sparse prefix-cache state for a batch: ``(prefix_inst, prefix_hit_len)``, int32 arrays
+    of shape (n_slots, N).  A share ``hit_share`` of the requests has a cached prefix in slot 0
+    (system prompts and multi-turn sessions); each further slot is filled for half of the
+    requests that filled the one before (replicated prefixes).  The instance is uniform over
+    the pool, the hit a uniform fraction of the prompt rounded down to whole KV blocks of
+    ``block`` tokens.  Empty slots hold instance -1 and length 0."""
+    n = requests.prompt_len.shape[0]
+    pi = np.full((n_slots, n), -1, np.int32)
+    ph = np.zeros((n_slots, n), np.int32)
+    has = np.ones(n, bool)
+    for k in range(n_slots):
+        u = _rng(seed, _S_PFX_HAS + 10 * k).random(n)
+        has = has & (u < (hit_share if k == 0 else 0.5))
+        g = _rng(seed, _S_PFX_INST + 10 * k).integers(0, n_instances, size=n, dtype=np.int64)
+        frac = _rng(seed, _S_PFX_LEN + 10 * k).random(n)
+        length = (np.floor(frac * requests.prompt_len.astype(np.float64)) // block * block).astype(np.int32)
+        pi[k] = np.where(has, g, -1).astype(np.int32)
+        ph[k] = np.where(has, length, 0).astype(np.int32)
+    return pi, ph
 
 
 def make_active(cfg: Config, types: TypeTable, n_instances: int, seed: int,
