@@ -9,6 +9,8 @@
  *                    restricted to instances with KV room, the "just-enough" choice
  *                    argmax d_g over that set, and the fallback argmin T when the set is
  *                    empty (Algorithm 1; Sec. 3.4).
+ *   gs_route_batch_prefix  the same round with Eq. 2's prefix-cache term: per request a
+ *                    few (instance, cached prefix length) pairs lower T on those instances.
  *   gs_risk_scan     for every active request, the SLO-violation risk test of Sec. 3.4
  *                    (expected finish time under the latest estimates exceeds the SLO) and
  *                    the ascending list of flagged requests (migration candidates).
@@ -170,6 +172,37 @@ GS_API int gs_route_batch(gs_ctx *ctx,
                    const gs_instances *inst, const gs_types *types, float ema_alpha,
                    int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
                    uint8_t *out_tier, unsigned flags, void *cuda_stream);
+
+/*
+ * One routing round with the prefix-cache term of Eq. 2,
+ *   T(r,g) = q_g + p_g * (L_in_r - H_{r,g}) + d_g * L_out_r,
+ * where H_{r,g} (Algorithm 1's ReusePrefix) is the number of prompt tokens of r already cached
+ * on g.  H is given in sparse form: n_slots (instance, hit length) pairs per request; every
+ * pair not named has H = 0.
+ *
+ * prefix_inst, prefix_hit_len: device arrays of n_slots * slot_stride int32 entries; slot k
+ * of request r is at index k * slot_stride + r.  slot_stride >= n_requests and a multiple of
+ * 4 (each slot's column starts 16-byte aligned, else GS_ERR_ALIGN).  0 <= n_slots <=
+ * GS_MAX_PREFIX_SLOTS; with n_slots == 0 the two pointers are not read and the result is that
+ * of gs_route_batch.
+ *   - a slot whose instance is negative is empty;
+ *   - an instance >= n_instances names nothing: the slot is ignored and GS_DEV_BAD_INSTANCE set;
+ *   - a hit length is clamped into [0, L_in]; one outside sets GS_DEV_BAD_VALUE;
+ *   - an instance named by several slots keeps its longest hit.
+ * The estimate is computed as fma(d, L_out, fma(p, L_in - H, q)) in float.  The memory
+ * constraint is the one of gs_route_batch (L_in + L_out <= free_kv_tokens): a cached prefix
+ * does not lower it.  Outputs, tiers, ties and feasibility as for gs_route_batch.  Does not
+ * touch the context's pending per-instance deltas.
+ */
+#define GS_MAX_PREFIX_SLOTS 8
+GS_API int gs_route_batch_prefix(gs_ctx *ctx,
+                   const int32_t *prompt_len, const int32_t *pred_decode_len,
+                   const float *slo_ms, int64_t n_requests,
+                   const int32_t *prefix_inst, const int32_t *prefix_hit_len, int n_slots,
+                   int64_t slot_stride,
+                   const gs_instances *inst, const gs_types *types, float ema_alpha,
+                   int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                   uint8_t *out_tier, void *cuda_stream);
 
 /*
  * Applies the deltas accumulated by gs_route_batch(..., GS_ROUTE_ACCUMULATE) since the last

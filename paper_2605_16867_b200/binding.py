@@ -84,6 +84,9 @@ def load_library(build_if_missing: bool = True):
     route_args = [vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types), f32, vp, vp, vp, vp]
     lib.gs_route_batch.argtypes = route_args + [u32, vp]
     lib.gs_route_batch_host.argtypes = route_args + [vp]
+    lib.gs_route_batch_prefix.argtypes = [vp, vp, vp, vp, i64, vp, vp, C.c_int, i64, C.POINTER(_Instances),
+                                          C.POINTER(_Types), f32, vp, vp, vp, vp, vp]
+    lib.gs_route_batch_prefix.restype = C.c_int
     lib.gs_advance_state.argtypes = [vp, C.POINTER(_InstancesMut), vp]
     risk_args = [vp, vp, vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types), vp, vp, i64, vp, vp]
     lib.gs_risk_scan.argtypes = risk_args
@@ -239,6 +242,28 @@ class GoodServe:
             _dev_ptr(out_slack_ms, f32, n, "out_slack_ms", dev),
             _dev_ptr(out_tier, torch.uint8, n, "out_tier", dev),
             GS_ROUTE_ACCUMULATE if accumulate else 0, self._stream(stream)))
+
+    def route_batch_prefix(self, prompt_len, pred_decode_len, slo_ms, prefix_inst, prefix_hit_len,
+                           n_slots: int, slot_stride: int, pool: InstancePool, ema_alpha: float,
+                           out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier=None,
+                           n_requests: Optional[int] = None, stream=None):
+        """``prefix_inst`` / ``prefix_hit_len``: 1-D int32 CUDA tensors of n_slots * slot_stride
+        entries, slot k of request r at k * slot_stride + r."""
+        n = int(prompt_len.numel()) if n_requests is None else int(n_requests)
+        dev, i32, f32 = self.device, torch.int32, torch.float32
+        inst, types = self._pool_structs(pool)
+        n_hits = max(int(n_slots), 0) * int(slot_stride)
+        self._check(self._lib.gs_route_batch_prefix(
+            self._h, _dev_ptr(prompt_len, i32, n, "prompt_len", dev),
+            _dev_ptr(pred_decode_len, i32, n, "pred_decode_len", dev),
+            _dev_ptr(slo_ms, f32, n, "slo_ms", dev), n,
+            _dev_ptr(prefix_inst, i32, n_hits, "prefix_inst", dev),
+            _dev_ptr(prefix_hit_len, i32, n_hits, "prefix_hit_len", dev), int(n_slots), int(slot_stride),
+            C.byref(inst), C.byref(types),
+            float(ema_alpha), _dev_ptr(out_instance_idx, i32, n, "out_instance_idx", dev),
+            _dev_ptr(out_est_e2e_ms, f32, n, "out_est_e2e_ms", dev),
+            _dev_ptr(out_slack_ms, f32, n, "out_slack_ms", dev),
+            _dev_ptr(out_tier, torch.uint8, n, "out_tier", dev), self._stream(stream)))
 
     def advance_state(self, pool: InstancePool, stream=None):
         M, dev, i32 = pool.n_instances, self.device, torch.int32

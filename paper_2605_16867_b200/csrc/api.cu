@@ -258,9 +258,40 @@ GS_API int gs_route_batch(gs_ctx *ctx, const int32_t *prompt_len, const int32_t 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, types->n_types,
+    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, types->n_types,
                          out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier,
                          (flags & GS_ROUTE_ACCUMULATE) != 0, st);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
+GS_API int gs_route_batch_prefix(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                          const float *slo_ms, int64_t n_requests,
+                          const int32_t *prefix_inst, const int32_t *prefix_hit_len, int n_slots,
+                          int64_t slot_stride,
+                          const gs_instances *inst, const gs_types *types, float ema_alpha,
+                          int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                          uint8_t *out_tier, void *cuda_stream)
+{
+    int rc = check_pool(ctx, inst, types, true);
+    if (rc != GS_OK) return rc;
+    if (n_requests < 0 || n_slots < 0 || n_slots > GS_MAX_PREFIX_SLOTS) return GS_ERR_INVALID_ARG;
+    if (n_slots > 0 && n_requests > 0) {
+        if (!prefix_inst || !prefix_hit_len || slot_stride < n_requests) return GS_ERR_INVALID_ARG;
+        if (misaligned(prefix_inst) || misaligned(prefix_hit_len) || (slot_stride & 3)) return GS_ERR_ALIGN;
+    }
+    if (n_requests > 0) {
+        const void *ptrs[] = {prompt_len, pred_decode_len, slo_ms, out_instance_idx, out_est_e2e_ms, out_slack_ms};
+        for (const void *p : ptrs) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+        if (out_tier && misaligned(out_tier)) return GS_ERR_ALIGN;
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    const gs::PrefixHits hits = {prefix_inst, prefix_hit_len, n_slots, slot_stride};
+    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, &hits, types->n_types,
+                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, false, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 

@@ -100,11 +100,20 @@ struct LaunchTimer {
     ~LaunchTimer();
 };
 
+// Sparse prefix-cache state of a batch (Eq. 2's H): n_slots (instance, hit length) pairs per
+// request, slot k of request r at k * slot_stride + r.
+struct PrefixHits {
+    const int32_t *inst;
+    const int32_t *hit_len;
+    int n_slots;
+    int64_t slot_stride;
+};
+
 // launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_types &types,
                             float ema_alpha, cudaStream_t st);
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
-                         const float *slo_ms, int64_t n, int n_types,
+                         const float *slo_ms, int64_t n, const PrefixHits *hits, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, cudaStream_t st);
 cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,

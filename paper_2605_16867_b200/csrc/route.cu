@@ -334,10 +334,10 @@ __device__ __forceinline__ void exhaustive_pick(const Row *rows, int M, float xs
     }
 }
 
-template <bool kAccumulate>
+template <bool kAccumulate, bool kPrefix>
 __global__ void __launch_bounds__(kRouteThreads, 4)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
-             const float *__restrict__ slo_ms, int64_t n, int n_types_alloc,
+             const float *__restrict__ slo_ms, int64_t n, const PrefixHits hits, int n_types_alloc,
              const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
              const unsigned char *__restrict__ g_start_table,
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
@@ -444,6 +444,54 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 }
             }
         }
+        // ---- prefix-cache term of Eq. 2: on the instances that hold a prefix of the request T
+        // is lower by p * H; each is scored again with its hit and merged into the answer ------
+        if (kPrefix) {
+            const bool full = kReqPerThread == 4 && first + kReqPerThread <= n;
+            for (int k = 0; k < hits.n_slots; ++k) {
+                const int32_t *col_g = hits.inst + (int64_t)k * hits.slot_stride;
+                const int32_t *col_h = hits.hit_len + (int64_t)k * hits.slot_stride;
+                int hg[kReqPerThread], hh[kReqPerThread];
+                if (full) {
+                    const int4 gv = __ldcs(reinterpret_cast<const int4 *>(col_g + first));
+                    const int4 hv = __ldcs(reinterpret_cast<const int4 *>(col_h + first));
+                    hg[0] = gv.x; hg[1] = gv.y; hg[2] = gv.z; hg[3] = gv.w;
+                    hh[0] = hv.x; hh[1] = hv.y; hh[2] = hv.z; hh[3] = hv.w;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kReqPerThread; ++j) {
+                        const bool v = first + j < n;
+                        hg[j] = v ? col_g[first + j] : -1;
+                        hh[j] = v ? col_h[first + j] : 0;
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < kReqPerThread; ++j) {
+                    const int g = hg[j];
+                    if (g < 0) continue;                                     // empty slot
+                    if (g >= M) { bad |= GS_DEV_BAD_INSTANCE; continue; }    // names nothing
+                    int h = hh[j];
+                    if (h < 0 || h > xi[j]) { bad |= GS_DEV_BAD_VALUE; h = h < 0 ? 0 : xi[j]; }
+                    const Row row = sh_rows[g];
+                    const float T = __fmaf_rn(row.d, __int2float_rn(yi[j]),
+                                              __fmaf_rn(row.p, __int2float_rn(xi[j] - h), row.q));
+                    const bool room = (unsigned)xi[j] + (unsigned)yi[j] <= (unsigned)row.kv;
+                    const unsigned tier = (tiers >> (8 * j)) & 0xFFu;
+                    const int g_cur = g_out[j];
+                    bool take;
+                    if (room && T <= D[j]) {                                 // feasible with its hit
+                        const float d_cur = tier == 1u ? sh_rows[g_cur].d : 0.f;
+                        take = tier != 1u || row.d > d_cur || (row.d == d_cur && g < g_cur) ||
+                               (g == g_cur && T < T_out[j]);
+                        if (take) tiers = (tiers & ~(0xFFu << (8 * j))) | (1u << (8 * j));
+                    } else {                                                 // may still lead the fallback
+                        take = tier >= 2u && (room || tier == 3u) &&
+                               (T < T_out[j] || (T == T_out[j] && g < g_cur));
+                    }
+                    if (take) { g_out[j] = g; T_out[j] = T; }
+                }
+            }
+        }
         if (kAccumulate) {
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j)
@@ -485,7 +533,7 @@ constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
 
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
-                         const float *slo_ms, int64_t n, int n_types,
+                         const float *slo_ms, int64_t n, const PrefixHits *hits, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, cudaStream_t st)
 {
@@ -495,16 +543,16 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm[n_types];
     if (blocks > cap) blocks = cap;
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
-    if (accumulate)
-        route_kernel<true><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, n_types, ctx->s.rows, ctx->s.row_bounds,
-            ctx->s.start_table, ctx->s.headers,
-            ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
-    else
-        route_kernel<false><<<(unsigned)blocks, kRouteThreads, smem, st>>>(
-            prompt_len, pred_decode_len, slo_ms, n, n_types, ctx->s.rows, ctx->s.row_bounds,
-            ctx->s.start_table, ctx->s.headers,
-            ctx->s.table_info, out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);
+    const PrefixHits none = {nullptr, nullptr, 0, 0};
+#define GS_LAUNCH_ROUTE(ACC, PFX)                                                                     \
+    route_kernel<ACC, PFX><<<(unsigned)blocks, kRouteThreads, smem, st>>>(                             \
+        prompt_len, pred_decode_len, slo_ms, n, hits ? *hits : none, n_types, ctx->s.rows,            \
+        ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, out_idx, out_est,   \
+        out_slack, out_tier, ctx->s.deltas, ctx->s.status)
+    if (hits && hits->n_slots > 0) GS_LAUNCH_ROUTE(false, true);      // (never with accumulate)
+    else if (accumulate) GS_LAUNCH_ROUTE(true, false);
+    else GS_LAUNCH_ROUTE(false, false);
+#undef GS_LAUNCH_ROUTE
     return cudaGetLastError();
 }
 
@@ -614,16 +662,18 @@ cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *
 cudaError_t configure_route(gs_ctx *ctx)
 {
     const size_t max_smem = kRouteSmemFixed + kRouteSmemPerType * GS_MAX_TYPES;
-    cudaError_t e = cudaFuncSetAttribute(route_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(route_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)(max_smem + kRouteSmemHist));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    e = cudaFuncSetAttribute(route_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(route_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
     for (int t = 0; t <= GS_MAX_TYPES; ++t) {
         int occ = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false>, kRouteThreads,
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false>, kRouteThreads,
                                                           kRouteSmemFixed + kRouteSmemPerType * t);
         if (e != cudaSuccess) return e;
         ctx->route_ctas_per_sm[t] = occ > 0 ? occ : 1;

@@ -36,6 +36,32 @@ def gpu_route(gs, pool, req, alpha, accumulate=False, with_tier=True):
                     tier.cpu().numpy() if with_tier else None)
 
 
+def gpu_route_prefix(gs, pool, req, alpha, prefix_inst, prefix_hit_len, pad_to=None):
+    """prefix_inst / prefix_hit_len: int32 arrays (n_slots, N); columns are padded to a stride
+    that is a multiple of 4 (``pad_to`` forces a larger one)."""
+    import torch
+    dev = gs.device
+    n = req.n
+    K = prefix_inst.shape[0]
+    stride = max((n + 3) // 4 * 4, pad_to or 0)
+    pi = np.full((K, stride), 12345, np.int32)          # padding must never be read as a slot
+    ph = np.full((K, stride), 999, np.int32)
+    pi[:, :n] = prefix_inst
+    ph[:, :n] = prefix_hit_len
+    x = torch.from_numpy(req.prompt_len).to(dev)
+    y = torch.from_numpy(req.pred_decode_len).to(dev)
+    D = torch.from_numpy(req.slo_ms).to(dev)
+    pi_d = torch.from_numpy(pi.reshape(-1)).to(dev)
+    ph_d = torch.from_numpy(ph.reshape(-1)).to(dev)
+    idx = torch.full((n,), -7, dtype=torch.int32, device=dev)
+    est = torch.full((n,), float("nan"), dtype=torch.float32, device=dev)
+    slack = torch.full((n,), float("nan"), dtype=torch.float32, device=dev)
+    tier = torch.zeros(n, dtype=torch.uint8, device=dev)
+    gs.route_batch_prefix(x, y, D, pi_d, ph_d, K, stride, pool, alpha, idx, est, slack, tier)
+    torch.cuda.synchronize(dev)
+    return GpuRoute(idx.cpu().numpy(), est.cpu().numpy(), slack.cpu().numpy(), tier.cpu().numpy())
+
+
 @dataclass
 class GpuRisk:
     flag_bits: np.ndarray     # uint32 words

@@ -9,7 +9,7 @@ import pytest
 import oracle
 import workloads as W
 from parity_util import (REL_TOL, assert_route_matches_f32_oracle, check_risk_against_f64,
-                         check_route_against_f64, gpu_risk, gpu_route, unpack_bits)
+                         check_route_against_f64, gpu_risk, gpu_route, gpu_route_prefix, unpack_bits)
 
 pytestmark = pytest.mark.gpu
 
@@ -511,3 +511,114 @@ def test_reroute_on_adversarial_pools(gs, case):
     prompt = np.clip(np.rint(np.exp(rng.normal(6.5, 1.2, act.n))), 0, 1 << 20).astype(np.int32)
     check_reroute(gs, types, inst, act, prompt, alpha=0.25)
     assert gs.device_status() == 0
+
+
+# --------------------------------------------------------------------------------------
+# routing with the prefix-cache term of Eq. 2
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("cfg_id,n_slots", [(0, 1), (1, 1), (1, 3), (2, 2)])
+def test_prefix_config_full_size(gs, cfg_id, n_slots):
+    wl = W.make_workload(cfg_id)
+    pool = pool_of(gs, wl.types, wl.instances)
+    t32 = oracle.instance_table(wl.types, wl.instances, wl.ema_alpha, "f32")
+    pi, ph = W.make_prefix_hits(wl.requests, t32.n_instances, seed=cfg_id, n_slots=n_slots)
+    got = gpu_route_prefix(gs, pool, wl.requests, wl.ema_alpha, pi, ph)
+    ref = oracle.route_prefix(t32, *wl.requests.columns(), pi, ph, threads=8)
+    assert_route_matches_f32_oracle(got, ref)
+    plain = oracle.route(t32, *wl.requests.columns(), threads=8)
+    print(f"cfg {cfg_id}, {n_slots} slot(s): {int((plain.instance_idx != ref.instance_idx).sum())} of "
+          f"{len(ref.tier)} answers moved by the hits")
+    assert gs.device_status() == 0
+
+
+def test_prefix_config3_sample(gs):
+    """Full-size launch; the oracle checks a strided sample of the requests."""
+    wl = W.make_workload(3)
+    pool = pool_of(gs, wl.types, wl.instances)
+    t32 = oracle.instance_table(wl.types, wl.instances, wl.ema_alpha, "f32")
+    pi, ph = W.make_prefix_hits(wl.requests, t32.n_instances, seed=3, n_slots=1)
+    got = gpu_route_prefix(gs, pool, wl.requests, wl.ema_alpha, pi, ph)
+    sel = np.arange(0, wl.requests.n, 61)
+    x, y, D = (c[sel] for c in wl.requests.columns())
+    ref = oracle.route_prefix(t32, x, y, D, pi[:, sel], ph[:, sel], threads=8)
+    np.testing.assert_array_equal(got.instance_idx[sel], ref.instance_idx)
+    np.testing.assert_array_equal(got.tier[sel], ref.tier)
+    np.testing.assert_array_equal(got.est_e2e_ms[sel], ref.est_e2e_ms)
+
+
+@pytest.mark.parametrize("n_slots", [0, 1, 2])
+def test_prefix_without_hits_equals_plain_routing(gs, n_slots):
+    wl = W.make_workload(1, n_requests=10001)
+    pool = pool_of(gs, wl.types, wl.instances)
+    n = wl.requests.n
+    pi = np.full((n_slots, n), -1, np.int32)
+    ph = np.full((n_slots, n), 50, np.int32)
+    a = gpu_route_prefix(gs, pool, wl.requests, 0.5, pi, ph)
+    b = gpu_route(gs, pool, wl.requests, 0.5)
+    for u, v in ((a.instance_idx, b.instance_idx), (a.est_e2e_ms, b.est_e2e_ms), (a.slack_ms, b.slack_ms), (a.tier, b.tier)):
+        np.testing.assert_array_equal(u, v)
+
+
+def test_prefix_handworked(gs):
+    from test_oracle_pins import fixture_pool, parse_slots, read_rows
+    for name, x, y, D, k0, k1, k2, slots, g, est, slack, tier in read_rows("handworked_prefix.txt"):
+        types, inst = fixture_pool((int(k0), int(k1), int(k2)))
+        pool = pool_of(gs, types, inst)
+        pi, ph = parse_slots(slots)
+        req = W.RequestBatch(np.array([int(x)], np.int32), np.array([int(y)], np.int32), np.array([float(D)], np.float32))
+        got = gpu_route_prefix(gs, pool, req, 0.5, pi, ph)
+        assert got.instance_idx[0] == int(g) and got.tier[0] == int(tier), name
+        assert got.est_e2e_ms[0] == pytest.approx(float(est), rel=1e-5), name
+        assert got.slack_ms[0] == pytest.approx(float(slack), rel=1e-4, abs=2e-3), name
+        gs.device_status()
+
+
+@pytest.mark.parametrize("case", [0, 1, 3, 5, 9, 13])
+def test_prefix_on_adversarial_pools(gs, case):
+    """Boundary deadlines, equal estimates, scarce KV, slots that are empty, unknown,
+    duplicated, negative or longer than the prompt; ragged batch size and padded stride."""
+    from paper_2605_16867_b200 import DeviceStatus
+    rng = np.random.default_rng(2000 + case)
+    types, inst = _random_pool(rng, **FUZZ_CASES[case])
+    pool = pool_of(gs, types, inst)
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    M = t32.n_instances
+    n = 6001
+    req = _boundary_requests(rng, t32, n)
+    K = 3
+    pi = rng.integers(-1, M + 1, (K, n)).astype(np.int32)
+    pi[2] = np.where(rng.random(n) < 0.5, pi[0], pi[2])                 # duplicates
+    ph = (rng.random((K, n)) * 1.2 * req.prompt_len - 2).astype(np.int32)
+    # deadlines that the hit decides: just below the hit-free estimate of the first slot's instance
+    g0 = np.clip(pi[0], 0, M - 1)
+    T0 = _canonical_T(t32, req.prompt_len, req.pred_decode_len)[np.arange(n), g0]
+    req.slo_ms[::4] = np.nextafter(T0, np.float32(-np.inf))[::4]
+    got = gpu_route_prefix(gs, pool, req, 0.5, pi, ph, pad_to=n + 37 + (4 - (n + 37) % 4) % 4)
+    ref = oracle.route_prefix(t32, *req.columns(), pi, ph, threads=4)
+    assert_route_matches_f32_oracle(got, ref)
+    assert gs.device_status() == ref.status == (DeviceStatus.BAD_VALUE | DeviceStatus.BAD_INSTANCE)
+
+
+def test_prefix_error_codes(gs):
+    from paper_2605_16867_b200 import GoodServeError
+    wl = W.make_workload(0, n_requests=64)
+    pool = pool_of(gs, wl.types, wl.instances)
+    dev = gs.device
+    x = torch.from_numpy(wl.requests.prompt_len).to(dev)
+    y = torch.from_numpy(wl.requests.pred_decode_len).to(dev)
+    D = torch.from_numpy(wl.requests.slo_ms).to(dev)
+    hits = torch.zeros(9 * 64 + 4, dtype=torch.int32, device=dev)
+    o_i = torch.zeros(64, dtype=torch.int32, device=dev)
+    o_f = torch.zeros(64, dtype=torch.float32, device=dev)
+    o_s = torch.zeros(64, dtype=torch.float32, device=dev)
+    for kwargs, code in ((dict(n_slots=9, slot_stride=64), -1),        # more slots than supported
+                         (dict(n_slots=-1, slot_stride=64), -1),
+                         (dict(n_slots=1, slot_stride=60), -1),        # stride shorter than the batch
+                         (dict(n_slots=1, slot_stride=66), -4)):       # stride not a multiple of 4
+        with pytest.raises(GoodServeError) as e:
+            gs.route_batch_prefix(x, y, D, hits, hits, kwargs["n_slots"], kwargs["slot_stride"], pool, 0.5, o_i, o_f, o_s)
+        assert e.value.code == code, kwargs
+    with pytest.raises(GoodServeError) as e:                            # misaligned hit column
+        gs.route_batch_prefix(x, y, D, hits[1:], hits, 1, 64, pool, 0.5, o_i, o_f, o_s)
+    assert e.value.code == -4
