@@ -41,9 +41,9 @@ ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-ins
 # Counters of one launch on config 3 taken with ncu (profiles/route_kernel_config3.md).  They
 # describe the kernel sources with this hash; after any change to those files they no longer
 # apply and the fields that use them become null until the kernel is profiled again.
-PROFILED_ROUTE = {"sources_sha1": "03458c74dc1f4239b529344bf78842b3d3547611", "config": 3,
-                  "dram_bytes_per_launch": 50_439_424 + 5_802_496,
-                  "warp_instructions_per_launch": 58_386_468}
+PROFILED_ROUTE = {"sources_sha1": "8092b819b153fba0346a9f54aee8675bd35aa484", "config": 3,
+                  "dram_bytes_per_launch": 50_451_200 + 5_850_880,
+                  "warp_instructions_per_launch": 57_344_633}
 
 
 def kernel_sources_sha1() -> str:
