@@ -112,6 +112,31 @@ def instance_table(types, inst, ema_alpha: float, precision: str = "f64") -> Ins
     return InstanceTable(q, p, d, kv, status.value, precision)
 
 
+def direct_table(q_ms, p_ms_per_tok, d_ms_per_tok, free_kv_tokens, precision: str = "f64") -> InstanceTable:
+    """The table of a round from coefficients given directly (black-box estimates, Sec. 3.3)."""
+    qi = _c(q_ms, np.float32); pi = _c(p_ms_per_tok, np.float32); di = _c(d_ms_per_tok, np.float32)
+    kvi = _c(free_kv_tokens, np.int32)
+    M = qi.shape[0]
+    real = np.float64 if precision == "f64" else np.float32
+    q = np.empty(M, real); p = np.empty(M, real); d = np.empty(M, real); kv = np.empty(M, np.int64)
+    status = C.c_uint(0)
+    getattr(_L(), f"gso_direct_table_{precision}")(C.c_int32(M), _p(qi), _p(pi), _p(di), _p(kvi),
+                                                   _p(q), _p(p), _p(d), _p(kv), C.byref(status))
+    return InstanceTable(q, p, d, kv, status.value, precision)
+
+
+def ema_update(alpha: float, observed, state, precision: str = "f64"):
+    """One EMA step of a coefficient column: returns (new state, status)."""
+    obs = _c(observed, np.float32)
+    real = np.float64 if precision == "f64" else np.float32
+    c_in = _c(state, real)
+    c_out = np.empty_like(c_in)
+    status = C.c_uint(0)
+    getattr(_L(), f"gso_ema_update_{precision}")(C.c_int32(obs.shape[0]), C.c_float(alpha), _p(obs), _p(c_in),
+                                                 _p(c_out), C.byref(status))
+    return c_out, status.value
+
+
 @dataclass
 class RouteResult:
     instance_idx: np.ndarray   # int32[N]

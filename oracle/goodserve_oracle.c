@@ -13,6 +13,8 @@
  *     can hold the request                                                      (Algorithm 1; Sec. 3.1 constraints)
  *   - just-enough choice  g* = argmax_{g in C} d_g                               (Algorithm 1; Sec. 3.4)
  *   - fallback  g* = argmin_g (T(r,g) - D_r)  when C is empty                    (Algorithm 1)
+ *   - black-box coefficient smoothing  c <- alpha * obs + (1 - alpha) * c  for q, p, d and
+ *     tables given directly                                                    (Sec. 3.3)
  *   - risk test: an ongoing request is flagged when its expected finish time under the
  *     latest estimates exceeds its SLO                                          (Sec. 3.4, second step)
  *
@@ -432,4 +434,69 @@ void gso_route_prefix_f32(int64_t N, const int32_t *prompt_len, const int32_t *p
                           unsigned *status)
 {
     GSO_ROUTE_PREFIX_BODY(float, fmaf(d[g], y, fmaf(p[g], xh, q[g])))
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Black-box coefficients (Sec. 3.3): q_g, p_g, d_g come straight from recent             */
+/* observations, each smoothed by an exponential moving average, with no reference to     */
+/* GPU type, batch size or queue content.                                                 */
+/*                                                                                        */
+/* Reading:                                                                               */
+/*   - one EMA step per coefficient and instance:  c <- alpha * obs + (1 - alpha) * c ;    */
+/*   - an observation that is negative or NaN is no observation: c stays, status bit;     */
+/*   - a table handed to the router directly is used as it is (no EMA step inside the      */
+/*     round); a negative or NaN coefficient is read as 0 and a negative KV count as 0,    */
+/*     with a status bit.                                                                 */
+/* ------------------------------------------------------------------------------------ */
+
+void gso_ema_update_f64(int32_t M, float alpha, const float *obs, const double *c_in, double *c_out,
+                        unsigned *status)
+{
+    double a = (double)alpha;
+    for (int32_t g = 0; g < M; ++g) {
+        double o = (double)obs[g];
+        if (!(o >= 0.0)) { *status |= GSO_BAD_VALUE; c_out[g] = c_in[g]; continue; }
+        c_out[g] = a * o + (1.0 - a) * c_in[g];
+    }
+}
+
+void gso_ema_update_f32(int32_t M, float alpha, const float *obs, const float *c_in, float *c_out,
+                        unsigned *status)
+{
+    float one_minus_alpha = 1.0f - alpha;
+    for (int32_t g = 0; g < M; ++g) {
+        float o = obs[g];
+        if (!(o >= 0.0f)) { *status |= GSO_BAD_VALUE; c_out[g] = c_in[g]; continue; }
+        float keep = one_minus_alpha * c_in[g];
+        c_out[g] = fmaf(alpha, o, keep);
+    }
+}
+
+/* the table of a round from directly given coefficients (float inputs, as the C ABI takes them) */
+void gso_direct_table_f64(int32_t M, const float *q_in, const float *p_in, const float *d_in,
+                          const int32_t *free_kv_tokens,
+                          double *q, double *p, double *d, int64_t *kv, unsigned *status)
+{
+    for (int32_t g = 0; g < M; ++g) {
+        double qv = (double)q_in[g], pv = (double)p_in[g], dv = (double)d_in[g];
+        if (!(qv >= 0.0)) { *status |= GSO_BAD_VALUE; qv = 0.0; }
+        if (!(pv >= 0.0)) { *status |= GSO_BAD_VALUE; pv = 0.0; }
+        if (!(dv >= 0.0)) { *status |= GSO_BAD_VALUE; dv = 0.0; }
+        q[g] = qv; p[g] = pv; d[g] = dv;
+        kv[g] = (int64_t)clamp_count(free_kv_tokens[g], status);
+    }
+}
+
+void gso_direct_table_f32(int32_t M, const float *q_in, const float *p_in, const float *d_in,
+                          const int32_t *free_kv_tokens,
+                          float *q, float *p, float *d, int64_t *kv, unsigned *status)
+{
+    for (int32_t g = 0; g < M; ++g) {
+        float qv = q_in[g], pv = p_in[g], dv = d_in[g];
+        if (!(qv >= 0.0f)) { *status |= GSO_BAD_VALUE; qv = 0.0f; }
+        if (!(pv >= 0.0f)) { *status |= GSO_BAD_VALUE; pv = 0.0f; }
+        if (!(dv >= 0.0f)) { *status |= GSO_BAD_VALUE; dv = 0.0f; }
+        q[g] = qv; p[g] = pv; d[g] = dv;
+        kv[g] = (int64_t)clamp_count(free_kv_tokens[g], status);
+    }
 }

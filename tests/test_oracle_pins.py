@@ -712,3 +712,89 @@ def test_prefix_threaded_split_is_identical():
     b = oracle.route_prefix(tab, *cols, pi, ph, threads=7)
     for u, v in ((a.instance_idx, b.instance_idx), (a.est_e2e_ms, b.est_e2e_ms), (a.tier, b.tier)):
         np.testing.assert_array_equal(u, v)
+
+
+# --------------------------------------------------------------------------------------
+# black-box coefficients: EMA step and directly given tables (Sec. 3.3)
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_ema_closed_form_and_special_cases(prec):
+    """n EMA steps unroll to  (1-a)^n c0 + a * sum_k (1-a)^(n-1-k) obs_k ; alpha = 0 keeps the
+    state, alpha = 1 replaces it, a constant observation is a fixed point's limit."""
+    rng = np.random.default_rng(8)
+    M, n, a = 50, 12, 0.3
+    c0 = rng.uniform(0, 100, M).astype(np.float32)
+    obs = rng.uniform(0, 100, (n, M)).astype(np.float32)
+    c = c0.astype(np.float64 if prec == "f64" else np.float32)
+    for k in range(n):
+        c, st = oracle.ema_update(a, obs[k], c, prec)
+        assert st == 0
+    a32 = float(np.float32(a))
+    want = (1 - a32) ** n * c0.astype(np.float64) + a32 * sum((1 - a32) ** (n - 1 - k) * obs[k].astype(np.float64) for k in range(n))
+    np.testing.assert_allclose(c, want, rtol=1e-12 if prec == "f64" else 2e-6)
+    same, _ = oracle.ema_update(0.0, obs[0], c0, prec)
+    np.testing.assert_array_equal(same, c0)
+    repl, _ = oracle.ema_update(1.0, obs[0], c0, prec)
+    np.testing.assert_array_equal(repl, obs[0])
+    c = c0.astype(np.float64 if prec == "f64" else np.float32)
+    for _ in range(200):
+        c, _ = oracle.ema_update(0.5, np.full(M, 42.0, np.float32), c, prec)
+    np.testing.assert_allclose(c, 42.0, rtol=1e-6)
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_ema_ignores_invalid_observations(prec):
+    c0 = np.array([5.0, 6.0, 7.0, 8.0], np.float32)
+    obs = np.array([1.0, -1.0, np.nan, 0.0], np.float32)
+    c, st = oracle.ema_update(0.5, obs, c0, prec)
+    np.testing.assert_allclose(c, [3.0, 6.0, 7.0, 4.0])
+    assert st == 4
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_ema_matches_the_queue_delay_step_of_the_typed_table(prec):
+    """The EMA step that instance_table() applies to q (pinned above by its own closed form) is
+    this same step with obs = w_g = queued * p."""
+    wl = W.make_workload(1, n_requests=8, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.3, prec)
+    p32 = wl.types.prefill_ms_per_tok[wl.instances.type_id]
+    if prec == "f64":
+        w = wl.instances.queued_prefill_tokens.astype(np.float64) * p32.astype(np.float64)
+        want = float(np.float32(0.3)) * w + (1 - float(np.float32(0.3))) * wl.instances.q_ema_ms.astype(np.float64)
+        np.testing.assert_allclose(tab.q, want, rtol=1e-12)
+    else:
+        w = (wl.instances.queued_prefill_tokens.astype(np.float32) * p32).astype(np.float32)
+        got, _ = oracle.ema_update(0.3, w, wl.instances.q_ema_ms, "f32")
+        np.testing.assert_array_equal(tab.q, got)
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_direct_table_is_the_identity_on_valid_input_and_clamps_the_rest(prec):
+    wl = W.make_workload(1, n_requests=2000, n_active=8)
+    bb = W.make_blackbox_table(wl.types, wl.instances, seed=1)
+    tab = oracle.direct_table(*bb.columns(), prec)
+    for got, src in ((tab.q, bb.q_ms), (tab.p, bb.p_ms_per_tok), (tab.d, bb.d_ms_per_tok), (tab.kv, bb.free_kv_tokens)):
+        np.testing.assert_array_equal(got, src.astype(got.dtype))
+    assert tab.status == 0
+    assert len(np.unique(bb.p_ms_per_tok)) > 0.9 * bb.n_instances          # no shared p: no GPU types to lean on
+    # routing on it obeys the declarative post-condition of Algorithm 1
+    x, y, D = wl.requests.columns()
+    res = oracle.route(tab, x, y, D)
+    check_postcondition(tab.q, tab.p, tab.d, tab.kv, x[:400], y[:400], D[:400], res.instance_idx, res.tier, prec)
+    bad = oracle.direct_table([1, -1, np.nan, 2], [0.1, 0.1, 0.1, -0.5], [3, 3, 3, np.nan], [5, 5, -2, 5], prec)
+    np.testing.assert_array_equal(bad.q, [1, 0, 0, 2])
+    np.testing.assert_array_equal(bad.p, np.array([0.1, 0.1, 0.1, 0], np.float32).astype(bad.p.dtype))
+    np.testing.assert_array_equal(bad.d, [3, 3, 3, 0])
+    np.testing.assert_array_equal(bad.kv, [5, 5, 0, 5])
+    assert bad.status == 4
+
+
+def test_direct_table_of_the_typed_coefficients_routes_like_the_typed_table():
+    wl = W.make_workload(1, n_requests=3000, n_active=8)
+    typed = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    direct = oracle.direct_table(typed.q, typed.p, typed.d, typed.kv.astype(np.int32), "f32")
+    a = oracle.route(typed, *wl.requests.columns())
+    b = oracle.route(direct, *wl.requests.columns())
+    np.testing.assert_array_equal(a.instance_idx, b.instance_idx)
+    np.testing.assert_array_equal(a.est_e2e_ms, b.est_e2e_ms)

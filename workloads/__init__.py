@@ -62,6 +62,7 @@ CONFIGS: Dict[int, Config] = {
 _S_TYPES, _S_INST, _S_PROMPT, _S_DECODE, _S_SLO, _S_MIX = 1, 2, 3, 4, 5, 6
 _S_A_INST, _S_A_PRED, _S_A_GEN, _S_A_PROMPT, _S_A_SLO, _S_A_ELAPSED = 10, 11, 12, 13, 14, 15
 _S_PFX_HAS, _S_PFX_INST, _S_PFX_LEN = 20, 21, 22
+_S_BB_Q, _S_BB_P, _S_BB_D, _S_BB_OBS = 60, 61, 62, 63
 _ROUND_STRIDE = 1000  # stream ids of round k are offset by k * _ROUND_STRIDE
 
 
@@ -222,6 +223,43 @@ def make_requests(cfg: Config, types: TypeTable, seed: int, n: Optional[int] = N
     scale = _rng(seed, _S_SLO + off).uniform(cfg.slo_lo, cfg.slo_hi, size=n)
     slo = (scale * _unloaded_latency_ms(types, prompt, decode)).astype(np.float32)
     return RequestBatch(prompt, decode, slo)
+
+
+@dataclass
+class BlackBoxTable:
+    """Per-instance coefficients of Eq. 2 as a monitor would report them (Sec. 3.3)."""
+    q_ms: np.ndarray            # f32[M]
+    p_ms_per_tok: np.ndarray    # f32[M]
+    d_ms_per_tok: np.ndarray    # f32[M]
+    free_kv_tokens: np.ndarray  # i32[M]
+
+    @property
+    def n_instances(self) -> int:
+        return int(self.q_ms.shape[0])
+
+    def columns(self):
+        return self.q_ms, self.p_ms_per_tok, self.d_ms_per_tok, self.free_kv_tokens
+
+
+def make_blackbox_table(types: TypeTable, inst: InstanceState, seed: int, jitter: float = 0.05) -> BlackBoxTable:
+    """What black-box monitoring of the pool ``(types, inst)`` would hand to the router: the
+    pool's nominal per-instance values, each with its own multiplicative measurement jitter
+    (so no two instances share p exactly, unlike the typed description)."""
+    M = inst.n_instances
+    t = inst.type_id
+    u = lambda sid: _rng(seed, sid).uniform(1.0 - jitter, 1.0 + jitter, size=M)
+    p = types.prefill_ms_per_tok[t].astype(np.float64) * u(_S_BB_P)
+    d = (types.tpot_a_ms[t].astype(np.float64)
+         + types.tpot_b_ms[t].astype(np.float64) * inst.decode_batch.astype(np.float64)) * u(_S_BB_D)
+    q = inst.q_ema_ms.astype(np.float64) * u(_S_BB_Q)
+    return BlackBoxTable(q.astype(np.float32), p.astype(np.float32), d.astype(np.float32),
+                         inst.free_kv_tokens.copy())
+
+
+def make_observations(column: np.ndarray, seed: int, step: int, jitter: float = 0.2) -> np.ndarray:
+    """A fresh noisy observation of a coefficient column (input of one EMA step)."""
+    u = _rng(seed, _S_BB_OBS + 7 * step).uniform(1.0 - jitter, 1.0 + jitter, size=column.shape[0])
+    return (column.astype(np.float64) * u).astype(np.float32)
 
 
 def make_prefix_hits(requests: RequestBatch, n_instances: int, seed: int, n_slots: int = 1,
