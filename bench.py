@@ -35,7 +35,7 @@ METRIC = "request-instance pairs scored/sec"
 UNIT = "pairs/s"
 ROUTE_BYTES_PER_REQUEST = 24      # 3 input columns + 3 output columns, 4 B each
 RISK_BYTES_PER_REQUEST = 20.125   # 5 input columns + 1 flag bit (candidate indices added per flag)
-KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter", "reroute")
+KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter", "reroute", "ema")
 ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-instruction per clock
 
 # Counters of one launch on config 3 taken with ncu (profiles/route_kernel_config3.md).  They
@@ -352,6 +352,27 @@ def run_gpu(args):
                   "algorithmic_GBps": N * (ROUTE_BYTES_PER_REQUEST + 8) / (ms / n_l * 1e-3) / 1e9}
         del pi_d, ph_d
         gs.route_batch(*req, pool, alpha, out_idx, out_est, out_slack, None, stream=stream)   # outputs of the timed step
+    # ---- the routing round against black-box coefficients given per instance (not timed) ----
+    direct = None
+    if not args.no_direct:
+        bb = W.make_blackbox_table(wl.types, wl.instances, seed=rank_seed(args.config, rank))
+        tab = [torch.from_numpy(c).to(dev) for c in bb.columns()]
+        obs = [torch.from_numpy(W.make_observations(c, seed=rank_seed(args.config, rank), step=k)).to(dev)
+               for k, c in enumerate(bb.columns()[:3])]
+        run = lambda: (gs.ema_update(alpha, *obs, *tab[:3], stream=stream),
+                       gs.route_batch_direct(*req, *tab, out_idx, out_est, out_slack, None, stream=stream))
+        run()
+        barrier()
+        gs.timing_enable(True)
+        for _ in range(max(3, args.steps // 2)):
+            run()
+        barrier()
+        t = {name: gs.timing_read(KERNEL_NAMES.index(name)) for name in ("ema", "prologue", "route")}
+        gs.timing_enable(False)
+        direct = {name + "_avg_us": ms / n_l * 1e3 for name, (ms, n_l) in t.items()}
+        direct["groups_of_p"] = 8
+        del tab, obs
+        gs.route_batch(*req, pool, alpha, out_idx, out_est, out_slack, None, stream=stream)   # outputs of the timed step
     t_wait = time.perf_counter()
     while len(sampler.rows) < 4 and time.perf_counter() - t_wait < 3.0:
         step()                                   # keep the same load up for the sampler (untimed)
@@ -450,7 +471,7 @@ def run_gpu(args):
         "route_requests_per_s": world * N / (route_ms * 1e-3) if route_ms else None,
         "step_hbm_frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "flagged_fraction": flagged / A, "device_status": status,
-        "roofline": roofline, "issue": issue, "kernels": per_kernel, "reroute": reroute, "prefix": prefix,
+        "roofline": roofline, "issue": issue, "kernels": per_kernel, "reroute": reroute, "prefix": prefix, "direct": direct,
         "kernel_timing": "serial pass of %d steps on one stream after the timed region, %.4f ms/step" % (
             args.steps, serial_ms_per_step),
         "e2e": None if args.no_e2e else
@@ -475,6 +496,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-reroute", action="store_true", help="skip the untimed re-route measurement")
+    ap.add_argument("--no-direct", action="store_true", help="skip the untimed black-box-table routing measurement")
     ap.add_argument("--no-prefix", action="store_true", help="skip the untimed prefix-cache routing measurement")
     ap.add_argument("--serial", action="store_true", help="route and scan on one stream instead of two")
     ap.add_argument("--print-kernel-hash", action="store_true", help="print the hash PROFILED_ROUTE refers to")

@@ -11,6 +11,8 @@
  *                    empty (Algorithm 1; Sec. 3.4).
  *   gs_route_batch_prefix  the same round with Eq. 2's prefix-cache term: per request a
  *                    few (instance, cached prefix length) pairs lower T on those instances.
+ *   gs_route_batch_direct / gs_ema_update   the same round against per-instance q, p, d given
+ *                    directly (black-box estimates smoothed by an EMA, Sec. 3.3).
  *   gs_risk_scan     for every active request, the SLO-violation risk test of Sec. 3.4
  *                    (expected finish time under the latest estimates exceeds the SLO) and
  *                    the ascending list of flagged requests (migration candidates).
@@ -139,7 +141,8 @@ enum gs_kernel {
     GS_K_RISK_FLAGS = 3,     /* risk test + flag words + per-chunk flag counts */
     GS_K_RISK_SCATTER = 4,   /* ordered candidate list */
     GS_K_REROUTE = 5,        /* re-routing of the candidates */
-    GS_K_COUNT = 6
+    GS_K_EMA = 6,            /* EMA step of directly given coefficients */
+    GS_K_COUNT = 7
 };
 
 /* Optional per-kernel timing for benchmarks.  While enabled (on != 0) every kernel launch of
@@ -201,6 +204,52 @@ GS_API int gs_route_batch_prefix(gs_ctx *ctx,
                    const int32_t *prefix_inst, const int32_t *prefix_hit_len, int n_slots,
                    int64_t slot_stride,
                    const gs_instances *inst, const gs_types *types, float ema_alpha,
+                   int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                   uint8_t *out_tier, void *cuda_stream);
+
+/*
+ * Black-box instance coefficients (Sec. 3.3): q_g, p_g and d_g of Eq. 2 estimated directly from
+ * their recent observed values and smoothed by an exponential moving average, with no
+ * reference to GPU type, batch size or queue content.
+ *
+ * Per-instance table, structure of arrays, n_instances entries each, DEVICE pointers:
+ *   q_ms            smoothed queueing delay q_g
+ *   p_ms_per_tok    smoothed per-token prefill latency p_g
+ *   d_ms_per_tok    smoothed per-token decode latency d_g
+ *   free_kv_tokens  bounds L_in + L_out of a request placed on g
+ */
+typedef struct gs_instance_table {
+    const float *q_ms;
+    const float *p_ms_per_tok;
+    const float *d_ms_per_tok;
+    const int32_t *free_kv_tokens;
+    int32_t n_instances;
+} gs_instance_table;
+
+/*
+ * One EMA step per instance for up to three coefficient columns, in place:
+ *   c[g] <- fma(alpha, obs[g], (1 - alpha) * c[g])                 for c in {q, p, d}.
+ * obs_* are device arrays of n_instances fresh observations; a NULL obs pointer skips that
+ * column (its state pointer is then not read and may be NULL too).  An observation that is
+ * negative or NaN is no observation: that entry keeps its value and GS_DEV_BAD_VALUE is set.
+ * 1 <= n_instances <= the context's max_instances.  Only enqueues work on the stream.
+ */
+GS_API int gs_ema_update(gs_ctx *ctx, float alpha, int32_t n_instances,
+                  const float *obs_q_ms, const float *obs_p_ms_per_tok, const float *obs_d_ms_per_tok,
+                  float *q_ms, float *p_ms_per_tok, float *d_ms_per_tok, void *cuda_stream);
+
+/*
+ * One routing round (as gs_route_batch) against coefficients given directly.  The table is
+ * used as it is: no EMA step is taken inside the round (gs_ema_update is that step).  A
+ * negative or NaN coefficient is read as 0 and a negative free_kv_tokens as 0, with
+ * GS_DEV_BAD_VALUE set; an infinite coefficient also sets it and makes every request of the
+ * round take the exhaustive (still exact) path.  Outputs, tiers, ties and feasibility as for
+ * gs_route_batch; the estimate is fma(d, L_out, fma(p, L_in, q)) in float.  Does not touch the
+ * context's pending per-instance deltas.
+ */
+GS_API int gs_route_batch_direct(gs_ctx *ctx,
+                   const int32_t *prompt_len, const int32_t *pred_decode_len,
+                   const float *slo_ms, int64_t n_requests, const gs_instance_table *table,
                    int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
                    uint8_t *out_tier, void *cuda_stream);
 

@@ -42,6 +42,11 @@ class _Types(C.Structure):
                 ("tpot_b_ms", C.c_void_p), ("n_types", C.c_int32)]
 
 
+class _InstanceTable(C.Structure):
+    _fields_ = [("q_ms", C.c_void_p), ("p_ms_per_tok", C.c_void_p), ("d_ms_per_tok", C.c_void_p),
+                ("free_kv_tokens", C.c_void_p), ("n_instances", C.c_int32)]
+
+
 class _InstancesMut(C.Structure):
     _fields_ = [("queued_prefill_tokens", C.c_void_p), ("decode_batch", C.c_void_p),
                 ("free_kv_tokens", C.c_void_p), ("q_ema_ms", C.c_void_p),
@@ -87,6 +92,10 @@ def load_library(build_if_missing: bool = True):
     lib.gs_route_batch_prefix.argtypes = [vp, vp, vp, vp, i64, vp, vp, C.c_int, i64, C.POINTER(_Instances),
                                           C.POINTER(_Types), f32, vp, vp, vp, vp, vp]
     lib.gs_route_batch_prefix.restype = C.c_int
+    lib.gs_route_batch_direct.argtypes = [vp, vp, vp, vp, i64, C.POINTER(_InstanceTable), vp, vp, vp, vp, vp]
+    lib.gs_route_batch_direct.restype = C.c_int
+    lib.gs_ema_update.argtypes = [vp, f32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.gs_ema_update.restype = C.c_int
     lib.gs_advance_state.argtypes = [vp, C.POINTER(_InstancesMut), vp]
     risk_args = [vp, vp, vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types), vp, vp, i64, vp, vp]
     lib.gs_risk_scan.argtypes = risk_args
@@ -264,6 +273,38 @@ class GoodServe:
             _dev_ptr(out_est_e2e_ms, f32, n, "out_est_e2e_ms", dev),
             _dev_ptr(out_slack_ms, f32, n, "out_slack_ms", dev),
             _dev_ptr(out_tier, torch.uint8, n, "out_tier", dev), self._stream(stream)))
+
+    def route_batch_direct(self, prompt_len, pred_decode_len, slo_ms, q_ms, p_ms_per_tok, d_ms_per_tok,
+                           free_kv_tokens, out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier=None,
+                           n_requests: Optional[int] = None, n_instances: Optional[int] = None, stream=None):
+        """Routing round against per-instance coefficients given directly (CUDA tensors)."""
+        n = int(prompt_len.numel()) if n_requests is None else int(n_requests)
+        M = int(q_ms.numel()) if n_instances is None else int(n_instances)
+        dev, i32, f32 = self.device, torch.int32, torch.float32
+        table = _InstanceTable(_dev_ptr(q_ms, f32, M, "q_ms", dev), _dev_ptr(p_ms_per_tok, f32, M, "p_ms_per_tok", dev),
+                               _dev_ptr(d_ms_per_tok, f32, M, "d_ms_per_tok", dev),
+                               _dev_ptr(free_kv_tokens, i32, M, "free_kv_tokens", dev), M)
+        self._check(self._lib.gs_route_batch_direct(
+            self._h, _dev_ptr(prompt_len, i32, n, "prompt_len", dev),
+            _dev_ptr(pred_decode_len, i32, n, "pred_decode_len", dev),
+            _dev_ptr(slo_ms, f32, n, "slo_ms", dev), n, C.byref(table),
+            _dev_ptr(out_instance_idx, i32, n, "out_instance_idx", dev),
+            _dev_ptr(out_est_e2e_ms, f32, n, "out_est_e2e_ms", dev),
+            _dev_ptr(out_slack_ms, f32, n, "out_slack_ms", dev),
+            _dev_ptr(out_tier, torch.uint8, n, "out_tier", dev), self._stream(stream)))
+
+    def ema_update(self, alpha: float, obs_q_ms, obs_p_ms_per_tok, obs_d_ms_per_tok, q_ms, p_ms_per_tok,
+                   d_ms_per_tok, n_instances: Optional[int] = None, stream=None):
+        """In-place EMA step of the coefficient columns; a ``None`` observation skips its column."""
+        cols = [t for t in (q_ms, p_ms_per_tok, d_ms_per_tok, obs_q_ms, obs_p_ms_per_tok, obs_d_ms_per_tok) if t is not None]
+        M = int(cols[0].numel()) if n_instances is None else int(n_instances)
+        dev, f32 = self.device, torch.float32
+        self._check(self._lib.gs_ema_update(
+            self._h, float(alpha), M, _dev_ptr(obs_q_ms, f32, M, "obs_q_ms", dev),
+            _dev_ptr(obs_p_ms_per_tok, f32, M, "obs_p_ms_per_tok", dev),
+            _dev_ptr(obs_d_ms_per_tok, f32, M, "obs_d_ms_per_tok", dev), _dev_ptr(q_ms, f32, M, "q_ms", dev),
+            _dev_ptr(p_ms_per_tok, f32, M, "p_ms_per_tok", dev), _dev_ptr(d_ms_per_tok, f32, M, "d_ms_per_tok", dev),
+            self._stream(stream)))
 
     def advance_state(self, pool: InstancePool, stream=None):
         M, dev, i32 = pool.n_instances, self.device, torch.int32

@@ -295,6 +295,50 @@ GS_API int gs_route_batch_prefix(gs_ctx *ctx, const int32_t *prompt_len, const i
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 
+GS_API int gs_ema_update(gs_ctx *ctx, float alpha, int32_t n_instances,
+                  const float *obs_q_ms, const float *obs_p_ms_per_tok, const float *obs_d_ms_per_tok,
+                  float *q_ms, float *p_ms_per_tok, float *d_ms_per_tok, void *cuda_stream)
+{
+    if (!ctx || n_instances < 1) return GS_ERR_INVALID_ARG;
+    if (n_instances > ctx->max_instances) return GS_ERR_CAPACITY;
+    const float *obs[3] = {obs_q_ms, obs_p_ms_per_tok, obs_d_ms_per_tok};
+    float *col[3] = {q_ms, p_ms_per_tok, d_ms_per_tok};
+    for (int c = 0; c < 3; ++c) {
+        if (!obs[c]) continue;
+        if (!col[c]) return GS_ERR_INVALID_ARG;
+        if (misaligned(obs[c]) || misaligned(col[c])) return GS_ERR_ALIGN;
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    const cudaError_t e = gs::launch_ema(ctx, alpha, n_instances, obs_q_ms, obs_p_ms_per_tok, obs_d_ms_per_tok,
+                                         q_ms, p_ms_per_tok, d_ms_per_tok, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
+GS_API int gs_route_batch_direct(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                          const float *slo_ms, int64_t n_requests, const gs_instance_table *table,
+                          int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                          uint8_t *out_tier, void *cuda_stream)
+{
+    if (!ctx || !table || n_requests < 0 || table->n_instances < 1) return GS_ERR_INVALID_ARG;
+    if (table->n_instances > ctx->max_instances) return GS_ERR_CAPACITY;
+    const void *cols[] = {table->q_ms, table->p_ms_per_tok, table->d_ms_per_tok, table->free_kv_tokens};
+    for (const void *p : cols) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+    if (n_requests > 0) {
+        const void *ptrs[] = {prompt_len, pred_decode_len, slo_ms, out_instance_idx, out_est_e2e_ms, out_slack_ms};
+        for (const void *p : ptrs) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+        if (out_tier && misaligned(out_tier)) return GS_ERR_ALIGN;
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = gs::launch_prologue_direct(ctx, *table, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, gs::kDirectGroups,
+                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, false, st);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
 GS_API int gs_advance_state(gs_ctx *ctx, const gs_instances_mut *inst, void *cuda_stream) {
     if (!ctx || !inst) return GS_ERR_INVALID_ARG;
     if (inst->n_instances < 1) return GS_ERR_INVALID_ARG;

@@ -33,6 +33,11 @@ __host__ __device__ __forceinline__ int row_slot(int i) {
 }
 
 constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low bits of a q word
+// groups of similar p that stand in for GPU types when the coefficients are given per instance
+#ifndef GS_DIRECT_GROUPS
+#define GS_DIRECT_GROUPS 8
+#endif
+constexpr int kDirectGroups = GS_DIRECT_GROUPS;
 constexpr int kMaxPaddedRows = GS_MAX_INSTANCES + GS_MAX_TYPES * 16;
 constexpr int kStartSlots = 64;
 constexpr int kStartBuckets = 32;         // two per octave of L_out; the last one is open-ended
@@ -112,6 +117,9 @@ struct PrefixHits {
 // launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_types &types,
                             float ema_alpha, cudaStream_t st);
+cudaError_t launch_ema(gs_ctx *ctx, float alpha, int M, const float *obs_q, const float *obs_p, const float *obs_d,
+                       float *q, float *p, float *d, cudaStream_t st);
+cudaError_t launch_prologue_direct(gs_ctx *ctx, const gs_instance_table &tab, cudaStream_t st);
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                          const float *slo_ms, int64_t n, const PrefixHits *hits, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,

@@ -62,6 +62,13 @@ __device__ __forceinline__ unsigned lower_bound_bits(float v) {
 // Lower bound of v >= 0 at full precision (no tag).
 __device__ __forceinline__ float lower_bound(float v) { return __fmul_rn(v, kShrink); }
 
+// kDirect = false: the coefficients come from the typed description of the pool (type
+// constants, batch, queue, carried EMA state).  kDirect = true: q, p, d are given per instance
+// (black-box estimates, Sec. 3.3; the first three pointers are then q, p, d reinterpreted, see
+// launch_prologue_direct) and the instances are grouped by p instead of by GPU type: the search
+// only needs groups whose members share a lower bound of p, and instances of similar p (the same
+// hardware, as a rule) make groups for which that bound is tight.
+template <bool kDirect>
 __global__ void __launch_bounds__(kPrologueThreads)
 prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__ queued,
                 const int32_t *__restrict__ batch, const int32_t *__restrict__ free_kv,
@@ -81,42 +88,44 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     __shared__ unsigned sh_qmin;
     __shared__ float sh_tp[GS_MAX_TYPES], sh_ta[GS_MAX_TYPES], sh_tb[GS_MAX_TYPES];   // type constants
     __shared__ int sh_unsafe, sh_fill;
+    __shared__ unsigned sh_pmin, sh_pmax, sh_pgrp[GS_MAX_TYPES];           // kDirect: range of p, least p per group
 
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
     const bool writer = blockIdx.x == 0;       // one CTA writes what does not depend on the type
     unsigned bad = 0;
     if (tid < GS_MAX_TYPES) { sh_cnt[tid] = 0; sh_dmax[tid] = 0u; }
-    if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; }
+    if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; sh_pmin = 0xFFFFFFFFu; sh_pmax = 0u; }
+    if (kDirect && tid < GS_MAX_TYPES) sh_pgrp[tid] = 0xFFFFFFFFu;
     __syncthreads();
 
     // ---- 1. coefficients of every instance (thread g owns instance g) -------------------------
     // all global loads are issued before anything depends on them
     const bool has = tid < M;
-    int r_type = 0, r_queued = 0, r_batch = 0, r_kv = 0;
-    float r_qema = 0.f;
-    if (has) {
-        r_type = type_id[tid]; r_queued = queued[tid]; r_batch = batch[tid];
-        r_kv = free_kv[tid]; r_qema = q_ema[tid];
-    }
-    if (tid < n_types) { sh_tp[tid] = p_type[tid]; sh_ta[tid] = a_type[tid]; sh_tb[tid] = b_type[tid]; }
-    __syncthreads();
-    {
-        int t = r_type;
-        if (has && (t < 0 || t >= n_types)) { bad |= GS_DEV_BAD_TYPE; t = 0; }
-        if (!has) t = -1;
-        float d = 0.f;
+    if (kDirect) {
+        // the same parameter slots carry the direct table: q, p, d (float) and free KV
+        const float *q_in = reinterpret_cast<const float *>(type_id);
+        const float *p_in = reinterpret_cast<const float *>(queued);
+        const float *d_in = reinterpret_cast<const float *>(batch);
+        float q = 0.f, p = 0.f, d = 0.f;
+        int kv = 0;
         if (has) {
-            const float Qtok = __int2float_rn(clamp_count(r_queued, bad));
-            const float B = __int2float_rn(clamp_count(r_batch, bad));
-            float qe = r_qema;
-            if (!(qe >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; qe = 0.0f; }
-            const int kv = clamp_count(r_kv, bad);
-            const float p = sh_tp[t];
-            d = __fmaf_rn(sh_tb[t], B, sh_ta[t]);               // loaded per-token decode latency
-            const float w = __fmul_rn(Qtok, p);                 // time to drain the queued prefill
-            const float keep = __fmul_rn(__fsub_rn(1.0f, alpha), qe);
-            const float q = __fmaf_rn(alpha, w, keep);          // EMA step
+            q = q_in[tid]; p = p_in[tid]; d = d_in[tid]; kv = clamp_count(free_kv[tid], bad);
+            if (!(q >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; q = 0.0f; }
+            if (!(p >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; p = 0.0f; }
+            if (!(d >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; d = 0.0f; }
+        }
+        // range of p over the pool (non-negative floats order like their bit patterns)
+        const unsigned pb = __float_as_uint(p) & 0x7FFFFFFFu;          // (a -0 counts as 0)
+        const unsigned wmin = __reduce_min_sync(0xFFFFFFFFu, has ? pb : 0xFFFFFFFFu);
+        const unsigned wmax = __reduce_max_sync(0xFFFFFFFFu, has ? pb : 0u);
+        if (lane == 0) { atomicMin(&sh_pmin, wmin); atomicMax(&sh_pmax, wmax); }
+        __syncthreads();
+        // group = equal slices of the bit-pattern range of p (close to equal ratios of p)
+        int t = -1;
+        if (has) {
+            const unsigned long long span = (unsigned long long)(sh_pmax - sh_pmin) + 1ull;
+            t = (int)(((unsigned long long)(pb - sh_pmin) * (unsigned long long)n_types) / span);
             sh_q[tid] = q; sh_d[tid] = d; sh_t[tid] = (unsigned char)t;
             if (writer) {
                 Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
@@ -124,19 +133,65 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 s.d_by_g[tid] = d;
                 s.q_by_g[tid] = q;
             }
-            // the bounds of the search tables need finite, non-negative coefficients
             const float big = 3.0e38f;
-            if (!(q >= 0.f && q < big && p >= 0.f && p < big && d >= 0.f && d < big)) atomicOr(&sh_unsafe, 1);
+            if (!(q < big && p < big && d < big)) atomicOr(&sh_unsafe, 1);
         }
-        // instances per type and each type's largest d: one shared-memory atomic per type and warp
         const unsigned peers = __match_any_sync(0xFFFFFFFFu, t);
         const unsigned dmax = __reduce_max_sync(peers, orderable(d));
+        const unsigned gmin = __reduce_min_sync(peers, pb);
         if (t >= 0 && lane == __ffs(peers) - 1) {
             atomicAdd(&sh_cnt[t], __popc(peers));
             atomicMax(&sh_dmax[t], dmax);
+            atomicMin(&sh_pgrp[t], gmin);
         }
+        __syncthreads();
+        if (tid < GS_MAX_TYPES) sh_tp[tid] = __uint_as_float(sh_pgrp[tid]);     // the group's least p
+    } else {
+        int r_type = 0, r_queued = 0, r_batch = 0, r_kv = 0;
+        float r_qema = 0.f;
+        if (has) {
+            r_type = type_id[tid]; r_queued = queued[tid]; r_batch = batch[tid];
+            r_kv = free_kv[tid]; r_qema = q_ema[tid];
+        }
+        if (tid < n_types) { sh_tp[tid] = p_type[tid]; sh_ta[tid] = a_type[tid]; sh_tb[tid] = b_type[tid]; }
+        __syncthreads();
+        {
+            int t = r_type;
+            if (has && (t < 0 || t >= n_types)) { bad |= GS_DEV_BAD_TYPE; t = 0; }
+            if (!has) t = -1;
+            float d = 0.f;
+            if (has) {
+                const float Qtok = __int2float_rn(clamp_count(r_queued, bad));
+                const float B = __int2float_rn(clamp_count(r_batch, bad));
+                float qe = r_qema;
+                if (!(qe >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; qe = 0.0f; }
+                const int kv = clamp_count(r_kv, bad);
+                const float p = sh_tp[t];
+                d = __fmaf_rn(sh_tb[t], B, sh_ta[t]);               // loaded per-token decode latency
+                const float w = __fmul_rn(Qtok, p);                 // time to drain the queued prefill
+                const float keep = __fmul_rn(__fsub_rn(1.0f, alpha), qe);
+                const float q = __fmaf_rn(alpha, w, keep);          // EMA step
+                sh_q[tid] = q; sh_d[tid] = d; sh_t[tid] = (unsigned char)t;
+                if (writer) {
+                    Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
+                    s.rows[tid] = row;
+                    s.d_by_g[tid] = d;
+                    s.q_by_g[tid] = q;
+                }
+                // the bounds of the search tables need finite, non-negative coefficients
+                const float big = 3.0e38f;
+                if (!(q >= 0.f && q < big && p >= 0.f && p < big && d >= 0.f && d < big)) atomicOr(&sh_unsafe, 1);
+            }
+            // instances per type and each type's largest d: one shared-memory atomic per type and warp
+            const unsigned peers = __match_any_sync(0xFFFFFFFFu, t);
+            const unsigned dmax = __reduce_max_sync(peers, orderable(d));
+            if (t >= 0 && lane == __ffs(peers) - 1) {
+                atomicAdd(&sh_cnt[t], __popc(peers));
+                atomicMax(&sh_dmax[t], dmax);
+            }
+        }
+        __syncthreads();
     }
-    __syncthreads();
 
     // ---- 2. order of the types (largest d first; ties: smaller type id) ----------------------
     if (tid < GS_MAX_TYPES) {
@@ -303,7 +358,10 @@ size_t prologue_dynamic_smem() { return (size_t)kPmFloats * sizeof(float); }   /
 
 cudaError_t configure_prologue()
 {
-    return cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(prologue_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)prologue_dynamic_smem());
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(prologue_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)prologue_dynamic_smem());
 }
 
@@ -311,10 +369,22 @@ cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_type
                             float ema_alpha, cudaStream_t st)
 {
     LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
-    prologue_kernel<<<GS_MAX_TYPES, kPrologueThreads, prologue_dynamic_smem(), st>>>(
+    prologue_kernel<false><<<GS_MAX_TYPES, kPrologueThreads, prologue_dynamic_smem(), st>>>(
         inst.type_id, inst.queued_prefill_tokens, inst.decode_batch, inst.free_kv_tokens,
         inst.q_ema_ms, inst.n_instances, types.prefill_ms_per_tok, types.tpot_a_ms,
         types.tpot_b_ms, types.n_types, ema_alpha, ctx->s);
+    return cudaGetLastError();
+}
+
+// Tables of a round from coefficients given per instance; the instances are put into
+// kDirectGroups groups of similar p, which take the place of the GPU types in the search.
+cudaError_t launch_prologue_direct(gs_ctx *ctx, const gs_instance_table &tab, cudaStream_t st)
+{
+    LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
+    prologue_kernel<true><<<GS_MAX_TYPES, kPrologueThreads, prologue_dynamic_smem(), st>>>(
+        reinterpret_cast<const int32_t *>(tab.q_ms), reinterpret_cast<const int32_t *>(tab.p_ms_per_tok),
+        reinterpret_cast<const int32_t *>(tab.d_ms_per_tok), tab.free_kv_tokens, nullptr, tab.n_instances,
+        nullptr, nullptr, nullptr, kDirectGroups, 0.f, ctx->s);
     return cudaGetLastError();
 }
 

@@ -717,4 +717,38 @@ cudaError_t launch_advance(gs_ctx *ctx, const gs_instances_mut &inst, cudaStream
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------
+// EMA step of the black-box coefficients (Sec. 3.3): c <- alpha * obs + (1 - alpha) * c
+// ---------------------------------------------------------------------------------------
+
+// One thread per instance and column; a column without observations (null) is left alone, and
+// so is an entry whose observation is negative or NaN (status bit).
+__global__ void ema_kernel(float alpha, int M, const float *__restrict__ obs_q, const float *__restrict__ obs_p,
+                           const float *__restrict__ obs_d, float *__restrict__ q, float *__restrict__ p,
+                           float *__restrict__ d, unsigned *__restrict__ status)
+{
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= M) return;
+    const float *obs[3] = {obs_q, obs_p, obs_d};
+    float *col[3] = {q, p, d};
+    const float one_minus_alpha = __fsub_rn(1.0f, alpha);
+    bool bad = false;
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        if (!obs[c]) continue;
+        const float o = obs[c][g];
+        if (!(o >= 0.0f)) { bad = true; continue; }
+        col[c][g] = __fmaf_rn(alpha, o, __fmul_rn(one_minus_alpha, col[c][g]));
+    }
+    if (bad) atomicOr(status, (unsigned)GS_DEV_BAD_VALUE);
+}
+
+cudaError_t launch_ema(gs_ctx *ctx, float alpha, int M, const float *obs_q, const float *obs_p, const float *obs_d,
+                       float *q, float *p, float *d, cudaStream_t st)
+{
+    LaunchTimer timer(ctx, GS_K_EMA, st);
+    ema_kernel<<<(M + 255) / 256, 256, 0, st>>>(alpha, M, obs_q, obs_p, obs_d, q, p, d, ctx->s.status);
+    return cudaGetLastError();
+}
+
 }  // namespace gs

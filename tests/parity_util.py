@@ -62,6 +62,24 @@ def gpu_route_prefix(gs, pool, req, alpha, prefix_inst, prefix_hit_len, pad_to=N
     return GpuRoute(idx.cpu().numpy(), est.cpu().numpy(), slack.cpu().numpy(), tier.cpu().numpy())
 
 
+def gpu_route_direct(gs, bb, req):
+    """bb: workloads.BlackBoxTable (or anything with .columns() -> q, p, d, kv as numpy)."""
+    import torch
+    dev = gs.device
+    n = req.n
+    q, p, d, kv = (torch.from_numpy(np.ascontiguousarray(c)).to(dev) for c in bb.columns())
+    x = torch.from_numpy(req.prompt_len).to(dev)
+    y = torch.from_numpy(req.pred_decode_len).to(dev)
+    D = torch.from_numpy(req.slo_ms).to(dev)
+    idx = torch.full((n,), -7, dtype=torch.int32, device=dev)
+    est = torch.full((n,), float("nan"), dtype=torch.float32, device=dev)
+    slack = torch.full((n,), float("nan"), dtype=torch.float32, device=dev)
+    tier = torch.zeros(n, dtype=torch.uint8, device=dev)
+    gs.route_batch_direct(x, y, D, q, p, d, kv, idx, est, slack, tier)
+    torch.cuda.synchronize(dev)
+    return GpuRoute(idx.cpu().numpy(), est.cpu().numpy(), slack.cpu().numpy(), tier.cpu().numpy())
+
+
 @dataclass
 class GpuRisk:
     flag_bits: np.ndarray     # uint32 words

@@ -9,7 +9,8 @@ import pytest
 import oracle
 import workloads as W
 from parity_util import (REL_TOL, assert_route_matches_f32_oracle, check_risk_against_f64,
-                         check_route_against_f64, gpu_risk, gpu_route, gpu_route_prefix, unpack_bits)
+                         check_route_against_f64, gpu_risk, gpu_route, gpu_route_direct, gpu_route_prefix,
+                         unpack_bits)
 
 pytestmark = pytest.mark.gpu
 
@@ -622,3 +623,131 @@ def test_prefix_error_codes(gs):
     with pytest.raises(GoodServeError) as e:                            # misaligned hit column
         gs.route_batch_prefix(x, y, D, hits[1:], hits, 1, 64, pool, 0.5, o_i, o_f, o_s)
     assert e.value.code == -4
+
+
+# --------------------------------------------------------------------------------------
+# black-box coefficients: directly given tables and their EMA step (Sec. 3.3)
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("cfg_id", [0, 1, 2])
+def test_direct_config_full_size(gs, cfg_id):
+    wl = W.make_workload(cfg_id)
+    bb = W.make_blackbox_table(wl.types, wl.instances, seed=cfg_id)
+    t32 = oracle.direct_table(*bb.columns(), "f32")
+    got = gpu_route_direct(gs, bb, wl.requests)
+    ref = oracle.route(t32, *wl.requests.columns(), threads=8)
+    assert_route_matches_f32_oracle(got, ref)
+    t64 = oracle.direct_table(*bb.columns(), "f64")
+    n_tie = check_route_against_f64(got, t64, wl.requests)
+    print(f"cfg {cfg_id} direct: tiers={[int((got.tier == k).sum()) for k in (1, 2, 3)]} near-ties vs fp64={n_tie}")
+    assert gs.device_status() == 0
+
+
+def test_direct_config3_sample(gs):
+    wl = W.make_workload(3)
+    bb = W.make_blackbox_table(wl.types, wl.instances, seed=3)
+    t32 = oracle.direct_table(*bb.columns(), "f32")
+    got = gpu_route_direct(gs, bb, wl.requests)
+    sel = np.arange(0, wl.requests.n, 37)
+    ref = oracle.route(t32, *(c[sel] for c in wl.requests.columns()), threads=8)
+    np.testing.assert_array_equal(got.instance_idx[sel], ref.instance_idx)
+    np.testing.assert_array_equal(got.tier[sel], ref.tier)
+    np.testing.assert_array_equal(got.est_e2e_ms[sel], ref.est_e2e_ms)
+
+
+def test_direct_table_of_typed_coefficients_equals_typed_routing(gs):
+    """Feeding the typed path's own coefficients through the direct interface must not change
+    a single output, although the search then runs on groups of p instead of GPU types."""
+    wl = W.make_workload(2, n_requests=200000)
+    pool = pool_of(gs, wl.types, wl.instances)
+    typed = gpu_route(gs, pool, wl.requests, wl.ema_alpha)
+    t32 = oracle.instance_table(wl.types, wl.instances, wl.ema_alpha, "f32")
+    bb = W.BlackBoxTable(t32.q, t32.p, t32.d, t32.kv.astype(np.int32))
+    direct = gpu_route_direct(gs, bb, wl.requests)
+    for u, v in ((typed.instance_idx, direct.instance_idx), (typed.est_e2e_ms, direct.est_e2e_ms),
+                 (typed.slack_ms, direct.slack_ms), (typed.tier, direct.tier)):
+        np.testing.assert_array_equal(u, v)
+
+
+@pytest.mark.parametrize("case", range(8))
+def test_direct_on_adversarial_tables(gs, case):
+    """Continuous p (no two instances alike), all p equal, p spanning orders of magnitude, zeros,
+    a single instance; deadlines on, one ulp below and one ulp above instance estimates."""
+    rng = np.random.default_rng(3000 + case)
+    M = [1024, 1000, 513, 64, 1, 17, 300, 1024][case]
+    q = rng.uniform(0, 500, M)
+    p = [rng.uniform(0.01, 0.2, M), np.full(M, 0.05), 10.0 ** rng.uniform(-6, 2, M), rng.uniform(0.01, 0.2, M),
+         np.array([0.03]), np.zeros(M), rng.choice([0.02, 0.05, 0.11], M) * rng.uniform(0.97, 1.03, M),
+         rng.uniform(0.01, 0.2, M)][case]
+    d = rng.uniform(4, 60, M)
+    if case == 3:
+        q[:] = 0.0; d[::2] = d[0]                      # equal d: ties go to the smaller index
+    if case == 7:
+        d[rng.random(M) < 0.3] = 0.0; q[rng.random(M) < 0.3] = 0.0
+    kv = rng.integers(0, 3000 if case in (2, 6) else 200001, M)
+    bb = W.BlackBoxTable(q.astype(np.float32), p.astype(np.float32), d.astype(np.float32), kv.astype(np.int32))
+    t32 = oracle.direct_table(*bb.columns(), "f32")
+    req = _boundary_requests(rng, t32, 6000)
+    got = gpu_route_direct(gs, bb, req)
+    ref = oracle.route(t32, *req.columns(), threads=4)
+    assert_route_matches_f32_oracle(got, ref)
+    assert gs.device_status() == 0
+
+
+def test_direct_invalid_coefficients(gs):
+    from paper_2605_16867_b200 import DeviceStatus
+    rng = np.random.default_rng(9)
+    M = 200
+    q = rng.uniform(0, 500, M).astype(np.float32); p = rng.uniform(0.01, 0.2, M).astype(np.float32)
+    d = rng.uniform(4, 60, M).astype(np.float32); kv = rng.integers(0, 200001, M).astype(np.int32)
+    q[3] = -1.0; p[5] = np.nan; d[7] = -2.0; kv[9] = -5
+    bb = W.BlackBoxTable(q, p, d, kv)
+    t32 = oracle.direct_table(*bb.columns(), "f32")
+    req = W.make_requests(W.CONFIGS[1], W.make_types(3, 0, perturb=False), seed=5, n=5000)
+    got = gpu_route_direct(gs, bb, req)
+    ref = oracle.route(t32, *req.columns())
+    assert_route_matches_f32_oracle(got, ref)
+    assert gs.device_status() == t32.status == DeviceStatus.BAD_VALUE
+    d[11] = np.inf                                     # bounds unusable: exhaustive path, still exact
+    bb = W.BlackBoxTable(q, p, d, kv)
+    t32 = oracle.direct_table(*bb.columns(), "f32")
+    got = gpu_route_direct(gs, bb, req)
+    ref = oracle.route(t32, *req.columns())
+    np.testing.assert_array_equal(got.instance_idx, ref.instance_idx)
+    np.testing.assert_array_equal(got.tier, ref.tier)
+    assert gs.device_status() & DeviceStatus.BAD_VALUE
+
+
+def test_ema_update_matches_oracle(gs):
+    from paper_2605_16867_b200 import DeviceStatus, GoodServeError
+    wl = W.make_workload(3, n_requests=8, n_active=8)
+    bb = W.make_blackbox_table(wl.types, wl.instances, seed=3)
+    dev = gs.device
+    M = bb.n_instances
+    state = [torch.from_numpy(c.copy()).to(dev) for c in (bb.q_ms, bb.p_ms_per_tok, bb.d_ms_per_tok)]
+    want = [c.copy() for c in (bb.q_ms, bb.p_ms_per_tok, bb.d_ms_per_tok)]
+    for step in range(5):
+        obs = [W.make_observations(c, seed=3 + k, step=step) for k, c in enumerate((bb.q_ms, bb.p_ms_per_tok, bb.d_ms_per_tok))]
+        if step == 2:
+            obs[1][4] = np.nan; obs[2][6] = -1.0
+        alpha = (0.3, 0.0, 0.5, 1.0, 0.125)[step]
+        skip_p = step == 3                            # a column without observations stays as it is
+        gs.ema_update(alpha, *(torch.from_numpy(o).to(dev) if not (skip_p and k == 1) else None for k, o in enumerate(obs)), *state)
+        st = 0
+        for k in range(3):
+            if skip_p and k == 1:
+                continue
+            want[k], s_k = oracle.ema_update(alpha, obs[k], want[k], "f32")
+            st |= s_k
+        for k in range(3):
+            np.testing.assert_array_equal(state[k].cpu().numpy(), want[k])
+        assert gs.device_status() == st == (DeviceStatus.BAD_VALUE if step == 2 else 0)
+    # the smoothed table routes like the oracle's
+    bb2 = W.BlackBoxTable(want[0], want[1], want[2], bb.free_kv_tokens)
+    req = W.make_requests(wl.cfg, wl.types, seed=3, n=20000)
+    got = gpu_route_direct(gs, bb2, req)
+    ref = oracle.route(oracle.direct_table(*bb2.columns(), "f32"), *req.columns(), threads=4)
+    assert_route_matches_f32_oracle(got, ref)
+    with pytest.raises(GoodServeError) as e:          # observations without a state column
+        gs.ema_update(0.5, state[0], None, None, None, None, None)
+    assert e.value.code == -1
