@@ -159,6 +159,7 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
     struct { void **p; size_t bytes; } allocs[] = {
         {(void **)&s.rows, Mx * sizeof(gs::Row)},
         {(void **)&s.row_bounds, gs::kMaxPaddedRows * sizeof(uint2)},
+        {(void **)&s.row_p, gs::kMaxPaddedRows * sizeof(float)},
         {(void **)&s.start_table, (size_t)GS_MAX_TYPES * gs::kStartBuckets * gs::kStartSlots},
         {(void **)&s.headers, GS_MAX_TYPES * sizeof(gs::TypeHeader)},
         {(void **)&s.table_info, 64},
@@ -186,7 +187,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.start_table, s.headers, s.table_info, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.group_totals, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.group_totals, s.status, ctx->stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);
@@ -260,7 +261,7 @@ GS_API int gs_route_batch(gs_ctx *ctx, const int32_t *prompt_len, const int32_t 
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, types->n_types,
                          out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier,
-                         (flags & GS_ROUTE_ACCUMULATE) != 0, st);
+                         (flags & GS_ROUTE_ACCUMULATE) != 0, false, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 
@@ -291,7 +292,7 @@ GS_API int gs_route_batch_prefix(gs_ctx *ctx, const int32_t *prompt_len, const i
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     const gs::PrefixHits hits = {prefix_inst, prefix_hit_len, n_slots, slot_stride};
     e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, &hits, types->n_types,
-                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, false, st);
+                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, false, false, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 
@@ -335,7 +336,7 @@ GS_API int gs_route_batch_direct(gs_ctx *ctx, const int32_t *prompt_len, const i
     cudaError_t e = gs::launch_prologue_direct(ctx, *table, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, gs::kDirectGroups,
-                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, false, st);
+                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, false, true, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 

@@ -58,6 +58,7 @@ constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 struct Scratch {
     Row *rows;                // [max_instances] exact coefficients, caller order
     uint2 *row_bounds;        // [kMaxPaddedRows]
+    float *row_p;             // [kMaxPaddedRows] lower bound of each row's p, in row order (unswizzled)
     unsigned char *start_table;   // [GS_MAX_TYPES * kStartBuckets * kStartSlots]
     TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)
     int *table_info;          // {padded rows, unsafe, n_instances, n_active_types}
@@ -76,6 +77,7 @@ struct gs_ctx {
     int max_instances;
     int max_types;
     int n_sm;
+    int route_ctas_per_sm_row_p;
     int route_ctas_per_sm[GS_MAX_TYPES + 1];   // by number of types (sets the shared-memory size)
     gs::Scratch s;
     size_t max_chunks, max_groups;   // capacity of the risk scan's count arrays
@@ -123,7 +125,7 @@ cudaError_t launch_prologue_direct(gs_ctx *ctx, const gs_instance_table &tab, cu
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                          const float *slo_ms, int64_t n, const PrefixHits *hits, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
-                         bool accumulate, cudaStream_t st);
+                         bool accumulate, bool row_p, cudaStream_t st);
 cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,
                            const int32_t *assigned, const int32_t *generated, const int32_t *pred_len,
                            const float *elapsed, const float *slo, const int32_t *prompt_len, int64_t n_active,

@@ -62,12 +62,42 @@ __device__ __forceinline__ unsigned lower_bound_bits(float v) {
 // Lower bound of v >= 0 at full precision (no tag).
 __device__ __forceinline__ float lower_bound(float v) { return __fmul_rn(v, kShrink); }
 
+// Bitonic sort of one 64-bit key per thread over the first n_sort threads' keys (n_sort a power
+// of two >= 32; all kPrologueThreads threads call it).  Partners closer than a warp exchange by
+// shuffle, farther ones through shared memory (two buffers, so one barrier per exchange).
+// Returns the key of rank tid.
+__device__ __forceinline__ unsigned long long bitonic_sort(unsigned long long key, int n_sort, int tid,
+                                                           unsigned long long (*sh_xchg)[GS_MAX_INSTANCES])
+{
+    int buf = 0;
+    for (int k = 2; k <= n_sort; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            unsigned long long other;
+            if (j >= 32) {
+                sh_xchg[buf][tid] = key;
+                __syncthreads();
+                other = sh_xchg[buf][tid ^ j];
+                buf ^= 1;
+            } else {
+                other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
+            }
+            const bool keep_min = ((tid & k) == 0) == ((tid & j) == 0);
+            key = (keep_min == (other < key)) ? other : key;
+        }
+    }
+    __syncthreads();
+    return key;
+}
+
 // kDirect = false: the coefficients come from the typed description of the pool (type
-// constants, batch, queue, carried EMA state).  kDirect = true: q, p, d are given per instance
-// (black-box estimates, Sec. 3.3; the first three pointers are then q, p, d reinterpreted, see
-// launch_prologue_direct) and the instances are grouped by p instead of by GPU type: the search
-// only needs groups whose members share a lower bound of p, and instances of similar p (the same
-// hardware, as a rule) make groups for which that bound is tight.
+// constants, batch, queue, carried EMA state) and the groups of the search are the GPU types.
+// kDirect = true: q, p, d are given per instance (black-box estimates, Sec. 3.3; the first
+// three pointers are then q, p, d reinterpreted, see launch_prologue_direct).  There are no
+// types to lean on, so the pool is cut into n_types groups of consecutive rank in the
+// preference order (d descending, index ascending): the groups are disjoint in d, so the first
+// group that yields a feasible row ends a request's search.  Inside a group p varies; the
+// header and the start table use the group's least p, and every row carries its own bound of p
+// (row_p) for the row tests.
 template <bool kDirect>
 __global__ void __launch_bounds__(kPrologueThreads)
 prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__ queued,
@@ -77,76 +107,78 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 const float *__restrict__ b_type, int n_types, float alpha,
                 Scratch s)
 {
-    __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];                // my type's rows, sorted
+    __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];                // my group's rows, sorted
     extern __shared__ unsigned long long sh_dyn[];                        // sort exchange buffers, then running minima
     unsigned long long (*sh_xchg)[GS_MAX_INSTANCES] = reinterpret_cast<unsigned long long (*)[GS_MAX_INSTANCES]>(sh_dyn);
     __shared__ float sh_q[GS_MAX_INSTANCES], sh_d[GS_MAX_INSTANCES];       // by instance index
-    __shared__ unsigned char sh_t[GS_MAX_INSTANCES];
+    __shared__ float sh_p[kDirect ? GS_MAX_INSTANCES : 1];                 // kDirect: p by instance index
+    __shared__ unsigned char sh_t[kDirect ? 1 : GS_MAX_INSTANCES];
     __shared__ float sh_rq[GS_MAX_INSTANCES], sh_rd[GS_MAX_INSTANCES];     // my rows: q_lo, d_lo (untagged)
     __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES];
     __shared__ unsigned sh_dmax[GS_MAX_TYPES];
-    __shared__ unsigned sh_qmin;
+    __shared__ unsigned sh_qmin, sh_pmin;
     __shared__ float sh_tp[GS_MAX_TYPES], sh_ta[GS_MAX_TYPES], sh_tb[GS_MAX_TYPES];   // type constants
     __shared__ int sh_unsafe, sh_fill;
-    __shared__ unsigned sh_pmin, sh_pmax, sh_pgrp[GS_MAX_TYPES];           // kDirect: range of p, least p per group
 
     const int tid = threadIdx.x;
-    const int lane = tid & 31, warp = tid >> 5;
-    const bool writer = blockIdx.x == 0;       // one CTA writes what does not depend on the type
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const bool writer = blockIdx.x == 0;       // one CTA writes what does not depend on the group
+    const int tr = blockIdx.x;                 // position of this CTA's group in the search order
     unsigned bad = 0;
     if (tid < GS_MAX_TYPES) { sh_cnt[tid] = 0; sh_dmax[tid] = 0u; }
-    if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; sh_pmin = 0xFFFFFFFFu; sh_pmax = 0u; }
-    if (kDirect && tid < GS_MAX_TYPES) sh_pgrp[tid] = 0xFFFFFFFFu;
+    if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; sh_pmin = 0xFFFFFFFFu; }
     __syncthreads();
 
-    // ---- 1. coefficients of every instance (thread g owns instance g) -------------------------
-    // all global loads are issued before anything depends on them
     const bool has = tid < M;
+    int base = 0, n_act = 0, padded_total = 0, n_t = 0;
+    float p_group = 0.f;                       // lower bound source: the least p of the group
+
     if (kDirect) {
-        // the same parameter slots carry the direct table: q, p, d (float) and free KV
+        // ---- 1. the coefficients as given (thread g owns instance g) ---------------------------
         const float *q_in = reinterpret_cast<const float *>(type_id);
         const float *p_in = reinterpret_cast<const float *>(queued);
         const float *d_in = reinterpret_cast<const float *>(batch);
-        float q = 0.f, p = 0.f, d = 0.f;
-        int kv = 0;
+        float q = 0.f, pv = 0.f, d = 0.f;
         if (has) {
-            q = q_in[tid]; p = p_in[tid]; d = d_in[tid]; kv = clamp_count(free_kv[tid], bad);
+            q = q_in[tid]; pv = p_in[tid]; d = d_in[tid];
+            const int kv = clamp_count(free_kv[tid], bad);
             if (!(q >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; q = 0.0f; }
-            if (!(p >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; p = 0.0f; }
+            if (!(pv >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; pv = 0.0f; }
             if (!(d >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; d = 0.0f; }
-        }
-        // range of p over the pool (non-negative floats order like their bit patterns)
-        const unsigned pb = __float_as_uint(p) & 0x7FFFFFFFu;          // (a -0 counts as 0)
-        const unsigned wmin = __reduce_min_sync(0xFFFFFFFFu, has ? pb : 0xFFFFFFFFu);
-        const unsigned wmax = __reduce_max_sync(0xFFFFFFFFu, has ? pb : 0u);
-        if (lane == 0) { atomicMin(&sh_pmin, wmin); atomicMax(&sh_pmax, wmax); }
-        __syncthreads();
-        // group = equal slices of the bit-pattern range of p (close to equal ratios of p)
-        int t = -1;
-        if (has) {
-            const unsigned long long span = (unsigned long long)(sh_pmax - sh_pmin) + 1ull;
-            t = (int)(((unsigned long long)(pb - sh_pmin) * (unsigned long long)n_types) / span);
-            sh_q[tid] = q; sh_d[tid] = d; sh_t[tid] = (unsigned char)t;
+            sh_q[tid] = q; sh_d[tid] = d; sh_p[tid] = pv;
             if (writer) {
-                Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
+                Row row; row.q = q; row.p = pv; row.d = d; row.kv = kv;
                 s.rows[tid] = row;
                 s.d_by_g[tid] = d;
                 s.q_by_g[tid] = q;
             }
-            const float big = 3.0e38f;
-            if (!(q < big && p < big && d < big)) atomicOr(&sh_unsafe, 1);
+            const float big = 3.0e38f;           // the bounds need finite coefficients
+            if (!(q < big && pv < big && d < big)) atomicOr(&sh_unsafe, 1);
         }
-        const unsigned peers = __match_any_sync(0xFFFFFFFFu, t);
-        const unsigned dmax = __reduce_max_sync(peers, orderable(d));
-        const unsigned gmin = __reduce_min_sync(peers, pb);
-        if (t >= 0 && lane == __ffs(peers) - 1) {
-            atomicAdd(&sh_cnt[t], __popc(peers));
-            atomicMax(&sh_dmax[t], dmax);
-            atomicMin(&sh_pgrp[t], gmin);
+        // ---- 2. preference order of the whole pool, cut into groups of consecutive rank -------
+        int n_sort = 32;
+        while (n_sort < M) n_sort <<= 1;
+        unsigned long long key = has ? (((unsigned long long)(~orderable(d)) << 16) | (unsigned)tid) : ~0ull;
+        key = bitonic_sort(key, n_sort, tid, sh_xchg);          // (its barriers also publish sh_unsafe)
+        const int group_rows = (((M + n_types - 1) / n_types) + 15) & ~15;
+        n_act = (M + group_rows - 1) / group_rows;
+        padded_total = (n_act - 1) * group_rows + ((M - (n_act - 1) * group_rows + 15) & ~15);
+        if (tr < n_act) {
+            base = tr * group_rows;
+            n_t = min(group_rows, M - base);
         }
+        // ---- 3. this CTA's slice of the order, and its least p ---------------------------------
+        const bool mine = tr < n_act && tid >= base && tid < base + n_t;      // tid = rank here
+        if (mine) sh_key[tid - base] = key;
+        const unsigned pb = mine ? (__float_as_uint(sh_p[(int)(key & 0xFFFFull)]) & 0x7FFFFFFFu) : 0xFFFFFFFFu;
+        const unsigned wmin = __reduce_min_sync(0xFFFFFFFFu, pb);   // non-negative floats order like their bits
+        if (lane == 0 && wmin != 0xFFFFFFFFu) atomicMin(&sh_pmin, wmin);
         __syncthreads();
-        if (tid < GS_MAX_TYPES) sh_tp[tid] = __uint_as_float(sh_pgrp[tid]);     // the group's least p
+        p_group = __uint_as_float(sh_pmin);
     } else {
+        // ---- 1. coefficients of every instance (thread g owns instance g) ----------------------
+        // all global loads are issued before anything depends on them
         int r_type = 0, r_queued = 0, r_batch = 0, r_kv = 0;
         float r_qema = 0.f;
         if (has) {
@@ -191,28 +223,42 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             }
         }
         __syncthreads();
-    }
 
-    // ---- 2. order of the types (largest d first; ties: smaller type id) ----------------------
-    if (tid < GS_MAX_TYPES) {
-        int rank = GS_MAX_TYPES;           // unused types sort last
-        if (sh_cnt[tid] > 0) {
-            rank = 0;
-            for (int o = 0; o < GS_MAX_TYPES; ++o)
-                if (sh_cnt[o] > 0 && (sh_dmax[o] > sh_dmax[tid] || (sh_dmax[o] == sh_dmax[tid] && o < tid))) ++rank;
+        // ---- 2. order of the types (largest d first; ties: smaller type id) --------------------
+        if (tid < GS_MAX_TYPES) {
+            int rank = GS_MAX_TYPES;           // unused types sort last
+            if (sh_cnt[tid] > 0) {
+                rank = 0;
+                for (int o = 0; o < GS_MAX_TYPES; ++o)
+                    if (sh_cnt[o] > 0 && (sh_dmax[o] > sh_dmax[tid] || (sh_dmax[o] == sh_dmax[tid] && o < tid))) ++rank;
+            }
+            sh_rank[tid] = rank;
         }
-        sh_rank[tid] = rank;
-    }
-    __syncthreads();
-    // the type this CTA builds, the padded rows before it, the number of types in use
-    int my_type = -1, base = 0, n_act = 0, padded_total = 0;
-    for (int o = 0; o < GS_MAX_TYPES; ++o) {
-        const int r = sh_rank[o], n = sh_cnt[o];
-        if (n == 0) continue;
-        ++n_act;
-        padded_total += (n + 15) & ~15;
-        if (r == (int)blockIdx.x) my_type = o;
-        if (r < (int)blockIdx.x) base += (n + 15) & ~15;
+        __syncthreads();
+        // the type this CTA builds, the padded rows before it, the number of types in use
+        int my_type = -1;
+        for (int o = 0; o < GS_MAX_TYPES; ++o) {
+            const int r = sh_rank[o], n = sh_cnt[o];
+            if (n == 0) continue;
+            ++n_act;
+            padded_total += (n + 15) & ~15;
+            if (r == tr) my_type = o;
+            if (r < tr) base += (n + 15) & ~15;
+        }
+        if (my_type >= 0) {
+            n_t = sh_cnt[my_type];
+            p_group = sh_tp[my_type];
+            // ---- 3. collect this type's rows and sort them by (d descending, index ascending) ---
+            if (has && sh_t[tid] == my_type)
+                sh_key[atomicAdd(&sh_fill, 1)] = ((unsigned long long)(~orderable(sh_d[tid])) << 16) | (unsigned)tid;
+        }
+        __syncthreads();
+        if (my_type >= 0) {                    // (uniform over the CTA)
+            int n_sort = 32;
+            while (n_sort < n_t) n_sort <<= 1;
+            const unsigned long long key = bitonic_sort(tid < n_t ? sh_key[tid] : ~0ull, n_sort, tid, sh_xchg);
+            sh_key[tid] = key;
+        }
     }
     if (writer && tid == 0) {
         s.table_info[0] = padded_total;
@@ -222,40 +268,8 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         if (sh_unsafe) atomicOr(s.status, (unsigned)GS_DEV_BAD_VALUE);
     }
     if (writer && bad) atomicOr(s.status, bad);
-    if (my_type < 0) return;
-    const int tr = blockIdx.x;
-    const int n_t = sh_cnt[my_type];
+    if (n_t == 0) return;                      // no group at this position
     const int n_padded = (n_t + 15) & ~15;
-
-    // ---- 3. collect this type's rows and sort them by (d descending, index ascending) --------
-    // bitonic network, one key per thread: partners closer than a warp exchange by shuffle,
-    // farther ones through shared memory (two buffers, so one barrier per exchange)
-    int n_sort = 32;
-    while (n_sort < n_t) n_sort <<= 1;
-    if (has && sh_t[tid] == my_type)
-        sh_key[atomicAdd(&sh_fill, 1)] = ((unsigned long long)(~orderable(sh_d[tid])) << 16) | (unsigned)tid;
-    __syncthreads();
-    {
-        unsigned long long key = tid < n_t ? sh_key[tid] : ~0ull;
-        int buf = 0;
-        for (int k = 2; k <= n_sort; k <<= 1) {
-            for (int j = k >> 1; j > 0; j >>= 1) {
-                unsigned long long other;
-                if (j >= 32) {
-                    sh_xchg[buf][tid] = key;
-                    __syncthreads();
-                    other = sh_xchg[buf][tid ^ j];
-                    buf ^= 1;
-                } else {
-                    other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
-                }
-                const bool keep_min = ((tid & k) == 0) == ((tid & j) == 0);
-                key = (keep_min == (other < key)) ? other : key;
-            }
-        }
-        __syncthreads();
-        sh_key[tid] = key;
-    }
     __syncthreads();
 
     // ---- 4. row bounds, least q of the type ---------------------------------------------------
@@ -273,6 +287,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             my_qmin = min(my_qmin, q_bits);             // non-negative floats order like their bits
         }
         s.row_bounds[row_slot(base + k)] = entry;
+        if (kDirect) s.row_p[base + k] = k < n_t ? lower_bound(sh_p[(int)(sh_key[k] & 0xFFFFull)]) : 0.f;
     }
     my_qmin = __reduce_min_sync(0xFFFFFFFFu, my_qmin);
     if (lane == 0) atomicMin(&sh_qmin, my_qmin);
@@ -286,7 +301,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     if (tid == 0) {
         const int first_inst = (int)(sh_key[0] & 0xFFFFull);
         TypeHeader h;
-        h.p_lo = __fmul_rn(sh_tp[my_type], kShrink);
+        h.p_lo = __fmul_rn(p_group, kShrink);
         h.q_lo = q0;
         h.d_lo = d_low;
         h.d_max = sh_d[first_inst];

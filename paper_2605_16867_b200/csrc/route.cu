@@ -71,6 +71,7 @@ struct Tables {
     const uint2 *row_bounds;
     const unsigned char *start_table;
     const Row *rows;
+    const float *row_p;       // per-row lower bound of p, in row order (only where p differs inside a group)
     int n_types;
 };
 
@@ -82,11 +83,15 @@ constexpr unsigned kNoRow = 0xFFFFFFFFu;
 #endif
 constexpr int kThreadFallbackMin = GS_THREAD_FALLBACK_MIN;
 
-// Bound test of one row: false only if the row certainly cannot be chosen.
-template <bool kCapped>
-__device__ __forceinline__ bool row_may_pass(unsigned q_word, unsigned d_word, float y, float R, float d_cap) {
+// Bound test of one row: false only if the row certainly cannot be chosen.  Where all rows of
+// a group share p (GPU types) the prefill term is already in R = D - p_lo x; with kRowP the row
+// brings its own bound of p and `R` is the deadline itself.
+template <bool kCapped, bool kRowP>
+__device__ __forceinline__ bool row_may_pass(unsigned q_word, unsigned d_word, float p_lo, float x, float y,
+                                             float R, float d_cap) {
     const float d_lo = __uint_as_float(d_word);
-    return __fmaf_rn(d_lo, y, __uint_as_float(q_word)) <= R && (!kCapped || d_lo < d_cap);
+    const float base = kRowP ? __fmaf_rn(p_lo, x, __uint_as_float(q_word)) : __uint_as_float(q_word);
+    return __fmaf_rn(d_lo, y, base) <= R && (!kCapped || d_lo < d_cap);
 }
 
 // Scores one row exactly and folds it into the running best.  Returns true when the search of
@@ -109,7 +114,7 @@ __device__ __forceinline__ bool score_row(const Tables &tb, int inst, float x, f
 
 // Just-enough pick for one request.  Returns the chosen instance or -1 (no feasible one, or a
 // request this search does not take).  `Dm` is the deadline plus a hair (see the caller).
-template <bool kCapped>
+template <bool kCapped, bool kRowP>
 __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y, float D, float Dm,
                                              unsigned need, float d_cap, float &T_out)
 {
@@ -133,12 +138,13 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
         const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);
         if (h.w < d_best) break;                                  // no later type can do better
         const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, inv_w, d0
-        const float R = __fmaf_rn(-h.x, x, Dm);
+        const float Rg = __fmaf_rn(-h.x, x, Dm);           // deadline less the group's least prefill time
+        const float R = kRowP ? Dm : Rg;                   // what a row's own bound is held against
         const float inv_w = __int_as_float(geo.z);
         int k = 0;
         if (inv_w > 0.f) {
             // largest d that can still meet the deadline -> slot -> first row worth a look
-            const float z = (R - h.y) * ry;
+            const float z = (Rg - h.y) * ry;
             const float sf = fminf(fmaxf((z - __int_as_float(geo.w)) * inv_w, 0.f), (float)(kStartSlots - 1));
             k = 8 * tb.start_table[(t * kStartBuckets + ybucket) * kStartSlots + __float2int_rd(sf)];
         }
@@ -154,14 +160,19 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
                 const uint4 r1 = *reinterpret_cast<const uint4 *>(grp + ((1 ^ sw) << 4));
                 const uint4 r2 = *reinterpret_cast<const uint4 *>(grp + ((2 ^ sw) << 4));
                 const uint4 r3 = *reinterpret_cast<const uint4 *>(grp + ((3 ^ sw) << 4));
-                first = row_may_pass<kCapped>(r3.z, r3.w, y, R, d_cap) ? r3.z : first;
-                first = row_may_pass<kCapped>(r3.x, r3.y, y, R, d_cap) ? r3.x : first;
-                first = row_may_pass<kCapped>(r2.z, r2.w, y, R, d_cap) ? r2.z : first;
-                first = row_may_pass<kCapped>(r2.x, r2.y, y, R, d_cap) ? r2.x : first;
-                first = row_may_pass<kCapped>(r1.z, r1.w, y, R, d_cap) ? r1.z : first;
-                first = row_may_pass<kCapped>(r1.x, r1.y, y, R, d_cap) ? r1.x : first;
-                first = row_may_pass<kCapped>(r0.z, r0.w, y, R, d_cap) ? r0.z : first;
-                first = row_may_pass<kCapped>(r0.x, r0.y, y, R, d_cap) ? r0.x : first;
+                float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;      // rows k..k+3, k+4..k+7
+                if (kRowP) {
+                    pa = *reinterpret_cast<const float4 *>(tb.row_p + k);
+                    pb = *reinterpret_cast<const float4 *>(tb.row_p + k + 4);
+                }
+                first = row_may_pass<kCapped, kRowP>(r3.z, r3.w, pb.w, x, y, R, d_cap) ? r3.z : first;
+                first = row_may_pass<kCapped, kRowP>(r3.x, r3.y, pb.z, x, y, R, d_cap) ? r3.x : first;
+                first = row_may_pass<kCapped, kRowP>(r2.z, r2.w, pb.y, x, y, R, d_cap) ? r2.z : first;
+                first = row_may_pass<kCapped, kRowP>(r2.x, r2.y, pb.x, x, y, R, d_cap) ? r2.x : first;
+                first = row_may_pass<kCapped, kRowP>(r1.z, r1.w, pa.w, x, y, R, d_cap) ? r1.z : first;
+                first = row_may_pass<kCapped, kRowP>(r1.x, r1.y, pa.z, x, y, R, d_cap) ? r1.x : first;
+                first = row_may_pass<kCapped, kRowP>(r0.z, r0.w, pa.y, x, y, R, d_cap) ? r0.z : first;
+                first = row_may_pass<kCapped, kRowP>(r0.x, r0.y, pa.x, x, y, R, d_cap) ? r0.x : first;
                 if (first != kNoRow) break;
             }
             if (first == kNoRow) break;                     // type exhausted
@@ -173,7 +184,7 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
             for (int j = 0; j < 8 && !over; ++j) {
                 const uint2 rb = tb.row_bounds[row_slot(k + j)];
                 if (!seen) { seen = (rb.x == first); continue; }
-                if (row_may_pass<kCapped>(rb.x, rb.y, y, R, d_cap))
+                if (row_may_pass<kCapped, kRowP>(rb.x, rb.y, kRowP ? tb.row_p[k + j] : 0.f, x, y, R, d_cap))
                     over = score_row<kCapped>(tb, (int)(rb.x & kRowTagMask), x, y, D, need, d_cap, g_best, d_best, T_best);
             }
             if (over) break;
@@ -193,12 +204,9 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
 // Returns -1 with tier 0 only when kCapped and no instance has d < d_cap.
 struct Pick { int g; float T; unsigned tier; };
 
-template <bool kCapped>
-__device__ __forceinline__ Pick fallback_pick(const TypeHeader *headers, const uint2 *row_bounds, const Row *rows,
-                                           int n_types, float x, float y, unsigned need, float d_cap)
+template <bool kCapped, bool kRowP>
+__device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y, unsigned need, float d_cap)
 {
-    Tables tb;
-    tb.headers = headers; tb.row_bounds = row_bounds; tb.rows = rows; tb.start_table = nullptr; tb.n_types = n_types;
     unsigned tier_out = 0;
     int g_best = -1;
     float T_best = __int_as_float(0x7F800000);            // +inf
@@ -209,8 +217,8 @@ __device__ __forceinline__ Pick fallback_pick(const TypeHeader *headers, const u
         for (int t = tb.n_types - 1; t >= 0; --t) {
             const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);   // p_lo, q_lo, d_lo, d_max
             if (kCapped && !(h.z < d_cap)) continue;
-            float R = __fmaf_rn(-h.x, x, T_best) + 1e-30f;
-            if (!(__fmaf_rn(h.z, y, h.y) <= R)) continue;
+            float Rg = __fmaf_rn(-h.x, x, T_best) + 1e-30f;      // best so far less the group's least prefill time
+            if (!(__fmaf_rn(h.z, y, h.y) <= Rg)) continue;
             const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, ..
 #pragma unroll 1
             for (int k = geo.x + geo.y - 8; k >= geo.x; k -= 8) {
@@ -229,13 +237,20 @@ __device__ __forceinline__ Pick fallback_pick(const TypeHeader *headers, const u
                     if (!have && __uint_as_float(r[c].z) == __uint_as_float(r[c].z)) { d_min = __uint_as_float(r[c].w); have = true; }
                     if (!have && __uint_as_float(r[c].x) == __uint_as_float(r[c].x)) { d_min = __uint_as_float(r[c].y); have = true; }
                 }
-                if (!(__fmaf_rn(d_min, y, h.y) <= R)) break;
+                if (!(__fmaf_rn(d_min, y, h.y) <= Rg)) break;
+                float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;
+                if (kRowP) {
+                    pa = *reinterpret_cast<const float4 *>(tb.row_p + k);
+                    pb = *reinterpret_cast<const float4 *>(tb.row_p + k + 4);
+                }
+                const float pl[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
 #pragma unroll
                 for (int c = 3; c >= 0; --c) {
 #pragma unroll
                     for (int e = 1; e >= 0; --e) {
                         const unsigned qw = e ? r[c].z : r[c].x, dw = e ? r[c].w : r[c].y;
-                        if (!row_may_pass<kCapped>(qw, dw, y, R, d_cap)) continue;
+                        const float R = kRowP ? T_best + 1e-30f : Rg;
+                        if (!row_may_pass<kCapped, kRowP>(qw, dw, pl[2 * c + e], x, y, R, d_cap)) continue;
                         const int inst = (int)(qw & kRowTagMask);
                         const Row row = tb.rows[inst];
                         if (kCapped && !(row.d < d_cap)) continue;
@@ -243,7 +258,7 @@ __device__ __forceinline__ Pick fallback_pick(const TypeHeader *headers, const u
                         const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));   // Eq. 2, H = 0
                         if (T < T_best || (T == T_best && inst < g_best) || g_best < 0) {
                             T_best = T; g_best = inst;
-                            R = __fmaf_rn(-h.x, x, T_best) + 1e-30f;
+                            Rg = __fmaf_rn(-h.x, x, T_best) + 1e-30f;
                         }
                     }
                 }
@@ -264,7 +279,8 @@ __device__ __forceinline__ unsigned char *stage_tables(unsigned char *smem, int 
                                                        const uint2 *__restrict__ g_row_bounds,
                                                        const unsigned char *__restrict__ g_start_table,
                                                        const TypeHeader *__restrict__ g_headers,
-                                                       const int *__restrict__ table_info, Tables &tb)
+                                                       const int *__restrict__ table_info, Tables &tb,
+                                                       const float *__restrict__ g_row_p = nullptr)
 {
     const int n_padded = table_info[0];
     const bool unsafe = table_info[1] != 0;
@@ -282,7 +298,15 @@ __device__ __forceinline__ unsigned char *stage_tables(unsigned char *smem, int 
     tb.headers = sh_headers; tb.row_bounds = sh_row_bounds;
     tb.start_table = sh_start; tb.rows = sh_rows;
     tb.n_types = unsafe ? 0 : n_act;          // unusable bounds: every request takes the exhaustive path
-    return sh_start + n_types_alloc * (kStartBuckets * kStartSlots);
+    unsigned char *end = sh_start + n_types_alloc * (kStartBuckets * kStartSlots);
+    tb.row_p = nullptr;
+    if (g_row_p) {                            // per-row bounds of p, after the start tables
+        float *sh_row_p = reinterpret_cast<float *>(end);
+        for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_p[k] = g_row_p[k];
+        tb.row_p = sh_row_p;
+        end += kMaxPaddedRows * sizeof(float);
+    }
+    return end;
 }
 
 // The definition evaluated in full by one warp for one request (same arguments in all lanes):
@@ -334,13 +358,14 @@ __device__ __forceinline__ void exhaustive_pick(const Row *rows, int M, float xs
     }
 }
 
-template <bool kAccumulate, bool kPrefix>
-__global__ void __launch_bounds__(kRouteThreads, 4)
+template <bool kAccumulate, bool kPrefix, bool kRowP>
+__global__ void __launch_bounds__(kRouteThreads, kRowP ? 3 : 4)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
              const float *__restrict__ slo_ms, int64_t n, const PrefixHits hits, int n_types_alloc,
              const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
              const unsigned char *__restrict__ g_start_table,
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
+             const float *__restrict__ g_row_p,
              int32_t *__restrict__ out_idx, float *__restrict__ out_est,
              float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
@@ -349,7 +374,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     const int M = table_info[2];
     Tables tb;
     unsigned char *after_tables = stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_start_table, g_headers,
-                                               table_info, tb);
+                                               table_info, tb, kRowP ? g_row_p : nullptr);
     const Row *sh_rows = tb.rows;
     unsigned long long *hist = reinterpret_cast<unsigned long long *>(after_tables);
     if (kAccumulate)
@@ -398,7 +423,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             // (the hair added to the deadline of the bound tests keeps them safe when a bound's
             // tag bits make a zero coefficient a denormal)
             const float Dj = (valid && yi[j] > 0) ? D[j] : -1.0f;
-            g_out[j] = pick_instance<false>(tb, x, y, Dj, Dj + 1e-30f, need, 0.f, T_out[j]);
+            g_out[j] = pick_instance<false, kRowP>(tb, x, y, Dj, Dj + 1e-30f, need, 0.f, T_out[j]);
         }
         // ---- requests still without an instance: nothing is feasible (the fallback of
         // Algorithm 1), or L_out == 0, or tables whose bounds cannot be used ----------------------
@@ -417,8 +442,8 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 for (int j = 0; j < kReqPerThread; ++j)
                     if ((mine >> j) & 1u) {
                         const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];
-                        const Pick r = fallback_pick<false>(tb.headers, tb.row_bounds, tb.rows, tb.n_types,
-                                                            __int2float_rn(xi[j]), __int2float_rn(yi[j]), need, 0.f);
+                        const Pick r = fallback_pick<false, kRowP>(tb, __int2float_rn(xi[j]), __int2float_rn(yi[j]),
+                                                                   need, 0.f);
                         g_out[j] = r.g; T_out[j] = r.T;
                         tiers = (tiers & ~(0xFFu << (8 * j))) | (r.tier << (8 * j));
                         pend &= ~(1u << j);
@@ -531,27 +556,31 @@ constexpr size_t kRouteSmemFixed = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_M
                                    (size_t)kMaxPaddedRows * sizeof(uint2);
 constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
+constexpr size_t kRouteSmemRowP = (size_t)kMaxPaddedRows * sizeof(float);
 
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                          const float *slo_ms, int64_t n, const PrefixHits *hits, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
-                         bool accumulate, cudaStream_t st)
+                         bool accumulate, bool row_p, cudaStream_t st)
 {
     if (n == 0) return cudaSuccess;
-    const size_t smem = kRouteSmemFixed + kRouteSmemPerType * n_types + (accumulate ? kRouteSmemHist : 0);
+    const size_t smem = kRouteSmemFixed + kRouteSmemPerType * n_types + (accumulate ? kRouteSmemHist : 0) +
+                        (row_p ? kRouteSmemRowP : 0);
     int64_t blocks = (n + kRouteTile - 1) / kRouteTile;
-    const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm[n_types];
+    const int64_t cap = (int64_t)ctx->n_sm * (row_p ? ctx->route_ctas_per_sm_row_p : ctx->route_ctas_per_sm[n_types]);
     if (blocks > cap) blocks = cap;
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     const PrefixHits none = {nullptr, nullptr, 0, 0};
-#define GS_LAUNCH_ROUTE(ACC, PFX)                                                                     \
-    route_kernel<ACC, PFX><<<(unsigned)blocks, kRouteThreads, smem, st>>>(                             \
+#define GS_LAUNCH_ROUTE(ACC, PFX, ROWP)                                                               \
+    route_kernel<ACC, PFX, ROWP><<<(unsigned)blocks, kRouteThreads, smem, st>>>(                       \
         prompt_len, pred_decode_len, slo_ms, n, hits ? *hits : none, n_types, ctx->s.rows,            \
-        ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, out_idx, out_est,   \
-        out_slack, out_tier, ctx->s.deltas, ctx->s.status)
-    if (hits && hits->n_slots > 0) GS_LAUNCH_ROUTE(false, true);      // (never with accumulate)
-    else if (accumulate) GS_LAUNCH_ROUTE(true, false);
-    else GS_LAUNCH_ROUTE(false, false);
+        ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, ctx->s.row_p,       \
+        out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status)
+    // (the prefix term and per-row p are never combined with accumulate, nor with each other)
+    if (row_p) GS_LAUNCH_ROUTE(false, false, true);
+    else if (hits && hits->n_slots > 0) GS_LAUNCH_ROUTE(false, true, false);
+    else if (accumulate) GS_LAUNCH_ROUTE(true, false, false);
+    else GS_LAUNCH_ROUTE(false, false, false);
 #undef GS_LAUNCH_ROUTE
     return cudaGetLastError();
 }
@@ -607,13 +636,13 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
         const float d_cap = tb.rows[c].d;
         float T = 0.f;
         const float Ds = (valid && rem > 0) ? D : -1.0f;      // see route_kernel: L_out == 0 skips the search
-        int g = pick_instance<true>(tb, x, y, Ds, Ds + 1e-30f, need, d_cap, T);
+        int g = pick_instance<true, false>(tb, x, y, Ds, Ds + 1e-30f, need, d_cap, T);
         unsigned tier = 1;
         bool settled = g >= 0;
         const bool fall = valid && !settled && rem > 0 && tb.n_types > 0;
         const int n_fall = __popc(__ballot_sync(0xFFFFFFFFu, fall));           // all lanes vote
         if (fall && n_fall >= kThreadFallbackMin) {
-            const Pick r = fallback_pick<true>(tb.headers, tb.row_bounds, tb.rows, tb.n_types, x, y, need, d_cap);
+            const Pick r = fallback_pick<true, false>(tb, x, y, need, d_cap);
             g = r.g; T = r.T; tier = r.tier;                                // may settle on "no move"
             settled = true;
         }
@@ -662,18 +691,28 @@ cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *
 cudaError_t configure_route(gs_ctx *ctx)
 {
     const size_t max_smem = kRouteSmemFixed + kRouteSmemPerType * GS_MAX_TYPES;
-    cudaError_t e = cudaFuncSetAttribute(route_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(route_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)(max_smem + kRouteSmemHist));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    e = cudaFuncSetAttribute(route_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    e = cudaFuncSetAttribute(route_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(route_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(max_smem + kRouteSmemRowP));
+    if (e != cudaSuccess) return e;
+    {
+        int occ = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false, true>, kRouteThreads,
+                                                          kRouteSmemFixed + kRouteSmemPerType * kDirectGroups + kRouteSmemRowP);
+        if (e != cudaSuccess) return e;
+        ctx->route_ctas_per_sm_row_p = occ > 0 ? occ : 1;
+    }
     e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
     for (int t = 0; t <= GS_MAX_TYPES; ++t) {
         int occ = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false>, kRouteThreads,
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false, false>, kRouteThreads,
                                                           kRouteSmemFixed + kRouteSmemPerType * t);
         if (e != cudaSuccess) return e;
         ctx->route_ctas_per_sm[t] = occ > 0 ? occ : 1;
