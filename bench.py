@@ -370,7 +370,7 @@ def run_gpu(args):
         t = {name: gs.timing_read(KERNEL_NAMES.index(name)) for name in ("ema", "prologue", "route")}
         gs.timing_enable(False)
         direct = {name + "_avg_us": ms / n_l * 1e3 for name, (ms, n_l) in t.items()}
-        direct["groups_of_p"] = 8
+        direct["groups"] = 8
         del tab, obs
         gs.route_batch(*req, pool, alpha, out_idx, out_est, out_slack, None, stream=stream)   # outputs of the timed step
     t_wait = time.perf_counter()
