@@ -217,6 +217,27 @@ def route_prefix(table: InstanceTable, prompt_len, pred_decode_len, slo_ms, pref
     return out
 
 
+def route_sequential(types, inst, ema_alpha: float, prompt_len, pred_decode_len, slo_ms) -> RouteResult:
+    """Algorithm 1 one request at a time, each seeing the state left by the ones before it.
+    ``inst`` (a workloads.InstanceState) is advanced in place.  Single precision."""
+    x = _c(prompt_len, np.int32); y = _c(pred_decode_len, np.int32); D = _c(slo_ms, np.float32)
+    N = x.shape[0]
+    for a in inst.columns():
+        assert a.flags.c_contiguous
+    out = RouteResult(np.empty(N, np.int32), np.empty(N, np.float32), np.empty(N, np.float32),
+                      np.empty(N, np.uint8), 0)
+    status = C.c_uint(0)
+    _L().gso_route_sequential_f32(
+        C.c_int64(N), _p(x), _p(y), _p(D), C.c_int32(inst.n_instances), C.c_int32(types.n_types),
+        _p(_c(inst.type_id, np.int32)), _p(inst.queued_prefill_tokens), _p(inst.decode_batch),
+        _p(inst.free_kv_tokens), _p(inst.q_ema_ms),
+        _p(_c(types.prefill_ms_per_tok, np.float32)), _p(_c(types.tpot_a_ms, np.float32)),
+        _p(_c(types.tpot_b_ms, np.float32)), C.c_float(ema_alpha),
+        _p(out.instance_idx), _p(out.est_e2e_ms), _p(out.slack_ms), _p(out.tier), C.byref(status))
+    out.status = status.value
+    return out
+
+
 @dataclass
 class RiskResult:
     flag: np.ndarray        # uint8[A]

@@ -500,3 +500,90 @@ void gso_direct_table_f32(int32_t M, const float *q_in, const float *p_in, const
         kv[g] = (int64_t)clamp_count(free_kv_tokens[g], status);
     }
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Algorithm 1 one request at a time (its literal reading): the requests of a batch are    */
+/* taken in arrival order, and each one sees the state left by the ones before it.         */
+/*                                                                                        */
+/* For request r:                                                                         */
+/*   1. every instance takes its EMA step on the current state:                            */
+/*        w_g = queued_g * p_g ,  q_g <- alpha * w_g + (1 - alpha) * q_g                   */
+/*      and d_g = a_t + b_t * batch_g is read from the current batch;                      */
+/*   2. T(r, g), the feasible set, the just-enough pick and the fallback as in gso_route;  */
+/*   3. the chosen instance takes the request: queued += L_in, batch += 1,                 */
+/*      free KV -= L_in + L_out (saturating like gso_advance), and the smoothed q of step 1 */
+/*      becomes the carried state of every instance.                                       */
+/* This is the same as rounds of one request each: gso_instance_table, gso_route,          */
+/* gso_advance.  Single precision only: the carried state is single precision, and one     */
+/* decision that differs changes every later one, so there is no double-precision          */
+/* authority to compare values with beyond the first near-tie.                             */
+/* The instance state arrays are updated in place.                                         */
+/* ------------------------------------------------------------------------------------ */
+
+void gso_route_sequential_f32(int64_t N, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                              const float *slo_ms, int32_t M, int32_t Tn, const int32_t *type_id,
+                              int32_t *queued_prefill_tokens, int32_t *decode_batch, int32_t *free_kv_tokens,
+                              float *q_ema_ms,
+                              const float *p_type, const float *a_type, const float *b_type, float ema_alpha,
+                              int32_t *instance_idx, float *est_e2e_ms, float *slack_ms, uint8_t *tier,
+                              unsigned *status)
+{
+    const int64_t I32_MAX = 2147483647LL;
+    float one_minus_alpha = 1.0f - ema_alpha;
+    for (int64_t r = 0; r < N; ++r) {
+        int32_t xi = clamp_count(prompt_len[r], status);
+        int32_t yi = clamp_count(pred_decode_len[r], status);
+        float x = (float)xi, y = (float)yi;
+        float D = slo_ms[r];
+        int64_t need = (int64_t)xi + (int64_t)yi;
+
+        int32_t best_c = -1, best_k = -1, best_a = -1;
+        float d_c = 0.0f, T_c = 0.0f, T_k = 0.0f, T_a = 0.0f;
+        for (int32_t g = 0; g < M; ++g) {
+            /* step 1: coefficients of g from the current state */
+            int32_t t = type_id[g];
+            if (t < 0 || t >= Tn) { *status |= GSO_BAD_TYPE; t = 0; }
+            float Qtok = (float)clamp_count(queued_prefill_tokens[g], status);
+            float B = (float)clamp_count(decode_batch[g], status);
+            float qe = q_ema_ms[g];
+            if (!(qe >= 0.0f)) { *status |= GSO_BAD_VALUE; qe = 0.0f; }
+            float p = p_type[t];
+            float d = fmaf(b_type[t], B, a_type[t]);
+            float w = Qtok * p;
+            float keep = one_minus_alpha * qe;
+            float q = fmaf(ema_alpha, w, keep);
+            q_ema_ms[g] = q;                               /* carried to the next request */
+            int64_t kv = (int64_t)clamp_count(free_kv_tokens[g], status);
+            /* step 2 */
+            float T = fmaf(d, y, fmaf(p, x, q));
+            int kv_ok = need <= kv;
+            if (kv_ok && T <= D) {
+                if (best_c < 0 || d > d_c) { best_c = g; d_c = d; T_c = T; }
+            }
+            if (kv_ok && (best_k < 0 || T < T_k)) { best_k = g; T_k = T; }
+            if (best_a < 0 || T < T_a) { best_a = g; T_a = T; }
+        }
+        int32_t g_star; float T_star; uint8_t tr;
+        if (best_c >= 0)      { g_star = best_c; T_star = T_c; tr = 1; }
+        else if (best_k >= 0) { g_star = best_k; T_star = T_k; tr = 2; }
+        else                  { g_star = best_a; T_star = T_a; tr = 3; }
+        instance_idx[r] = g_star;
+        est_e2e_ms[r] = T_star;
+        slack_ms[r] = D - T_star;
+        if (tier) tier[r] = tr;
+        /* step 3: every instance's counts leave this step clamped as gso_advance leaves them */
+        for (int32_t g = 0; g < M; ++g) {
+            int64_t Q = queued_prefill_tokens[g] < 0 ? 0 : queued_prefill_tokens[g];
+            int64_t Bc = decode_batch[g] < 0 ? 0 : decode_batch[g];
+            int64_t K = free_kv_tokens[g] < 0 ? 0 : free_kv_tokens[g];
+            if (g == g_star) {
+                Q += xi; if (Q > I32_MAX) Q = I32_MAX;
+                Bc += 1; if (Bc > I32_MAX) Bc = I32_MAX;
+                K -= need; if (K < 0) K = 0;
+            }
+            queued_prefill_tokens[g] = (int32_t)Q;
+            decode_batch[g] = (int32_t)Bc;
+            free_kv_tokens[g] = (int32_t)K;
+        }
+    }
+}

@@ -798,3 +798,61 @@ def test_direct_table_of_the_typed_coefficients_routes_like_the_typed_table():
     b = oracle.route(direct, *wl.requests.columns())
     np.testing.assert_array_equal(a.instance_idx, b.instance_idx)
     np.testing.assert_array_equal(a.est_e2e_ms, b.est_e2e_ms)
+
+
+# --------------------------------------------------------------------------------------
+# Algorithm 1 one request at a time
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("cfg_id,alpha", [(0, 0.5), (1, 0.5), (1, 0.0), (1, 1.0)])
+def test_sequential_equals_rounds_of_one_request(cfg_id, alpha):
+    """The sequential reading is, by definition, rounds of a single request: table, route,
+    advance -- three functions pinned above, composed here in Python."""
+    wl = W.make_workload(cfg_id, n_requests=300, n_active=8)
+    x, y, D = wl.requests.columns()
+    D = D.copy(); D[::5] *= 0.3                       # some requests fall back
+    state = wl.instances.copy()
+    state.free_kv_tokens[::2] = 4000                  # KV room runs out along the way
+    seq_state = state.copy()
+    seq = oracle.route_sequential(wl.types, seq_state, alpha, x, y, D)
+    for r in range(len(x)):
+        tab = oracle.instance_table(wl.types, state, alpha, "f32")
+        one = oracle.route(tab, x[r:r + 1], y[r:r + 1], D[r:r + 1])
+        assert seq.instance_idx[r] == one.instance_idx[0], r
+        assert seq.tier[r] == one.tier[0] and seq.est_e2e_ms[r] == one.est_e2e_ms[0], r
+        assert seq.slack_ms[r] == one.slack_ms[0], r
+        oracle.advance(state, tab, one.instance_idx, x[r:r + 1], y[r:r + 1])
+    for a, b in zip(seq_state.columns(), state.columns()):
+        np.testing.assert_array_equal(a, b)
+    assert {1, 2} <= set(seq.tier.tolist())
+
+
+def test_sequential_moves_on_when_the_deadline_binds():
+    """Identical requests against identical idle instances.  The snapshot reading sends all of
+    them to instance 0.  One at a time with a loose deadline they still all go there (the
+    instance just used has the larger batch, hence the larger d, and just-enough prefers it);
+    with a deadline that the growing queue breaks, later requests move to other instances."""
+    types = base_types()
+    M = 8
+    inst = W.InstanceState(np.zeros(M, np.int32), np.zeros(M, np.int32), np.zeros(M, np.int32),
+                           np.full(M, 10**6, np.int32), np.zeros(M, np.float32))
+    n = 64
+    x = np.full(n, 1000, np.int32); y = np.full(n, 100, np.int32)
+    loose = np.full(n, 1e9, np.float32)
+    snap = oracle.route(oracle.instance_table(types, inst, 0.5, "f32"), x, y, loose)
+    assert (snap.instance_idx == 0).all()
+    seq = oracle.route_sequential(types, inst.copy(), 0.5, x, y, loose)
+    assert (seq.instance_idx == 0).all() and (seq.tier == 1).all()
+    assert (np.diff(seq.est_e2e_ms) > 0).all()                       # each one waits behind the ones before
+    tight = np.full(n, 8.0 * 100 + 0.025 * 1000 + 30.0, np.float32)   # unloaded T (825 ms) + 30 ms
+    seq_tight = oracle.route_sequential(types, inst.copy(), 0.5, x, y, tight)
+    assert seq_tight.instance_idx[0] == 0 and (seq_tight.tier[:2] == 1).all()
+    assert len(set(seq_tight.instance_idx.tolist())) > 1
+
+
+def test_sequential_first_request_is_the_batch_answer():
+    wl = W.make_workload(1, n_requests=50, n_active=8)
+    tab = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    batch = oracle.route(tab, *wl.requests.columns())
+    seq = oracle.route_sequential(wl.types, wl.instances.copy(), 0.5, *wl.requests.columns())
+    assert seq.instance_idx[0] == batch.instance_idx[0] and seq.est_e2e_ms[0] == batch.est_e2e_ms[0]
