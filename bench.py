@@ -35,7 +35,7 @@ METRIC = "request-instance pairs scored/sec"
 UNIT = "pairs/s"
 ROUTE_BYTES_PER_REQUEST = 24      # 3 input columns + 3 output columns, 4 B each
 RISK_BYTES_PER_REQUEST = 20.125   # 5 input columns + 1 flag bit (candidate indices added per flag)
-KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter", "reroute", "ema")
+KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter", "reroute", "ema", "sequential")
 ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-instruction per clock
 
 # Counters of one launch on config 3 taken with ncu (profiles/route_kernel_config3.md).  They
@@ -373,6 +373,20 @@ def run_gpu(args):
         direct["groups"] = 8
         del tab, obs
         gs.route_batch(*req, pool, alpha, out_idx, out_est, out_slack, None, stream=stream)   # outputs of the timed step
+    # ---- Algorithm 1 one request at a time: a single dependent chain (not timed) ----
+    sequential = None
+    if not args.no_sequential:
+        n_seq = min(N, 262144)
+        seq_pool = InstancePool.from_host(wl.types, wl.instances, dev)      # advanced in place
+        gs.timing_enable(True)
+        gs.route_sequential(*req, seq_pool, alpha, out_idx, out_est, out_slack, None, n_requests=n_seq, stream=stream)
+        barrier()
+        ms, n_l = gs.timing_read(KERNEL_NAMES.index("sequential"))
+        gs.timing_enable(False)
+        sequential = {"requests": n_seq, "ms": ms / n_l, "requests_per_s": n_seq / (ms / n_l * 1e-3),
+                      "ns_per_request": ms / n_l * 1e6 / n_seq}
+        del seq_pool
+        gs.route_batch(*req, pool, alpha, out_idx, out_est, out_slack, None, stream=stream)   # outputs of the timed step
     t_wait = time.perf_counter()
     while len(sampler.rows) < 4 and time.perf_counter() - t_wait < 3.0:
         step()                                   # keep the same load up for the sampler (untimed)
@@ -471,7 +485,7 @@ def run_gpu(args):
         "route_requests_per_s": world * N / (route_ms * 1e-3) if route_ms else None,
         "step_hbm_frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "flagged_fraction": flagged / A, "device_status": status,
-        "roofline": roofline, "issue": issue, "kernels": per_kernel, "reroute": reroute, "prefix": prefix, "direct": direct,
+        "roofline": roofline, "issue": issue, "kernels": per_kernel, "reroute": reroute, "prefix": prefix, "direct": direct, "sequential": sequential,
         "kernel_timing": "serial pass of %d steps on one stream after the timed region, %.4f ms/step" % (
             args.steps, serial_ms_per_step),
         "e2e": None if args.no_e2e else
@@ -497,6 +511,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-reroute", action="store_true", help="skip the untimed re-route measurement")
     ap.add_argument("--no-direct", action="store_true", help="skip the untimed black-box-table routing measurement")
+    ap.add_argument("--no-sequential", action="store_true", help="skip the untimed one-at-a-time routing measurement")
     ap.add_argument("--no-prefix", action="store_true", help="skip the untimed prefix-cache routing measurement")
     ap.add_argument("--serial", action="store_true", help="route and scan on one stream instead of two")
     ap.add_argument("--print-kernel-hash", action="store_true", help="print the hash PROFILED_ROUTE refers to")

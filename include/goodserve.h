@@ -13,6 +13,8 @@
  *                    few (instance, cached prefix length) pairs lower T on those instances.
  *   gs_route_batch_direct / gs_ema_update   the same round against per-instance q, p, d given
  *                    directly (black-box estimates smoothed by an EMA, Sec. 3.3).
+ *   gs_route_sequential  Algorithm 1 one request at a time, each seeing the state left by the
+ *                    ones before it (the literal reading; a single dependent chain).
  *   gs_risk_scan     for every active request, the SLO-violation risk test of Sec. 3.4
  *                    (expected finish time under the latest estimates exceeds the SLO) and
  *                    the ascending list of flagged requests (migration candidates).
@@ -142,7 +144,8 @@ enum gs_kernel {
     GS_K_RISK_SCATTER = 4,   /* ordered candidate list */
     GS_K_REROUTE = 5,        /* re-routing of the candidates */
     GS_K_EMA = 6,            /* EMA step of directly given coefficients */
-    GS_K_COUNT = 7
+    GS_K_SEQUENTIAL = 7,     /* one-request-at-a-time routing */
+    GS_K_COUNT = 8
 };
 
 /* Optional per-kernel timing for benchmarks.  While enabled (on != 0) every kernel launch of
@@ -250,6 +253,36 @@ GS_API int gs_ema_update(gs_ctx *ctx, float alpha, int32_t n_instances,
 GS_API int gs_route_batch_direct(gs_ctx *ctx,
                    const int32_t *prompt_len, const int32_t *pred_decode_len,
                    const float *slo_ms, int64_t n_requests, const gs_instance_table *table,
+                   int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                   uint8_t *out_tier, void *cuda_stream);
+
+/*
+ * Algorithm 1 one request at a time (its literal reading): the requests are taken in array
+ * order and each one sees the instance state left by the ones before it.  For every request
+ *   1. every instance takes the EMA step on the current state (w_g = queued_g * p_g,
+ *      q_g <- alpha * w_g + (1 - alpha) * q_g) and d_g = a_t + b_t * batch_g is read from the
+ *      current batch,
+ *   2. T(r,g), the feasible set, the just-enough pick and the fallback are those of
+ *      gs_route_batch,
+ *   3. the chosen instance takes the request (queued += L_in, batch += 1,
+ *      free KV -= L_in + L_out, saturating as in gs_advance_state) and the smoothed q_g of
+ *      step 1 becomes the carried state of every instance.
+ * This equals n_requests rounds of gs_route_batch(ACCUMULATE) + gs_advance_state with one
+ * request each.  `type_id` (n_instances entries) is read; `state` is advanced IN PLACE and is
+ * the pool's state after the last request when the stream reaches the end of the call.
+ * The requests form one dependent chain, so a single thread block does the work, one thread
+ * for up to four instances: about 1.5 million requests per second at 1,024 instances, whatever
+ * the GPU's size (every request updates and scores every instance: the chain is bound by the
+ * instructions one SM can issue per request).
+ * It exists to measure what the snapshot reading of gs_route_batch changes (the herd onto
+ * one instance within a round), not as the fast path.  Outputs and error behaviour as for
+ * gs_route_batch; n_requests == 0 enqueues nothing and leaves the state as it is.
+ */
+GS_API int gs_route_sequential(gs_ctx *ctx,
+                   const int32_t *prompt_len, const int32_t *pred_decode_len,
+                   const float *slo_ms, int64_t n_requests,
+                   const int32_t *type_id, const gs_instances_mut *state, const gs_types *types,
+                   float ema_alpha,
                    int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
                    uint8_t *out_tier, void *cuda_stream);
 

@@ -96,6 +96,9 @@ def load_library(build_if_missing: bool = True):
     lib.gs_route_batch_direct.restype = C.c_int
     lib.gs_ema_update.argtypes = [vp, f32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.gs_ema_update.restype = C.c_int
+    lib.gs_route_sequential.argtypes = [vp, vp, vp, vp, i64, vp, C.POINTER(_InstancesMut), C.POINTER(_Types), f32,
+                                        vp, vp, vp, vp, vp]
+    lib.gs_route_sequential.restype = C.c_int
     lib.gs_advance_state.argtypes = [vp, C.POINTER(_InstancesMut), vp]
     risk_args = [vp, vp, vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types), vp, vp, i64, vp, vp]
     lib.gs_risk_scan.argtypes = risk_args
@@ -305,6 +308,27 @@ class GoodServe:
             _dev_ptr(obs_d_ms_per_tok, f32, M, "obs_d_ms_per_tok", dev), _dev_ptr(q_ms, f32, M, "q_ms", dev),
             _dev_ptr(p_ms_per_tok, f32, M, "p_ms_per_tok", dev), _dev_ptr(d_ms_per_tok, f32, M, "d_ms_per_tok", dev),
             self._stream(stream)))
+
+    def route_sequential(self, prompt_len, pred_decode_len, slo_ms, pool: InstancePool, ema_alpha: float,
+                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier=None,
+                         n_requests: Optional[int] = None, stream=None):
+        """One request at a time; ``pool``'s state tensors are advanced in place."""
+        n = int(prompt_len.numel()) if n_requests is None else int(n_requests)
+        M, dev, i32, f32 = pool.n_instances, self.device, torch.int32, torch.float32
+        _, types = self._pool_structs(pool)
+        mut = _InstancesMut(_dev_ptr(pool.queued_prefill_tokens, i32, M, "queued_prefill_tokens", dev),
+                            _dev_ptr(pool.decode_batch, i32, M, "decode_batch", dev),
+                            _dev_ptr(pool.free_kv_tokens, i32, M, "free_kv_tokens", dev),
+                            _dev_ptr(pool.q_ema_ms, f32, M, "q_ema_ms", dev), M)
+        self._check(self._lib.gs_route_sequential(
+            self._h, _dev_ptr(prompt_len, i32, n, "prompt_len", dev),
+            _dev_ptr(pred_decode_len, i32, n, "pred_decode_len", dev),
+            _dev_ptr(slo_ms, f32, n, "slo_ms", dev), n, _dev_ptr(pool.type_id, i32, M, "type_id", dev),
+            C.byref(mut), C.byref(types), float(ema_alpha),
+            _dev_ptr(out_instance_idx, i32, n, "out_instance_idx", dev),
+            _dev_ptr(out_est_e2e_ms, f32, n, "out_est_e2e_ms", dev),
+            _dev_ptr(out_slack_ms, f32, n, "out_slack_ms", dev),
+            _dev_ptr(out_tier, torch.uint8, n, "out_tier", dev), self._stream(stream)))
 
     def advance_state(self, pool: InstancePool, stream=None):
         M, dev, i32 = pool.n_instances, self.device, torch.int32

@@ -11,7 +11,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libgoodserve.so")
-SOURCES = ("api.cu", "prologue.cu", "route.cu", "risk.cu")
+SOURCES = ("api.cu", "prologue.cu", "route.cu", "risk.cu", "sequential.cu")
 NVCC_FLAGS = ("-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--shared",
               "-cudart", "shared")

@@ -340,6 +340,32 @@ GS_API int gs_route_batch_direct(gs_ctx *ctx, const int32_t *prompt_len, const i
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 
+GS_API int gs_route_sequential(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                        const float *slo_ms, int64_t n_requests,
+                        const int32_t *type_id, const gs_instances_mut *state, const gs_types *types,
+                        float ema_alpha,
+                        int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                        uint8_t *out_tier, void *cuda_stream)
+{
+    if (!ctx || !state || !types || !type_id || n_requests < 0) return GS_ERR_INVALID_ARG;
+    if (state->n_instances < 1 || types->n_types < 1) return GS_ERR_INVALID_ARG;
+    if (state->n_instances > ctx->max_instances || types->n_types > ctx->max_types) return GS_ERR_CAPACITY;
+    const void *pool[] = {type_id, state->queued_prefill_tokens, state->decode_batch, state->free_kv_tokens,
+                          state->q_ema_ms, types->prefill_ms_per_tok, types->tpot_a_ms, types->tpot_b_ms};
+    for (const void *p : pool) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+    if (n_requests > 0) {
+        const void *ptrs[] = {prompt_len, pred_decode_len, slo_ms, out_instance_idx, out_est_e2e_ms, out_slack_ms};
+        for (const void *p : ptrs) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
+        if (out_tier && misaligned(out_tier)) return GS_ERR_ALIGN;
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    const cudaError_t e = gs::launch_sequential(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, type_id, *state,
+                                                *types, ema_alpha, out_instance_idx, out_est_e2e_ms, out_slack_ms,
+                                                out_tier, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
 GS_API int gs_advance_state(gs_ctx *ctx, const gs_instances_mut *inst, void *cuda_stream) {
     if (!ctx || !inst) return GS_ERR_INVALID_ARG;
     if (inst->n_instances < 1) return GS_ERR_INVALID_ARG;

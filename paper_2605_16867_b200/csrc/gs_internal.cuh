@@ -119,6 +119,11 @@ struct PrefixHits {
 // launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_types &types,
                             float ema_alpha, cudaStream_t st);
+cudaError_t launch_sequential(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                              const float *slo_ms, int64_t n, const int32_t *type_id,
+                              const gs_instances_mut &state, const gs_types &types, float alpha,
+                              int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
+                              cudaStream_t st);
 cudaError_t launch_ema(gs_ctx *ctx, float alpha, int M, const float *obs_q, const float *obs_p, const float *obs_d,
                        float *q, float *p, float *d, cudaStream_t st);
 cudaError_t launch_prologue_direct(gs_ctx *ctx, const gs_instance_table &tab, cudaStream_t st);

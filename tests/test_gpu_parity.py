@@ -751,3 +751,104 @@ def test_ema_update_matches_oracle(gs):
     with pytest.raises(GoodServeError) as e:          # observations without a state column
         gs.ema_update(0.5, state[0], None, None, None, None, None)
     assert e.value.code == -1
+
+
+# --------------------------------------------------------------------------------------
+# Algorithm 1 one request at a time
+# --------------------------------------------------------------------------------------
+
+def gpu_sequential(gs, types, inst, req, alpha):
+    pool = pool_of(gs, types, inst)
+    dev = gs.device
+    n = req.n
+    x = torch.from_numpy(req.prompt_len).to(dev)
+    y = torch.from_numpy(req.pred_decode_len).to(dev)
+    D = torch.from_numpy(req.slo_ms).to(dev)
+    idx = torch.full((max(n, 1),), -7, dtype=torch.int32, device=dev)
+    est = torch.zeros(max(n, 1), dtype=torch.float32, device=dev)
+    slack = torch.zeros(max(n, 1), dtype=torch.float32, device=dev)
+    tier = torch.zeros(max(n, 1), dtype=torch.uint8, device=dev)
+    gs.route_sequential(x, y, D, pool, alpha, idx, est, slack, tier, n_requests=n)
+    torch.cuda.synchronize(dev)
+    state = W.InstanceState(pool.type_id.cpu().numpy(), pool.queued_prefill_tokens.cpu().numpy(),
+                            pool.decode_batch.cpu().numpy(), pool.free_kv_tokens.cpu().numpy(),
+                            pool.q_ema_ms.cpu().numpy())
+    return (idx.cpu().numpy()[:n], est.cpu().numpy()[:n], slack.cpu().numpy()[:n], tier.cpu().numpy()[:n]), state
+
+
+def assert_sequential_matches(got, state, ref, ref_state):
+    for u, v in zip(got, (ref.instance_idx, ref.est_e2e_ms, ref.slack_ms, ref.tier)):
+        np.testing.assert_array_equal(u, v)
+    for u, v in zip(state.columns(), ref_state.columns()):
+        np.testing.assert_array_equal(u, v)
+
+
+@pytest.mark.parametrize("cfg_id,n", [(0, 256), (1, 65536), (2, 150000), (3, 100000)])
+def test_sequential_configs(gs, cfg_id, n):
+    wl = W.make_workload(cfg_id, n_requests=n)
+    req = wl.requests
+    req.slo_ms[::7] *= 0.3                                   # some requests fall back
+    ref_state = wl.instances.copy()
+    ref = oracle.route_sequential(wl.types, ref_state, wl.ema_alpha, *req.columns())
+    got, state = gpu_sequential(gs, wl.types, wl.instances, req, wl.ema_alpha)
+    assert_sequential_matches(got, state, ref, ref_state)
+    snap = oracle.route(oracle.instance_table(wl.types, wl.instances, wl.ema_alpha, "f32"), *req.columns(), threads=8)
+    print(f"cfg {cfg_id}: {n} requests one at a time, tiers={[int((ref.tier == k).sum()) for k in (1, 2, 3)]}; "
+          f"busiest instance takes {np.bincount(ref.instance_idx).max()} (snapshot round: {np.bincount(snap.instance_idx).max()})")
+    assert gs.device_status() == 0
+
+
+@pytest.mark.parametrize("M", [1, 31, 33, 1000])
+@pytest.mark.parametrize("n", [0, 1, 255, 257, 3000])
+def test_sequential_ragged_sizes(gs, M, n):
+    rng = np.random.default_rng(M * 7 + n)
+    types, inst = _random_pool(rng, M, 3, scarce_kv=(M == 33))
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    req = _boundary_requests(rng, t32, max(n, 1))
+    req = W.RequestBatch(req.prompt_len[:n], req.pred_decode_len[:n], req.slo_ms[:n])
+    ref_state = inst.copy()
+    ref = oracle.route_sequential(types, ref_state, 0.5, *req.columns())
+    got, state = gpu_sequential(gs, types, inst, req, 0.5)
+    assert_sequential_matches(got, state, ref, ref_state)
+    assert gs.device_status() == 0
+
+
+def test_sequential_equals_rounds_of_one_request_on_the_gpu(gs):
+    """What the header promises: n rounds of gs_route_batch(ACCUMULATE) + gs_advance_state with
+    one request each give the same assignments and the same final state."""
+    wl = W.make_workload(1, n_requests=200)
+    req = wl.requests
+    got, state = gpu_sequential(gs, wl.types, wl.instances, req, 0.5)
+    pool = pool_of(gs, wl.types, wl.instances)
+    dev = gs.device
+    x = torch.from_numpy(req.prompt_len).to(dev); y = torch.from_numpy(req.pred_decode_len).to(dev)
+    D = torch.from_numpy(req.slo_ms).to(dev)
+    idx = torch.zeros(req.n, dtype=torch.int32, device=dev)
+    est = torch.zeros(req.n, dtype=torch.float32, device=dev)
+    slack = torch.zeros(req.n, dtype=torch.float32, device=dev)
+    for r in range(req.n):
+        one_i = torch.zeros(4, dtype=torch.int32, device=dev); one_e = torch.zeros(4, device=dev); one_s = torch.zeros(4, device=dev)
+        gs.route_batch(x[r:r + 1].clone(), y[r:r + 1].clone(), D[r:r + 1].clone(), pool, 0.5, one_i, one_e, one_s,
+                       None, accumulate=True, n_requests=1)
+        gs.advance_state(pool)
+        idx[r] = one_i[0]; est[r] = one_e[0]
+    torch.cuda.synchronize(dev)
+    np.testing.assert_array_equal(idx.cpu().numpy(), got[0])
+    np.testing.assert_array_equal(est.cpu().numpy(), got[1])
+    np.testing.assert_array_equal(pool.queued_prefill_tokens.cpu().numpy(), state.queued_prefill_tokens)
+    np.testing.assert_array_equal(pool.q_ema_ms.cpu().numpy(), state.q_ema_ms)
+
+
+def test_sequential_invalid_data(gs):
+    from paper_2605_16867_b200 import DeviceStatus
+    rng = np.random.default_rng(12)
+    types, inst = _random_pool(rng, 100, 3)
+    inst.type_id[3] = 9; inst.queued_prefill_tokens[5] = -4; inst.q_ema_ms[7] = np.nan; inst.free_kv_tokens[9] = -1
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    req = _boundary_requests(rng, t32, 500)
+    req.prompt_len[11] = -3
+    ref_state = inst.copy()
+    ref = oracle.route_sequential(types, ref_state, 0.5, *req.columns())
+    got, state = gpu_sequential(gs, types, inst, req, 0.5)
+    assert_sequential_matches(got, state, ref, ref_state)
+    assert gs.device_status() == ref.status == (DeviceStatus.BAD_TYPE | DeviceStatus.BAD_VALUE)
