@@ -39,8 +39,18 @@ constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low
 #endif
 constexpr int kDirectGroups = GS_DIRECT_GROUPS;
 constexpr int kMaxPaddedRows = GS_MAX_INSTANCES + GS_MAX_TYPES * 16;
-constexpr int kStartSlots = 64;
-constexpr int kStartBuckets = 32;         // two per octave of L_out; the last one is open-ended
+#ifndef GS_START_MB
+#define GS_START_MB 1
+#endif
+#ifndef GS_START_SLOTS
+#define GS_START_SLOTS 64
+#endif
+#ifndef GS_SLOT_WIDEN
+#define GS_SLOT_WIDEN 1.0625f
+#endif
+constexpr int kStartSlots = GS_START_SLOTS;
+constexpr int kBucketBits = GS_START_MB;  // mantissa bits of L_out that pick the bucket: 2^bits buckets per octave
+constexpr int kStartBuckets = 16 << kBucketBits;   // sixteen octaves of L_out; the last bucket is open-ended
 
 // One GPU type's entry: bound over all its rows, where its rows are, start-table geometry.
 struct __align__(16) TypeHeader {
@@ -50,6 +60,12 @@ struct __align__(16) TypeHeader {
     float inv_w;        // slots per unit of d; 0 = no start table, begin at group 0
     float d0;           // d at the low edge of slot 0
 };
+
+// Candidate table: which GPU types (bit = position in the search order) can hold a feasible
+// instance at all, by the slot of D / L_out among the types' least d (a type needs
+// d_lo * L_out <= D).  The top slot and a pool whose types all have about the same least d
+// name every type.
+constexpr int kCandSlots = 64;
 
 constexpr int kRiskChunk = 1024;        // requests per warp-chunk of the risk scan (32 flag words)
 constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
@@ -61,7 +77,9 @@ struct Scratch {
     float *row_p;             // [kMaxPaddedRows] lower bound of each row's p, in row order (unswizzled)
     unsigned char *start_table;   // [GS_MAX_TYPES * kStartBuckets * kStartSlots]
     TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)
-    int *table_info;          // {padded rows, unsafe, n_instances, n_active_types}
+    int *table_info;          // {padded rows, unsafe, n_instances, n_active_types, bits of the candidate
+                              //  table's origin (least d_lo of any type), bits of its slots per unit of d}
+    unsigned short *cand_table;   // [kCandSlots] candidate types by slot of D / L_out
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
     float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out
@@ -79,6 +97,7 @@ struct gs_ctx {
     int n_sm;
     int route_ctas_per_sm_row_p;
     int route_ctas_per_sm[GS_MAX_TYPES + 1];   // by number of types (sets the shared-memory size)
+    int reroute_ctas_per_sm[GS_MAX_TYPES + 1];
     gs::Scratch s;
     size_t max_chunks, max_groups;   // capacity of the risk scan's count arrays
     unsigned scan_epoch;             // its parity selects the group-total buffer of the next scan

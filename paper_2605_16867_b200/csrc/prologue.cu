@@ -48,8 +48,9 @@ constexpr float kShrink = 1.0f - 1.9073486328125e-6f;   // 1 - 2^-19
 
 // Upper edge of bucket b of L_out: buckets split every octave at 1.5, b = 2 * exponent + (mantissa >= 1.5).
 __device__ __forceinline__ float bucket_upper_edge(int b) {
-    const unsigned e = 127u + (unsigned)(b >> 1);
-    return __uint_as_float((b & 1) ? ((e + 1u) << 23) : ((e << 23) | 0x400000u));
+    const unsigned e = 127u + (unsigned)(b >> kBucketBits);
+    const unsigned m = ((unsigned)b & ((1u << kBucketBits) - 1u)) + 1u;
+    return __uint_as_float((m >> kBucketBits) ? ((e + 1u) << 23) : ((e << 23) | (m << (23 - kBucketBits))));
 }
 constexpr unsigned kPadQ = 0x7FC00000u;                 // NaN: compares false with everything
 
@@ -115,7 +116,8 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     __shared__ unsigned char sh_t[kDirect ? 1 : GS_MAX_INSTANCES];
     __shared__ float sh_rq[GS_MAX_INSTANCES], sh_rd[GS_MAX_INSTANCES];     // my rows: q_lo, d_lo (untagged)
     __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES];
-    __shared__ unsigned sh_dmax[GS_MAX_TYPES];
+    __shared__ unsigned sh_dmax[GS_MAX_TYPES], sh_dmin[GS_MAX_TYPES];      // by type: largest / least d
+    __shared__ unsigned sh_dlow_pos[GS_MAX_TYPES];                         // least d by position in the search order
     __shared__ unsigned sh_qmin, sh_pmin;
     __shared__ float sh_tp[GS_MAX_TYPES], sh_ta[GS_MAX_TYPES], sh_tb[GS_MAX_TYPES];   // type constants
     __shared__ int sh_unsafe, sh_fill;
@@ -126,7 +128,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     const bool writer = blockIdx.x == 0;       // one CTA writes what does not depend on the group
     const int tr = blockIdx.x;                 // position of this CTA's group in the search order
     unsigned bad = 0;
-    if (tid < GS_MAX_TYPES) { sh_cnt[tid] = 0; sh_dmax[tid] = 0u; }
+    if (tid < GS_MAX_TYPES) { sh_cnt[tid] = 0; sh_dmax[tid] = 0u; sh_dmin[tid] = 0xFFFFFFFFu; }
     if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; sh_pmin = 0xFFFFFFFFu; }
     __syncthreads();
 
@@ -169,7 +171,9 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             n_t = min(group_rows, M - base);
         }
         // ---- 3. this CTA's slice of the order, and its least p ---------------------------------
-        const bool mine = tr < n_act && tid >= base && tid < base + n_t;      // tid = rank here
+        // the least d of every group: that of its last row (tid = rank here)
+        if (has && (tid == M - 1 || (tid + 1) % group_rows == 0)) sh_dlow_pos[tid / group_rows] = ~(unsigned)(key >> 16);
+        const bool mine = tr < n_act && tid >= base && tid < base + n_t;
         if (mine) sh_key[tid - base] = key;
         const unsigned pb = mine ? (__float_as_uint(sh_p[(int)(key & 0xFFFFull)]) & 0x7FFFFFFFu) : 0xFFFFFFFFu;
         const unsigned wmin = __reduce_min_sync(0xFFFFFFFFu, pb);   // non-negative floats order like their bits
@@ -217,9 +221,11 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             // instances per type and each type's largest d: one shared-memory atomic per type and warp
             const unsigned peers = __match_any_sync(0xFFFFFFFFu, t);
             const unsigned dmax = __reduce_max_sync(peers, orderable(d));
+            const unsigned dmin = __reduce_min_sync(peers, orderable(d));
             if (t >= 0 && lane == __ffs(peers) - 1) {
                 atomicAdd(&sh_cnt[t], __popc(peers));
                 atomicMax(&sh_dmax[t], dmax);
+                atomicMin(&sh_dmin[t], dmin);
             }
         }
         __syncthreads();
@@ -233,6 +239,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                     if (sh_cnt[o] > 0 && (sh_dmax[o] > sh_dmax[tid] || (sh_dmax[o] == sh_dmax[tid] && o < tid))) ++rank;
             }
             sh_rank[tid] = rank;
+            if (rank < GS_MAX_TYPES) sh_dlow_pos[rank] = sh_dmin[tid];
         }
         __syncthreads();
         // the type this CTA builds, the padded rows before it, the number of types in use
@@ -268,6 +275,28 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         if (sh_unsafe) atomicOr(s.status, (unsigned)GS_DEV_BAD_VALUE);
     }
     if (writer && bad) atomicOr(s.status, bad);
+    // candidate table: a type can hold a feasible instance only if its least d_lo times L_out is
+    // within the deadline, so the slot of D / L_out names the types worth an entry test (slots
+    // widened by a sixteenth against the rounding of the kernel's own slot computation)
+    if (writer && tid < kCandSlots) {
+        float z0 = 3.4e38f, z1 = 0.f;
+        for (int r = 0; r < n_act; ++r) {
+            const float v = lower_bound(__uint_as_float(sh_dlow_pos[r] & 0x7FFFFFFFu));
+            z0 = fminf(z0, v); z1 = fmaxf(z1, v);
+        }
+        const bool usable = (z1 - z0) > z1 * (1.0f / 1024.0f);
+        const float edge = (z0 + ((float)tid + 1.0625f) * ((z1 - z0) / (float)kCandSlots)) * 1.00002f;
+        unsigned mask = 0;
+        for (int r = 0; r < n_act; ++r) {
+            const float v = lower_bound(__uint_as_float(sh_dlow_pos[r] & 0x7FFFFFFFu));
+            if (!usable || tid == kCandSlots - 1 || v <= edge) mask |= 1u << r;
+        }
+        s.cand_table[tid] = (unsigned short)mask;
+        if (tid == 0) {
+            s.table_info[4] = __float_as_int(z0);
+            s.table_info[5] = __float_as_int(usable ? (float)kCandSlots / (z1 - z0) : 0.f);
+        }
+    }
     if (n_t == 0) return;                      // no group at this position
     const int n_padded = (n_t + 15) & ~15;
     __syncthreads();
@@ -318,10 +347,15 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     // With P_k the running minimum of H over rows 0..k, the first row that can pass is the first
     // k with P_k <= y_hi z_edge: a binary search per slot.  Eight buckets are done at a time,
     // one warp each for the running minima, then one (bucket, slot) cell per thread.
+    if (!(inv_w > 0.f)) {       // no start table: every search of this type begins at its first row
+        for (int c = tid; c < kStartBuckets * kStartSlots; c += kPrologueThreads)
+            s.start_table[tr * kStartBuckets * kStartSlots + c] = 0;
+    }
     if (inv_w > 0.f) {
         float *sh_pm = reinterpret_cast<float *>(sh_dyn);   // [buckets per batch][n_t] running minima
         const float w_slot = 1.0f / inv_w;
         int per_batch = kPmFloats / n_t;                    // n_t <= 1024: at least 8
+        if (per_batch > kPrologueThreads / 32) per_batch = kPrologueThreads / 32;   // one warp per bucket
         if (per_batch > kStartBuckets) per_batch = kStartBuckets;
         __syncthreads();                                    // the sort is done with sh_dyn
         for (int b0 = 0; b0 < kStartBuckets; b0 += per_batch) {
@@ -352,7 +386,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 if (b >= kStartBuckets) break;
                 const bool open_ended = b == kStartBuckets - 1;
                 const float y_hi = bucket_upper_edge(b) * 1.00002f;
-                const float z_edge = d_low + (float)(slot + 2) * w_slot;
+                const float z_edge = d_low + ((float)slot + GS_SLOT_WIDEN) * w_slot;
                 const float limit = (open_ended ? z_edge : y_hi * z_edge) * 1.00002f;
                 const float *pm = sh_pm + bw * n_t;
                 int lo = 0, hi = n_t;                       // rows [0, lo) cannot pass
@@ -362,7 +396,8 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 }
                 // the top slot also takes every z beyond the table: nothing can be ruled out there
                 if (slot == kStartSlots - 1) lo = 0;
-                s.start_table[(tr * kStartBuckets + b) * kStartSlots + slot] = (unsigned char)(lo >> 3);
+                // (a cell that no row can pass begins at the type's last group: searches always have eight rows to test)
+                s.start_table[(tr * kStartBuckets + b) * kStartSlots + slot] = (unsigned char)min(lo >> 3, (n_padded >> 3) - 1);
             }
             __syncthreads();
         }

@@ -26,7 +26,14 @@
 
 namespace gs {
 
-constexpr int kRouteThreads = 256;
+#ifndef GS_ROUTE_THREADS
+#define GS_ROUTE_THREADS 256
+#endif
+#ifndef GS_ROUTE_MIN_CTAS
+#define GS_ROUTE_MIN_CTAS 4
+#endif
+constexpr int kRouteThreads = GS_ROUTE_THREADS;
+constexpr int kRouteMinCtas = GS_ROUTE_MIN_CTAS;
 #ifndef GS_REQ_PER_THREAD
 #define GS_REQ_PER_THREAD 4
 #endif
@@ -72,6 +79,7 @@ struct Tables {
     const unsigned char *start_table;
     const Row *rows;
     const float *row_p;       // per-row lower bound of p, in row order (only where p differs inside a group)
+    const unsigned short *cand;   // candidate types by slot of D / L_out
     int n_types;
 };
 
@@ -130,7 +138,7 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
     float d_best = -1.0f, T_best = 0.f;
     const float ry = __frcp_rn(y);
     // bucket of L_out: exponent and top mantissa bit of y (y >= 1 here)
-    const int ybucket = min((int)(__float_as_uint(y) >> 22) - 254, kStartBuckets - 1);
+    const int ybucket = min((int)(__float_as_uint(y) >> (23 - kBucketBits)) - (127 << kBucketBits), kStartBuckets - 1);
     // 2. search them, largest d first
     while (alive) {
         const int t = __ffs(alive) - 1;
@@ -358,41 +366,239 @@ __device__ __forceinline__ void exhaustive_pick(const Row *rows, int M, float xs
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// the routing round
+// ---------------------------------------------------------------------------------------
+
+// First row of the eight at padded index k (a multiple of 8) whose bound passes: its tag word
+// replaces `first`; rows are tested last to first so that the earliest one wins.
+template <bool kRowP>
+__device__ __forceinline__ unsigned first_pass_of_eight(const Tables &tb, int k, float x, float y, float R, unsigned first)
+{
+    const char *grp = reinterpret_cast<const char *>(tb.row_bounds + k);
+    const int sw = (k >> 4) & 3;                // see row_slot()
+    const uint4 r0 = *reinterpret_cast<const uint4 *>(grp + ((0 ^ sw) << 4));
+    const uint4 r1 = *reinterpret_cast<const uint4 *>(grp + ((1 ^ sw) << 4));
+    const uint4 r2 = *reinterpret_cast<const uint4 *>(grp + ((2 ^ sw) << 4));
+    const uint4 r3 = *reinterpret_cast<const uint4 *>(grp + ((3 ^ sw) << 4));
+    float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;      // rows k..k+3, k+4..k+7
+    if (kRowP) {
+        pa = *reinterpret_cast<const float4 *>(tb.row_p + k);
+        pb = *reinterpret_cast<const float4 *>(tb.row_p + k + 4);
+    }
+    first = row_may_pass<false, kRowP>(r3.z, r3.w, pb.w, x, y, R, 0.f) ? r3.z : first;
+    first = row_may_pass<false, kRowP>(r3.x, r3.y, pb.z, x, y, R, 0.f) ? r3.x : first;
+    first = row_may_pass<false, kRowP>(r2.z, r2.w, pb.y, x, y, R, 0.f) ? r2.z : first;
+    first = row_may_pass<false, kRowP>(r2.x, r2.y, pb.x, x, y, R, 0.f) ? r2.x : first;
+    first = row_may_pass<false, kRowP>(r1.z, r1.w, pa.w, x, y, R, 0.f) ? r1.z : first;
+    first = row_may_pass<false, kRowP>(r1.x, r1.y, pa.z, x, y, R, 0.f) ? r1.x : first;
+    first = row_may_pass<false, kRowP>(r0.z, r0.w, pa.y, x, y, R, 0.f) ? r0.z : first;
+    first = row_may_pass<false, kRowP>(r0.x, r0.y, pa.x, x, y, R, 0.f) ? r0.x : first;
+    return first;
+}
+
+// The short way to the just-enough pick, taken by every request first.  Straight-line code
+// but for two short loops over GPU types:
+//   1. the candidate table names the types whose least d fits D / L_out at all; the first of
+//      them (largest d first) that passes its entry test is searched;
+//   2. the start table gives the first group of eight rows worth a look; sixteen row bounds
+//      from there are tested, and the first row that passes is scored exactly as the
+//      definition says and checked against the deadline and the instance's free KV;
+//   3. no later type may be able to do better: its largest d is below the pick's, or even its
+//      least q with the pick's d misses the deadline.
+// Returns false whenever this does not settle the request (nothing passed within the sixteen
+// rows, the scored row is not feasible, another type may hold a better instance, no type
+// passes its entry test); the request is then queued for the full search.  When it returns
+// true the pick is the definition's: every row ranked before it was ruled out by a true lower
+// bound of its T, and every type that could rank before it by one of its whole type.
+template <bool kRowP>
+__device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float cand_inv, float x, float y,
+                                          float D, unsigned need, int &g_out, float &T_out)
+{
+    const float Dm = D + 1e-30f;                 // see route_kernel
+    float ry;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(ry) : "f"(y));
+    const float sc = fminf(fmaxf((Dm * ry - cand_z0) * cand_inv, 0.f), (float)(kCandSlots - 1));
+    unsigned mask = tb.cand[__float2int_rd(sc)];
+    int t = -1;
+    float4 h = make_float4(0.f, 0.f, 0.f, 0.f);
+    float Rg = 0.f;
+    while (mask) {
+        const int tt = __ffs(mask) - 1;
+        mask &= mask - 1;
+        h = *reinterpret_cast<const float4 *>(&tb.headers[tt]);               // p_lo, q_lo, d_lo, d_max
+        Rg = __fmaf_rn(-h.x, x, Dm);
+        if (__fmaf_rn(h.z, y, h.y) <= Rg) { t = tt; break; }
+    }
+    if (t < 0) return false;
+    const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, inv_w, d0
+    const int ybucket = min((int)(__float_as_uint(y) >> (23 - kBucketBits)) - (127 << kBucketBits), kStartBuckets - 1);
+    const float z = (Rg - h.y) * ry;             // about the largest d that can still meet the deadline
+    const float sf = fminf(fmaxf((z - __int_as_float(geo.w)) * __int_as_float(geo.z), 0.f), (float)(kStartSlots - 1));
+    const int k = geo.x + 8 * tb.start_table[(t * kStartBuckets + ybucket) * kStartSlots + __float2int_rd(sf)];
+    const int k2 = min(k + 8, geo.x + geo.y - 8);        // (the last group of a type is tested twice)
+    const float R = kRowP ? Dm : Rg;
+    unsigned first = first_pass_of_eight<kRowP>(tb, k2, x, y, R, kNoRow);
+    first = first_pass_of_eight<kRowP>(tb, k, x, y, R, first);
+    if (first == kNoRow) return false;
+    const int inst = (int)(first & kRowTagMask);
+    const Row row = tb.rows[inst];
+    const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));          // Eq. 2, H = 0
+    if (!(T <= D && need <= (unsigned)row.kv)) return false;
+    const float d_floor = __fmul_rn(row.d, 1.0f - 1.9073486328125e-6f);       // the bound every row with d >= the pick's carries
+    while (mask) {
+        const int tt = __ffs(mask) - 1;
+        mask &= mask - 1;
+        const float4 h2 = *reinterpret_cast<const float4 *>(&tb.headers[tt]);
+        if (h2.w < row.d) break;                                              // nor can any type after it
+        if (__fmaf_rn(fmaxf(h2.z, d_floor), y, h2.y) <= __fmaf_rn(-h2.x, x, Dm)) return false;
+    }
+    g_out = inst;
+    T_out = T;
+    return true;
+}
+
+// The full search for one request per lane (lanes without a request pass active = false):
+// the just-enough pick over all types, then the fallback of Algorithm 1 -- by the lane itself
+// when several lanes need it, by the whole warp otherwise and for requests that the tables
+// cannot serve (L_out == 0, unusable coefficients).
+template <bool kRowP>
+__device__ __noinline__ Pick full_pick(const Tables tb, int M, int lane, bool active, int xi, int yi, float D)
+{
+    const unsigned need = (unsigned)xi + (unsigned)yi;      // < 2^32, no overflow
+    const float x = __int2float_rn(xi), y = __int2float_rn(yi);
+    // an empty lane, or L_out == 0 (the start table divides by it), skips the search; the hair
+    // added to the deadline of the bound tests keeps them safe when a bound's tag bits make a
+    // zero coefficient a denormal
+    const float Dj = (active && yi > 0) ? D : -1.0f;
+    Pick out;
+    out.T = 0.f;
+    out.g = pick_instance<false, kRowP>(tb, x, y, Dj, Dj + 1e-30f, need, 0.f, out.T);
+    out.tier = 1u;
+    bool open = active && out.g < 0;
+    const bool mine = open && yi > 0 && tb.n_types > 0;
+    const int n_fall = __popc(__ballot_sync(0xFFFFFFFFu, mine));
+    if (mine && n_fall >= kThreadFallbackMin) {
+        out = fallback_pick<false, kRowP>(tb, x, y, need, 0.f);
+        open = false;
+    }
+    unsigned todo = __ballot_sync(0xFFFFFFFFu, open);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const float xs = __shfl_sync(0xFFFFFFFFu, x, src), ys = __shfl_sync(0xFFFFFFFFu, y, src);
+        const float Ds = __shfl_sync(0xFFFFFFFFu, D, src);
+        const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
+        int gg; float TT; unsigned tt;
+        exhaustive_pick<false>(tb.rows, M, xs, ys, Ds, needs, 0.f, lane, gg, TT, tt);
+        if (lane == src) { out.g = gg; out.T = TT; out.tier = tt; }
+    }
+    return out;
+}
+
+// Prefix-cache term of Eq. 2 for one (instance, hit length) pair of a request whose hit-free
+// pick is (g_cur, T_cur, tier): on the named instance T is lower by p * H; it is scored again
+// with its hit and merged into the answer.
+__device__ __forceinline__ void merge_hit(const Row *rows, int M, int g, int h, int xi, int yi, float D,
+                                          int &g_cur, float &T_cur, unsigned &tier, unsigned &bad)
+{
+    if (g < 0) return;                                       // empty slot
+    if (g >= M) { bad |= GS_DEV_BAD_INSTANCE; return; }      // names nothing
+    if (h < 0 || h > xi) { bad |= GS_DEV_BAD_VALUE; h = h < 0 ? 0 : xi; }
+    const Row row = rows[g];
+    const float T = __fmaf_rn(row.d, __int2float_rn(yi), __fmaf_rn(row.p, __int2float_rn(xi - h), row.q));
+    const bool room = (unsigned)xi + (unsigned)yi <= (unsigned)row.kv;
+    bool take;
+    if (room && T <= D) {                                    // feasible with its hit
+        const float d_cur = tier == 1u ? rows[g_cur].d : 0.f;
+        take = tier != 1u || row.d > d_cur || (row.d == d_cur && g < g_cur) || (g == g_cur && T < T_cur);
+        if (take) tier = 1u;
+    } else {                                                 // may still lead the fallback
+        take = tier >= 2u && (room || tier == 3u) && (T < T_cur || (T == T_cur && g < g_cur));
+    }
+    if (take) { g_cur = g; T_cur = T; }
+}
+
+constexpr int kQueueCap = 64;           // per warp: at most 31 left over + 32 new entries
+
+// A warp takes 128 consecutive requests at a time, four per lane (128-bit column loads and
+// stores).  Every request first tries fast_pick; the ones it does not settle are put on the
+// warp's queue in shared memory, and whenever 32 have gathered each lane takes one of them
+// through full_pick, so the long, divergent search always runs with all lanes busy.  Their
+// results are stored one by one over the placeholders that the tile's vector stores left.
 template <bool kAccumulate, bool kPrefix, bool kRowP>
-__global__ void __launch_bounds__(kRouteThreads, kRowP ? 3 : 4)
+__global__ void __launch_bounds__(kRouteThreads, kRowP ? (kRouteMinCtas > 3 ? 3 : kRouteMinCtas) : kRouteMinCtas)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
              const float *__restrict__ slo_ms, int64_t n, const PrefixHits hits, int n_types_alloc,
              const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
              const unsigned char *__restrict__ g_start_table,
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
-             const float *__restrict__ g_row_p,
+             const unsigned short *__restrict__ g_cand, const float *__restrict__ g_row_p,
              int32_t *__restrict__ out_idx, float *__restrict__ out_est,
              float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     const int M = table_info[2];
+    const float cand_z0 = __int_as_float(table_info[4]), cand_inv = __int_as_float(table_info[5]);
     Tables tb;
     unsigned char *after_tables = stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_start_table, g_headers,
                                                table_info, tb, kRowP ? g_row_p : nullptr);
-    const Row *sh_rows = tb.rows;
+    unsigned short *sh_cand = reinterpret_cast<unsigned short *>(after_tables);
+    if (threadIdx.x < kCandSlots) sh_cand[threadIdx.x] = g_cand[threadIdx.x];
+    tb.cand = sh_cand;
+    after_tables += kCandSlots * sizeof(unsigned short);
+    // the warps' queues: {L_in, L_out, bits of D, low word of the request index}, high word
+    int4 *queue = reinterpret_cast<int4 *>(after_tables) + (threadIdx.x >> 5) * kQueueCap;
+    after_tables += (kRouteThreads / 32) * kQueueCap * sizeof(int4);
+    int *queue_hi = reinterpret_cast<int *>(after_tables) + (threadIdx.x >> 5) * kQueueCap;
+    after_tables += (kRouteThreads / 32) * kQueueCap * sizeof(int);
     unsigned long long *hist = reinterpret_cast<unsigned long long *>(after_tables);
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
     __syncthreads();
 
     const int lane = threadIdx.x & 31;
+    const bool fast_on = tb.n_types > 0;          // unusable bounds: every request takes the full search
     unsigned bad = 0;
-    // a warp takes 128 consecutive requests at a time; nothing below needs a CTA barrier
+    int q_count = 0;                               // entries on this warp's queue (same in all lanes)
+
+    // takes up to 32 queued requests (the newest) through the full search and stores their results
+    auto drain = [&]() {
+        const int cnt = min(q_count, 32);
+        q_count -= cnt;
+        const bool active = lane < cnt;
+        int4 e = make_int4(0, 0, 0, 0);
+        int e_hi = 0;
+        if (active) { e = queue[q_count + lane]; e_hi = queue_hi[q_count + lane]; }
+        __syncwarp();                              // the slots may be written again
+        const int64_t r = ((int64_t)e_hi << 32) | (unsigned)e.w;
+        const float D = __int_as_float(e.z);
+        const Pick pk = full_pick<kRowP>(tb, M, lane, active, e.x, e.y, D);
+        int g = pk.g; float T = pk.T; unsigned tier = pk.tier;
+        if (kPrefix && active)
+            for (int k = 0; k < hits.n_slots; ++k)
+                merge_hit(tb.rows, M, hits.inst[(int64_t)k * hits.slot_stride + r],
+                          hits.hit_len[(int64_t)k * hits.slot_stride + r], e.x, e.y, D, g, T, tier, bad);
+        if (kAccumulate) accumulate_choice(hist, M, active ? g : -1, (unsigned)e.x, (unsigned)e.x + (unsigned)e.y);
+        if (active) {
+            out_idx[r] = g;
+            out_est[r] = T;
+            out_slack[r] = __fsub_rn(D, T);
+            if (out_tier) out_tier[r] = (uint8_t)tier;
+        }
+    };
+
     constexpr int kWarpTile = 32 * kReqPerThread;
     const int64_t n_wtiles = (n + kWarpTile - 1) / kWarpTile;
     const int64_t warp_stride = (int64_t)gridDim.x * (kRouteThreads / 32);
     for (int64_t wt = (int64_t)blockIdx.x * (kRouteThreads / 32) + (threadIdx.x >> 5); wt < n_wtiles;
          wt += warp_stride) {
         const int64_t first = wt * kWarpTile + (int64_t)lane * kReqPerThread;
+        const bool full = first + kReqPerThread <= n;
         int xi[kReqPerThread], yi[kReqPerThread];
         float D[kReqPerThread];
-        if (kReqPerThread == 4 && first + kReqPerThread <= n) {
+        if (full) {
             const int4 xv = __ldcs(reinterpret_cast<const int4 *>(prompt_len + first));
             const int4 yv = __ldcs(reinterpret_cast<const int4 *>(pred_decode_len + first));
             const float4 dv = __ldcs(reinterpret_cast<const float4 *>(slo_ms + first));
@@ -408,71 +614,28 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 D[j] = v ? slo_ms[first + j] : -1.0f;
             }
         }
+        if ((xi[0] | xi[1] | xi[2] | xi[3] | yi[0] | yi[1] | yi[2] | yi[3]) < 0) {      // negative counts read as 0
+#pragma unroll
+            for (int j = 0; j < kReqPerThread; ++j) { xi[j] = max(xi[j], 0); yi[j] = max(yi[j], 0); }
+            bad |= GS_DEV_BAD_VALUE;
+        }
         int g_out[kReqPerThread];
         float T_out[kReqPerThread];
         unsigned tiers = 0x01010101u;             // one byte per request
+        unsigned slow = 0;                        // bit j: request j of this lane goes to the queue
 #pragma unroll
         for (int j = 0; j < kReqPerThread; ++j) {
-            if (xi[j] < 0) { xi[j] = 0; bad |= GS_DEV_BAD_VALUE; }
-            if (yi[j] < 0) { yi[j] = 0; bad |= GS_DEV_BAD_VALUE; }
-            const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];      // < 2^32, no overflow
             const bool valid = first + j < n;
-            const float x = __int2float_rn(xi[j]), y = __int2float_rn(yi[j]);
-            // an empty slot, or L_out == 0 (the start table divides by it), skips the search;
-            // a real request that comes back empty-handed goes to the exhaustive path below.
-            // (the hair added to the deadline of the bound tests keeps them safe when a bound's
-            // tag bits make a zero coefficient a denormal)
-            const float Dj = (valid && yi[j] > 0) ? D[j] : -1.0f;
-            g_out[j] = pick_instance<false, kRowP>(tb, x, y, Dj, Dj + 1e-30f, need, 0.f, T_out[j]);
+            g_out[j] = -1; T_out[j] = 0.f;
+            // (an empty slot, or L_out == 0, which the start table cannot take, gets a deadline that
+            // nothing meets and so ends up in the full search)
+            bool settled = false;
+            if (fast_on)
+                settled = fast_pick<kRowP>(tb, cand_z0, cand_inv, __int2float_rn(xi[j]), __int2float_rn(yi[j]),
+                                           (valid && yi[j] > 0) ? D[j] : -1.0f, (unsigned)xi[j] + (unsigned)yi[j], g_out[j], T_out[j]);
+            if (valid && !settled) slow |= 1u << j;
         }
-        // ---- requests still without an instance: nothing is feasible (the fallback of
-        // Algorithm 1), or L_out == 0, or tables whose bounds cannot be used ----------------------
-        unsigned pend = 0, mine = 0;                 // bit j: request j of this lane is open / may search by itself
-#pragma unroll
-        for (int j = 0; j < kReqPerThread; ++j) {
-            const bool open = first + j < n && g_out[j] < 0;
-            pend |= (unsigned)open << j;
-            mine |= (unsigned)(open && yi[j] > 0 && tb.n_types > 0) << j;
-        }
-        if (__any_sync(0xFFFFFFFFu, pend != 0)) {
-            // several in the warp: each lane searches for its own; few: the warp shares each one
-            const int n_fall = (int)__reduce_add_sync(0xFFFFFFFFu, (unsigned)__popc(mine));
-            if (n_fall >= kThreadFallbackMin) {
-#pragma unroll
-                for (int j = 0; j < kReqPerThread; ++j)
-                    if ((mine >> j) & 1u) {
-                        const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];
-                        const Pick r = fallback_pick<false, kRowP>(tb, __int2float_rn(xi[j]), __int2float_rn(yi[j]),
-                                                                   need, 0.f);
-                        g_out[j] = r.g; T_out[j] = r.T;
-                        tiers = (tiers & ~(0xFFu << (8 * j))) | (r.tier << (8 * j));
-                        pend &= ~(1u << j);
-                    }
-            }
-#pragma unroll
-            for (int j = 0; j < kReqPerThread; ++j) {
-                unsigned todo = __ballot_sync(0xFFFFFFFFu, (pend >> j) & 1u);
-                const unsigned need = (unsigned)xi[j] + (unsigned)yi[j];
-                while (todo) {
-                    const int src = __ffs(todo) - 1;
-                    todo &= todo - 1;
-                    const float xs = __shfl_sync(0xFFFFFFFFu, __int2float_rn(xi[j]), src);
-                    const float ys = __shfl_sync(0xFFFFFFFFu, __int2float_rn(yi[j]), src);
-                    const float Ds = __shfl_sync(0xFFFFFFFFu, D[j], src);
-                    const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
-                    int g; float T; unsigned tier;
-                    exhaustive_pick<false>(sh_rows, M, xs, ys, Ds, needs, 0.f, lane, g, T, tier);
-                    if (lane == src) {
-                        g_out[j] = g; T_out[j] = T;
-                        tiers = (tiers & ~(0xFFu << (8 * j))) | (tier << (8 * j));
-                    }
-                }
-            }
-        }
-        // ---- prefix-cache term of Eq. 2: on the instances that hold a prefix of the request T
-        // is lower by p * H; each is scored again with its hit and merged into the answer ------
         if (kPrefix) {
-            const bool full = kReqPerThread == 4 && first + kReqPerThread <= n;
             for (int k = 0; k < hits.n_slots; ++k) {
                 const int32_t *col_g = hits.inst + (int64_t)k * hits.slot_stride;
                 const int32_t *col_h = hits.hit_len + (int64_t)k * hits.slot_stride;
@@ -492,38 +655,18 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 }
 #pragma unroll
                 for (int j = 0; j < kReqPerThread; ++j) {
-                    const int g = hg[j];
-                    if (g < 0) continue;                                     // empty slot
-                    if (g >= M) { bad |= GS_DEV_BAD_INSTANCE; continue; }    // names nothing
-                    int h = hh[j];
-                    if (h < 0 || h > xi[j]) { bad |= GS_DEV_BAD_VALUE; h = h < 0 ? 0 : xi[j]; }
-                    const Row row = sh_rows[g];
-                    const float T = __fmaf_rn(row.d, __int2float_rn(yi[j]),
-                                              __fmaf_rn(row.p, __int2float_rn(xi[j] - h), row.q));
-                    const bool room = (unsigned)xi[j] + (unsigned)yi[j] <= (unsigned)row.kv;
-                    const unsigned tier = (tiers >> (8 * j)) & 0xFFu;
-                    const int g_cur = g_out[j];
-                    bool take;
-                    if (room && T <= D[j]) {                                 // feasible with its hit
-                        const float d_cur = tier == 1u ? sh_rows[g_cur].d : 0.f;
-                        take = tier != 1u || row.d > d_cur || (row.d == d_cur && g < g_cur) ||
-                               (g == g_cur && T < T_out[j]);
-                        if (take) tiers = (tiers & ~(0xFFu << (8 * j))) | (1u << (8 * j));
-                    } else {                                                 // may still lead the fallback
-                        take = tier >= 2u && (room || tier == 3u) &&
-                               (T < T_out[j] || (T == T_out[j] && g < g_cur));
-                    }
-                    if (take) { g_out[j] = g; T_out[j] = T; }
+                    if (g_out[j] < 0) continue;                      // queued: merged after the full search
+                    unsigned tier = 1u;
+                    merge_hit(tb.rows, M, hg[j], hh[j], xi[j], yi[j], D[j], g_out[j], T_out[j], tier, bad);
                 }
             }
         }
         if (kAccumulate) {
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j)
-                accumulate_choice(hist, M, first + j < n ? g_out[j] : -1, (unsigned)xi[j],
-                                  (unsigned)xi[j] + (unsigned)yi[j]);
+                accumulate_choice(hist, M, g_out[j], (unsigned)xi[j], (unsigned)xi[j] + (unsigned)yi[j]);
         }
-        if (kReqPerThread == 4 && first + kReqPerThread <= n) {
+        if (full) {
             __stcs(reinterpret_cast<int4 *>(out_idx + first), make_int4(g_out[0], g_out[1], g_out[2], g_out[3]));
             __stcs(reinterpret_cast<float4 *>(out_est + first), make_float4(T_out[0], T_out[1], T_out[2], T_out[3]));
             __stcs(reinterpret_cast<float4 *>(out_slack + first),
@@ -537,10 +680,30 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                     out_idx[first + j] = g_out[j];
                     out_est[first + j] = T_out[j];
                     out_slack[first + j] = __fsub_rn(D[j], T_out[j]);
-                    if (out_tier) out_tier[first + j] = (uint8_t)((tiers >> (8 * j)) & 0xFFu);
+                    if (out_tier) out_tier[first + j] = (uint8_t)1;
                 }
         }
+        // ---- queue what is open; run the full search whenever 32 requests have gathered ---------
+        if (__any_sync(0xFFFFFFFFu, slow != 0)) {
+            __syncwarp();                          // the stores above come before the drain's
+#pragma unroll
+            for (int j = 0; j < kReqPerThread; ++j) {
+                const bool push = (slow >> j) & 1u;
+                const unsigned votes = __ballot_sync(0xFFFFFFFFu, push);
+                if (votes == 0) continue;
+                if (push) {
+                    const int pos = q_count + __popc(votes & ((1u << lane) - 1u));
+                    const int64_t r = first + j;
+                    queue[pos] = make_int4(xi[j], yi[j], __float_as_int(D[j]), (int)(unsigned)(r & 0xFFFFFFFFll));
+                    queue_hi[pos] = (int)(r >> 32);
+                }
+                q_count += __popc(votes);
+                __syncwarp();
+                if (q_count >= 32) drain();
+            }
+        }
     }
+    while (q_count > 0) { __syncwarp(); drain(); }
     if (bad) atomicOr(status, bad);
 
     if (kAccumulate) {
@@ -552,8 +715,10 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     }
 }
 
-constexpr size_t kRouteSmemFixed = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
-                                   (size_t)kMaxPaddedRows * sizeof(uint2);
+constexpr size_t kTablesSmemFixed = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
+                                    (size_t)kMaxPaddedRows * sizeof(uint2);
+constexpr size_t kRouteSmemFixed = kTablesSmemFixed + kCandSlots * sizeof(unsigned short) +
+                                   (size_t)(kRouteThreads / 32) * kQueueCap * (sizeof(int4) + sizeof(int));
 constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
 constexpr size_t kRouteSmemRowP = (size_t)kMaxPaddedRows * sizeof(float);
@@ -574,7 +739,8 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
 #define GS_LAUNCH_ROUTE(ACC, PFX, ROWP)                                                               \
     route_kernel<ACC, PFX, ROWP><<<(unsigned)blocks, kRouteThreads, smem, st>>>(                       \
         prompt_len, pred_decode_len, slo_ms, n, hits ? *hits : none, n_types, ctx->s.rows,            \
-        ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, ctx->s.row_p,       \
+        ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, ctx->s.cand_table,  \
+        ctx->s.row_p,                                                                                 \
         out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status)
     // (the prefix term and per-row p are never combined with accumulate, nor with each other)
     if (row_p) GS_LAUNCH_ROUTE(false, false, true);
@@ -593,7 +759,7 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
 // into the request that a token-ID migration would pose to the target (re-prefill prompt +
 // generated tokens, decode what is left, within the time that is left) and runs the same
 // search as the routing round, restricted to instances with d < d of the current instance.
-__global__ void __launch_bounds__(kRouteThreads, 4)
+__global__ void __launch_bounds__(kRouteThreads, 1024 / kRouteThreads)
 reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__ cand_count, int64_t cand_capacity,
                const int32_t *__restrict__ assigned, const int32_t *__restrict__ generated,
                const int32_t *__restrict__ pred_len, const float *__restrict__ elapsed,
@@ -674,9 +840,9 @@ cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *
                            cudaStream_t st)
 {
     if (cand_capacity == 0) return cudaSuccess;
-    const size_t smem = kRouteSmemFixed + kRouteSmemPerType * n_types;
+    const size_t smem = kTablesSmemFixed + kRouteSmemPerType * n_types;
     int64_t blocks = (cand_capacity + kRouteThreads - 1) / kRouteThreads;
-    const int64_t cap = (int64_t)ctx->n_sm * ctx->route_ctas_per_sm[n_types];
+    const int64_t cap = (int64_t)ctx->n_sm * ctx->reroute_ctas_per_sm[n_types];
     if (blocks > cap) blocks = cap;
     LaunchTimer timer(ctx, GS_K_REROUTE, st);
     reroute_kernel<<<(unsigned)blocks, kRouteThreads, smem, st>>>(
@@ -716,6 +882,10 @@ cudaError_t configure_route(gs_ctx *ctx)
                                                           kRouteSmemFixed + kRouteSmemPerType * t);
         if (e != cudaSuccess) return e;
         ctx->route_ctas_per_sm[t] = occ > 0 ? occ : 1;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, reroute_kernel, kRouteThreads,
+                                                          kTablesSmemFixed + kRouteSmemPerType * t);
+        if (e != cudaSuccess) return e;
+        ctx->reroute_ctas_per_sm[t] = occ > 0 ? occ : 1;
     }
     return cudaSuccess;
 }
