@@ -164,6 +164,9 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
         {(void **)&s.headers, GS_MAX_TYPES * sizeof(gs::TypeHeader)},
         {(void **)&s.table_info, 64},
         {(void **)&s.cand_table, gs::kCandSlots * sizeof(unsigned short)},
+        {(void **)&s.pool, gs::kPoolEntries * sizeof(uint2)},
+        {(void **)&s.bucket_list, (size_t)GS_MAX_TYPES * gs::kStartBuckets * sizeof(unsigned short)},
+        {(void **)&s.start_list, (size_t)GS_MAX_TYPES * gs::kStartBuckets * gs::kStartSlots},
         {(void **)&s.d_by_g, Mx * sizeof(float)},
         {(void **)&s.q_by_g, Mx * sizeof(float)},
         {(void **)&s.deltas, 3 * Mx * sizeof(unsigned long long)},
@@ -188,7 +191,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.group_totals, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.group_totals, s.status, ctx->stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);

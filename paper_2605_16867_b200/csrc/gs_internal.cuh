@@ -67,6 +67,18 @@ struct __align__(16) TypeHeader {
 // name every type.
 constexpr int kCandSlots = 64;
 
+// Record lists (typed pools).  For every GPU type and bucket of L_out the rows that can be the
+// first of their type to pass a bound test (see the prologue), as {q word, d_lo} entries in one
+// pool; a list ends in kListWindow entries that never pass, so a window of that many entries
+// read from any start inside the list stays inside it.
+#ifndef GS_POOL_ENTRIES
+#define GS_POOL_ENTRIES 8192
+#endif
+constexpr int kPoolEntries = GS_POOL_ENTRIES;
+constexpr int kListWindow = 4;             // entries the first attempt tests
+constexpr int kListMax = 510;              // longer lists are not stored (start_list counts pairs of entries in a byte)
+constexpr unsigned short kNoList = 0xFFFFu;
+
 constexpr int kRiskChunk = 1024;        // requests per warp-chunk of the risk scan (32 flag words)
 constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 
@@ -78,8 +90,12 @@ struct Scratch {
     unsigned char *start_table;   // [GS_MAX_TYPES * kStartBuckets * kStartSlots]
     TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)
     int *table_info;          // {padded rows, unsafe, n_instances, n_active_types, bits of the candidate
-                              //  table's origin (least d_lo of any type), bits of its slots per unit of d}
+                              //  table's origin (least d_lo of any type), bits of its slots per unit of d,
+                              //  pool entries handed out to the types}
     unsigned short *cand_table;   // [kCandSlots] candidate types by slot of D / L_out
+    uint2 *pool;              // [kPoolEntries] record lists
+    unsigned short *bucket_list;  // [GS_MAX_TYPES * kStartBuckets] first pool entry of the list, halved; kNoList = none
+    unsigned char *start_list;    // [GS_MAX_TYPES * kStartBuckets * kStartSlots] like start_table, in pairs of list entries
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
     float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out

@@ -54,6 +54,9 @@ __device__ __forceinline__ float bucket_upper_edge(int b) {
 }
 constexpr unsigned kPadQ = 0x7FC00000u;                 // NaN: compares false with everything
 
+// Entries of the record-list pool that a type with n of the pool's M instances may use.
+__device__ __forceinline__ int pool_share_of(int n, int M) { return (int)(((long long)kPoolEntries * n) / M) & ~3; }
+
 // Bit pattern of a lower bound of v >= 0 whose low tag bits are zero and may be overwritten.
 __device__ __forceinline__ unsigned lower_bound_bits(float v) {
     const unsigned b = __float_as_uint(__fmul_rn(v, kShrink)) & ~kRowTagMask;
@@ -114,13 +117,14 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     __shared__ float sh_q[GS_MAX_INSTANCES], sh_d[GS_MAX_INSTANCES];       // by instance index
     __shared__ float sh_p[kDirect ? GS_MAX_INSTANCES : 1];                 // kDirect: p by instance index
     __shared__ unsigned char sh_t[kDirect ? 1 : GS_MAX_INSTANCES];
-    __shared__ float sh_rq[GS_MAX_INSTANCES], sh_rd[GS_MAX_INSTANCES];     // my rows: q_lo, d_lo (untagged)
+    __shared__ float sh_rq[GS_MAX_INSTANCES], sh_rd[GS_MAX_INSTANCES];     // my rows: q_lo (tagged), d_lo
     __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES];
     __shared__ unsigned sh_dmax[GS_MAX_TYPES], sh_dmin[GS_MAX_TYPES];      // by type: largest / least d
     __shared__ unsigned sh_dlow_pos[GS_MAX_TYPES];                         // least d by position in the search order
     __shared__ unsigned sh_qmin, sh_pmin;
     __shared__ float sh_tp[GS_MAX_TYPES], sh_ta[GS_MAX_TYPES], sh_tb[GS_MAX_TYPES];   // type constants
     __shared__ int sh_unsafe, sh_fill;
+    __shared__ int sh_len[kPrologueThreads / 32], sh_off[kPrologueThreads / 32], sh_pool_used;
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -134,6 +138,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
 
     const bool has = tid < M;
     int base = 0, n_act = 0, padded_total = 0, n_t = 0;
+    int pool_base = 0, pool_share = 0, pool_total = 0;     // record lists: this type's part of the pool
     float p_group = 0.f;                       // lower bound source: the least p of the group
 
     if (kDirect) {
@@ -249,8 +254,9 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             if (n == 0) continue;
             ++n_act;
             padded_total += (n + 15) & ~15;
-            if (r == tr) my_type = o;
-            if (r < tr) base += (n + 15) & ~15;
+            if (r == tr) { my_type = o; pool_share = pool_share_of(n, M); }
+            if (r < tr) { base += (n + 15) & ~15; pool_base += pool_share_of(n, M); }
+            pool_total += pool_share_of(n, M);
         }
         if (my_type >= 0) {
             n_t = sh_cnt[my_type];
@@ -272,6 +278,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         s.table_info[1] = sh_unsafe;
         s.table_info[2] = M;
         s.table_info[3] = n_act;
+        s.table_info[6] = pool_total;
         if (sh_unsafe) atomicOr(s.status, (unsigned)GS_DEV_BAD_VALUE);
     }
     if (writer && bad) atomicOr(s.status, bad);
@@ -311,7 +318,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             const unsigned q_bits = lower_bound_bits(sh_q[inst]);
             const float d_lo = lower_bound(sh_d[inst]);
             entry = make_uint2(q_bits | (unsigned)inst, __float_as_uint(d_lo));
-            sh_rq[k] = __uint_as_float(q_bits);
+            sh_rq[k] = __uint_as_float(q_bits | (unsigned)inst);    // as the kernel tests it
             sh_rd[k] = d_lo;
             my_qmin = min(my_qmin, q_bits);             // non-negative floats order like their bits
         }
@@ -326,7 +333,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     const float q0 = __uint_as_float(sh_qmin);
     const float d_hi = sh_rd[0], d_low = sh_rd[n_t - 1];
     float inv_w = 0.f;              // slots per unit of d; 0 = no start table (search from row 0)
-    if (n_t > 16 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f)) inv_w = (float)kStartSlots / (d_hi - d_low);
+    if (n_t > 4 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f)) inv_w = (float)kStartSlots / (d_hi - d_low);
     if (tid == 0) {
         const int first_inst = (int)(sh_key[0] & 0xFFFFull);
         TypeHeader h;
@@ -341,70 +348,122 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         s.headers[tr] = h;
     }
 
-    // ---- 6. start table -------------------------------------------------------------------------
-    // For bucket b put  H_k = (q_lo_k - q0) + y_hi d_lo_k.  A row can pass only if
-    // H_k <= y_hi z_edge (see the header comment; rows with d_lo above z_edge fail that too).
-    // With P_k the running minimum of H over rows 0..k, the first row that can pass is the first
-    // k with P_k <= y_hi z_edge: a binary search per slot.  Eight buckets are done at a time,
-    // one warp each for the running minima, then one (bucket, slot) cell per thread.
-    if (!(inv_w > 0.f)) {       // no start table: every search of this type begins at its first row
-        for (int c = tid; c < kStartBuckets * kStartSlots; c += kPrologueThreads)
-            s.start_table[tr * kStartBuckets * kStartSlots + c] = 0;
-    }
-    if (inv_w > 0.f) {
-        float *sh_pm = reinterpret_cast<float *>(sh_dyn);   // [buckets per batch][n_t] running minima
-        const float w_slot = 1.0f / inv_w;
+    // ---- 6. start tables and record lists -----------------------------------------------------
+    // For bucket b put  H_k = (q_k - q0) + y_hi d_lo_k  with q_k the row's tagged bound, the value
+    // the kernel tests.  A row can pass only if H_k <= y_hi z_edge (see the header comment; rows
+    // with d_lo above z_edge fail that too).  With P_k the running minimum of H over rows 0..k,
+    // the first row that can pass is the first k with P_k <= y_hi z_edge: a binary search per
+    // slot.
+    // Record list.  Row k is a record of the bucket if H_k < P_(k-1).  A row that is not has an
+    // earlier row j with q_j + y_hi d_lo_j <= q_k + y_hi d_lo_k and d_lo_j >= d_lo_k, hence
+    // q_j + y d_lo_j <= q_k + y d_lo_k for every y <= y_hi: whenever its bound passes so does
+    // that of row j, so it is never the first row to pass and the kernel's first attempt need
+    // not look at it.  Each bucket's records are stored as a list of their own (while the
+    // type's share of the pool lasts, shortest lists first) with a second start table that
+    // counts in list entries.  Up to 32 buckets are done at a time, one warp each for the
+    // running minima and record counts, then one (bucket, slot) cell per thread.
+    {
+        float *sh_pm = reinterpret_cast<float *>(sh_dyn);                         // [buckets per batch][n_t] running minima
+        unsigned short *sh_pc = reinterpret_cast<unsigned short *>(sh_pm + kPmFloats);   // records before each row
+        const float w_slot = inv_w > 0.f ? 1.0f / inv_w : 0.f;
         int per_batch = kPmFloats / n_t;                    // n_t <= 1024: at least 8
         if (per_batch > kPrologueThreads / 32) per_batch = kPrologueThreads / 32;   // one warp per bucket
         if (per_batch > kStartBuckets) per_batch = kStartBuckets;
+        if (tid == 0) sh_pool_used = 0;
         __syncthreads();                                    // the sort is done with sh_dyn
         for (int b0 = 0; b0 < kStartBuckets; b0 += per_batch) {
-            if (warp < per_batch && b0 + warp < kStartBuckets) {
+            const bool my_bucket = warp < per_batch && b0 + warp < kStartBuckets;
+            if (my_bucket) {
                 const int b = b0 + warp;
                 // bucket b holds y in [2^e (1 + m/2), 2^e (1 + (m+1)/2)),  e = b >> 1, m = b & 1;
                 // the last bucket has no upper edge: there only d_lo <= z_edge can be required
                 const bool open_ended = b == kStartBuckets - 1;
                 const float y_hi = bucket_upper_edge(b) * 1.00002f;
                 float carry = 3.4e38f;
+                int n_rec = 0;
                 for (int k0 = 0; k0 < n_t; k0 += 32) {
                     const int k = k0 + lane;
-                    float h = 3.4e38f;
-                    if (k < n_t) h = open_ended ? sh_rd[k] : __fmaf_rn(y_hi, sh_rd[k], sh_rq[k] - q0);
+                    float own = 3.4e38f;
+                    if (k < n_t) own = open_ended ? sh_rd[k] : __fmaf_rn(y_hi, sh_rd[k], sh_rq[k] - q0);
+                    float h = own;
 #pragma unroll
                     for (int off = 1; off < 32; off <<= 1) {
                         const float up = __shfl_up_sync(0xFFFFFFFFu, h, off);
                         if (lane >= off) h = fminf(h, up);
                     }
                     h = fminf(h, carry);
-                    if (k < n_t) sh_pm[warp * n_t + k] = h;
+                    float before = __shfl_up_sync(0xFFFFFFFFu, h, 1);       // minimum over the rows before k
+                    if (lane == 0) before = carry;
+                    // (kept unless an earlier row is below it by more than the rounding of H)
+                    const bool rec = k < n_t && !(before * 1.000001f <= own);
+                    const unsigned votes = __ballot_sync(0xFFFFFFFFu, rec);
+                    if (k < n_t) {
+                        sh_pm[warp * n_t + k] = h;
+                        sh_pc[warp * n_t + k] = (unsigned short)(n_rec + __popc(votes & ((1u << lane) - 1u)));
+                    }
+                    n_rec += __popc(votes);
                     carry = __shfl_sync(0xFFFFFFFFu, h, 31);
                 }
+                if (lane == 0) sh_len[warp] = n_rec;
             }
             __syncthreads();
+            if (tid == 0) {                                 // room in the pool, in bucket order
+                int used = sh_pool_used;
+                for (int wb = 0; wb < per_batch && b0 + wb < kStartBuckets; ++wb) {
+                    const int len = sh_len[wb];
+                    const int need = (len + kListWindow + 1) & ~1;      // padded: a window never leaves its list
+                    const bool fits = !kDirect && b0 + wb != kStartBuckets - 1 && len <= kListMax &&
+                                      used + need <= pool_share;
+                    sh_off[wb] = fits ? pool_base + used : -1;
+                    if (fits) used += need;
+                }
+                sh_pool_used = used;
+            }
+            __syncthreads();
+            if (my_bucket && !kDirect) {
+                const int off = sh_off[warp], len = sh_len[warp];
+                if (off >= 0) {
+                    const unsigned short *pc = sh_pc + warp * n_t;
+                    for (int k = lane; k < n_t; k += 32) {
+                        const int c = pc[k], c_next = k + 1 < n_t ? pc[k + 1] : len;
+                        if (c_next != c)
+                            s.pool[off + c] = make_uint2(__float_as_uint(sh_rq[k]), __float_as_uint(sh_rd[k]));
+                    }
+                    for (int k = len + lane; k < ((len + kListWindow + 1) & ~1); k += 32)
+                        s.pool[off + k] = make_uint2(kPadQ, 0u);
+                }
+                if (lane == 0)
+                    s.bucket_list[tr * kStartBuckets + b0 + warp] = off >= 0 ? (unsigned short)(off >> 1) : kNoList;
+            }
             for (int c = tid; c < per_batch * kStartSlots; c += kPrologueThreads) {
                 const int bw = c / kStartSlots, slot = c % kStartSlots, b = b0 + bw;
                 if (b >= kStartBuckets) break;
-                const bool open_ended = b == kStartBuckets - 1;
-                const float y_hi = bucket_upper_edge(b) * 1.00002f;
-                const float z_edge = d_low + ((float)slot + GS_SLOT_WIDEN) * w_slot;
-                const float limit = (open_ended ? z_edge : y_hi * z_edge) * 1.00002f;
-                const float *pm = sh_pm + bw * n_t;
-                int lo = 0, hi = n_t;                       // rows [0, lo) cannot pass
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    if (pm[mid] > limit) lo = mid + 1; else hi = mid;
+                int lo = 0;                                 // rows [0, lo) cannot pass
+                if (inv_w > 0.f && slot != kStartSlots - 1) {   // (the top slot also takes every z beyond the table)
+                    const bool open_ended = b == kStartBuckets - 1;
+                    const float y_hi = bucket_upper_edge(b) * 1.00002f;
+                    const float z_edge = d_low + ((float)slot + GS_SLOT_WIDEN) * w_slot;
+                    const float limit = (open_ended ? z_edge : y_hi * z_edge) * 1.00002f;
+                    const float *pm = sh_pm + bw * n_t;
+                    int hi = n_t;
+                    while (lo < hi) {
+                        const int mid = (lo + hi) >> 1;
+                        if (pm[mid] > limit) lo = mid + 1; else hi = mid;
+                    }
                 }
-                // the top slot also takes every z beyond the table: nothing can be ruled out there
-                if (slot == kStartSlots - 1) lo = 0;
                 // (a cell that no row can pass begins at the type's last group: searches always have eight rows to test)
                 s.start_table[(tr * kStartBuckets + b) * kStartSlots + slot] = (unsigned char)min(lo >> 3, (n_padded >> 3) - 1);
+                if (!kDirect) {
+                    const int before = lo < n_t ? sh_pc[bw * n_t + lo] : sh_len[bw];    // records among rows [0, lo)
+                    s.start_list[(tr * kStartBuckets + b) * kStartSlots + slot] = (unsigned char)min(before >> 1, 255);
+                }
             }
             __syncthreads();
         }
     }
 }
 
-size_t prologue_dynamic_smem() { return (size_t)kPmFloats * sizeof(float); }   // >= 2 sort buffers
+size_t prologue_dynamic_smem() { return (size_t)kPmFloats * (sizeof(float) + sizeof(unsigned short)); }   // >= 2 sort buffers
 
 cudaError_t configure_prologue()
 {

@@ -27,18 +27,20 @@
 namespace gs {
 
 #ifndef GS_ROUTE_THREADS
-#define GS_ROUTE_THREADS 256
+#define GS_ROUTE_THREADS 1024
 #endif
 #ifndef GS_ROUTE_MIN_CTAS
-#define GS_ROUTE_MIN_CTAS 4
+#define GS_ROUTE_MIN_CTAS 1
 #endif
 constexpr int kRouteThreads = GS_ROUTE_THREADS;
 constexpr int kRouteMinCtas = GS_ROUTE_MIN_CTAS;
+constexpr int kRerouteThreads = 256;
+// (with per-row p the search holds more state: fewer threads, more registers each)
+__host__ __device__ constexpr int route_threads(bool row_p) { return row_p ? (kRouteThreads * 3) / 4 : kRouteThreads; }
 #ifndef GS_REQ_PER_THREAD
 #define GS_REQ_PER_THREAD 4
 #endif
 constexpr int kReqPerThread = GS_REQ_PER_THREAD;
-constexpr int kRouteTile = kRouteThreads * kReqPerThread;
 
 // T(r,g) of Eq. 2 with H = 0, each step rounded once.
 __device__ __forceinline__ float latency(const Row &r, float x, float y) {
@@ -80,10 +82,23 @@ struct Tables {
     const Row *rows;
     const float *row_p;       // per-row lower bound of p, in row order (only where p differs inside a group)
     const unsigned short *cand;   // candidate types by slot of D / L_out
+    const uint2 *pool;            // record lists (typed pools)
+    const unsigned short *bucket_list;
+    const unsigned char *start_list;
     int n_types;
 };
 
 constexpr unsigned kNoRow = 0xFFFFFFFFu;
+
+// Slot of the start tables for a request: z, about the largest d that can still meet the
+// deadline R with the type's least q, in units of the table.  R is raised by a hair first: a row
+// passes its test when its rounded bound is <= R, which lets the unrounded one exceed R by half
+// an ulp, and where q dominates that half ulp can be worth whole slots of d.  (ry: 1 / L_out to
+// within an ulp or two; the tables' slots are widened against what remains.)
+__device__ __forceinline__ int start_slot(float R, float q_lo, float ry, float d0, float inv_w) {
+    const float z = (__fmaf_rn(R, 4.76837158203125e-7f, R) - q_lo) * ry;
+    return __float2int_rd(fminf(fmaxf((z - d0) * inv_w, 0.f), (float)(kStartSlots - 1)));
+}
 // Lanes of a warp that must need the fallback before each runs its own search; below that the
 // warp-wide scoring of every instance is the shorter way.
 #ifndef GS_THREAD_FALLBACK_MIN
@@ -152,9 +167,8 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
         int k = 0;
         if (inv_w > 0.f) {
             // largest d that can still meet the deadline -> slot -> first row worth a look
-            const float z = (Rg - h.y) * ry;
-            const float sf = fminf(fmaxf((z - __int_as_float(geo.w)) * inv_w, 0.f), (float)(kStartSlots - 1));
-            k = 8 * tb.start_table[(t * kStartBuckets + ybucket) * kStartSlots + __float2int_rd(sf)];
+            k = 8 * tb.start_table[(t * kStartBuckets + ybucket) * kStartSlots +
+                                   start_slot(Rg, h.y, ry, __int_as_float(geo.w), inv_w)];
         }
         const int k_end = geo.x + geo.y;
         k += geo.x;                                         // padded row index, a multiple of 8
@@ -401,13 +415,15 @@ __device__ __forceinline__ unsigned first_pass_of_eight(const Tables &tb, int k,
 // but for two short loops over GPU types:
 //   1. the candidate table names the types whose least d fits D / L_out at all; the first of
 //      them (largest d first) that passes its entry test is searched;
-//   2. the start table gives the first group of eight rows worth a look; sixteen row bounds
-//      from there are tested, and the first row that passes is scored exactly as the
-//      definition says and checked against the deadline and the instance's free KV;
+//   2. the start table gives the first entry worth a look in the record list of that type and
+//      bucket of L_out (the rows that can be the first of the type to pass; see the prologue);
+//      four entries from there are tested (with per-row p, where there are no such lists:
+//      sixteen row bounds of the full list), and the first row that passes is scored exactly
+//      as the definition says and checked against the deadline and the instance's free KV;
 //   3. no later type may be able to do better: its largest d is below the pick's, or even its
 //      least q with the pick's d misses the deadline.
-// Returns false whenever this does not settle the request (nothing passed within the sixteen
-// rows, the scored row is not feasible, another type may hold a better instance, no type
+// Returns false whenever this does not settle the request (nothing passed among the entries
+// tested, there is no list, the scored row is not feasible, another type may hold a better instance, no type
 // passes its entry test); the request is then queued for the full search.  When it returns
 // true the pick is the definition's: every row ranked before it was ruled out by a true lower
 // bound of its T, and every type that could rank before it by one of its whole type.
@@ -433,13 +449,26 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
     if (t < 0) return false;
     const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, inv_w, d0
     const int ybucket = min((int)(__float_as_uint(y) >> (23 - kBucketBits)) - (127 << kBucketBits), kStartBuckets - 1);
-    const float z = (Rg - h.y) * ry;             // about the largest d that can still meet the deadline
-    const float sf = fminf(fmaxf((z - __int_as_float(geo.w)) * __int_as_float(geo.z), 0.f), (float)(kStartSlots - 1));
-    const int k = geo.x + 8 * tb.start_table[(t * kStartBuckets + ybucket) * kStartSlots + __float2int_rd(sf)];
-    const int k2 = min(k + 8, geo.x + geo.y - 8);        // (the last group of a type is tested twice)
-    const float R = kRowP ? Dm : Rg;
-    unsigned first = first_pass_of_eight<kRowP>(tb, k2, x, y, R, kNoRow);
-    first = first_pass_of_eight<kRowP>(tb, k, x, y, R, first);
+    const int cell = (t * kStartBuckets + ybucket) * kStartSlots +
+                     start_slot(Rg, h.y, ry, __int_as_float(geo.w), __int_as_float(geo.z));
+    unsigned first = kNoRow;
+    if (kRowP) {
+        // rows of a group differ in p: sixteen row bounds of the group's full list
+        const int k = geo.x + 8 * tb.start_table[cell];
+        const int k2 = min(k + 8, geo.x + geo.y - 8);    // (the last group of a type is tested twice)
+        first = first_pass_of_eight<kRowP>(tb, k2, x, y, Dm, kNoRow);
+        first = first_pass_of_eight<kRowP>(tb, k, x, y, Dm, first);
+    } else {
+        // the record list of this type and bucket of L_out: only rows that can be the first to pass
+        const unsigned list = tb.bucket_list[t * kStartBuckets + ybucket];
+        if (list == kNoList) return false;
+        const uint4 *w = reinterpret_cast<const uint4 *>(tb.pool) + (list + tb.start_list[cell]);
+        const uint4 r0 = w[0], r1 = w[1];
+        first = row_may_pass<false, false>(r1.z, r1.w, 0.f, x, y, Rg, 0.f) ? r1.z : first;
+        first = row_may_pass<false, false>(r1.x, r1.y, 0.f, x, y, Rg, 0.f) ? r1.x : first;
+        first = row_may_pass<false, false>(r0.z, r0.w, 0.f, x, y, Rg, 0.f) ? r0.z : first;
+        first = row_may_pass<false, false>(r0.x, r0.y, 0.f, x, y, Rg, 0.f) ? r0.x : first;
+    }
     if (first == kNoRow) return false;
     const int inst = (int)(first & kRowTagMask);
     const Row row = tb.rows[inst];
@@ -527,13 +556,15 @@ constexpr int kQueueCap = 64;           // per warp: at most 31 left over + 32 n
 // through full_pick, so the long, divergent search always runs with all lanes busy.  Their
 // results are stored one by one over the placeholders that the tile's vector stores left.
 template <bool kAccumulate, bool kPrefix, bool kRowP>
-__global__ void __launch_bounds__(kRouteThreads, kRowP ? (kRouteMinCtas > 3 ? 3 : kRouteMinCtas) : kRouteMinCtas)
+__global__ void __launch_bounds__(route_threads(kRowP), kRouteMinCtas)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
              const float *__restrict__ slo_ms, int64_t n, const PrefixHits hits, int n_types_alloc,
              const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
              const unsigned char *__restrict__ g_start_table,
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
-             const unsigned short *__restrict__ g_cand, const float *__restrict__ g_row_p,
+             const unsigned short *__restrict__ g_cand, const uint2 *__restrict__ g_pool,
+             const unsigned short *__restrict__ g_bucket_list, const unsigned char *__restrict__ g_start_list,
+             const float *__restrict__ g_row_p,
              int32_t *__restrict__ out_idx, float *__restrict__ out_est,
              float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
@@ -548,11 +579,30 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     if (threadIdx.x < kCandSlots) sh_cand[threadIdx.x] = g_cand[threadIdx.x];
     tb.cand = sh_cand;
     after_tables += kCandSlots * sizeof(unsigned short);
+    tb.pool = nullptr; tb.bucket_list = nullptr; tb.start_list = nullptr;
+    if (!kRowP) {                                  // record lists and their start table
+        const int n_act = table_info[3], pool_n = table_info[6];
+        uint4 *sh_start_list = reinterpret_cast<uint4 *>(after_tables);
+        for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
+            sh_start_list[k] = reinterpret_cast<const uint4 *>(g_start_list)[k];
+        after_tables += (size_t)n_types_alloc * kStartBuckets * kStartSlots;
+        uint4 *sh_bucket = reinterpret_cast<uint4 *>(after_tables);
+        for (int k = threadIdx.x; k < n_act * (kStartBuckets * (int)sizeof(unsigned short) / 16); k += blockDim.x)
+            sh_bucket[k] = reinterpret_cast<const uint4 *>(g_bucket_list)[k];
+        after_tables += (size_t)n_types_alloc * kStartBuckets * sizeof(unsigned short);
+        uint4 *sh_pool = reinterpret_cast<uint4 *>(after_tables);
+        for (int k = threadIdx.x; k < pool_n / 2; k += blockDim.x)
+            sh_pool[k] = reinterpret_cast<const uint4 *>(g_pool)[k];
+        after_tables += (size_t)kPoolEntries * sizeof(uint2);
+        tb.start_list = reinterpret_cast<const unsigned char *>(sh_start_list);
+        tb.bucket_list = reinterpret_cast<const unsigned short *>(sh_bucket);
+        tb.pool = reinterpret_cast<const uint2 *>(sh_pool);
+    }
     // the warps' queues: {L_in, L_out, bits of D, low word of the request index}, high word
     int4 *queue = reinterpret_cast<int4 *>(after_tables) + (threadIdx.x >> 5) * kQueueCap;
-    after_tables += (kRouteThreads / 32) * kQueueCap * sizeof(int4);
+    after_tables += (route_threads(kRowP) / 32) * kQueueCap * sizeof(int4);
     int *queue_hi = reinterpret_cast<int *>(after_tables) + (threadIdx.x >> 5) * kQueueCap;
-    after_tables += (kRouteThreads / 32) * kQueueCap * sizeof(int);
+    after_tables += (route_threads(kRowP) / 32) * kQueueCap * sizeof(int);
     unsigned long long *hist = reinterpret_cast<unsigned long long *>(after_tables);
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
@@ -591,8 +641,8 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
 
     constexpr int kWarpTile = 32 * kReqPerThread;
     const int64_t n_wtiles = (n + kWarpTile - 1) / kWarpTile;
-    const int64_t warp_stride = (int64_t)gridDim.x * (kRouteThreads / 32);
-    for (int64_t wt = (int64_t)blockIdx.x * (kRouteThreads / 32) + (threadIdx.x >> 5); wt < n_wtiles;
+    const int64_t warp_stride = (int64_t)gridDim.x * (route_threads(kRowP) / 32);
+    for (int64_t wt = (int64_t)blockIdx.x * (route_threads(kRowP) / 32) + (threadIdx.x >> 5); wt < n_wtiles;
          wt += warp_stride) {
         const int64_t first = wt * kWarpTile + (int64_t)lane * kReqPerThread;
         const bool full = first + kReqPerThread <= n;
@@ -722,6 +772,15 @@ constexpr size_t kRouteSmemFixed = kTablesSmemFixed + kCandSlots * sizeof(unsign
 constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
 constexpr size_t kRouteSmemRowP = (size_t)kMaxPaddedRows * sizeof(float);
+constexpr size_t kRouteSmemPerTypeLists = (size_t)kStartBuckets * kStartSlots + kStartBuckets * sizeof(unsigned short);
+constexpr size_t kRouteSmemPool = (size_t)kPoolEntries * sizeof(uint2);
+
+// Dynamic shared memory of one route CTA: the tables of n_types types (with record lists for a
+// typed pool, per-row p for coefficients given per instance), the warps' queues, the histogram.
+static size_t route_smem_bytes(int n_types, bool accumulate, bool row_p) {
+    return kRouteSmemFixed + kRouteSmemPerType * n_types + (accumulate ? kRouteSmemHist : 0) +
+           (row_p ? kRouteSmemRowP : kRouteSmemPerTypeLists * n_types + kRouteSmemPool);
+}
 
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                          const float *slo_ms, int64_t n, const PrefixHits *hits, int n_types,
@@ -729,18 +788,18 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
                          bool accumulate, bool row_p, cudaStream_t st)
 {
     if (n == 0) return cudaSuccess;
-    const size_t smem = kRouteSmemFixed + kRouteSmemPerType * n_types + (accumulate ? kRouteSmemHist : 0) +
-                        (row_p ? kRouteSmemRowP : 0);
-    int64_t blocks = (n + kRouteTile - 1) / kRouteTile;
+    const size_t smem = route_smem_bytes(n_types, accumulate, row_p);
+    const int64_t tile = (int64_t)route_threads(row_p) * kReqPerThread;
+    int64_t blocks = (n + tile - 1) / tile;
     const int64_t cap = (int64_t)ctx->n_sm * (row_p ? ctx->route_ctas_per_sm_row_p : ctx->route_ctas_per_sm[n_types]);
     if (blocks > cap) blocks = cap;
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     const PrefixHits none = {nullptr, nullptr, 0, 0};
 #define GS_LAUNCH_ROUTE(ACC, PFX, ROWP)                                                               \
-    route_kernel<ACC, PFX, ROWP><<<(unsigned)blocks, kRouteThreads, smem, st>>>(                       \
+    route_kernel<ACC, PFX, ROWP><<<(unsigned)blocks, route_threads(ROWP), smem, st>>>(                       \
         prompt_len, pred_decode_len, slo_ms, n, hits ? *hits : none, n_types, ctx->s.rows,            \
         ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, ctx->s.cand_table,  \
-        ctx->s.row_p,                                                                                 \
+        ctx->s.pool, ctx->s.bucket_list, ctx->s.start_list, ctx->s.row_p,                             \
         out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status)
     // (the prefix term and per-row p are never combined with accumulate, nor with each other)
     if (row_p) GS_LAUNCH_ROUTE(false, false, true);
@@ -759,7 +818,7 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
 // into the request that a token-ID migration would pose to the target (re-prefill prompt +
 // generated tokens, decode what is left, within the time that is left) and runs the same
 // search as the routing round, restricted to instances with d < d of the current instance.
-__global__ void __launch_bounds__(kRouteThreads, 1024 / kRouteThreads)
+__global__ void __launch_bounds__(kRerouteThreads, 4)
 reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__ cand_count, int64_t cand_capacity,
                const int32_t *__restrict__ assigned, const int32_t *__restrict__ generated,
                const int32_t *__restrict__ pred_len, const float *__restrict__ elapsed,
@@ -841,11 +900,11 @@ cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *
 {
     if (cand_capacity == 0) return cudaSuccess;
     const size_t smem = kTablesSmemFixed + kRouteSmemPerType * n_types;
-    int64_t blocks = (cand_capacity + kRouteThreads - 1) / kRouteThreads;
+    int64_t blocks = (cand_capacity + kRerouteThreads - 1) / kRerouteThreads;
     const int64_t cap = (int64_t)ctx->n_sm * ctx->reroute_ctas_per_sm[n_types];
     if (blocks > cap) blocks = cap;
     LaunchTimer timer(ctx, GS_K_REROUTE, st);
-    reroute_kernel<<<(unsigned)blocks, kRouteThreads, smem, st>>>(
+    reroute_kernel<<<(unsigned)blocks, kRerouteThreads, smem, st>>>(
         cand_idx, cand_count, cand_capacity, assigned, generated, pred_len, elapsed, slo, prompt_len, n_active,
         n_types, ctx->s.rows, ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info,
         out_inst, out_est, out_slack, out_tier, ctx->s.status);
@@ -856,33 +915,35 @@ cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *
 // on an SM for each table size (called once per context).
 cudaError_t configure_route(gs_ctx *ctx)
 {
-    const size_t max_smem = kRouteSmemFixed + kRouteSmemPerType * GS_MAX_TYPES;
     cudaError_t e = cudaFuncSetAttribute(route_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(max_smem + kRouteSmemHist));
+                                         (int)route_smem_bytes(GS_MAX_TYPES, true, false));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    e = cudaFuncSetAttribute(route_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)route_smem_bytes(GS_MAX_TYPES, false, false));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    e = cudaFuncSetAttribute(route_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)route_smem_bytes(GS_MAX_TYPES, false, false));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(route_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(max_smem + kRouteSmemRowP));
+                             (int)route_smem_bytes(GS_MAX_TYPES, false, true));
     if (e != cudaSuccess) return e;
     {
         int occ = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false, true>, kRouteThreads,
-                                                          kRouteSmemFixed + kRouteSmemPerType * kDirectGroups + kRouteSmemRowP);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false, true>, route_threads(true),
+                                                          route_smem_bytes(kDirectGroups, false, true));
         if (e != cudaSuccess) return e;
         ctx->route_ctas_per_sm_row_p = occ > 0 ? occ : 1;
     }
-    e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(kTablesSmemFixed + kRouteSmemPerType * GS_MAX_TYPES));
     if (e != cudaSuccess) return e;
     for (int t = 0; t <= GS_MAX_TYPES; ++t) {
         int occ = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false, false>, kRouteThreads,
-                                                          kRouteSmemFixed + kRouteSmemPerType * t);
+                                                          route_smem_bytes(t, false, false));
         if (e != cudaSuccess) return e;
         ctx->route_ctas_per_sm[t] = occ > 0 ? occ : 1;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, reroute_kernel, kRouteThreads,
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, reroute_kernel, kRerouteThreads,
                                                           kTablesSmemFixed + kRouteSmemPerType * t);
         if (e != cudaSuccess) return e;
         ctx->reroute_ctas_per_sm[t] = occ > 0 ? occ : 1;
