@@ -75,7 +75,7 @@ constexpr int kCandSlots = 64;
 #define GS_POOL_ENTRIES 8192
 #endif
 constexpr int kPoolEntries = GS_POOL_ENTRIES;
-constexpr int kListWindow = 4;             // entries the first attempt tests
+constexpr int kListWindow = 8;             // entries the first attempt may test (four, then four more)
 constexpr int kListMax = 510;              // longer lists are not stored (start_list counts pairs of entries in a byte)
 constexpr unsigned short kNoList = 0xFFFFu;
 

@@ -27,7 +27,7 @@
 namespace gs {
 
 #ifndef GS_ROUTE_THREADS
-#define GS_ROUTE_THREADS 1024
+#define GS_ROUTE_THREADS 768
 #endif
 #ifndef GS_ROUTE_MIN_CTAS
 #define GS_ROUTE_MIN_CTAS 1
@@ -41,6 +41,11 @@ __host__ __device__ constexpr int route_threads(bool row_p) { return row_p ? (kR
 #define GS_REQ_PER_THREAD 4
 #endif
 constexpr int kReqPerThread = GS_REQ_PER_THREAD;
+
+// Where the exact coefficients of instance g sit in the shared-memory copy of the table.  Lanes
+// often ask for instances a fixed stride apart (all of one GPU type when types are dealt round
+// robin); the low bits are mixed with the next ones so that such lanes spread over the banks.
+__device__ __forceinline__ int row_pos(int g) { return g ^ (((g >> 3) ^ (g >> 6)) & 7); }
 
 // T(r,g) of Eq. 2 with H = 0, each step rounded once.
 __device__ __forceinline__ float latency(const Row &r, float x, float y) {
@@ -125,7 +130,7 @@ template <bool kCapped>
 __device__ __forceinline__ bool score_row(const Tables &tb, int inst, float x, float y, float D, unsigned need,
                                           float d_cap, int &g_best, float &d_best, float &T_best)
 {
-    const Row row = tb.rows[inst];
+    const Row row = tb.rows[row_pos(inst)];
     const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));      // Eq. 2, H = 0
     const bool feasible = (T <= D) && (need <= (unsigned)row.kv) && (!kCapped || row.d < d_cap);
     const bool worse = row.d < d_best;
@@ -274,7 +279,7 @@ __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y
                         const float R = kRowP ? T_best + 1e-30f : Rg;
                         if (!row_may_pass<kCapped, kRowP>(qw, dw, pl[2 * c + e], x, y, R, d_cap)) continue;
                         const int inst = (int)(qw & kRowTagMask);
-                        const Row row = tb.rows[inst];
+                        const Row row = tb.rows[row_pos(inst)];
                         if (kCapped && !(row.d < d_cap)) continue;
                         if (!any_kv && !(need <= (unsigned)row.kv)) continue;
                         const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));   // Eq. 2, H = 0
@@ -312,7 +317,7 @@ __device__ __forceinline__ unsigned char *stage_tables(unsigned char *smem, int 
     TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
     uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
     unsigned char *sh_start = reinterpret_cast<unsigned char *>(sh_row_bounds + kMaxPaddedRows);
-    for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[k] = g_rows[k];
+    for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[row_pos(k)] = g_rows[k];
     for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
     for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
         reinterpret_cast<uint4 *>(sh_start)[k] = reinterpret_cast<const uint4 *>(g_start_table)[k];
@@ -344,7 +349,7 @@ __device__ __forceinline__ void exhaustive_pick(const Row *rows, int M, float xs
     unsigned long long k_room = ~0ull, k_all = ~0ull;    // min over KV-ok / all: (T, index)
     float T_feas = 0.f;
     for (int inst = lane; inst < M; inst += 32) {
-        const Row row = rows[inst];
+        const Row row = rows[row_pos(inst)];
         if (kCapped && !(row.d < d_cap)) continue;
         const float Tr = latency(row, xs, ys);
         const bool room = needs <= (unsigned)row.kv;
@@ -468,10 +473,17 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
         first = row_may_pass<false, false>(r1.x, r1.y, 0.f, x, y, Rg, 0.f) ? r1.x : first;
         first = row_may_pass<false, false>(r0.z, r0.w, 0.f, x, y, Rg, 0.f) ? r0.z : first;
         first = row_may_pass<false, false>(r0.x, r0.y, 0.f, x, y, Rg, 0.f) ? r0.x : first;
+        if (first == kNoRow) {                   // one lane in a hundred: the next four entries
+            const uint4 r2 = w[2], r3 = w[3];    // (still inside the list or its padding: see below)
+            first = row_may_pass<false, false>(r3.z, r3.w, 0.f, x, y, Rg, 0.f) ? r3.z : first;
+            first = row_may_pass<false, false>(r3.x, r3.y, 0.f, x, y, Rg, 0.f) ? r3.x : first;
+            first = row_may_pass<false, false>(r2.z, r2.w, 0.f, x, y, Rg, 0.f) ? r2.z : first;
+            first = row_may_pass<false, false>(r2.x, r2.y, 0.f, x, y, Rg, 0.f) ? r2.x : first;
+        }
     }
     if (first == kNoRow) return false;
     const int inst = (int)(first & kRowTagMask);
-    const Row row = tb.rows[inst];
+    const Row row = tb.rows[row_pos(inst)];
     const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));          // Eq. 2, H = 0
     if (!(T <= D && need <= (unsigned)row.kv)) return false;
     const float d_floor = __fmul_rn(row.d, 1.0f - 1.9073486328125e-6f);       // the bound every row with d >= the pick's carries
@@ -534,12 +546,12 @@ __device__ __forceinline__ void merge_hit(const Row *rows, int M, int g, int h, 
     if (g < 0) return;                                       // empty slot
     if (g >= M) { bad |= GS_DEV_BAD_INSTANCE; return; }      // names nothing
     if (h < 0 || h > xi) { bad |= GS_DEV_BAD_VALUE; h = h < 0 ? 0 : xi; }
-    const Row row = rows[g];
+    const Row row = rows[row_pos(g)];
     const float T = __fmaf_rn(row.d, __int2float_rn(yi), __fmaf_rn(row.p, __int2float_rn(xi - h), row.q));
     const bool room = (unsigned)xi + (unsigned)yi <= (unsigned)row.kv;
     bool take;
     if (room && T <= D) {                                    // feasible with its hit
-        const float d_cur = tier == 1u ? rows[g_cur].d : 0.f;
+        const float d_cur = tier == 1u ? rows[row_pos(g_cur)].d : 0.f;
         take = tier != 1u || row.d > d_cur || (row.d == d_cur && g < g_cur) || (g == g_cur && T < T_cur);
         if (take) tier = 1u;
     } else {                                                 // may still lead the fallback
@@ -570,6 +582,38 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
+    static_assert(kReqPerThread == 4, "four requests per lane: 128-bit column loads");
+    const int lane = threadIdx.x & 31;
+    constexpr int kWarpTile = 32 * kReqPerThread;
+    const int64_t n_wtiles = (n + kWarpTile - 1) / kWarpTile;
+    const int64_t warp_stride = (int64_t)gridDim.x * (route_threads(kRowP) / 32);
+    const int64_t wt0 = (int64_t)blockIdx.x * (route_threads(kRowP) / 32) + (threadIdx.x >> 5);
+    // the request columns of a warp's tile, four requests per lane; slots past the end read as
+    // requests that nothing can serve
+    auto load_tile = [&](int64_t tile, int4 &xv, int4 &yv, float4 &dv) {
+        const int64_t first = tile * kWarpTile + (int64_t)lane * kReqPerThread;
+        if (first + kReqPerThread <= n) {
+            xv = __ldcs(reinterpret_cast<const int4 *>(prompt_len + first));
+            yv = __ldcs(reinterpret_cast<const int4 *>(pred_decode_len + first));
+            dv = __ldcs(reinterpret_cast<const float4 *>(slo_ms + first));
+        } else {
+            int xs[kReqPerThread], ys[kReqPerThread];
+            float ds[kReqPerThread];
+#pragma unroll
+            for (int j = 0; j < kReqPerThread; ++j) {
+                const bool v = first + j < n;
+                xs[j] = v ? prompt_len[first + j] : 0;
+                ys[j] = v ? pred_decode_len[first + j] : 0;
+                ds[j] = v ? slo_ms[first + j] : -1.0f;
+            }
+            xv = make_int4(xs[0], xs[1], xs[2], xs[3]);
+            yv = make_int4(ys[0], ys[1], ys[2], ys[3]);
+            dv = make_float4(ds[0], ds[1], ds[2], ds[3]);
+        }
+    };
+    int4 xv = make_int4(0, 0, 0, 0), yv = xv;
+    float4 dv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (wt0 < n_wtiles) load_tile(wt0, xv, yv, dv);          // under way while the tables are staged
     const int M = table_info[2];
     const float cand_z0 = __int_as_float(table_info[4]), cand_inv = __int_as_float(table_info[5]);
     Tables tb;
@@ -599,29 +643,24 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         tb.pool = reinterpret_cast<const uint2 *>(sh_pool);
     }
     // the warps' queues: {L_in, L_out, bits of D, low word of the request index}, high word
-    int4 *queue = reinterpret_cast<int4 *>(after_tables) + (threadIdx.x >> 5) * kQueueCap;
+    constexpr int kWarps = route_threads(kRowP) / 32;
+    int4 *queue_all = reinterpret_cast<int4 *>(after_tables);
+    int4 *queue = queue_all + (threadIdx.x >> 5) * kQueueCap;
     after_tables += (route_threads(kRowP) / 32) * kQueueCap * sizeof(int4);
-    int *queue_hi = reinterpret_cast<int *>(after_tables) + (threadIdx.x >> 5) * kQueueCap;
+    int *queue_hi_all = reinterpret_cast<int *>(after_tables);
+    int *queue_hi = queue_hi_all + (threadIdx.x >> 5) * kQueueCap;
     after_tables += (route_threads(kRowP) / 32) * kQueueCap * sizeof(int);
     unsigned long long *hist = reinterpret_cast<unsigned long long *>(after_tables);
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
     __syncthreads();
 
-    const int lane = threadIdx.x & 31;
     const bool fast_on = tb.n_types > 0;          // unusable bounds: every request takes the full search
     unsigned bad = 0;
     int q_count = 0;                               // entries on this warp's queue (same in all lanes)
 
-    // takes up to 32 queued requests (the newest) through the full search and stores their results
-    auto drain = [&]() {
-        const int cnt = min(q_count, 32);
-        q_count -= cnt;
-        const bool active = lane < cnt;
-        int4 e = make_int4(0, 0, 0, 0);
-        int e_hi = 0;
-        if (active) { e = queue[q_count + lane]; e_hi = queue_hi[q_count + lane]; }
-        __syncwarp();                              // the slots may be written again
+    // takes one queued request per lane through the full search and stores the results
+    auto settle = [&](bool active, int4 e, int e_hi) {
         const int64_t r = ((int64_t)e_hi << 32) | (unsigned)e.w;
         const float D = __int_as_float(e.z);
         const Pick pk = full_pick<kRowP>(tb, M, lane, active, e.x, e.y, D);
@@ -638,32 +677,29 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             if (out_tier) out_tier[r] = (uint8_t)tier;
         }
     };
+    // ... the newest (up to) 32 of this warp's queue
+    auto drain = [&]() {
+        const int cnt = min(q_count, 32);
+        q_count -= cnt;
+        const bool active = lane < cnt;
+        int4 e = make_int4(0, 0, 0, 0);
+        int e_hi = 0;
+        if (active) { e = queue[q_count + lane]; e_hi = queue_hi[q_count + lane]; }
+        __syncwarp();                              // the slots may be written again
+        settle(active, e, e_hi);
+    };
 
-    constexpr int kWarpTile = 32 * kReqPerThread;
-    const int64_t n_wtiles = (n + kWarpTile - 1) / kWarpTile;
-    const int64_t warp_stride = (int64_t)gridDim.x * (route_threads(kRowP) / 32);
-    for (int64_t wt = (int64_t)blockIdx.x * (route_threads(kRowP) / 32) + (threadIdx.x >> 5); wt < n_wtiles;
-         wt += warp_stride) {
+    int64_t wt = wt0;
+    while (wt < n_wtiles) {
         const int64_t first = wt * kWarpTile + (int64_t)lane * kReqPerThread;
         const bool full = first + kReqPerThread <= n;
         int xi[kReqPerThread], yi[kReqPerThread];
         float D[kReqPerThread];
-        if (full) {
-            const int4 xv = __ldcs(reinterpret_cast<const int4 *>(prompt_len + first));
-            const int4 yv = __ldcs(reinterpret_cast<const int4 *>(pred_decode_len + first));
-            const float4 dv = __ldcs(reinterpret_cast<const float4 *>(slo_ms + first));
-            xi[0] = xv.x; xi[1] = xv.y; xi[2] = xv.z; xi[3] = xv.w;
-            yi[0] = yv.x; yi[1] = yv.y; yi[2] = yv.z; yi[3] = yv.w;
-            D[0] = dv.x; D[1] = dv.y; D[2] = dv.z; D[3] = dv.w;
-        } else {
-#pragma unroll
-            for (int j = 0; j < kReqPerThread; ++j) {
-                const bool v = first + j < n;
-                xi[j] = v ? prompt_len[first + j] : 0;
-                yi[j] = v ? pred_decode_len[first + j] : 0;
-                D[j] = v ? slo_ms[first + j] : -1.0f;
-            }
-        }
+        xi[0] = xv.x; xi[1] = xv.y; xi[2] = xv.z; xi[3] = xv.w;
+        yi[0] = yv.x; yi[1] = yv.y; yi[2] = yv.z; yi[3] = yv.w;
+        D[0] = dv.x; D[1] = dv.y; D[2] = dv.z; D[3] = dv.w;
+        wt += warp_stride;
+        if (wt < n_wtiles) load_tile(wt, xv, yv, dv);        // the next tile is on its way while this one is searched
         if ((xi[0] | xi[1] | xi[2] | xi[3] | yi[0] | yi[1] | yi[2] | yi[3]) < 0) {      // negative counts read as 0
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j) { xi[j] = max(xi[j], 0); yi[j] = max(yi[j], 0); }
@@ -753,7 +789,29 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             }
         }
     }
-    while (q_count > 0) { __syncwarp(); drain(); }
+    // What is left on the warps' queues (fewer than 32 each) is pooled: the CTA's warps take it
+    // 32 requests at a time, so the full search still runs with its lanes busy.
+    {
+        __shared__ int sh_left[kWarps];
+        const int warp = threadIdx.x >> 5;
+        if (lane == 0) sh_left[warp] = q_count;
+        __syncthreads();
+        int total = 0;
+        for (int w = 0; w < kWarps; ++w) total += sh_left[w];
+        for (int v0 = warp * 32; v0 < total; v0 += kWarps * 32) {
+            const int v = v0 + lane;
+            const bool active = v < total;
+            int owner = 0, before = 0;             // whose queue entry v is, and how many entries come before that queue
+            for (int w = 0; w < kWarps - 1; ++w) {
+                const int c = sh_left[w];
+                if (v >= before + c && owner == w) { before += c; owner = w + 1; }
+            }
+            int4 e = make_int4(0, 0, 0, 0);
+            int e_hi = 0;
+            if (active) { e = queue_all[owner * kQueueCap + v - before]; e_hi = queue_hi_all[owner * kQueueCap + v - before]; }
+            settle(active, e, e_hi);
+        }
+    }
     if (bad) atomicOr(status, bad);
 
     if (kAccumulate) {
@@ -858,7 +916,7 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
         const unsigned need = need64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (unsigned)need64;   // kv < 2^31 anyway
         const float x = __uint2float_rn(xu), y = __uint2float_rn(rem);
         const float D = __fsub_rn(slo[i], elapsed[i]);                        // time left
-        const float d_cap = tb.rows[c].d;
+        const float d_cap = tb.rows[row_pos(c)].d;
         float T = 0.f;
         const float Ds = (valid && rem > 0) ? D : -1.0f;      // see route_kernel: L_out == 0 skips the search
         int g = pick_instance<true, false>(tb, x, y, Ds, Ds + 1e-30f, need, d_cap, T);
