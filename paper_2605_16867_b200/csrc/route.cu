@@ -586,8 +586,14 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     const int lane = threadIdx.x & 31;
     constexpr int kWarpTile = 32 * kReqPerThread;
     const int64_t n_wtiles = (n + kWarpTile - 1) / kWarpTile;
-    const int64_t warp_stride = (int64_t)gridDim.x * (route_threads(kRowP) / 32);
-    const int64_t wt0 = (int64_t)blockIdx.x * (route_threads(kRowP) / 32) + (threadIdx.x >> 5);
+    // A CTA owns a contiguous run of warp tiles; its warps take them one at a time from a shared
+    // counter, so a warp that is held up by a full search simply takes fewer.
+    const int64_t tiles_per_cta = (n_wtiles + gridDim.x - 1) / gridDim.x;
+    const int64_t cta_first = (int64_t)blockIdx.x * tiles_per_cta;
+    const int64_t cta_end = min(cta_first + tiles_per_cta, n_wtiles);
+    __shared__ int sh_next_tile;
+    if (threadIdx.x == 0) sh_next_tile = route_threads(kRowP) / 32;     // the first round is dealt by warp number
+    const int64_t wt0 = cta_first + (threadIdx.x >> 5);
     // the request columns of a warp's tile, four requests per lane; slots past the end read as
     // requests that nothing can serve
     auto load_tile = [&](int64_t tile, int4 &xv, int4 &yv, float4 &dv) {
@@ -613,7 +619,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     };
     int4 xv = make_int4(0, 0, 0, 0), yv = xv;
     float4 dv = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (wt0 < n_wtiles) load_tile(wt0, xv, yv, dv);          // under way while the tables are staged
+    if (wt0 < cta_end) load_tile(wt0, xv, yv, dv);           // under way while the tables are staged
     const int M = table_info[2];
     const float cand_z0 = __int_as_float(table_info[4]), cand_inv = __int_as_float(table_info[5]);
     Tables tb;
@@ -690,7 +696,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     };
 
     int64_t wt = wt0;
-    while (wt < n_wtiles) {
+    while (wt < cta_end) {
         const int64_t first = wt * kWarpTile + (int64_t)lane * kReqPerThread;
         const bool full = first + kReqPerThread <= n;
         int xi[kReqPerThread], yi[kReqPerThread];
@@ -698,8 +704,12 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         xi[0] = xv.x; xi[1] = xv.y; xi[2] = xv.z; xi[3] = xv.w;
         yi[0] = yv.x; yi[1] = yv.y; yi[2] = yv.z; yi[3] = yv.w;
         D[0] = dv.x; D[1] = dv.y; D[2] = dv.z; D[3] = dv.w;
-        wt += warp_stride;
-        if (wt < n_wtiles) load_tile(wt, xv, yv, dv);        // the next tile is on its way while this one is searched
+        {
+            int t = 0;
+            if (lane == 0) t = atomicAdd(&sh_next_tile, 1);
+            wt = cta_first + __shfl_sync(0xFFFFFFFFu, t, 0);
+        }
+        if (wt < cta_end) load_tile(wt, xv, yv, dv);         // the next tile is on its way while this one is searched
         if ((xi[0] | xi[1] | xi[2] | xi[3] | yi[0] | yi[1] | yi[2] | yi[3]) < 0) {      // negative counts read as 0
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j) { xi[j] = max(xi[j], 0); yi[j] = max(yi[j], 0); }
