@@ -560,13 +560,14 @@ __device__ __forceinline__ void merge_hit(const Row *rows, int M, int g, int h, 
     if (take) { g_cur = g; T_cur = T; }
 }
 
-constexpr int kQueueCap = 64;           // per warp: at most 31 left over + 32 new entries
+constexpr int kQueueCap = 160;          // per warp: at most 31 left over + the 128 requests of a tile
 
 // A warp takes 128 consecutive requests at a time, four per lane (128-bit column loads and
 // stores).  Every request first tries fast_pick; the ones it does not settle are put on the
-// warp's queue in shared memory, and whenever 32 have gathered each lane takes one of them
-// through full_pick, so the long, divergent search always runs with all lanes busy.  Their
-// results are stored one by one over the placeholders that the tile's vector stores left.
+// warp's queue in shared memory (by their index: the columns are read again), and whenever 32
+// have gathered, between two tiles, each lane takes one of them through full_pick, so the
+// long, divergent search always runs with all lanes busy.  Their results are stored one by one
+// over the placeholders that the tile's vector stores left.
 template <bool kAccumulate, bool kPrefix, bool kRowP>
 __global__ void __launch_bounds__(route_threads(kRowP), kRouteMinCtas)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
@@ -650,12 +651,12 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     }
     // the warps' queues: {L_in, L_out, bits of D, low word of the request index}, high word
     constexpr int kWarps = route_threads(kRowP) / 32;
-    int4 *queue_all = reinterpret_cast<int4 *>(after_tables);
-    int4 *queue = queue_all + (threadIdx.x >> 5) * kQueueCap;
-    after_tables += (route_threads(kRowP) / 32) * kQueueCap * sizeof(int4);
-    int *queue_hi_all = reinterpret_cast<int *>(after_tables);
-    int *queue_hi = queue_hi_all + (threadIdx.x >> 5) * kQueueCap;
-    after_tables += (route_threads(kRowP) / 32) * kQueueCap * sizeof(int);
+    // (entries: the request's index less that of the CTA's first request; a CTA's run of requests
+    // is far below 2^32)
+    unsigned *queue_all = reinterpret_cast<unsigned *>(after_tables);
+    unsigned *queue = queue_all + (threadIdx.x >> 5) * kQueueCap;
+    after_tables += kWarps * kQueueCap * sizeof(unsigned);
+    const int64_t cta_first_request = cta_first * kWarpTile;
     unsigned long long *hist = reinterpret_cast<unsigned long long *>(after_tables);
     if (kAccumulate)
         for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
@@ -666,9 +667,11 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     int q_count = 0;                               // entries on this warp's queue (same in all lanes)
 
     // takes one queued request per lane through the full search and stores the results
-    auto settle = [&](bool active, int4 e, int e_hi) {
-        const int64_t r = ((int64_t)e_hi << 32) | (unsigned)e.w;
-        const float D = __int_as_float(e.z);
+    auto settle = [&](bool active, unsigned entry) {
+        const int64_t r = cta_first_request + entry;
+        int4 e = make_int4(0, 0, 0, 0);
+        float D = -1.0f;
+        if (active) { e.x = max(prompt_len[r], 0); e.y = max(pred_decode_len[r], 0); D = slo_ms[r]; }
         const Pick pk = full_pick<kRowP>(tb, M, lane, active, e.x, e.y, D);
         int g = pk.g; float T = pk.T; unsigned tier = pk.tier;
         if (kPrefix && active)
@@ -688,15 +691,16 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         const int cnt = min(q_count, 32);
         q_count -= cnt;
         const bool active = lane < cnt;
-        int4 e = make_int4(0, 0, 0, 0);
-        int e_hi = 0;
-        if (active) { e = queue[q_count + lane]; e_hi = queue_hi[q_count + lane]; }
+        unsigned entry = 0;
+        if (active) entry = queue[q_count + lane];
         __syncwarp();                              // the slots may be written again
-        settle(active, e, e_hi);
+        settle(active, entry);
     };
 
     int64_t wt = wt0;
-    while (wt < cta_end) {
+    for (;;) {
+    // (the full search is kept out of this loop: it runs between two tiles, further down)
+    while (wt < cta_end && q_count < 32) {
         const int64_t first = wt * kWarpTile + (int64_t)lane * kReqPerThread;
         const bool full = first + kReqPerThread <= n;
         int xi[kReqPerThread], yi[kReqPerThread];
@@ -779,25 +783,20 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                     if (out_tier) out_tier[first + j] = (uint8_t)1;
                 }
         }
-        // ---- queue what is open; run the full search whenever 32 requests have gathered ---------
+        // ---- queue what is open ---------------------------------------------------------------
         if (__any_sync(0xFFFFFFFFu, slow != 0)) {
-            __syncwarp();                          // the stores above come before the drain's
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j) {
                 const bool push = (slow >> j) & 1u;
                 const unsigned votes = __ballot_sync(0xFFFFFFFFu, push);
-                if (votes == 0) continue;
-                if (push) {
-                    const int pos = q_count + __popc(votes & ((1u << lane) - 1u));
-                    const int64_t r = first + j;
-                    queue[pos] = make_int4(xi[j], yi[j], __float_as_int(D[j]), (int)(unsigned)(r & 0xFFFFFFFFll));
-                    queue_hi[pos] = (int)(r >> 32);
-                }
+                if (push) queue[q_count + __popc(votes & ((1u << lane) - 1u))] = (unsigned)(first + j - cta_first_request);
                 q_count += __popc(votes);
-                __syncwarp();
-                if (q_count >= 32) drain();
             }
+            __syncwarp();                          // the entries, and the stores above, come before the full search
         }
+    }
+    if (q_count < 32) break;                       // out of tiles
+    do drain(); while (q_count >= 32);
     }
     // What is left on the warps' queues (fewer than 32 each) is pooled: the CTA's warps take it
     // 32 requests at a time, so the full search still runs with its lanes busy.
@@ -816,10 +815,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 const int c = sh_left[w];
                 if (v >= before + c && owner == w) { before += c; owner = w + 1; }
             }
-            int4 e = make_int4(0, 0, 0, 0);
-            int e_hi = 0;
-            if (active) { e = queue_all[owner * kQueueCap + v - before]; e_hi = queue_hi_all[owner * kQueueCap + v - before]; }
-            settle(active, e, e_hi);
+            settle(active, active ? queue_all[owner * kQueueCap + v - before] : 0u);
         }
     }
     if (bad) atomicOr(status, bad);
@@ -836,7 +832,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
 constexpr size_t kTablesSmemFixed = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
                                     (size_t)kMaxPaddedRows * sizeof(uint2);
 constexpr size_t kRouteSmemFixed = kTablesSmemFixed + kCandSlots * sizeof(unsigned short) +
-                                   (size_t)(kRouteThreads / 32) * kQueueCap * (sizeof(int4) + sizeof(int));
+                                   (size_t)(kRouteThreads / 32) * kQueueCap * sizeof(unsigned);
 constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
 constexpr size_t kRouteSmemRowP = (size_t)kMaxPaddedRows * sizeof(float);
