@@ -38,22 +38,33 @@ RISK_BYTES_PER_REQUEST = 20.125   # 5 input columns + 1 flag bit (candidate indi
 KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter", "reroute", "ema", "sequential")
 ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-instruction per clock
 
-# Counters of one launch on config 3 taken with ncu (profiles/route_kernel_config3.md).  They
-# describe the kernel sources with this hash; after any change to those files they no longer
-# apply and the fields that use them become null until the kernel is profiled again.
-PROFILED_ROUTE = {"sources_sha1": "8092b819b153fba0346a9f54aee8675bd35aa484", "config": 3,
-                  "dram_bytes_per_launch": 50_451_200 + 5_850_880,
-                  "warp_instructions_per_launch": 57_344_633}
+# Counters of one launch on config 3 taken with ncu (profiles/route_kernel_config3.md,
+# profiles/risk_flags_kernel_config3.md).  They describe the kernel sources with these hashes;
+# after any change to those files they no longer apply and the fields that use them become
+# null until the kernel is profiled again.
+PROFILED_ROUTE = {"sources_sha1": "44a17f186ef9d74c2bc7d4d3fc0bc9bd6ed54858", "config": 3,
+                  "dram_bytes_per_launch": 52_436_992 + 7_620_864,
+                  "warp_instructions_per_launch": 25_137_038}
+PROFILED_RISK_FLAGS = {"sources_sha1": "f8e31b7c345a323b00a561cf8750b4981dfafdb6", "config": 3,
+                       "dram_bytes_per_launch": 335_563_008 + 5_301_760}
 
 
-def kernel_sources_sha1() -> str:
+def _sources_sha1(names) -> str:
     import hashlib
     h = hashlib.sha1()
     base = os.path.join(ROOT, "paper_2605_16867_b200", "csrc")
-    for name in ("gs_internal.cuh", "prologue.cu", "route.cu"):
+    for name in names:
         with open(os.path.join(base, name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
+
+
+def kernel_sources_sha1() -> str:
+    return _sources_sha1(("gs_internal.cuh", "prologue.cu", "route.cu"))
+
+
+def risk_sources_sha1() -> str:
+    return _sources_sha1(("gs_internal.cuh", "risk.cu"))
 
 
 # --------------------------------------------------------------------------------------
@@ -449,12 +460,15 @@ def run_gpu(args):
     issue = None
     profiled = (PROFILED_ROUTE if PROFILED_ROUTE["sources_sha1"] == kernel_sources_sha1()
                 and PROFILED_ROUTE["config"] == args.config else None)
+    profiled_risk = (PROFILED_RISK_FLAGS if PROFILED_RISK_FLAGS["sources_sha1"] == risk_sources_sha1()
+                     and PROFILED_RISK_FLAGS["config"] == args.config else None)
     if dominant in alg_bytes:
         ms, n = kernel_ms[dominant]
         achieved = alg_bytes[dominant] / (ms / n * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak,
-                    "traffic": profiled["dram_bytes_per_launch"] if profiled and dominant == "route" else None,
+                    "traffic": (profiled["dram_bytes_per_launch"] if profiled and dominant == "route" else
+                                profiled_risk["dram_bytes_per_launch"] if profiled_risk and dominant == "risk_flags" else None),
                     "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": alg_bytes[dominant]}
     if profiled and "route" in kernel_ms:
         ms, n = kernel_ms["route"]
@@ -468,6 +482,10 @@ def run_gpu(args):
             gbs = alg_bytes[name] / (per_kernel[name]["avg_us"] * 1e-6) / 1e9
             per_kernel[name]["algorithmic_GBps"] = gbs
             per_kernel[name]["frac_of_hbm_peak"] = gbs / peak
+    if profiled and "route" in per_kernel:
+        per_kernel["route"]["dram_bytes_per_launch"] = profiled["dram_bytes_per_launch"]
+    if profiled_risk and "risk_flags" in per_kernel:
+        per_kernel["risk_flags"]["dram_bytes_per_launch"] = profiled_risk["dram_bytes_per_launch"]
     route_ms = sum(kernel_ms[k][0] for k in ("prologue", "route") if k in kernel_ms) / args.steps   # serial pass
     risk_ms = sum(kernel_ms[k][0] for k in ("risk_flags", "risk_scatter") if k in kernel_ms) / args.steps
     step_bytes = ROUTE_BYTES_PER_REQUEST * N + RISK_BYTES_PER_REQUEST * A + 4 * flagged
@@ -517,7 +535,7 @@ def main():
     ap.add_argument("--print-kernel-hash", action="store_true", help="print the hash PROFILED_ROUTE refers to")
     args = ap.parse_args()
     if args.print_kernel_hash:
-        print(kernel_sources_sha1())
+        print(kernel_sources_sha1(), risk_sources_sha1())
         return
     if args.impl == "reference":
         run_reference(args)
