@@ -379,6 +379,50 @@ def test_pruned_search_is_exact_on_adversarial_pools(gs, case):
     assert gs.device_status() == 0
 
 
+RECORD_LIST_CASES = [
+    dict(M=1024, Tn=8),                    # the benchmark's shape: every type gets a share of the pool
+    dict(M=1024, Tn=1),                    # one type of 1,024 rows: long lists, the pool runs out at some bucket
+    dict(M=1024, Tn=2, scarce_kv=True),    # picks that lack KV room leave the lists' promise
+    dict(M=600, Tn=3, zero_queue=True),    # equal q: a type's records collapse to its first row
+    dict(M=96, Tn=16),                     # six rows a type: lists shorter than the window
+]
+
+
+@pytest.mark.parametrize("case", range(len(RECORD_LIST_CASES)))
+def test_record_lists_at_bucket_edges_and_row_deadlines(gs, case):
+    """The first attempt of the route kernel looks at a few entries of a per-type, per-bucket
+    list of rows; what it cannot prove goes to the full search.  L_out on, just below and just
+    above every bucket edge (powers of two and 1.5 times them, up to beyond the last bucket),
+    deadlines exactly on, one ulp below and one ulp above the estimate of every instance of a
+    request's row, so that each list entry is the pick of some request and each of its
+    neighbours is refused by one ulp."""
+    rng = np.random.default_rng(7000 + case)
+    types, inst = _random_pool(rng, **RECORD_LIST_CASES[case])
+    pool = pool_of(gs, types, inst)
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    M = inst.n_instances
+    edges = []
+    for e in range(0, 19):
+        for base in (1 << e, 3 << e >> 1):
+            edges += [base - 1, base, base + 1]
+    y_vals = np.array(sorted({v for v in edges if v >= 1}), np.int32)
+    reps = -(-3 * M // len(y_vals))                     # every instance gets on/below/above deadlines
+    y = np.tile(y_vals, reps * 8)[: 24 * M]
+    n = y.size
+    x = np.clip(np.rint(np.exp(rng.normal(6.0, 1.5, n))), 0, 1 << 18).astype(np.int32)
+    T = _canonical_T(t32, x, y)
+    g = np.arange(n) % M
+    D = T[np.arange(n), g].copy()
+    kind = (np.arange(n) // M) % 3
+    D = np.where(kind == 1, np.nextafter(D, np.float32(-np.inf)), D)
+    D = np.where(kind == 2, np.nextafter(D, np.float32(np.inf)), D)
+    req = W.RequestBatch(x, y.astype(np.int32), D.astype(np.float32))
+    got = gpu_route(gs, pool, req, 0.5)
+    ref = oracle.route(t32, *req.columns(), threads=4)
+    assert_route_matches_f32_oracle(got, ref)
+    assert gs.device_status() == 0
+
+
 @pytest.mark.parametrize("share", [1.0, 0.3, 0.01])
 @pytest.mark.parametrize("scarce_kv", [False, True])
 def test_fallback_heavy_and_sparse_batches(gs, share, scarce_kv):
