@@ -111,9 +111,7 @@ struct gs_ctx {
     int max_instances;
     int max_types;
     int n_sm;
-    int route_ctas_per_sm_row_p;
-    int route_ctas_per_sm[GS_MAX_TYPES + 1];   // by number of types (sets the shared-memory size)
-    int reroute_ctas_per_sm[GS_MAX_TYPES + 1];
+    int reroute_ctas_per_sm[GS_MAX_TYPES + 1];   // by number of types (sets the shared-memory size)
     gs::Scratch s;
     size_t max_chunks, max_groups;   // capacity of the risk scan's count arrays
     unsigned scan_epoch;             // its parity selects the group-total buffer of the next scan

@@ -36,11 +36,13 @@ constexpr int kRouteThreads = GS_ROUTE_THREADS;
 constexpr int kRouteMinCtas = GS_ROUTE_MIN_CTAS;
 constexpr int kRerouteThreads = 256;
 // (with per-row p the search holds more state: fewer threads, more registers each)
-__host__ __device__ constexpr int route_threads(bool row_p) { return row_p ? (kRouteThreads * 3) / 4 : kRouteThreads; }
-#ifndef GS_REQ_PER_THREAD
-#define GS_REQ_PER_THREAD 4
-#endif
-constexpr int kReqPerThread = GS_REQ_PER_THREAD;
+// Requests per lane: four (128-bit column loads) for large batches; one for small ones, where
+// shorter tiles spread over more warps count for more than wide loads (fewer registers: a
+// third more threads).
+__host__ __device__ constexpr int route_threads(bool row_p, int req = 4) {
+    return (row_p ? (kRouteThreads * 3) / 4 : kRouteThreads) * (req == 1 ? 4 : 3) / 3;
+}
+constexpr int64_t kSmallBatch = 1 << 21;        // below this many requests: one per lane
 
 // Where the exact coefficients of instance g sit in the shared-memory copy of the table.  Lanes
 // often ask for instances a fixed stride apart (all of one GPU type when types are dealt round
@@ -568,8 +570,8 @@ constexpr int kQueueCap = 160;          // per warp: at most 31 left over + the 
 // have gathered, between two tiles, each lane takes one of them through full_pick, so the
 // long, divergent search always runs with all lanes busy.  Their results are stored one by one
 // over the placeholders that the tile's vector stores left.
-template <bool kAccumulate, bool kPrefix, bool kRowP>
-__global__ void __launch_bounds__(route_threads(kRowP), kRouteMinCtas)
+template <bool kAccumulate, bool kPrefix, bool kRowP, int kReqPerThread>
+__global__ void __launch_bounds__(route_threads(kRowP, kReqPerThread), kRouteMinCtas)
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
              const float *__restrict__ slo_ms, int64_t n, const PrefixHits hits, int n_types_alloc,
              const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
@@ -583,7 +585,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    static_assert(kReqPerThread == 4, "four requests per lane: 128-bit column loads");
+    static_assert(kReqPerThread == 4 || kReqPerThread == 1, "four requests per lane (128-bit column loads) or one");
     const int lane = threadIdx.x & 31;
     constexpr int kWarpTile = 32 * kReqPerThread;
     const int64_t n_wtiles = (n + kWarpTile - 1) / kWarpTile;
@@ -593,34 +595,35 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     const int64_t cta_first = (int64_t)blockIdx.x * tiles_per_cta;
     const int64_t cta_end = min(cta_first + tiles_per_cta, n_wtiles);
     __shared__ int sh_next_tile;
-    if (threadIdx.x == 0) sh_next_tile = route_threads(kRowP) / 32;     // the first round is dealt by warp number
+    if (threadIdx.x == 0) sh_next_tile = route_threads(kRowP, kReqPerThread) / 32;     // the first round is dealt by warp number
     const int64_t wt0 = cta_first + (threadIdx.x >> 5);
     // the request columns of a warp's tile, four requests per lane; slots past the end read as
     // requests that nothing can serve
-    auto load_tile = [&](int64_t tile, int4 &xv, int4 &yv, float4 &dv) {
+    auto load_tile = [&](int64_t tile, int (&xs)[kReqPerThread], int (&ys)[kReqPerThread], float (&ds)[kReqPerThread]) {
         const int64_t first = tile * kWarpTile + (int64_t)lane * kReqPerThread;
-        if (first + kReqPerThread <= n) {
-            xv = __ldcs(reinterpret_cast<const int4 *>(prompt_len + first));
-            yv = __ldcs(reinterpret_cast<const int4 *>(pred_decode_len + first));
-            dv = __ldcs(reinterpret_cast<const float4 *>(slo_ms + first));
+        if (kReqPerThread == 4 && first + kReqPerThread <= n) {
+            const int4 xv = __ldcs(reinterpret_cast<const int4 *>(prompt_len + first));
+            const int4 yv = __ldcs(reinterpret_cast<const int4 *>(pred_decode_len + first));
+            const float4 dv = __ldcs(reinterpret_cast<const float4 *>(slo_ms + first));
+            const int xa[4] = {xv.x, xv.y, xv.z, xv.w}, ya[4] = {yv.x, yv.y, yv.z, yv.w};
+            const float da[4] = {dv.x, dv.y, dv.z, dv.w};
+#pragma unroll
+            for (int j = 0; j < kReqPerThread; ++j) { xs[j] = xa[j]; ys[j] = ya[j]; ds[j] = da[j]; }
         } else {
-            int xs[kReqPerThread], ys[kReqPerThread];
-            float ds[kReqPerThread];
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j) {
                 const bool v = first + j < n;
-                xs[j] = v ? prompt_len[first + j] : 0;
-                ys[j] = v ? pred_decode_len[first + j] : 0;
-                ds[j] = v ? slo_ms[first + j] : -1.0f;
+                xs[j] = v ? __ldcs(prompt_len + first + j) : 0;
+                ys[j] = v ? __ldcs(pred_decode_len + first + j) : 0;
+                ds[j] = v ? __ldcs(slo_ms + first + j) : -1.0f;
             }
-            xv = make_int4(xs[0], xs[1], xs[2], xs[3]);
-            yv = make_int4(ys[0], ys[1], ys[2], ys[3]);
-            dv = make_float4(ds[0], ds[1], ds[2], ds[3]);
         }
     };
-    int4 xv = make_int4(0, 0, 0, 0), yv = xv;
-    float4 dv = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (wt0 < cta_end) load_tile(wt0, xv, yv, dv);           // under way while the tables are staged
+    int nx[kReqPerThread], ny[kReqPerThread];      // the tile on its way
+    float nd[kReqPerThread];
+#pragma unroll
+    for (int j = 0; j < kReqPerThread; ++j) { nx[j] = 0; ny[j] = 0; nd[j] = -1.0f; }
+    if (wt0 < cta_end) load_tile(wt0, nx, ny, nd);           // under way while the tables are staged
     const int M = table_info[2];
     const float cand_z0 = __int_as_float(table_info[4]), cand_inv = __int_as_float(table_info[5]);
     Tables tb;
@@ -650,7 +653,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         tb.pool = reinterpret_cast<const uint2 *>(sh_pool);
     }
     // the warps' queues: {L_in, L_out, bits of D, low word of the request index}, high word
-    constexpr int kWarps = route_threads(kRowP) / 32;
+    constexpr int kWarps = route_threads(kRowP, kReqPerThread) / 32;
     // (entries: the request's index less that of the CTA's first request; a CTA's run of requests
     // is far below 2^32)
     unsigned *queue_all = reinterpret_cast<unsigned *>(after_tables);
@@ -702,19 +705,21 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     // (the full search is kept out of this loop: it runs between two tiles, further down)
     while (wt < cta_end && q_count < 32) {
         const int64_t first = wt * kWarpTile + (int64_t)lane * kReqPerThread;
-        const bool full = first + kReqPerThread <= n;
+        const bool full = kReqPerThread == 4 && first + kReqPerThread <= n;
         int xi[kReqPerThread], yi[kReqPerThread];
         float D[kReqPerThread];
-        xi[0] = xv.x; xi[1] = xv.y; xi[2] = xv.z; xi[3] = xv.w;
-        yi[0] = yv.x; yi[1] = yv.y; yi[2] = yv.z; yi[3] = yv.w;
-        D[0] = dv.x; D[1] = dv.y; D[2] = dv.z; D[3] = dv.w;
+#pragma unroll
+        for (int j = 0; j < kReqPerThread; ++j) { xi[j] = nx[j]; yi[j] = ny[j]; D[j] = nd[j]; }
         {
             int t = 0;
             if (lane == 0) t = atomicAdd(&sh_next_tile, 1);
             wt = cta_first + __shfl_sync(0xFFFFFFFFu, t, 0);
         }
-        if (wt < cta_end) load_tile(wt, xv, yv, dv);         // the next tile is on its way while this one is searched
-        if ((xi[0] | xi[1] | xi[2] | xi[3] | yi[0] | yi[1] | yi[2] | yi[3]) < 0) {      // negative counts read as 0
+        if (wt < cta_end) load_tile(wt, nx, ny, nd);         // the next tile is on its way while this one is searched
+        int any_sign = 0;
+#pragma unroll
+        for (int j = 0; j < kReqPerThread; ++j) any_sign |= xi[j] | yi[j];
+        if (any_sign < 0) {                                  // negative counts read as 0
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j) { xi[j] = max(xi[j], 0); yi[j] = max(yi[j], 0); }
             bad |= GS_DEV_BAD_VALUE;
@@ -743,8 +748,9 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 if (full) {
                     const int4 gv = __ldcs(reinterpret_cast<const int4 *>(col_g + first));
                     const int4 hv = __ldcs(reinterpret_cast<const int4 *>(col_h + first));
-                    hg[0] = gv.x; hg[1] = gv.y; hg[2] = gv.z; hg[3] = gv.w;
-                    hh[0] = hv.x; hh[1] = hv.y; hh[2] = hv.z; hh[3] = hv.w;
+                    const int ga[4] = {gv.x, gv.y, gv.z, gv.w}, ha[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+                    for (int j = 0; j < kReqPerThread; ++j) { hg[j] = ga[j]; hh[j] = ha[j]; }
                 } else {
 #pragma unroll
                     for (int j = 0; j < kReqPerThread; ++j) {
@@ -767,19 +773,20 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
                 accumulate_choice(hist, M, g_out[j], (unsigned)xi[j], (unsigned)xi[j] + (unsigned)yi[j]);
         }
         if (full) {
-            __stcs(reinterpret_cast<int4 *>(out_idx + first), make_int4(g_out[0], g_out[1], g_out[2], g_out[3]));
-            __stcs(reinterpret_cast<float4 *>(out_est + first), make_float4(T_out[0], T_out[1], T_out[2], T_out[3]));
+            constexpr int k1 = kReqPerThread > 1 ? 1 : 0, k2 = kReqPerThread > 2 ? 2 : 0, k3 = kReqPerThread > 3 ? 3 : 0;
+            __stcs(reinterpret_cast<int4 *>(out_idx + first), make_int4(g_out[0], g_out[k1], g_out[k2], g_out[k3]));
+            __stcs(reinterpret_cast<float4 *>(out_est + first), make_float4(T_out[0], T_out[k1], T_out[k2], T_out[k3]));
             __stcs(reinterpret_cast<float4 *>(out_slack + first),
-                   make_float4(__fsub_rn(D[0], T_out[0]), __fsub_rn(D[1], T_out[1]),
-                               __fsub_rn(D[2], T_out[2]), __fsub_rn(D[3], T_out[3])));
+                   make_float4(__fsub_rn(D[0], T_out[0]), __fsub_rn(D[k1], T_out[k1]),
+                               __fsub_rn(D[k2], T_out[k2]), __fsub_rn(D[k3], T_out[k3])));
             if (out_tier) *reinterpret_cast<unsigned *>(out_tier + first) = tiers;
         } else {
 #pragma unroll
             for (int j = 0; j < kReqPerThread; ++j)
                 if (first + j < n) {
-                    out_idx[first + j] = g_out[j];
-                    out_est[first + j] = T_out[j];
-                    out_slack[first + j] = __fsub_rn(D[j], T_out[j]);
+                    __stcs(out_idx + first + j, g_out[j]);
+                    __stcs(out_est + first + j, T_out[j]);
+                    __stcs(out_slack + first + j, __fsub_rn(D[j], T_out[j]));
                     if (out_tier) out_tier[first + j] = (uint8_t)1;
                 }
         }
@@ -832,7 +839,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
 constexpr size_t kTablesSmemFixed = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
                                     (size_t)kMaxPaddedRows * sizeof(uint2);
 constexpr size_t kRouteSmemFixed = kTablesSmemFixed + kCandSlots * sizeof(unsigned short) +
-                                   (size_t)(kRouteThreads / 32) * kQueueCap * sizeof(unsigned);
+                                   (size_t)(route_threads(false, 1) / 32) * kQueueCap * sizeof(unsigned);
 constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
 constexpr size_t kRouteSmemRowP = (size_t)kMaxPaddedRows * sizeof(float);
@@ -853,14 +860,16 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
 {
     if (n == 0) return cudaSuccess;
     const size_t smem = route_smem_bytes(n_types, accumulate, row_p);
-    const int64_t tile = (int64_t)route_threads(row_p) * kReqPerThread;
+    const int req = n < kSmallBatch ? 1 : 4;
+    const int64_t tile = (int64_t)route_threads(row_p, req) * req;
     int64_t blocks = (n + tile - 1) / tile;
-    const int64_t cap = (int64_t)ctx->n_sm * (row_p ? ctx->route_ctas_per_sm_row_p : ctx->route_ctas_per_sm[n_types]);
-    if (blocks > cap) blocks = cap;
+    if (blocks > ctx->n_sm) blocks = ctx->n_sm;   // one CTA per SM: its tables fill most of the shared memory
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     const PrefixHits none = {nullptr, nullptr, 0, 0};
 #define GS_LAUNCH_ROUTE(ACC, PFX, ROWP)                                                               \
-    route_kernel<ACC, PFX, ROWP><<<(unsigned)blocks, route_threads(ROWP), smem, st>>>(                       \
+    if (req == 1) GS_LAUNCH_ROUTE_R(ACC, PFX, ROWP, 1); else GS_LAUNCH_ROUTE_R(ACC, PFX, ROWP, 4)
+#define GS_LAUNCH_ROUTE_R(ACC, PFX, ROWP, REQ)                                                        \
+    route_kernel<ACC, PFX, ROWP, REQ><<<(unsigned)blocks, route_threads(ROWP, REQ), smem, st>>>(      \
         prompt_len, pred_decode_len, slo_ms, n, hits ? *hits : none, n_types, ctx->s.rows,            \
         ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, ctx->s.cand_table,  \
         ctx->s.pool, ctx->s.bucket_list, ctx->s.start_list, ctx->s.row_p,                             \
@@ -871,6 +880,7 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     else if (accumulate) GS_LAUNCH_ROUTE(true, false, false);
     else GS_LAUNCH_ROUTE(false, false, false);
 #undef GS_LAUNCH_ROUTE
+#undef GS_LAUNCH_ROUTE_R
     return cudaGetLastError();
 }
 
@@ -977,36 +987,33 @@ cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *
 
 // Raises the dynamic shared-memory limit of the route kernels and looks up how many CTAs fit
 // on an SM for each table size (called once per context).
-cudaError_t configure_route(gs_ctx *ctx)
+template <int kReq>
+static cudaError_t configure_route_kernels()
 {
-    cudaError_t e = cudaFuncSetAttribute(route_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(route_kernel<true, false, false, kReq>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)route_smem_bytes(GS_MAX_TYPES, true, false));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(route_kernel<false, false, false, kReq>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)route_smem_bytes(GS_MAX_TYPES, false, false));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(route_kernel<false, true, false, kReq>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)route_smem_bytes(GS_MAX_TYPES, false, false));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)route_smem_bytes(GS_MAX_TYPES, false, true));
+    return cudaFuncSetAttribute(route_kernel<false, false, true, kReq>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)route_smem_bytes(GS_MAX_TYPES, false, true));
+}
+
+cudaError_t configure_route(gs_ctx *ctx)
+{
+    cudaError_t e = configure_route_kernels<1>();
     if (e != cudaSuccess) return e;
-    {
-        int occ = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false, true>, route_threads(true),
-                                                          route_smem_bytes(kDirectGroups, false, true));
-        if (e != cudaSuccess) return e;
-        ctx->route_ctas_per_sm_row_p = occ > 0 ? occ : 1;
-    }
+    e = configure_route_kernels<4>();
+    if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kTablesSmemFixed + kRouteSmemPerType * GS_MAX_TYPES));
     if (e != cudaSuccess) return e;
     for (int t = 0; t <= GS_MAX_TYPES; ++t) {
         int occ = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_kernel<false, false, false>, kRouteThreads,
-                                                          route_smem_bytes(t, false, false));
-        if (e != cudaSuccess) return e;
-        ctx->route_ctas_per_sm[t] = occ > 0 ? occ : 1;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, reroute_kernel, kRerouteThreads,
                                                           kTablesSmemFixed + kRouteSmemPerType * t);
         if (e != cudaSuccess) return e;
