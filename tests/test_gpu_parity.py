@@ -423,6 +423,46 @@ def test_record_lists_at_bucket_edges_and_row_deadlines(gs, case):
     assert gs.device_status() == 0
 
 
+@pytest.mark.parametrize("variant", ["plain", "accumulate", "prefix", "direct"])
+def test_large_batches_take_the_wide_kernel(gs, variant):
+    """From 2,097,152 requests on, the route kernel reads four requests per lane with 128-bit
+    loads (below: one per lane).  Every variant of it runs here on a batch just over that size,
+    ragged at the end, with a tenth of the deadlines out of reach so that the queue and the
+    fallback see traffic too."""
+    n = (1 << 21) + 37
+    wl = W.make_workload(3, n_requests=n, n_active=1024)
+    req = wl.requests
+    rng = np.random.default_rng(99)
+    hopeless = rng.random(n) < 0.1
+    req = W.RequestBatch(req.prompt_len, req.pred_decode_len,
+                         np.where(hopeless, req.slo_ms * np.float32(0.3), req.slo_ms).astype(np.float32))
+    t32 = oracle.instance_table(wl.types, wl.instances, wl.ema_alpha, "f32")
+    if variant == "direct":
+        bb = W.make_blackbox_table(wl.types, wl.instances, seed=3)
+        t32 = oracle.direct_table(*bb.columns(), "f32")
+        got = gpu_route_direct(gs, bb, req)
+        ref = oracle.route(t32, *req.columns(), threads=8)
+    elif variant == "prefix":
+        pool = pool_of(gs, wl.types, wl.instances)
+        pi, ph = W.make_prefix_hits(req, t32.n_instances, seed=3, n_slots=2)
+        got = gpu_route_prefix(gs, pool, req, wl.ema_alpha, pi, ph)
+        ref = oracle.route_prefix(t32, *req.columns(), pi, ph, threads=8)
+    else:
+        pool = pool_of(gs, wl.types, wl.instances)
+        got = gpu_route(gs, pool, req, wl.ema_alpha, accumulate=variant == "accumulate")
+        ref = oracle.route(t32, *req.columns(), threads=8)
+        if variant == "accumulate":
+            gs.advance_state(pool)
+            state = wl.instances.copy()
+            oracle.advance(state, t32, ref.instance_idx, req.prompt_len, req.pred_decode_len)
+            np.testing.assert_array_equal(pool.queued_prefill_tokens.cpu().numpy(), state.queued_prefill_tokens)
+            np.testing.assert_array_equal(pool.decode_batch.cpu().numpy(), state.decode_batch)
+            np.testing.assert_array_equal(pool.free_kv_tokens.cpu().numpy(), state.free_kv_tokens)
+    assert_route_matches_f32_oracle(got, ref)
+    assert (ref.tier >= 2).mean() > 0.05
+    assert gs.device_status() == 0
+
+
 @pytest.mark.parametrize("share", [1.0, 0.3, 0.01])
 @pytest.mark.parametrize("scarce_kv", [False, True])
 def test_fallback_heavy_and_sparse_batches(gs, share, scarce_kv):
