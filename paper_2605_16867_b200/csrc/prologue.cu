@@ -24,8 +24,9 @@
 // For all requests with y <= y_hi and z < z_edge the right side is at most
 // max(z_edge - d_lo, 0) * y_hi, so a row whose q_lo - q0 exceeds that is out for all of them,
 // and the search may begin at the first row that is not out.  The table is indexed by the
-// bucket of y (upper edge y_hi) and the slot of z (upper edge z_edge, widened by two slots
-// against the rounding of the kernel's own slot computation).
+// bucket of y (upper edge y_hi) and the slot of z (upper edge z_edge, widened by a sixteenth of
+// a slot against the rounding of the kernel's own slot computation, which stays below 0.03
+// slots because a table is only built where the type's range of d exceeds d / 1024).
 #include "gs_internal.cuh"
 
 namespace gs {
@@ -262,8 +263,13 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             n_t = sh_cnt[my_type];
             p_group = sh_tp[my_type];
             // ---- 3. collect this type's rows and sort them by (d descending, index ascending) ---
-            if (has && sh_t[tid] == my_type)
-                sh_key[atomicAdd(&sh_fill, 1)] = ((unsigned long long)(~orderable(sh_d[tid])) << 16) | (unsigned)tid;
+            // (one shared-memory atomic per warp; the order inside the list does not matter yet)
+            const bool mine = has && sh_t[tid] == my_type;
+            const unsigned votes = __ballot_sync(0xFFFFFFFFu, mine);
+            int at = 0;
+            if (lane == 0 && votes) at = atomicAdd(&sh_fill, __popc(votes));
+            at = __shfl_sync(0xFFFFFFFFu, at, 0) + __popc(votes & ((1u << lane) - 1u));
+            if (mine) sh_key[at] = ((unsigned long long)(~orderable(sh_d[tid])) << 16) | (unsigned)tid;
         }
         __syncthreads();
         if (my_type >= 0) {                    // (uniform over the CTA)
@@ -407,17 +413,25 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 if (lane == 0) sh_len[warp] = n_rec;
             }
             __syncthreads();
-            if (tid == 0) {                                 // room in the pool, in bucket order
-                int used = sh_pool_used;
-                for (int wb = 0; wb < per_batch && b0 + wb < kStartBuckets; ++wb) {
-                    const int len = sh_len[wb];
-                    const int need = (len + kListWindow + 1) & ~1;      // padded: a window never leaves its list
-                    const bool fits = !kDirect && b0 + wb != kStartBuckets - 1 && len <= kListMax &&
-                                      used + need <= pool_share;
-                    sh_off[wb] = fits ? pool_base + used : -1;
-                    if (fits) used += need;
+            if (warp == 0) {                                // room in the pool, in bucket order (lane = bucket of the batch)
+                const bool listed = !kDirect && lane < per_batch && b0 + lane < kStartBuckets - 1 &&
+                                    sh_len[lane < per_batch ? lane : 0] <= kListMax;
+                // padded: a window never leaves its list
+                const int need = listed ? (sh_len[lane] + kListWindow + 1) & ~1 : 0;
+                int upto = need;                            // entries wanted by this bucket and the ones before it
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int v = __shfl_up_sync(0xFFFFFFFFu, upto, off);
+                    if (lane >= off) upto += v;
                 }
-                sh_pool_used = used;
+                const int used = sh_pool_used;
+                const bool fits = listed && used + upto <= pool_share;     // (lists only get longer with the bucket)
+                if (lane < per_batch) sh_off[lane] = fits ? pool_base + used + upto - need : -1;
+                const unsigned got = __ballot_sync(0xFFFFFFFFu, fits);
+                const int last = got ? 31 - __clz(got) : -1;
+                const int used_now = last >= 0 ? __shfl_sync(0xFFFFFFFFu, upto, last) : 0;
+                __syncwarp();
+                if (lane == 0) sh_pool_used = used + used_now;
             }
             __syncthreads();
             if (my_bucket && !kDirect) {
