@@ -159,6 +159,7 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
     struct { void **p; size_t bytes; } allocs[] = {
         {(void **)&s.rows, Mx * sizeof(gs::Row)},
         {(void **)&s.row_bounds, gs::kMaxPaddedRows * sizeof(uint2)},
+        {(void **)&s.group_bounds, gs::kMaxPaddedRows / 8 * sizeof(float2)},
         {(void **)&s.row_p, gs::kMaxPaddedRows * sizeof(float)},
         {(void **)&s.start_table, (size_t)GS_MAX_TYPES * gs::kStartBuckets * gs::kStartSlots},
         {(void **)&s.headers, GS_MAX_TYPES * sizeof(gs::TypeHeader)},
@@ -191,7 +192,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.group_totals, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.group_totals, s.status, ctx->stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);

@@ -86,6 +86,7 @@ constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 struct Scratch {
     Row *rows;                // [max_instances] exact coefficients, caller order
     uint2 *row_bounds;        // [kMaxPaddedRows]
+    float2 *group_bounds;     // [kMaxPaddedRows / 8] per eight rows: {least q word as a float, d_lo of the last row}; +inf, 0 = padding only
     float *row_p;             // [kMaxPaddedRows] lower bound of each row's p, in row order (unswizzled)
     unsigned char *start_table;   // [GS_MAX_TYPES * kStartBuckets * kStartSlots]
     TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)

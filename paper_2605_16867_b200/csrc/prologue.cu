@@ -335,6 +335,14 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     if (lane == 0) atomicMin(&sh_qmin, my_qmin);
     __syncthreads();
 
+    // bounds over every eight rows (the fallback's search skips a group whole with them)
+    for (int g = tid; g < n_padded / 8; g += kPrologueThreads) {
+        float q_least = __int_as_float(0x7F800000);         // +inf: a group of padding only
+        float d_last = 0.f;
+        for (int k = 8 * g; k < 8 * g + 8 && k < n_t; ++k) { q_least = fminf(q_least, sh_rq[k]); d_last = sh_rd[k]; }
+        s.group_bounds[(base >> 3) + g] = make_float2(q_least, d_last);
+    }
+
     // ---- 5. header ----------------------------------------------------------------------------
     const float q0 = __uint_as_float(sh_qmin);
     const float d_hi = sh_rd[0], d_low = sh_rd[n_t - 1];

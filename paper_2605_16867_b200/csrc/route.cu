@@ -85,6 +85,7 @@ __device__ __forceinline__ void accumulate_choice(unsigned long long *hist, int 
 struct Tables {
     const TypeHeader *headers;
     const uint2 *row_bounds;
+    const float2 *group_bounds;   // per eight rows: {least q word, d_lo of the last row}
     const unsigned char *start_table;
     const Row *rows;
     const float *row_p;       // per-row lower bound of p, in row order (only where p differs inside a group)
@@ -251,22 +252,19 @@ __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y
             const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, ..
 #pragma unroll 1
             for (int k = geo.x + geo.y - 8; k >= geo.x; k -= 8) {
+                // the group's rows have d_lo >= gb.y (its last row's) and q words >= gb.x: if even
+                // the type's least q with that d misses the best, so does everything from here up;
+                // if the group's own least q with it does, the group holds nothing better
+                const float2 gb = tb.group_bounds[k >> 3];
+                if (!(__fmaf_rn(gb.y, y, h.y) <= Rg)) break;
+                if (kRowP ? !(__fmaf_rn(gb.y, y, __fmaf_rn(h.x, x, gb.x)) <= T_best + 1e-30f)
+                          : !(__fmaf_rn(gb.y, y, gb.x) <= Rg)) continue;
                 const char *grp = reinterpret_cast<const char *>(tb.row_bounds + k);
                 const int sw = (k >> 4) & 3;                // see row_slot()
                 uint4 r[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) r[c] = *reinterpret_cast<const uint4 *>(grp + ((c ^ sw) << 4));
-                // rows k .. k+7 in order: (r[0].x,y) (r[0].z,w) (r[1].x,y) ...; larger d first.
-                // the last real row of the group has the group's smallest d: if even q0 with that
-                // d misses the best, so does everything from here up
-                float d_min = 0.f;                          // a group of padding only: nothing to conclude
-                bool have = false;
-#pragma unroll
-                for (int c = 3; c >= 0; --c) {              // padding (NaN q) only follows a type's last row
-                    if (!have && __uint_as_float(r[c].z) == __uint_as_float(r[c].z)) { d_min = __uint_as_float(r[c].w); have = true; }
-                    if (!have && __uint_as_float(r[c].x) == __uint_as_float(r[c].x)) { d_min = __uint_as_float(r[c].y); have = true; }
-                }
-                if (!(__fmaf_rn(d_min, y, h.y) <= Rg)) break;
+                // rows k .. k+7 in order: (r[0].x,y) (r[0].z,w) (r[1].x,y) ...; larger d first
                 float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;
                 if (kRowP) {
                     pa = *reinterpret_cast<const float4 *>(tb.row_p + k);
@@ -306,6 +304,7 @@ __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y
 __device__ __forceinline__ unsigned char *stage_tables(unsigned char *smem, int n_types_alloc,
                                                        const Row *__restrict__ g_rows,
                                                        const uint2 *__restrict__ g_row_bounds,
+                                                       const float2 *__restrict__ g_group_bounds,
                                                        const unsigned char *__restrict__ g_start_table,
                                                        const TypeHeader *__restrict__ g_headers,
                                                        const int *__restrict__ table_info, Tables &tb,
@@ -318,13 +317,15 @@ __device__ __forceinline__ unsigned char *stage_tables(unsigned char *smem, int 
     Row *sh_rows = reinterpret_cast<Row *>(smem);
     TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
     uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
-    unsigned char *sh_start = reinterpret_cast<unsigned char *>(sh_row_bounds + kMaxPaddedRows);
+    float2 *sh_group_bounds = reinterpret_cast<float2 *>(sh_row_bounds + kMaxPaddedRows);
+    unsigned char *sh_start = reinterpret_cast<unsigned char *>(sh_group_bounds + kMaxPaddedRows / 8);
     for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[row_pos(k)] = g_rows[k];
     for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
+    for (int k = threadIdx.x; k < n_padded / 8; k += blockDim.x) sh_group_bounds[k] = g_group_bounds[k];
     for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
         reinterpret_cast<uint4 *>(sh_start)[k] = reinterpret_cast<const uint4 *>(g_start_table)[k];
     if (threadIdx.x < n_act) sh_headers[threadIdx.x] = g_headers[threadIdx.x];
-    tb.headers = sh_headers; tb.row_bounds = sh_row_bounds;
+    tb.headers = sh_headers; tb.row_bounds = sh_row_bounds; tb.group_bounds = sh_group_bounds;
     tb.start_table = sh_start; tb.rows = sh_rows;
     tb.n_types = unsafe ? 0 : n_act;          // unusable bounds: every request takes the exhaustive path
     unsigned char *end = sh_start + n_types_alloc * (kStartBuckets * kStartSlots);
@@ -575,6 +576,7 @@ __global__ void __launch_bounds__(route_threads(kRowP, kReqPerThread), kRouteMin
 route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__ pred_decode_len,
              const float *__restrict__ slo_ms, int64_t n, const PrefixHits hits, int n_types_alloc,
              const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
+             const float2 *__restrict__ g_group_bounds,
              const unsigned char *__restrict__ g_start_table,
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
              const unsigned short *__restrict__ g_cand, const uint2 *__restrict__ g_pool,
@@ -627,7 +629,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     const int M = table_info[2];
     const float cand_z0 = __int_as_float(table_info[4]), cand_inv = __int_as_float(table_info[5]);
     Tables tb;
-    unsigned char *after_tables = stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_start_table, g_headers,
+    unsigned char *after_tables = stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_group_bounds, g_start_table, g_headers,
                                                table_info, tb, kRowP ? g_row_p : nullptr);
     unsigned short *sh_cand = reinterpret_cast<unsigned short *>(after_tables);
     if (threadIdx.x < kCandSlots) sh_cand[threadIdx.x] = g_cand[threadIdx.x];
@@ -837,7 +839,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
 }
 
 constexpr size_t kTablesSmemFixed = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
-                                    (size_t)kMaxPaddedRows * sizeof(uint2);
+                                    (size_t)kMaxPaddedRows * sizeof(uint2) + kMaxPaddedRows / 8 * sizeof(float2);
 constexpr size_t kRouteSmemFixed = kTablesSmemFixed + kCandSlots * sizeof(unsigned short) +
                                    (size_t)(route_threads(false, 1) / 32) * kQueueCap * sizeof(unsigned);
 constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
@@ -871,7 +873,7 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
 #define GS_LAUNCH_ROUTE_R(ACC, PFX, ROWP, REQ)                                                        \
     route_kernel<ACC, PFX, ROWP, REQ><<<(unsigned)blocks, route_threads(ROWP, REQ), smem, st>>>(      \
         prompt_len, pred_decode_len, slo_ms, n, hits ? *hits : none, n_types, ctx->s.rows,            \
-        ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, ctx->s.cand_table,  \
+        ctx->s.row_bounds, ctx->s.group_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, ctx->s.cand_table,  \
         ctx->s.pool, ctx->s.bucket_list, ctx->s.start_list, ctx->s.row_p,                             \
         out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status)
     // (the prefix term and per-row p are never combined with accumulate, nor with each other)
@@ -899,6 +901,7 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
                const float *__restrict__ slo, const int32_t *__restrict__ prompt_len, int64_t n_active,
                int n_types_alloc,
                const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
+             const float2 *__restrict__ g_group_bounds,
                const unsigned char *__restrict__ g_start_table,
                const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
                int32_t *__restrict__ out_inst, float *__restrict__ out_est,
@@ -907,7 +910,7 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
     extern __shared__ __align__(16) unsigned char smem[];
     const int M = table_info[2];
     Tables tb;
-    stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_start_table, g_headers, table_info, tb);
+    stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_group_bounds, g_start_table, g_headers, table_info, tb);
     __syncthreads();
 
     int64_t n = *cand_count;
@@ -980,7 +983,7 @@ cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *
     LaunchTimer timer(ctx, GS_K_REROUTE, st);
     reroute_kernel<<<(unsigned)blocks, kRerouteThreads, smem, st>>>(
         cand_idx, cand_count, cand_capacity, assigned, generated, pred_len, elapsed, slo, prompt_len, n_active,
-        n_types, ctx->s.rows, ctx->s.row_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info,
+        n_types, ctx->s.rows, ctx->s.row_bounds, ctx->s.group_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info,
         out_inst, out_est, out_slack, out_tier, ctx->s.status);
     return cudaGetLastError();
 }
