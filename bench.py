@@ -42,11 +42,11 @@ ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-ins
 # profiles/risk_flags_kernel_config3.md).  They describe the kernel sources with these hashes;
 # after any change to those files they no longer apply and the fields that use them become
 # null until the kernel is profiled again.
-PROFILED_ROUTE = {"sources_sha1": "44a17f186ef9d74c2bc7d4d3fc0bc9bd6ed54858", "config": 3,
-                  "dram_bytes_per_launch": 52_436_992 + 7_620_864,
-                  "warp_instructions_per_launch": 25_137_038}
-PROFILED_RISK_FLAGS = {"sources_sha1": "f8e31b7c345a323b00a561cf8750b4981dfafdb6", "config": 3,
-                       "dram_bytes_per_launch": 335_563_008 + 5_301_760}
+PROFILED_ROUTE = {"sources_sha1": "58d1cdce5b807a322ce0423c56df0f812499423e", "config": 3,
+                  "dram_bytes_per_launch": 52_283_136 + 8_322_048,
+                  "warp_instructions_per_launch": 24_754_981}
+PROFILED_RISK_FLAGS = {"sources_sha1": "23376727e5a3e7bc33cc0aaa3cba258afd1240c6", "config": 3,
+                       "dram_bytes_per_launch": 335_588_608 + 3_752_448}
 
 
 def _sources_sha1(names) -> str:
