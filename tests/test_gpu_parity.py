@@ -256,6 +256,27 @@ def test_accumulate_and_advance_saturate(gs):
     np.testing.assert_array_equal(pool.decode_batch.cpu().numpy(), state.decode_batch)
 
 
+def test_accumulate_with_the_most_types(gs):
+    """Sixteen GPU types make the route kernel's tables as large as they get; with the
+    per-instance sums of the accumulate variant beside them the CTA's shared memory is at its
+    fullest.  Decisions and the advanced state must still be the oracle's."""
+    rng = np.random.default_rng(16)
+    types, inst = _random_pool(rng, 1024, 16)
+    pool = pool_of(gs, types, inst)
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    req = _boundary_requests(rng, t32, 9000)
+    got = gpu_route(gs, pool, req, 0.5, accumulate=True)
+    gs.advance_state(pool)
+    ref = oracle.route(t32, *req.columns(), threads=4)
+    assert_route_matches_f32_oracle(got, ref)
+    state = inst.copy()
+    oracle.advance(state, t32, ref.instance_idx, req.prompt_len, req.pred_decode_len)
+    np.testing.assert_array_equal(pool.queued_prefill_tokens.cpu().numpy(), state.queued_prefill_tokens)
+    np.testing.assert_array_equal(pool.decode_batch.cpu().numpy(), state.decode_batch)
+    np.testing.assert_array_equal(pool.free_kv_tokens.cpu().numpy(), state.free_kv_tokens)
+    assert gs.device_status() == 0
+
+
 def test_route_without_accumulate_leaves_state_alone(gs):
     wl = W.make_workload(1, n_requests=4096, n_active=16)
     pool = pool_of(gs, wl.types, wl.instances)
