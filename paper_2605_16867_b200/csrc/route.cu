@@ -108,9 +108,13 @@ __device__ __forceinline__ int start_slot(float R, float q_lo, float ry, float d
     return __float2int_rd(fminf(fmaxf((z - d0) * inv_w, 0.f), (float)(kStartSlots - 1)));
 }
 // Lanes of a warp that must need the fallback before each runs its own search; below that the
-// warp-wide scoring of every instance is the shorter way.
+// whole warp would score every instance for each of them.  The full search only ever sees
+// requests that the first attempt left open, a few to a warp at the end of the kernel, and
+// there one lane's own search (about 700 instructions) is shorter than the warp's scan of all
+// instances (about 800 for each such request), so the lane always searches for itself; the
+// warp-wide scan remains for requests that the tables cannot serve.
 #ifndef GS_THREAD_FALLBACK_MIN
-#define GS_THREAD_FALLBACK_MIN 3
+#define GS_THREAD_FALLBACK_MIN 1
 #endif
 constexpr int kThreadFallbackMin = GS_THREAD_FALLBACK_MIN;
 
