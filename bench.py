@@ -42,11 +42,11 @@ ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-ins
 # profiles/risk_flags_kernel_config3.md).  They describe the kernel sources with these hashes;
 # after any change to those files they no longer apply and the fields that use them become
 # null until the kernel is profiled again.
-PROFILED_ROUTE = {"sources_sha1": "58d1cdce5b807a322ce0423c56df0f812499423e", "config": 3,
-                  "dram_bytes_per_launch": 52_283_136 + 8_322_048,
-                  "warp_instructions_per_launch": 24_754_981}
+PROFILED_ROUTE = {"sources_sha1": "aabfbd386a434106d3a56a21b5d4f4681f8870af", "config": 3,
+                  "dram_bytes_per_launch": 52_352_256 + 7_199_488,
+                  "warp_instructions_per_launch": 24_600_939}
 PROFILED_RISK_FLAGS = {"sources_sha1": "23376727e5a3e7bc33cc0aaa3cba258afd1240c6", "config": 3,
-                       "dram_bytes_per_launch": 335_588_608 + 3_752_448}
+                       "dram_bytes_per_launch": 335_564_032 + 4_064_256}
 
 
 def _sources_sha1(names) -> str:
