@@ -42,7 +42,7 @@ ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-ins
 # profiles/risk_flags_kernel_config3.md).  They describe the kernel sources with these hashes;
 # after any change to those files they no longer apply and the fields that use them become
 # null until the kernel is profiled again.
-PROFILED_ROUTE = {"sources_sha1": "aabfbd386a434106d3a56a21b5d4f4681f8870af", "config": 3,
+PROFILED_ROUTE = {"sources_sha1": "bac3726b1cb32d3d74d0cdb6b491727579021779", "config": 3,
                   "dram_bytes_per_launch": 52_352_256 + 7_199_488,
                   "warp_instructions_per_launch": 24_600_939}
 PROFILED_RISK_FLAGS = {"sources_sha1": "23376727e5a3e7bc33cc0aaa3cba258afd1240c6", "config": 3,

@@ -170,7 +170,8 @@ GS_API int gs_timing_read(gs_ctx *ctx, int kernel, double *total_ms, int64_t *la
  *                     3 = no instance has KV room: minimum T among all.
  * Ties (equal d_g, or equal T in the fallback) go to the smallest instance index.
  * Feasibility is T <= D (a request whose estimate equals its deadline is feasible).
- * n_requests == 0 is valid and enqueues nothing.  Never writes the instance state.
+ * n_requests == 0 is valid and enqueues nothing; more than 2^36 requests in one call is refused
+ * (GS_ERR_CUDA, invalid value).  Never writes the instance state.
  */
 GS_API int gs_route_batch(gs_ctx *ctx,
                    const int32_t *prompt_len, const int32_t *pred_decode_len,

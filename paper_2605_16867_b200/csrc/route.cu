@@ -865,6 +865,9 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
                          bool accumulate, bool row_p, cudaStream_t st)
 {
     if (n == 0) return cudaSuccess;
+    // (the kernel's queues hold a request's index within its CTA's run as 32 bits; with at most one
+    // CTA per SM that bounds a batch far beyond what fits in device memory)
+    if (n > ((int64_t)1 << 36)) return cudaErrorInvalidValue;
     const size_t smem = route_smem_bytes(n_types, accumulate, row_p);
     const int req = n < kSmallBatch ? 1 : 4;
     const int64_t tile = (int64_t)route_threads(row_p, req) * req;
