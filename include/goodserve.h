@@ -375,15 +375,15 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx,
  * plugin running inside someone else's memory pool, a latency-critical loop where an
  * allocation's implicit device synchronisation is unacceptable.  Such callers cannot create
  * a gs_ctx (gs_create allocates), so this call takes none: the scratch that gs_risk_scan
- * keeps in its context (the flag counts its two passes exchange) lives instead
- * in a fixed array inside the library image, 66 KB that every GPU loading the library
+ * keeps in its context (the per-CTA flag counts its two passes exchange) lives instead
+ * in a fixed array inside the library image, 16 KB that every GPU loading the library
  * holds until the process exits.  It computes exactly what gs_risk_scan computes, with the
  * same kernels; inputs, outputs and their layout are the same and still belong to the caller.
  *
  *   - Runs on the CURRENT device (cudaGetDevice) and enqueues on `cuda_stream`, which must
  *     belong to it.  No cudaMalloc, cudaFree or allocating library routine is called.
- *   - n_active may not exceed GS_NOALLOC_MAX_ACTIVE (the array is sized for that); a larger
- *     value returns GS_ERR_TOO_LARGE and enqueues nothing.
+ *   - n_active may not exceed GS_NOALLOC_MAX_ACTIVE (the stated limit of this entry point); a
+ *     larger value returns GS_ERR_TOO_LARGE and enqueues nothing.
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress).  Make that first call outside any stream capture.
  *   - All calls on one GPU share the one array, and it keeps the previous call's contents;

@@ -273,9 +273,9 @@ void gso_advance(int32_t M, int64_t N, const int32_t *instance_idx,
 
 /* ------------------------------------------------------------------------------------ */
 /* Re-routing of flagged requests (Sec. 3.4): a request whose expected finish exceeds its */
-/* SLO is re-routed "to another GPU with stronger processing capability (still following  */
-/* the just-enough heuristic)"; the migration moves token IDs, so the target re-prefills   */
-/* the whole context (prompt + tokens generated so far).                                   */
+/* SLO moves to a faster instance, chosen again by the just-enough rule; the migration    */
+/* moves token IDs, so the target re-prefills the whole context (prompt + tokens          */
+/* generated so far).                                                                      */
 /*                                                                                        */
 /* Reading: for candidate i on instance c                                                  */
 /*   x' = prompt_len + generated,  y' = max(pred_len - generated, 0),  D' = slo - elapsed  */

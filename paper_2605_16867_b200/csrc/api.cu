@@ -151,8 +151,6 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
     ctx->pending = new (std::nothrow) std::vector<gs_ctx::TimedLaunch>();
     ctx->free_events = new (std::nothrow) std::vector<cudaEvent_t>();
     if (!ctx->pending || !ctx->free_events) { delete ctx->pending; delete ctx->free_events; delete ctx; return GS_ERR_INVALID_ARG; }
-    ctx->max_chunks = ((size_t)gs::kMaxActive + gs::kRiskChunk - 1) / gs::kRiskChunk;
-    ctx->max_groups = (ctx->max_chunks + 63) / 64;
 
     const size_t Mx = GS_MAX_INSTANCES;
     gs::Scratch &s = ctx->s;
@@ -171,8 +169,7 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
         {(void **)&s.d_by_g, Mx * sizeof(float)},
         {(void **)&s.q_by_g, Mx * sizeof(float)},
         {(void **)&s.deltas, 3 * Mx * sizeof(unsigned long long)},
-        {(void **)&s.chunk_counts, ctx->max_chunks * sizeof(unsigned)},
-        {(void **)&s.group_totals, 2 * ctx->max_groups * sizeof(unsigned)},
+        {(void **)&s.scan_counts, gs::kMaxScanCtas * sizeof(unsigned)},
         {(void **)&s.status, 256},
     };
     for (auto &a : allocs) {
@@ -192,7 +189,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.d_by_g, s.q_by_g, s.deltas, s.chunk_counts, s.group_totals, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.d_by_g, s.q_by_g, s.deltas, s.scan_counts, s.status, ctx->stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);

@@ -79,7 +79,7 @@ constexpr int kListWindow = 8;             // entries the first attempt may test
 constexpr int kListMax = 510;              // longer lists are not stored (start_list counts pairs of entries in a byte)
 constexpr unsigned short kNoList = 0xFFFFu;
 
-constexpr int kRiskChunk = 1024;        // requests per warp-chunk of the risk scan (32 flag words)
+constexpr int kMaxScanCtas = 4096;      // CTAs of one risk scan (a few per SM), one flag count each
 constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 
 // Device scratch owned by a context.
@@ -100,8 +100,7 @@ struct Scratch {
     float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
     float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out
-    unsigned *chunk_counts;   // [max_chunks] risk scan: flags per chunk of 1024 requests
-    unsigned *group_totals;   // [2 * max_groups] risk scan: flags per 64 chunks, two parities
+    unsigned *scan_counts;    // [kMaxScanCtas] risk scan: requests flagged by each CTA of pass 1
     unsigned *status;         // device status word
 };
 
@@ -114,9 +113,6 @@ struct gs_ctx {
     int n_sm;
     int reroute_ctas_per_sm[GS_MAX_TYPES + 1];   // by number of types (sets the shared-memory size)
     gs::Scratch s;
-    size_t max_chunks, max_groups;   // capacity of the risk scan's count arrays
-    unsigned scan_epoch;             // its parity selects the group-total buffer of the next scan
-    int64_t scan_dirty[2];           // entries of each group-total buffer that may be non-zero
     int64_t launches;
     int last_cuda_error;
     // staging for the *_host entry points (device memory, grown on demand)

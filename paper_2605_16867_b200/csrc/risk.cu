@@ -1,19 +1,25 @@
 // gs_risk_scan: the SLO-violation risk test of Sec. 3.4 over all active requests and the
 // ordered compaction of the flagged ones (migration candidates).
 //
-// Pass 1 (risk_flags_kernel) streams the five request columns once.  Each CTA first computes
-// d_g = a_t + b_t * batch_g for every instance into shared memory; a warp then takes chunks of
-// 1024 requests, gathers d_g of the assigned instance, and emits one flag word per 32 requests
-// with a warp ballot.  It leaves the chunk's number of flags, and adds it to the total of the
-// chunk's group of 64 chunks.
-// Pass 2 (scatter_candidates_kernel) re-reads only the flag words.  Every warp owns a
-// contiguous run of chunks; it sums the group totals and chunk counts that precede its run
-// once, then keeps a running offset, and writes the ascending candidate list: a request's
-// position is that offset plus popc of the lower flags.
-// There is no device-side wait anywhere in the scan.
+// The requests are cut into steps of 128 (four flag words) and the steps dealt out evenly: CTA b
+// of G owns the contiguous run of steps [b S / G, (b + 1) S / G).  Both passes use the same G.
 //
-// The group totals are double-buffered by call parity: pass 2 of one call clears the buffer
-// that pass 1 of the next call adds into.
+// Pass 1 (risk_flags_kernel) streams the five request columns once.  Each CTA first computes
+// d_g = a_t + b_t * batch_g for every instance into shared memory; its warps then take the
+// CTA's steps in turn, four consecutive requests per lane (128-bit column loads), gather d_g of
+// the assigned instance and assemble the flag words (a nibble per lane, OR-reduced over each
+// eight lanes).  The CTA leaves one number: how many requests it flagged.
+// Pass 2 (scatter_candidates_kernel) re-reads only the flag words.  CTA b sums the counts of
+// the CTAs before it, then walks its own run 8 x 1024 requests at a time: a warp counts the
+// flags of its 1024 requests, the counts of the eight warps are exchanged through shared memory,
+// and each warp writes its part of the ascending candidate list word by word: a flagged
+// request's position is the running offset plus the number of flagged requests below it in its
+// word, so the lanes that hold a flag store to consecutive entries.
+//
+// Nothing is accumulated with atomics and nothing survives a call: every word of scratch that
+// pass 2 reads was stored by pass 1 of the same call.  There is no device-side wait.  Pass 2 is
+// launched as a programmatic dependent of pass 1 (its launch overlaps pass 1's tail; it waits
+// for pass 1's memory before it reads anything).
 #include <mutex>
 
 #include "gs_internal.cuh"
@@ -22,161 +28,293 @@ namespace gs {
 
 constexpr int kRiskThreads = 256;
 constexpr int kRiskWarps = kRiskThreads / 32;
-constexpr int kRiskUnroll = 4;          // independent 32-request groups in flight per warp
-constexpr int kGroupShift = 6;          // 64 chunks per group
+#ifndef GS_RISK_UNROLL
+#define GS_RISK_UNROLL 1
+#endif
+#ifndef GS_RISK_MIN_CTAS
+#define GS_RISK_MIN_CTAS 4
+#endif
+#ifndef GS_RISK_PDL
+#define GS_RISK_PDL 2       // pass 2 as a programmatic dependent of pass 1: 0 no, 1 set up from pass 1's start, 2 from its end
+#endif
+constexpr int kRiskUnroll = GS_RISK_UNROLL;   // steps of 128 requests a warp works on at a time (as many again are on their way)
+constexpr int kRiskMinCtas = GS_RISK_MIN_CTAS;
+constexpr int kStepShift = 7;                 // 128 requests per step
 
-__global__ void __launch_bounds__(kRiskThreads)
+// First step of CTA b's run when S steps are dealt to G CTAs.
+__host__ __device__ __forceinline__ int64_t first_step_of(int64_t b, int64_t S, int64_t G) { return b * S / G; }
+
+// Risk test of one request (Sec. 3.4): expected finish = elapsed + d_assigned * tokens left;
+// flagged when it exceeds the SLO.  Out-of-range data is clamped and reported in `bad`.
+__device__ __forceinline__ bool risk_flag(const float *sh_d, int M, int g, int gen, int tot, float el, float dl,
+                                          unsigned &bad)
+{
+    if ((unsigned)g >= (unsigned)M) { g = g < 0 ? 0 : M - 1; bad |= GS_DEV_BAD_INSTANCE; }
+    if ((gen | tot) < 0) { gen = max(gen, 0); tot = max(tot, 0); bad |= GS_DEV_BAD_VALUE; }
+    const int rem = max(tot - gen, 0);
+    return __fmaf_rn(sh_d[g], __int2float_rn(rem), el) > dl;
+}
+
+// The five columns of one step (128 requests), four consecutive requests per lane.
+struct StepData {
+    int4 g, gen, tot;
+    float4 el, dl;
+};
+
+__device__ __forceinline__ void load_step(StepData &d, const int32_t *__restrict__ assigned,
+                                          const int32_t *__restrict__ generated, const int32_t *__restrict__ pred_len,
+                                          const float *__restrict__ elapsed, const float *__restrict__ slo,
+                                          int64_t step, int lane)
+{
+    const int64_t i = (step << kStepShift) + lane * 4;
+    d.g = __ldcs(reinterpret_cast<const int4 *>(assigned + i));
+    d.gen = __ldcs(reinterpret_cast<const int4 *>(generated + i));
+    d.tot = __ldcs(reinterpret_cast<const int4 *>(pred_len + i));
+    d.el = __ldcs(reinterpret_cast<const float4 *>(elapsed + i));
+    d.dl = __ldcs(reinterpret_cast<const float4 *>(slo + i));
+}
+
+__global__ void __launch_bounds__(kRiskThreads, kRiskMinCtas)
 risk_flags_kernel(const int32_t *__restrict__ assigned, const int32_t *__restrict__ generated,
                   const int32_t *__restrict__ pred_len, const float *__restrict__ elapsed,
                   const float *__restrict__ slo, int64_t n,
                   const int32_t *__restrict__ type_id, const int32_t *__restrict__ batch, int M,
                   const float *__restrict__ a_type, const float *__restrict__ b_type, int n_types,
-                  uint32_t *__restrict__ flag_bits, unsigned *__restrict__ chunk_counts,
-                  unsigned *__restrict__ group_totals, int64_t n_chunks, unsigned *__restrict__ status)
+                  uint32_t *__restrict__ flag_bits, unsigned *__restrict__ cta_counts,
+                  int64_t n_steps, unsigned *__restrict__ status)
 {
+#if GS_RISK_PDL == 1
+    // the dependent launch (pass 2) may be set up from now on; it still waits for this grid's end
+    asm volatile("griddepcontrol.launch_dependents;");
+#endif
     __shared__ float sh_d[GS_MAX_INSTANCES];
+    __shared__ float sh_a[GS_MAX_TYPES], sh_b[GS_MAX_TYPES];
+    __shared__ unsigned sh_count;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int64_t s_begin = first_step_of(blockIdx.x, n_steps, gridDim.x);
+    const int64_t s_end = first_step_of((int64_t)blockIdx.x + 1, n_steps, gridDim.x);
+    // steps that lie wholly inside the batch and inside this CTA's run take the 128-bit path
+    const int64_t s_fast = min(s_end, n >> kStepShift);
+
+    // the warp's first steps are on their way while the CTA works out d_g
+    StepData cur[kRiskUnroll];
+    int64_t s0 = s_begin + warp;             // warp w takes the steps w, w + 8, .. of the run
+#pragma unroll
+    for (int u = 0; u < kRiskUnroll; ++u)
+        if (s0 + u * kRiskWarps < s_fast) load_step(cur[u], assigned, generated, pred_len, elapsed, slo, s0 + u * kRiskWarps, lane);
+
+    // d_g for every instance: all global loads are issued together (one round trip, not one per
+    // dependent step), the type constants go through shared memory
     unsigned bad = 0;
-    for (int g = threadIdx.x; g < M; g += blockDim.x) {
-        int t = type_id[g];
+    constexpr int kPerThread = GS_MAX_INSTANCES / kRiskThreads;
+    int r_type[kPerThread], r_batch[kPerThread];
+#pragma unroll
+    for (int k = 0; k < kPerThread; ++k) {
+        const int g = threadIdx.x + k * kRiskThreads;
+        r_type[k] = g < M ? type_id[g] : 0;
+        r_batch[k] = g < M ? batch[g] : 0;
+    }
+    if (threadIdx.x < n_types) { sh_a[threadIdx.x] = a_type[threadIdx.x]; sh_b[threadIdx.x] = b_type[threadIdx.x]; }
+    if (threadIdx.x == 0) sh_count = 0u;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kPerThread; ++k) {
+        const int g = threadIdx.x + k * kRiskThreads;
+        if (g >= M) break;
+        int t = r_type[k], B = r_batch[k];
         if (t < 0 || t >= n_types) { bad |= GS_DEV_BAD_TYPE; t = 0; }
-        int B = batch[g];
         if (B < 0) { bad |= GS_DEV_BAD_VALUE; B = 0; }
-        sh_d[g] = __fmaf_rn(b_type[t], __int2float_rn(B), a_type[t]);   // loaded per-token decode latency
+        sh_d[g] = __fmaf_rn(sh_b[t], __int2float_rn(B), sh_a[t]);       // loaded per-token decode latency
     }
     if (blockIdx.x != 0) bad = 0;           // one CTA reports bad pool data
     __syncthreads();
 
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    const int64_t n_words = (n + 31) >> 5;
+    const unsigned oct_mask = 0xFFu << (lane & 24);     // the eight lanes that share a flag word
+    const int nib_shift = (lane & 7) << 2;
+    unsigned flagged = 0;                               // flags this lane has seen (its own nibbles)
 
-    for (int64_t chunk = (int64_t)blockIdx.x * kRiskWarps + warp; chunk < n_chunks;
-         chunk += (int64_t)gridDim.x * kRiskWarps) {
-        const int64_t first = chunk * kRiskChunk;
-        uint32_t my_word = 0;               // lane l ends up holding word l of the chunk
 #pragma unroll 1
-        for (int w0 = 0; w0 < 32; w0 += kRiskUnroll) {
-            int g[kRiskUnroll], gen[kRiskUnroll], tot[kRiskUnroll];
-            float el[kRiskUnroll], dl[kRiskUnroll];
-            bool valid[kRiskUnroll];
+    for (; s0 < s_end; s0 += kRiskWarps * kRiskUnroll) {
+        const int64_t s_next = s0 + kRiskWarps * kRiskUnroll;
+        StepData nxt[kRiskUnroll];
 #pragma unroll
-            for (int u = 0; u < kRiskUnroll; ++u) {
-                const int64_t i = first + (int64_t)(w0 + u) * 32 + lane;
-                valid[u] = i < n;
-                g[u] = valid[u] ? __ldcs(assigned + i) : 0;
-                gen[u] = valid[u] ? __ldcs(generated + i) : 0;
-                tot[u] = valid[u] ? __ldcs(pred_len + i) : 0;
-                el[u] = valid[u] ? __ldcs(elapsed + i) : 0.f;
-                dl[u] = valid[u] ? __ldcs(slo + i) : 0.f;
-            }
+        for (int u = 0; u < kRiskUnroll; ++u)            // the next steps are requested before these are worked on
+            if (s_next + u * kRiskWarps < s_fast) load_step(nxt[u], assigned, generated, pred_len, elapsed, slo, s_next + u * kRiskWarps, lane);
 #pragma unroll
-            for (int u = 0; u < kRiskUnroll; ++u) {
-                int gi = g[u];
-                if (gi < 0) { gi = 0; bad |= GS_DEV_BAD_INSTANCE; }
-                if (gi >= M) { gi = M - 1; bad |= GS_DEV_BAD_INSTANCE; }
-                int ge = gen[u], to = tot[u];
-                if (ge < 0) { ge = 0; bad |= GS_DEV_BAD_VALUE; }
-                if (to < 0) { to = 0; bad |= GS_DEV_BAD_VALUE; }
-                const int rem = max(to - ge, 0);
-                const float finish = __fmaf_rn(sh_d[gi], __int2float_rn(rem), el[u]);
-                const bool flag = valid[u] && (finish > dl[u]);
-                const uint32_t word = __ballot_sync(0xFFFFFFFFu, flag);
-                if (lane == w0 + u) my_word = word;
+        for (int u = 0; u < kRiskUnroll; ++u) {
+            const int64_t s = s0 + u * kRiskWarps;
+            if (s >= s_end) break;
+            unsigned nib = 0;
+            if (s < s_fast) {
+                const StepData &d = cur[u];
+                nib = risk_flag(sh_d, M, d.g.x, d.gen.x, d.tot.x, d.el.x, d.dl.x, bad) ? 1u : 0u;
+                nib |= risk_flag(sh_d, M, d.g.y, d.gen.y, d.tot.y, d.el.y, d.dl.y, bad) ? 2u : 0u;
+                nib |= risk_flag(sh_d, M, d.g.z, d.gen.z, d.tot.z, d.el.z, d.dl.z, bad) ? 4u : 0u;
+                nib |= risk_flag(sh_d, M, d.g.w, d.gen.w, d.tot.w, d.el.w, d.dl.w, bad) ? 8u : 0u;
+            } else {
+                // the ragged last step of the batch: request by request
+                const int64_t i0 = (s << kStepShift) + lane * 4;
+                for (int j = 0; j < 4; ++j)
+                    if (i0 + j < n && risk_flag(sh_d, M, assigned[i0 + j], generated[i0 + j], pred_len[i0 + j],
+                                                elapsed[i0 + j], slo[i0 + j], bad))
+                        nib |= 1u << j;
             }
+            flagged += __popc(nib);
+            // lanes 8w .. 8w+7 hold the eight nibbles of word w of this step
+            const uint32_t word = __reduce_or_sync(oct_mask, nib << nib_shift);
+            const int64_t wi = (s << 2) + (lane >> 3);
+            if ((lane & 7) == 0 && wi < ((n + 31) >> 5)) flag_bits[wi] = word;
         }
-        const int64_t wi = chunk * 32 + lane;
-        if (wi < n_words) flag_bits[wi] = my_word;
-        const unsigned total = __reduce_add_sync(0xFFFFFFFFu, (unsigned)__popc(my_word));
-        if (lane == 0) {
-            chunk_counts[chunk] = total;
-            if (total) atomicAdd(group_totals + (chunk >> kGroupShift), total);
-        }
+#pragma unroll
+        for (int u = 0; u < kRiskUnroll; ++u) cur[u] = nxt[u];
     }
+#if GS_RISK_PDL == 2
+    // pass 2 may be set up from now on (it still waits for this whole grid before it reads): at
+    // 16 M requests that is worth nothing, at 2 M and below it hides pass 2's launch (2 us)
+    asm volatile("griddepcontrol.launch_dependents;");
+#endif
+    flagged = __reduce_add_sync(0xFFFFFFFFu, flagged);
+    if (lane == 0 && flagged) atomicAdd(&sh_count, flagged);
+    __syncthreads();
+    if (threadIdx.x == 0) cta_counts[blockIdx.x] = sh_count;
     if (bad) atomicOr(status, bad);
 }
 
+constexpr int kScatterBlocks = 4;           // blocks of 32 flag words (1024 requests) per warp and round
+
 __global__ void __launch_bounds__(kRiskThreads)
 scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_words,
-                          const unsigned *__restrict__ chunk_counts,
-                          const unsigned *__restrict__ group_totals, unsigned *__restrict__ next_group_totals,
-                          int64_t n_clear, int64_t n_chunks, int64_t chunks_per_warp,
+                          const unsigned *__restrict__ cta_counts, int64_t n_steps,
                           int32_t *__restrict__ cand_idx, int64_t cand_capacity,
                           int64_t *__restrict__ cand_count, unsigned *__restrict__ status)
 {
     const int lane = threadIdx.x & 31;
-    const int64_t gwarp = (int64_t)blockIdx.x * kRiskWarps + (threadIdx.x >> 5);
-     // clear what an earlier call left in the other parity's group totals, for the next call
-    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n_clear;
-         k += (int64_t)gridDim.x * blockDim.x)
-        next_group_totals[k] = 0u;
+    const int warp = threadIdx.x >> 5;
+    __shared__ unsigned sh_part[kRiskWarps];
+    __shared__ unsigned sh_cnt[2][kRiskWarps * kScatterBlocks];
+    __shared__ uint2 sh_words[kRiskWarps][32];
+    // the CTA's run of flag words; a round covers 8 warps x 4 blocks of 32 words, warp w the
+    // blocks w, w + 8, w + 16, w + 24 of the round
+    const int64_t w_begin = first_step_of(blockIdx.x, n_steps, gridDim.x) << 2;
+    const int64_t w_end = min(first_step_of((int64_t)blockIdx.x + 1, n_steps, gridDim.x) << 2, n_words);
+    // everything read below is written by pass 1: wait until that grid is done and visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    const int64_t c0 = gwarp * chunks_per_warp;
-    if (c0 >= n_chunks) return;
-    const int64_t c1 = min(c0 + chunks_per_warp, n_chunks);
-
-    // flags before chunk c0: whole groups, then the chunks of c0's own group
+    // flags before this CTA's run: the counts of the CTAs before it (fewer than 2^31 in all)
     unsigned part = 0;
-    const int64_t g0 = c0 >> kGroupShift;
-    for (int64_t k = lane; k < g0; k += 32 * 8) {           // eight independent loads in flight
-        unsigned v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = k + 32 * u < g0 ? group_totals[k + 32 * u] : 0u;
-#pragma unroll
-        for (int u = 0; u < 8; ++u) part += v[u];
-    }
-    {
-        const int64_t k = (g0 << kGroupShift) + lane;       // at most 64 chunks of c0's own group
-        part += (k < c0 ? chunk_counts[k] : 0u) + (k + 32 < c0 ? chunk_counts[k + 32] : 0u);
-    }
-    int64_t base = (int64_t)__reduce_add_sync(0xFFFFFFFFu, part);
+    for (int k = threadIdx.x; k < (int)blockIdx.x; k += kRiskThreads) part += __ldcg(cta_counts + k);
+    part = __reduce_add_sync(0xFFFFFFFFu, part);
+    if (lane == 0) sh_part[warp] = part;
 
-    __shared__ unsigned short sh_stage[kRiskWarps][kRiskChunk];   // a chunk's flagged positions, in order
-    unsigned short *stage = sh_stage[threadIdx.x >> 5];
-    for (int64_t chunk = c0; chunk < c1; ++chunk) {
-        const int64_t wi = chunk * 32 + lane;
-        uint32_t word = wi < n_words ? __ldcs(flag_bits + wi) : 0u;
-        const unsigned c = __popc(word);
+    const unsigned lane_bit = 1u << lane, below = lane_bit - 1u;
+    int64_t base = 0;
+    int buf = 0;
+    for (int64_t w0 = w_begin; w0 < w_end; w0 += kRiskWarps * kScatterBlocks * 32, buf ^= 1) {
+        uint32_t word[kScatterBlocks];
+#pragma unroll
+        for (int k = 0; k < kScatterBlocks; ++k) {
+            const int64_t wi = w0 + (k * kRiskWarps + warp) * 32 + lane;
+            word[k] = wi < w_end ? __ldcs(flag_bits + wi) : 0u;
+        }
+#pragma unroll
+        for (int k = 0; k < kScatterBlocks; ++k) {
+            const unsigned total = __reduce_add_sync(0xFFFFFFFFu, (unsigned)__popc(word[k]));
+            if (lane == 0) sh_cnt[buf][k * kRiskWarps + warp] = total;
+        }
+        __syncthreads();                    // (the other buffer is free again after the next barrier)
+        if (w0 == w_begin) {
+#pragma unroll
+            for (int w = 0; w < kRiskWarps; ++w) base += sh_part[w];
+        }
+        // lane b holds the count of block b of the round: flags before each block, and in all
+        const unsigned c = sh_cnt[buf][lane];
         unsigned incl = c;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const unsigned v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
             if (lane >= off) incl += v;
         }
-        const unsigned total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-        // each lane lists the set bits of its own word behind those of the lower words ...
-        unsigned at = incl - c;
-        const unsigned lane_base = (unsigned)lane << 5;
-        while (word) {
-            stage[at++] = (unsigned short)(lane_base + (__ffs(word) - 1));
-            word &= word - 1;
+        const unsigned all = __shfl_sync(0xFFFFFFFFu, incl, 31);
+#pragma unroll
+        for (int k = 0; k < kScatterBlocks; ++k) {
+            const int blk = k * kRiskWarps + warp;
+            const unsigned total = __shfl_sync(0xFFFFFFFFu, c, blk);
+            const unsigned before = __shfl_sync(0xFFFFFFFFu, incl - c, blk);
+            if (total == 0) continue;
+            // flags in the block's words before each word (lane = word), then every word and its
+            // offset go through shared memory so that the loop below reads them as broadcasts
+            unsigned w_incl = __popc(word[k]);
+            const unsigned w_cnt = w_incl;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned v = __shfl_up_sync(0xFFFFFFFFu, w_incl, off);
+                if (lane >= off) w_incl += v;
+            }
+            __syncwarp();                   // (the previous block's entries have been read)
+            sh_words[warp][lane] = make_uint2(word[k], w_incl - w_cnt);
+            __syncwarp();
+            const int64_t mine = base + before;             // list position of the block's first flag
+            int32_t *out = cand_idx + mine;
+            const int32_t idx0 = (int32_t)((w0 + blk * 32) << 5) + lane;     // n_active < 2^31
+            if (mine + total <= cand_capacity) {
+#pragma unroll
+                for (int w = 0; w < 32; ++w) {
+                    const uint2 e = sh_words[warp][w];      // {flag word, flags before it}: same address in all lanes
+                    if (e.x & lane_bit) out[e.y + __popc(e.x & below)] = idx0 + (w << 5);
+                }
+            } else {
+                // the list ends inside this block (or has already ended): entries still free
+                const int64_t room64 = cand_capacity - mine;
+                const unsigned room = room64 <= 0 ? 0u : (unsigned)room64;      // < total <= 1024
+#pragma unroll 1
+                for (int w = 0; w < 32; ++w) {
+                    const uint2 e = sh_words[warp][w];
+                    const unsigned at = e.y + __popc(e.x & below);
+                    if ((e.x & lane_bit) && at < room) out[at] = idx0 + (w << 5);
+                }
+            }
         }
-        __syncwarp();
-        // ... and the warp copies the list out with contiguous stores
-        const int32_t idx0 = (int32_t)(chunk * kRiskChunk);             // n_active < 2^31
-        const int64_t room = cand_capacity - base;
-        const unsigned n_out = room <= 0 ? 0u : (room < (int64_t)total ? (unsigned)room : total);
-        int32_t *out = cand_idx + base;
-        for (unsigned i = lane; i < n_out; i += 32) out[i] = idx0 + (int32_t)stage[i];
-        __syncwarp();
-        base += total;
+        base += all;
     }
-    if (c1 == n_chunks && lane == 0) {      // the warp that owns the last chunk knows the total
+    if (w_begin >= w_end) {                 // (a CTA without words still has to know the total if it is the last)
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < kRiskWarps; ++w) base += sh_part[w];
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {     // the last CTA knows the total
         *cand_count = base;
         if (base > cand_capacity) atomicOr(status, (unsigned)GS_DEV_CAND_TRUNCATED);
     }
 }
 
-// Host side of one scan; `epoch` (host) selects the group-total buffer of this call and
-// `dirty[b]` (host) is how many entries of buffer b may be non-zero.
-struct ScanLaunch {
-    unsigned *chunk_counts;
-    unsigned *group_totals;     // two buffers of max_groups entries, both zero before the first call
-    size_t max_groups;
-    unsigned *epoch;
-    int64_t *dirty;
-};
+// CTAs of pass 1 that fit on one SM (looked up once per device).
+static int risk_ctas_per_sm(int dev)
+{
+    static std::mutex mu;
+    static int cached[64];
+    std::lock_guard<std::mutex> lock(mu);
+    if (dev < 0 || dev >= 64) return kRiskMinCtas;
+    if (cached[dev] == 0) {
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, risk_flags_kernel, kRiskThreads, 0) != cudaSuccess || occ < 1)
+            occ = kRiskMinCtas;
+        cached[dev] = occ;
+    }
+    return cached[dev];
+}
 
-static cudaError_t enqueue_scan(const ScanLaunch &sl, int n_sm, gs_ctx *timing_ctx,
+// Number of CTAs (of both passes) for a scan of n requests on a GPU with n_sm SMs: every SM
+// full, but no CTA with less than one round of its warps' steps.
+static int64_t scan_grid(int64_t n_steps, int dev, int n_sm)
+{
+    int64_t blocks = (n_steps + kRiskWarps * kRiskUnroll - 1) / (kRiskWarps * kRiskUnroll);
+    const int64_t cap = (int64_t)n_sm * risk_ctas_per_sm(dev);
+    return blocks > cap ? cap : blocks;
+}
+
+// One scan: cta_counts is scratch for one count per CTA (kMaxScanCtas entries).
+static cudaError_t enqueue_scan(unsigned *cta_counts, int dev, int n_sm, gs_ctx *timing_ctx,
                                 const int32_t *assigned, const int32_t *generated, const int32_t *pred_len,
                                 const float *elapsed, const float *slo, int64_t n,
                                 const gs_instances &inst, const gs_types &types,
@@ -184,33 +322,34 @@ static cudaError_t enqueue_scan(const ScanLaunch &sl, int n_sm, gs_ctx *timing_c
                                 int64_t *cand_count, unsigned *status, cudaStream_t st)
 {
     if (n == 0) return cudaMemsetAsync(cand_count, 0, sizeof(int64_t), st);
-    const int64_t n_chunks = (n + kRiskChunk - 1) / kRiskChunk;
+    const int64_t n_steps = (n + (1 << kStepShift) - 1) >> kStepShift;
     const int64_t n_words = (n + 31) >> 5;
-    const unsigned parity = (*sl.epoch)++ & 1u;
-    unsigned *totals = sl.group_totals + parity * sl.max_groups;
-    unsigned *next_totals = sl.group_totals + (parity ^ 1u) * sl.max_groups;
-    int64_t blocks = (n_chunks + kRiskWarps - 1) / kRiskWarps;
-    const int64_t cap = (int64_t)n_sm * 8;
-    if (blocks > cap) blocks = cap;
+    int64_t blocks = scan_grid(n_steps, dev, n_sm);
+    if (blocks > kMaxScanCtas) blocks = kMaxScanCtas;
     cudaError_t e;
     {
         LaunchTimer timer(timing_ctx, GS_K_RISK_FLAGS, st);
         risk_flags_kernel<<<(unsigned)blocks, kRiskThreads, 0, st>>>(
             assigned, generated, pred_len, elapsed, slo, n, inst.type_id, inst.decode_batch, inst.n_instances,
-            types.tpot_a_ms, types.tpot_b_ms, types.n_types, flag_bits, sl.chunk_counts, totals, n_chunks, status);
+            types.tpot_a_ms, types.tpot_b_ms, types.n_types, flag_bits, cta_counts, n_steps, status);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     {
-        const int64_t warps = blocks * kRiskWarps;
-        const int64_t chunks_per_warp = (n_chunks + warps - 1) / warps;
         LaunchTimer timer(timing_ctx, GS_K_RISK_SCATTER, st);
-        scatter_candidates_kernel<<<(unsigned)blocks, kRiskThreads, 0, st>>>(
-            flag_bits, n_words, sl.chunk_counts, totals, next_totals, sl.dirty[parity ^ 1u], n_chunks,
-            chunks_per_warp, cand_idx, cand_capacity, cand_count, status);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks);           // the same runs of steps as pass 1
+        cfg.blockDim = dim3(kRiskThreads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = GS_RISK_PDL ? 1 : 0;
+        e = cudaLaunchKernelEx(&cfg, scatter_candidates_kernel, (const uint32_t *)flag_bits, n_words,
+                               (const unsigned *)cta_counts, n_steps, cand_idx, cand_capacity, cand_count, status);
+        if (e != cudaSuccess) return e;
     }
-    sl.dirty[parity] = (n_chunks + (1 << kGroupShift) - 1) >> kGroupShift;
-    sl.dirty[parity ^ 1u] = 0;
     return cudaSuccess;
 }
 
@@ -220,25 +359,20 @@ cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *gen
                         uint32_t *flag_bits, int32_t *cand_idx, int64_t cand_capacity,
                         int64_t *cand_count, cudaStream_t st)
 {
-    ScanLaunch sl{ctx->s.chunk_counts, ctx->s.group_totals, ctx->max_groups, &ctx->scan_epoch, ctx->scan_dirty};
-    return enqueue_scan(sl, ctx->n_sm, ctx, assigned, generated, pred_len, elapsed, slo, n, inst, types,
-                        flag_bits, cand_idx, cand_capacity, cand_count, ctx->s.status, st);
+    return enqueue_scan(ctx->s.scan_counts, ctx->device, ctx->n_sm, ctx, assigned, generated, pred_len, elapsed, slo, n,
+                        inst, types, flag_bits, cand_idx, cand_capacity, cand_count, ctx->s.status, st);
 }
 
 // ---------------------------------------------------------------------------------------
 // gs_risk_scan_noalloc: the same scan for callers that cannot allocate device memory
 // ---------------------------------------------------------------------------------------
 
-constexpr size_t kNoAllocChunks = (GS_NOALLOC_MAX_ACTIVE + kRiskChunk - 1) / kRiskChunk;
-constexpr size_t kNoAllocGroups = (kNoAllocChunks + (1u << kGroupShift) - 1) >> kGroupShift;
-
-// All scratch of the no-allocation entry point.  It lives in the library image: every GPU
-// that loads the library holds these 66 KB until the process exits.  Zero-initialised.  The
-// chunk counts are rewritten by every call before they are read; of the two group-total
-// buffers each call adds into one (cleared by the call before it) and clears the other.
+// All scratch of the no-allocation entry point: the per-CTA flag counts that the scan's two
+// passes exchange, and a status word.  It lives in the library image: every GPU that loads the
+// library holds these 16 KB until the process exits.  Every call stores each count before it
+// reads it, so nothing a call computes depends on what an earlier call left here.
 struct NoAllocScratch {
-    unsigned chunk_counts[kNoAllocChunks];
-    unsigned group_totals[2 * kNoAllocGroups];
+    unsigned cta_counts[kMaxScanCtas];
     unsigned status;
 };
 static __device__ __align__(256) NoAllocScratch g_noalloc_scratch;
@@ -249,14 +383,11 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 // Per GPU: the device address of g_noalloc_scratch, resolved on that GPU's first call (in host
-// code the symbol's name is only a handle, never an address a kernel may use), and the host
-// side of the scan's bookkeeping.
+// code the symbol's name is only a handle, never an address a kernel may use).
 struct NoAllocDevice {
     gs::NoAllocScratch *ptr = nullptr;
     cudaError_t err = cudaSuccess;
     bool ready = false;
-    unsigned epoch = 0;
-    int64_t dirty[2] = {0, 0};
 };
 NoAllocDevice g_noalloc[kMaxDevices];
 std::mutex g_noalloc_mutex;     // guards g_noalloc
@@ -298,8 +429,7 @@ extern "C" GS_API int gs_risk_scan_noalloc(
     NoAllocScratch *sc = nd.ptr;
     int n_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1) n_sm = 148;
-    ScanLaunch sl{sc->chunk_counts, sc->group_totals, kNoAllocGroups, &nd.epoch, nd.dirty};
-    const cudaError_t e = enqueue_scan(sl, n_sm, nullptr, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms,
+    const cudaError_t e = enqueue_scan(sc->cta_counts, dev, n_sm, nullptr, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms,
                                        n_active, *inst, *types, out_flag_bits, out_cand_idx, cand_capacity,
                                        out_cand_count, out_status_bits ? out_status_bits : &sc->status,
                                        (cudaStream_t)cuda_stream);

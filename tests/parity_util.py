@@ -140,9 +140,7 @@ def check_route_against_f64(got: GpuRoute, tab64, req, max_explain=5):
         g = int(got.instance_idx[r])
         order = np.arange(len(T))
         preferred = (tab64.d > tab64.d[g]) | ((tab64.d == tab64.d[g]) & (order < g))
-        # d_g itself is rounded differently in the two precisions: equal-within-rounding d also ties
-        close_d = np.abs(tab64.d - tab64.d[g]) <= 1e-6 * np.abs(tab64.d[g])
-        tier1_ok = maybe[g] and not (definitely & preferred & ~close_d).any()
+        tier1_ok = maybe[g] and not (definitely & preferred).any()
         pool = ok if ok.any() else np.ones_like(ok)
         tmin = T[pool].min()
         fb_ok = (not definitely.any()) and pool[g] and (T[g] - tmin) <= REL_TOL * abs(tmin)
