@@ -261,7 +261,7 @@ GS_API int gs_route_batch(gs_ctx *ctx, const int32_t *prompt_len, const int32_t 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, types->n_types,
+    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, inst->n_instances, types->n_types,
                          out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier,
                          (flags & GS_ROUTE_ACCUMULATE) != 0, false, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
@@ -293,7 +293,7 @@ GS_API int gs_route_batch_prefix(gs_ctx *ctx, const int32_t *prompt_len, const i
     cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     const gs::PrefixHits hits = {prefix_inst, prefix_hit_len, n_slots, slot_stride};
-    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, &hits, types->n_types,
+    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, &hits, inst->n_instances, types->n_types,
                          out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, false, false, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
@@ -337,7 +337,7 @@ GS_API int gs_route_batch_direct(gs_ctx *ctx, const int32_t *prompt_len, const i
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = gs::launch_prologue_direct(ctx, *table, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, gs::kDirectGroups,
+    e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, table->n_instances, gs::kDirectGroups,
                          out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, false, true, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }

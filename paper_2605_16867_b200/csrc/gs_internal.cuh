@@ -32,6 +32,12 @@ __host__ __device__ __forceinline__ int row_slot(int i) {
     return (group << 3) | (((pair ^ ((group >> 1) & 3)) << 1) | (i & 1));
 }
 
+// Where the exact coefficients of instance g sit in the table `rows` (in global memory and in its
+// shared-memory copies).  Lanes often ask for instances a fixed stride apart (all of one GPU type
+// when types are dealt round robin); the low bits are mixed with the next ones so that such lanes
+// spread over the shared-memory banks.  A permutation inside every aligned block of eight.
+__host__ __device__ __forceinline__ int row_pos(int g) { return g ^ (((g >> 3) ^ (g >> 6)) & 7); }
+
 constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low bits of a q word
 // groups of similar p that stand in for GPU types when the coefficients are given per instance
 #ifndef GS_DIRECT_GROUPS
@@ -84,7 +90,7 @@ constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 
 // Device scratch owned by a context.
 struct Scratch {
-    Row *rows;                // [max_instances] exact coefficients, caller order
+    Row *rows;                // [GS_MAX_INSTANCES] exact coefficients, instance g at row_pos(g)
     uint2 *row_bounds;        // [kMaxPaddedRows]
     float2 *group_bounds;     // [kMaxPaddedRows / 8] per eight rows: {least q word as a float, d_lo of the last row}; +inf, 0 = padding only
     float *row_p;             // [kMaxPaddedRows] lower bound of each row's p, in row order (unswizzled)
@@ -158,7 +164,7 @@ cudaError_t launch_ema(gs_ctx *ctx, float alpha, int M, const float *obs_q, cons
                        float *q, float *p, float *d, cudaStream_t st);
 cudaError_t launch_prologue_direct(gs_ctx *ctx, const gs_instance_table &tab, cudaStream_t st);
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
-                         const float *slo_ms, int64_t n, const PrefixHits *hits, int n_types,
+                         const float *slo_ms, int64_t n, const PrefixHits *hits, int n_instances, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, bool row_p, cudaStream_t st);
 cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,

@@ -33,6 +33,7 @@ namespace gs {
 
 constexpr int kPrologueThreads = GS_MAX_INSTANCES;      // one thread per instance
 constexpr int kPmFloats = 8192;                         // shared-memory floats for the running minima
+constexpr int kCountSortMax = 256;                      // a group of up to this many rows is ranked by counting
 
 __device__ __forceinline__ int clamp_count(int v, unsigned &bad) {
     if (v < 0) { bad |= GS_DEV_BAD_VALUE; return 0; }
@@ -56,7 +57,8 @@ __device__ __forceinline__ float bucket_upper_edge(int b) {
 constexpr unsigned kPadQ = 0x7FC00000u;                 // NaN: compares false with everything
 
 // Entries of the record-list pool that a type with n of the pool's M instances may use.
-__device__ __forceinline__ int pool_share_of(int n, int M) { return (int)(((long long)kPoolEntries * n) / M) & ~3; }
+// (kPoolEntries * n <= 2^23: plain 32-bit arithmetic)
+__device__ __forceinline__ int pool_share_of(int n, int M) { return (int)((unsigned)(kPoolEntries * n) / (unsigned)M) & ~3; }
 
 // Bit pattern of a lower bound of v >= 0 whose low tag bits are zero and may be overwritten.
 __device__ __forceinline__ unsigned lower_bound_bits(float v) {
@@ -68,22 +70,23 @@ __device__ __forceinline__ unsigned lower_bound_bits(float v) {
 __device__ __forceinline__ float lower_bound(float v) { return __fmul_rn(v, kShrink); }
 
 // Bitonic sort of one 64-bit key per thread over the first n_sort threads' keys (n_sort a power
-// of two >= 32; all kPrologueThreads threads call it).  Partners closer than a warp exchange by
-// shuffle, farther ones through shared memory (two buffers, so one barrier per exchange).
-// Returns the key of rank tid.
+// of two >= 32; all kPrologueThreads threads call it, the warps beyond n_sort only meet the
+// barriers).  Partners closer than a warp exchange by shuffle, farther ones through shared
+// memory (two buffers, so one barrier per exchange).  Returns the key of rank tid (tid < n_sort).
 __device__ __forceinline__ unsigned long long bitonic_sort(unsigned long long key, int n_sort, int tid,
                                                            unsigned long long (*sh_xchg)[GS_MAX_INSTANCES])
 {
     int buf = 0;
+    const bool works = tid < n_sort;            // whole warps: n_sort is a multiple of 32
     for (int k = 2; k <= n_sort; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
-            unsigned long long other;
+            unsigned long long other = key;
             if (j >= 32) {
-                sh_xchg[buf][tid] = key;
+                if (works) sh_xchg[buf][tid] = key;
                 __syncthreads();
-                other = sh_xchg[buf][tid ^ j];
+                if (works) other = sh_xchg[buf][tid ^ j];
                 buf ^= 1;
-            } else {
+            } else if (works) {
                 other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
             }
             const bool keep_min = ((tid & k) == 0) == ((tid & j) == 0);
@@ -112,14 +115,15 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 const float *__restrict__ b_type, int n_types, float alpha,
                 Scratch s)
 {
-    __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];                // my group's rows, sorted
+    __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];                // my group's rows as collected
+    __shared__ unsigned long long sh_sorted[GS_MAX_INSTANCES];             // ... in preference order
     extern __shared__ unsigned long long sh_dyn[];                        // sort exchange buffers, then running minima
     unsigned long long (*sh_xchg)[GS_MAX_INSTANCES] = reinterpret_cast<unsigned long long (*)[GS_MAX_INSTANCES]>(sh_dyn);
     __shared__ float sh_q[GS_MAX_INSTANCES], sh_d[GS_MAX_INSTANCES];       // by instance index
     __shared__ float sh_p[kDirect ? GS_MAX_INSTANCES : 1];                 // kDirect: p by instance index
     __shared__ unsigned char sh_t[kDirect ? 1 : GS_MAX_INSTANCES];
     __shared__ float sh_rq[GS_MAX_INSTANCES], sh_rd[GS_MAX_INSTANCES];     // my rows: q_lo (tagged), d_lo
-    __shared__ int sh_cnt[GS_MAX_TYPES], sh_rank[GS_MAX_TYPES];
+    __shared__ int sh_cnt[GS_MAX_TYPES], sh_plan[8];
     __shared__ unsigned sh_dmax[GS_MAX_TYPES], sh_dmin[GS_MAX_TYPES];      // by type: largest / least d
     __shared__ unsigned sh_dlow_pos[GS_MAX_TYPES];                         // least d by position in the search order
     __shared__ unsigned sh_qmin, sh_pmin;
@@ -127,17 +131,30 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     __shared__ int sh_unsafe, sh_fill;
     __shared__ int sh_len[kPrologueThreads / 32], sh_off[kPrologueThreads / 32], sh_pool_used;
 
+    // the kernel that follows in the stream (the routing round) may be set up from now on; it
+    // waits for this whole grid before it reads a table
+    asm volatile("griddepcontrol.launch_dependents;");
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
     const bool writer = blockIdx.x == 0;       // one CTA writes what does not depend on the group
     const int tr = blockIdx.x;                 // position of this CTA's group in the search order
     unsigned bad = 0;
+    const bool has = tid < M;
+    // typed pools: all global loads are issued before anything else is done
+    int r_type = 0, r_queued = 0, r_batch = 0, r_kv = 0;
+    float r_qema = 0.f;
+    if (!kDirect) {
+        if (has) {
+            r_type = type_id[tid]; r_queued = queued[tid]; r_batch = batch[tid];
+            r_kv = free_kv[tid]; r_qema = q_ema[tid];
+        }
+        if (tid < n_types) { sh_tp[tid] = p_type[tid]; sh_ta[tid] = a_type[tid]; sh_tb[tid] = b_type[tid]; }
+    }
     if (tid < GS_MAX_TYPES) { sh_cnt[tid] = 0; sh_dmax[tid] = 0u; sh_dmin[tid] = 0xFFFFFFFFu; }
     if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; sh_pmin = 0xFFFFFFFFu; }
     __syncthreads();
 
-    const bool has = tid < M;
     int base = 0, n_act = 0, padded_total = 0, n_t = 0;
     int pool_base = 0, pool_share = 0, pool_total = 0;     // record lists: this type's part of the pool
     float p_group = 0.f;                       // lower bound source: the least p of the group
@@ -157,7 +174,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             sh_q[tid] = q; sh_d[tid] = d; sh_p[tid] = pv;
             if (writer) {
                 Row row; row.q = q; row.p = pv; row.d = d; row.kv = kv;
-                s.rows[tid] = row;
+                s.rows[row_pos(tid)] = row;
                 s.d_by_g[tid] = d;
                 s.q_by_g[tid] = q;
             }
@@ -180,7 +197,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         // the least d of every group: that of its last row (tid = rank here)
         if (has && (tid == M - 1 || (tid + 1) % group_rows == 0)) sh_dlow_pos[tid / group_rows] = ~(unsigned)(key >> 16);
         const bool mine = tr < n_act && tid >= base && tid < base + n_t;
-        if (mine) sh_key[tid - base] = key;
+        if (mine) sh_sorted[tid - base] = key;
         const unsigned pb = mine ? (__float_as_uint(sh_p[(int)(key & 0xFFFFull)]) & 0x7FFFFFFFu) : 0xFFFFFFFFu;
         const unsigned wmin = __reduce_min_sync(0xFFFFFFFFu, pb);   // non-negative floats order like their bits
         if (lane == 0 && wmin != 0xFFFFFFFFu) atomicMin(&sh_pmin, wmin);
@@ -188,15 +205,6 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         p_group = __uint_as_float(sh_pmin);
     } else {
         // ---- 1. coefficients of every instance (thread g owns instance g) ----------------------
-        // all global loads are issued before anything depends on them
-        int r_type = 0, r_queued = 0, r_batch = 0, r_kv = 0;
-        float r_qema = 0.f;
-        if (has) {
-            r_type = type_id[tid]; r_queued = queued[tid]; r_batch = batch[tid];
-            r_kv = free_kv[tid]; r_qema = q_ema[tid];
-        }
-        if (tid < n_types) { sh_tp[tid] = p_type[tid]; sh_ta[tid] = a_type[tid]; sh_tb[tid] = b_type[tid]; }
-        __syncthreads();
         {
             int t = r_type;
             if (has && (t < 0 || t >= n_types)) { bad |= GS_DEV_BAD_TYPE; t = 0; }
@@ -216,7 +224,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 sh_q[tid] = q; sh_d[tid] = d; sh_t[tid] = (unsigned char)t;
                 if (writer) {
                     Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
-                    s.rows[tid] = row;
+                    s.rows[row_pos(tid)] = row;
                     s.d_by_g[tid] = d;
                     s.q_by_g[tid] = q;
                 }
@@ -224,43 +232,64 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 const float big = 3.0e38f;
                 if (!(q >= 0.f && q < big && p >= 0.f && p < big && d >= 0.f && d < big)) atomicOr(&sh_unsafe, 1);
             }
-            // instances per type and each type's largest d: one shared-memory atomic per type and warp
-            const unsigned peers = __match_any_sync(0xFFFFFFFFu, t);
-            const unsigned dmax = __reduce_max_sync(peers, orderable(d));
-            const unsigned dmin = __reduce_min_sync(peers, orderable(d));
-            if (t >= 0 && lane == __ffs(peers) - 1) {
-                atomicAdd(&sh_cnt[t], __popc(peers));
-                atomicMax(&sh_dmax[t], dmax);
-                atomicMin(&sh_dmin[t], dmin);
+            // instances per type and each type's largest and least d: the warp goes through the
+            // types together (no divergence), lane o keeps type o's figures and adds them to the
+            // CTA's with one shared-memory atomic each
+            const unsigned od = orderable(d);
+            int w_cnt = 0;
+            unsigned w_max = 0u, w_min = 0xFFFFFFFFu;
+            for (int o = 0; o < n_types; ++o) {
+                const bool is = t == o;
+                const int c = __popc(__ballot_sync(0xFFFFFFFFu, is));
+                const unsigned mx = __reduce_max_sync(0xFFFFFFFFu, is ? od : 0u);
+                const unsigned mn = __reduce_min_sync(0xFFFFFFFFu, is ? od : 0xFFFFFFFFu);
+                if (lane == o) { w_cnt = c; w_max = mx; w_min = mn; }
+            }
+            if (w_cnt > 0) {
+                atomicAdd(&sh_cnt[lane], w_cnt);
+                atomicMax(&sh_dmax[lane], w_max);
+                atomicMin(&sh_dmin[lane], w_min);
             }
         }
         __syncthreads();
 
         // ---- 2. order of the types (largest d first; ties: smaller type id) --------------------
-        if (tid < GS_MAX_TYPES) {
-            int rank = GS_MAX_TYPES;           // unused types sort last
-            if (sh_cnt[tid] > 0) {
-                rank = 0;
-                for (int o = 0; o < GS_MAX_TYPES; ++o)
-                    if (sh_cnt[o] > 0 && (sh_dmax[o] > sh_dmax[tid] || (sh_dmax[o] == sh_dmax[tid] && o < tid))) ++rank;
+        // One warp works it out, lane o for type o, and leaves the CTA's plan in shared memory.
+        if (warp == 0) {
+            const bool is_type = lane < GS_MAX_TYPES;
+            const int cnt_o = is_type ? sh_cnt[lane] : 0;
+            const unsigned dmax_o = is_type ? sh_dmax[lane] : 0u;
+            int rank_o = 0;
+#pragma unroll
+            for (int k = 0; k < GS_MAX_TYPES; ++k) {
+                const int cnt_k = __shfl_sync(0xFFFFFFFFu, cnt_o, k);
+                const unsigned dmax_k = __shfl_sync(0xFFFFFFFFu, dmax_o, k);
+                if (cnt_k > 0 && (dmax_k > dmax_o || (dmax_k == dmax_o && k < lane))) ++rank_o;
             }
-            sh_rank[tid] = rank;
-            if (rank < GS_MAX_TYPES) sh_dlow_pos[rank] = sh_dmin[tid];
+            if (cnt_o == 0) rank_o = GS_MAX_TYPES;              // unused types sort last
+            const int padded_o = cnt_o > 0 ? (cnt_o + 15) & ~15 : 0;
+            const int share_o = cnt_o > 0 ? pool_share_of(cnt_o, M) : 0;
+            if (cnt_o > 0) sh_dlow_pos[rank_o] = sh_dmin[lane];
+            const int v_act = __popc(__ballot_sync(0xFFFFFFFFu, cnt_o > 0));
+            const int v_padded = __reduce_add_sync(0xFFFFFFFFu, padded_o);
+            const int v_pool = __reduce_add_sync(0xFFFFFFFFu, share_o);
+            const int v_base = __reduce_add_sync(0xFFFFFFFFu, rank_o < tr ? padded_o : 0);
+            const int v_pool_base = __reduce_add_sync(0xFFFFFFFFu, rank_o < tr ? share_o : 0);
+            // the type this CTA builds: the one at position tr of the order
+            const unsigned at_tr = __ballot_sync(0xFFFFFFFFu, cnt_o > 0 && rank_o == tr);
+            const int v_type = at_tr ? __ffs(at_tr) - 1 : -1;
+            const int v_nt = __shfl_sync(0xFFFFFFFFu, cnt_o, v_type < 0 ? 0 : v_type);
+            const int v_share = __shfl_sync(0xFFFFFFFFu, share_o, v_type < 0 ? 0 : v_type);
+            if (lane == 0) {
+                sh_plan[0] = v_type; sh_plan[1] = v_type < 0 ? 0 : v_nt; sh_plan[2] = v_type < 0 ? 0 : v_share;
+                sh_plan[3] = v_act; sh_plan[4] = v_padded; sh_plan[5] = v_pool; sh_plan[6] = v_base; sh_plan[7] = v_pool_base;
+            }
         }
         __syncthreads();
-        // the type this CTA builds, the padded rows before it, the number of types in use
-        int my_type = -1;
-        for (int o = 0; o < GS_MAX_TYPES; ++o) {
-            const int r = sh_rank[o], n = sh_cnt[o];
-            if (n == 0) continue;
-            ++n_act;
-            padded_total += (n + 15) & ~15;
-            if (r == tr) { my_type = o; pool_share = pool_share_of(n, M); }
-            if (r < tr) { base += (n + 15) & ~15; pool_base += pool_share_of(n, M); }
-            pool_total += pool_share_of(n, M);
-        }
+        const int my_type = sh_plan[0];
+        n_t = sh_plan[1]; pool_share = sh_plan[2]; n_act = sh_plan[3]; padded_total = sh_plan[4];
+        pool_total = sh_plan[5]; base = sh_plan[6]; pool_base = sh_plan[7];
         if (my_type >= 0) {
-            n_t = sh_cnt[my_type];
             p_group = sh_tp[my_type];
             // ---- 3. collect this type's rows and sort them by (d descending, index ascending) ---
             // (one shared-memory atomic per warp; the order inside the list does not matter yet)
@@ -272,11 +301,25 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             if (mine) sh_key[at] = ((unsigned long long)(~orderable(sh_d[tid])) << 16) | (unsigned)tid;
         }
         __syncthreads();
-        if (my_type >= 0) {                    // (uniform over the CTA)
+        if (my_type >= 0 && n_t <= kCountSortMax) {
+            // Rank by counting: the keys are distinct (the index is part of them), so a row's place
+            // is the number of keys below its own.  n_pow^2 / 1024 compares per thread, P threads
+            // per row (consecutive lanes take consecutive keys: no bank conflicts), no barrier
+            // until the places are known.
+            int n_pow = 32;
+            while (n_pow < n_t) n_pow <<= 1;
+            const int P = kPrologueThreads / n_pow;             // 4 .. 32 threads per row
+            const int i = tid / P, part = tid % P;
+            const unsigned long long key_i = i < n_t ? sh_key[i] : 0ull;
+            int below_i = 0;
+            for (int j = part; j < n_t; j += P) below_i += sh_key[j] < key_i ? 1 : 0;
+            for (int off = P >> 1; off > 0; off >>= 1) below_i += __shfl_xor_sync(0xFFFFFFFFu, below_i, off);
+            if (part == 0 && i < n_t) sh_sorted[below_i] = key_i;    // (published by the barrier further down)
+        } else if (my_type >= 0) {             // (uniform over the CTA)
             int n_sort = 32;
             while (n_sort < n_t) n_sort <<= 1;
             const unsigned long long key = bitonic_sort(tid < n_t ? sh_key[tid] : ~0ull, n_sort, tid, sh_xchg);
-            sh_key[tid] = key;
+            sh_sorted[tid] = key;
         }
     }
     if (writer && tid == 0) {
@@ -319,7 +362,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     for (int k = tid; k < n_padded; k += kPrologueThreads) {
         uint2 entry = make_uint2(kPadQ, 0u);
         if (k < n_t) {
-            const int inst = (int)(sh_key[k] & 0xFFFFull);
+            const int inst = (int)(sh_sorted[k] & 0xFFFFull);
             // the tag rides on q: d multiplies L_out, so its bound is kept at full precision
             const unsigned q_bits = lower_bound_bits(sh_q[inst]);
             const float d_lo = lower_bound(sh_d[inst]);
@@ -329,14 +372,15 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             my_qmin = min(my_qmin, q_bits);             // non-negative floats order like their bits
         }
         s.row_bounds[row_slot(base + k)] = entry;
-        if (kDirect) s.row_p[base + k] = k < n_t ? lower_bound(sh_p[(int)(sh_key[k] & 0xFFFFull)]) : 0.f;
+        if (kDirect) s.row_p[base + k] = k < n_t ? lower_bound(sh_p[(int)(sh_sorted[k] & 0xFFFFull)]) : 0.f;
     }
     my_qmin = __reduce_min_sync(0xFFFFFFFFu, my_qmin);
     if (lane == 0) atomicMin(&sh_qmin, my_qmin);
     __syncthreads();
 
     // bounds over every eight rows (the fallback's search skips a group whole with them)
-    for (int g = tid; g < n_padded / 8; g += kPrologueThreads) {
+    for (int g = tid - 64; g < n_padded / 8; g += kPrologueThreads - 64) {   // (warps 0 and 1 have other work below)
+        if (g < 0) break;
         float q_least = __int_as_float(0x7F800000);         // +inf: a group of padding only
         float d_last = 0.f;
         for (int k = 8 * g; k < 8 * g + 8 && k < n_t; ++k) { q_least = fminf(q_least, sh_rq[k]); d_last = sh_rd[k]; }
@@ -348,8 +392,8 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     const float d_hi = sh_rd[0], d_low = sh_rd[n_t - 1];
     float inv_w = 0.f;              // slots per unit of d; 0 = no start table (search from row 0)
     if (n_t > 4 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f)) inv_w = (float)kStartSlots / (d_hi - d_low);
-    if (tid == 0) {
-        const int first_inst = (int)(sh_key[0] & 0xFFFFull);
+    if (tid == 32) {
+        const int first_inst = (int)(sh_sorted[0] & 0xFFFFull);
         TypeHeader h;
         h.p_lo = __fmul_rn(p_group, kShrink);
         h.q_lo = q0;
@@ -384,7 +428,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         if (per_batch > kPrologueThreads / 32) per_batch = kPrologueThreads / 32;   // one warp per bucket
         if (per_batch > kStartBuckets) per_batch = kStartBuckets;
         if (tid == 0) sh_pool_used = 0;
-        __syncthreads();                                    // the sort is done with sh_dyn
+        if (kDirect || n_t > kCountSortMax) __syncthreads();       // the bitonic sort is done with sh_dyn
         for (int b0 = 0; b0 < kStartBuckets; b0 += per_batch) {
             const bool my_bucket = warp < per_batch && b0 + warp < kStartBuckets;
             if (my_bucket) {
@@ -441,23 +485,10 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 __syncwarp();
                 if (lane == 0) sh_pool_used = used + used_now;
             }
-            __syncthreads();
-            if (my_bucket && !kDirect) {
-                const int off = sh_off[warp], len = sh_len[warp];
-                if (off >= 0) {
-                    const unsigned short *pc = sh_pc + warp * n_t;
-                    for (int k = lane; k < n_t; k += 32) {
-                        const int c = pc[k], c_next = k + 1 < n_t ? pc[k + 1] : len;
-                        if (c_next != c)
-                            s.pool[off + c] = make_uint2(__float_as_uint(sh_rq[k]), __float_as_uint(sh_rd[k]));
-                    }
-                    for (int k = len + lane; k < ((len + kListWindow + 1) & ~1); k += 32)
-                        s.pool[off + k] = make_uint2(kPadQ, 0u);
-                }
-                if (lane == 0)
-                    s.bucket_list[tr * kStartBuckets + b0 + warp] = off >= 0 ? (unsigned short)(off >> 1) : kNoList;
-            }
-            for (int c = tid; c < per_batch * kStartSlots; c += kPrologueThreads) {
+            // (the cells below need the running minima and record counts only, not the pool
+            // offsets that warp 0 has just worked out: no barrier in between)
+            for (int c = tid - 32; c < per_batch * kStartSlots; c += kPrologueThreads - 32) {
+                if (c < 0) break;                           // warp 0 is busy with the pool
                 const int bw = c / kStartSlots, slot = c % kStartSlots, b = b0 + bw;
                 if (b >= kStartBuckets) break;
                 int lo = 0;                                 // rows [0, lo) cannot pass
@@ -481,6 +512,22 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 }
             }
             __syncthreads();
+            if (my_bucket && !kDirect) {
+                const int off = sh_off[warp], len = sh_len[warp];
+                if (off >= 0) {
+                    const unsigned short *pc = sh_pc + warp * n_t;
+                    for (int k = lane; k < n_t; k += 32) {
+                        const int c = pc[k], c_next = k + 1 < n_t ? pc[k + 1] : len;
+                        if (c_next != c)
+                            s.pool[off + c] = make_uint2(__float_as_uint(sh_rq[k]), __float_as_uint(sh_rd[k]));
+                    }
+                    for (int k = len + lane; k < ((len + kListWindow + 1) & ~1); k += 32)
+                        s.pool[off + k] = make_uint2(kPadQ, 0u);
+                }
+                if (lane == 0)
+                    s.bucket_list[tr * kStartBuckets + b0 + warp] = off >= 0 ? (unsigned short)(off >> 1) : kNoList;
+            }
+            if (b0 + per_batch < kStartBuckets) __syncthreads();     // the next batch writes the same shared arrays
         }
     }
 }

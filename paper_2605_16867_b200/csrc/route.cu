@@ -44,11 +44,6 @@ __host__ __device__ constexpr int route_threads(bool row_p, int req = 4) {
 }
 constexpr int64_t kSmallBatch = 1 << 21;        // below this many requests: one per lane
 
-// Where the exact coefficients of instance g sit in the shared-memory copy of the table.  Lanes
-// often ask for instances a fixed stride apart (all of one GPU type when types are dealt round
-// robin); the low bits are mixed with the next ones so that such lanes spread over the banks.
-__device__ __forceinline__ int row_pos(int g) { return g ^ (((g >> 3) ^ (g >> 6)) & 7); }
-
 // T(r,g) of Eq. 2 with H = 0, each step rounded once.
 __device__ __forceinline__ float latency(const Row &r, float x, float y) {
     return __fmaf_rn(r.d, y, __fmaf_rn(r.p, x, r.q));
@@ -323,7 +318,7 @@ __device__ __forceinline__ unsigned char *stage_tables(unsigned char *smem, int 
     uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
     float2 *sh_group_bounds = reinterpret_cast<float2 *>(sh_row_bounds + kMaxPaddedRows);
     unsigned char *sh_start = reinterpret_cast<unsigned char *>(sh_group_bounds + kMaxPaddedRows / 8);
-    for (int k = threadIdx.x; k < M; k += blockDim.x) sh_rows[row_pos(k)] = g_rows[k];
+    for (int k = threadIdx.x; k < ((M + 7) & ~7); k += blockDim.x) sh_rows[k] = g_rows[k];   // (stored position-mixed: row_pos)
     for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
     for (int k = threadIdx.x; k < n_padded / 8; k += blockDim.x) sh_group_bounds[k] = g_group_bounds[k];
     for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
@@ -395,6 +390,58 @@ __device__ __forceinline__ void exhaustive_pick(const Row *rows, int M, float xs
 // ---------------------------------------------------------------------------------------
 // the routing round
 // ---------------------------------------------------------------------------------------
+
+// Bulk asynchronous copies (global -> this CTA's shared memory, this GPU's memory only, no
+// multicast) that report to an mbarrier.  Addresses and sizes are multiples of 16 bytes.
+__device__ __forceinline__ unsigned shared_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void bulk_copy_to_shared(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(shared_addr(dst)), "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(shared_addr(bar)) : "memory");
+}
+
+// Waits for phase `parity` of the barrier, at most kBarrierTries tries (each try itself gives up
+// after a hardware time limit): a wait that cannot end turns into `false`, never into a hang.
+constexpr int kBarrierTries = 1 << 20;
+__device__ __forceinline__ bool wait_barrier(unsigned long long *bar, unsigned parity) {
+    unsigned done = 0;
+    for (int it = 0; it < kBarrierTries && !done; ++it)
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(shared_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+
+// Shared-memory image of the round's tables for the route kernel, in the order it is carved.
+struct TableImage {
+    Row *rows; TypeHeader *headers; uint2 *row_bounds; float2 *group_bounds; unsigned char *start_table;
+    unsigned short *cand; unsigned char *start_list; unsigned short *bucket_list; uint2 *pool; float *row_p;
+    int *info; unsigned long long *bar; unsigned char *end;
+};
+
+template <bool kRowP>
+__device__ __forceinline__ TableImage carve_tables(unsigned char *smem, int n_types_alloc) {
+    TableImage im;
+    im.rows = reinterpret_cast<Row *>(smem);
+    im.headers = reinterpret_cast<TypeHeader *>(im.rows + GS_MAX_INSTANCES);
+    im.row_bounds = reinterpret_cast<uint2 *>(im.headers + GS_MAX_TYPES);
+    im.group_bounds = reinterpret_cast<float2 *>(im.row_bounds + kMaxPaddedRows);
+    im.start_table = reinterpret_cast<unsigned char *>(im.group_bounds + kMaxPaddedRows / 8);
+    unsigned char *at = im.start_table + (size_t)n_types_alloc * (kStartBuckets * kStartSlots);
+    im.row_p = nullptr; im.start_list = nullptr; im.bucket_list = nullptr; im.pool = nullptr;
+    if (kRowP) {
+        im.row_p = reinterpret_cast<float *>(at); at += kMaxPaddedRows * sizeof(float);
+    }
+    im.cand = reinterpret_cast<unsigned short *>(at); at += kCandSlots * sizeof(unsigned short);
+    if (!kRowP) {
+        im.start_list = at; at += (size_t)n_types_alloc * kStartBuckets * kStartSlots;
+        im.bucket_list = reinterpret_cast<unsigned short *>(at); at += (size_t)n_types_alloc * kStartBuckets * sizeof(unsigned short);
+        im.pool = reinterpret_cast<uint2 *>(at); at += (size_t)kPoolEntries * sizeof(uint2);
+    }
+    im.info = reinterpret_cast<int *>(at); at += 64;
+    im.bar = reinterpret_cast<unsigned long long *>(at); at += 16;
+    im.end = at;
+    return im;
+}
 
 // First row of the eight at padded index k (a multiple of 8) whose bound passes: its tag word
 // replaces `first`; rows are tested last to first so that the earliest one wins.
@@ -585,7 +632,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
              const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
              const unsigned short *__restrict__ g_cand, const uint2 *__restrict__ g_pool,
              const unsigned short *__restrict__ g_bucket_list, const unsigned char *__restrict__ g_start_list,
-             const float *__restrict__ g_row_p,
+             const float *__restrict__ g_row_p, int m_rows, int n_padded_max,
              int32_t *__restrict__ out_idx, float *__restrict__ out_est,
              float *__restrict__ out_slack, uint8_t *__restrict__ out_tier,
              unsigned long long *__restrict__ deltas, unsigned *__restrict__ status)
@@ -630,34 +677,46 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
 #pragma unroll
     for (int j = 0; j < kReqPerThread; ++j) { nx[j] = 0; ny[j] = 0; nd[j] = -1.0f; }
     if (wt0 < cta_end) load_tile(wt0, nx, ny, nd);           // under way while the tables are staged
-    const int M = table_info[2];
-    const float cand_z0 = __int_as_float(table_info[4]), cand_inv = __int_as_float(table_info[5]);
-    Tables tb;
-    unsigned char *after_tables = stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_group_bounds, g_start_table, g_headers,
-                                               table_info, tb, kRowP ? g_row_p : nullptr);
-    unsigned short *sh_cand = reinterpret_cast<unsigned short *>(after_tables);
-    if (threadIdx.x < kCandSlots) sh_cand[threadIdx.x] = g_cand[threadIdx.x];
-    tb.cand = sh_cand;
-    after_tables += kCandSlots * sizeof(unsigned short);
-    tb.pool = nullptr; tb.bucket_list = nullptr; tb.start_list = nullptr;
-    if (!kRowP) {                                  // record lists and their start table
-        const int n_act = table_info[3], pool_n = table_info[6];
-        uint4 *sh_start_list = reinterpret_cast<uint4 *>(after_tables);
-        for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
-            sh_start_list[k] = reinterpret_cast<const uint4 *>(g_start_list)[k];
-        after_tables += (size_t)n_types_alloc * kStartBuckets * kStartSlots;
-        uint4 *sh_bucket = reinterpret_cast<uint4 *>(after_tables);
-        for (int k = threadIdx.x; k < n_act * (kStartBuckets * (int)sizeof(unsigned short) / 16); k += blockDim.x)
-            sh_bucket[k] = reinterpret_cast<const uint4 *>(g_bucket_list)[k];
-        after_tables += (size_t)n_types_alloc * kStartBuckets * sizeof(unsigned short);
-        uint4 *sh_pool = reinterpret_cast<uint4 *>(after_tables);
-        for (int k = threadIdx.x; k < pool_n / 2; k += blockDim.x)
-            sh_pool[k] = reinterpret_cast<const uint4 *>(g_pool)[k];
-        after_tables += (size_t)kPoolEntries * sizeof(uint2);
-        tb.start_list = reinterpret_cast<const unsigned char *>(sh_start_list);
-        tb.bucket_list = reinterpret_cast<const unsigned short *>(sh_bucket);
-        tb.pool = reinterpret_cast<const uint2 *>(sh_pool);
+    // The kernel is launched as a programmatic dependent of the prologue: everything above ran
+    // beside it; the tables may be read once that whole grid is done and its stores are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // The tables come in by bulk asynchronous copies, all in flight together, one barrier for
+    // all of them.  The sizes are upper bounds that the host knows (what lies beyond the round's
+    // own entries is never looked at); the few numbers that only the prologue knows are copied
+    // along (info).
+    const TableImage im = carve_tables<kRowP>(smem, n_types_alloc);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(shared_addr(im.bar)) : "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned b_rows = (unsigned)m_rows * sizeof(Row), b_headers = (unsigned)n_types_alloc * sizeof(TypeHeader);
+        const unsigned b_bounds = (unsigned)n_padded_max * sizeof(uint2), b_groups = (unsigned)n_padded_max / 8 * sizeof(float2);
+        const unsigned b_start = (unsigned)n_types_alloc * (kStartBuckets * kStartSlots);
+        const unsigned b_cand = kCandSlots * sizeof(unsigned short), b_info = 64u;
+        const unsigned b_rowp = kRowP ? (unsigned)n_padded_max * sizeof(float) : 0u;
+        const unsigned b_bucket = kRowP ? 0u : (unsigned)n_types_alloc * kStartBuckets * sizeof(unsigned short);
+        const unsigned b_pool = kRowP ? 0u : (unsigned)kPoolEntries * sizeof(uint2);
+        const unsigned total = b_rows + b_headers + b_bounds + b_groups + b_start + b_cand + b_info + b_rowp +
+                               (kRowP ? 0u : b_start) + b_bucket + b_pool;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(shared_addr(im.bar)), "r"(total) : "memory");
+        bulk_copy_to_shared(im.info, table_info, b_info, im.bar);
+        bulk_copy_to_shared(im.cand, g_cand, b_cand, im.bar);
+        bulk_copy_to_shared(im.headers, g_headers, b_headers, im.bar);
+        bulk_copy_to_shared(im.rows, g_rows, b_rows, im.bar);
+        if (kRowP) {
+            bulk_copy_to_shared(im.row_p, g_row_p, b_rowp, im.bar);
+        } else {
+            bulk_copy_to_shared(im.bucket_list, g_bucket_list, b_bucket, im.bar);
+            bulk_copy_to_shared(im.start_list, g_start_list, b_start, im.bar);
+            bulk_copy_to_shared(im.pool, g_pool, b_pool, im.bar);
+        }
+        bulk_copy_to_shared(im.start_table, g_start_table, b_start, im.bar);
+        bulk_copy_to_shared(im.row_bounds, g_row_bounds, b_bounds, im.bar);
+        bulk_copy_to_shared(im.group_bounds, g_group_bounds, b_groups, im.bar);
+    }
+    unsigned char *after_tables = im.end;
     // the warps' queues: {L_in, L_out, bits of D, low word of the request index}, high word
     constexpr int kWarps = route_threads(kRowP, kReqPerThread) / 32;
     // (entries: the request's index less that of the CTA's first request; a CTA's run of requests
@@ -668,8 +727,25 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     const int64_t cta_first_request = cta_first * kWarpTile;
     unsigned long long *hist = reinterpret_cast<unsigned long long *>(after_tables);
     if (kAccumulate)
-        for (int k = threadIdx.x; k < 3 * M; k += blockDim.x) hist[k] = 0ull;
-    __syncthreads();
+        for (int k = threadIdx.x; k < 3 * GS_MAX_INSTANCES; k += blockDim.x) hist[k] = 0ull;
+    // every thread waits for the tables itself (the barrier's phase is what makes them visible)
+    {
+        const bool arrived = wait_barrier(im.bar, 0u);
+        if (!__syncthreads_and(arrived)) {
+            // the copies did not complete in time: report it, give them one more chance to land
+            // (nothing may still be writing this CTA's shared memory when it exits) and leave
+            if (threadIdx.x == 0) atomicOr(status, (unsigned)GS_DEV_TIMEOUT);
+            wait_barrier(im.bar, 0u);
+            return;
+        }
+    }
+    const int M = im.info[2];
+    const float cand_z0 = __int_as_float(im.info[4]), cand_inv = __int_as_float(im.info[5]);
+    Tables tb;
+    tb.headers = im.headers; tb.row_bounds = im.row_bounds; tb.group_bounds = im.group_bounds;
+    tb.start_table = im.start_table; tb.rows = im.rows; tb.row_p = im.row_p; tb.cand = im.cand;
+    tb.pool = im.pool; tb.bucket_list = im.bucket_list; tb.start_list = im.start_list;
+    tb.n_types = im.info[1] != 0 ? 0 : im.info[3];       // unusable bounds: every request takes the exhaustive path
 
     const bool fast_on = tb.n_types > 0;          // unusable bounds: every request takes the full search
     unsigned bad = 0;
@@ -844,7 +920,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
 
 constexpr size_t kTablesSmemFixed = (size_t)GS_MAX_INSTANCES * sizeof(Row) + GS_MAX_TYPES * sizeof(TypeHeader) +
                                     (size_t)kMaxPaddedRows * sizeof(uint2) + kMaxPaddedRows / 8 * sizeof(float2);
-constexpr size_t kRouteSmemFixed = kTablesSmemFixed + kCandSlots * sizeof(unsigned short) +
+constexpr size_t kRouteSmemFixed = kTablesSmemFixed + kCandSlots * sizeof(unsigned short) + 64 + 16 +   // info, barrier
                                    (size_t)(route_threads(false, 1) / 32) * kQueueCap * sizeof(unsigned);
 constexpr size_t kRouteSmemPerType = (size_t)kStartBuckets * kStartSlots;
 constexpr size_t kRouteSmemHist = (size_t)3 * GS_MAX_INSTANCES * sizeof(unsigned long long);
@@ -860,7 +936,7 @@ static size_t route_smem_bytes(int n_types, bool accumulate, bool row_p) {
 }
 
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
-                         const float *slo_ms, int64_t n, const PrefixHits *hits, int n_types,
+                         const float *slo_ms, int64_t n, const PrefixHits *hits, int n_instances, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
                          bool accumulate, bool row_p, cudaStream_t st)
 {
@@ -869,20 +945,42 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     // CTA per SM that bounds a batch far beyond what fits in device memory)
     if (n > ((int64_t)1 << 36)) return cudaErrorInvalidValue;
     const size_t smem = route_smem_bytes(n_types, accumulate, row_p);
+    // upper bounds of what the kernel copies of the round's tables: the rows (position-mixed in
+    // blocks of eight) and the padded rows of all groups (each group adds less than 16 of padding)
+    const int m_rows = (n_instances + 7) & ~7;
+    int n_padded_max = (n_instances + 16 * n_types + 15) & ~15;
+    if (n_padded_max > kMaxPaddedRows) n_padded_max = kMaxPaddedRows;
     const int req = n < kSmallBatch ? 1 : 4;
     const int64_t tile = (int64_t)route_threads(row_p, req) * req;
     int64_t blocks = (n + tile - 1) / tile;
     if (blocks > ctx->n_sm) blocks = ctx->n_sm;   // one CTA per SM: its tables fill most of the shared memory
     LaunchTimer timer(ctx, GS_K_ROUTE, st);
     const PrefixHits none = {nullptr, nullptr, 0, 0};
+    // a programmatic dependent of the kernel before it in the stream (the prologue): it may be
+    // set up, and read its first requests, while that kernel still runs
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t err = cudaSuccess;
 #define GS_LAUNCH_ROUTE(ACC, PFX, ROWP)                                                               \
     if (req == 1) GS_LAUNCH_ROUTE_R(ACC, PFX, ROWP, 1); else GS_LAUNCH_ROUTE_R(ACC, PFX, ROWP, 4)
 #define GS_LAUNCH_ROUTE_R(ACC, PFX, ROWP, REQ)                                                        \
-    route_kernel<ACC, PFX, ROWP, REQ><<<(unsigned)blocks, route_threads(ROWP, REQ), smem, st>>>(      \
-        prompt_len, pred_decode_len, slo_ms, n, hits ? *hits : none, n_types, ctx->s.rows,            \
-        ctx->s.row_bounds, ctx->s.group_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info, ctx->s.cand_table,  \
-        ctx->s.pool, ctx->s.bucket_list, ctx->s.start_list, ctx->s.row_p,                             \
-        out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status)
+    do {                                                                                              \
+        cfg.blockDim = dim3(route_threads(ROWP, REQ));                                                \
+        err = cudaLaunchKernelEx(&cfg, route_kernel<ACC, PFX, ROWP, REQ>,                             \
+            prompt_len, pred_decode_len, slo_ms, n, hits ? *hits : none, n_types, (const Row *)ctx->s.rows,            \
+            (const uint2 *)ctx->s.row_bounds, (const float2 *)ctx->s.group_bounds, (const unsigned char *)ctx->s.start_table, \
+            (const TypeHeader *)ctx->s.headers, (const int *)ctx->s.table_info, (const unsigned short *)ctx->s.cand_table,  \
+            (const uint2 *)ctx->s.pool, (const unsigned short *)ctx->s.bucket_list, (const unsigned char *)ctx->s.start_list, \
+            (const float *)ctx->s.row_p, m_rows, n_padded_max,                                        \
+            out_idx, out_est, out_slack, out_tier, ctx->s.deltas, ctx->s.status);                     \
+    } while (0)
     // (the prefix term and per-row p are never combined with accumulate, nor with each other)
     if (row_p) GS_LAUNCH_ROUTE(false, false, true);
     else if (hits && hits->n_slots > 0) GS_LAUNCH_ROUTE(false, true, false);
@@ -890,7 +988,7 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     else GS_LAUNCH_ROUTE(false, false, false);
 #undef GS_LAUNCH_ROUTE
 #undef GS_LAUNCH_ROUTE_R
-    return cudaGetLastError();
+    return err;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -915,6 +1013,7 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
                float *__restrict__ out_slack, uint8_t *__restrict__ out_tier, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // (the tables are the prologue's)
     const int M = table_info[2];
     Tables tb;
     stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_group_bounds, g_start_table, g_headers, table_info, tb);
