@@ -135,6 +135,17 @@ GS_API int gs_device_status(gs_ctx *ctx, void *cuda_stream, unsigned *out_bits);
 /* Number of kernels this context has launched since it was created. */
 GS_API int64_t gs_launch_count(const gs_ctx *ctx);
 
+/* Work counters of the routing kernels, for benchmarks.  Synchronises `cuda_stream`, copies the
+ * GS_EVAL_COUNT counters to `out` (host) and clears them if `clear` != 0.  They count, since they
+ * were last cleared: [0] request-instance pairs scored exactly (T of Eq. 2 evaluated in full),
+ * [1] per-instance lower bounds of T tested, [2] whole-type lower bounds tested, [3] requests that
+ * the straight-line first attempt left to the full search, [4] requests that ran the fallback
+ * (Algorithm 1's else branch), [5] requests scored against every instance by a whole warp.
+ * Only a library built with -DGS_COUNT_EVALS counts (one global atomic per event: a measuring
+ * build, many times slower); the regular build returns zeros. */
+#define GS_EVAL_COUNT 8
+GS_API int gs_eval_counters(gs_ctx *ctx, void *cuda_stream, uint64_t *out, int clear);
+
 /* Kernels of the library, for gs_timing_read. */
 enum gs_kernel {
     GS_K_PROLOGUE = 0,       /* instance coefficients + preference order (per round) */

@@ -230,6 +230,18 @@ GS_API int gs_timing_read(gs_ctx *ctx, int kernel, double *total_ms, int64_t *la
 
 GS_API int gs_last_cuda_error(const gs_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
+GS_API int gs_eval_counters(gs_ctx *ctx, void *cuda_stream, uint64_t *out, int clear) {
+    if (!ctx || !out) return GS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+    unsigned long long v[gs::kCountN];
+    if (e == cudaSuccess) e = gs::read_eval_counters(v, clear != 0);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    for (int k = 0; k < gs::kCountN; ++k) out[k] = v[k];
+    return GS_OK;
+}
+
 GS_API int64_t gs_launch_count(const gs_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
 GS_API int gs_device_status(gs_ctx *ctx, void *cuda_stream, unsigned *out_bits) {

@@ -11,6 +11,19 @@
 
 namespace gs {
 
+// Work counters of the routing kernels, only in a library built with -DGS_COUNT_EVALS (the
+// benchmark's second build; one global atomic per event, far too slow for anything else).
+enum EvalCounter {
+    kCountExact = 0,        // pairs (request, instance) scored exactly, T of Eq. 2 in full
+    kCountBound = 1,        // row bounds tested (a lower bound of T for one pair)
+    kCountTypeTest = 2,     // whole-type bounds tested
+    kCountQueued = 3,       // requests that the first attempt left to the full search
+    kCountFallback = 4,     // requests that ran the per-lane fallback (no feasible instance)
+    kCountExhaustive = 5,   // requests scored against every instance by a whole warp
+    kCountN = 8
+};
+cudaError_t read_eval_counters(unsigned long long *out, bool clear);     // zeros unless GS_COUNT_EVALS
+
 // Exact per-instance coefficients of Eq. 2 for the current round, in caller order.
 struct __align__(16) Row {
     float q, p, d;

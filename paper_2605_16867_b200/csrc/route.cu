@@ -26,6 +26,28 @@
 
 namespace gs {
 
+#ifdef GS_COUNT_EVALS
+__device__ unsigned long long g_eval_counts[kCountN];
+#define GS_COUNT(k, v) atomicAdd(&gs::g_eval_counts[k], (unsigned long long)(v))
+#else
+#define GS_COUNT(k, v) ((void)0)
+#endif
+cudaError_t read_eval_counters(unsigned long long *out, bool clear)
+{
+    for (int k = 0; k < kCountN; ++k) out[k] = 0ull;
+#ifdef GS_COUNT_EVALS
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_eval_counts, sizeof(unsigned long long) * kCountN);
+    if (e != cudaSuccess) return e;
+    if (clear) {
+        unsigned long long zeros[kCountN] = {};
+        return cudaMemcpyToSymbol(g_eval_counts, zeros, sizeof(zeros));
+    }
+#else
+    (void)clear;
+#endif
+    return cudaSuccess;
+}
+
 #ifndef GS_ROUTE_THREADS
 #define GS_ROUTE_THREADS 768
 #endif
@@ -119,6 +141,7 @@ constexpr int kThreadFallbackMin = GS_THREAD_FALLBACK_MIN;
 template <bool kCapped, bool kRowP>
 __device__ __forceinline__ bool row_may_pass(unsigned q_word, unsigned d_word, float p_lo, float x, float y,
                                              float R, float d_cap) {
+    GS_COUNT(kCountBound, 1);
     const float d_lo = __uint_as_float(d_word);
     const float base = kRowP ? __fmaf_rn(p_lo, x, __uint_as_float(q_word)) : __uint_as_float(q_word);
     return __fmaf_rn(d_lo, y, base) <= R && (!kCapped || d_lo < d_cap);
@@ -132,6 +155,7 @@ template <bool kCapped>
 __device__ __forceinline__ bool score_row(const Tables &tb, int inst, float x, float y, float D, unsigned need,
                                           float d_cap, int &g_best, float &d_best, float &T_best)
 {
+    GS_COUNT(kCountExact, 1);
     const Row row = tb.rows[row_pos(inst)];
     const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));      // Eq. 2, H = 0
     const bool feasible = (T <= D) && (need <= (unsigned)row.kv) && (!kCapped || row.d < d_cap);
@@ -154,6 +178,7 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
     for (int t = 0; t < tb.n_types; ++t) {
         const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);   // p_lo, q_lo, d_lo, d_max
         // (a type whose least d_lo is not below the cap has no eligible instance: d_lo <= d)
+        if (D >= 0.f) GS_COUNT(kCountTypeTest, 1);
         if (__fmaf_rn(h.z, y, h.y) <= __fmaf_rn(-h.x, x, Dm) && (!kCapped || h.z < d_cap)) alive |= 1u << t;
     }
     int g_best = -1;
@@ -281,6 +306,7 @@ __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y
                         const Row row = tb.rows[row_pos(inst)];
                         if (kCapped && !(row.d < d_cap)) continue;
                         if (!any_kv && !(need <= (unsigned)row.kv)) continue;
+                        GS_COUNT(kCountExact, 1);
                         const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));   // Eq. 2, H = 0
                         if (T < T_best || (T == T_best && inst < g_best) || g_best < 0) {
                             T_best = T; g_best = inst;
@@ -353,6 +379,7 @@ __device__ __forceinline__ void exhaustive_pick(const Row *rows, int M, float xs
     for (int inst = lane; inst < M; inst += 32) {
         const Row row = rows[row_pos(inst)];
         if (kCapped && !(row.d < d_cap)) continue;
+        GS_COUNT(kCountExact, 1);
         const float Tr = latency(row, xs, ys);
         const bool room = needs <= (unsigned)row.kv;
         const unsigned long long kt = ((unsigned long long)orderable_bits(Tr) << 32) | (unsigned)inst;
@@ -503,6 +530,7 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
         mask &= mask - 1;
         h = *reinterpret_cast<const float4 *>(&tb.headers[tt]);               // p_lo, q_lo, d_lo, d_max
         Rg = __fmaf_rn(-h.x, x, Dm);
+        GS_COUNT(kCountTypeTest, 1);
         if (__fmaf_rn(h.z, y, h.y) <= Rg) { t = tt; break; }
     }
     if (t < 0) return false;
@@ -537,6 +565,7 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
     }
     if (first == kNoRow) return false;
     const int inst = (int)(first & kRowTagMask);
+    GS_COUNT(kCountExact, 1);
     const Row row = tb.rows[row_pos(inst)];
     const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));          // Eq. 2, H = 0
     if (!(T <= D && need <= (unsigned)row.kv)) return false;
@@ -546,6 +575,7 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
         mask &= mask - 1;
         const float4 h2 = *reinterpret_cast<const float4 *>(&tb.headers[tt]);
         if (h2.w < row.d) break;                                              // nor can any type after it
+        GS_COUNT(kCountTypeTest, 1);
         if (__fmaf_rn(fmaxf(h2.z, d_floor), y, h2.y) <= __fmaf_rn(-h2.x, x, Dm)) return false;
     }
     g_out = inst;
@@ -574,6 +604,7 @@ __device__ __noinline__ Pick full_pick(const Tables tb, int M, int lane, bool ac
     const bool mine = open && yi > 0 && tb.n_types > 0;
     const int n_fall = __popc(__ballot_sync(0xFFFFFFFFu, mine));
     if (mine && n_fall >= kThreadFallbackMin) {
+        GS_COUNT(kCountFallback, 1);
         out = fallback_pick<false, kRowP>(tb, x, y, need, 0.f);
         open = false;
     }
@@ -585,6 +616,7 @@ __device__ __noinline__ Pick full_pick(const Tables tb, int M, int lane, bool ac
         const float Ds = __shfl_sync(0xFFFFFFFFu, D, src);
         const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
         int gg; float TT; unsigned tt;
+        if (lane == 0) GS_COUNT(kCountExhaustive, 1);
         exhaustive_pick<false>(tb.rows, M, xs, ys, Ds, needs, 0.f, lane, gg, TT, tt);
         if (lane == src) { out.g = gg; out.T = TT; out.tier = tt; }
     }
@@ -820,7 +852,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             if (fast_on)
                 settled = fast_pick<kRowP>(tb, cand_z0, cand_inv, __int2float_rn(xi[j]), __int2float_rn(yi[j]),
                                            (valid && yi[j] > 0) ? D[j] : -1.0f, (unsigned)xi[j] + (unsigned)yi[j], g_out[j], T_out[j]);
-            if (valid && !settled) slow |= 1u << j;
+            if (valid && !settled) { slow |= 1u << j; GS_COUNT(kCountQueued, 1); }
         }
         if (kPrefix) {
             for (int k = 0; k < hits.n_slots; ++k) {
@@ -887,26 +919,10 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     if (q_count < 32) break;                       // out of tiles
     do drain(); while (q_count >= 32);
     }
-    // What is left on the warps' queues (fewer than 32 each) is pooled: the CTA's warps take it
-    // 32 requests at a time, so the full search still runs with its lanes busy.
-    {
-        __shared__ int sh_left[kWarps];
-        const int warp = threadIdx.x >> 5;
-        if (lane == 0) sh_left[warp] = q_count;
-        __syncthreads();
-        int total = 0;
-        for (int w = 0; w < kWarps; ++w) total += sh_left[w];
-        for (int v0 = warp * 32; v0 < total; v0 += kWarps * 32) {
-            const int v = v0 + lane;
-            const bool active = v < total;
-            int owner = 0, before = 0;             // whose queue entry v is, and how many entries come before that queue
-            for (int w = 0; w < kWarps - 1; ++w) {
-                const int c = sh_left[w];
-                if (v >= before + c && owner == w) { before += c; owner = w + 1; }
-            }
-            settle(active, active ? queue_all[owner * kQueueCap + v - before] : 0u);
-        }
-    }
+    // What is left on the warp's queue (fewer than 32) it finishes itself, right after its last
+    // tile: the warps of a CTA end up to a tile apart, so these searches overlap the other warps'
+    // last tiles, and a handful of lanes per warp diverge far less than 32 would.
+    while (q_count > 0) drain();
     if (bad) atomicOr(status, bad);
 
     if (kAccumulate) {
