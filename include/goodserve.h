@@ -30,7 +30,9 @@
  *     buffers owned by the context.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *     Device entry points only enqueue work on it and return; they do not synchronise.
- *   - Return value: GS_OK or a negative gs_error.  On an error nothing has been enqueued.
+ *   - Return value: GS_OK or a negative gs_error.  Every error but GS_ERR_CUDA is found in the
+ *     arguments before anything is enqueued; GS_ERR_CUDA (a launch or copy that the CUDA runtime
+ *     refused) can leave the part of the call that came before it on the stream.
  *   - Invalid DATA never faults or traps: negative token counts and negative/NaN q_ema are
  *     read as 0, a type id outside [0, n_types) as type 0, an assigned instance outside
  *     [0, n_instances) is clamped into range; a bit of the device status word records it
@@ -74,7 +76,8 @@ enum gs_dev_status {
     GS_DEV_BAD_INSTANCE = 1,    /* assigned_inst outside [0, n_instances) was clamped */
     GS_DEV_BAD_TYPE = 2,        /* type_id outside [0, n_types) was read as 0 */
     GS_DEV_BAD_VALUE = 4,       /* negative count or negative/NaN q_ema was read as 0 */
-    GS_DEV_TIMEOUT = 8,         /* a bounded device-side wait expired (results of that call are invalid) */
+    GS_DEV_TIMEOUT = 8,         /* a bounded device-side wait expired (the route kernel's wait for its table
+                                   copies); the outputs of that call are invalid */
     GS_DEV_CAND_TRUNCATED = 16  /* more flagged requests than cand_capacity; list was cut */
 };
 
@@ -181,8 +184,8 @@ GS_API int gs_timing_read(gs_ctx *ctx, int kernel, double *total_ms, int64_t *la
  *                     3 = no instance has KV room: minimum T among all.
  * Ties (equal d_g, or equal T in the fallback) go to the smallest instance index.
  * Feasibility is T <= D (a request whose estimate equals its deadline is feasible).
- * n_requests == 0 is valid and enqueues nothing; more than 2^36 requests in one call is refused
- * (GS_ERR_CUDA, invalid value).  Never writes the instance state.
+ * n_requests == 0 is valid; more than 2^36 requests in one call is refused (GS_ERR_INVALID_ARG,
+ * nothing enqueued).  Never writes the instance state.
  */
 GS_API int gs_route_batch(gs_ctx *ctx,
                    const int32_t *prompt_len, const int32_t *pred_decode_len,
@@ -303,7 +306,8 @@ GS_API int gs_route_sequential(gs_ctx *ctx,
  * advance: per instance g,  queued_prefill_tokens += sum of L_in routed to g  (saturating at
  * INT32_MAX), decode_batch += number of requests routed to g (saturating),
  * free_kv_tokens = max(free_kv_tokens - sum of (L_in + L_out), 0), and q_ema_ms = q_g of the
- * latest round.  Clears the pending deltas.  Integer sums, so the result does not depend on
+ * latest GS_ROUTE_ACCUMULATE round (other routing calls in between do not disturb it; without
+ * such a round since the last advance q_ema_ms is left as it is).  Clears the pending deltas.  Integer sums, so the result does not depend on
  * the order in which requests were processed.
  */
 GS_API int gs_advance_state(gs_ctx *ctx, const gs_instances_mut *inst, void *cuda_stream);

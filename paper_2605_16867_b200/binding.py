@@ -53,30 +53,16 @@ class _InstancesMut(C.Structure):
                 ("n_instances", C.c_int32)]
 
 
-def library_path() -> str:
-    return os.path.join(_PKG, "libgoodserve.so")
+def library_path(counting: bool = False) -> str:
+    return os.path.join(_PKG, "libgoodserve_count.so" if counting else "libgoodserve.so")
 
 
 _lib = None
+_count_lib = None
 
 
-def load_library(build_if_missing: bool = True):
-    """Loads libgoodserve.so (building it with nvcc first if it is absent or stale).
-    Raises if that fails -- there is no other implementation to fall back to."""
-    global _lib
-    if _lib is not None:
-        return _lib
-    path = library_path()
-    if build_if_missing:
-        from .build import build_library
-        try:
-            build_library()
-        except Exception as exc:                      # nvcc missing on a box that has the .so
-            if not os.path.exists(path):
-                raise RuntimeError(f"libgoodserve.so is missing and could not be built: {exc}") from exc
-    if not os.path.exists(path):
-        raise RuntimeError(f"{path} not found; run paper_2605_16867_b200/build.py")
-    lib = C.CDLL(path)
+def _declare(lib):
+    """Argument and result types of every entry point of include/goodserve.h."""
     vp, i32, i64, f32, u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_uint
     lib.gs_create.argtypes = [C.POINTER(vp), C.c_int, C.c_int, C.c_int]
     lib.gs_destroy.argtypes = [vp]
@@ -86,6 +72,8 @@ def load_library(build_if_missing: bool = True):
     lib.gs_device_status.argtypes = [vp, vp, C.POINTER(u32)]
     lib.gs_launch_count.argtypes = [vp]
     lib.gs_launch_count.restype = i64
+    lib.gs_eval_counters.argtypes = [vp, vp, C.POINTER(C.c_uint64), C.c_int]
+    lib.gs_eval_counters.restype = C.c_int
     route_args = [vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types), f32, vp, vp, vp, vp]
     lib.gs_route_batch.argtypes = route_args + [u32, vp]
     lib.gs_route_batch_host.argtypes = route_args + [vp]
@@ -114,7 +102,33 @@ def load_library(build_if_missing: bool = True):
     for name in ("gs_timing_enable", "gs_timing_read", "gs_create", "gs_destroy", "gs_last_cuda_error", "gs_device_status", "gs_route_batch",
                  "gs_route_batch_host", "gs_advance_state", "gs_risk_scan", "gs_risk_scan_host"):
         getattr(lib, name).restype = C.c_int
-    _lib = lib
+    return lib
+
+
+def load_library(build_if_missing: bool = True, counting: bool = False):
+    """Loads libgoodserve.so (building it with nvcc first if it is absent or stale).
+    Raises if that fails -- there is no other implementation to fall back to.
+    ``counting=True`` loads the measuring build instead (-DGS_COUNT_EVALS: the work counters
+    behind gs_eval_counters tick; many times slower, for benchmarks only)."""
+    global _lib, _count_lib
+    cached = _count_lib if counting else _lib
+    if cached is not None:
+        return cached
+    path = library_path(counting)
+    if build_if_missing:
+        from .build import build_library
+        try:
+            build_library(counting=counting)
+        except Exception as exc:                      # nvcc missing on a box that has the .so
+            if not os.path.exists(path):
+                raise RuntimeError(f"{os.path.basename(path)} is missing and could not be built: {exc}") from exc
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} not found; run paper_2605_16867_b200/build.py")
+    lib = _declare(C.CDLL(path))
+    if counting:
+        _count_lib = lib
+    else:
+        _lib = lib
     return lib
 
 
@@ -180,10 +194,10 @@ class InstancePool:
 class GoodServe:
     """One library context (gs_create / gs_destroy) bound to a CUDA device."""
 
-    def __init__(self, device: int = 0, max_instances: int = 1024, max_types: int = 16):
+    def __init__(self, device: int = 0, max_instances: int = 1024, max_types: int = 16, counting: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("GoodServe needs a CUDA device; there is no CPU implementation")
-        self._lib = load_library()
+        self._lib = load_library(counting=counting)
         self.device = torch.device("cuda", device)
         torch.cuda.init()
         with torch.cuda.device(self.device):
@@ -412,6 +426,13 @@ class GoodServe:
         bits = C.c_uint(0)
         self._check(self._lib.gs_device_status(self._h, self._stream(stream), C.byref(bits)))
         return int(bits.value)
+
+    def eval_counters(self, clear: bool = True, stream=None):
+        """Work counters of the routing kernels (all zero unless the library was built with
+        -DGS_COUNT_EVALS): exact scorings, row bounds, type bounds, queued, fallback, exhaustive."""
+        out = (C.c_uint64 * 8)()
+        self._check(self._lib.gs_eval_counters(self._h, self._stream(stream), out, 1 if clear else 0))
+        return [int(v) for v in out]
 
     def launch_count(self) -> int:
         return int(self._lib.gs_launch_count(self._h))

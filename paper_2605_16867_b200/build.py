@@ -11,6 +11,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libgoodserve.so")
+COUNT_LIB_PATH = os.path.join(_PKG, "libgoodserve_count.so")    # the measuring build (-DGS_COUNT_EVALS)
 SOURCES = ("api.cu", "prologue.cu", "route.cu", "risk.cu", "sequential.cu")
 NVCC_FLAGS = ("-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--shared",
@@ -24,26 +25,32 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found: libgoodserve.so cannot be built")
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def _stale(path: str) -> bool:
+    if not os.path.exists(path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(path)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "goodserve.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
-    if not force and not _stale():
-        return LIB_PATH
+def build_library(force: bool = False, verbose: bool = False, extra_flags=(), counting: bool = False) -> str:
+    """Builds libgoodserve.so, or with ``counting`` the measuring build whose work counters tick."""
+    path = COUNT_LIB_PATH if counting else LIB_PATH
+    if not force and not _stale(path):
+        return path
+    if counting:
+        extra_flags = (*extra_flags, "-DGS_COUNT_EVALS")
     cmd = [_nvcc(), *NVCC_FLAGS, *extra_flags, "-I", INCLUDE, "-I", CSRC,
-           *[os.path.join(CSRC, s) for s in SOURCES], "-o", LIB_PATH + ".tmp"]
+           *[os.path.join(CSRC, s) for s in SOURCES], "-o", path + ".tmp"]
     if verbose:
         print(" ".join(cmd), file=sys.stderr)
     subprocess.run(cmd, check=True)
-    os.replace(LIB_PATH + ".tmp", LIB_PATH)
-    return LIB_PATH
+    os.replace(path + ".tmp", path)
+    return path
 
 
 if __name__ == "__main__":
     print(build_library(force="--force" in sys.argv, verbose=True,
                         extra_flags=("-Xptxas", "-v") if "--ptxas" in sys.argv else ()))
+    if "--counting" in sys.argv:
+        print(build_library(force="--force" in sys.argv, verbose=True, counting=True))

@@ -166,7 +166,6 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
         {(void **)&s.pool, gs::kPoolEntries * sizeof(uint2)},
         {(void **)&s.bucket_list, (size_t)GS_MAX_TYPES * gs::kStartBuckets * sizeof(unsigned short)},
         {(void **)&s.start_list, (size_t)GS_MAX_TYPES * gs::kStartBuckets * gs::kStartSlots},
-        {(void **)&s.d_by_g, Mx * sizeof(float)},
         {(void **)&s.q_by_g, Mx * sizeof(float)},
         {(void **)&s.deltas, 3 * Mx * sizeof(unsigned long long)},
         {(void **)&s.scan_counts, gs::kMaxScanCtas * sizeof(unsigned)},
@@ -189,7 +188,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.d_by_g, s.q_by_g, s.deltas, s.scan_counts, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.q_by_g, s.deltas, s.scan_counts, s.status, ctx->stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);
@@ -262,7 +261,7 @@ GS_API int gs_route_batch(gs_ctx *ctx, const int32_t *prompt_len, const int32_t 
 {
     int rc = check_pool(ctx, inst, types, true);
     if (rc != GS_OK) return rc;
-    if (n_requests < 0 || (flags & ~GS_ROUTE_ACCUMULATE)) return GS_ERR_INVALID_ARG;
+    if (n_requests < 0 || n_requests > gs::kMaxRouteRequests || (flags & ~GS_ROUTE_ACCUMULATE)) return GS_ERR_INVALID_ARG;
     if (n_requests > 0) {
         const void *ptrs[] = {prompt_len, pred_decode_len, slo_ms, out_instance_idx, out_est_e2e_ms, out_slack_ms};
         for (const void *p : ptrs) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
@@ -271,7 +270,8 @@ GS_API int gs_route_batch(gs_ctx *ctx, const int32_t *prompt_len, const int32_t 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GS_ERR_NO_DEVICE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
+    if (n_requests == 0 && !(flags & GS_ROUTE_ACCUMULATE)) return GS_OK;
+    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, (flags & GS_ROUTE_ACCUMULATE) != 0, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, inst->n_instances, types->n_types,
                          out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier,
@@ -289,7 +289,8 @@ GS_API int gs_route_batch_prefix(gs_ctx *ctx, const int32_t *prompt_len, const i
 {
     int rc = check_pool(ctx, inst, types, true);
     if (rc != GS_OK) return rc;
-    if (n_requests < 0 || n_slots < 0 || n_slots > GS_MAX_PREFIX_SLOTS) return GS_ERR_INVALID_ARG;
+    if (n_requests < 0 || n_requests > gs::kMaxRouteRequests || n_slots < 0 || n_slots > GS_MAX_PREFIX_SLOTS)
+        return GS_ERR_INVALID_ARG;
     if (n_slots > 0 && n_requests > 0) {
         if (!prefix_inst || !prefix_hit_len || slot_stride < n_requests) return GS_ERR_INVALID_ARG;
         if (misaligned(prefix_inst) || misaligned(prefix_hit_len) || (slot_stride & 3)) return GS_ERR_ALIGN;
@@ -302,7 +303,8 @@ GS_API int gs_route_batch_prefix(gs_ctx *ctx, const int32_t *prompt_len, const i
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GS_ERR_NO_DEVICE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
+    if (n_requests == 0) return GS_OK;
+    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, false, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     const gs::PrefixHits hits = {prefix_inst, prefix_hit_len, n_slots, slot_stride};
     e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, &hits, inst->n_instances, types->n_types,
@@ -335,7 +337,8 @@ GS_API int gs_route_batch_direct(gs_ctx *ctx, const int32_t *prompt_len, const i
                           int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
                           uint8_t *out_tier, void *cuda_stream)
 {
-    if (!ctx || !table || n_requests < 0 || table->n_instances < 1) return GS_ERR_INVALID_ARG;
+    if (!ctx || !table || n_requests < 0 || n_requests > gs::kMaxRouteRequests || table->n_instances < 1)
+        return GS_ERR_INVALID_ARG;
     if (table->n_instances > ctx->max_instances) return GS_ERR_CAPACITY;
     const void *cols[] = {table->q_ms, table->p_ms_per_tok, table->d_ms_per_tok, table->free_kv_tokens};
     for (const void *p : cols) { if (!p) return GS_ERR_INVALID_ARG; if (misaligned(p)) return GS_ERR_ALIGN; }
@@ -347,6 +350,7 @@ GS_API int gs_route_batch_direct(gs_ctx *ctx, const int32_t *prompt_len, const i
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GS_ERR_NO_DEVICE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (n_requests == 0) return GS_OK;
     cudaError_t e = gs::launch_prologue_direct(ctx, *table, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     e = gs::launch_route(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, nullptr, table->n_instances, gs::kDirectGroups,
@@ -440,7 +444,8 @@ GS_API int gs_reroute_candidates(gs_ctx *ctx, const int32_t *cand_idx, const int
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GS_ERR_NO_DEVICE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, st);
+    if (cand_capacity == 0) return GS_OK;
+    cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, false, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     e = gs::launch_reroute(ctx, cand_idx, cand_count, cand_capacity, assigned_inst, generated_tokens, pred_len,
                            elapsed_ms, slo_ms, prompt_len, n_active, types->n_types,

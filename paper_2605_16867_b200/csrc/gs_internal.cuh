@@ -52,7 +52,8 @@ __host__ __device__ __forceinline__ int row_slot(int i) {
 __host__ __device__ __forceinline__ int row_pos(int g) { return g ^ (((g >> 3) ^ (g >> 6)) & 7); }
 
 constexpr unsigned kRowTagMask = 0x3FFu;            // instance index in the low bits of a q word
-// groups of similar p that stand in for GPU types when the coefficients are given per instance
+// groups of consecutive rank (d descending) that stand in for GPU types when the coefficients
+// are given per instance
 #ifndef GS_DIRECT_GROUPS
 #define GS_DIRECT_GROUPS 8
 #endif
@@ -98,6 +99,8 @@ constexpr int kListWindow = 8;             // entries the first attempt may test
 constexpr int kListMax = 510;              // longer lists are not stored (start_list counts pairs of entries in a byte)
 constexpr unsigned short kNoList = 0xFFFFu;
 
+constexpr int64_t kMaxRouteRequests = (int64_t)1 << 36;   // per routing call (the kernel's queues hold a request's
+                                                          // index within its CTA's run of requests in 32 bits)
 constexpr int kMaxScanCtas = 4096;      // CTAs of one risk scan (a few per SM), one flag count each
 constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 
@@ -111,13 +114,12 @@ struct Scratch {
     TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)
     int *table_info;          // {padded rows, unsafe, n_instances, n_active_types, bits of the candidate
                               //  table's origin (least d_lo of any type), bits of its slots per unit of d,
-                              //  pool entries handed out to the types}
+                              //  pool entries handed out to the types, 1 = q_by_g holds a round to carry}
     unsigned short *cand_table;   // [kCandSlots] candidate types by slot of D / L_out
     uint2 *pool;              // [kPoolEntries] record lists
     unsigned short *bucket_list;  // [GS_MAX_TYPES * kStartBuckets] first pool entry of the list, halved; kNoList = none
     unsigned char *start_list;    // [GS_MAX_TYPES * kStartBuckets * kStartSlots] like start_table, in pairs of list entries
-    float *d_by_g;            // [max_instances] d_g in caller order (risk scan gather)
-    float *q_by_g;            // [max_instances] q_g in caller order (carried by advance)
+    float *q_by_g;            // [max_instances] q_g of the latest ACCUMULATE round, caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out
     unsigned *scan_counts;    // [kMaxScanCtas] risk scan: requests flagged by each CTA of pass 1
     unsigned *status;         // device status word
@@ -167,7 +169,7 @@ struct PrefixHits {
 
 // launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_types &types,
-                            float ema_alpha, cudaStream_t st);
+                            float ema_alpha, bool carry_q, cudaStream_t st);
 cudaError_t launch_sequential(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                               const float *slo_ms, int64_t n, const int32_t *type_id,
                               const gs_instances_mut &state, const gs_types &types, float alpha,

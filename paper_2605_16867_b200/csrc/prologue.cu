@@ -112,7 +112,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 const int32_t *__restrict__ batch, const int32_t *__restrict__ free_kv,
                 const float *__restrict__ q_ema, int M,
                 const float *__restrict__ p_type, const float *__restrict__ a_type,
-                const float *__restrict__ b_type, int n_types, float alpha,
+                const float *__restrict__ b_type, int n_types, float alpha, int carry_q,
                 Scratch s)
 {
     __shared__ unsigned long long sh_key[GS_MAX_INSTANCES];                // my group's rows as collected
@@ -175,8 +175,6 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             if (writer) {
                 Row row; row.q = q; row.p = pv; row.d = d; row.kv = kv;
                 s.rows[row_pos(tid)] = row;
-                s.d_by_g[tid] = d;
-                s.q_by_g[tid] = q;
             }
             const float big = 3.0e38f;           // the bounds need finite coefficients
             if (!(q < big && pv < big && d < big)) atomicOr(&sh_unsafe, 1);
@@ -225,8 +223,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 if (writer) {
                     Row row; row.q = q; row.p = p; row.d = d; row.kv = kv;
                     s.rows[row_pos(tid)] = row;
-                    s.d_by_g[tid] = d;
-                    s.q_by_g[tid] = q;
+                    if (carry_q) s.q_by_g[tid] = q;     // the smoothed delay that gs_advance_state carries on
                 }
                 // the bounds of the search tables need finite, non-negative coefficients
                 const float big = 3.0e38f;
@@ -328,6 +325,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         s.table_info[2] = M;
         s.table_info[3] = n_act;
         s.table_info[6] = pool_total;
+        if (carry_q) s.table_info[7] = 1;      // a round whose q_g is to be carried is pending
         if (sh_unsafe) atomicOr(s.status, (unsigned)GS_DEV_BAD_VALUE);
     }
     if (writer && bad) atomicOr(s.status, bad);
@@ -544,25 +542,26 @@ cudaError_t configure_prologue()
 }
 
 cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_types &types,
-                            float ema_alpha, cudaStream_t st)
+                            float ema_alpha, bool carry_q, cudaStream_t st)
 {
     LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
     prologue_kernel<false><<<GS_MAX_TYPES, kPrologueThreads, prologue_dynamic_smem(), st>>>(
         inst.type_id, inst.queued_prefill_tokens, inst.decode_batch, inst.free_kv_tokens,
         inst.q_ema_ms, inst.n_instances, types.prefill_ms_per_tok, types.tpot_a_ms,
-        types.tpot_b_ms, types.n_types, ema_alpha, ctx->s);
+        types.tpot_b_ms, types.n_types, ema_alpha, carry_q ? 1 : 0, ctx->s);
     return cudaGetLastError();
 }
 
 // Tables of a round from coefficients given per instance; the instances are put into
-// kDirectGroups groups of similar p, which take the place of the GPU types in the search.
+// kDirectGroups groups of consecutive rank in the preference order, which take the place of the
+// GPU types in the search.
 cudaError_t launch_prologue_direct(gs_ctx *ctx, const gs_instance_table &tab, cudaStream_t st)
 {
     LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
     prologue_kernel<true><<<GS_MAX_TYPES, kPrologueThreads, prologue_dynamic_smem(), st>>>(
         reinterpret_cast<const int32_t *>(tab.q_ms), reinterpret_cast<const int32_t *>(tab.p_ms_per_tok),
         reinterpret_cast<const int32_t *>(tab.d_ms_per_tok), tab.free_kv_tokens, nullptr, tab.n_instances,
-        nullptr, nullptr, nullptr, kDirectGroups, 0.f, ctx->s);
+        nullptr, nullptr, nullptr, kDirectGroups, 0.f, 0, ctx->s);
     return cudaGetLastError();
 }
 

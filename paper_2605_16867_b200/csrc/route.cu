@@ -49,20 +49,21 @@ cudaError_t read_eval_counters(unsigned long long *out, bool clear)
 }
 
 #ifndef GS_ROUTE_THREADS
-#define GS_ROUTE_THREADS 768
+#define GS_ROUTE_THREADS 896
 #endif
 #ifndef GS_ROUTE_MIN_CTAS
 #define GS_ROUTE_MIN_CTAS 1
 #endif
-constexpr int kRouteThreads = GS_ROUTE_THREADS;
+constexpr int kRouteThreads = GS_ROUTE_THREADS;     // four requests per lane (large batches)
+constexpr int kRouteThreadsSmall = 1024;            // one request per lane (small batches)
 constexpr int kRouteMinCtas = GS_ROUTE_MIN_CTAS;
 constexpr int kRerouteThreads = 256;
-// (with per-row p the search holds more state: fewer threads, more registers each)
 // Requests per lane: four (128-bit column loads) for large batches; one for small ones, where
-// shorter tiles spread over more warps count for more than wide loads (fewer registers: a
-// third more threads).
+// shorter tiles spread over more warps count for more than wide loads (fewer registers: more
+// threads).  With per-row p the search holds more state: a quarter fewer threads, more
+// registers each.
 __host__ __device__ constexpr int route_threads(bool row_p, int req = 4) {
-    return (row_p ? (kRouteThreads * 3) / 4 : kRouteThreads) * (req == 1 ? 4 : 3) / 3;
+    return ((req == 1 ? kRouteThreadsSmall : kRouteThreads) * (row_p ? 3 : 4) / 4) & ~31;
 }
 constexpr int64_t kSmallBatch = 1 << 21;        // below this many requests: one per lane
 
@@ -957,9 +958,7 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
                          bool accumulate, bool row_p, cudaStream_t st)
 {
     if (n == 0) return cudaSuccess;
-    // (the kernel's queues hold a request's index within its CTA's run as 32 bits; with at most one
-    // CTA per SM that bounds a batch far beyond what fits in device memory)
-    if (n > ((int64_t)1 << 36)) return cudaErrorInvalidValue;
+    if (n > kMaxRouteRequests) return cudaErrorInvalidValue;      // (the entry points refuse it first)
     const size_t smem = route_smem_bytes(n_types, accumulate, row_p);
     // upper bounds of what the kernel copies of the round's tables: the rows (position-mixed in
     // blocks of eight) and the padded rows of all groups (each group adds less than 16 of padding)
@@ -1151,12 +1150,18 @@ cudaError_t configure_route(gs_ctx *ctx)
 // state advance between rounds of a stream
 // ---------------------------------------------------------------------------------------
 
-__global__ void advance_kernel(int32_t *__restrict__ queued, int32_t *__restrict__ batch,
-                               int32_t *__restrict__ free_kv, float *__restrict__ q_ema, int M,
-                               unsigned long long *__restrict__ deltas,
-                               const float *__restrict__ q_by_g)
+// One CTA, one thread per instance.  The smoothed queue delay is carried only when an ACCUMULATE
+// round has left one since the last advance (the prologue of such a round raises pending[0]).
+__global__ void __launch_bounds__(GS_MAX_INSTANCES)
+advance_kernel(int32_t *__restrict__ queued, int32_t *__restrict__ batch,
+               int32_t *__restrict__ free_kv, float *__restrict__ q_ema, int M,
+               unsigned long long *__restrict__ deltas,
+               const float *__restrict__ q_by_g, int *__restrict__ pending)
 {
-    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    const int g = threadIdx.x;
+    const bool carry = pending[0] != 0;
+    __syncthreads();
+    if (g == 0) pending[0] = 0;
     if (g >= M) return;
     const long long kMax = 2147483647ll;
     const long long dq = (long long)deltas[g];
@@ -1170,16 +1175,16 @@ __global__ void advance_kernel(int32_t *__restrict__ queued, int32_t *__restrict
     queued[g] = (int32_t)Q;
     batch[g] = (int32_t)B;
     free_kv[g] = (int32_t)K;
-    q_ema[g] = q_by_g[g];
+    if (carry) q_ema[g] = q_by_g[g];
 }
 
 cudaError_t launch_advance(gs_ctx *ctx, const gs_instances_mut &inst, cudaStream_t st)
 {
     const int M = inst.n_instances;
     LaunchTimer timer(ctx, GS_K_ADVANCE, st);
-    advance_kernel<<<(M + 255) / 256, 256, 0, st>>>(inst.queued_prefill_tokens, inst.decode_batch,
-                                                    inst.free_kv_tokens, inst.q_ema_ms, M,
-                                                    ctx->s.deltas, ctx->s.q_by_g);
+    advance_kernel<<<1, GS_MAX_INSTANCES, 0, st>>>(inst.queued_prefill_tokens, inst.decode_batch,
+                                                   inst.free_kv_tokens, inst.q_ema_ms, M,
+                                                   ctx->s.deltas, ctx->s.q_by_g, ctx->s.table_info + 7);
     return cudaGetLastError();
 }
 

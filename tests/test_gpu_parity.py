@@ -286,6 +286,36 @@ def test_route_without_accumulate_leaves_state_alone(gs):
     np.testing.assert_array_equal(pool.decode_batch.cpu().numpy(), wl.instances.decode_batch)
 
 
+def test_advance_carries_the_queue_delay_of_the_accumulate_round_only(gs):
+    """gs_advance_state writes back q_g of the latest ACCUMULATE round.  Routing calls that do not
+    accumulate (another alpha, another pool) between that round and the advance must not change
+    what is carried, and an advance with no round pending leaves q_ema alone."""
+    import torch
+    wl = W.make_workload(1, n_requests=3000, n_active=16)
+    pool = pool_of(gs, wl.types, wl.instances)
+    q0 = pool.q_ema_ms.cpu().numpy().copy()
+    gs.advance_state(pool)                                     # nothing pending
+    np.testing.assert_array_equal(pool.q_ema_ms.cpu().numpy().view(np.uint32), q0.view(np.uint32))
+    gpu_route(gs, pool, wl.requests, 0.25)                     # no accumulate: nothing to carry
+    gs.advance_state(pool)
+    np.testing.assert_array_equal(pool.q_ema_ms.cpu().numpy().view(np.uint32), q0.view(np.uint32))
+    t32 = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    got = gpu_route(gs, pool, wl.requests, 0.5, accumulate=True)
+    # other rounds in between: a plain one with another alpha, and one against a smaller pool
+    gpu_route(gs, pool, wl.requests, 0.9)
+    other = W.make_workload(0, n_requests=64, n_active=16)
+    gpu_route(gs, pool_of(gs, other.types, other.instances), other.requests, 0.1)
+    gs.advance_state(pool)
+    torch.cuda.synchronize()
+    ref = oracle.route(t32, *wl.requests.columns())
+    assert_route_matches_f32_oracle(got, ref)
+    state = wl.instances.copy()
+    oracle.advance(state, t32, ref.instance_idx, wl.requests.prompt_len, wl.requests.pred_decode_len)
+    np.testing.assert_array_equal(pool.q_ema_ms.cpu().numpy().view(np.uint32), state.q_ema_ms.view(np.uint32))
+    np.testing.assert_array_equal(pool.decode_batch.cpu().numpy(), state.decode_batch)
+    assert gs.device_status() == 0
+
+
 def test_host_entry_points_match_device_ones(gs):
     wl = W.make_workload(1, n_requests=20_001, n_active=70_003)
     pool = pool_of(gs, wl.types, wl.instances)
