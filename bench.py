@@ -7,6 +7,12 @@ requests (instance prologue, pair scoring, selection, risk test, candidate compa
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 3] [--impl reference]
 
+Besides the step of the largest workload (the headline), rank 0 of a one-GPU run measures
+every one of the five workload shapes (`per_config`): each entry point called back to back and
+one call at a time, inputs rotated through several device copies so that L2 cannot serve them,
+the 64-round stream of config 4 replayed from a CUDA graph, and the work the routing search
+does per request (from the library's counting build).
+
 Prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) every rank
 runs the same-size workload on its own GPU with its own seed -- requests are independent, so
 the path shards with no collective -- and the reported value is all ranks' units over the
@@ -36,17 +42,16 @@ UNIT = "pairs/s"
 ROUTE_BYTES_PER_REQUEST = 24      # 3 input columns + 3 output columns, 4 B each
 RISK_BYTES_PER_REQUEST = 20.125   # 5 input columns + 1 flag bit (candidate indices added per flag)
 KERNEL_NAMES = ("prologue", "route", "advance", "risk_flags", "risk_scatter", "reroute", "ema", "sequential")
-ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9   # SMs x schedulers x 1 warp-instruction per clock
+SCHEDULERS_PER_SM = 4             # one warp-instruction per scheduler and clock
 
-# Counters of one launch on config 3 taken with ncu (profiles/route_kernel_config3.md,
-# profiles/risk_flags_kernel_config3.md).  They describe the kernel sources with these hashes;
-# after any change to those files they no longer apply and the fields that use them become
-# null until the kernel is profiled again.
-PROFILED_ROUTE = {"sources_sha1": "bac3726b1cb32d3d74d0cdb6b491727579021779", "config": 3,
-                  "dram_bytes_per_launch": 52_352_256 + 7_199_488,
-                  "warp_instructions_per_launch": 24_600_939}
-PROFILED_RISK_FLAGS = {"sources_sha1": "23376727e5a3e7bc33cc0aaa3cba258afd1240c6", "config": 3,
-                       "dram_bytes_per_launch": 335_564_032 + 4_064_256}
+# Counters of one launch on config 3 taken with ncu (the committed ncu summaries).  They describe
+# the kernel sources with these hashes; after any change to those files they no longer apply and
+# the fields that use them become null until the kernel is profiled again.
+PROFILED_ROUTE = {"sources_sha1": "", "config": 3,
+                  "dram_bytes_per_launch": 0,
+                  "warp_instructions_per_launch": 0}
+PROFILED_RISK_FLAGS = {"sources_sha1": "", "config": 3,
+                       "dram_bytes_per_launch": 0}
 
 
 def _sources_sha1(names) -> str:
@@ -180,11 +185,18 @@ def cpu_baseline(wl, seconds_target: float = 12.0):
     scale = max(1.0, min(seconds_target / max(t_route, 1e-3) * 0.5, wl.requests.n / n_req))
     n_req = int(n_req * scale)
     t_route, t_risk = oracle_step(wl, n_req, n_act, threads)
+    # the same plain loop on one thread, on a sample sized for a few seconds
+    n1 = max(1024, min(n_req, int(n_req / max(threads, 1) * 0.5)))
+    a1 = max(1024, min(n_act, 1 << 20))
+    t1_route, t1_risk = oracle_step(wl, n1, a1, 1)
     return {"value": n_req * M / (t_route + t_risk), "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"fp64 oracle, first {n_req} of {wl.requests.n} requests x {M} instances "
                       f"({t_route:.2f} s) + risk scan of first {n_act} of {wl.active.n} active requests "
                       f"({t_risk:.2f} s), {threads} threads over contiguous request ranges",
-            "route_pairs_per_s": n_req * M / t_route, "risk_scan_requests_per_s": n_act / t_risk}
+            "route_pairs_per_s": n_req * M / t_route, "risk_scan_requests_per_s": n_act / t_risk,
+            "one_thread": {"route_pairs_per_s": n1 * M / t1_route, "risk_scan_requests_per_s": a1 / t1_risk,
+                           "sample": f"first {n1} requests x {M} instances ({t1_route:.2f} s), first {a1} active "
+                                     f"requests ({t1_risk:.2f} s)"}}
 
 
 def run_reference(args):
@@ -205,7 +217,8 @@ def run_reference(args):
     dt = time.perf_counter() - t0
     value = args.steps * n_req * M / dt
     sample = (f"each step: fp64 oracle over {n_req} requests x {M} instances + risk scan over {n_act} "
-              f"active requests (bounded sample of config {args.config}), {threads} threads")
+              f"active requests (bounded sample of config {args.config}: the full workload would take the "
+              f"oracle seconds per step, so rates, not step times, are what compares), {threads} threads")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
@@ -220,6 +233,189 @@ def workload_name(cfg_id: int) -> str:
     c = W.CONFIGS[cfg_id]
     return (f"config {cfg_id}: {c.n_requests} pending requests x {c.n_instances} instances of "
             f"{c.n_types} GPU types, SLO U[{c.slo_lo},{c.slo_hi}] x ideal; risk scan over {c.n_active} active requests")
+
+
+# --------------------------------------------------------------------------------------
+# timing of one entry point, and the five workload shapes
+# --------------------------------------------------------------------------------------
+
+def time_back_to_back(fn, stream, inner: int = 20, outer: int = 7) -> float:
+    """Microseconds per call when `inner` calls are enqueued back to back (what a stream of
+    rounds sees): one event pair around the batch, median over `outer` batches."""
+    import torch
+    fn(0)
+    out = []
+    k = 1
+    for _ in range(outer):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(inner):
+            fn(k)
+            k += 1
+        e1.record(stream)
+        torch.cuda.synchronize()
+        out.append(e0.elapsed_time(e1) / inner * 1e3)
+    return statistics.median(out)
+
+
+def time_isolated(fn, stream, reps: int = 25) -> float:
+    """Microseconds of one call on an idle GPU: every call between its own pair of events
+    (the pair itself costs a few microseconds), median over `reps` calls."""
+    import torch
+    fn(0)
+    out = []
+    for k in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        fn(k + 1)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        out.append(e0.elapsed_time(e1) * 1e3)
+    return statistics.median(out)
+
+
+def n_copies(bytes_per_copy: int) -> int:
+    """Device copies of an input set to rotate through: at least four while the set is smaller
+    than 256 MB (then L2 could serve a repeated one), enough to reach 512 MB, at most 16."""
+    if bytes_per_copy >= 256e6:
+        return 2
+    return int(max(4, min(16, 512e6 // max(bytes_per_copy, 1) + 1)))
+
+
+def measure_config(gs, cfg_id: int, seed: int, dev, peak_gbs: float, gs_count=None):
+    """Every entry point of the hot path on one workload shape at full size."""
+    import torch
+    from paper_2605_16867_b200 import InstancePool
+    wl = W.make_workload(cfg_id, seed=seed)
+    N, M, A, Tn = wl.requests.n, wl.instances.n_instances, wl.active.n, wl.types.n_types
+    alpha = wl.ema_alpha
+    stream = torch.cuda.current_stream(dev)
+    pool = InstancePool.from_host(wl.types, wl.instances, dev)
+    res = {"n_requests": N, "n_instances": M, "n_types": Tn, "n_active": A}
+
+    # ---- the routing round -------------------------------------------------------------
+    nc = n_copies(24 * N)
+    reqs = [[torch.from_numpy(c).to(dev) for c in wl.requests.columns()] for _ in range(nc)]
+    outs = [(torch.empty(N, dtype=torch.int32, device=dev), torch.empty(N, dtype=torch.float32, device=dev),
+             torch.empty(N, dtype=torch.float32, device=dev)) for _ in range(nc)]
+    tier = torch.empty(N, dtype=torch.uint8, device=dev)
+    route = lambda k: gs.route_batch(*reqs[k % nc], pool, alpha, *outs[k % nc], None, stream=stream)   # noqa: E731
+    for k in range(3):
+        route(k)
+    t_b2b = time_back_to_back(route, stream)
+    t_iso = time_isolated(route, stream)
+    gs.timing_enable(True)
+    for k in range(20):
+        route(k)
+    torch.cuda.synchronize(dev)
+    t_pro, t_rt = gs.timing_read(KERNEL_NAMES.index("prologue")), gs.timing_read(KERNEL_NAMES.index("route"))
+    gs.timing_enable(False)
+    gs.route_batch(*reqs[0], pool, alpha, *outs[0], tier, stream=stream)
+    torch.cuda.synchronize(dev)
+    hist = torch.bincount(tier.to(torch.int64), minlength=4).cpu().tolist()
+    by = ROUTE_BYTES_PER_REQUEST * N + 20 * M
+    res["route"] = {
+        "call_us": t_b2b, "call_us_isolated": t_iso, "input_copies_rotated": nc,
+        "requests_per_s": N / (t_b2b * 1e-6), "logical_pairs_per_s": N * M / (t_b2b * 1e-6),
+        "algorithmic_GBps": by / (t_b2b * 1e-6) / 1e9, "frac_of_hbm_peak": by / (t_b2b * 1e-6) / 1e9 / peak_gbs,
+        "frac_of_hbm_peak_isolated": by / (t_iso * 1e-6) / 1e9 / peak_gbs,
+        "kernel_us": {"prologue": t_pro[0] / t_pro[1] * 1e3, "route": t_rt[0] / t_rt[1] * 1e3},
+        "tier_histogram": {"just_enough": hist[1], "fallback_kv_ok": hist[2], "fallback_any": hist[3]},
+    }
+    if gs_count is not None:
+        # the search's work per request, from the counting build (same kernels, counters on)
+        gs_count.eval_counters(clear=True)
+        gs_count.route_batch(*reqs[0], pool, alpha, *outs[0], None, stream=stream)
+        c = gs_count.eval_counters(clear=True)
+        res["route"]["evaluated_per_request"] = {
+            "pairs_scored_exactly": c[0] / N, "row_bounds_tested": c[1] / N, "type_bounds_tested": c[2] / N,
+            "logical_pairs": M, "share_left_to_full_search": c[3] / N, "share_fallback": c[4] / N,
+            "share_scored_by_a_whole_warp": c[5] / N}
+    del reqs, outs, tier
+
+    # ---- the risk scan -------------------------------------------------------------------
+    nc = n_copies(20 * A)
+    acts = [[torch.from_numpy(c).to(dev) for c in wl.active.columns()] for _ in range(nc)]
+    bits = torch.empty((A + 31) // 32, dtype=torch.int32, device=dev)
+    cand = torch.empty(A, dtype=torch.int32, device=dev)
+    count = torch.zeros(1, dtype=torch.int64, device=dev)
+    scan = lambda k: gs.risk_scan(*acts[k % nc], pool, bits, cand, count, stream=stream)   # noqa: E731
+    for k in range(3):
+        scan(k)
+    t_b2b = time_back_to_back(scan, stream)
+    t_iso = time_isolated(scan, stream)
+    gs.timing_enable(True)
+    for k in range(20):
+        scan(k)
+    torch.cuda.synchronize(dev)
+    t_fl, t_sc = gs.timing_read(KERNEL_NAMES.index("risk_flags")), gs.timing_read(KERNEL_NAMES.index("risk_scatter"))
+    gs.timing_enable(False)
+    flagged = int(count.item())
+    by = RISK_BYTES_PER_REQUEST * A + 4 * flagged
+    res["risk_scan"] = {
+        "call_us": t_b2b, "call_us_isolated": t_iso, "input_copies_rotated": nc, "flagged_fraction": flagged / A,
+        "requests_per_s": A / (t_b2b * 1e-6), "algorithmic_GBps": by / (t_b2b * 1e-6) / 1e9,
+        "frac_of_hbm_peak": by / (t_b2b * 1e-6) / 1e9 / peak_gbs,
+        "frac_of_hbm_peak_isolated": by / (t_iso * 1e-6) / 1e9 / peak_gbs,
+        "kernel_us": {"risk_flags": t_fl[0] / t_fl[1] * 1e3, "risk_scatter": t_sc[0] / t_sc[1] * 1e3},
+    }
+
+    # ---- config 4: the stream of dependent rounds (route + advance, a scan after every round) ----
+    if wl.cfg.n_rounds > 1:
+        R = wl.cfg.n_rounds
+        rounds = [[torch.from_numpy(c).to(dev) for c in W.make_round_requests(wl, k).columns()] for k in range(R)]
+        o_idx = torch.empty(N, dtype=torch.int32, device=dev)
+        o_est = torch.empty(N, dtype=torch.float32, device=dev)
+        o_slack = torch.empty(N, dtype=torch.float32, device=dev)
+        state0 = InstancePool.from_host(wl.types, wl.instances, dev)
+        live = InstancePool.from_host(wl.types, wl.instances, dev)
+
+        def reset_state():
+            for name in ("queued_prefill_tokens", "decode_batch", "free_kv_tokens", "q_ema_ms"):
+                getattr(live, name).copy_(getattr(state0, name))
+
+        def enqueue_stream(st):
+            for k in range(R):
+                gs.route_batch(*rounds[k], live, alpha, o_idx, o_est, o_slack, None, accumulate=True, stream=st)
+                gs.advance_state(live, stream=st)
+                gs.risk_scan(*acts[k % nc], live, bits, cand, count, stream=st)
+
+        side = torch.cuda.Stream(dev)
+        how = "CUDA graph of the 64 rounds, replayed"
+        graph = None
+        try:
+            reset_state()
+            torch.cuda.synchronize(dev)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                enqueue_stream(side)
+        except Exception as exc:                      # capture refused: enqueue the rounds one by one
+            graph = None
+            how = "rounds enqueued one by one from the host (graph capture failed: %s)" % type(exc).__name__
+        torch.cuda.synchronize(dev)
+        times = []
+        for _ in range(7):
+            reset_state()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(dev)
+            e0.record(stream)
+            if graph is not None:
+                graph.replay()
+            else:
+                enqueue_stream(stream)
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            times.append(e0.elapsed_time(e1))
+        ms = statistics.median(times)
+        res["stream"] = {"rounds": R, "ms": ms, "us_per_round": ms / R * 1e3, "how": how,
+                         "requests_per_s": R * N / (ms * 1e-3), "logical_pairs_per_s": R * N * M / (ms * 1e-3),
+                         "scans": R, "scan_requests_per_s": R * A / (ms * 1e-3),
+                         "what": "per round: gs_route_batch(ACCUMULATE) + gs_advance_state + gs_risk_scan over the advanced state"}
+    status = gs.device_status()
+    res["device_status"] = status
+    return res
 
 
 # --------------------------------------------------------------------------------------
@@ -247,6 +443,8 @@ def run_gpu(args):
     alpha = wl.ema_alpha
 
     gs = GoodServe(local_rank)
+    props = torch.cuda.get_device_properties(dev)
+    n_sm = int(props.multi_processor_count)
     pool = InstancePool.from_host(wl.types, wl.instances, dev)
     req = [torch.from_numpy(c).to(dev) for c in wl.requests.columns()]
     act = [torch.from_numpy(c).to(dev) for c in wl.active.columns()]
@@ -398,6 +596,22 @@ def run_gpu(args):
                       "ns_per_request": ms / n_l * 1e6 / n_seq}
         del seq_pool
         gs.route_batch(*req, pool, alpha, out_idx, out_est, out_slack, None, stream=stream)   # outputs of the timed step
+    # ---- every workload shape, each entry point by itself (rank 0 of a one-GPU run) ----
+    peak, peak_kind = load_peaks()
+    per_config = None
+    if world == 1 and not args.no_per_config:
+        gs_count = None
+        if not args.no_count:
+            try:
+                gs_count = GoodServe(local_rank, counting=True)
+            except Exception as exc:                   # the counting build is optional equipment
+                print(f"counting build unavailable: {exc}", file=sys.stderr)
+        per_config = {}
+        for cid in sorted(W.CONFIGS):
+            per_config[str(cid)] = measure_config(gs, cid, rank_seed(cid, rank), dev, peak, gs_count)
+            torch.cuda.empty_cache()
+        if gs_count is not None:
+            gs_count.close()
     t_wait = time.perf_counter()
     while len(sampler.rows) < 4 and time.perf_counter() - t_wait < 3.0:
         step()                                   # keep the same load up for the sampler (untimed)
@@ -448,7 +662,8 @@ def run_gpu(args):
         return
 
     # ---- roofline of the dominant kernel ---------------------------------------------
-    peak, peak_kind = load_peaks()
+    sm_max_hz = (clocks.get("sm_max_mhz") or 1965.0) * 1e6
+    issue_peak = n_sm * SCHEDULERS_PER_SM * sm_max_hz      # SM count from the device, clock from nvidia-smi
     per_kernel = {}
     for name, (ms, n) in kernel_ms.items():
         per_kernel[name] = {"launches": n, "avg_us": ms / n * 1e3}
@@ -473,10 +688,11 @@ def run_gpu(args):
     if profiled and "route" in kernel_ms:
         ms, n = kernel_ms["route"]
         rate = profiled["warp_instructions_per_launch"] / (ms / n * 1e-3)
-        issue = {"kernel": "route", "bound": "alu", "achieved": rate, "peak": ISSUE_PEAK_WARP_INST_PER_S,
-                 "unit": "warp-instructions/s", "frac": rate / ISSUE_PEAK_WARP_INST_PER_S,
+        issue = {"kernel": "route", "bound": "alu", "achieved": rate, "peak": issue_peak,
+                 "unit": "warp-instructions/s", "frac": rate / issue_peak,
                  "warp_instructions_per_request": profiled["warp_instructions_per_launch"] / N,
-                 "note": "instruction count from ncu; peak = 148 SMs x 4 schedulers x 1.965 GHz"}
+                 "note": "instruction count from ncu; peak = %d SMs x %d schedulers x %.3f GHz" % (
+                     n_sm, SCHEDULERS_PER_SM, sm_max_hz / 1e9)}
     for name in per_kernel:
         if name in alg_bytes:
             gbs = alg_bytes[name] / (per_kernel[name]["avg_us"] * 1e-6) / 1e9
@@ -499,12 +715,26 @@ def run_gpu(args):
                    "streams": 1 if args.serial else 2,
                    "per_rank_seed": "config id + 1000 * rank", "sharding": "independent batches per rank, no collective"},
         "risk_scan_requests_per_s": world * A / (risk_ms * 1e-3) if risk_ms else None,
-        "route_pairs_per_s": world * N * M / (route_ms * 1e-3) if route_ms else None,
+        "value_note": "logical pairs: N x M per routing round -- pairs decided, not pairs scored; the search scores "
+                      "about one pair per request exactly (per_config.*.route.evaluated_per_request)",
+        "route_logical_pairs_per_s": world * N * M / (route_ms * 1e-3) if route_ms else None,
         "route_requests_per_s": world * N / (route_ms * 1e-3) if route_ms else None,
         "step_hbm_frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "flagged_fraction": flagged / A, "device_status": status,
-        "roofline": roofline, "issue": issue, "kernels": per_kernel, "reroute": reroute, "prefix": prefix, "direct": direct, "sequential": sequential,
-        "kernel_timing": "serial pass of %d steps on one stream after the timed region, %.4f ms/step" % (
+        "roofline": roofline, "issue": issue, "kernels": per_kernel,
+        "route_call": None if not per_config else {
+            "us": per_config[str(args.config)]["route"]["call_us"],
+            "algorithmic_GBps": per_config[str(args.config)]["route"]["algorithmic_GBps"],
+            "frac_of_hbm_peak": per_config[str(args.config)]["route"]["frac_of_hbm_peak"],
+            "what": "gs_route_batch (prologue + route kernel) called back to back, inputs rotated"},
+        "scan_call": None if not per_config else {
+            "us": per_config[str(args.config)]["risk_scan"]["call_us"],
+            "algorithmic_GBps": per_config[str(args.config)]["risk_scan"]["algorithmic_GBps"],
+            "frac_of_hbm_peak": per_config[str(args.config)]["risk_scan"]["frac_of_hbm_peak"],
+            "what": "gs_risk_scan (both passes) called back to back, inputs rotated"},
+        "per_config": per_config, "reroute": reroute, "prefix": prefix, "direct": direct, "sequential": sequential,
+        "kernel_timing": "serial pass of %d steps on one stream after the timed region, every launch between its own "
+                         "pair of CUDA events (the pair adds about 3 us to each duration), %.4f ms/step" % (
             args.steps, serial_ms_per_step),
         "e2e": None if args.no_e2e else
                {"value": e2e_pairs / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -531,6 +761,8 @@ def main():
     ap.add_argument("--no-direct", action="store_true", help="skip the untimed black-box-table routing measurement")
     ap.add_argument("--no-sequential", action="store_true", help="skip the untimed one-at-a-time routing measurement")
     ap.add_argument("--no-prefix", action="store_true", help="skip the untimed prefix-cache routing measurement")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the per-config block (all five workload shapes)")
+    ap.add_argument("--no-count", action="store_true", help="skip the counting build (work per request)")
     ap.add_argument("--serial", action="store_true", help="route and scan on one stream instead of two")
     ap.add_argument("--print-kernel-hash", action="store_true", help="print the hash PROFILED_ROUTE refers to")
     args = ap.parse_args()

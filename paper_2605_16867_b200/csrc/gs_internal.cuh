@@ -114,7 +114,8 @@ struct Scratch {
     TypeHeader *headers;      // [GS_MAX_TYPES] in search order (largest d first)
     int *table_info;          // {padded rows, unsafe, n_instances, n_active_types, bits of the candidate
                               //  table's origin (least d_lo of any type), bits of its slots per unit of d,
-                              //  pool entries handed out to the types, 1 = q_by_g holds a round to carry}
+                              //  pool entries handed out to the types, 1 = q_by_g holds a round to carry,
+                              //  the most free KV of any instance}
     unsigned short *cand_table;   // [kCandSlots] candidate types by slot of D / L_out
     uint2 *pool;              // [kPoolEntries] record lists
     unsigned short *bucket_list;  // [GS_MAX_TYPES * kStartBuckets] first pool entry of the list, halved; kNoList = none

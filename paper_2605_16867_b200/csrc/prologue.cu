@@ -127,6 +127,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     __shared__ unsigned sh_dmax[GS_MAX_TYPES], sh_dmin[GS_MAX_TYPES];      // by type: largest / least d
     __shared__ unsigned sh_dlow_pos[GS_MAX_TYPES];                         // least d by position in the search order
     __shared__ unsigned sh_qmin, sh_pmin;
+    __shared__ int sh_kvmax;                                               // most free KV of any instance
     __shared__ float sh_tp[GS_MAX_TYPES], sh_ta[GS_MAX_TYPES], sh_tb[GS_MAX_TYPES];   // type constants
     __shared__ int sh_unsafe, sh_fill;
     __shared__ int sh_len[kPrologueThreads / 32], sh_off[kPrologueThreads / 32], sh_pool_used;
@@ -152,12 +153,13 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         if (tid < n_types) { sh_tp[tid] = p_type[tid]; sh_ta[tid] = a_type[tid]; sh_tb[tid] = b_type[tid]; }
     }
     if (tid < GS_MAX_TYPES) { sh_cnt[tid] = 0; sh_dmax[tid] = 0u; sh_dmin[tid] = 0xFFFFFFFFu; }
-    if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; sh_pmin = 0xFFFFFFFFu; }
+    if (tid == 0) { sh_unsafe = 0; sh_fill = 0; sh_qmin = 0xFFFFFFFFu; sh_pmin = 0xFFFFFFFFu; sh_kvmax = 0; }
     __syncthreads();
 
     int base = 0, n_act = 0, padded_total = 0, n_t = 0;
     int pool_base = 0, pool_share = 0, pool_total = 0;     // record lists: this type's part of the pool
     float p_group = 0.f;                       // lower bound source: the least p of the group
+    int my_kv = 0;                             // free KV of this thread's instance
 
     if (kDirect) {
         // ---- 1. the coefficients as given (thread g owns instance g) ---------------------------
@@ -168,6 +170,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         if (has) {
             q = q_in[tid]; pv = p_in[tid]; d = d_in[tid];
             const int kv = clamp_count(free_kv[tid], bad);
+            my_kv = kv;
             if (!(q >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; q = 0.0f; }
             if (!(pv >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; pv = 0.0f; }
             if (!(d >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; d = 0.0f; }
@@ -178,6 +181,10 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             }
             const float big = 3.0e38f;           // the bounds need finite coefficients
             if (!(q < big && pv < big && d < big)) atomicOr(&sh_unsafe, 1);
+        }
+        {
+            const int wmax = __reduce_max_sync(0xFFFFFFFFu, my_kv);
+            if (lane == 0 && wmax > 0) atomicMax(&sh_kvmax, wmax);
         }
         // ---- 2. preference order of the whole pool, cut into groups of consecutive rank -------
         int n_sort = 32;
@@ -214,6 +221,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 float qe = r_qema;
                 if (!(qe >= 0.0f)) { bad |= GS_DEV_BAD_VALUE; qe = 0.0f; }
                 const int kv = clamp_count(r_kv, bad);
+                my_kv = kv;
                 const float p = sh_tp[t];
                 d = __fmaf_rn(sh_tb[t], B, sh_ta[t]);               // loaded per-token decode latency
                 const float w = __fmul_rn(Qtok, p);                 // time to drain the queued prefill
@@ -242,6 +250,8 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 const unsigned mn = __reduce_min_sync(0xFFFFFFFFu, is ? od : 0xFFFFFFFFu);
                 if (lane == o) { w_cnt = c; w_max = mx; w_min = mn; }
             }
+            const int wmax = __reduce_max_sync(0xFFFFFFFFu, my_kv);
+            if (lane == 0 && wmax > 0) atomicMax(&sh_kvmax, wmax);
             if (w_cnt > 0) {
                 atomicAdd(&sh_cnt[lane], w_cnt);
                 atomicMax(&sh_dmax[lane], w_max);
@@ -326,6 +336,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         s.table_info[3] = n_act;
         s.table_info[6] = pool_total;
         if (carry_q) s.table_info[7] = 1;      // a round whose q_g is to be carried is pending
+        s.table_info[8] = sh_kvmax;            // no instance has more free KV than this
         if (sh_unsafe) atomicOr(s.status, (unsigned)GS_DEV_BAD_VALUE);
     }
     if (writer && bad) atomicOr(s.status, bad);

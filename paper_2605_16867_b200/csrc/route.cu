@@ -259,14 +259,16 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
 // Returns -1 with tier 0 only when kCapped and no instance has d < d_cap.
 struct Pick { int g; float T; unsigned tier; };
 
+// `first_pass` = 1 skips the pass over instances with KV room (the caller knows there is none).
 template <bool kCapped, bool kRowP>
-__device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y, unsigned need, float d_cap)
+__device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y, unsigned need, float d_cap,
+                                              int first_pass = 0)
 {
     unsigned tier_out = 0;
     int g_best = -1;
     float T_best = __int_as_float(0x7F800000);            // +inf
 #pragma unroll 1
-    for (int pass = 0; pass < 2 && g_best < 0; ++pass) {  // pass 0: instances with KV room only
+    for (int pass = first_pass; pass < 2 && g_best < 0; ++pass) {  // pass 0: instances with KV room only
         const bool any_kv = pass == 1;
 #pragma unroll 1
         for (int t = tb.n_types - 1; t >= 0; --t) {
@@ -588,15 +590,18 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
 // the just-enough pick over all types, then the fallback of Algorithm 1 -- by the lane itself
 // when several lanes need it, by the whole warp otherwise and for requests that the tables
 // cannot serve (L_out == 0, unusable coefficients).
+// A request that needs more KV than any instance has free (need > kv_max) cannot be served in
+// tier 1 or 2: it goes straight to the minimum of T over all instances (tier 3).
 template <bool kRowP>
-__device__ __noinline__ Pick full_pick(const Tables tb, int M, int lane, bool active, int xi, int yi, float D)
+__device__ __noinline__ Pick full_pick(const Tables tb, int M, unsigned kv_max, int lane, bool active, int xi, int yi, float D)
 {
     const unsigned need = (unsigned)xi + (unsigned)yi;      // < 2^32, no overflow
+    const bool room_somewhere = need <= kv_max;
     const float x = __int2float_rn(xi), y = __int2float_rn(yi);
     // an empty lane, or L_out == 0 (the start table divides by it), skips the search; the hair
     // added to the deadline of the bound tests keeps them safe when a bound's tag bits make a
     // zero coefficient a denormal
-    const float Dj = (active && yi > 0) ? D : -1.0f;
+    const float Dj = (active && yi > 0 && room_somewhere) ? D : -1.0f;
     Pick out;
     out.T = 0.f;
     out.g = pick_instance<false, kRowP>(tb, x, y, Dj, Dj + 1e-30f, need, 0.f, out.T);
@@ -606,7 +611,7 @@ __device__ __noinline__ Pick full_pick(const Tables tb, int M, int lane, bool ac
     const int n_fall = __popc(__ballot_sync(0xFFFFFFFFu, mine));
     if (mine && n_fall >= kThreadFallbackMin) {
         GS_COUNT(kCountFallback, 1);
-        out = fallback_pick<false, kRowP>(tb, x, y, need, 0.f);
+        out = fallback_pick<false, kRowP>(tb, x, y, need, 0.f, room_somewhere ? 0 : 1);
         open = false;
     }
     unsigned todo = __ballot_sync(0xFFFFFFFFu, open);
@@ -773,6 +778,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         }
     }
     const int M = im.info[2];
+    const unsigned kv_max = (unsigned)im.info[8];         // no instance has more free KV than this
     const float cand_z0 = __int_as_float(im.info[4]), cand_inv = __int_as_float(im.info[5]);
     Tables tb;
     tb.headers = im.headers; tb.row_bounds = im.row_bounds; tb.group_bounds = im.group_bounds;
@@ -790,7 +796,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
         int4 e = make_int4(0, 0, 0, 0);
         float D = -1.0f;
         if (active) { e.x = max(prompt_len[r], 0); e.y = max(pred_decode_len[r], 0); D = slo_ms[r]; }
-        const Pick pk = full_pick<kRowP>(tb, M, lane, active, e.x, e.y, D);
+        const Pick pk = full_pick<kRowP>(tb, M, kv_max, lane, active, e.x, e.y, D);
         int g = pk.g; float T = pk.T; unsigned tier = pk.tier;
         if (kPrefix && active)
             for (int k = 0; k < hits.n_slots; ++k)
@@ -850,7 +856,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             // (an empty slot, or L_out == 0, which the start table cannot take, gets a deadline that
             // nothing meets and so ends up in the full search)
             bool settled = false;
-            if (fast_on)
+            if (fast_on && (unsigned)xi[j] + (unsigned)yi[j] <= kv_max)
                 settled = fast_pick<kRowP>(tb, cand_z0, cand_inv, __int2float_rn(xi[j]), __int2float_rn(yi[j]),
                                            (valid && yi[j] > 0) ? D[j] : -1.0f, (unsigned)xi[j] + (unsigned)yi[j], g_out[j], T_out[j]);
             if (valid && !settled) { slow |= 1u << j; GS_COUNT(kCountQueued, 1); }
@@ -1014,6 +1020,18 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
 // into the request that a token-ID migration would pose to the target (re-prefill prompt +
 // generated tokens, decode what is left, within the time that is left) and runs the same
 // search as the routing round, restricted to instances with d < d of the current instance.
+// Candidates for which that search finds no feasible faster instance (nearly half of them at
+// config 3) need Algorithm 1's fallback, a much longer search: their positions go on the warp's
+// queue, and whenever 32 have gathered each lane takes one of them through the fallback, so that
+// the long path runs with all lanes busy instead of the few of each 32 that need it.
+constexpr int kRerouteQueue = 64;           // per warp: at most 31 left over + the 32 of a step
+
+struct Candidate {
+    float x, y, D, d_cap;
+    unsigned need, rem;
+    bool valid;
+};
+
 __global__ void __launch_bounds__(kRerouteThreads, 4)
 reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__ cand_count, int64_t cand_capacity,
                const int32_t *__restrict__ assigned, const int32_t *__restrict__ generated,
@@ -1030,64 +1048,100 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
     extern __shared__ __align__(16) unsigned char smem[];
     asm volatile("griddepcontrol.wait;" ::: "memory");       // (the tables are the prologue's)
     const int M = table_info[2];
+    const unsigned kv_max = (unsigned)table_info[8];      // no instance has more free KV than this
     Tables tb;
-    stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_group_bounds, g_start_table, g_headers, table_info, tb);
+    unsigned char *after = stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_group_bounds, g_start_table, g_headers,
+                                        table_info, tb);
+    unsigned *queue = reinterpret_cast<unsigned *>(after) + (threadIdx.x >> 5) * kRerouteQueue;
     __syncthreads();
 
     int64_t n = *cand_count;
     if (n > cand_capacity) n = cand_capacity;
     const int lane = threadIdx.x & 31;
     unsigned bad = 0;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31); base < n; base += stride) {
-        const int64_t j = base + lane;
-        const bool valid = j < n;
+    int q_count = 0;                               // entries on this warp's queue (same in all lanes)
+
+    // the request that candidate j poses (j < n < 2^31)
+    auto load_candidate = [&](int64_t j, bool valid) {
+        Candidate c;
         int64_t i = valid ? (int64_t)cand_idx[j] : 0;
         if (i < 0 || i >= n_active) { i = 0; if (valid) bad |= GS_DEV_BAD_INSTANCE; }
-        int c = assigned[i], gen = generated[i], tot = pred_len[i], xin = prompt_len[i];
-        if (c < 0) { c = 0; bad |= GS_DEV_BAD_INSTANCE; }
-        if (c >= M) { c = M - 1; bad |= GS_DEV_BAD_INSTANCE; }
+        int cur = assigned[i], gen = generated[i], tot = pred_len[i], xin = prompt_len[i];
+        if (cur < 0) { cur = 0; bad |= GS_DEV_BAD_INSTANCE; }
+        if (cur >= M) { cur = M - 1; bad |= GS_DEV_BAD_INSTANCE; }
         if (gen < 0) { gen = 0; bad |= GS_DEV_BAD_VALUE; }
         if (tot < 0) { tot = 0; bad |= GS_DEV_BAD_VALUE; }
         if (xin < 0) { xin = 0; bad |= GS_DEV_BAD_VALUE; }
-        const unsigned rem = (unsigned)max(tot - gen, 0);
+        c.rem = (unsigned)max(tot - gen, 0);
         const unsigned xu = (unsigned)xin + (unsigned)gen;                    // < 2^32
-        const unsigned long long need64 = (unsigned long long)xu + rem;
-        const unsigned need = need64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (unsigned)need64;   // kv < 2^31 anyway
-        const float x = __uint2float_rn(xu), y = __uint2float_rn(rem);
-        const float D = __fsub_rn(slo[i], elapsed[i]);                        // time left
-        const float d_cap = tb.rows[row_pos(c)].d;
-        float T = 0.f;
-        const float Ds = (valid && rem > 0) ? D : -1.0f;      // see route_kernel: L_out == 0 skips the search
-        int g = pick_instance<true, false>(tb, x, y, Ds, Ds + 1e-30f, need, d_cap, T);
-        unsigned tier = 1;
-        bool settled = g >= 0;
-        const bool fall = valid && !settled && rem > 0 && tb.n_types > 0;
-        const int n_fall = __popc(__ballot_sync(0xFFFFFFFFu, fall));           // all lanes vote
-        if (fall && n_fall >= kThreadFallbackMin) {
-            const Pick r = fallback_pick<true, false>(tb, x, y, need, d_cap);
+        const unsigned long long need64 = (unsigned long long)xu + c.rem;
+        c.need = need64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (unsigned)need64;     // kv < 2^31 anyway
+        c.x = __uint2float_rn(xu); c.y = __uint2float_rn(c.rem);
+        c.D = __fsub_rn(slo[i], elapsed[i]);                                  // time left
+        c.d_cap = tb.rows[row_pos(cur)].d;
+        c.valid = valid;
+        return c;
+    };
+    auto store = [&](int64_t j, int g, float T, unsigned tier, float D) {
+        out_inst[j] = g;
+        out_est[j] = T;
+        out_slack[j] = tier ? __fsub_rn(D, T) : 0.f;
+        if (out_tier) out_tier[j] = (uint8_t)tier;
+    };
+    // the fallback for (up to) the newest 32 candidates of the queue, one per lane
+    auto drain = [&]() {
+        const int cnt = min(q_count, 32);
+        q_count -= cnt;
+        const bool active = lane < cnt;
+        const int64_t j = active ? (int64_t)queue[q_count + lane] : 0;
+        __syncwarp();                              // the slots may be written again
+        const Candidate c = load_candidate(j, active);
+        int g = -1; float T = 0.f; unsigned tier = 0;
+        bool settled = !active;
+        if (active && c.rem > 0 && tb.n_types > 0) {
+            const Pick r = fallback_pick<true, false>(tb, c.x, c.y, c.need, c.d_cap, c.need <= kv_max ? 0 : 1);
             g = r.g; T = r.T; tier = r.tier;                                // may settle on "no move"
             settled = true;
         }
-        unsigned todo = __ballot_sync(0xFFFFFFFFu, valid && !settled);
+        // what the tables cannot serve (nothing left to decode, unusable coefficients): the whole
+        // warp scores every instance
+        unsigned todo = __ballot_sync(0xFFFFFFFFu, !settled);
         while (todo) {
             const int src = __ffs(todo) - 1;
             todo &= todo - 1;
-            const float xs = __shfl_sync(0xFFFFFFFFu, x, src), ys = __shfl_sync(0xFFFFFFFFu, y, src);
-            const float Dsrc = __shfl_sync(0xFFFFFFFFu, D, src), caps = __shfl_sync(0xFFFFFFFFu, d_cap, src);
-            const unsigned needs = __shfl_sync(0xFFFFFFFFu, need, src);
+            const float xs = __shfl_sync(0xFFFFFFFFu, c.x, src), ys = __shfl_sync(0xFFFFFFFFu, c.y, src);
+            const float Dsrc = __shfl_sync(0xFFFFFFFFu, c.D, src), caps = __shfl_sync(0xFFFFFFFFu, c.d_cap, src);
+            const unsigned needs = __shfl_sync(0xFFFFFFFFu, c.need, src);
             int gg; float TT; unsigned tt;
             exhaustive_pick<true>(tb.rows, M, xs, ys, Dsrc, needs, caps, lane, gg, TT, tt);
             if (lane == src) { g = gg; T = TT; tier = tt; }
         }
-        if (valid) {
-            out_inst[j] = g;
-            out_est[j] = T;
-            out_slack[j] = tier ? __fsub_rn(D, T) : 0.f;
-            if (out_tier) out_tier[j] = (uint8_t)tier;
-        }
+        if (active) store(j, g, T, tier, c.D);
+    };
+
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31); base < n; base += stride) {
+        const int64_t j = base + lane;
+        const Candidate c = load_candidate(j, j < n);
+        float T = 0.f;
+        // (see route_kernel: L_out == 0 skips the search; so does a request that fits no instance's free KV)
+        const float Ds = (c.valid && c.rem > 0 && c.need <= kv_max) ? c.D : -1.0f;
+        const int g = pick_instance<true, false>(tb, c.x, c.y, Ds, Ds + 1e-30f, c.need, c.d_cap, T);
+        if (c.valid && g >= 0) store(j, g, T, 1u, c.D);
+        // the rest is queued for the fallback
+        const bool push = c.valid && g < 0;
+        const unsigned votes = __ballot_sync(0xFFFFFFFFu, push);
+        if (push) queue[q_count + __popc(votes & ((1u << lane) - 1u))] = (unsigned)j;
+        q_count += __popc(votes);
+        __syncwarp();
+        while (q_count >= 32) drain();
     }
+    while (q_count > 0) drain();
     if (bad) atomicOr(status, bad);
+}
+
+static size_t reroute_smem_bytes(int n_types) {       // the tables of n_types types and the warps' queues
+    return kTablesSmemFixed + kRouteSmemPerType * n_types + (size_t)(kRerouteThreads / 32) * kRerouteQueue * sizeof(unsigned);
 }
 
 cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,
@@ -1097,7 +1151,7 @@ cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *
                            cudaStream_t st)
 {
     if (cand_capacity == 0) return cudaSuccess;
-    const size_t smem = kTablesSmemFixed + kRouteSmemPerType * n_types;
+    const size_t smem = reroute_smem_bytes(n_types);
     int64_t blocks = (cand_capacity + kRerouteThreads - 1) / kRerouteThreads;
     const int64_t cap = (int64_t)ctx->n_sm * ctx->reroute_ctas_per_sm[n_types];
     if (blocks > cap) blocks = cap;
@@ -1134,12 +1188,12 @@ cudaError_t configure_route(gs_ctx *ctx)
     e = configure_route_kernels<4>();
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(kTablesSmemFixed + kRouteSmemPerType * GS_MAX_TYPES));
+                             (int)reroute_smem_bytes(GS_MAX_TYPES));
     if (e != cudaSuccess) return e;
     for (int t = 0; t <= GS_MAX_TYPES; ++t) {
         int occ = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, reroute_kernel, kRerouteThreads,
-                                                          kTablesSmemFixed + kRouteSmemPerType * t);
+                                                          reroute_smem_bytes(t));
         if (e != cudaSuccess) return e;
         ctx->reroute_ctas_per_sm[t] = occ > 0 ? occ : 1;
     }
