@@ -181,9 +181,14 @@ risk_flags_kernel(const int32_t *__restrict__ assigned, const int32_t *__restric
     if (bad) atomicOr(status, bad);
 }
 
-constexpr int kScatterBlocks = 4;           // blocks of 32 flag words (1024 requests) per warp and round
+#ifndef GS_SCATTER_THREADS
+#define GS_SCATTER_THREADS 512
+#endif
+constexpr int kScatterThreads = GS_SCATTER_THREADS;      // pass 2 runs more warps per CTA than pass 1: it is bound by latency
+constexpr int kScatterWarps = kScatterThreads / 32;
+constexpr int kScatterBlocks = 32 / kScatterWarps;        // blocks of 32 flag words (1024 requests) per warp and round: 32 blocks a round
 
-__global__ void __launch_bounds__(kRiskThreads)
+__global__ void __launch_bounds__(kScatterThreads, 2048 / kScatterThreads)
 scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_words,
                           const unsigned *__restrict__ cta_counts, int64_t n_steps,
                           int32_t *__restrict__ cand_idx, int64_t cand_capacity,
@@ -191,11 +196,11 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
 {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    __shared__ unsigned sh_part[kRiskWarps];
-    __shared__ unsigned sh_cnt[2][kRiskWarps * kScatterBlocks];
-    __shared__ uint2 sh_words[kRiskWarps][32];
-    // the CTA's run of flag words; a round covers 8 warps x 4 blocks of 32 words, warp w the
-    // blocks w, w + 8, w + 16, w + 24 of the round
+    __shared__ unsigned sh_part[kScatterWarps];
+    __shared__ unsigned sh_cnt[2][kScatterWarps * kScatterBlocks];
+    __shared__ uint2 sh_words[kScatterWarps][32];
+    // the CTA's run of flag words; a round covers 32 blocks of 32 words, warp w the blocks
+    // w, w + kScatterWarps, .. of the round
     const int64_t w_begin = first_step_of(blockIdx.x, n_steps, gridDim.x) << 2;
     const int64_t w_end = min(first_step_of((int64_t)blockIdx.x + 1, n_steps, gridDim.x) << 2, n_words);
     // everything read below is written by pass 1: wait until that grid is done and visible
@@ -203,29 +208,29 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
 
     // flags before this CTA's run: the counts of the CTAs before it (fewer than 2^31 in all)
     unsigned part = 0;
-    for (int k = threadIdx.x; k < (int)blockIdx.x; k += kRiskThreads) part += __ldcg(cta_counts + k);
+    for (int k = threadIdx.x; k < (int)blockIdx.x; k += kScatterThreads) part += __ldcg(cta_counts + k);
     part = __reduce_add_sync(0xFFFFFFFFu, part);
     if (lane == 0) sh_part[warp] = part;
 
     const unsigned lane_bit = 1u << lane, below = lane_bit - 1u;
     int64_t base = 0;
     int buf = 0;
-    for (int64_t w0 = w_begin; w0 < w_end; w0 += kRiskWarps * kScatterBlocks * 32, buf ^= 1) {
+    for (int64_t w0 = w_begin; w0 < w_end; w0 += kScatterWarps * kScatterBlocks * 32, buf ^= 1) {
         uint32_t word[kScatterBlocks];
 #pragma unroll
         for (int k = 0; k < kScatterBlocks; ++k) {
-            const int64_t wi = w0 + (k * kRiskWarps + warp) * 32 + lane;
+            const int64_t wi = w0 + (k * kScatterWarps + warp) * 32 + lane;
             word[k] = wi < w_end ? __ldcs(flag_bits + wi) : 0u;
         }
 #pragma unroll
         for (int k = 0; k < kScatterBlocks; ++k) {
             const unsigned total = __reduce_add_sync(0xFFFFFFFFu, (unsigned)__popc(word[k]));
-            if (lane == 0) sh_cnt[buf][k * kRiskWarps + warp] = total;
+            if (lane == 0) sh_cnt[buf][k * kScatterWarps + warp] = total;
         }
         __syncthreads();                    // (the other buffer is free again after the next barrier)
         if (w0 == w_begin) {
 #pragma unroll
-            for (int w = 0; w < kRiskWarps; ++w) base += sh_part[w];
+            for (int w = 0; w < kScatterWarps; ++w) base += sh_part[w];
         }
         // lane b holds the count of block b of the round: flags before each block, and in all
         const unsigned c = sh_cnt[buf][lane];
@@ -238,7 +243,7 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
         const unsigned all = __shfl_sync(0xFFFFFFFFu, incl, 31);
 #pragma unroll
         for (int k = 0; k < kScatterBlocks; ++k) {
-            const int blk = k * kRiskWarps + warp;
+            const int blk = k * kScatterWarps + warp;
             const unsigned total = __shfl_sync(0xFFFFFFFFu, c, blk);
             const unsigned before = __shfl_sync(0xFFFFFFFFu, incl - c, blk);
             if (total == 0) continue;
@@ -280,7 +285,7 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
     if (w_begin >= w_end) {                 // (a CTA without words still has to know the total if it is the last)
         __syncthreads();
 #pragma unroll
-        for (int w = 0; w < kRiskWarps; ++w) base += sh_part[w];
+        for (int w = 0; w < kScatterWarps; ++w) base += sh_part[w];
     }
     if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {     // the last CTA knows the total
         *cand_count = base;
@@ -338,7 +343,7 @@ static cudaError_t enqueue_scan(unsigned *cta_counts, int dev, int n_sm, gs_ctx 
         LaunchTimer timer(timing_ctx, GS_K_RISK_SCATTER, st);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)blocks);           // the same runs of steps as pass 1
-        cfg.blockDim = dim3(kRiskThreads);
+        cfg.blockDim = dim3(kScatterThreads);
         cfg.dynamicSmemBytes = 0;
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
