@@ -192,6 +192,11 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);
+    if (ctx->host_pipe_ready) {
+        cudaStreamDestroy(ctx->host_out_stream);
+        for (cudaEvent_t ev : ctx->host_events) cudaEventDestroy(ev);
+        cudaFreeHost(ctx->host_counts);
+    }
     delete ctx->pending;
     delete ctx->free_events;
     delete ctx;
@@ -453,6 +458,27 @@ GS_API int gs_reroute_candidates(gs_ctx *ctx, const int32_t *cand_idx, const int
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 
+// The *_host entry points work through their input in pieces: while the kernels of piece k run
+// and its results travel back on a second stream, the inputs of piece k + 1 are already on
+// their way -- the link to the host carries traffic in both directions at once.
+static int ensure_host_pipe(gs_ctx *ctx) {
+    if (ctx->host_pipe_ready) return GS_OK;
+    cudaError_t e = cudaStreamCreateWithFlags(&ctx->host_out_stream, cudaStreamNonBlocking);
+    for (int k = 0; k < GS_HOST_PIECES && e == cudaSuccess; ++k)
+        e = cudaEventCreateWithFlags(&ctx->host_events[k], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaHostAlloc((void **)&ctx->host_counts, GS_HOST_PIECES * sizeof(int64_t), cudaHostAllocDefault);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->host_pipe_ready = true;
+    return GS_OK;
+}
+
+// Requests per piece: a multiple of 1024 (pieces start 16-byte aligned and on whole flag words).
+static int64_t host_piece(int64_t n) {
+    int64_t piece = (n + GS_HOST_PIECES - 1) / GS_HOST_PIECES;
+    if (piece < gs::kHostPieceMin) piece = gs::kHostPieceMin;
+    return (piece + 1023) & ~(int64_t)1023;
+}
+
 GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                         const float *slo_ms, int64_t n_requests,
                         const gs_instances *inst, const gs_types *types, float ema_alpha,
@@ -461,17 +487,18 @@ GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int
 {
     int rc = check_pool(ctx, inst, types, false);
     if (rc != GS_OK) return rc;
-    if (n_requests < 0) return GS_ERR_INVALID_ARG;
+    if (n_requests < 0 || n_requests > gs::kMaxRouteRequests) return GS_ERR_INVALID_ARG;
     if (n_requests > 0 && (!prompt_len || !pred_decode_len || !slo_ms || !out_instance_idx ||
                            !out_est_e2e_ms || !out_slack_ms)) return GS_ERR_INVALID_ARG;
     if (n_requests == 0) return GS_OK;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GS_ERR_NO_DEVICE;
+    if ((rc = ensure_host_pipe(ctx)) != GS_OK) return rc;
     const size_t n = (size_t)n_requests;
     const size_t bytes = pool_stage_bytes(inst->n_instances, types->n_types) + 6 * pad256(n * 4) + pad256(n);
     rc = ensure_stage(ctx, bytes);
     if (rc != GS_OK) return rc;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaStream_t st = (cudaStream_t)cuda_stream, out = ctx->host_out_stream;
     Carver c{ctx->stage};
     PoolStage pool;
     cudaError_t e = stage_pool(c, inst, types, &pool, st);
@@ -481,20 +508,31 @@ GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int
     int32_t *didx = c.take<int32_t>(n);
     float *dest = c.take<float>(n), *dslack = c.take<float>(n);
     uint8_t *dtier = out_tier ? c.take<uint8_t>(n) : nullptr;
-    if ((e = cudaMemcpyAsync(dx, prompt_len, n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(dy, pred_decode_len, n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(dD, slo_ms, n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-        return cuda_fail(ctx, e);
-    rc = gs_route_batch(ctx, dx, dy, dD, n_requests, &pool.inst, &pool.types, ema_alpha,
-                        didx, dest, dslack, dtier, 0u, cuda_stream);
-    if (rc != GS_OK) return rc;
-    if ((e = cudaMemcpyAsync(out_instance_idx, didx, n * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(out_est_e2e_ms, dest, n * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(out_slack_ms, dslack, n * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-        return cuda_fail(ctx, e);
-    if (out_tier && (e = cudaMemcpyAsync(out_tier, dtier, n, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-        return cuda_fail(ctx, e);
-    e = cudaStreamSynchronize(st);
+    if ((e = gs::launch_prologue(ctx, pool.inst, pool.types, ema_alpha, false, st)) != cudaSuccess) return cuda_fail(ctx, e);
+    const int64_t piece = host_piece(n_requests);
+    int k = 0;
+    for (int64_t off = 0; off < n_requests; off += piece, ++k) {
+        const size_t len = (size_t)(n_requests - off < piece ? n_requests - off : piece);
+        if ((e = cudaMemcpyAsync(dx + off, prompt_len + off, len * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(dy + off, pred_decode_len + off, len * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(dD + off, slo_ms + off, len * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+            break;
+        if ((e = gs::launch_route(ctx, dx + off, dy + off, dD + off, (int64_t)len, nullptr, inst->n_instances,
+                                  types->n_types, didx + off, dest + off, dslack + off, dtier ? dtier + off : nullptr,
+                                  false, false, st)) != cudaSuccess) break;
+        // the piece's results go back on the second stream as soon as they exist
+        if ((e = cudaEventRecord(ctx->host_events[k], st)) != cudaSuccess ||
+            (e = cudaStreamWaitEvent(out, ctx->host_events[k], 0)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(out_instance_idx + off, didx + off, len * 4, cudaMemcpyDeviceToHost, out)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(out_est_e2e_ms + off, dest + off, len * 4, cudaMemcpyDeviceToHost, out)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(out_slack_ms + off, dslack + off, len * 4, cudaMemcpyDeviceToHost, out)) != cudaSuccess)
+            break;
+        if (out_tier && (e = cudaMemcpyAsync(out_tier + off, dtier + off, len, cudaMemcpyDeviceToHost, out)) != cudaSuccess)
+            break;
+    }
+    // (also after an error: nothing may still be using the staging buffers when the call returns)
+    const cudaError_t e1 = cudaStreamSynchronize(st), e2 = cudaStreamSynchronize(out);
+    if (e == cudaSuccess) e = e1 != cudaSuccess ? e1 : e2;
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 
@@ -511,8 +549,10 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx, const int32_t *assigned_inst, const in
     if (cand_capacity > 0 && !out_cand_idx) return GS_ERR_INVALID_ARG;
     if (n_active > 0 && (!assigned_inst || !generated_tokens || !pred_len || !elapsed_ms || !slo_ms ||
                          !out_flag_bits)) return GS_ERR_INVALID_ARG;
+    if (n_active == 0) { *out_cand_count = 0; return GS_OK; }
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GS_ERR_NO_DEVICE;
+    if ((rc = ensure_host_pipe(ctx)) != GS_OK) return rc;
     const size_t n = (size_t)n_active;
     const size_t words = (n + 31) / 32;
     const size_t cap = (size_t)(cand_capacity < n_active ? cand_capacity : n_active);
@@ -520,7 +560,7 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx, const int32_t *assigned_inst, const in
                          pad256(words * 4) + pad256(cap * 4) + 256;
     rc = ensure_stage(ctx, bytes);
     if (rc != GS_OK) return rc;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaStream_t st = (cudaStream_t)cuda_stream, out = ctx->host_out_stream;
     Carver c{ctx->stage};
     PoolStage pool;
     cudaError_t e = stage_pool(c, inst, types, &pool, st);
@@ -529,28 +569,43 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx, const int32_t *assigned_inst, const in
     float *del = c.take<float>(n), *dslo = c.take<float>(n);
     uint32_t *dbits = c.take<uint32_t>(words);
     int32_t *dcand = c.take<int32_t>(cap);
-    int64_t *dcount = c.take<int64_t>(1);
+    int64_t *dcount = c.take<int64_t>(2);           // running totals, two slots taken in turn
     const void *src[] = {assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms};
     void *dst[] = {dg, dgen, dtot, del, dslo};
-    for (int k = 0; k < 5 && n > 0; ++k)
-        if ((e = cudaMemcpyAsync(dst[k], src[k], n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-            return cuda_fail(ctx, e);
-    rc = gs_risk_scan(ctx, dg, dgen, dtot, del, dslo, n_active, &pool.inst, &pool.types,
-                      dbits, cap ? dcand : nullptr, (int64_t)cap, dcount, cuda_stream);
-    if (rc != GS_OK) return rc;
-    int64_t count = 0;
-    if ((e = cudaMemcpyAsync(&count, dcount, sizeof(count), cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-        return cuda_fail(ctx, e);
-    if (words && (e = cudaMemcpyAsync(out_flag_bits, dbits, words * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-        return cuda_fail(ctx, e);
-    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(ctx, e);
-    *out_cand_count = count;
-    const size_t n_out = (size_t)(count < (int64_t)cap ? count : (int64_t)cap);
-    if (n_out) {
-        e = cudaMemcpyAsync(out_cand_idx, dcand, n_out * 4, cudaMemcpyDeviceToHost, st);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    // every piece's copies and kernels are enqueued first: piece k scans its own requests, lists
+    // its candidates behind those of the pieces before it and leaves the running total
+    const int64_t piece = host_piece(n_active);
+    int n_pieces = 0;
+    for (int64_t off = 0; off < n_active && e == cudaSuccess; off += piece, ++n_pieces) {
+        const int k = n_pieces;
+        const size_t len = (size_t)(n_active - off < piece ? n_active - off : piece);
+        for (int col = 0; col < 5 && e == cudaSuccess; ++col)
+            e = cudaMemcpyAsync((char *)dst[col] + off * 4, (const char *)src[col] + off * 4, len * 4, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) break;
+        e = gs::launch_risk(ctx, dg + off, dgen + off, dtot + off, del + off, dslo + off, (int64_t)len, pool.inst, pool.types,
+                            dbits + off / 32, cap ? dcand : nullptr, (int64_t)cap, dcount + (k & 1), st,
+                            k ? dcount + ((k - 1) & 1) : nullptr, (int32_t)off);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->host_counts + k, dcount + (k & 1), sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->host_events[k], st);
     }
+    // then, piece by piece as the totals arrive: its flag words and its stretch of the list go back
+    // on the second stream while later pieces are still being copied in and scanned
+    int64_t before = 0;
+    for (int k = 0; k < n_pieces && e == cudaSuccess; ++k) {
+        const int64_t off = (int64_t)k * piece;
+        const size_t len = (size_t)(n_active - off < piece ? n_active - off : piece);
+        if ((e = cudaEventSynchronize(ctx->host_events[k])) != cudaSuccess) break;
+        const int64_t total = ctx->host_counts[k];
+        e = cudaMemcpyAsync(out_flag_bits + off / 32, dbits + off / 32, ((len + 31) / 32) * 4, cudaMemcpyDeviceToHost, out);
+        const int64_t lo = before < (int64_t)cap ? before : (int64_t)cap, hi = total < (int64_t)cap ? total : (int64_t)cap;
+        if (e == cudaSuccess && hi > lo)
+            e = cudaMemcpyAsync(out_cand_idx + lo, dcand + lo, (size_t)(hi - lo) * 4, cudaMemcpyDeviceToHost, out);
+        before = total;
+    }
+    const cudaError_t e1 = cudaStreamSynchronize(st), e2 = cudaStreamSynchronize(out);
+    if (e == cudaSuccess) e = e1 != cudaSuccess ? e1 : e2;
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    *out_cand_count = before;
     return GS_OK;
 }
 

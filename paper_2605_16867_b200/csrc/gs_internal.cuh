@@ -101,6 +101,8 @@ constexpr unsigned short kNoList = 0xFFFFu;
 
 constexpr int64_t kMaxRouteRequests = (int64_t)1 << 36;   // per routing call (the kernel's queues hold a request's
                                                           // index within its CTA's run of requests in 32 bits)
+#define GS_HOST_PIECES 8                 // the *_host entry points work through their input in up to this many pieces
+constexpr int64_t kHostPieceMin = 1 << 18;   // ... of at least this many requests
 constexpr int kMaxScanCtas = 4096;      // CTAs of one risk scan (a few per SM), one flag count each
 constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
 
@@ -137,9 +139,14 @@ struct gs_ctx {
     gs::Scratch s;
     int64_t launches;
     int last_cuda_error;
-    // staging for the *_host entry points (device memory, grown on demand)
+    // staging for the *_host entry points (device memory, grown on demand), and what their
+    // pipeline of copies and kernels needs (created by the first such call)
     char *stage;
     size_t stage_bytes;
+    cudaStream_t host_out_stream;            // results travel back on it while the next piece's inputs arrive
+    cudaEvent_t host_events[GS_HOST_PIECES]; // piece k computed
+    int64_t *host_counts;                    // pinned: candidates up to and including piece k
+    bool host_pipe_ready;
     // optional per-kernel timing (gs_timing_enable)
     bool timing;
     struct TimedLaunch { int kernel; cudaEvent_t start, stop; };
@@ -195,6 +202,7 @@ cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *gen
                         const int32_t *pred_len, const float *elapsed, const float *slo,
                         int64_t n_active, const gs_instances &inst, const gs_types &types,
                         uint32_t *flag_bits, int32_t *cand_idx, int64_t cand_capacity,
-                        int64_t *cand_count, cudaStream_t st);
+                        int64_t *cand_count, cudaStream_t st,
+                        const int64_t *prev_count = nullptr, int32_t index_base = 0);   // a scan in pieces: see risk.cu
 
 }  // namespace gs

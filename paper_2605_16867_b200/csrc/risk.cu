@@ -192,7 +192,8 @@ __global__ void __launch_bounds__(kScatterThreads, 2048 / kScatterThreads)
 scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_words,
                           const unsigned *__restrict__ cta_counts, int64_t n_steps,
                           int32_t *__restrict__ cand_idx, int64_t cand_capacity,
-                          int64_t *__restrict__ cand_count, unsigned *__restrict__ status)
+                          int64_t *__restrict__ cand_count, unsigned *__restrict__ status,
+                          const int64_t *__restrict__ prev_count, int32_t index_base)
 {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -213,7 +214,9 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
     if (lane == 0) sh_part[warp] = part;
 
     const unsigned lane_bit = 1u << lane, below = lane_bit - 1u;
-    int64_t base = 0;
+    // (a scan that continues an earlier one -- the host entry point scans in pieces -- starts
+    // its list where that one ended and numbers its requests from index_base)
+    int64_t base = prev_count ? *prev_count : 0;
     int buf = 0;
     for (int64_t w0 = w_begin; w0 < w_end; w0 += kScatterWarps * kScatterBlocks * 32, buf ^= 1) {
         uint32_t word[kScatterBlocks];
@@ -261,7 +264,7 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
             __syncwarp();
             const int64_t mine = base + before;             // list position of the block's first flag
             int32_t *out = cand_idx + mine;
-            const int32_t idx0 = (int32_t)((w0 + blk * 32) << 5) + lane;     // n_active < 2^31
+            const int32_t idx0 = index_base + (int32_t)((w0 + blk * 32) << 5) + lane;    // n_active < 2^31
             if (mine + total <= cand_capacity) {
 #pragma unroll
                 for (int w = 0; w < 32; ++w) {
@@ -324,7 +327,8 @@ static cudaError_t enqueue_scan(unsigned *cta_counts, int dev, int n_sm, gs_ctx 
                                 const float *elapsed, const float *slo, int64_t n,
                                 const gs_instances &inst, const gs_types &types,
                                 uint32_t *flag_bits, int32_t *cand_idx, int64_t cand_capacity,
-                                int64_t *cand_count, unsigned *status, cudaStream_t st)
+                                int64_t *cand_count, unsigned *status, cudaStream_t st,
+                                const int64_t *prev_count = nullptr, int32_t index_base = 0)
 {
     if (n == 0) return cudaMemsetAsync(cand_count, 0, sizeof(int64_t), st);
     const int64_t n_steps = (n + (1 << kStepShift) - 1) >> kStepShift;
@@ -352,7 +356,8 @@ static cudaError_t enqueue_scan(unsigned *cta_counts, int dev, int n_sm, gs_ctx 
         cfg.attrs = attr;
         cfg.numAttrs = GS_RISK_PDL ? 1 : 0;
         e = cudaLaunchKernelEx(&cfg, scatter_candidates_kernel, (const uint32_t *)flag_bits, n_words,
-                               (const unsigned *)cta_counts, n_steps, cand_idx, cand_capacity, cand_count, status);
+                               (const unsigned *)cta_counts, n_steps, cand_idx, cand_capacity, cand_count, status,
+                               prev_count, index_base);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -362,10 +367,11 @@ cudaError_t launch_risk(gs_ctx *ctx, const int32_t *assigned, const int32_t *gen
                         const int32_t *pred_len, const float *elapsed, const float *slo,
                         int64_t n, const gs_instances &inst, const gs_types &types,
                         uint32_t *flag_bits, int32_t *cand_idx, int64_t cand_capacity,
-                        int64_t *cand_count, cudaStream_t st)
+                        int64_t *cand_count, cudaStream_t st, const int64_t *prev_count, int32_t index_base)
 {
     return enqueue_scan(ctx->s.scan_counts, ctx->device, ctx->n_sm, ctx, assigned, generated, pred_len, elapsed, slo, n,
-                        inst, types, flag_bits, cand_idx, cand_capacity, cand_count, ctx->s.status, st);
+                        inst, types, flag_bits, cand_idx, cand_capacity, cand_count, ctx->s.status, st, prev_count,
+                        index_base);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -316,8 +316,13 @@ def test_advance_carries_the_queue_delay_of_the_accumulate_round_only(gs):
     assert gs.device_status() == 0
 
 
-def test_host_entry_points_match_device_ones(gs):
-    wl = W.make_workload(1, n_requests=20_001, n_active=70_003)
+@pytest.mark.parametrize("n_req,n_act", [(20_001, 70_003), (700_001, 1_000_003)])
+def test_host_entry_points_match_device_ones(gs, n_req, n_act):
+    """The host-buffer entry points work through their input in pieces (copies in, kernels and
+    copies out overlap); the larger size spans several pieces with a ragged last one.  Results
+    must equal the device entry points' bit for bit, also with a candidate buffer that ends
+    inside a piece."""
+    wl = W.make_workload(1, n_requests=n_req, n_active=n_act)
     pool = pool_of(gs, wl.types, wl.instances)
     dev = gpu_route(gs, pool, wl.requests, 0.5)
     n = wl.requests.n
@@ -335,6 +340,13 @@ def test_host_entry_points_match_device_ones(gs):
     assert count == risk.count
     np.testing.assert_array_equal(bits, risk.flag_bits)
     np.testing.assert_array_equal(cand[:count], risk.cand_idx)
+    assert gs.device_status() == 0
+    # a candidate buffer that holds two thirds of the list: the true count, the list's head
+    small = np.full(2 * count // 3, -5, np.int32)
+    count2 = gs.risk_scan_host(*wl.active.columns(), wl.types, wl.instances, bits, small)
+    assert count2 == risk.count
+    np.testing.assert_array_equal(small, risk.cand_idx[:small.size])
+    assert gs.device_status() == 16                              # GS_DEV_CAND_TRUNCATED
 
 
 def test_error_codes(gs):
