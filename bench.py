@@ -395,21 +395,27 @@ def measure_config(gs, cfg_id: int, seed: int, dev, peak_gbs: float, gs_count=No
             graph = None
             how = "rounds enqueued one by one from the host (graph capture failed: %s)" % type(exc).__name__
         torch.cuda.synchronize(dev)
-        times = []
-        for _ in range(7):
-            reset_state()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize(dev)
-            e0.record(stream)
-            if graph is not None:
-                graph.replay()
-            else:
-                enqueue_stream(stream)
-            e1.record(stream)
-            torch.cuda.synchronize(dev)
-            times.append(e0.elapsed_time(e1))
-        ms = statistics.median(times)
+
+        def time_stream(use_graph):
+            times = []
+            for _ in range(7):
+                reset_state()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize(dev)
+                e0.record(stream)
+                if use_graph:
+                    graph.replay()
+                else:
+                    enqueue_stream(stream)
+                e1.record(stream)
+                torch.cuda.synchronize(dev)
+                times.append(e0.elapsed_time(e1))
+            return statistics.median(times)
+
+        ms_host = time_stream(False)                  # enqueued call by call from Python
+        ms = time_stream(True) if graph is not None else ms_host
         res["stream"] = {"rounds": R, "ms": ms, "us_per_round": ms / R * 1e3, "how": how,
+                         "ms_enqueued_from_host": ms_host,
                          "requests_per_s": R * N / (ms * 1e-3), "logical_pairs_per_s": R * N * M / (ms * 1e-3),
                          "scans": R, "scan_requests_per_s": R * A / (ms * 1e-3),
                          "what": "per round: gs_route_batch(ACCUMULATE) + gs_advance_state + gs_risk_scan over the advanced state"}
