@@ -421,8 +421,8 @@ __device__ __forceinline__ void exhaustive_pick(const Row *rows, int M, float xs
 // the routing round
 // ---------------------------------------------------------------------------------------
 
-// Bulk asynchronous copies (global -> this CTA's shared memory, this GPU's memory only, no
-// multicast) that report to an mbarrier.  Addresses and sizes are multiples of 16 bytes.
+// Bulk asynchronous copies (global -> this one CTA's shared memory, from this GPU's own memory)
+// that report to an mbarrier.  Addresses and sizes are multiples of 16 bytes.
 __device__ __forceinline__ unsigned shared_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void bulk_copy_to_shared(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
