@@ -349,6 +349,31 @@ def test_host_entry_points_match_device_ones(gs, n_req, n_act):
     assert gs.device_status() == 16                              # GS_DEV_CAND_TRUNCATED
 
 
+def test_work_counters_of_the_counting_build(gs):
+    """The measuring build (-DGS_COUNT_EVALS) runs the same kernels with its counters on: its
+    answers are still the oracle's, every request is scored exactly at least once, far fewer
+    pairs are scored than the N x M the definition names, and the regular build counts nothing."""
+    from paper_2605_16867_b200 import GoodServe
+    wl = W.make_workload(1, n_requests=30_000, n_active=16)
+    t32 = oracle.instance_table(wl.types, wl.instances, wl.ema_alpha, "f32")
+    ref = oracle.route(t32, *wl.requests.columns())
+    counting = GoodServe(0, counting=True)
+    try:
+        counting.eval_counters(clear=True)
+        got = gpu_route(counting, pool_of(counting, wl.types, wl.instances), wl.requests, wl.ema_alpha)
+        assert_route_matches_f32_oracle(got, ref)
+        c = counting.eval_counters(clear=True)
+        n, M = wl.requests.n, wl.instances.n_instances
+        assert n <= c[0] < n * M // 4                      # pairs scored exactly
+        assert c[1] >= c[0] and c[2] >= n                  # row bounds, type bounds
+        assert 0 <= c[3] < n and c[4] <= c[3]              # left to the full search, of which fallback
+        assert counting.eval_counters() == [0] * 8         # cleared
+    finally:
+        counting.close()
+    gpu_route(gs, pool_of(gs, wl.types, wl.instances), wl.requests, wl.ema_alpha)
+    assert gs.eval_counters() == [0] * 8
+
+
 def test_error_codes(gs):
     from paper_2605_16867_b200 import GoodServe, GoodServeError, InstancePool
     types, inst = W.make_pool(16, 4, seed=1)
