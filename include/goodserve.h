@@ -78,7 +78,9 @@ enum gs_dev_status {
     GS_DEV_BAD_VALUE = 4,       /* negative count or negative/NaN q_ema was read as 0 */
     GS_DEV_TIMEOUT = 8,         /* a bounded device-side wait expired (the route kernel's wait for its table
                                    copies); the outputs of that call are invalid */
-    GS_DEV_CAND_TRUNCATED = 16  /* more flagged requests than cand_capacity; list was cut */
+    GS_DEV_CAND_TRUNCATED = 16, /* more flagged requests than cand_capacity; list was cut */
+    GS_DEV_INTERNAL = 32        /* only from a library built with -DGS_DEBUG: one of its index checks failed
+                                   (a table index computed by the search fell outside its table) */
 };
 
 /* gs_route_batch flags */

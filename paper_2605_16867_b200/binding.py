@@ -23,6 +23,7 @@ class DeviceStatus:
     BAD_VALUE = 4
     TIMEOUT = 8
     CAND_TRUNCATED = 16
+    INTERNAL = 32
 
 
 class GoodServeError(RuntimeError):
@@ -53,12 +54,12 @@ class _InstancesMut(C.Structure):
                 ("n_instances", C.c_int32)]
 
 
-def library_path(counting: bool = False) -> str:
-    return os.path.join(_PKG, "libgoodserve_count.so" if counting else "libgoodserve.so")
+def library_path(counting: bool = False, checking: bool = False) -> str:
+    name = "libgoodserve_count.so" if counting else "libgoodserve_debug.so" if checking else "libgoodserve.so"
+    return os.path.join(_PKG, name)
 
 
-_lib = None
-_count_lib = None
+_libs = {}
 
 
 def _declare(lib):
@@ -105,31 +106,27 @@ def _declare(lib):
     return lib
 
 
-def load_library(build_if_missing: bool = True, counting: bool = False):
+def load_library(build_if_missing: bool = True, counting: bool = False, checking: bool = False):
     """Loads libgoodserve.so (building it with nvcc first if it is absent or stale).
     Raises if that fails -- there is no other implementation to fall back to.
     ``counting=True`` loads the measuring build instead (-DGS_COUNT_EVALS: the work counters
-    behind gs_eval_counters tick; many times slower, for benchmarks only)."""
-    global _lib, _count_lib
-    cached = _count_lib if counting else _lib
-    if cached is not None:
-        return cached
-    path = library_path(counting)
+    behind gs_eval_counters tick; many times slower, for benchmarks only); ``checking=True`` the
+    build with table index checks compiled in (-DGS_DEBUG; GS_DEV_INTERNAL reports a failure)."""
+    kind = "counting" if counting else "checking" if checking else "regular"
+    if kind in _libs:
+        return _libs[kind]
+    path = library_path(counting, checking)
     if build_if_missing:
         from .build import build_library
         try:
-            build_library(counting=counting)
+            build_library(counting=counting, checking=checking)
         except Exception as exc:                      # nvcc missing on a box that has the .so
             if not os.path.exists(path):
                 raise RuntimeError(f"{os.path.basename(path)} is missing and could not be built: {exc}") from exc
     if not os.path.exists(path):
         raise RuntimeError(f"{path} not found; run paper_2605_16867_b200/build.py")
-    lib = _declare(C.CDLL(path))
-    if counting:
-        _count_lib = lib
-    else:
-        _lib = lib
-    return lib
+    _libs[kind] = _declare(C.CDLL(path))
+    return _libs[kind]
 
 
 def _dev_ptr(t: Optional[torch.Tensor], dtype: torch.dtype, n: Optional[int], name: str, device) -> Optional[int]:
@@ -194,10 +191,11 @@ class InstancePool:
 class GoodServe:
     """One library context (gs_create / gs_destroy) bound to a CUDA device."""
 
-    def __init__(self, device: int = 0, max_instances: int = 1024, max_types: int = 16, counting: bool = False):
+    def __init__(self, device: int = 0, max_instances: int = 1024, max_types: int = 16, counting: bool = False,
+                 checking: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("GoodServe needs a CUDA device; there is no CPU implementation")
-        self._lib = load_library(counting=counting)
+        self._lib = load_library(counting=counting, checking=checking)
         self.device = torch.device("cuda", device)
         torch.cuda.init()
         with torch.cuda.device(self.device):

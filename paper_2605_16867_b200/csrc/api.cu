@@ -255,7 +255,10 @@ GS_API int gs_device_status(gs_ctx *ctx, void *cuda_stream, unsigned *out_bits) 
     cudaError_t e = cudaStreamSynchronize(st);
     if (e == cudaSuccess) e = cudaMemcpy(out_bits, ctx->s.status, sizeof(unsigned), cudaMemcpyDeviceToHost);
     if (e == cudaSuccess) e = cudaMemset(ctx->s.status, 0, sizeof(unsigned));
-    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    // (the checking build's index tests; always 0 in the regular build)
+    if (gs::route_index_errors(true) | gs::prologue_index_errors(true)) *out_bits |= (unsigned)GS_DEV_INTERNAL;
+    return GS_OK;
 }
 
 GS_API int gs_route_batch(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,

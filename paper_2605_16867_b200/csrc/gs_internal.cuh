@@ -24,6 +24,25 @@ enum EvalCounter {
 };
 cudaError_t read_eval_counters(unsigned long long *out, bool clear);     // zeros unless GS_COUNT_EVALS
 
+// Checking build (-DGS_DEBUG), in place of a memory checker: every index into a shared-memory
+// table that the search computes from table contents, and every position the prologue writes a
+// table entry to, is tested against the table's size first.  A failed test is counted in a
+// per-file device counter and the index pulled to 0, so the access that follows stays legal;
+// nothing traps.  gs_device_status then reports GS_DEV_INTERNAL.  (GS_CHECKED compiles to the
+// bare index in the regular build.)
+#ifdef GS_DEBUG
+#define GS_DEBUG_COUNTER(name) __device__ unsigned name
+#define GS_CHECKED(counter, idx, limit) gs::checked_index(&(counter), (int)(idx), (int)(limit))
+__device__ __forceinline__ int checked_index(unsigned *counter, int idx, int limit) {
+    if ((unsigned)idx >= (unsigned)limit) { atomicAdd(counter, 1u); return 0; }
+    return idx;
+}
+#else
+#define GS_CHECKED(counter, idx, limit) (idx)
+#endif
+unsigned route_index_errors(bool clear);       // failed index checks since the last clear (0 unless GS_DEBUG)
+unsigned prologue_index_errors(bool clear);
+
 // Exact per-instance coefficients of Eq. 2 for the current round, in caller order.
 struct __align__(16) Row {
     float q, p, d;

@@ -31,6 +31,21 @@
 
 namespace gs {
 
+#ifdef GS_DEBUG
+GS_DEBUG_COUNTER(g_prologue_index_errors);
+#endif
+unsigned prologue_index_errors(bool clear)
+{
+    unsigned v = 0;
+#ifdef GS_DEBUG
+    if (cudaMemcpyFromSymbol(&v, g_prologue_index_errors, sizeof(v)) != cudaSuccess) return ~0u;
+    if (clear) { const unsigned zero = 0; cudaMemcpyToSymbol(g_prologue_index_errors, &zero, sizeof(zero)); }
+#else
+    (void)clear;
+#endif
+    return v;
+}
+
 constexpr int kPrologueThreads = GS_MAX_INSTANCES;      // one thread per instance
 constexpr int kPmFloats = 8192;                         // shared-memory floats for the running minima
 constexpr int kCountSortMax = 256;                      // a group of up to this many rows is ranked by counting
@@ -380,7 +395,11 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             sh_rd[k] = d_lo;
             my_qmin = min(my_qmin, q_bits);             // non-negative floats order like their bits
         }
-        s.row_bounds[row_slot(base + k)] = entry;
+#ifdef GS_DEBUG
+        // the order must be a strict one (a permutation of the group's rows, no key twice)
+        if (k > 0 && k < n_t && !(sh_sorted[k - 1] < sh_sorted[k])) atomicAdd(&g_prologue_index_errors, 1u);
+#endif
+        s.row_bounds[GS_CHECKED(g_prologue_index_errors, row_slot(base + k), kMaxPaddedRows)] = entry;
         if (kDirect) s.row_p[base + k] = k < n_t ? lower_bound(sh_p[(int)(sh_sorted[k] & 0xFFFFull)]) : 0.f;
     }
     my_qmin = __reduce_min_sync(0xFFFFFFFFu, my_qmin);
@@ -514,7 +533,8 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                     }
                 }
                 // (a cell that no row can pass begins at the type's last group: searches always have eight rows to test)
-                s.start_table[(tr * kStartBuckets + b) * kStartSlots + slot] = (unsigned char)min(lo >> 3, (n_padded >> 3) - 1);
+                s.start_table[GS_CHECKED(g_prologue_index_errors, (tr * kStartBuckets + b) * kStartSlots + slot,
+                                         GS_MAX_TYPES * kStartBuckets * kStartSlots)] = (unsigned char)min(lo >> 3, (n_padded >> 3) - 1);
                 if (!kDirect) {
                     const int before = lo < n_t ? sh_pc[bw * n_t + lo] : sh_len[bw];    // records among rows [0, lo)
                     s.start_list[(tr * kStartBuckets + b) * kStartSlots + slot] = (unsigned char)min(before >> 1, 255);
@@ -528,10 +548,11 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                     for (int k = lane; k < n_t; k += 32) {
                         const int c = pc[k], c_next = k + 1 < n_t ? pc[k + 1] : len;
                         if (c_next != c)
-                            s.pool[off + c] = make_uint2(__float_as_uint(sh_rq[k]), __float_as_uint(sh_rd[k]));
+                            s.pool[GS_CHECKED(g_prologue_index_errors, off + c, pool_base + pool_share)] =
+                                make_uint2(__float_as_uint(sh_rq[k]), __float_as_uint(sh_rd[k]));
                     }
                     for (int k = len + lane; k < ((len + kListWindow + 1) & ~1); k += 32)
-                        s.pool[off + k] = make_uint2(kPadQ, 0u);
+                        s.pool[GS_CHECKED(g_prologue_index_errors, off + k, pool_base + pool_share)] = make_uint2(kPadQ, 0u);
                 }
                 if (lane == 0)
                     s.bucket_list[tr * kStartBuckets + b0 + warp] = off >= 0 ? (unsigned short)(off >> 1) : kNoList;

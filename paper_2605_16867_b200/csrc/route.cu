@@ -26,6 +26,21 @@
 
 namespace gs {
 
+#ifdef GS_DEBUG
+GS_DEBUG_COUNTER(g_route_index_errors);
+#endif
+unsigned route_index_errors(bool clear)
+{
+    unsigned v = 0;
+#ifdef GS_DEBUG
+    if (cudaMemcpyFromSymbol(&v, g_route_index_errors, sizeof(v)) != cudaSuccess) return ~0u;
+    if (clear) { const unsigned zero = 0; cudaMemcpyToSymbol(g_route_index_errors, &zero, sizeof(zero)); }
+#else
+    (void)clear;
+#endif
+    return v;
+}
+
 #ifdef GS_COUNT_EVALS
 __device__ unsigned long long g_eval_counts[kCountN];
 #define GS_COUNT(k, v) atomicAdd(&gs::g_eval_counts[k], (unsigned long long)(v))
@@ -157,7 +172,7 @@ __device__ __forceinline__ bool score_row(const Tables &tb, int inst, float x, f
                                           float d_cap, int &g_best, float &d_best, float &T_best)
 {
     GS_COUNT(kCountExact, 1);
-    const Row row = tb.rows[row_pos(inst)];
+    const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
     const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));      // Eq. 2, H = 0
     const bool feasible = (T <= D) && (need <= (unsigned)row.kv) && (!kCapped || row.d < d_cap);
     const bool worse = row.d < d_best;
@@ -200,8 +215,8 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
         int k = 0;
         if (inv_w > 0.f) {
             // largest d that can still meet the deadline -> slot -> first row worth a look
-            k = 8 * tb.start_table[(t * kStartBuckets + ybucket) * kStartSlots +
-                                   start_slot(Rg, h.y, ry, __int_as_float(geo.w), inv_w)];
+            k = 8 * tb.start_table[GS_CHECKED(g_route_index_errors, (t * kStartBuckets + ybucket) * kStartSlots +
+                                   start_slot(Rg, h.y, ry, __int_as_float(geo.w), inv_w), tb.n_types * kStartBuckets * kStartSlots)];
         }
         const int k_end = geo.x + geo.y;
         k += geo.x;                                         // padded row index, a multiple of 8
@@ -209,7 +224,7 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
             // tag word of the first row, from k on, whose bound passes
             unsigned first = kNoRow;
             for (; k < k_end; k += 8) {
-                const char *grp = reinterpret_cast<const char *>(tb.row_bounds + k);
+                const char *grp = reinterpret_cast<const char *>(tb.row_bounds + GS_CHECKED(g_route_index_errors, k, kMaxPaddedRows - 7));
                 const int sw = (k >> 4) & 3;                // see row_slot()
                 const uint4 r0 = *reinterpret_cast<const uint4 *>(grp + ((0 ^ sw) << 4));
                 const uint4 r1 = *reinterpret_cast<const uint4 *>(grp + ((1 ^ sw) << 4));
@@ -282,7 +297,7 @@ __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y
                 // the group's rows have d_lo >= gb.y (its last row's) and q words >= gb.x: if even
                 // the type's least q with that d misses the best, so does everything from here up;
                 // if the group's own least q with it does, the group holds nothing better
-                const float2 gb = tb.group_bounds[k >> 3];
+                const float2 gb = tb.group_bounds[GS_CHECKED(g_route_index_errors, k >> 3, kMaxPaddedRows / 8)];
                 if (!(__fmaf_rn(gb.y, y, h.y) <= Rg)) break;
                 if (kRowP ? !(__fmaf_rn(gb.y, y, __fmaf_rn(h.x, x, gb.x)) <= T_best + 1e-30f)
                           : !(__fmaf_rn(gb.y, y, gb.x) <= Rg)) continue;
@@ -306,7 +321,7 @@ __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y
                         const float R = kRowP ? T_best + 1e-30f : Rg;
                         if (!row_may_pass<kCapped, kRowP>(qw, dw, pl[2 * c + e], x, y, R, d_cap)) continue;
                         const int inst = (int)(qw & kRowTagMask);
-                        const Row row = tb.rows[row_pos(inst)];
+                        const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
                         if (kCapped && !(row.d < d_cap)) continue;
                         if (!any_kv && !(need <= (unsigned)row.kv)) continue;
                         GS_COUNT(kCountExact, 1);
@@ -524,7 +539,7 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
     float ry;
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(ry) : "f"(y));
     const float sc = fminf(fmaxf((Dm * ry - cand_z0) * cand_inv, 0.f), (float)(kCandSlots - 1));
-    unsigned mask = tb.cand[__float2int_rd(sc)];
+    unsigned mask = tb.cand[GS_CHECKED(g_route_index_errors, __float2int_rd(sc), kCandSlots)];
     int t = -1;
     float4 h = make_float4(0.f, 0.f, 0.f, 0.f);
     float Rg = 0.f;
@@ -539,8 +554,8 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
     if (t < 0) return false;
     const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, inv_w, d0
     const int ybucket = min((int)(__float_as_uint(y) >> (23 - kBucketBits)) - (127 << kBucketBits), kStartBuckets - 1);
-    const int cell = (t * kStartBuckets + ybucket) * kStartSlots +
-                     start_slot(Rg, h.y, ry, __int_as_float(geo.w), __int_as_float(geo.z));
+    const int cell = GS_CHECKED(g_route_index_errors, (t * kStartBuckets + ybucket) * kStartSlots +
+                     start_slot(Rg, h.y, ry, __int_as_float(geo.w), __int_as_float(geo.z)), tb.n_types * kStartBuckets * kStartSlots);
     unsigned first = kNoRow;
     if (kRowP) {
         // rows of a group differ in p: sixteen row bounds of the group's full list
@@ -552,7 +567,9 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
         // the record list of this type and bucket of L_out: only rows that can be the first to pass
         const unsigned list = tb.bucket_list[t * kStartBuckets + ybucket];
         if (list == kNoList) return false;
-        const uint4 *w = reinterpret_cast<const uint4 *>(tb.pool) + (list + tb.start_list[cell]);
+        // (the window of four pairs of entries read from there must end inside the pool)
+        const uint4 *w = reinterpret_cast<const uint4 *>(tb.pool) +
+                         GS_CHECKED(g_route_index_errors, list + tb.start_list[cell], kPoolEntries / 2 - 3);
         const uint4 r0 = w[0], r1 = w[1];
         first = row_may_pass<false, false>(r1.z, r1.w, 0.f, x, y, Rg, 0.f) ? r1.z : first;
         first = row_may_pass<false, false>(r1.x, r1.y, 0.f, x, y, Rg, 0.f) ? r1.x : first;
@@ -569,7 +586,7 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
     if (first == kNoRow) return false;
     const int inst = (int)(first & kRowTagMask);
     GS_COUNT(kCountExact, 1);
-    const Row row = tb.rows[row_pos(inst)];
+    const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
     const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));          // Eq. 2, H = 0
     if (!(T <= D && need <= (unsigned)row.kv)) return false;
     const float d_floor = __fmul_rn(row.d, 1.0f - 1.9073486328125e-6f);       // the bound every row with d >= the pick's carries
@@ -917,7 +934,8 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             for (int j = 0; j < kReqPerThread; ++j) {
                 const bool push = (slow >> j) & 1u;
                 const unsigned votes = __ballot_sync(0xFFFFFFFFu, push);
-                if (push) queue[q_count + __popc(votes & ((1u << lane) - 1u))] = (unsigned)(first + j - cta_first_request);
+                if (push) queue[GS_CHECKED(g_route_index_errors, q_count + __popc(votes & ((1u << lane) - 1u)), kQueueCap)] =
+                              (unsigned)(first + j - cta_first_request);
                 q_count += __popc(votes);
             }
             __syncwarp();                          // the entries, and the stores above, come before the full search
