@@ -194,6 +194,28 @@ struct PrefixHits {
     int64_t slot_stride;
 };
 
+// Launches `kernel` as a programmatic dependent of the kernel before it in the stream: the launch
+// may be set up, and the CTAs placed, while that kernel still runs (once all its CTAs have said so
+// with griddepcontrol.launch_dependents, or have ended).  Every kernel launched this way waits
+// (griddepcontrol.wait: the whole earlier grid done, its stores visible) before it reads or
+// writes anything an earlier kernel of the stream may touch.  Hides a launch latency per kernel.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_types &types,
                             float ema_alpha, bool carry_q, cudaStream_t st);

@@ -148,8 +148,10 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     __shared__ int sh_len[kPrologueThreads / 32], sh_off[kPrologueThreads / 32], sh_pool_used;
 
     // the kernel that follows in the stream (the routing round) may be set up from now on; it
-    // waits for this whole grid before it reads a table
+    // waits for this whole grid before it reads a table.  This kernel itself is launched the same
+    // way: the kernel before it may still be running, and may be the one that writes the pool's state.
     asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
@@ -577,11 +579,10 @@ cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_type
                             float ema_alpha, bool carry_q, cudaStream_t st)
 {
     LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
-    prologue_kernel<false><<<GS_MAX_TYPES, kPrologueThreads, prologue_dynamic_smem(), st>>>(
-        inst.type_id, inst.queued_prefill_tokens, inst.decode_batch, inst.free_kv_tokens,
-        inst.q_ema_ms, inst.n_instances, types.prefill_ms_per_tok, types.tpot_a_ms,
-        types.tpot_b_ms, types.n_types, ema_alpha, carry_q ? 1 : 0, ctx->s);
-    return cudaGetLastError();
+    return launch_dependent(prologue_kernel<false>, dim3(GS_MAX_TYPES), dim3(kPrologueThreads), prologue_dynamic_smem(), st,
+                            inst.type_id, inst.queued_prefill_tokens, inst.decode_batch, inst.free_kv_tokens,
+                            inst.q_ema_ms, inst.n_instances, types.prefill_ms_per_tok, types.tpot_a_ms,
+                            types.tpot_b_ms, types.n_types, ema_alpha, carry_q ? 1 : 0, ctx->s);
 }
 
 // Tables of a round from coefficients given per instance; the instances are put into
@@ -590,11 +591,11 @@ cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_type
 cudaError_t launch_prologue_direct(gs_ctx *ctx, const gs_instance_table &tab, cudaStream_t st)
 {
     LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
-    prologue_kernel<true><<<GS_MAX_TYPES, kPrologueThreads, prologue_dynamic_smem(), st>>>(
-        reinterpret_cast<const int32_t *>(tab.q_ms), reinterpret_cast<const int32_t *>(tab.p_ms_per_tok),
-        reinterpret_cast<const int32_t *>(tab.d_ms_per_tok), tab.free_kv_tokens, nullptr, tab.n_instances,
-        nullptr, nullptr, nullptr, kDirectGroups, 0.f, 0, ctx->s);
-    return cudaGetLastError();
+    return launch_dependent(prologue_kernel<true>, dim3(GS_MAX_TYPES), dim3(kPrologueThreads), prologue_dynamic_smem(), st,
+                            reinterpret_cast<const int32_t *>(tab.q_ms), reinterpret_cast<const int32_t *>(tab.p_ms_per_tok),
+                            reinterpret_cast<const int32_t *>(tab.d_ms_per_tok), tab.free_kv_tokens, (const float *)nullptr,
+                            tab.n_instances, (const float *)nullptr, (const float *)nullptr, (const float *)nullptr,
+                            kDirectGroups, 0.f, 0, ctx->s);
 }
 
 }  // namespace gs

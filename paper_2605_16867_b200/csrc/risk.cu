@@ -87,6 +87,9 @@ risk_flags_kernel(const int32_t *__restrict__ assigned, const int32_t *__restric
     // the dependent launch (pass 2) may be set up from now on; it still waits for this grid's end
     asm volatile("griddepcontrol.launch_dependents;");
 #endif
+    // (launched as a programmatic dependent: the kernel before it may be the one that writes the
+    // pool's state, or the previous scan still reading the scratch this one overwrites)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __shared__ float sh_d[GS_MAX_INSTANCES];
     __shared__ float sh_a[GS_MAX_TYPES], sh_b[GS_MAX_TYPES];
     __shared__ unsigned sh_count;
@@ -212,6 +215,8 @@ scatter_candidates_kernel(const uint32_t *__restrict__ flag_bits, int64_t n_word
     for (int k = threadIdx.x; k < (int)blockIdx.x; k += kScatterThreads) part += __ldcg(cta_counts + k);
     part = __reduce_add_sync(0xFFFFFFFFu, part);
     if (lane == 0) sh_part[warp] = part;
+    // (the kernel after this one in the stream may be set up from now on)
+    asm volatile("griddepcontrol.launch_dependents;");
 
     const unsigned lane_bit = 1u << lane, below = lane_bit - 1u;
     // (a scan that continues an earlier one -- the host entry point scans in pieces -- starts
@@ -338,10 +343,10 @@ static cudaError_t enqueue_scan(unsigned *cta_counts, int dev, int n_sm, gs_ctx 
     cudaError_t e;
     {
         LaunchTimer timer(timing_ctx, GS_K_RISK_FLAGS, st);
-        risk_flags_kernel<<<(unsigned)blocks, kRiskThreads, 0, st>>>(
-            assigned, generated, pred_len, elapsed, slo, n, inst.type_id, inst.decode_batch, inst.n_instances,
-            types.tpot_a_ms, types.tpot_b_ms, types.n_types, flag_bits, cta_counts, n_steps, status);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        e = launch_dependent(risk_flags_kernel, dim3((unsigned)blocks), dim3(kRiskThreads), 0, st,
+                             assigned, generated, pred_len, elapsed, slo, n, inst.type_id, inst.decode_batch, inst.n_instances,
+                             types.tpot_a_ms, types.tpot_b_ms, types.n_types, flag_bits, cta_counts, n_steps, status);
+        if (e != cudaSuccess) return e;
     }
     {
         LaunchTimer timer(timing_ctx, GS_K_RISK_SCATTER, st);

@@ -944,6 +944,8 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     if (q_count < 32) break;                       // out of tiles
     do drain(); while (q_count >= 32);
     }
+    // (the kernel after this one in the stream may be set up from now on)
+    asm volatile("griddepcontrol.launch_dependents;");
     // What is left on the warp's queue (fewer than 32) it finishes itself, right after its last
     // tile: the warps of a CTA end up to a tile apart, so these searches overlap the other warps'
     // last tiles, and a handful of lanes per warp diverge far less than 32 would.
@@ -1230,6 +1232,8 @@ advance_kernel(int32_t *__restrict__ queued, int32_t *__restrict__ batch,
                unsigned long long *__restrict__ deltas,
                const float *__restrict__ q_by_g, int *__restrict__ pending)
 {
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // (launched as a programmatic dependent of the routing round)
     const int g = threadIdx.x;
     const bool carry = pending[0] != 0;
     __syncthreads();
@@ -1254,10 +1258,9 @@ cudaError_t launch_advance(gs_ctx *ctx, const gs_instances_mut &inst, cudaStream
 {
     const int M = inst.n_instances;
     LaunchTimer timer(ctx, GS_K_ADVANCE, st);
-    advance_kernel<<<1, GS_MAX_INSTANCES, 0, st>>>(inst.queued_prefill_tokens, inst.decode_batch,
-                                                   inst.free_kv_tokens, inst.q_ema_ms, M,
-                                                   ctx->s.deltas, ctx->s.q_by_g, ctx->s.table_info + 7);
-    return cudaGetLastError();
+    return launch_dependent(advance_kernel, dim3(1), dim3(GS_MAX_INSTANCES), 0, st, inst.queued_prefill_tokens,
+                            inst.decode_batch, inst.free_kv_tokens, inst.q_ema_ms, M, ctx->s.deltas,
+                            (const float *)ctx->s.q_by_g, ctx->s.table_info + 7);
 }
 
 // ---------------------------------------------------------------------------------------
