@@ -166,6 +166,7 @@ GS_API int gs_create(gs_ctx **out, int device, int max_instances, int max_types)
         {(void **)&s.pool, gs::kPoolEntries * sizeof(uint2)},
         {(void **)&s.bucket_list, (size_t)GS_MAX_TYPES * gs::kStartBuckets * sizeof(unsigned short)},
         {(void **)&s.start_list, (size_t)GS_MAX_TYPES * gs::kStartBuckets * gs::kStartSlots},
+        {(void **)&s.chord, (size_t)GS_MAX_TYPES * gs::kStartBuckets * sizeof(float4)},
         {(void **)&s.q_by_g, Mx * sizeof(float)},
         {(void **)&s.deltas, 3 * Mx * sizeof(unsigned long long)},
         {(void **)&s.scan_counts, gs::kMaxScanCtas * sizeof(unsigned)},
@@ -188,7 +189,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.q_by_g, s.deltas, s.scan_counts, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.chord, s.q_by_g, s.deltas, s.scan_counts, s.status, ctx->stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);
@@ -456,7 +457,7 @@ GS_API int gs_reroute_candidates(gs_ctx *ctx, const int32_t *cand_idx, const int
     cudaError_t e = gs::launch_prologue(ctx, *inst, *types, ema_alpha, false, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     e = gs::launch_reroute(ctx, cand_idx, cand_count, cand_capacity, assigned_inst, generated_tokens, pred_len,
-                           elapsed_ms, slo_ms, prompt_len, n_active, types->n_types,
+                           elapsed_ms, slo_ms, prompt_len, n_active, inst->n_instances, types->n_types,
                            out_new_instance, out_est_ms, out_slack_ms, out_tier, st);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }

@@ -117,6 +117,7 @@ constexpr int kPoolEntries = GS_POOL_ENTRIES;
 constexpr int kListWindow = 8;             // entries the first attempt may test (four, then four more)
 constexpr int kListMax = 510;              // longer lists are not stored (start_list counts pairs of entries in a byte)
 constexpr unsigned short kNoList = 0xFFFFu;
+constexpr unsigned kPadQ = 0x7FC00000u;    // q word of a padding entry (a NaN: its bound test is false); no row has it
 
 constexpr int64_t kMaxRouteRequests = (int64_t)1 << 36;   // per routing call (the kernel's queues hold a request's
                                                           // index within its CTA's run of requests in 32 bits)
@@ -141,6 +142,8 @@ struct Scratch {
     uint2 *pool;              // [kPoolEntries] record lists
     unsigned short *bucket_list;  // [GS_MAX_TYPES * kStartBuckets] first pool entry of the list, halved; kNoList = none
     unsigned char *start_list;    // [GS_MAX_TYPES * kStartBuckets * kStartSlots] like start_table, in pairs of list entries
+    float4 *chord;            // [GS_MAX_TYPES * kStartBuckets] {a, s, p_lo, -}: a + s * L_out is below every row bound of
+                              //  the type for L_out in the bucket (typed pools; see the prologue)
     float *q_by_g;            // [max_instances] q_g of the latest ACCUMULATE round, caller order (carried by advance)
     unsigned long long *deltas;   // [3 * max_instances] pending sums: L_in, count, L_in + L_out
     unsigned *scan_counts;    // [kMaxScanCtas] risk scan: requests flagged by each CTA of pass 1
@@ -154,7 +157,6 @@ struct gs_ctx {
     int max_instances;
     int max_types;
     int n_sm;
-    int reroute_ctas_per_sm[GS_MAX_TYPES + 1];   // by number of types (sets the shared-memory size)
     gs::Scratch s;
     int64_t launches;
     int last_cuda_error;
@@ -234,7 +236,7 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
 cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,
                            const int32_t *assigned, const int32_t *generated, const int32_t *pred_len,
                            const float *elapsed, const float *slo, const int32_t *prompt_len, int64_t n_active,
-                           int n_types, int32_t *out_inst, float *out_est, float *out_slack, uint8_t *out_tier,
+                           int n_instances, int n_types, int32_t *out_inst, float *out_est, float *out_slack, uint8_t *out_tier,
                            cudaStream_t st);
 cudaError_t configure_route(gs_ctx *ctx);
 cudaError_t configure_prologue();

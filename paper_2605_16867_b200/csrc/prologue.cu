@@ -63,13 +63,17 @@ __device__ __forceinline__ unsigned orderable(float f) {
 
 constexpr float kShrink = 1.0f - 1.9073486328125e-6f;   // 1 - 2^-19
 
+// Least value of a warp's lanes (non-negative floats: they order like their bits).
+__device__ __forceinline__ float warp_min_nonneg(float v) {
+    return __uint_as_float(__reduce_min_sync(0xFFFFFFFFu, __float_as_uint(v)));
+}
+
 // Upper edge of bucket b of L_out: buckets split every octave at 1.5, b = 2 * exponent + (mantissa >= 1.5).
 __device__ __forceinline__ float bucket_upper_edge(int b) {
     const unsigned e = 127u + (unsigned)(b >> kBucketBits);
     const unsigned m = ((unsigned)b & ((1u << kBucketBits) - 1u)) + 1u;
     return __uint_as_float((m >> kBucketBits) ? ((e + 1u) << 23) : ((e << 23) | (m << (23 - kBucketBits))));
 }
-constexpr unsigned kPadQ = 0x7FC00000u;                 // NaN: compares false with everything
 
 // Entries of the record-list pool that a type with n of the pool's M instances may use.
 // (kPoolEntries * n <= 2^23: plain 32-bit arithmetic)
@@ -469,10 +473,17 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 const float y_hi = bucket_upper_edge(b) * 1.00002f;
                 float carry = 3.4e38f;
                 int n_rec = 0;
+                // (for the chord, below: the least row bound at either end of the bucket)
+                const float y_lo = b == 0 ? 1.0f : bucket_upper_edge(b - 1) * 0.99998f;
+                float f_lo = 3.4e38f, f_hi = 3.4e38f;
                 for (int k0 = 0; k0 < n_t; k0 += 32) {
                     const int k = k0 + lane;
                     float own = 3.4e38f;
                     if (k < n_t) own = open_ended ? sh_rd[k] : __fmaf_rn(y_hi, sh_rd[k], sh_rq[k] - q0);
+                    if (!kDirect && k < n_t) {
+                        f_lo = fminf(f_lo, __fmaf_rn(y_lo, sh_rd[k], sh_rq[k]));
+                        f_hi = fminf(f_hi, __fmaf_rn(y_hi, sh_rd[k], sh_rq[k]));
+                    }
                     float h = own;
 #pragma unroll
                     for (int off = 1; off < 32; off <<= 1) {
@@ -493,6 +504,26 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                     carry = __shfl_sync(0xFFFFFFFFu, h, 31);
                 }
                 if (lane == 0) sh_len[warp] = n_rec;
+                if (!kDirect) {
+                    // Chord.  F(y) = least row bound of the type at L_out = y, the minimum of the
+                    // lines q_k + d_lo_k y, is concave: between two points it lies on or above the
+                    // straight line through them.  The line through (y_lo, F(y_lo)) and
+                    // (y_hi, F(y_hi)), the ends of the bucket pushed outwards a little, is therefore
+                    // below every row bound for every L_out of the bucket: a request whose
+                    // R = D - p_lo L_in is below that line can pass no row bound of the type.  Beyond
+                    // the last bucket's lower end F grows at least as fast as the least d_lo.  Line
+                    // and offset are lowered by 2^-16 of F, far more than the roundings here
+                    // and in the kernel's tests add up to (a few 2^-20 of F).
+                    f_lo = warp_min_nonneg(f_lo);
+                    f_hi = warp_min_nonneg(f_hi);
+                    float slope = open_ended ? sh_rd[n_t - 1] : (f_hi - f_lo) / (y_hi - y_lo);
+                    slope = fmaxf(slope, 0.f);
+                    const float offset = f_lo - slope * y_lo;
+                    const float kMargin = 1.52587890625e-5f;            // 2^-16
+                    if (lane == 0)
+                        s.chord[tr * kStartBuckets + b] = make_float4(offset - kMargin * f_lo, slope * (1.0f - kMargin),
+                                                                  __fmul_rn(p_group, kShrink), 0.f);
+                }
             }
             __syncthreads();
             if (warp == 0) {                                // room in the pool, in bucket order (lane = bucket of the batch)

@@ -66,13 +66,15 @@ cudaError_t read_eval_counters(unsigned long long *out, bool clear)
 #ifndef GS_ROUTE_THREADS
 #define GS_ROUTE_THREADS 896
 #endif
+#ifndef GS_REROUTE_THREADS
+#define GS_REROUTE_THREADS 1024
+#endif
 #ifndef GS_ROUTE_MIN_CTAS
 #define GS_ROUTE_MIN_CTAS 1
 #endif
 constexpr int kRouteThreads = GS_ROUTE_THREADS;     // four requests per lane (large batches)
 constexpr int kRouteThreadsSmall = 1024;            // one request per lane (small batches)
 constexpr int kRouteMinCtas = GS_ROUTE_MIN_CTAS;
-constexpr int kRerouteThreads = 256;
 // Requests per lane: four (128-bit column loads) for large batches; one for small ones, where
 // shorter tiles spread over more warps count for more than wide loads (fewer registers: more
 // threads).  With per-row p the search holds more state: a quarter fewer threads, more
@@ -126,6 +128,7 @@ struct Tables {
     const uint2 *pool;            // record lists (typed pools)
     const unsigned short *bucket_list;
     const unsigned char *start_list;
+    const float4 *chord;          // per type and bucket of L_out: a line below every row bound (re-routing only)
     int n_types;
 };
 
@@ -268,13 +271,78 @@ __device__ __forceinline__ int pick_instance(const Tables &tb, float x, float y,
 // Fallback of Algorithm 1 for one request, by one thread: the smallest T among instances with
 // KV room (tier 2), else among all (tier 3); ties to the smallest index.  Branch and bound over
 // the same tables: the best T found so far plays the deadline's part in the bound tests, so a
-// row is skipped only when its exactly-rounded T is proven larger.  Types are visited fastest
-// first and each type's rows from its smallest d upwards, which is where the minimum lives;
-// the walk up a type stops at the first group whose smallest d alone already exceeds the best.
-// Returns -1 with tier 0 only when kCapped and no instance has d < d_cap.
+// row is skipped only when its exactly-rounded T is proven larger.
 struct Pick { int g; float T; unsigned tier; };
 
-// `first_pass` = 1 skips the pass over instances with KV room (the caller knows there is none).
+// The eight rows at padded index k (a multiple of 8) of a type with least prefill coefficient
+// p_lo, held against the best found so far; Rg = (T_best less the type's least prefill time).
+template <bool kCapped, bool kRowP>
+__device__ __forceinline__ void search_eight(const Tables &tb, int k, float x, float y, unsigned need, float d_cap,
+                                             bool any_kv, float p_lo, int &g_best, float &T_best, float &Rg)
+{
+    const char *grp = reinterpret_cast<const char *>(tb.row_bounds + k);
+    const int sw = (k >> 4) & 3;                // see row_slot()
+    uint4 r[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) r[c] = *reinterpret_cast<const uint4 *>(grp + ((c ^ sw) << 4));
+    // rows k .. k+7 in order: (r[0].x,y) (r[0].z,w) (r[1].x,y) ...; larger d first
+    float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;
+    if (kRowP) {
+        pa = *reinterpret_cast<const float4 *>(tb.row_p + k);
+        pb = *reinterpret_cast<const float4 *>(tb.row_p + k + 4);
+    }
+    const float pl[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+    // the eight bounds at once (NaN, which passes no test, for padding and for rows that the
+    // cap excludes) ...
+    GS_COUNT(kCountBound, 8);
+    float b[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const unsigned qw = (j & 1) ? r[j >> 1].z : r[j >> 1].x, dw = (j & 1) ? r[j >> 1].w : r[j >> 1].y;
+        const float d_lo = __uint_as_float(dw);
+        const float base = kRowP ? __fmaf_rn(pl[j], x, __uint_as_float(qw)) : __uint_as_float(qw);
+        b[j] = __fmaf_rn(d_lo, y, base);
+        if (kCapped) b[j] = d_lo < d_cap ? b[j] : __int_as_float(0x7FC00000);
+    }
+    // ... then the rows whose bound passes, one at a time, smallest d first (one copy of the
+    // scoring code, run as often as the busiest lane has rows to score).  While nothing has been
+    // found the row with the least bound goes first and the others are then held against its T.
+    auto passing = [&](float limit) {
+        unsigned m = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) m |= (b[j] <= limit) ? (1u << j) : 0u;
+        return m;
+    };
+    bool blind = g_best < 0;
+    unsigned m = passing(blind ? fminf(fminf(fminf(b[0], b[1]), fminf(b[2], b[3])), fminf(fminf(b[4], b[5]), fminf(b[6], b[7])))
+                               : (kRowP ? T_best + 1e-30f : Rg));
+    unsigned done = 0;
+    while (m) {
+        const int j = 31 - __clz(m);
+        m &= ~(1u << j);
+        done |= 1u << j;
+        const int inst = (int)(tb.row_bounds[k + ((((j >> 1) ^ sw) << 1) | (j & 1))].x & kRowTagMask);
+        const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
+        if ((!kCapped || row.d < d_cap) && (any_kv || need <= (unsigned)row.kv)) {
+            GS_COUNT(kCountExact, 1);
+            const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));   // Eq. 2, H = 0
+            if (T < T_best || (T == T_best && inst < g_best) || g_best < 0) {
+                T_best = T; g_best = inst;
+                Rg = __fmaf_rn(-p_lo, x, T_best) + 1e-30f;
+            }
+        }
+        if (blind && m == 0) {                 // the rest of the group, against what is known now
+            blind = false;
+            m = passing(kRowP ? T_best + 1e-30f : Rg) & ~done;
+        }
+    }
+}
+
+// Types are visited fastest first and each type's rows from its smallest d upwards, which is
+// where the minimum lives; the walk up a type stops at the first group whose smallest d alone
+// already exceeds the best.  Returns -1 with tier 0 only when kCapped and no instance has
+// d < d_cap.  `first_pass` = 1 skips the pass over instances with KV room (the caller knows
+// there is none).
 template <bool kCapped, bool kRowP>
 __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y, unsigned need, float d_cap,
                                               int first_pass = 0)
@@ -301,37 +369,7 @@ __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y
                 if (!(__fmaf_rn(gb.y, y, h.y) <= Rg)) break;
                 if (kRowP ? !(__fmaf_rn(gb.y, y, __fmaf_rn(h.x, x, gb.x)) <= T_best + 1e-30f)
                           : !(__fmaf_rn(gb.y, y, gb.x) <= Rg)) continue;
-                const char *grp = reinterpret_cast<const char *>(tb.row_bounds + k);
-                const int sw = (k >> 4) & 3;                // see row_slot()
-                uint4 r[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) r[c] = *reinterpret_cast<const uint4 *>(grp + ((c ^ sw) << 4));
-                // rows k .. k+7 in order: (r[0].x,y) (r[0].z,w) (r[1].x,y) ...; larger d first
-                float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;
-                if (kRowP) {
-                    pa = *reinterpret_cast<const float4 *>(tb.row_p + k);
-                    pb = *reinterpret_cast<const float4 *>(tb.row_p + k + 4);
-                }
-                const float pl[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-#pragma unroll
-                for (int c = 3; c >= 0; --c) {
-#pragma unroll
-                    for (int e = 1; e >= 0; --e) {
-                        const unsigned qw = e ? r[c].z : r[c].x, dw = e ? r[c].w : r[c].y;
-                        const float R = kRowP ? T_best + 1e-30f : Rg;
-                        if (!row_may_pass<kCapped, kRowP>(qw, dw, pl[2 * c + e], x, y, R, d_cap)) continue;
-                        const int inst = (int)(qw & kRowTagMask);
-                        const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
-                        if (kCapped && !(row.d < d_cap)) continue;
-                        if (!any_kv && !(need <= (unsigned)row.kv)) continue;
-                        GS_COUNT(kCountExact, 1);
-                        const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));   // Eq. 2, H = 0
-                        if (T < T_best || (T == T_best && inst < g_best) || g_best < 0) {
-                            T_best = T; g_best = inst;
-                            Rg = __fmaf_rn(-h.x, x, T_best) + 1e-30f;
-                        }
-                    }
-                }
+                search_eight<kCapped, kRowP>(tb, k, x, y, need, d_cap, any_kv, h.x, g_best, T_best, Rg);
             }
         }
         tier_out = any_kv ? 3u : 2u;
@@ -340,46 +378,6 @@ __device__ __forceinline__ Pick fallback_pick(const Tables &tb, float x, float y
     Pick r;
     r.g = g_best; r.T = T_best; r.tier = tier_out;
     return r;
-}
-
-// Copies the round's tables into shared memory (all threads of the CTA; the caller
-// synchronises).  Returns the first shared-memory byte after them.
-__device__ __forceinline__ unsigned char *stage_tables(unsigned char *smem, int n_types_alloc,
-                                                       const Row *__restrict__ g_rows,
-                                                       const uint2 *__restrict__ g_row_bounds,
-                                                       const float2 *__restrict__ g_group_bounds,
-                                                       const unsigned char *__restrict__ g_start_table,
-                                                       const TypeHeader *__restrict__ g_headers,
-                                                       const int *__restrict__ table_info, Tables &tb,
-                                                       const float *__restrict__ g_row_p = nullptr)
-{
-    const int n_padded = table_info[0];
-    const bool unsafe = table_info[1] != 0;
-    const int M = table_info[2];
-    const int n_act = table_info[3];
-    Row *sh_rows = reinterpret_cast<Row *>(smem);
-    TypeHeader *sh_headers = reinterpret_cast<TypeHeader *>(sh_rows + GS_MAX_INSTANCES);
-    uint2 *sh_row_bounds = reinterpret_cast<uint2 *>(sh_headers + GS_MAX_TYPES);
-    float2 *sh_group_bounds = reinterpret_cast<float2 *>(sh_row_bounds + kMaxPaddedRows);
-    unsigned char *sh_start = reinterpret_cast<unsigned char *>(sh_group_bounds + kMaxPaddedRows / 8);
-    for (int k = threadIdx.x; k < ((M + 7) & ~7); k += blockDim.x) sh_rows[k] = g_rows[k];   // (stored position-mixed: row_pos)
-    for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_bounds[k] = g_row_bounds[k];
-    for (int k = threadIdx.x; k < n_padded / 8; k += blockDim.x) sh_group_bounds[k] = g_group_bounds[k];
-    for (int k = threadIdx.x; k < n_act * (kStartBuckets * kStartSlots / 16); k += blockDim.x)
-        reinterpret_cast<uint4 *>(sh_start)[k] = reinterpret_cast<const uint4 *>(g_start_table)[k];
-    if (threadIdx.x < n_act) sh_headers[threadIdx.x] = g_headers[threadIdx.x];
-    tb.headers = sh_headers; tb.row_bounds = sh_row_bounds; tb.group_bounds = sh_group_bounds;
-    tb.start_table = sh_start; tb.rows = sh_rows;
-    tb.n_types = unsafe ? 0 : n_act;          // unusable bounds: every request takes the exhaustive path
-    unsigned char *end = sh_start + n_types_alloc * (kStartBuckets * kStartSlots);
-    tb.row_p = nullptr;
-    if (g_row_p) {                            // per-row bounds of p, after the start tables
-        float *sh_row_p = reinterpret_cast<float *>(end);
-        for (int k = threadIdx.x; k < n_padded; k += blockDim.x) sh_row_p[k] = g_row_p[k];
-        tb.row_p = sh_row_p;
-        end += kMaxPaddedRows * sizeof(float);
-    }
-    return end;
 }
 
 // The definition evaluated in full by one warp for one request (same arguments in all lanes):
@@ -459,11 +457,11 @@ __device__ __forceinline__ bool wait_barrier(unsigned long long *bar, unsigned p
 // Shared-memory image of the round's tables for the route kernel, in the order it is carved.
 struct TableImage {
     Row *rows; TypeHeader *headers; uint2 *row_bounds; float2 *group_bounds; unsigned char *start_table;
-    unsigned short *cand; unsigned char *start_list; unsigned short *bucket_list; uint2 *pool; float *row_p;
+    unsigned short *cand; unsigned char *start_list; unsigned short *bucket_list; uint2 *pool; float *row_p; float4 *chord;
     int *info; unsigned long long *bar; unsigned char *end;
 };
 
-template <bool kRowP>
+template <bool kRowP, bool kChord = false>
 __device__ __forceinline__ TableImage carve_tables(unsigned char *smem, int n_types_alloc) {
     TableImage im;
     im.rows = reinterpret_cast<Row *>(smem);
@@ -472,7 +470,7 @@ __device__ __forceinline__ TableImage carve_tables(unsigned char *smem, int n_ty
     im.group_bounds = reinterpret_cast<float2 *>(im.row_bounds + kMaxPaddedRows);
     im.start_table = reinterpret_cast<unsigned char *>(im.group_bounds + kMaxPaddedRows / 8);
     unsigned char *at = im.start_table + (size_t)n_types_alloc * (kStartBuckets * kStartSlots);
-    im.row_p = nullptr; im.start_list = nullptr; im.bucket_list = nullptr; im.pool = nullptr;
+    im.row_p = nullptr; im.start_list = nullptr; im.bucket_list = nullptr; im.pool = nullptr; im.chord = nullptr;
     if (kRowP) {
         im.row_p = reinterpret_cast<float *>(at); at += kMaxPaddedRows * sizeof(float);
     }
@@ -482,10 +480,55 @@ __device__ __forceinline__ TableImage carve_tables(unsigned char *smem, int n_ty
         im.bucket_list = reinterpret_cast<unsigned short *>(at); at += (size_t)n_types_alloc * kStartBuckets * sizeof(unsigned short);
         im.pool = reinterpret_cast<uint2 *>(at); at += (size_t)kPoolEntries * sizeof(uint2);
     }
+    if (kChord) {
+        im.chord = reinterpret_cast<float4 *>(at); at += (size_t)n_types_alloc * kStartBuckets * sizeof(float4);
+    }
     im.info = reinterpret_cast<int *>(at); at += 64;
     im.bar = reinterpret_cast<unsigned long long *>(at); at += 16;
     im.end = at;
     return im;
+}
+
+// Where the round's tables lie in global memory, and upper bounds, known to the host, of how much
+// of each the round can use (what lies beyond the round's own entries is never looked at).
+struct TableSource {
+    const Row *rows; const uint2 *row_bounds; const float2 *group_bounds; const unsigned char *start_table;
+    const TypeHeader *headers; const int *info; const unsigned short *cand; const uint2 *pool;
+    const unsigned short *bucket_list; const unsigned char *start_list; const float *row_p; const float4 *chord;
+    int n_types_alloc, m_rows, n_padded_max;
+};
+
+// Starts the bulk copies of all tables into the image, all in flight together, one barrier for
+// all of them (one thread).  The few numbers that only the prologue knows are copied along (info).
+template <bool kRowP, bool kChord = false>
+__device__ __forceinline__ void start_table_copies(const TableImage &im, const TableSource &src)
+{
+    const unsigned b_rows = (unsigned)src.m_rows * sizeof(Row), b_headers = (unsigned)src.n_types_alloc * sizeof(TypeHeader);
+    const unsigned b_bounds = (unsigned)src.n_padded_max * sizeof(uint2), b_groups = (unsigned)src.n_padded_max / 8 * sizeof(float2);
+    const unsigned b_start = (unsigned)src.n_types_alloc * (kStartBuckets * kStartSlots);
+    const unsigned b_cand = kCandSlots * sizeof(unsigned short), b_info = 64u;
+    const unsigned b_rowp = kRowP ? (unsigned)src.n_padded_max * sizeof(float) : 0u;
+    const unsigned b_bucket = kRowP ? 0u : (unsigned)src.n_types_alloc * kStartBuckets * sizeof(unsigned short);
+    const unsigned b_pool = kRowP ? 0u : (unsigned)kPoolEntries * sizeof(uint2);
+    const unsigned b_chord = kChord ? (unsigned)src.n_types_alloc * kStartBuckets * sizeof(float4) : 0u;
+    const unsigned total = b_rows + b_headers + b_bounds + b_groups + b_start + b_cand + b_info + b_rowp +
+                           (kRowP ? 0u : b_start) + b_bucket + b_pool + b_chord;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(shared_addr(im.bar)), "r"(total) : "memory");
+    bulk_copy_to_shared(im.info, src.info, b_info, im.bar);
+    bulk_copy_to_shared(im.cand, src.cand, b_cand, im.bar);
+    bulk_copy_to_shared(im.headers, src.headers, b_headers, im.bar);
+    bulk_copy_to_shared(im.rows, src.rows, b_rows, im.bar);
+    if (kRowP) {
+        bulk_copy_to_shared(im.row_p, src.row_p, b_rowp, im.bar);
+    } else {
+        bulk_copy_to_shared(im.bucket_list, src.bucket_list, b_bucket, im.bar);
+        bulk_copy_to_shared(im.start_list, src.start_list, b_start, im.bar);
+        bulk_copy_to_shared(im.pool, src.pool, b_pool, im.bar);
+    }
+    if (kChord) bulk_copy_to_shared(im.chord, src.chord, b_chord, im.bar);
+    bulk_copy_to_shared(im.start_table, src.start_table, b_start, im.bar);
+    bulk_copy_to_shared(im.row_bounds, src.row_bounds, b_bounds, im.bar);
+    bulk_copy_to_shared(im.group_bounds, src.group_bounds, b_groups, im.bar);
 }
 
 // First row of the eight at padded index k (a multiple of 8) whose bound passes: its tag word
@@ -735,10 +778,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     // The kernel is launched as a programmatic dependent of the prologue: everything above ran
     // beside it; the tables may be read once that whole grid is done and its stores are visible.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // The tables come in by bulk asynchronous copies, all in flight together, one barrier for
-    // all of them.  The sizes are upper bounds that the host knows (what lies beyond the round's
-    // own entries is never looked at); the few numbers that only the prologue knows are copied
-    // along (info).
+    // The tables come in by bulk asynchronous copies (start_table_copies).
     const TableImage im = carve_tables<kRowP>(smem, n_types_alloc);
     if (threadIdx.x == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(shared_addr(im.bar)) : "memory");
@@ -746,30 +786,9 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        const unsigned b_rows = (unsigned)m_rows * sizeof(Row), b_headers = (unsigned)n_types_alloc * sizeof(TypeHeader);
-        const unsigned b_bounds = (unsigned)n_padded_max * sizeof(uint2), b_groups = (unsigned)n_padded_max / 8 * sizeof(float2);
-        const unsigned b_start = (unsigned)n_types_alloc * (kStartBuckets * kStartSlots);
-        const unsigned b_cand = kCandSlots * sizeof(unsigned short), b_info = 64u;
-        const unsigned b_rowp = kRowP ? (unsigned)n_padded_max * sizeof(float) : 0u;
-        const unsigned b_bucket = kRowP ? 0u : (unsigned)n_types_alloc * kStartBuckets * sizeof(unsigned short);
-        const unsigned b_pool = kRowP ? 0u : (unsigned)kPoolEntries * sizeof(uint2);
-        const unsigned total = b_rows + b_headers + b_bounds + b_groups + b_start + b_cand + b_info + b_rowp +
-                               (kRowP ? 0u : b_start) + b_bucket + b_pool;
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(shared_addr(im.bar)), "r"(total) : "memory");
-        bulk_copy_to_shared(im.info, table_info, b_info, im.bar);
-        bulk_copy_to_shared(im.cand, g_cand, b_cand, im.bar);
-        bulk_copy_to_shared(im.headers, g_headers, b_headers, im.bar);
-        bulk_copy_to_shared(im.rows, g_rows, b_rows, im.bar);
-        if (kRowP) {
-            bulk_copy_to_shared(im.row_p, g_row_p, b_rowp, im.bar);
-        } else {
-            bulk_copy_to_shared(im.bucket_list, g_bucket_list, b_bucket, im.bar);
-            bulk_copy_to_shared(im.start_list, g_start_list, b_start, im.bar);
-            bulk_copy_to_shared(im.pool, g_pool, b_pool, im.bar);
-        }
-        bulk_copy_to_shared(im.start_table, g_start_table, b_start, im.bar);
-        bulk_copy_to_shared(im.row_bounds, g_row_bounds, b_bounds, im.bar);
-        bulk_copy_to_shared(im.group_bounds, g_group_bounds, b_groups, im.bar);
+        const TableSource src = {g_rows, g_row_bounds, g_group_bounds, g_start_table, g_headers, table_info, g_cand, g_pool,
+                                 g_bucket_list, g_start_list, g_row_p, nullptr, n_types_alloc, m_rows, n_padded_max};
+        start_table_copies<kRowP>(im, src);
     }
     unsigned char *after_tables = im.end;
     // the warps' queues: {L_in, L_out, bits of D, low word of the request index}, high word
@@ -800,7 +819,7 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
     Tables tb;
     tb.headers = im.headers; tb.row_bounds = im.row_bounds; tb.group_bounds = im.group_bounds;
     tb.start_table = im.start_table; tb.rows = im.rows; tb.row_p = im.row_p; tb.cand = im.cand;
-    tb.pool = im.pool; tb.bucket_list = im.bucket_list; tb.start_list = im.start_list;
+    tb.pool = im.pool; tb.bucket_list = im.bucket_list; tb.start_list = im.start_list; tb.chord = nullptr;
     tb.n_types = im.info[1] != 0 ? 0 : im.info[3];       // unusable bounds: every request takes the exhaustive path
 
     const bool fast_on = tb.n_types > 0;          // unusable bounds: every request takes the full search
@@ -978,6 +997,22 @@ static size_t route_smem_bytes(int n_types, bool accumulate, bool row_p) {
            (row_p ? kRouteSmemRowP : kRouteSmemPerTypeLists * n_types + kRouteSmemPool);
 }
 
+// The context's tables as a kernel argument, with the upper bounds of what a kernel copies of
+// them: the rows (position-mixed in blocks of eight) and the padded rows of all groups (each
+// group adds less than 16 of padding).
+static TableSource table_source(const gs_ctx *ctx, int n_instances, int n_types) {
+    TableSource src;
+    src.rows = ctx->s.rows; src.row_bounds = ctx->s.row_bounds; src.group_bounds = ctx->s.group_bounds;
+    src.start_table = ctx->s.start_table; src.headers = ctx->s.headers; src.info = ctx->s.table_info;
+    src.cand = ctx->s.cand_table; src.pool = ctx->s.pool; src.bucket_list = ctx->s.bucket_list;
+    src.start_list = ctx->s.start_list; src.row_p = ctx->s.row_p; src.chord = ctx->s.chord;
+    src.n_types_alloc = n_types;
+    src.m_rows = (n_instances + 7) & ~7;
+    src.n_padded_max = (n_instances + 16 * n_types + 15) & ~15;
+    if (src.n_padded_max > kMaxPaddedRows) src.n_padded_max = kMaxPaddedRows;
+    return src;
+}
+
 cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
                          const float *slo_ms, int64_t n, const PrefixHits *hits, int n_instances, int n_types,
                          int32_t *out_idx, float *out_est, float *out_slack, uint8_t *out_tier,
@@ -986,11 +1021,8 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
     if (n == 0) return cudaSuccess;
     if (n > kMaxRouteRequests) return cudaErrorInvalidValue;      // (the entry points refuse it first)
     const size_t smem = route_smem_bytes(n_types, accumulate, row_p);
-    // upper bounds of what the kernel copies of the round's tables: the rows (position-mixed in
-    // blocks of eight) and the padded rows of all groups (each group adds less than 16 of padding)
-    const int m_rows = (n_instances + 7) & ~7;
-    int n_padded_max = (n_instances + 16 * n_types + 15) & ~15;
-    if (n_padded_max > kMaxPaddedRows) n_padded_max = kMaxPaddedRows;
+    const TableSource src = table_source(ctx, n_instances, n_types);
+    const int m_rows = src.m_rows, n_padded_max = src.n_padded_max;
     const int req = n < kSmallBatch ? 1 : 4;
     const int64_t tile = (int64_t)route_threads(row_p, req) * req;
     int64_t blocks = (n + tile - 1) / tile;
@@ -1036,68 +1068,180 @@ cudaError_t launch_route(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *
 // re-routing of the scan's candidates among strictly faster instances (Sec. 3.4)
 // ---------------------------------------------------------------------------------------
 
-// One thread per candidate: gathers the flagged request's columns through cand_idx, turns it
-// into the request that a token-ID migration would pose to the target (re-prefill prompt +
-// generated tokens, decode what is left, within the time that is left) and runs the same
-// search as the routing round, restricted to instances with d < d of the current instance.
-// Candidates for which that search finds no feasible faster instance (nearly half of them at
-// config 3) need Algorithm 1's fallback, a much longer search: their positions go on the warp's
-// queue, and whenever 32 have gathered each lane takes one of them through the fallback, so that
-// the long path runs with all lanes busy instead of the few of each 32 that need it.
-constexpr int kRerouteQueue = 64;           // per warp: at most 31 left over + the 32 of a step
+// The short way for a re-routed candidate, modelled on fast_pick.  The search without the cap is
+// tried: if its pick happens to be strictly faster than the current instance it is the capped
+// search's pick as well (the eligible instances are a subset that holds the unrestricted
+// optimum), and a request that is at risk where it runs can only be feasible on a faster
+// instance, so this is the usual case.  Going through the candidate types in search order:
+//   * a type that fails its entry test (R below the type's chord for this bucket of L_out: see
+//     the prologue) holds no feasible instance;
+//   * nor does a type whose record list, from the start cell on, ends inside the eight entries
+//     tested without one of them passing (a row that is not a record passes only if a record
+//     before it does, and the records before the start cell cannot pass);
+//   * the first row that passes is scored exactly; if it is feasible and below the cap, and no
+//     later type can rank before it, it is the answer.
+// Returns 1 (settled: g_out, T_out), -1 (no instance at all is feasible, capped or not: the
+// fallback decides) or 0 (not settled: the capped search in full).
+__device__ __forceinline__ int capped_first_attempt(const Tables &tb, float x, float y,
+                                                    float D, unsigned need, float d_cap, int &g_out, float &T_out)
+{
+    const float Dm = D + 1e-30f;
+    float ry;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(ry) : "f"(y));
+    const int ybucket = min((int)(__float_as_uint(y) >> (23 - kBucketBits)) - (127 << kBucketBits), kStartBuckets - 1);
+    // which types pass their entry test: all of them at once, the same work in every lane
+    unsigned mask = 0;
+    for (int t = 0; t < tb.n_types; ++t) {
+        const float4 line = tb.chord[t * kStartBuckets + ybucket];               // offset, slope, p_lo
+        GS_COUNT(kCountTypeTest, 1);
+        if (__fmaf_rn(line.y, y, line.x) <= __fmaf_rn(-line.z, x, Dm)) mask |= 1u << t;
+    }
+    for (;;) {
+        if (!mask) return -1;
+        const int t = __ffs(mask) - 1;
+        mask &= mask - 1;
+        const float4 h = *reinterpret_cast<const float4 *>(&tb.headers[t]);       // p_lo, q_lo, d_lo, d_max
+        const float Rg = __fmaf_rn(-h.x, x, Dm);
+        const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, inv_w, d0
+        const int cell = GS_CHECKED(g_route_index_errors, (t * kStartBuckets + ybucket) * kStartSlots +
+                         start_slot(Rg, h.y, ry, __int_as_float(geo.w), __int_as_float(geo.z)), tb.n_types * kStartBuckets * kStartSlots);
+        const unsigned list = tb.bucket_list[t * kStartBuckets + ybucket];
+        if (list == kNoList) return 0;
+        const uint4 *w = reinterpret_cast<const uint4 *>(tb.pool) +
+                         GS_CHECKED(g_route_index_errors, list + tb.start_list[cell], kPoolEntries / 2 - 3);
+        const uint4 r0 = w[0], r1 = w[1];
+        unsigned first = kNoRow;
+        first = row_may_pass<false, false>(r1.z, r1.w, 0.f, x, y, Rg, 0.f) ? r1.z : first;
+        first = row_may_pass<false, false>(r1.x, r1.y, 0.f, x, y, Rg, 0.f) ? r1.x : first;
+        first = row_may_pass<false, false>(r0.z, r0.w, 0.f, x, y, Rg, 0.f) ? r0.z : first;
+        first = row_may_pass<false, false>(r0.x, r0.y, 0.f, x, y, Rg, 0.f) ? r0.x : first;
+        if (first == kNoRow) {
+            const uint4 r2 = w[2], r3 = w[3];
+            first = row_may_pass<false, false>(r3.z, r3.w, 0.f, x, y, Rg, 0.f) ? r3.z : first;
+            first = row_may_pass<false, false>(r3.x, r3.y, 0.f, x, y, Rg, 0.f) ? r3.x : first;
+            first = row_may_pass<false, false>(r2.z, r2.w, 0.f, x, y, Rg, 0.f) ? r2.z : first;
+            first = row_may_pass<false, false>(r2.x, r2.y, 0.f, x, y, Rg, 0.f) ? r2.x : first;
+            if (first == kNoRow) {
+                if (r3.z == kPadQ) continue;         // the list ended inside the window: nothing of this type
+                return 0;
+            }
+        }
+        const int inst = (int)(first & kRowTagMask);
+        GS_COUNT(kCountExact, 1);
+        const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
+        const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));          // Eq. 2, H = 0
+        if (!(T <= D && need <= (unsigned)row.kv && row.d < d_cap)) return 0;
+        const float d_floor = __fmul_rn(row.d, 1.0f - 1.9073486328125e-6f);       // the bound every row with d >= the pick's carries
+        while (mask) {
+            const int tt = __ffs(mask) - 1;
+            mask &= mask - 1;
+            const float4 h2 = *reinterpret_cast<const float4 *>(&tb.headers[tt]);
+            if (h2.w < row.d) break;                                              // nor can any type after it
+            GS_COUNT(kCountTypeTest, 1);
+            if (__fmaf_rn(fmaxf(h2.z, d_floor), y, h2.y) <= __fmaf_rn(-h2.x, x, Dm)) return 0;
+        }
+        g_out = inst;
+        T_out = T;
+        return 1;
+    }
+}
+
+// A warp takes 32 candidates at a time, one per lane: it gathers the flagged request's columns
+// through cand_idx (the next step's are on their way while this one is searched), turns it into
+// the request that a token-ID migration would pose to the target (re-prefill prompt + generated
+// tokens, decode what is left, within the time that is left) and runs capped_first_attempt.
+// What that does not settle goes on one of the warp's two queues in shared memory, by position
+// in cand_idx: candidates that still need the capped search in full, and candidates for which
+// no feasible instance exists (half of them at the largest configuration), which need
+// Algorithm 1's fallback among the faster instances.  Whenever 32 have gathered on a queue each
+// lane takes one of them, so the long, divergent searches always run with all lanes busy.
+constexpr int kRerouteThreads = GS_REROUTE_THREADS;
+constexpr int kRerouteQueue = 64;           // per warp and queue: at most 31 left over + the 32 of a step
 
 struct Candidate {
     float x, y, D, d_cap;
     unsigned need, rem;
     bool valid;
 };
+struct RawCandidate { int cur, gen, tot, xin; float slo, elapsed; };
 
-__global__ void __launch_bounds__(kRerouteThreads, 4)
+__global__ void __launch_bounds__(kRerouteThreads, 1)
 reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__ cand_count, int64_t cand_capacity,
                const int32_t *__restrict__ assigned, const int32_t *__restrict__ generated,
                const int32_t *__restrict__ pred_len, const float *__restrict__ elapsed,
                const float *__restrict__ slo, const int32_t *__restrict__ prompt_len, int64_t n_active,
-               int n_types_alloc,
-               const Row *__restrict__ g_rows, const uint2 *__restrict__ g_row_bounds,
-             const float2 *__restrict__ g_group_bounds,
-               const unsigned char *__restrict__ g_start_table,
-               const TypeHeader *__restrict__ g_headers, const int *__restrict__ table_info,
+               const TableSource src,
                int32_t *__restrict__ out_inst, float *__restrict__ out_est,
                float *__restrict__ out_slack, uint8_t *__restrict__ out_tier, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    asm volatile("griddepcontrol.wait;" ::: "memory");       // (the tables are the prologue's)
-    const int M = table_info[2];
-    const unsigned kv_max = (unsigned)table_info[8];      // no instance has more free KV than this
-    Tables tb;
-    unsigned char *after = stage_tables(smem, n_types_alloc, g_rows, g_row_bounds, g_group_bounds, g_start_table, g_headers,
-                                        table_info, tb);
-    unsigned *queue = reinterpret_cast<unsigned *>(after) + (threadIdx.x >> 5) * kRerouteQueue;
+    constexpr int kWarps = kRerouteThreads / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // (the tables are the prologue's, the candidates the scan's)
+    const TableImage im = carve_tables<false, true>(smem, src.n_types_alloc);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(shared_addr(im.bar)) : "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
     __syncthreads();
+    if (threadIdx.x == 0) start_table_copies<false, true>(im, src);
+    unsigned *queue_full = reinterpret_cast<unsigned *>(im.end) + warp * (2 * kRerouteQueue);
+    unsigned *queue_fall = queue_full + kRerouteQueue;
 
     int64_t n = *cand_count;
     if (n > cand_capacity) n = cand_capacity;
-    const int lane = threadIdx.x & 31;
     unsigned bad = 0;
-    int q_count = 0;                               // entries on this warp's queue (same in all lanes)
-
-    // the request that candidate j poses (j < n < 2^31)
-    auto load_candidate = [&](int64_t j, bool valid) {
-        Candidate c;
-        int64_t i = valid ? (int64_t)cand_idx[j] : 0;
+    // position in cand_idx -> index of the active request (-1 past the end), and its columns
+    auto index_at = [&](int64_t j) { return j < n ? cand_idx[j] : -1; };
+    auto gather = [&](int idx, bool valid) {
+        int64_t i = idx;
         if (i < 0 || i >= n_active) { i = 0; if (valid) bad |= GS_DEV_BAD_INSTANCE; }
-        int cur = assigned[i], gen = generated[i], tot = pred_len[i], xin = prompt_len[i];
-        if (cur < 0) { cur = 0; bad |= GS_DEV_BAD_INSTANCE; }
-        if (cur >= M) { cur = M - 1; bad |= GS_DEV_BAD_INSTANCE; }
-        if (gen < 0) { gen = 0; bad |= GS_DEV_BAD_VALUE; }
-        if (tot < 0) { tot = 0; bad |= GS_DEV_BAD_VALUE; }
-        if (xin < 0) { xin = 0; bad |= GS_DEV_BAD_VALUE; }
+        RawCandidate r;
+        r.cur = assigned[i]; r.gen = generated[i]; r.tot = pred_len[i]; r.xin = prompt_len[i];
+        r.slo = slo[i]; r.elapsed = elapsed[i];
+        return r;
+    };
+    const int64_t n_steps = (n + 31) >> 5;
+    const int64_t stride = (int64_t)gridDim.x * kWarps;
+    int64_t step = (int64_t)blockIdx.x * kWarps + warp;
+    // two steps ahead: the indices; one step ahead: the columns
+    int idx_next = step < n_steps ? index_at(step * 32 + lane) : -1;
+    RawCandidate raw_next = gather(idx_next, step < n_steps && step * 32 + lane < n);
+    idx_next = step + stride < n_steps ? index_at((step + stride) * 32 + lane) : -1;
+
+    {
+        const bool arrived = wait_barrier(im.bar, 0u);
+        if (!__syncthreads_and(arrived)) {         // see route_kernel
+            if (threadIdx.x == 0) atomicOr(status, (unsigned)GS_DEV_TIMEOUT);
+            wait_barrier(im.bar, 0u);
+            return;
+        }
+    }
+    const int M = im.info[2];
+    const unsigned kv_max = (unsigned)im.info[8];         // no instance has more free KV than this
+    Tables tb;
+    tb.headers = im.headers; tb.row_bounds = im.row_bounds; tb.group_bounds = im.group_bounds;
+    tb.start_table = im.start_table; tb.rows = im.rows; tb.row_p = nullptr; tb.cand = im.cand;
+    tb.pool = im.pool; tb.bucket_list = im.bucket_list; tb.start_list = im.start_list; tb.chord = im.chord;
+    tb.n_types = im.info[1] != 0 ? 0 : im.info[3];       // unusable bounds: every candidate is scored against every instance
+    int n_full = 0, n_fall = 0;                           // entries on the warp's queues (same in all lanes)
+
+    // the request that a candidate poses
+    auto pose = [&](const RawCandidate &r, bool valid) {
+        Candidate c;
+        int cur = r.cur, gen = r.gen, tot = r.tot, xin = r.xin;
+        if (cur < 0) { cur = 0; if (valid) bad |= GS_DEV_BAD_INSTANCE; }
+        if (cur >= M) { cur = M - 1; if (valid) bad |= GS_DEV_BAD_INSTANCE; }
+        if ((gen | tot | xin) < 0) {
+            gen = max(gen, 0); tot = max(tot, 0); xin = max(xin, 0);
+            if (valid) bad |= GS_DEV_BAD_VALUE;
+        }
         c.rem = (unsigned)max(tot - gen, 0);
         const unsigned xu = (unsigned)xin + (unsigned)gen;                    // < 2^32
         const unsigned long long need64 = (unsigned long long)xu + c.rem;
         c.need = need64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (unsigned)need64;     // kv < 2^31 anyway
         c.x = __uint2float_rn(xu); c.y = __uint2float_rn(c.rem);
-        c.D = __fsub_rn(slo[i], elapsed[i]);                                  // time left
+        c.D = __fsub_rn(r.slo, r.elapsed);                                    // time left
         c.d_cap = tb.rows[row_pos(cur)].d;
         c.valid = valid;
         return c;
@@ -1108,14 +1252,20 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
         out_slack[j] = tier ? __fsub_rn(D, T) : 0.f;
         if (out_tier) out_tier[j] = (uint8_t)tier;
     };
-    // the fallback for (up to) the newest 32 candidates of the queue, one per lane
-    auto drain = [&]() {
-        const int cnt = min(q_count, 32);
-        q_count -= cnt;
+    // appends the lanes that vote `push` to a queue
+    auto append = [&](unsigned *queue, int &count, bool push, unsigned entry) {
+        const unsigned votes = __ballot_sync(0xFFFFFFFFu, push);
+        if (push) queue[GS_CHECKED(g_route_index_errors, count + __popc(votes & ((1u << lane) - 1u)), kRerouteQueue)] = entry;
+        count += __popc(votes);
+    };
+    // the fallback for (up to) the newest 32 candidates of its queue, one per lane
+    auto drain_fall = [&]() {
+        const int cnt = min(n_fall, 32);
+        n_fall -= cnt;
         const bool active = lane < cnt;
-        const int64_t j = active ? (int64_t)queue[q_count + lane] : 0;
+        const int64_t j = active ? (int64_t)queue_fall[n_fall + lane] : 0;
         __syncwarp();                              // the slots may be written again
-        const Candidate c = load_candidate(j, active);
+        const Candidate c = pose(gather(active ? cand_idx[j] : 0, active), active);
         int g = -1; float T = 0.f; unsigned tier = 0;
         bool settled = !active;
         if (active && c.rem > 0 && tb.n_types > 0) {
@@ -1127,59 +1277,85 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
         // warp scores every instance
         unsigned todo = __ballot_sync(0xFFFFFFFFu, !settled);
         while (todo) {
-            const int src = __ffs(todo) - 1;
+            const int from = __ffs(todo) - 1;
             todo &= todo - 1;
-            const float xs = __shfl_sync(0xFFFFFFFFu, c.x, src), ys = __shfl_sync(0xFFFFFFFFu, c.y, src);
-            const float Dsrc = __shfl_sync(0xFFFFFFFFu, c.D, src), caps = __shfl_sync(0xFFFFFFFFu, c.d_cap, src);
-            const unsigned needs = __shfl_sync(0xFFFFFFFFu, c.need, src);
+            const float xs = __shfl_sync(0xFFFFFFFFu, c.x, from), ys = __shfl_sync(0xFFFFFFFFu, c.y, from);
+            const float Ds = __shfl_sync(0xFFFFFFFFu, c.D, from), caps = __shfl_sync(0xFFFFFFFFu, c.d_cap, from);
+            const unsigned needs = __shfl_sync(0xFFFFFFFFu, c.need, from);
             int gg; float TT; unsigned tt;
-            exhaustive_pick<true>(tb.rows, M, xs, ys, Dsrc, needs, caps, lane, gg, TT, tt);
-            if (lane == src) { g = gg; T = TT; tier = tt; }
+            exhaustive_pick<true>(tb.rows, M, xs, ys, Ds, needs, caps, lane, gg, TT, tt);
+            if (lane == from) { g = gg; T = TT; tier = tt; }
         }
         if (active) store(j, g, T, tier, c.D);
     };
-
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31); base < n; base += stride) {
-        const int64_t j = base + lane;
-        const Candidate c = load_candidate(j, j < n);
-        float T = 0.f;
-        // (see route_kernel: L_out == 0 skips the search; so does a request that fits no instance's free KV)
-        const float Ds = (c.valid && c.rem > 0 && c.need <= kv_max) ? c.D : -1.0f;
-        const int g = pick_instance<true, false>(tb, c.x, c.y, Ds, Ds + 1e-30f, c.need, c.d_cap, T);
-        if (c.valid && g >= 0) store(j, g, T, 1u, c.D);
-        // the rest is queued for the fallback
-        const bool push = c.valid && g < 0;
-        const unsigned votes = __ballot_sync(0xFFFFFFFFu, push);
-        if (push) queue[q_count + __popc(votes & ((1u << lane) - 1u))] = (unsigned)j;
-        q_count += __popc(votes);
+    // the capped search in full for (up to) the newest 32 candidates of its queue
+    auto drain_full = [&]() {
+        const int cnt = min(n_full, 32);
+        n_full -= cnt;
+        const bool active = lane < cnt;
+        const int64_t j = active ? (int64_t)queue_full[n_full + lane] : 0;
         __syncwarp();
-        while (q_count >= 32) drain();
+        const Candidate c = pose(gather(active ? cand_idx[j] : 0, active), active);
+        float T = 0.f;
+        const float Ds = active ? c.D : -1.0f;     // (queued here: rem > 0, need <= kv_max)
+        const int g = pick_instance<true, false>(tb, c.x, c.y, Ds, Ds + 1e-30f, c.need, c.d_cap, T);
+        if (active && g >= 0) store(j, g, T, 1u, c.D);
+        append(queue_fall, n_fall, active && g < 0, (unsigned)j);
+        __syncwarp();
+    };
+
+    for (; step < n_steps; step += stride) {
+        const int64_t j = step * 32 + lane;
+        const RawCandidate raw = raw_next;
+        const bool valid = j < n;
+        // the columns of the next step, the indices of the one after it
+        raw_next = gather(idx_next, step + stride < n_steps && (step + stride) * 32 + lane < n);
+        idx_next = step + 2 * stride < n_steps ? index_at((step + 2 * stride) * 32 + lane) : -1;
+        const Candidate c = pose(raw, valid);
+        int g = -1; float T = 0.f;
+        int verdict = -1;          // nothing left to decode, more KV than any instance has free, unusable tables: the fallback's queue
+        if (valid && c.rem > 0 && c.need <= kv_max && tb.n_types > 0)
+            verdict = capped_first_attempt(tb, c.x, c.y, c.D, c.need, c.d_cap, g, T);
+        if (valid && verdict > 0) store(j, g, T, 1u, c.D);
+        if (valid && verdict <= 0) GS_COUNT(kCountQueued, 1);
+        if (valid && verdict < 0) GS_COUNT(kCountFallback, 1);
+        append(queue_full, n_full, valid && verdict == 0, (unsigned)j);
+        append(queue_fall, n_fall, valid && verdict < 0, (unsigned)j);
+        __syncwarp();
+        for (;;) {
+            if (n_fall >= 32) drain_fall();
+            else if (n_full >= 32) drain_full();
+            else break;
+        }
     }
-    while (q_count > 0) drain();
+    while (n_full > 0) {
+        drain_full();
+        if (n_fall >= 32) drain_fall();
+    }
+    while (n_fall > 0) drain_fall();
     if (bad) atomicOr(status, bad);
 }
 
 static size_t reroute_smem_bytes(int n_types) {       // the tables of n_types types and the warps' queues
-    return kTablesSmemFixed + kRouteSmemPerType * n_types + (size_t)(kRerouteThreads / 32) * kRerouteQueue * sizeof(unsigned);
+    return route_smem_bytes(n_types, false, false) - (size_t)(route_threads(false, 1) / 32) * kQueueCap * sizeof(unsigned) +
+           (size_t)(kRerouteThreads / 32) * 2 * kRerouteQueue * sizeof(unsigned) + (size_t)n_types * kStartBuckets * sizeof(float4);
 }
 
 cudaError_t launch_reroute(gs_ctx *ctx, const int32_t *cand_idx, const int64_t *cand_count, int64_t cand_capacity,
                            const int32_t *assigned, const int32_t *generated, const int32_t *pred_len,
                            const float *elapsed, const float *slo, const int32_t *prompt_len, int64_t n_active,
-                           int n_types, int32_t *out_inst, float *out_est, float *out_slack, uint8_t *out_tier,
+                           int n_instances, int n_types, int32_t *out_inst, float *out_est, float *out_slack, uint8_t *out_tier,
                            cudaStream_t st)
 {
     if (cand_capacity == 0) return cudaSuccess;
     const size_t smem = reroute_smem_bytes(n_types);
     int64_t blocks = (cand_capacity + kRerouteThreads - 1) / kRerouteThreads;
-    const int64_t cap = (int64_t)ctx->n_sm * ctx->reroute_ctas_per_sm[n_types];
-    if (blocks > cap) blocks = cap;
+    if (blocks > ctx->n_sm) blocks = ctx->n_sm;       // one CTA per SM: its tables fill most of the shared memory
     LaunchTimer timer(ctx, GS_K_REROUTE, st);
+    const TableSource src = table_source(ctx, n_instances, n_types);
     reroute_kernel<<<(unsigned)blocks, kRerouteThreads, smem, st>>>(
         cand_idx, cand_count, cand_capacity, assigned, generated, pred_len, elapsed, slo, prompt_len, n_active,
-        n_types, ctx->s.rows, ctx->s.row_bounds, ctx->s.group_bounds, ctx->s.start_table, ctx->s.headers, ctx->s.table_info,
-        out_inst, out_est, out_slack, out_tier, ctx->s.status);
+        src, out_inst, out_est, out_slack, out_tier, ctx->s.status);
     return cudaGetLastError();
 }
 
@@ -1210,13 +1386,6 @@ cudaError_t configure_route(gs_ctx *ctx)
     e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)reroute_smem_bytes(GS_MAX_TYPES));
     if (e != cudaSuccess) return e;
-    for (int t = 0; t <= GS_MAX_TYPES; ++t) {
-        int occ = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, reroute_kernel, kRerouteThreads,
-                                                          reroute_smem_bytes(t));
-        if (e != cudaSuccess) return e;
-        ctx->reroute_ctas_per_sm[t] = occ > 0 ? occ : 1;
-    }
     return cudaSuccess;
 }
 

@@ -76,6 +76,16 @@ def test_reroute_on_adversarial_pools(checked, case):
     T.test_reroute_on_adversarial_pools(checked, case)
 
 
+@pytest.mark.parametrize("case", [3, 8])
+def test_reroute_of_requests_that_are_not_at_risk(checked, case):
+    T.test_reroute_of_requests_that_are_not_at_risk(checked, case)
+
+
+@pytest.mark.parametrize("case", [4, 9])
+def test_reroute_with_time_left_on_instance_estimates(checked, case):
+    T.test_reroute_with_time_left_on_instance_estimates(checked, case)
+
+
 @pytest.mark.parametrize("case", [0, 5, 13])
 def test_prefix_on_adversarial_pools(checked, case):
     T.test_prefix_on_adversarial_pools(checked, case)

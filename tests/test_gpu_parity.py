@@ -686,6 +686,82 @@ def test_reroute_on_adversarial_pools(gs, case):
     assert gs.device_status() == 0
 
 
+def gpu_reroute_listed(gs, pool, act, prompt, alpha, cand_idx):
+    """Re-routes the listed active requests (a caller-made list: the scan is not involved)."""
+    dev = gs.device
+    cols = [torch.from_numpy(c).to(dev) for c in act.columns()]
+    x = torch.from_numpy(prompt).to(dev)
+    c = len(cand_idx)
+    cand = torch.from_numpy(np.ascontiguousarray(cand_idx, np.int32)).to(dev)
+    count = torch.tensor([c], dtype=torch.int64, device=dev)
+    new_inst = torch.full((c + 3,), -7, dtype=torch.int32, device=dev)
+    est = torch.full((c + 3,), float("nan"), dtype=torch.float32, device=dev)
+    slack = torch.full((c + 3,), float("nan"), dtype=torch.float32, device=dev)
+    tier = torch.full((c + 3,), 9, dtype=torch.uint8, device=dev)
+    gs.reroute_candidates(cand, count, *cols, x, pool, alpha, new_inst, est, slack, tier, cand_capacity=c)
+    torch.cuda.synchronize(dev)
+    assert (new_inst[c:] == -7).all() and (tier[c:] == 9).all()
+    return new_inst.cpu().numpy()[:c], est.cpu().numpy()[:c], slack.cpu().numpy()[:c], tier.cpu().numpy()[:c]
+
+
+def assert_reroute_matches(got, ref):
+    new_inst, est, slack, tier = got
+    np.testing.assert_array_equal(new_inst, ref.new_instance)
+    np.testing.assert_array_equal(tier, ref.tier)
+    np.testing.assert_array_equal(est.view(np.uint32), ref.est_ms.view(np.uint32))
+    np.testing.assert_array_equal(slack.view(np.uint32), ref.slack_ms.view(np.uint32))
+
+
+@pytest.mark.parametrize("case", [0, 2, 3, 5, 8, 10])
+def test_reroute_of_requests_that_are_not_at_risk(gs, case):
+    """The candidate list is the caller's: requests with time to spare, whose unrestricted pick is
+    often an instance no faster than the current one, must still be held to faster instances."""
+    rng = np.random.default_rng(2100 + case)
+    types, inst = _random_pool(rng, **FUZZ_CASES[case])
+    act = W.make_active(W.CONFIGS[3], types, inst.n_instances, seed=40 + case, n=30_000)
+    act.slo_ms[:] = act.elapsed_ms + np.exp(rng.uniform(np.log(5.0), np.log(4.0e5), act.n)).astype(np.float32)
+    act.generated_tokens[::13] = act.pred_len[::13]              # nothing left to decode
+    prompt = np.clip(np.rint(np.exp(rng.normal(6.0, 1.5, act.n))), 0, 1 << 20).astype(np.int32)
+    cand = np.sort(rng.choice(act.n, size=act.n * 3 // 4, replace=False)).astype(np.int32)
+    pool = pool_of(gs, types, inst)
+    t32 = oracle.instance_table(types, inst, 0.25, "f32")
+    ref = oracle.reroute(t32, cand, *act.columns(), prompt)
+    assert_reroute_matches(gpu_reroute_listed(gs, pool, act, prompt, 0.25, cand), ref)
+    if case == 5:                  # identical instances: nothing is strictly faster, nobody moves
+        assert (ref.tier == 0).all() and (ref.new_instance == -1).all()
+    else:
+        assert (ref.tier == 1).any() and (ref.tier != 1).any()
+    cur_d = t32.d[act.assigned_inst[cand]]
+    assert (t32.d[ref.new_instance[ref.tier > 0]] < cur_d[ref.tier > 0]).all()   # only strictly faster instances
+    assert gs.device_status() == 0
+
+
+@pytest.mark.parametrize("case", [0, 4, 7, 9])
+def test_reroute_with_time_left_on_instance_estimates(gs, case):
+    """Time left equal to, one ulp below and one ulp above the exact T of some instance for the
+    re-posed request: the feasibility tests and every bound before them sit on their edge."""
+    rng = np.random.default_rng(2200 + case)
+    types, inst = _random_pool(rng, **FUZZ_CASES[case])
+    t32 = oracle.instance_table(types, inst, 0.5, "f32")
+    n = 24_000
+    act = W.make_active(W.CONFIGS[3], types, inst.n_instances, seed=60 + case, n=n)
+    prompt = np.clip(np.rint(np.exp(rng.normal(6.0, 1.0, n))), 1, 1 << 18).astype(np.int32)
+    x = (prompt.astype(np.int64) + act.generated_tokens).astype(np.float32)
+    y = np.maximum(act.pred_len - act.generated_tokens, 0).astype(np.float32)
+    target = rng.integers(0, inst.n_instances, n)
+    t1 = (x.astype(np.float64) * t32.p[target].astype(np.float64) + t32.q[target].astype(np.float64)).astype(np.float32)
+    T = (y.astype(np.float64) * t32.d[target].astype(np.float64) + t1.astype(np.float64)).astype(np.float32)   # see _canonical_T
+    step = rng.integers(-1, 2, n)
+    T = np.where(step < 0, np.nextafter(T, np.float32(-np.inf)), np.where(step > 0, np.nextafter(T, np.float32(np.inf)), T))
+    act.elapsed_ms[:] = 0.0                                      # time left = slo, bit for bit
+    act.slo_ms[:] = T.astype(np.float32)
+    cand = np.arange(n, dtype=np.int32)
+    pool = pool_of(gs, types, inst)
+    ref = oracle.reroute(t32, cand, *act.columns(), prompt)
+    assert_reroute_matches(gpu_reroute_listed(gs, pool, act, prompt, 0.5, cand), ref)
+    assert gs.device_status() == 0
+
+
 # --------------------------------------------------------------------------------------
 # routing with the prefix-cache term of Eq. 2
 # --------------------------------------------------------------------------------------
