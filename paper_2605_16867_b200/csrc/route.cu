@@ -565,7 +565,7 @@ __device__ __forceinline__ unsigned first_pass_of_eight(const Tables &tb, int k,
 //   2. the start table gives the first entry worth a look in the record list of that type and
 //      bucket of L_out (the rows that can be the first of the type to pass; see the prologue);
 //      four entries from there are tested (with per-row p, where there are no such lists:
-//      sixteen row bounds of the full list), and the first row that passes is scored exactly
+//      eight row bounds of the full list), and the first row that passes is scored exactly
 //      as the definition says and checked against the deadline and the instance's free KV;
 //   3. no later type may be able to do better: its largest d is below the pick's, or even its
 //      least q with the pick's d misses the deadline.
@@ -601,11 +601,9 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
                      start_slot(Rg, h.y, ry, __int_as_float(geo.w), __int_as_float(geo.z)), tb.n_types * kStartBuckets * kStartSlots);
     unsigned first = kNoRow;
     if (kRowP) {
-        // rows of a group differ in p: sixteen row bounds of the group's full list
+        // rows of a group differ in p: eight row bounds of the group's full list
         const int k = geo.x + 8 * tb.start_table[cell];
-        const int k2 = min(k + 8, geo.x + geo.y - 8);    // (the last group of a type is tested twice)
-        first = first_pass_of_eight<kRowP>(tb, k2, x, y, Dm, kNoRow);
-        first = first_pass_of_eight<kRowP>(tb, k, x, y, Dm, first);
+        first = first_pass_of_eight<kRowP>(tb, k, x, y, Dm, kNoRow);
     } else {
         // the record list of this type and bucket of L_out: only rows that can be the first to pass
         const unsigned list = tb.bucket_list[t * kStartBuckets + ybucket];
