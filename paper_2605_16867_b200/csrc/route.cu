@@ -292,48 +292,23 @@ __device__ __forceinline__ void search_eight(const Tables &tb, int k, float x, f
         pb = *reinterpret_cast<const float4 *>(tb.row_p + k + 4);
     }
     const float pl[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-    // the eight bounds at once (NaN, which passes no test, for padding and for rows that the
-    // cap excludes) ...
-    GS_COUNT(kCountBound, 8);
-    float b[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const unsigned qw = (j & 1) ? r[j >> 1].z : r[j >> 1].x, dw = (j & 1) ? r[j >> 1].w : r[j >> 1].y;
-        const float d_lo = __uint_as_float(dw);
-        const float base = kRowP ? __fmaf_rn(pl[j], x, __uint_as_float(qw)) : __uint_as_float(qw);
-        b[j] = __fmaf_rn(d_lo, y, base);
-        if (kCapped) b[j] = d_lo < d_cap ? b[j] : __int_as_float(0x7FC00000);
-    }
-    // ... then the rows whose bound passes, one at a time, smallest d first (one copy of the
-    // scoring code, run as often as the busiest lane has rows to score).  While nothing has been
-    // found the row with the least bound goes first and the others are then held against its T.
-    auto passing = [&](float limit) {
-        unsigned m = 0;
+    for (int c = 3; c >= 0; --c) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) m |= (b[j] <= limit) ? (1u << j) : 0u;
-        return m;
-    };
-    bool blind = g_best < 0;
-    unsigned m = passing(blind ? fminf(fminf(fminf(b[0], b[1]), fminf(b[2], b[3])), fminf(fminf(b[4], b[5]), fminf(b[6], b[7])))
-                               : (kRowP ? T_best + 1e-30f : Rg));
-    unsigned done = 0;
-    while (m) {
-        const int j = 31 - __clz(m);
-        m &= ~(1u << j);
-        done |= 1u << j;
-        const int inst = (int)(tb.row_bounds[k + ((((j >> 1) ^ sw) << 1) | (j & 1))].x & kRowTagMask);
-        const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
-        if ((!kCapped || row.d < d_cap) && (any_kv || need <= (unsigned)row.kv)) {
+        for (int e = 1; e >= 0; --e) {
+            const unsigned qw = e ? r[c].z : r[c].x, dw = e ? r[c].w : r[c].y;
+            const float R = kRowP ? T_best + 1e-30f : Rg;
+            if (!row_may_pass<kCapped, kRowP>(qw, dw, pl[2 * c + e], x, y, R, d_cap)) continue;
+            const int inst = (int)(qw & kRowTagMask);
+            const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
+            if (kCapped && !(row.d < d_cap)) continue;
+            if (!any_kv && !(need <= (unsigned)row.kv)) continue;
             GS_COUNT(kCountExact, 1);
             const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));   // Eq. 2, H = 0
             if (T < T_best || (T == T_best && inst < g_best) || g_best < 0) {
                 T_best = T; g_best = inst;
                 Rg = __fmaf_rn(-p_lo, x, T_best) + 1e-30f;
             }
-        }
-        if (blind && m == 0) {                 // the rest of the group, against what is known now
-            blind = false;
-            m = passing(kRowP ? T_best + 1e-30f : Rg) & ~done;
         }
     }
 }
@@ -565,7 +540,7 @@ __device__ __forceinline__ unsigned first_pass_of_eight(const Tables &tb, int k,
 //   2. the start table gives the first entry worth a look in the record list of that type and
 //      bucket of L_out (the rows that can be the first of the type to pass; see the prologue);
 //      four entries from there are tested (with per-row p, where there are no such lists:
-//      eight row bounds of the full list), and the first row that passes is scored exactly
+//      sixteen row bounds of the full list), and the first row that passes is scored exactly
 //      as the definition says and checked against the deadline and the instance's free KV;
 //   3. no later type may be able to do better: its largest d is below the pick's, or even its
 //      least q with the pick's d misses the deadline.
@@ -601,9 +576,11 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
                      start_slot(Rg, h.y, ry, __int_as_float(geo.w), __int_as_float(geo.z)), tb.n_types * kStartBuckets * kStartSlots);
     unsigned first = kNoRow;
     if (kRowP) {
-        // rows of a group differ in p: eight row bounds of the group's full list
+        // rows of a group differ in p: sixteen row bounds of the group's full list
         const int k = geo.x + 8 * tb.start_table[cell];
-        first = first_pass_of_eight<kRowP>(tb, k, x, y, Dm, kNoRow);
+        const int k2 = min(k + 8, geo.x + geo.y - 8);    // (the last group of a type is tested twice)
+        first = first_pass_of_eight<kRowP>(tb, k2, x, y, Dm, kNoRow);
+        first = first_pass_of_eight<kRowP>(tb, k, x, y, Dm, first);
     } else {
         // the record list of this type and bucket of L_out: only rows that can be the first to pass
         const unsigned list = tb.bucket_list[t * kStartBuckets + ybucket];
