@@ -621,6 +621,88 @@ __device__ __forceinline__ bool fast_pick(const Tables &tb, float cand_z0, float
     return true;
 }
 
+// The same first attempt for pools whose types overlap in d, where a later type often may hold
+// a better instance than the first one's pick: instead of giving up there it goes on to that
+// type (and on a type whose record list ends inside the window without a row passing), keeping
+// the best pick so far; it gives up only where a type's answer stays open (no list, nothing
+// passes among the entries tested although the list goes on, the scored row is not feasible).
+// Costs a few instructions more per request than fast_pick even when one type settles it, so
+// the kernel for small batches (one request per lane) uses it and the one for large batches
+// does not.
+template <bool kRowP>
+__device__ __forceinline__ bool fast_pick_several(const Tables &tb, float cand_z0, float cand_inv, float x, float y,
+                                          float D, unsigned need, int &g_out, float &T_out)
+{
+    const float Dm = D + 1e-30f;                 // see route_kernel
+    float ry;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(ry) : "f"(y));
+    const float sc = fminf(fmaxf((Dm * ry - cand_z0) * cand_inv, 0.f), (float)(kCandSlots - 1));
+    unsigned mask = tb.cand[GS_CHECKED(g_route_index_errors, __float2int_rd(sc), kCandSlots)];
+    const int ybucket = min((int)(__float_as_uint(y) >> (23 - kBucketBits)) - (127 << kBucketBits), kStartBuckets - 1);
+    int g_best = -1;
+    float T_best = 0.f, d_best = -1.0f, d_floor = 0.f;
+    for (;;) {
+        int t = -1;
+        float4 h = make_float4(0.f, 0.f, 0.f, 0.f);
+        float Rg = 0.f;
+        while (mask) {
+            const int tt = __ffs(mask) - 1;
+            mask &= mask - 1;
+            h = *reinterpret_cast<const float4 *>(&tb.headers[tt]);               // p_lo, q_lo, d_lo, d_max
+            if (h.w < d_best) { mask = 0; break; }                                // nor can any type after it
+            Rg = __fmaf_rn(-h.x, x, Dm);
+            GS_COUNT(kCountTypeTest, 1);
+            if (__fmaf_rn(fmaxf(h.z, d_floor), y, h.y) <= Rg) { t = tt; break; }
+        }
+        if (t < 0) break;
+        const int4 geo = *(reinterpret_cast<const int4 *>(&tb.headers[t]) + 1);   // base, n_padded, inv_w, d0
+        const int cell = GS_CHECKED(g_route_index_errors, (t * kStartBuckets + ybucket) * kStartSlots +
+                         start_slot(Rg, h.y, ry, __int_as_float(geo.w), __int_as_float(geo.z)), tb.n_types * kStartBuckets * kStartSlots);
+        unsigned first = kNoRow;
+        if (kRowP) {
+            const int k = geo.x + 8 * tb.start_table[cell];
+            const int k2 = min(k + 8, geo.x + geo.y - 8);
+            first = first_pass_of_eight<kRowP>(tb, k2, x, y, Dm, kNoRow);
+            first = first_pass_of_eight<kRowP>(tb, k, x, y, Dm, first);
+            if (first == kNoRow) return false;
+        } else {
+            const unsigned list = tb.bucket_list[t * kStartBuckets + ybucket];
+            if (list == kNoList) return false;
+            const uint4 *w = reinterpret_cast<const uint4 *>(tb.pool) +
+                             GS_CHECKED(g_route_index_errors, list + tb.start_list[cell], kPoolEntries / 2 - 3);
+            const uint4 r0 = w[0], r1 = w[1];
+            first = row_may_pass<false, false>(r1.z, r1.w, 0.f, x, y, Rg, 0.f) ? r1.z : first;
+            first = row_may_pass<false, false>(r1.x, r1.y, 0.f, x, y, Rg, 0.f) ? r1.x : first;
+            first = row_may_pass<false, false>(r0.z, r0.w, 0.f, x, y, Rg, 0.f) ? r0.z : first;
+            first = row_may_pass<false, false>(r0.x, r0.y, 0.f, x, y, Rg, 0.f) ? r0.x : first;
+            if (first == kNoRow) {
+                const uint4 r2 = w[2], r3 = w[3];
+                first = row_may_pass<false, false>(r3.z, r3.w, 0.f, x, y, Rg, 0.f) ? r3.z : first;
+                first = row_may_pass<false, false>(r3.x, r3.y, 0.f, x, y, Rg, 0.f) ? r3.x : first;
+                first = row_may_pass<false, false>(r2.z, r2.w, 0.f, x, y, Rg, 0.f) ? r2.z : first;
+                first = row_may_pass<false, false>(r2.x, r2.y, 0.f, x, y, Rg, 0.f) ? r2.x : first;
+                if (first == kNoRow) {
+                    if (r3.z == kPadQ) continue;
+                    return false;
+                }
+            }
+        }
+        const int inst = (int)(first & kRowTagMask);
+        GS_COUNT(kCountExact, 1);
+        const Row row = tb.rows[GS_CHECKED(g_route_index_errors, row_pos(inst), GS_MAX_INSTANCES)];
+        const float T = __fmaf_rn(row.d, y, __fmaf_rn(row.p, x, row.q));          // Eq. 2, H = 0
+        if (!(T <= D && need <= (unsigned)row.kv)) return false;
+        if (g_best < 0 || row.d > d_best || (row.d == d_best && inst < g_best)) {
+            g_best = inst; T_best = T; d_best = row.d;
+            d_floor = __fmul_rn(row.d, 1.0f - 1.9073486328125e-6f);
+        }
+    }
+    if (g_best < 0) return false;
+    g_out = g_best;
+    T_out = T_best;
+    return true;
+}
+
 // The full search for one request per lane (lanes without a request pass active = false):
 // the just-enough pick over all types, then the fallback of Algorithm 1 -- by the lane itself
 // when several lanes need it, by the whole warp otherwise and for requests that the tables
@@ -868,8 +950,11 @@ route_kernel(const int32_t *__restrict__ prompt_len, const int32_t *__restrict__
             // nothing meets and so ends up in the full search)
             bool settled = false;
             if (fast_on && (unsigned)xi[j] + (unsigned)yi[j] <= kv_max)
-                settled = fast_pick<kRowP>(tb, cand_z0, cand_inv, __int2float_rn(xi[j]), __int2float_rn(yi[j]),
-                                           (valid && yi[j] > 0) ? D[j] : -1.0f, (unsigned)xi[j] + (unsigned)yi[j], g_out[j], T_out[j]);
+                settled = kReqPerThread == 1
+                    ? fast_pick_several<kRowP>(tb, cand_z0, cand_inv, __int2float_rn(xi[j]), __int2float_rn(yi[j]),
+                                               (valid && yi[j] > 0) ? D[j] : -1.0f, (unsigned)xi[j] + (unsigned)yi[j], g_out[j], T_out[j])
+                    : fast_pick<kRowP>(tb, cand_z0, cand_inv, __int2float_rn(xi[j]), __int2float_rn(yi[j]),
+                                       (valid && yi[j] > 0) ? D[j] : -1.0f, (unsigned)xi[j] + (unsigned)yi[j], g_out[j], T_out[j]);
             if (valid && !settled) { slow |= 1u << j; GS_COUNT(kCountQueued, 1); }
         }
         if (kPrefix) {
