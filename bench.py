@@ -640,9 +640,13 @@ def run_gpu(args):
     h_bits = torch.empty((A + 31) // 32, dtype=torch.int32).pin_memory()
     h_cand = torch.empty(A, dtype=torch.int32).pin_memory()
 
+    # (the routing round's results travel back while the scan's inputs arrive: the first call
+    # returns once it is enqueued, the second one waits for both)
     def e2e_step():
-        gs.route_batch_host(*h_req, wl.types, wl.instances, alpha, h_idx, h_est, h_slack, stream=stream)
-        return gs.risk_scan_host(*h_act, wl.types, wl.instances, h_bits, h_cand, stream=stream)
+        gs.route_batch_host(*h_req, wl.types, wl.instances, alpha, h_idx, h_est, h_slack, stream=stream, wait=False)
+        n_flagged = gs.risk_scan_host(*h_act, wl.types, wl.instances, h_bits, h_cand, stream=stream)
+        gs.host_wait(stream)
+        return n_flagged
 
     e2e_steps = max(1, min(args.steps, 5))
     n_flag = flagged

@@ -384,6 +384,28 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx,
                       int64_t *out_cand_count, void *cuda_stream);
 
 /*
+ * gs_route_batch_host that returns as soon as all its copies and kernels are enqueued, so that
+ * the results of the routing round (Algorithm 1) travel back to the host while the caller's
+ * next call -- typically gs_risk_scan_host for the same scheduling tick (Sec. 3.4) -- already
+ * sends its inputs the other way.  Same arguments, same results.  The input and output buffers
+ * must stay untouched, and the outputs are not valid, until gs_host_wait, or any later
+ * gs_route_batch_host / gs_risk_scan_host call on this context, has returned GS_OK.  With
+ * pageable (not pinned) host memory the copies, and so the call, block as usual.
+ * Errors: as gs_route_batch_host; what fails on the device later is reported by the call that
+ * waits.
+ */
+GS_API int gs_route_batch_host_deferred(gs_ctx *ctx,
+                        const int32_t *prompt_len, const int32_t *pred_decode_len,
+                        const float *slo_ms, int64_t n_requests,
+                        const gs_instances *inst, const gs_types *types, float ema_alpha,
+                        int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                        uint8_t *out_tier, void *cuda_stream);
+
+/* Waits for everything the *_host calls of this context have enqueued on `cuda_stream` and on
+ * the context's own copy stream.  GS_ERR_CUDA if any of it failed. */
+GS_API int gs_host_wait(gs_ctx *ctx, void *cuda_stream);
+
+/*
  * Risk scan without any allocation.  (The paper has no counterpart: this entry point exists
  * only because of how some callers must run, not because of the method.)
  *

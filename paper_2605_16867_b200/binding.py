@@ -78,6 +78,8 @@ def _declare(lib):
     route_args = [vp, vp, vp, vp, i64, C.POINTER(_Instances), C.POINTER(_Types), f32, vp, vp, vp, vp]
     lib.gs_route_batch.argtypes = route_args + [u32, vp]
     lib.gs_route_batch_host.argtypes = route_args + [vp]
+    lib.gs_route_batch_host_deferred.argtypes = route_args + [vp]
+    lib.gs_host_wait.argtypes = [vp, vp]
     lib.gs_route_batch_prefix.argtypes = [vp, vp, vp, vp, i64, vp, vp, C.c_int, i64, C.POINTER(_Instances),
                                           C.POINTER(_Types), f32, vp, vp, vp, vp, vp]
     lib.gs_route_batch_prefix.restype = C.c_int
@@ -101,7 +103,7 @@ def _declare(lib):
                                          vp, vp, i64, vp, vp, vp]
     lib.gs_risk_scan_noalloc.restype = C.c_int
     for name in ("gs_timing_enable", "gs_timing_read", "gs_create", "gs_destroy", "gs_last_cuda_error", "gs_device_status", "gs_route_batch",
-                 "gs_route_batch_host", "gs_advance_state", "gs_risk_scan", "gs_risk_scan_host"):
+                 "gs_route_batch_host", "gs_route_batch_host_deferred", "gs_host_wait", "gs_advance_state", "gs_risk_scan", "gs_risk_scan_host"):
         getattr(lib, name).restype = C.c_int
     return lib
 
@@ -203,6 +205,7 @@ class GoodServe:
         h = C.c_void_p()
         self._check(self._lib.gs_create(C.byref(h), device, max_instances, max_types))
         self._h = h
+        self._deferred = None
 
     # -- plumbing ------------------------------------------------------------------------
     def _check(self, rc: int):
@@ -390,11 +393,18 @@ class GoodServe:
             _dev_ptr(out_tier, torch.uint8, cap, "out_tier", dev), self._stream(stream)))
 
     def route_batch_host(self, prompt_len, pred_decode_len, slo_ms, types, inst, ema_alpha: float,
-                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier=None, stream=None):
-        """Host-buffer variant: numpy arrays or (pinned) host tensors in and out."""
+                         out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier=None, stream=None,
+                         wait: bool = True):
+        """Host-buffer variant: numpy arrays or (pinned) host tensors in and out.  With
+        ``wait=False`` the call returns once everything is enqueued (gs_route_batch_host_deferred):
+        the outputs are valid after ``host_wait()`` or the next host-buffer call has returned."""
         n = int(prompt_len.shape[0])
         hi, ht = self._host_pool_structs(types, inst)
-        self._check(self._lib.gs_route_batch_host(
+        fn = self._lib.gs_route_batch_host if wait else self._lib.gs_route_batch_host_deferred
+        if not wait:        # what the enqueued copies read and write stays referenced until the wait
+            self._deferred = (prompt_len, pred_decode_len, slo_ms, types, inst, hi, ht,
+                              out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier)
+        self._check(fn(
             self._h, _host_ptr(prompt_len, np.int32, n, "prompt_len"),
             _host_ptr(pred_decode_len, np.int32, n, "pred_decode_len"),
             _host_ptr(slo_ms, np.float32, n, "slo_ms"), n, C.byref(hi), C.byref(ht), float(ema_alpha),
@@ -402,6 +412,11 @@ class GoodServe:
             _host_ptr(out_est_e2e_ms, np.float32, n, "out_est_e2e_ms"),
             _host_ptr(out_slack_ms, np.float32, n, "out_slack_ms"),
             _host_ptr(out_tier, np.uint8, n, "out_tier"), self._stream(stream)))
+
+    def host_wait(self, stream=None):
+        """Waits for what the host-buffer calls have enqueued (gs_host_wait)."""
+        self._check(self._lib.gs_host_wait(self._h, self._stream(stream)))
+        self._deferred = None
 
     def risk_scan_host(self, assigned_inst, generated_tokens, pred_len, elapsed_ms, slo_ms, types, inst,
                        out_flag_bits, out_cand_idx, stream=None) -> int:

@@ -39,13 +39,15 @@ int check_pool(const gs_ctx *ctx, const gs_instances *inst, const gs_types *type
     return GS_OK;
 }
 
-int ensure_stage(gs_ctx *ctx, size_t bytes) {
-    if (bytes <= ctx->stage_bytes) return GS_OK;
-    if (ctx->stage) { cudaFree(ctx->stage); ctx->stage = nullptr; ctx->stage_bytes = 0; }
+// Grows one of the context's staging buffers.  (cudaFree waits for everything the device still
+// has to do, so a buffer that copies enqueued earlier still use is never pulled from under them.)
+int ensure_stage(gs_ctx *ctx, char **stage, size_t *stage_bytes, size_t bytes) {
+    if (bytes <= *stage_bytes) return GS_OK;
+    if (*stage) { cudaFree(*stage); *stage = nullptr; *stage_bytes = 0; }
     const size_t want = bytes + bytes / 8 + 4096;
-    cudaError_t e = cudaMalloc(&ctx->stage, want);
+    cudaError_t e = cudaMalloc(stage, want);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    ctx->stage_bytes = want;
+    *stage_bytes = want;
     return GS_OK;
 }
 
@@ -189,7 +191,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
     if (!ctx) return GS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     gs::Scratch &s = ctx->s;
-    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.chord, s.q_by_g, s.deltas, s.scan_counts, s.status, ctx->stage};
+    void *ptrs[] = {s.rows, s.row_bounds, s.group_bounds, s.row_p, s.start_table, s.headers, s.table_info, s.cand_table, s.pool, s.bucket_list, s.start_list, s.chord, s.q_by_g, s.deltas, s.scan_counts, s.status, ctx->stage, ctx->scan_stage};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->pending) for (auto &t : *ctx->pending) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->free_events) for (cudaEvent_t ev : *ctx->free_events) cudaEventDestroy(ev);
@@ -483,11 +485,11 @@ static int64_t host_piece(int64_t n) {
     return (piece + 1023) & ~(int64_t)1023;
 }
 
-GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
-                        const float *slo_ms, int64_t n_requests,
-                        const gs_instances *inst, const gs_types *types, float ema_alpha,
-                        int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
-                        uint8_t *out_tier, void *cuda_stream)
+static int route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                            const float *slo_ms, int64_t n_requests,
+                            const gs_instances *inst, const gs_types *types, float ema_alpha,
+                            int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                            uint8_t *out_tier, void *cuda_stream, bool wait)
 {
     int rc = check_pool(ctx, inst, types, false);
     if (rc != GS_OK) return rc;
@@ -500,9 +502,11 @@ GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int
     if ((rc = ensure_host_pipe(ctx)) != GS_OK) return rc;
     const size_t n = (size_t)n_requests;
     const size_t bytes = pool_stage_bytes(inst->n_instances, types->n_types) + 6 * pad256(n * 4) + pad256(n);
-    rc = ensure_stage(ctx, bytes);
-    if (rc != GS_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream, out = ctx->host_out_stream;
+    // (an earlier deferred round may still be sending results back from the same buffers)
+    if (cudaStreamSynchronize(out) != cudaSuccess) return cuda_fail(ctx, cudaGetLastError());
+    rc = ensure_stage(ctx, &ctx->stage, &ctx->stage_bytes, bytes);
+    if (rc != GS_OK) return rc;
     Carver c{ctx->stage};
     PoolStage pool;
     cudaError_t e = stage_pool(c, inst, types, &pool, st);
@@ -534,9 +538,41 @@ GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int
         if (out_tier && (e = cudaMemcpyAsync(out_tier + off, dtier + off, len, cudaMemcpyDeviceToHost, out)) != cudaSuccess)
             break;
     }
-    // (also after an error: nothing may still be using the staging buffers when the call returns)
-    const cudaError_t e1 = cudaStreamSynchronize(st), e2 = cudaStreamSynchronize(out);
-    if (e == cudaSuccess) e = e1 != cudaSuccess ? e1 : e2;
+    // (after an error always: nothing may still be using the staging buffers when the call returns)
+    if (wait || e != cudaSuccess) {
+        const cudaError_t e1 = cudaStreamSynchronize(st), e2 = cudaStreamSynchronize(out);
+        if (e == cudaSuccess) e = e1 != cudaSuccess ? e1 : e2;
+    }
+    return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
+}
+
+GS_API int gs_route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                        const float *slo_ms, int64_t n_requests,
+                        const gs_instances *inst, const gs_types *types, float ema_alpha,
+                        int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                        uint8_t *out_tier, void *cuda_stream)
+{
+    return route_batch_host(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, inst, types, ema_alpha,
+                            out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, cuda_stream, true);
+}
+
+GS_API int gs_route_batch_host_deferred(gs_ctx *ctx, const int32_t *prompt_len, const int32_t *pred_decode_len,
+                        const float *slo_ms, int64_t n_requests,
+                        const gs_instances *inst, const gs_types *types, float ema_alpha,
+                        int32_t *out_instance_idx, float *out_est_e2e_ms, float *out_slack_ms,
+                        uint8_t *out_tier, void *cuda_stream)
+{
+    return route_batch_host(ctx, prompt_len, pred_decode_len, slo_ms, n_requests, inst, types, ema_alpha,
+                            out_instance_idx, out_est_e2e_ms, out_slack_ms, out_tier, cuda_stream, false);
+}
+
+GS_API int gs_host_wait(gs_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return GS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GS_ERR_NO_DEVICE;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+    if (e == cudaSuccess && ctx->host_pipe_ready) e = cudaStreamSynchronize(ctx->host_out_stream);
     return e == cudaSuccess ? GS_OK : cuda_fail(ctx, e);
 }
 
@@ -562,10 +598,10 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx, const int32_t *assigned_inst, const in
     const size_t cap = (size_t)(cand_capacity < n_active ? cand_capacity : n_active);
     const size_t bytes = pool_stage_bytes(inst->n_instances, types->n_types) + 5 * pad256(n * 4) +
                          pad256(words * 4) + pad256(cap * 4) + 256;
-    rc = ensure_stage(ctx, bytes);
+    rc = ensure_stage(ctx, &ctx->scan_stage, &ctx->scan_stage_bytes, bytes);
     if (rc != GS_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream, out = ctx->host_out_stream;
-    Carver c{ctx->stage};
+    Carver c{ctx->scan_stage};
     PoolStage pool;
     cudaError_t e = stage_pool(c, inst, types, &pool, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);

@@ -162,8 +162,10 @@ struct gs_ctx {
     int last_cuda_error;
     // staging for the *_host entry points (device memory, grown on demand), and what their
     // pipeline of copies and kernels needs (created by the first such call)
-    char *stage;
+    char *stage;                             // ... of gs_route_batch_host
     size_t stage_bytes;
+    char *scan_stage;                        // ... of gs_risk_scan_host (its own: a routing round's results may still be
+    size_t scan_stage_bytes;                 //     on their way back when the scan's inputs arrive)
     cudaStream_t host_out_stream;            // results travel back on it while the next piece's inputs arrive
     cudaEvent_t host_events[GS_HOST_PIECES]; // piece k computed
     int64_t *host_counts;                    // pinned: candidates up to and including piece k

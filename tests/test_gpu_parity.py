@@ -8,7 +8,7 @@ import pytest
 
 import oracle
 import workloads as W
-from parity_util import (REL_TOL, assert_route_matches_f32_oracle, check_risk_against_f64,
+from parity_util import (REL_TOL, GpuRoute, assert_route_matches_f32_oracle, check_risk_against_f64,
                          check_route_against_f64, gpu_risk, gpu_route, gpu_route_direct, gpu_route_prefix,
                          unpack_bits)
 
@@ -347,6 +347,40 @@ def test_host_entry_points_match_device_ones(gs, n_req, n_act):
     assert count2 == risk.count
     np.testing.assert_array_equal(small, risk.cand_idx[:small.size])
     assert gs.device_status() == 16                              # GS_DEV_CAND_TRUNCATED
+
+
+def test_deferred_host_routing_overlaps_the_scan_and_changes_nothing(gs):
+    """gs_route_batch_host_deferred returns once its work is enqueued; the scan's host call that
+    follows sends its inputs while the round's results come back.  Pinned buffers (the copies are
+    then really asynchronous); twice in a row, so that the second round meets the first one's
+    buffers; the results are the blocking calls', and the oracle's."""
+    wl = W.make_workload(2, n_requests=600_001, n_active=900_003)
+    t32 = oracle.instance_table(wl.types, wl.instances, 0.5, "f32")
+    ref = oracle.route(t32, *wl.requests.columns(), threads=8)
+    flags = oracle.risk(t32, *wl.active.columns(), threads=8).flag
+    rbits, rcand, rcount = oracle.compact(flags)
+    pin = lambda a: torch.from_numpy(a).pin_memory()            # noqa: E731
+    req = [pin(c) for c in wl.requests.columns()]
+    act = [pin(c) for c in wl.active.columns()]
+    n, a = wl.requests.n, wl.active.n
+    for rep in range(2):
+        idx = torch.full((n,), -7, dtype=torch.int32).pin_memory()
+        est = torch.zeros(n, dtype=torch.float32).pin_memory()
+        slack = torch.zeros(n, dtype=torch.float32).pin_memory()
+        tier = torch.zeros(n, dtype=torch.uint8).pin_memory()
+        bits = torch.zeros((a + 31) // 32, dtype=torch.int32).pin_memory()
+        cand = torch.zeros(a, dtype=torch.int32).pin_memory()
+        gs.route_batch_host(*req, wl.types, wl.instances, 0.5, idx, est, slack, tier, wait=False)
+        if rep == 1:       # a second deferred round right behind the first
+            gs.route_batch_host(*req, wl.types, wl.instances, 0.5, idx, est, slack, tier, wait=False)
+        count = gs.risk_scan_host(*act, wl.types, wl.instances, bits, cand)
+        gs.host_wait()
+        got = GpuRoute(idx.numpy(), est.numpy(), slack.numpy(), tier.numpy())
+        assert_route_matches_f32_oracle(got, ref)
+        assert count == rcount
+        np.testing.assert_array_equal(bits.numpy().view(np.uint32), rbits)
+        np.testing.assert_array_equal(cand.numpy()[:count], rcand)
+    assert gs.device_status() == 0
 
 
 def test_work_counters_of_the_counting_build(gs):
