@@ -121,7 +121,9 @@ constexpr unsigned kPadQ = 0x7FC00000u;    // q word of a padding entry (a NaN: 
 
 constexpr int64_t kMaxRouteRequests = (int64_t)1 << 36;   // per routing call (the kernel's queues hold a request's
                                                           // index within its CTA's run of requests in 32 bits)
-#define GS_HOST_PIECES 8                 // the *_host entry points work through their input in up to this many pieces
+#ifndef GS_HOST_PIECES
+#define GS_HOST_PIECES 4                 // the *_host entry points work through their input in up to this many pieces
+#endif
 constexpr int64_t kHostPieceMin = 1 << 18;   // ... of at least this many requests
 constexpr int kMaxScanCtas = 4096;      // CTAs of one risk scan (a few per SM), one flag count each
 constexpr int kMaxActive = 2147483647;  // n_active < 2^31 (indices are int32)
