@@ -71,9 +71,12 @@ struct PoolStage {
 
 size_t pool_stage_bytes(int M, int Tn) { return 5 * pad256((size_t)M * 4) + 3 * pad256((size_t)Tn * 4); }
 
+// The eight small arrays are first put together in a pinned image laid out like their device
+// copies and then sent as one copy (a copy costs some 20 us beside its bytes).
 cudaError_t stage_pool(Carver &c, const gs_instances *h_inst, const gs_types *h_types,
-                       PoolStage *out, cudaStream_t st) {
+                       PoolStage *out, char *pinned_image, cudaStream_t st) {
     const int M = h_inst->n_instances, Tn = h_types->n_types;
+    char *const first = c.base + c.off;
     int32_t *type_id = c.take<int32_t>(M), *queued = c.take<int32_t>(M), *batch = c.take<int32_t>(M),
             *kv = c.take<int32_t>(M);
     float *qe = c.take<float>(M), *p = c.take<float>(Tn), *a = c.take<float>(Tn), *b = c.take<float>(Tn);
@@ -81,11 +84,10 @@ cudaError_t stage_pool(Carver &c, const gs_instances *h_inst, const gs_types *h_
                          h_inst->free_kv_tokens, h_inst->q_ema_ms, h_types->prefill_ms_per_tok,
                          h_types->tpot_a_ms, h_types->tpot_b_ms};
     void *dst[] = {type_id, queued, batch, kv, qe, p, a, b};
-    for (int k = 0; k < 8; ++k) {
-        cudaError_t e = cudaMemcpyAsync(dst[k], src[k], (size_t)(k < 5 ? M : Tn) * 4,
-                                        cudaMemcpyHostToDevice, st);
-        if (e != cudaSuccess) return e;
-    }
+    for (int k = 0; k < 8; ++k)
+        memcpy(pinned_image + ((char *)dst[k] - first), src[k], (size_t)(k < 5 ? M : Tn) * 4);
+    const cudaError_t e = cudaMemcpyAsync(first, pinned_image, (size_t)(c.base + c.off - first), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return e;
     out->inst = gs_instances{type_id, queued, batch, kv, qe, M};
     out->types = gs_types{p, a, b, Tn};
     return cudaSuccess;
@@ -199,6 +201,7 @@ GS_API int gs_destroy(gs_ctx *ctx) {
         cudaStreamDestroy(ctx->host_out_stream);
         for (cudaEvent_t ev : ctx->host_events) cudaEventDestroy(ev);
         cudaFreeHost(ctx->host_counts);
+        for (char *image : ctx->host_pool_image) cudaFreeHost(image);
     }
     delete ctx->pending;
     delete ctx->free_events;
@@ -473,6 +476,8 @@ static int ensure_host_pipe(gs_ctx *ctx) {
     for (int k = 0; k < GS_HOST_PIECES && e == cudaSuccess; ++k)
         e = cudaEventCreateWithFlags(&ctx->host_events[k], cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&ctx->host_counts, GS_HOST_PIECES * sizeof(int64_t), cudaHostAllocDefault);
+    for (int k = 0; k < 2 && e == cudaSuccess; ++k)
+        e = cudaHostAlloc((void **)&ctx->host_pool_image[k], pool_stage_bytes(ctx->max_instances, ctx->max_types), cudaHostAllocDefault);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->host_pipe_ready = true;
     return GS_OK;
@@ -509,7 +514,7 @@ static int route_batch_host(gs_ctx *ctx, const int32_t *prompt_len, const int32_
     if (rc != GS_OK) return rc;
     Carver c{ctx->stage};
     PoolStage pool;
-    cudaError_t e = stage_pool(c, inst, types, &pool, st);
+    cudaError_t e = stage_pool(c, inst, types, &pool, ctx->host_pool_image[0], st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     int32_t *dx = c.take<int32_t>(n), *dy = c.take<int32_t>(n);
     float *dD = c.take<float>(n);
@@ -603,7 +608,7 @@ GS_API int gs_risk_scan_host(gs_ctx *ctx, const int32_t *assigned_inst, const in
     cudaStream_t st = (cudaStream_t)cuda_stream, out = ctx->host_out_stream;
     Carver c{ctx->scan_stage};
     PoolStage pool;
-    cudaError_t e = stage_pool(c, inst, types, &pool, st);
+    cudaError_t e = stage_pool(c, inst, types, &pool, ctx->host_pool_image[1], st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     int32_t *dg = c.take<int32_t>(n), *dgen = c.take<int32_t>(n), *dtot = c.take<int32_t>(n);
     float *del = c.take<float>(n), *dslo = c.take<float>(n);

@@ -171,6 +171,8 @@ struct gs_ctx {
     cudaStream_t host_out_stream;            // results travel back on it while the next piece's inputs arrive
     cudaEvent_t host_events[GS_HOST_PIECES]; // piece k computed
     int64_t *host_counts;                    // pinned: candidates up to and including piece k
+    char *host_pool_image[2];                // pinned: the pool description as it is laid out on the device, one copy
+                                             //  each for the routing and the scan entry point (they may overlap)
     bool host_pipe_ready;
     // optional per-kernel timing (gs_timing_enable)
     bool timing;
