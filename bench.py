@@ -47,11 +47,11 @@ SCHEDULERS_PER_SM = 4             # one warp-instruction per scheduler and clock
 # Counters of one launch on config 3 taken with ncu (the committed ncu summaries).  They describe
 # the kernel sources with these hashes; after any change to those files they no longer apply and
 # the fields that use them become null until the kernel is profiled again.
-PROFILED_ROUTE = {"sources_sha1": "b932c0e4c2f46e7db2f05cb4b61729ee9a3d55cd", "config": 3,
-                  "dram_bytes_per_launch": 52_257_280 + 7_742_464,
-                  "warp_instructions_per_launch": 28_149_367}
-PROFILED_RISK_FLAGS = {"sources_sha1": "711aa064e5105af7036f441a8b5619083510d284", "config": 3,
-                       "dram_bytes_per_launch": 335_603_456 + 4_643_840}
+PROFILED_ROUTE = {"sources_sha1": "a6f981f5085ca21a5b87f2cd588d356a5b0a067a", "config": 3,
+                  "dram_bytes_per_launch": 52_209_408 + 7_099_136,
+                  "warp_instructions_per_launch": 28_148_324}
+PROFILED_RISK_FLAGS = {"sources_sha1": "924a286221ab49a6ca09c606b4dc3cc192a2ea7b", "config": 3,
+                       "dram_bytes_per_launch": 335_576_832 + 4_612_096}
 
 
 def _sources_sha1(names) -> str:
