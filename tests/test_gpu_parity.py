@@ -796,6 +796,31 @@ def test_reroute_with_time_left_on_instance_estimates(gs, case):
     assert gs.device_status() == 0
 
 
+def test_reroute_invalid_data_and_unusable_coefficients(gs):
+    """Bad entries in the active columns are read as the oracle reads them (status bits); a pool
+    whose coefficients the bounds cannot take (an infinite decode time) is still served exactly,
+    every candidate scored against every instance."""
+    from paper_2605_16867_b200 import DeviceStatus
+    rng = np.random.default_rng(31)
+    types, inst = _random_pool(rng, 300, 5)
+    act = W.make_active(W.CONFIGS[3], types, inst.n_instances, seed=77, n=6000)
+    act.pred_len[:] = np.maximum(act.pred_len, act.generated_tokens + 1)      # something left to decode everywhere
+    prompt = np.clip(np.rint(np.exp(rng.normal(6.0, 1.0, act.n))), 1, 1 << 18).astype(np.int32)
+    act.assigned_inst[5] = inst.n_instances; act.assigned_inst[6] = -1
+    act.generated_tokens[7] = -3; prompt[9] = -20
+    cand = np.arange(act.n, dtype=np.int32)
+    for unusable in (False, True):
+        if unusable:
+            types.tpot_a_ms[2] = np.inf
+        pool = pool_of(gs, types, inst)
+        t32 = oracle.instance_table(types, inst, 0.5, "f32")
+        ref = oracle.reroute(t32, cand, *act.columns(), prompt)
+        assert_reroute_matches(gpu_reroute_listed(gs, pool, act, prompt, 0.5, cand), ref)
+        st = gs.device_status()
+        assert st & DeviceStatus.BAD_INSTANCE and st & DeviceStatus.BAD_VALUE
+        assert ref.status & DeviceStatus.BAD_INSTANCE and ref.status & DeviceStatus.BAD_VALUE
+
+
 # --------------------------------------------------------------------------------------
 # routing with the prefix-cache term of Eq. 2
 # --------------------------------------------------------------------------------------
