@@ -1373,14 +1373,14 @@ reroute_kernel(const int32_t *__restrict__ cand_idx, const int64_t *__restrict__
         idx_next = step + 2 * stride < n_steps ? index_at((step + 2 * stride) * 32 + lane) : -1;
         const Candidate c = pose(raw, valid);
         int g = -1; float T = 0.f;
-        int verdict = -1;          // nothing left to decode, more KV than any instance has free, unusable tables: the fallback's queue
+        int outcome = -1;          // nothing left to decode, more KV than any instance has free, unusable tables: the fallback's queue
         if (valid && c.rem > 0 && c.need <= kv_max && tb.n_types > 0)
-            verdict = capped_first_attempt(tb, c.x, c.y, c.D, c.need, c.d_cap, g, T);
-        if (valid && verdict > 0) store(j, g, T, 1u, c.D);
-        if (valid && verdict <= 0) GS_COUNT(kCountQueued, 1);
-        if (valid && verdict < 0) GS_COUNT(kCountFallback, 1);
-        append(queue_full, n_full, valid && verdict == 0, (unsigned)j);
-        append(queue_fall, n_fall, valid && verdict < 0, (unsigned)j);
+            outcome = capped_first_attempt(tb, c.x, c.y, c.D, c.need, c.d_cap, g, T);
+        if (valid && outcome > 0) store(j, g, T, 1u, c.D);
+        if (valid && outcome <= 0) GS_COUNT(kCountQueued, 1);
+        if (valid && outcome < 0) GS_COUNT(kCountFallback, 1);
+        append(queue_full, n_full, valid && outcome == 0, (unsigned)j);
+        append(queue_fall, n_fall, valid && outcome < 0, (unsigned)j);
         __syncwarp();
         for (;;) {
             if (n_fall >= 32) drain_fall();
