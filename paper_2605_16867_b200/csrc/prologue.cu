@@ -49,6 +49,14 @@ unsigned prologue_index_errors(bool clear)
 constexpr int kPrologueThreads = GS_MAX_INSTANCES;      // one thread per instance
 constexpr int kPmFloats = 8192;                         // shared-memory floats for the running minima
 constexpr int kCountSortMax = 256;                      // a group of up to this many rows is ranked by counting
+// CTAs per group.  Every one of them works out the group's order, bounds and running minima
+// (the same on every SM it runs on: nothing to exchange); the start cells and record lists, a
+// third of the kernel's time on one SM, are then shared out by bucket of L_out.
+#ifndef GS_PROLOGUE_SPLIT
+#define GS_PROLOGUE_SPLIT 8
+#endif
+constexpr int kPrologueSplit = GS_PROLOGUE_SPLIT;
+static_assert(kStartBuckets % kPrologueSplit == 0, "the buckets are dealt out evenly");
 
 __device__ __forceinline__ int clamp_count(int v, unsigned &bad) {
     if (v < 0) { bad |= GS_DEV_BAD_VALUE; return 0; }
@@ -160,7 +168,10 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     const int lane = tid & 31;
     const int warp = tid >> 5;
     const bool writer = blockIdx.x == 0;       // one CTA writes what does not depend on the group
-    const int tr = blockIdx.x;                 // position of this CTA's group in the search order
+    const int tr = blockIdx.x / kPrologueSplit;    // position of this CTA's group in the search order
+    const int part = blockIdx.x % kPrologueSplit;  // which of the group's CTAs this is: part 0 writes what the
+                                                   // group has once; each part the cells and lists of its buckets
+    const int b_lo = part * (kStartBuckets / kPrologueSplit), b_hi = b_lo + kStartBuckets / kPrologueSplit;
     unsigned bad = 0;
     const bool has = tid < M;
     // typed pools: all global loads are issued before anything else is done
@@ -405,8 +416,10 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
         // the order must be a strict one (a permutation of the group's rows, no key twice)
         if (k > 0 && k < n_t && !(sh_sorted[k - 1] < sh_sorted[k])) atomicAdd(&g_prologue_index_errors, 1u);
 #endif
-        s.row_bounds[GS_CHECKED(g_prologue_index_errors, row_slot(base + k), kMaxPaddedRows)] = entry;
-        if (kDirect) s.row_p[base + k] = k < n_t ? lower_bound(sh_p[(int)(sh_sorted[k] & 0xFFFFull)]) : 0.f;
+        if (part == 0) {
+            s.row_bounds[GS_CHECKED(g_prologue_index_errors, row_slot(base + k), kMaxPaddedRows)] = entry;
+            if (kDirect) s.row_p[base + k] = k < n_t ? lower_bound(sh_p[(int)(sh_sorted[k] & 0xFFFFull)]) : 0.f;
+        }
     }
     my_qmin = __reduce_min_sync(0xFFFFFFFFu, my_qmin);
     if (lane == 0) atomicMin(&sh_qmin, my_qmin);
@@ -414,7 +427,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
 
     // bounds over every eight rows (the fallback's search skips a group whole with them)
     for (int g = tid - 64; g < n_padded / 8; g += kPrologueThreads - 64) {   // (warps 0 and 1 have other work below)
-        if (g < 0) break;
+        if (g < 0 || part != 0) break;
         float q_least = __int_as_float(0x7F800000);         // +inf: a group of padding only
         float d_last = 0.f;
         for (int k = 8 * g; k < 8 * g + 8 && k < n_t; ++k) { q_least = fminf(q_least, sh_rq[k]); d_last = sh_rd[k]; }
@@ -426,7 +439,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
     const float d_hi = sh_rd[0], d_low = sh_rd[n_t - 1];
     float inv_w = 0.f;              // slots per unit of d; 0 = no start table (search from row 0)
     if (n_t > 4 && (d_hi - d_low) > d_hi * (1.0f / 1024.0f)) inv_w = (float)kStartSlots / (d_hi - d_low);
-    if (tid == 32) {
+    if (tid == 32 && part == 0) {
         const int first_inst = (int)(sh_sorted[0] & 0xFFFFull);
         TypeHeader h;
         h.p_lo = __fmul_rn(p_group, kShrink);
@@ -520,7 +533,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                     slope = fmaxf(slope, 0.f);
                     const float offset = f_lo - slope * y_lo;
                     const float kMargin = 1.52587890625e-5f;            // 2^-16
-                    if (lane == 0)
+                    if (lane == 0 && b >= b_lo && b < b_hi)
                         s.chord[tr * kStartBuckets + b] = make_float4(offset - kMargin * f_lo, slope * (1.0f - kMargin),
                                                                   __fmul_rn(p_group, kShrink), 0.f);
                 }
@@ -548,10 +561,11 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
             }
             // (the cells below need the running minima and record counts only, not the pool
             // offsets that warp 0 has just worked out: no barrier in between)
-            for (int c = tid - 32; c < per_batch * kStartSlots; c += kPrologueThreads - 32) {
-                if (c < 0) break;                           // warp 0 is busy with the pool
+            // (this CTA's buckets among those of the batch)
+            const int bw_lo = max(b_lo - b0, 0), bw_hi = min(min(b_hi, kStartBuckets) - b0, per_batch);
+            for (int c = bw_lo * kStartSlots + tid - 32; c < bw_hi * kStartSlots; c += kPrologueThreads - 32) {
+                if (tid < 32) break;                        // warp 0 is busy with the pool
                 const int bw = c / kStartSlots, slot = c % kStartSlots, b = b0 + bw;
-                if (b >= kStartBuckets) break;
                 int lo = 0;                                 // rows [0, lo) cannot pass
                 if (inv_w > 0.f && slot != kStartSlots - 1) {   // (the top slot also takes every z beyond the table)
                     const bool open_ended = b == kStartBuckets - 1;
@@ -574,7 +588,7 @@ prologue_kernel(const int32_t *__restrict__ type_id, const int32_t *__restrict__
                 }
             }
             __syncthreads();
-            if (my_bucket && !kDirect) {
+            if (my_bucket && !kDirect && b0 + warp >= b_lo && b0 + warp < b_hi) {
                 const int off = sh_off[warp], len = sh_len[warp];
                 if (off >= 0) {
                     const unsigned short *pc = sh_pc + warp * n_t;
@@ -610,7 +624,7 @@ cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_type
                             float ema_alpha, bool carry_q, cudaStream_t st)
 {
     LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
-    return launch_dependent(prologue_kernel<false>, dim3(GS_MAX_TYPES), dim3(kPrologueThreads), prologue_dynamic_smem(), st,
+    return launch_dependent(prologue_kernel<false>, dim3(GS_MAX_TYPES * kPrologueSplit), dim3(kPrologueThreads), prologue_dynamic_smem(), st,
                             inst.type_id, inst.queued_prefill_tokens, inst.decode_batch, inst.free_kv_tokens,
                             inst.q_ema_ms, inst.n_instances, types.prefill_ms_per_tok, types.tpot_a_ms,
                             types.tpot_b_ms, types.n_types, ema_alpha, carry_q ? 1 : 0, ctx->s);
@@ -622,7 +636,7 @@ cudaError_t launch_prologue(gs_ctx *ctx, const gs_instances &inst, const gs_type
 cudaError_t launch_prologue_direct(gs_ctx *ctx, const gs_instance_table &tab, cudaStream_t st)
 {
     LaunchTimer timer(ctx, GS_K_PROLOGUE, st);
-    return launch_dependent(prologue_kernel<true>, dim3(GS_MAX_TYPES), dim3(kPrologueThreads), prologue_dynamic_smem(), st,
+    return launch_dependent(prologue_kernel<true>, dim3(GS_MAX_TYPES * kPrologueSplit), dim3(kPrologueThreads), prologue_dynamic_smem(), st,
                             reinterpret_cast<const int32_t *>(tab.q_ms), reinterpret_cast<const int32_t *>(tab.p_ms_per_tok),
                             reinterpret_cast<const int32_t *>(tab.d_ms_per_tok), tab.free_kv_tokens, (const float *)nullptr,
                             tab.n_instances, (const float *)nullptr, (const float *)nullptr, (const float *)nullptr,
